@@ -1,0 +1,155 @@
+"""ctypes face of the CPU oracle (``ivf_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the benchmark's CPU-baseline leg load
+this; the product path never does.  The arithmetic is all in the C file; this module only
+marshals numpy arrays and compiles the C on first use (gcc, -O2, OpenMP over rows).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ivf_oracle.c")
+_LIB = os.path.join(_HERE, "libivf_oracle.so")
+
+F32, U8 = 0, 1
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle's C file into a shared object next to it."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared",
+                               "-ffp-contract=off", _SRC, "-o", tmp, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        i64, i32, vp = ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p
+        _lib.oracle_route.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, vp, i32, i32, vp, vp, vp]
+        _lib.oracle_assign.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, vp, i32, vp, vp]
+        _lib.oracle_pair_dists.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, i64, vp, vp, vp]
+        _lib.oracle_sqnorms.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, vp]
+        _lib.oracle_update.argtypes = [vp, ctypes.c_int, vp, i64, ctypes.c_int, i32, vp, vp]
+        _lib.oracle_finalize.argtypes = [vp, vp, i32, ctypes.c_int, vp]
+        _lib.oracle_lloyd.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, i32, ctypes.c_int, vp, vp, vp]
+        _lib.oracle_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def _rows(x: np.ndarray):
+    """(contiguous array, dtype code) for a float32 or uint8 row matrix."""
+    if x.dtype == np.uint8:
+        return np.ascontiguousarray(x), U8
+    if x.dtype == np.float32:
+        return np.ascontiguousarray(x), F32
+    raise TypeError(f"oracle takes float32 or uint8 rows, got {x.dtype}")
+
+
+def _cent(c: np.ndarray) -> np.ndarray:
+    if c.dtype != np.float32:
+        raise TypeError("centroids must be float32")
+    return np.ascontiguousarray(c)
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def route(x: np.ndarray, c: np.ndarray, k: int):
+    """(ids [n,k] int32, dists [n,k] float64, next [n] float64): the k nearest centroids of every
+    row in ascending (distance, id) order and the (k+1)-th distance."""
+    x, xt = _rows(x)
+    c = _cent(c)
+    n, d = x.shape
+    nlist = c.shape[0]
+    assert c.shape[1] == d
+    ids = np.empty((n, k), np.int32)
+    dists = np.empty((n, k), np.float64)
+    nxt = np.empty((n,), np.float64)
+    rc = _load().oracle_route(_p(x), xt, n, d, _p(c), nlist, k, _p(ids), _p(dists), _p(nxt))
+    if rc != 0:
+        raise ValueError("oracle_route: bad arguments")
+    return ids, dists, nxt
+
+
+def assign(x: np.ndarray, c: np.ndarray):
+    """(ids [n] int32, dists [n] float64): nearest centroid of every row."""
+    x, xt = _rows(x)
+    c = _cent(c)
+    n, d = x.shape
+    ids = np.empty((n,), np.int32)
+    dists = np.empty((n,), np.float64)
+    rc = _load().oracle_assign(_p(x), xt, n, d, _p(c), c.shape[0], _p(ids), _p(dists))
+    if rc != 0:
+        raise ValueError("oracle_assign: bad arguments")
+    return ids, dists
+
+
+def pair_dists(x: np.ndarray, c: np.ndarray, rows: np.ndarray, cols: np.ndarray) -> np.ndarray:
+    """Squared distances of the given (row of x, row of c) pairs, float64."""
+    x, xt = _rows(x)
+    c = _cent(c)
+    rows = np.ascontiguousarray(rows, np.int64)
+    cols = np.ascontiguousarray(cols, np.int32)
+    out = np.empty(rows.shape, np.float64)
+    _load().oracle_pair_dists(_p(x), xt, x.shape[1], _p(c), rows.size, _p(rows), _p(cols), _p(out))
+    return out
+
+
+def sqnorms(x: np.ndarray) -> np.ndarray:
+    x, xt = _rows(x)
+    out = np.empty((x.shape[0],), np.float64)
+    _load().oracle_sqnorms(_p(x), xt, x.shape[0], x.shape[1], _p(out))
+    return out
+
+
+def update(x: np.ndarray, ids: np.ndarray, nlist: int, sums: np.ndarray | None = None,
+           counts: np.ndarray | None = None):
+    """Accumulate per-list sums (float64 [nlist,d]) and counts (int64 [nlist]); returns
+    (sums, counts, ok) where ok is False if some id was out of range (that row is skipped)."""
+    x, xt = _rows(x)
+    n, d = x.shape
+    ids = np.ascontiguousarray(ids, np.int32)
+    if sums is None:
+        sums = np.zeros((nlist, d), np.float64)
+    if counts is None:
+        counts = np.zeros((nlist,), np.int64)
+    assert sums.dtype == np.float64 and counts.dtype == np.int64 and sums.flags.c_contiguous
+    rc = _load().oracle_update(_p(x), xt, _p(ids), n, d, nlist, _p(sums), _p(counts))
+    return sums, counts, rc == 0
+
+
+def finalize(sums: np.ndarray, counts: np.ndarray, centroids: np.ndarray) -> np.ndarray:
+    """New float32 centroids: mean per list, empty lists keep the row of ``centroids``."""
+    out = np.array(centroids, dtype=np.float32, order="C", copy=True)
+    sums = np.ascontiguousarray(sums, np.float64)
+    counts = np.ascontiguousarray(counts, np.int64)
+    _load().oracle_finalize(_p(sums), _p(counts), out.shape[0], out.shape[1], _p(out))
+    return out
+
+
+def lloyd(x: np.ndarray, init_centroids: np.ndarray, iters: int):
+    """(centroids float32, ids int32 of the last iteration, inertia float64 [iters])."""
+    x, xt = _rows(x)
+    c = np.array(init_centroids, dtype=np.float32, order="C", copy=True)
+    n, d = x.shape
+    ids = np.empty((n,), np.int32)
+    inertia = np.empty((iters,), np.float64)
+    rc = _load().oracle_lloyd(_p(x), xt, n, d, c.shape[0], iters, _p(c), _p(ids), _p(inertia))
+    if rc != 0:
+        raise ValueError("oracle_lloyd failed")
+    return c, ids, inertia
