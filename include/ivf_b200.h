@@ -1,0 +1,138 @@
+/*
+ * ivf_b200 -- C-ABI of the B200 (sm_100a) IVF coarse-routing / assignment / Lloyd-update library.
+ *
+ * The one computation behind every call is the batched squared-L2 distance from each row of a
+ * point matrix to every centroid, with the k smallest per row kept on the device:
+ *   - coarse search (Eq. 1): the P nearest lists of each query, P = nprobe;
+ *   - distances come from inner products and precomputed norms,
+ *     |x-c|^2 = |x|^2 + |c|^2 - 2 x.c  (Sec. 4.1, Eq. 3), as a dense tensor-core contraction;
+ *   - only ids and optional distances, O(B*P), leave the kernel (Sec. 4.1, on-device list
+ *     selection); the B x N_list distance matrix is never written to memory;
+ *   - index construction assigns every vector to its nearest centroid (Sec. 3.1, Sec. 5.5) -- the
+ *     k = 1 case -- and Lloyd iterations recompute each centroid as the mean of its members.
+ *
+ * Conventions shared by all calls
+ *   Layout     every matrix is dense row-major with contiguous rows (leading dimension = d).
+ *   Pointers   "device" = memory of the current CUDA device; "host" = page-locked host memory.
+ *              The caller owns every buffer; the library keeps none past stream completion.
+ *   Streams    work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = legacy default
+ *              stream) and the call returns without waiting, except where stated.
+ *   Workspace  the library keeps one grow-only device workspace per device; it grows with a
+ *              stream-ordered allocation on `stream`.  Calls that share a device must therefore be
+ *              issued in stream order with respect to each other (one stream, or streams the
+ *              caller has ordered with events).
+ *   Errors     every call returns IVF_OK or a negative ivf_status.  Argument errors are detected
+ *              before anything is enqueued.  Device-side problems (a bounded wait that expired, an
+ *              id out of range) set a sticky per-device status word that ivf_check reads.
+ *   Limits     d must be a multiple of 16, 16 <= d <= 256.  1 <= nprobe <= min(nlist, 512).
+ *              nlist < 2^31.  n == 0 is IVF_OK and enqueues nothing.
+ *   Non-finite inputs give unspecified (but memory-safe) results.
+ *
+ * The problem statement gives neither the element type of the points nor d for the update; both are
+ * needed, so the signatures below carry `ptype` and `d` in addition.
+ */
+#ifndef IVF_B200_H
+#define IVF_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { IVF_F32 = 0, IVF_U8 = 1 } ivf_dtype;
+
+typedef enum {
+    IVF_OK = 0,
+    IVF_ERR_INVALID_ARG = -1,    /* null pointer, negative size, pageable host memory ...        */
+    IVF_ERR_UNSUPPORTED = -2,    /* d, nprobe or nlist outside the limits above                   */
+    IVF_ERR_ALLOC = -3,          /* workspace allocation failed                                   */
+    IVF_ERR_CUDA = -4,           /* a CUDA runtime/driver call failed (see ivf_last_error)        */
+    IVF_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait expired; results are invalid       */
+    IVF_ERR_BAD_ID = -6          /* ivf_centroid_update met an id outside [0, nlist); row skipped */
+} ivf_status;
+
+/*
+ * Coarse routing (Eq. 1; Sec. 4.1 dense centroid evaluation + on-device list selection).
+ *   queries    [nq, d] float32 or uint8 (qtype); device, or page-locked host (then the rows are
+ *              streamed through the device in chunks, the copies overlapping the kernels)
+ *   centroids  [nlist, d] float32, device
+ *   out_ids    [nq, nprobe] int32, device: the nprobe nearest centroids of every query, ascending
+ *              by (distance, id) -- equal distances are ordered by the lower id
+ *   out_dists  [nq, nprobe] float32 squared L2 distances (clamped at 0), device; may be NULL
+ */
+int ivf_route(const void* queries, int64_t nq, int d, ivf_dtype qtype,
+              const float* centroids, int nlist, int nprobe,
+              int32_t* out_ids, float* out_dists, void* stream);
+
+/*
+ * Assignment to the nearest centroid (Sec. 3.1 index layout; Sec. 5.5 full-mode construction).
+ * Same as ivf_route with nprobe = 1: out_ids [n] int32, out_dists [n] float32 (may be NULL).
+ * `points` may be device or page-locked host memory as for ivf_route.
+ */
+int ivf_assign(const void* points, int64_t n, int d, ivf_dtype ptype,
+               const float* centroids, int nlist,
+               int32_t* out_ids, float* out_dists, void* stream);
+
+/*
+ * Lloyd accumulation (Sec. 5.5, "Lloyd iterations"):
+ *   sums[l, :] += sum of the rows i with ids[i] == l      [nlist, d] float32, device
+ *   counts[l]  += number of such rows                     [nlist]    int64,   device
+ * ACCUMULATES into sums/counts so that chunks of one iteration compose; the caller zeroes them
+ * at the start of an iteration.  points [n, d] (ptype) and ids [n] int32 are device pointers.
+ * A row whose id is outside [0, nlist) is skipped and flags IVF_ERR_BAD_ID in the status word.
+ * For uint8 points the sums are exact while every list sum stays below 2^24.
+ */
+int ivf_centroid_update(const void* points, ivf_dtype ptype, const int32_t* ids, int64_t n, int d,
+                        int nlist, float* sums, int64_t* counts, void* stream);
+
+/*
+ * Helper: new centroid = sums / counts per list (float32 divide); a list with count 0 keeps its
+ * row of centroids_inout (the paper does not say what an empty list does).  All device pointers.
+ */
+int ivf_centroid_finalize(const float* sums, const int64_t* counts, int nlist, int d,
+                          float* centroids_inout, void* stream);
+
+/*
+ * Helper: one pass of a Lloyd iteration over a point set that may exceed device memory
+ * (Table 3: assignment in batches of 1,048,576 vectors; Table 1: the host link is the scarce
+ * resource).  For each chunk of `chunk_rows` rows: copy to the device if `points` is page-locked
+ * host memory (double-buffered on an internal copy stream), assign (k = 1), accumulate
+ * sums/counts.  Each chunk crosses the host link once.  out_ids [n] int32 and out_dists [n]
+ * float32 are device pointers and may be NULL.  chunk_rows <= 0 selects 1,048,576.
+ */
+int ivf_assign_update(const void* points, int64_t n, int d, ivf_dtype ptype,
+                      const float* centroids, int nlist,
+                      int32_t* out_ids, float* out_dists,
+                      float* sums, int64_t* counts, int64_t chunk_rows, void* stream);
+
+/* Synchronises `stream`, then returns and clears the sticky device status of the current device. */
+int ivf_check(void* stream);
+
+/* Message of the last error returned on this host thread ("" if none). */
+const char* ivf_last_error(void);
+
+/* Frees the current device's workspace (after synchronising the device). */
+int ivf_release_workspace(void);
+
+/* Number of kernels this library has launched on this host process so far (all devices). */
+int64_t ivf_launch_count(void);
+
+/*
+ * Test hooks (host logic only; no kernel is launched).
+ *   ivf_debug_plan   the persistent schedule of the fused kernel for a problem size on a device
+ *                    with `num_sms` SMs: writes {row_tiles, col_tiles, ctas, max_partials_per_row_tile,
+ *                    block_n, k_slices, stages, smem_bytes} to out[8].
+ *   ivf_debug_span   first unit and one-past-last unit of CTA `cta` in that schedule.
+ *   ivf_debug_set_wait_limit_ns   time limit of every device-side wait (0 restores the default
+ *                    of 2 s); with a tiny limit a launch reports IVF_ERR_DEVICE_TIMEOUT through
+ *                    ivf_check and still returns normally.
+ */
+int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[8]);
+int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int64_t out[2]);
+int ivf_debug_set_wait_limit_ns(int64_t ns);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IVF_B200_H */

@@ -1,0 +1,238 @@
+"""Python face of the C-ABI library (``include/ivf_b200.h``): argument marshalling only.
+
+Every function takes torch tensors (CUDA tensors, or page-locked CPU tensors where the C function
+accepts host memory), checks dtype / shape / contiguity, and passes raw pointers and sizes plus
+the current CUDA stream to the library.  No step of the computation runs in Python or in torch.
+There is no fallback: if the library cannot be loaded the import of a symbol raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+IVF_F32, IVF_U8 = 0, 1
+IVF_OK = 0
+IVF_ERR_INVALID_ARG, IVF_ERR_UNSUPPORTED, IVF_ERR_ALLOC = -1, -2, -3
+IVF_ERR_CUDA, IVF_ERR_DEVICE_TIMEOUT, IVF_ERR_BAD_ID = -4, -5, -6
+
+EXPORTS = (
+    "ivf_route", "ivf_assign", "ivf_centroid_update", "ivf_centroid_finalize", "ivf_assign_update",
+    "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
+    "ivf_debug_plan", "ivf_debug_span", "ivf_debug_set_wait_limit_ns",
+)
+
+_lib = None
+
+
+class IvfError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"ivf_b200 error {code}: {message}")
+        self.code = code
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library; built in-tree first if it is missing or older than its sources."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB_PATH
+    if not os.path.exists(path) or _build._stale():
+        try:
+            path = _build.build()
+        except Exception as exc:  # no nvcc on this machine: use what travelled with the tree
+            if not os.path.exists(path):
+                raise RuntimeError(f"libivf_b200.so is missing and could not be built: {exc}") from exc
+    L = ctypes.CDLL(path)
+    vp, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+    L.ivf_route.argtypes = [vp, i64, i32, i32, vp, i32, i32, vp, vp, vp]
+    L.ivf_assign.argtypes = [vp, i64, i32, i32, vp, i32, vp, vp, vp]
+    L.ivf_centroid_update.argtypes = [vp, i32, vp, i64, i32, i32, vp, vp, vp]
+    L.ivf_centroid_finalize.argtypes = [vp, vp, i32, i32, vp, vp]
+    L.ivf_assign_update.argtypes = [vp, i64, i32, i32, vp, i32, vp, vp, vp, vp, i64, vp]
+    L.ivf_check.argtypes = [vp]
+    L.ivf_last_error.restype = ctypes.c_char_p
+    L.ivf_launch_count.restype = i64
+    L.ivf_debug_plan.argtypes = [i64, i32, i32, i32, i32, ctypes.POINTER(i64)]
+    L.ivf_debug_span.argtypes = [i64, i32, i32, i32, i32, i32, ctypes.POINTER(i64)]
+    L.ivf_debug_set_wait_limit_ns.argtypes = [i64]
+    for name in EXPORTS:
+        if name not in ("ivf_last_error", "ivf_launch_count"):
+            getattr(L, name).restype = i32
+    _lib = L
+    return L
+
+
+def _raise(code: int):
+    raise IvfError(code, lib().ivf_last_error().decode())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return IVF_F32
+    if t.dtype == torch.uint8:
+        return IVF_U8
+    raise TypeError(f"points must be float32 or uint8, got {t.dtype}")
+
+
+def _rows(t: torch.Tensor, name: str) -> torch.Tensor:
+    if t.dim() != 2 or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous 2-D tensor")
+    if not (t.is_cuda or t.is_pinned()):
+        raise ValueError(f"{name} must be a CUDA tensor or a pinned CPU tensor")
+    return t
+
+
+def _dev(t: torch.Tensor, name: str, dtype: torch.dtype) -> torch.Tensor:
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+def _stream(device) -> int:
+    return torch.cuda.current_stream(device).cuda_stream
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def ivf_route(queries: torch.Tensor, centroids: torch.Tensor, nprobe: int,
+              out_ids: torch.Tensor | None = None, out_dists: torch.Tensor | None = None,
+              want_dists: bool = True):
+    """ids [nq, nprobe] int32 (and squared distances [nq, nprobe] float32) of the nprobe nearest
+    centroids of every query, ascending by (distance, id).  Enqueued on the current stream."""
+    _rows(queries, "queries")
+    _dev(centroids, "centroids", torch.float32)
+    nq, d = queries.shape
+    nlist = centroids.shape[0]
+    dev = centroids.device
+    if out_ids is None:
+        out_ids = torch.empty((nq, nprobe), dtype=torch.int32, device=dev)
+    if out_dists is None and want_dists:
+        out_dists = torch.empty((nq, nprobe), dtype=torch.float32, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib().ivf_route(_ptr(queries), nq, d, _dtype_code(queries), _ptr(centroids), nlist, nprobe,
+                             _ptr(_dev(out_ids, "out_ids", torch.int32)),
+                             _ptr(out_dists), _stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
+    return out_ids, out_dists
+
+
+def ivf_assign(points: torch.Tensor, centroids: torch.Tensor,
+               out_ids: torch.Tensor | None = None, out_dists: torch.Tensor | None = None,
+               want_dists: bool = True):
+    """ids [n] int32 (and squared distances [n] float32) of the nearest centroid of every row."""
+    _rows(points, "points")
+    _dev(centroids, "centroids", torch.float32)
+    n, d = points.shape
+    dev = centroids.device
+    if out_ids is None:
+        out_ids = torch.empty((n,), dtype=torch.int32, device=dev)
+    if out_dists is None and want_dists:
+        out_dists = torch.empty((n,), dtype=torch.float32, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib().ivf_assign(_ptr(points), n, d, _dtype_code(points), _ptr(centroids), centroids.shape[0],
+                              _ptr(_dev(out_ids, "out_ids", torch.int32)), _ptr(out_dists), _stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
+    return out_ids, out_dists
+
+
+def ivf_centroid_update(points: torch.Tensor, ids: torch.Tensor, sums: torch.Tensor, counts: torch.Tensor):
+    """sums[l] += member rows, counts[l] += members; accumulates in place (all CUDA tensors)."""
+    if not points.is_cuda:
+        raise ValueError("points must be a CUDA tensor")
+    _rows(points, "points")
+    _dev(ids, "ids", torch.int32)
+    _dev(sums, "sums", torch.float32)
+    _dev(counts, "counts", torch.int64)
+    n, d = points.shape
+    nlist = sums.shape[0]
+    if sums.shape != (nlist, d) or counts.shape != (nlist,) or ids.shape != (n,):
+        raise ValueError("shape mismatch between points, ids, sums and counts")
+    dev = points.device
+    with torch.cuda.device(dev):
+        rc = lib().ivf_centroid_update(_ptr(points), _dtype_code(points), _ptr(ids), n, d, nlist,
+                                       _ptr(sums), _ptr(counts), _stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
+
+
+def ivf_centroid_finalize(sums: torch.Tensor, counts: torch.Tensor, centroids: torch.Tensor):
+    """centroids[l] = sums[l] / counts[l] in place; lists with count 0 keep their row."""
+    _dev(sums, "sums", torch.float32)
+    _dev(counts, "counts", torch.int64)
+    _dev(centroids, "centroids", torch.float32)
+    nlist, d = centroids.shape
+    dev = centroids.device
+    with torch.cuda.device(dev):
+        rc = lib().ivf_centroid_finalize(_ptr(sums), _ptr(counts), nlist, d, _ptr(centroids), _stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
+
+
+def ivf_assign_update(points: torch.Tensor, centroids: torch.Tensor, sums: torch.Tensor, counts: torch.Tensor,
+                      out_ids: torch.Tensor | None = None, out_dists: torch.Tensor | None = None,
+                      chunk_rows: int = 0):
+    """One streamed pass of a Lloyd iteration: per chunk copy (if host), assign, accumulate."""
+    _rows(points, "points")
+    _dev(centroids, "centroids", torch.float32)
+    _dev(sums, "sums", torch.float32)
+    _dev(counts, "counts", torch.int64)
+    n, d = points.shape
+    dev = centroids.device
+    if out_ids is not None:
+        _dev(out_ids, "out_ids", torch.int32)
+    if out_dists is not None:
+        _dev(out_dists, "out_dists", torch.float32)
+    with torch.cuda.device(dev):
+        rc = lib().ivf_assign_update(_ptr(points), n, d, _dtype_code(points), _ptr(centroids), centroids.shape[0],
+                                     _ptr(out_ids), _ptr(out_dists), _ptr(sums), _ptr(counts), chunk_rows,
+                                     _stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
+
+
+def ivf_check(device=None) -> None:
+    """Synchronises the current stream and raises if a kernel recorded a device-side problem."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    with torch.cuda.device(dev):
+        rc = lib().ivf_check(_stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
+
+
+def ivf_launch_count() -> int:
+    return int(lib().ivf_launch_count())
+
+
+def ivf_release_workspace() -> None:
+    rc = lib().ivf_release_workspace()
+    if rc != IVF_OK:
+        _raise(rc)
+
+
+def ivf_debug_plan(n: int, nlist: int, d: int, k: int, num_sms: int = 148) -> dict:
+    out = (ctypes.c_int64 * 8)()
+    rc = lib().ivf_debug_plan(n, nlist, d, k, num_sms, out)
+    if rc != IVF_OK:
+        _raise(rc)
+    keys = ("row_tiles", "col_tiles", "ctas", "partials", "block_n", "k_slices", "stages", "smem_bytes")
+    return dict(zip(keys, (int(v) for v in out)))
+
+
+def ivf_debug_span(n: int, nlist: int, d: int, k: int, num_sms: int, cta: int):
+    out = (ctypes.c_int64 * 2)()
+    rc = lib().ivf_debug_span(n, nlist, d, k, num_sms, cta, out)
+    if rc != IVF_OK:
+        _raise(rc)
+    return int(out[0]), int(out[1])
+
+
+def ivf_debug_set_wait_limit_ns(ns: int) -> None:
+    lib().ivf_debug_set_wait_limit_ns(ns)

@@ -1,0 +1,603 @@
+// Host side of the C-ABI library: argument checks, the per-device workspace, the persistent
+// schedule, kernel launches, and the chunk pipeline for point sets that live in page-locked host
+// memory (Table 3: assignment proceeds in batches; Table 1: the host link is the scarce resource,
+// so every chunk crosses it exactly once and the copy of chunk i+1 overlaps the kernels of chunk i).
+#include "../../include/ivf_b200.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <string>
+#include <type_traits>
+
+#include "fused_topk.cuh"
+#include "merge.cuh"
+#include "prep.cuh"
+#include "update.cuh"
+
+namespace {
+
+using namespace ivf;
+
+thread_local std::string g_err;
+std::atomic<int64_t> g_launches{0};
+std::atomic<uint64_t> g_wait_limit_ns{2000000000ull};  // 2 s per device-side wait
+std::mutex g_mu;
+
+int fail(int code, const char* fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_err = buf;
+    return code;
+}
+
+#define CUDA_TRY(expr)                                                                         \
+    do {                                                                                       \
+        cudaError_t e__ = (expr);                                                              \
+        if (e__ != cudaSuccess)                                                                \
+            return fail(IVF_ERR_CUDA, "%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__), \
+                        __FILE__, __LINE__);                                                   \
+    } while (0)
+
+#define LAUNCH_CHECK()                    \
+    do {                                  \
+        g_launches.fetch_add(1);          \
+        CUDA_TRY(cudaGetLastError());     \
+    } while (0)
+
+// ------------------------------------------------------------------ workspace
+enum WsSlot {
+    WS_X16, WS_C16, WS_XN, WS_CN, WS_SCAL, WS_BITS, WS_PART, WS_PARTCNT,
+    WS_UCNT, WS_UOFF, WS_UCUR, WS_UPERM, WS_IDS, WS_CHUNK0, WS_CHUNK1, WS_NUM
+};
+struct Buf {
+    void* p = nullptr;
+    size_t cap = 0;
+};
+struct DeviceCtx {
+    bool init = false;
+    int num_sms = 0;
+    int* status = nullptr;
+    Buf bufs[WS_NUM];
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_copied[2] = {nullptr, nullptr};
+    cudaEvent_t ev_free[2] = {nullptr, nullptr};
+    cudaEvent_t ev_ready = nullptr;
+    bool smem_attr_set = false;
+};
+constexpr int kMaxDevices = 64;
+DeviceCtx g_ctx[kMaxDevices];
+
+int get_ctx(DeviceCtx** out) {
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(IVF_ERR_CUDA, "device index %d out of range", dev);
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx& c = g_ctx[dev];
+    if (!c.init) {
+        cudaDeviceProp prop;
+        CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
+        if (prop.major != 10)
+            return fail(IVF_ERR_UNSUPPORTED, "this library runs on sm_100 devices only (found sm_%d%d)", prop.major,
+                        prop.minor);
+        c.num_sms = prop.multiProcessorCount;
+        CUDA_TRY(cudaMalloc(&c.status, 4 * sizeof(int)));
+        CUDA_TRY(cudaMemset(c.status, 0, 4 * sizeof(int)));
+        CUDA_TRY(cudaStreamCreateWithFlags(&c.copy_stream, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+            CUDA_TRY(cudaEventCreateWithFlags(&c.ev_copied[i], cudaEventDisableTiming));
+            CUDA_TRY(cudaEventCreateWithFlags(&c.ev_free[i], cudaEventDisableTiming));
+        }
+        CUDA_TRY(cudaEventCreateWithFlags(&c.ev_ready, cudaEventDisableTiming));
+        c.init = true;
+    }
+    *out = &c;
+    return IVF_OK;
+}
+
+// Grow-only, stream-ordered.
+int ws_get(DeviceCtx& c, WsSlot slot, size_t bytes, cudaStream_t stream, void** out) {
+    Buf& b = c.bufs[slot];
+    if (bytes > b.cap) {
+        if (b.p) CUDA_TRY(cudaFreeAsync(b.p, stream));
+        b.p = nullptr;
+        b.cap = 0;
+        size_t want = bytes + bytes / 8;
+        want = (want + 255) & ~size_t(255);
+        void* p = nullptr;
+        cudaError_t e = cudaMallocAsync(&p, want, stream);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            return fail(IVF_ERR_ALLOC, "workspace allocation of %zu bytes failed: %s", want, cudaGetErrorString(e));
+        }
+        b.p = p;
+        b.cap = want;
+    }
+    *out = b.p;
+    return IVF_OK;
+}
+#define WS(slot, bytes, ptrvar)                                                              \
+    do {                                                                                     \
+        void* p__ = nullptr;                                                                 \
+        int rc__ = ws_get(ctx, slot, bytes, stream, &p__);                                   \
+        if (rc__ != IVF_OK) return rc__;                                                     \
+        ptrvar = reinterpret_cast<typename std::remove_reference<decltype(ptrvar)>::type>(p__);                                    \
+    } while (0)
+
+// ------------------------------------------------------------------ schedule
+struct Plan {
+    int kp, kslices, ksteps, block_n, nstage;
+    int64_t row_tiles;
+    int col_tiles;
+    int64_t total_units;
+    int ctas;
+    int partials;
+    int cap;
+    size_t smem;
+};
+
+constexpr size_t kSmemLimit = 227 * 1024;
+
+int make_plan(int64_t n, int nlist, int d, int k, int num_sms, Plan* pl) {
+    pl->kp = (d + 63) / 64 * 64;
+    pl->kslices = pl->kp / 64;
+    pl->ksteps = (d + 15) / 16;
+    pl->block_n = pl->kslices <= 2 ? 256 : 128;
+    int nstage = kMaxStages;
+    while (nstage > 1 && fused_smem_bytes(pl->kslices, pl->block_n, nstage) > kSmemLimit) --nstage;
+    if (nstage < 2) return fail(IVF_ERR_UNSUPPORTED, "d = %d does not fit the shared-memory ring", d);
+    pl->nstage = nstage;
+    pl->smem = fused_smem_bytes(pl->kslices, pl->block_n, nstage);
+    pl->row_tiles = (n + kBlockM - 1) / kBlockM;
+    pl->col_tiles = (nlist + pl->block_n - 1) / pl->block_n;
+    pl->total_units = pl->row_tiles * pl->col_tiles;
+    pl->ctas = static_cast<int>(pl->total_units < num_sms ? pl->total_units : num_sms);
+    const int64_t lmin = pl->total_units / pl->ctas;
+    int64_t parts = (pl->col_tiles + lmin - 1) / lmin + 1;
+    if (parts > pl->ctas) parts = pl->ctas;
+    pl->partials = static_cast<int>(parts);
+    pl->cap = (k == 1) ? 1 : (4 * k > 128 ? 4 * k : 128);
+    return IVF_OK;
+}
+
+// rows per launch so that the per-launch scratch stays bounded
+int64_t rows_per_launch(int d, int k) {
+    const int kp = (d + 63) / 64 * 64;
+    const int cap = (k == 1) ? 1 : (4 * k > 128 ? 4 * k : 128);
+    const int64_t per_row = static_cast<int64_t>(kp) * 2 + 3ll * cap * 8;  // fp16 copy + ~3 partial logs
+    int64_t rows = (int64_t(2) << 30) / per_row;
+    rows = rows / kBlockM * kBlockM;
+    if (rows < kBlockM) rows = kBlockM;
+    if (rows > (int64_t(4) << 20)) rows = int64_t(4) << 20;
+    return rows;
+}
+
+// ------------------------------------------------------------------ tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+int get_encode() {
+    if (g_encode) return IVF_OK;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (qres != cudaDriverEntryPointSuccess || !fn)
+        return fail(IVF_ERR_CUDA, "cuTensorMapEncodeTiled is not available in this driver");
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    return IVF_OK;
+}
+
+// fp16 matrix [rows][kp] row-major; box = 64 columns x box_rows rows; 128-byte swizzle.
+int make_tmap(CUtensorMap* map, const void* base, int64_t rows, int kp, int box_rows) {
+    cuuint64_t dims[2] = {static_cast<cuuint64_t>(kp), static_cast<cuuint64_t>(rows)};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(kp) * 2};
+    cuuint32_t box[2] = {static_cast<cuuint32_t>(kSliceK), static_cast<cuuint32_t>(box_rows)};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(IVF_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return IVF_OK;
+}
+
+// ------------------------------------------------------------------ argument checks (no CUDA calls)
+int check_common(const void* points, int64_t n, int d, int ptype, const float* centroids, int nlist, int k,
+                 const int32_t* out_ids) {
+    if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
+    if (ptype != IVF_F32 && ptype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", ptype);
+    if (d < 16 || d > 256 || d % 16 != 0)
+        return fail(IVF_ERR_UNSUPPORTED, "d = %d: must be a multiple of 16 in [16, 256]", d);
+    if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
+    if (k < 1 || k > nlist || k > 512)
+        return fail(IVF_ERR_UNSUPPORTED, "nprobe = %d: must be in [1, min(nlist, 512)] (nlist = %d)", k, nlist);
+    if (n == 0) return IVF_OK;
+    if (!points || !centroids || !out_ids) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    if ((reinterpret_cast<uintptr_t>(points) & 15) || (reinterpret_cast<uintptr_t>(centroids) & 15))
+        return fail(IVF_ERR_INVALID_ARG, "points and centroids must be 16-byte aligned");
+    return IVF_OK;
+}
+
+// 0 = device (or managed), 1 = page-locked host, <0 = error
+int classify_pointer(const void* p) {
+    cudaPointerAttributes attr;
+    cudaError_t e = cudaPointerGetAttributes(&attr, p);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return fail(IVF_ERR_CUDA, "cudaPointerGetAttributes failed: %s", cudaGetErrorString(e));
+    }
+    if (attr.type == cudaMemoryTypeDevice || attr.type == cudaMemoryTypeManaged) return 0;
+    if (attr.type == cudaMemoryTypeHost) return 1;
+    return fail(IVF_ERR_INVALID_ARG, "pageable host memory is not accepted: pass device or page-locked host memory");
+}
+
+// ------------------------------------------------------------------ device-resident building blocks
+struct CentroidPrep {
+    __half* c16;
+    float* cn;
+    float* scal;
+    unsigned int* bits;
+    CUtensorMap tmap_c;
+};
+
+int prepare_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, const Plan& pl, cudaStream_t stream,
+                      CentroidPrep* cp) {
+    const int64_t padded = static_cast<int64_t>(pl.col_tiles) * pl.block_n;
+    WS(WS_C16, static_cast<size_t>(nlist) * pl.kp * sizeof(__half), cp->c16);
+    WS(WS_CN, static_cast<size_t>(padded) * sizeof(float), cp->cn);
+    WS(WS_SCAL, 4 * sizeof(float), cp->scal);
+    WS(WS_BITS, 2 * sizeof(unsigned int), cp->bits);
+    CUDA_TRY(cudaMemsetAsync(cp->bits, 0, 2 * sizeof(unsigned int), stream));
+    const int64_t count = static_cast<int64_t>(nlist) * d;
+    int blocks = static_cast<int>((count + 256 * 8 - 1) / (256 * 8));
+    if (blocks > ctx.num_sms * 8) blocks = ctx.num_sms * 8;
+    maxabs_kernel<<<blocks, 256, 0, stream>>>(centroids, count, cp->bits + 1);
+    LAUNCH_CHECK();
+    scales_kernel<<<1, 1, 0, stream>>>(cp->bits, 1, cp->scal);
+    LAUNCH_CHECK();
+    const int64_t threads = padded * 32;
+    convert_rows_kernel<float><<<static_cast<unsigned>((threads + 255) / 256), 256, 0, stream>>>(
+        centroids, nlist, padded, d, pl.kp, cp->scal, 1, cp->c16, cp->cn);
+    LAUNCH_CHECK();
+    return make_tmap(&cp->tmap_c, cp->c16, nlist, pl.kp, pl.block_n);
+}
+
+// Routes `n` device-resident rows against prepared centroids (one fused launch + one merge).
+int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int ptype, int nlist, int k,
+                      const CentroidPrep& cp, int32_t* out_ids, float* out_dists, cudaStream_t stream) {
+    Plan pl;
+    int rc = make_plan(n, nlist, d, k, ctx.num_sms, &pl);
+    if (rc != IVF_OK) return rc;
+    __half* x16;
+    float* xn;
+    Entry* part;
+    int* part_cnt = nullptr;
+    WS(WS_X16, static_cast<size_t>(n) * pl.kp * sizeof(__half), x16);
+    WS(WS_XN, static_cast<size_t>(n) * sizeof(float), xn);
+    WS(WS_PART, static_cast<size_t>(n) * pl.partials * pl.cap * sizeof(Entry), part);
+    if (k > 1) WS(WS_PARTCNT, static_cast<size_t>(n) * pl.partials * sizeof(int), part_cnt);
+
+    const int u8 = ptype == IVF_U8;
+    if (!u8) {
+        CUDA_TRY(cudaMemsetAsync(cp.bits, 0, sizeof(unsigned int), stream));
+        const int64_t count = n * d;
+        int blocks = static_cast<int>((count + 256 * 8 - 1) / (256 * 8));
+        if (blocks > ctx.num_sms * 8) blocks = ctx.num_sms * 8;
+        maxabs_kernel<<<blocks, 256, 0, stream>>>(static_cast<const float*>(points), count, cp.bits);
+        LAUNCH_CHECK();
+    }
+    scales_kernel<<<1, 1, 0, stream>>>(cp.bits, u8, cp.scal);
+    LAUNCH_CHECK();
+    const int64_t threads = n * 32;
+    const unsigned cblocks = static_cast<unsigned>((threads + 255) / 256);
+    if (u8)
+        convert_rows_kernel<uint8_t><<<cblocks, 256, 0, stream>>>(static_cast<const uint8_t*>(points), n, n, d, pl.kp,
+                                                                  cp.scal, 0, x16, xn);
+    else
+        convert_rows_kernel<float><<<cblocks, 256, 0, stream>>>(static_cast<const float*>(points), n, n, d, pl.kp,
+                                                                cp.scal, 0, x16, xn);
+    LAUNCH_CHECK();
+
+    CUtensorMap tmap_x;
+    rc = make_tmap(&tmap_x, x16, n, pl.kp, kBlockM);
+    if (rc != IVF_OK) return rc;
+
+    FusedParams fp;
+    fp.n = n;
+    fp.nlist = nlist;
+    fp.k = k;
+    fp.mode = (k == 1) ? MODE_ARGMIN : MODE_APPEND;
+    fp.ksteps = pl.ksteps;
+    fp.kslices = pl.kslices;
+    fp.block_n = pl.block_n;
+    fp.nstage = pl.nstage;
+    fp.col_tiles = pl.col_tiles;
+    fp.total_units = pl.total_units;
+    fp.partials = pl.partials;
+    fp.cap = pl.cap;
+    fp.cn = cp.cn;
+    fp.scal = cp.scal;
+    fp.part = part;
+    fp.part_cnt = part_cnt;
+    fp.status = ctx.status;
+    fp.wait_limit_ns = g_wait_limit_ns.load();
+    if (!ctx.smem_attr_set) {
+        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      static_cast<int>(kSmemLimit)));
+        ctx.smem_attr_set = true;
+    }
+    fused_topk_kernel<<<pl.ctas, kFusedThreads, pl.smem, stream>>>(tmap_x, cp.tmap_c, fp);
+    LAUNCH_CHECK();
+
+    MergeParams mp;
+    mp.n = n;
+    mp.k = k;
+    mp.partials = pl.partials;
+    mp.cap = pl.cap;
+    mp.col_tiles = pl.col_tiles;
+    mp.total_units = pl.total_units;
+    mp.ctas = pl.ctas;
+    mp.part = part;
+    mp.part_cnt = part_cnt;
+    mp.xn = xn;
+    mp.out_ids = out_ids;
+    mp.out_dists = out_dists;
+    if (k == 1) {
+        merge_argmin_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(mp);
+    } else {
+        merge_select_kernel<<<static_cast<unsigned>(n), kMergeThreads, 0, stream>>>(mp);
+    }
+    LAUNCH_CHECK();
+    return IVF_OK;
+}
+
+int update_device(DeviceCtx& ctx, const void* points, int ptype, const int32_t* ids, int64_t n, int d, int nlist,
+                  float* sums, int64_t* counts, cudaStream_t stream) {
+    int *cnt, *off, *cur, *perm;
+    WS(WS_UCNT, static_cast<size_t>(nlist) * sizeof(int), cnt);
+    WS(WS_UOFF, (static_cast<size_t>(nlist) + 1) * sizeof(int), off);
+    WS(WS_UCUR, static_cast<size_t>(nlist) * sizeof(int), cur);
+    WS(WS_UPERM, static_cast<size_t>(n) * sizeof(int), perm);
+    CUDA_TRY(cudaMemsetAsync(cnt, 0, static_cast<size_t>(nlist) * sizeof(int), stream));
+    const unsigned rb = static_cast<unsigned>((n + 255) / 256);
+    update_hist_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, cnt, ctx.status);
+    LAUNCH_CHECK();
+    update_scan_kernel<<<1, 1024, 0, stream>>>(cnt, nlist, off, cur);
+    LAUNCH_CHECK();
+    update_fill_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, off, cur, perm);
+    LAUNCH_CHECK();
+    const unsigned lb = static_cast<unsigned>((static_cast<int64_t>(nlist) * 32 + 255) / 256);
+    if (ptype == IVF_U8)
+        update_reduce_kernel<uint8_t><<<lb, 256, 0, stream>>>(static_cast<const uint8_t*>(points), perm, off, nlist, d,
+                                                              sums, reinterpret_cast<long long*>(counts));
+    else
+        update_reduce_kernel<float><<<lb, 256, 0, stream>>>(static_cast<const float*>(points), perm, off, nlist, d,
+                                                            sums, reinterpret_cast<long long*>(counts));
+    LAUNCH_CHECK();
+    return IVF_OK;
+}
+
+// ------------------------------------------------------------------ the chunk pipeline
+// Walks the rows in chunks; a host-resident chunk is staged through one of two device buffers on
+// the copy stream.  `with_update` adds the Lloyd accumulation of each chunk.
+int run_chunks(const void* points, int64_t n, int d, int ptype, const float* centroids, int nlist, int k,
+               int32_t* out_ids, float* out_dists, bool with_update, float* sums, int64_t* counts,
+               int64_t chunk_rows, cudaStream_t stream) {
+    DeviceCtx* pctx = nullptr;
+    int rc = get_ctx(&pctx);
+    if (rc != IVF_OK) return rc;
+    DeviceCtx& ctx = *pctx;
+    rc = get_encode();
+    if (rc != IVF_OK) return rc;
+    const int where = classify_pointer(points);
+    if (where < 0) return where;
+    const bool host = where == 1;
+    const size_t esize = ptype == IVF_U8 ? 1 : 4;
+
+    int64_t rows = rows_per_launch(d, k);
+    if (chunk_rows <= 0) chunk_rows = int64_t(1) << 20;
+    if ((host || with_update) && rows > chunk_rows) rows = chunk_rows;
+    if (rows > n) rows = n;
+    const int64_t nchunks = (n + rows - 1) / rows;
+
+    Plan pl0;
+    rc = make_plan(rows, nlist, d, k, ctx.num_sms, &pl0);
+    if (rc != IVF_OK) return rc;
+    CentroidPrep cp;
+    rc = prepare_centroids(ctx, centroids, nlist, d, pl0, stream, &cp);
+    if (rc != IVF_OK) return rc;
+
+    uint8_t* stage[2] = {nullptr, nullptr};
+    int32_t* tmp_ids = nullptr;
+    if (host) {
+        WS(WS_CHUNK0, static_cast<size_t>(rows) * d * esize, stage[0]);
+        if (nchunks > 1) WS(WS_CHUNK1, static_cast<size_t>(rows) * d * esize, stage[1]);
+        // the copy stream may touch the staging buffers only after their allocation on `stream`
+        CUDA_TRY(cudaEventRecord(ctx.ev_ready, stream));
+        CUDA_TRY(cudaStreamWaitEvent(ctx.copy_stream, ctx.ev_ready, 0));
+    }
+    if (with_update && !out_ids) WS(WS_IDS, static_cast<size_t>(rows) * sizeof(int32_t), tmp_ids);
+
+    auto issue_copy = [&](int64_t c) -> int {
+        const int64_t r0 = c * rows;
+        const int64_t nr = (n - r0 < rows) ? (n - r0) : rows;
+        const int sb = static_cast<int>(c & 1);
+        CUDA_TRY(cudaStreamWaitEvent(ctx.copy_stream, ctx.ev_free[sb], 0));
+        CUDA_TRY(cudaMemcpyAsync(stage[sb], static_cast<const uint8_t*>(points) + static_cast<size_t>(r0) * d * esize,
+                                 static_cast<size_t>(nr) * d * esize, cudaMemcpyHostToDevice, ctx.copy_stream));
+        CUDA_TRY(cudaEventRecord(ctx.ev_copied[sb], ctx.copy_stream));
+        return IVF_OK;
+    };
+
+    if (host) {
+        rc = issue_copy(0);
+        if (rc != IVF_OK) return rc;
+    }
+    for (int64_t c = 0; c < nchunks; ++c) {
+        const int64_t r0 = c * rows;
+        const int64_t nr = (n - r0 < rows) ? (n - r0) : rows;
+        const int sb = static_cast<int>(c & 1);
+        const void* chunk;
+        if (host) {
+            if (c + 1 < nchunks) {
+                rc = issue_copy(c + 1);
+                if (rc != IVF_OK) return rc;
+            }
+            CUDA_TRY(cudaStreamWaitEvent(stream, ctx.ev_copied[sb], 0));
+            chunk = stage[sb];
+        } else {
+            chunk = static_cast<const uint8_t*>(points) + static_cast<size_t>(r0) * d * esize;
+        }
+        int32_t* ids_c = out_ids ? out_ids + r0 * k : tmp_ids;
+        float* dists_c = out_dists ? out_dists + r0 * k : nullptr;
+        rc = route_rows_device(ctx, chunk, nr, d, ptype, nlist, k, cp, ids_c, dists_c, stream);
+        if (rc != IVF_OK) return rc;
+        if (with_update) {
+            rc = update_device(ctx, chunk, ptype, ids_c, nr, d, nlist, sums, counts, stream);
+            if (rc != IVF_OK) return rc;
+        }
+        if (host) CUDA_TRY(cudaEventRecord(ctx.ev_free[sb], stream));
+    }
+    return IVF_OK;
+}
+
+}  // namespace
+
+// ====================================================================== exported C functions
+extern "C" {
+
+int ivf_route(const void* queries, int64_t nq, int d, ivf_dtype qtype, const float* centroids, int nlist, int nprobe,
+              int32_t* out_ids, float* out_dists, void* stream) {
+    int rc = check_common(queries, nq, d, qtype, centroids, nlist, nprobe, out_ids);
+    if (rc != IVF_OK || nq == 0) return rc;
+    return run_chunks(queries, nq, d, qtype, centroids, nlist, nprobe, out_ids, out_dists, false, nullptr, nullptr, 0,
+                      static_cast<cudaStream_t>(stream));
+}
+
+int ivf_assign(const void* points, int64_t n, int d, ivf_dtype ptype, const float* centroids, int nlist,
+               int32_t* out_ids, float* out_dists, void* stream) {
+    int rc = check_common(points, n, d, ptype, centroids, nlist, 1, out_ids);
+    if (rc != IVF_OK || n == 0) return rc;
+    return run_chunks(points, n, d, ptype, centroids, nlist, 1, out_ids, out_dists, false, nullptr, nullptr, 0,
+                      static_cast<cudaStream_t>(stream));
+}
+
+int ivf_centroid_update(const void* points, ivf_dtype ptype, const int32_t* ids, int64_t n, int d, int nlist,
+                        float* sums, int64_t* counts, void* stream) {
+    if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
+    if (ptype != IVF_F32 && ptype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
+    if (d < 16 || d > 256 || d % 16 != 0)
+        return fail(IVF_ERR_UNSUPPORTED, "d = %d: must be a multiple of 16 in [16, 256]", d);
+    if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
+    if (n >= (int64_t(1) << 31)) return fail(IVF_ERR_UNSUPPORTED, "n = %lld: at most 2^31 - 1 rows per call", (long long)n);
+    if (n == 0) return IVF_OK;
+    if (!points || !ids || !sums || !counts) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    if ((reinterpret_cast<uintptr_t>(points) & 15) || (reinterpret_cast<uintptr_t>(sums) & 15))
+        return fail(IVF_ERR_INVALID_ARG, "points and sums must be 16-byte aligned");
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != IVF_OK) return rc;
+    return update_device(*ctx, points, ptype, ids, n, d, nlist, sums, counts, static_cast<cudaStream_t>(stream));
+}
+
+int ivf_centroid_finalize(const float* sums, const int64_t* counts, int nlist, int d, float* centroids_inout,
+                          void* stream) {
+    if (nlist < 1 || d < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d, d = %d", nlist, d);
+    if (!sums || !counts || !centroids_inout) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    const int64_t total = static_cast<int64_t>(nlist) * d;
+    finalize_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        sums, reinterpret_cast<const long long*>(counts), nlist, d, centroids_inout);
+    LAUNCH_CHECK();
+    return IVF_OK;
+}
+
+int ivf_assign_update(const void* points, int64_t n, int d, ivf_dtype ptype, const float* centroids, int nlist,
+                      int32_t* out_ids, float* out_dists, float* sums, int64_t* counts, int64_t chunk_rows,
+                      void* stream) {
+    int32_t dummy = 0;
+    int rc = check_common(points, n, d, ptype, centroids, nlist, 1, out_ids ? out_ids : &dummy);
+    if (rc != IVF_OK || n == 0) return rc;
+    if (!sums || !counts) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    if (reinterpret_cast<uintptr_t>(sums) & 15) return fail(IVF_ERR_INVALID_ARG, "sums must be 16-byte aligned");
+    return run_chunks(points, n, d, ptype, centroids, nlist, 1, out_ids, out_dists, true, sums, counts, chunk_rows,
+                      static_cast<cudaStream_t>(stream));
+}
+
+int ivf_check(void* stream) {
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != IVF_OK) return rc;
+    CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    int h[4] = {0, 0, 0, 0};
+    CUDA_TRY(cudaMemcpy(h, ctx->status, sizeof h, cudaMemcpyDeviceToHost));
+    if (h[0] != 0) {
+        CUDA_TRY(cudaMemset(ctx->status, 0, sizeof h));
+        if (h[0] == IVF_ERR_DEVICE_TIMEOUT)
+            return fail(IVF_ERR_DEVICE_TIMEOUT, "a device-side wait expired (wait site %d, block %d)", h[1], h[2]);
+        if (h[0] == IVF_ERR_BAD_ID) return fail(IVF_ERR_BAD_ID, "ivf_centroid_update skipped ids outside [0, nlist)");
+        return fail(h[0], "device status %d", h[0]);
+    }
+    return IVF_OK;
+}
+
+const char* ivf_last_error(void) { return g_err.c_str(); }
+
+int ivf_release_workspace(void) {
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    CUDA_TRY(cudaDeviceSynchronize());
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx& c = g_ctx[dev];
+    for (Buf& b : c.bufs) {
+        if (b.p) CUDA_TRY(cudaFree(b.p));
+        b.p = nullptr;
+        b.cap = 0;
+    }
+    return IVF_OK;
+}
+
+int64_t ivf_launch_count(void) { return g_launches.load(); }
+
+int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[8]) {
+    if (n < 1 || nlist < 1 || num_sms < 1 || !out) return fail(IVF_ERR_INVALID_ARG, "bad plan arguments");
+    if (d < 16 || d > 256 || d % 16 != 0) return fail(IVF_ERR_UNSUPPORTED, "d = %d", d);
+    Plan pl;
+    int rc = make_plan(n, nlist, d, k, num_sms, &pl);
+    if (rc != IVF_OK) return rc;
+    out[0] = pl.row_tiles;
+    out[1] = pl.col_tiles;
+    out[2] = pl.ctas;
+    out[3] = pl.partials;
+    out[4] = pl.block_n;
+    out[5] = pl.kslices;
+    out[6] = pl.nstage;
+    out[7] = static_cast<int64_t>(pl.smem);
+    return IVF_OK;
+}
+
+int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int64_t out[2]) {
+    if (n < 1 || nlist < 1 || num_sms < 1 || !out) return fail(IVF_ERR_INVALID_ARG, "bad plan arguments");
+    Plan pl;
+    int rc = make_plan(n, nlist, d, k, num_sms, &pl);
+    if (rc != IVF_OK) return rc;
+    if (cta < 0 || cta >= pl.ctas) return fail(IVF_ERR_INVALID_ARG, "cta %d outside [0, %d)", cta, pl.ctas);
+    out[0] = span_begin(pl.total_units, pl.ctas, cta);
+    out[1] = span_begin(pl.total_units, pl.ctas, cta + 1);
+    return IVF_OK;
+}
+
+int ivf_debug_set_wait_limit_ns(int64_t ns) {
+    g_wait_limit_ns.store(ns > 0 ? static_cast<uint64_t>(ns) : 2000000000ull);
+    return IVF_OK;
+}
+
+}  // extern "C"

