@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the IVF routing / assignment hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic input:
+    route   10,000 uint8 queries (d = 128) against 65,536 float32 centroids, nprobe = 64
+            (the SIFT-shaped routing configuration)
+    assign  one 1,048,576-row uint8 chunk of the IVF-build configuration against the same number
+            of centroids (k = 1), with the per-list sum/count update of that chunk
+    finalize  new centroids from the sums and counts
+Inputs are resident in HBM before the timed region; `e2e` repeats the routing through the same C
+calls with the queries in page-locked host memory and the results copied back to the host.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Under torchrun (N > 1) every rank runs the same per-GPU workload on its own rows (weak scaling);
+the only exchange is the all-reduce of the Lloyd sums and counts before the finalize.
+`--impl reference` times the CPU oracle, as it stands, on a bounded sample of the routing rows.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+NQ, NLIST, D, NPROBE = 10_000, 65_536, 128, 64
+CHUNK = 1 << 20
+WORKLOAD = ("C1 SIFT-shaped routing (10000 u8 queries x 65536 f32 centroids, d=128, nprobe=64) + one 1048576-row "
+            "u8 chunk of the IVF-build configuration: assign (k=1) + per-list sum/count update + finalize")
+METRIC = "routed queries/s"
+UNIT = "queries/s"
+
+# DRAM bytes (read + write) per launch of the dominant kernel from the ncu capture summarised in
+# profiles/; None until a capture exists.
+TRAFFIC_FUSED_ARGMIN_BYTES = None
+TRAFFIC_FUSED_TOPK_BYTES = None
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "tf_burst": p["bf16_tflops"], "tf_sustained": p["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tf_burst": 1590.0, "tf_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx = [], []
+        reasons = set()
+        try:
+            for line in open(self.path):
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 8:
+                    continue
+                try:
+                    sm.append(float(parts[0]))
+                    mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     parts[4:8]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            # under load = the upper half of the samples (idle gaps between steps read lower clocks)
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def make_inputs(rank: int):
+    from paper_2608_08751_b200 import synth
+    cent = synth.sift_like_centroids(NLIST, D)
+    if rank == 0:
+        queries = synth.sift_like_queries(NQ, D)
+    else:
+        queries = synth.sift_like_rows(1000 + rank, rows=NQ)
+    chunk = synth.sift_like_rows(rank, rows=CHUNK)
+    return queries, cent, chunk
+
+
+def run_reference(args, rank: int, world: int):
+    """The CPU oracle, as it stands, on a bounded sample of the routing rows (rank 0 only)."""
+    if rank != 0:
+        return
+    from oracle import oracle
+    from paper_2608_08751_b200 import synth
+    cores = oracle.num_threads()
+    rows = max(32, 16 * cores)
+    q = synth.sift_like_queries(NQ, D)
+    c = synth.sift_like_centroids(NLIST, D)
+    sample = np.ascontiguousarray(q[np.random.default_rng(0).choice(NQ, rows, replace=False)])
+    for _ in range(args.warmup):
+        oracle.route(sample[: max(8, rows // 8)], c, NPROBE)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.route(sample, c, NPROBE)
+    dt = time.perf_counter() - t0
+    value = rows * args.steps / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": f"{rows} of the {NQ} routing rows per step, full centroid width"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{rows} seeded rows of the C1 routing batch per step x {args.steps} steps"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else max(args.warmup, 0)
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2608_08751_b200 import binding as B
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    distributed = world > 1
+    if distributed:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    queries_np, cent_np, chunk_np = make_inputs(rank)
+    queries = torch.from_numpy(queries_np).to(dev)
+    cent_route = torch.from_numpy(cent_np).to(dev)
+    cent_lloyd = cent_route.clone()
+    chunk = torch.from_numpy(chunk_np).to(dev)
+    q_host = torch.from_numpy(queries_np).pin_memory()
+    out_ids = torch.empty((NQ, NPROBE), dtype=torch.int32, device=dev)
+    out_dists = torch.empty((NQ, NPROBE), dtype=torch.float32, device=dev)
+    ids_host = torch.empty((NQ, NPROBE), dtype=torch.int32).pin_memory()
+    dists_host = torch.empty((NQ, NPROBE), dtype=torch.float32).pin_memory()
+    a_ids = torch.empty((CHUNK,), dtype=torch.int32, device=dev)
+    a_dists = torch.empty((CHUNK,), dtype=torch.float32, device=dev)
+    sums = torch.zeros((NLIST, D), dtype=torch.float32, device=dev)
+    counts = torch.zeros((NLIST,), dtype=torch.int64, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)  # > 126 MB of L2
+
+    def step(ev=None):
+        if ev:
+            ev[0].record()
+        B.ivf_route(queries, cent_route, NPROBE, out_ids, out_dists)
+        if ev:
+            ev[1].record()
+        sums.zero_()
+        counts.zero_()
+        B.ivf_assign_update(chunk, cent_lloyd, sums, counts, a_ids, a_dists)
+        if distributed:
+            dist.all_reduce(sums)
+            dist.all_reduce(counts)
+        if ev:
+            ev[2].record()
+        B.ivf_centroid_finalize(sums, counts, cent_lloyd)
+        if ev:
+            ev[3].record()
+
+    for _ in range(args.warmup):
+        step()
+        flush.zero_()
+    B.ivf_check(dev)
+
+    def barrier():
+        if distributed:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    sampler = ClockSampler(local_rank)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    B.ivf_debug_timing(True)
+    launches0 = B.ivf_launch_count()
+    barrier()
+    sampler.start()
+    t_wall = time.perf_counter()
+    for s in range(args.steps):
+        step(events[s])
+        flush.zero_()  # L2 flush between timed iterations (outside the per-step events)
+    barrier()
+    t_wall = time.perf_counter() - t_wall
+    clocks = sampler.stop()
+    launches = B.ivf_launch_count() - launches0
+    fam = B.ivf_debug_timing_read()
+    B.ivf_debug_timing(False)
+    B.ivf_check(dev)
+
+    t_route = sum(e[0].elapsed_time(e[1]) for e in events)
+    t_assign = sum(e[1].elapsed_time(e[2]) for e in events)
+    t_final = sum(e[2].elapsed_time(e[3]) for e in events)
+    t_step = sum(e[0].elapsed_time(e[3]) for e in events)
+    times = torch.tensor([t_route, t_assign, t_final, t_step], dtype=torch.float64, device=dev)
+    if distributed:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    t_route, t_assign, t_final, t_step = (float(v) for v in times.cpu())
+
+    # ---- end to end: queries in page-locked host memory, results copied back to the host
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(2):
+        B.ivf_route(q_host, cent_route, NPROBE, out_ids, out_dists)
+        ids_host.copy_(out_ids, non_blocking=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        B.ivf_route(q_host, cent_route, NPROBE, out_ids, out_dists)
+        ids_host.copy_(out_ids, non_blocking=True)
+        dists_host.copy_(out_dists, non_blocking=True)
+    e1.record()
+    barrier()
+    t_e2e = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if distributed:
+        dist.all_reduce(t_e2e, op=dist.ReduceOp.MAX)
+    t_e2e = float(t_e2e.cpu()[0])
+    B.ivf_check(dev)
+
+    if rank != 0:
+        if distributed:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    K = args.steps
+    qps = world * NQ * K / (t_route / 1e3)
+    vps = world * CHUNK * K / (t_assign / 1e3)
+    arg_ms, arg_n = fam["fused_argmin"]
+    top_ms, top_n = fam["fused_topk"]
+    upd_ms, upd_n = fam["update"]
+    mrg_ms, mrg_n = fam["merge"]
+    prep_ms, prep_n = fam["prep"]
+    flops_assign = 2.0 * CHUNK * NLIST * D
+    flops_route = 2.0 * NQ * NLIST * D
+    peak_tf = pk["tf_sustained"]
+    ach_arg = flops_assign / (arg_ms / max(arg_n, 1) / 1e3) / 1e12 if arg_n else None
+    ach_top = flops_route / (top_ms / max(top_n, 1) / 1e3) / 1e12 if top_n else None
+    upd_bytes = CHUNK * D + CHUNK * 4 * 3 + NLIST * D * 4 * 2 + NLIST * 8 * 2
+    line = {
+        "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+        "ms_per_step": t_step / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f16 operands (uint8 exact), f32 accumulate", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "l2": "256 MB buffer rewritten between timed steps, outside the per-step events",
+                   "exchange": "all-reduce of sums/counts per step" if distributed else "none (1 GPU)"},
+        "assigned_vectors_per_s": vps,
+        "phases_ms_per_step": {"route": t_route / K, "assign_update": t_assign / K, "finalize": t_final / K},
+        "kernel_ms_per_launch": {
+            "prep": prep_ms / max(prep_n, 1), "fused_topk_k64": top_ms / max(top_n, 1),
+            "fused_argmin_k1": arg_ms / max(arg_n, 1), "merge": mrg_ms / max(mrg_n, 1),
+            "centroid_update": upd_ms / max(upd_n, 1)},
+        "roofline": {"kernel": "fused_topk_kernel (k=1, 1048576 x 65536 x 128)", "bound": "tensor",
+                     "achieved": ach_arg, "peak": peak_tf, "unit": "TFLOP/s",
+                     "frac": (ach_arg / peak_tf) if ach_arg else None, "traffic": TRAFFIC_FUSED_ARGMIN_BYTES,
+                     "peak_source": f"{pk['source']}: 16-bit dense, sustained"},
+        "roofline_route": {"kernel": "fused_topk_kernel (k=64, 10000 x 65536 x 128)", "bound": "tensor",
+                           "achieved": ach_top, "peak": pk["tf_burst"], "unit": "TFLOP/s",
+                           "frac": (ach_top / pk["tf_burst"]) if ach_top else None,
+                           "traffic": TRAFFIC_FUSED_TOPK_BYTES, "peak_source": f"{pk['source']}: 16-bit dense, burst"},
+        "roofline_update": {"kernel": "centroid update (hist+scan+fill+reduce)", "bound": "hbm",
+                            "achieved": upd_bytes / (upd_ms / max(upd_n, 1) / 1e3) / 1e9 if upd_n else None,
+                            "peak": pk["hbm_gbs"], "unit": "GB/s",
+                            "frac": (upd_bytes / (upd_ms / max(upd_n, 1) / 1e3) / 1e9 / pk["hbm_gbs"]) if upd_n else None,
+                            "traffic": None, "peak_source": pk["source"]},
+        "e2e": {"value": world * NQ * K / (t_e2e / 1e3), "unit": UNIT, "h2d_bytes_per_step": NQ * D,
+                "d2h_bytes_per_step": NQ * NPROBE * 8},
+        "gpu_launches": int(launches),
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"]},
+        "wall_s_timed_region": t_wall,
+    }
+
+    if not args.no_cpu_baseline and world == 1:
+        from oracle import oracle
+        cores = oracle.num_threads()
+        rows = max(64, 48 * cores)
+        sel = np.random.default_rng(1).choice(NQ, rows, replace=False)
+        sample = np.ascontiguousarray(queries_np[sel])
+        t0 = time.perf_counter()
+        o_ids, o_d, _ = oracle.route(sample, cent_np, NPROBE)
+        dt = time.perf_counter() - t0
+        g_ids = out_ids.cpu().numpy()[sel]
+        line["cpu_baseline"] = {"value": rows / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{rows} seeded rows of the C1 routing batch, full centroid width, {dt:.1f} s",
+                                "ids_identical_to_gpu": float((g_ids == o_ids).all(axis=1).mean())}
+    print(json.dumps(line), flush=True)
+    if distributed:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -125,12 +125,26 @@ int64_t ivf_launch_count(void);
  *                    block_n, k_slices, stages, smem_bytes} to out[8].
  *   ivf_debug_span   first unit and one-past-last unit of CTA `cta` in that schedule.
  *   ivf_debug_set_wait_limit_ns   time limit of every device-side wait (0 restores the default
- *                    of 2 s); with a tiny limit a launch reports IVF_ERR_DEVICE_TIMEOUT through
- *                    ivf_check and still returns normally.
+ *                    of 2 s).
+ *   ivf_debug_wait_probe   launches a one-warp kernel that waits, with the library's bounded wait,
+ *                    on a barrier nothing ever completes: after the limit it records
+ *                    IVF_ERR_DEVICE_TIMEOUT (wait site 99) in the status word and returns normally.
  */
 int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[8]);
 int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int64_t out[2]);
 int ivf_debug_set_wait_limit_ns(int64_t ns);
+int ivf_debug_wait_probe(void* stream);
+
+/*
+ * Measurement hooks.  ivf_debug_timing(1) makes every later call bracket its kernels with CUDA
+ * events on the caller's stream, grouped into five families: 0 operand preparation (norms,
+ * fp16 copies), 1 fused distance+argmin (k = 1), 2 fused distance+top-k (k > 1), 3 merge of
+ * partial results, 4 centroid update.  ivf_debug_timing_read synchronises the device, writes the
+ * summed milliseconds and launch-group counts of each family since the last read, and clears
+ * them.  ivf_debug_timing(0) switches the events off (the default).
+ */
+int ivf_debug_timing(int enable);
+int ivf_debug_timing_read(double ms[5], int64_t launches[5]);
 
 #ifdef __cplusplus
 }

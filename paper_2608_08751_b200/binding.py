@@ -23,6 +23,7 @@ EXPORTS = (
     "ivf_route", "ivf_assign", "ivf_centroid_update", "ivf_centroid_finalize", "ivf_assign_update",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
     "ivf_debug_plan", "ivf_debug_span", "ivf_debug_set_wait_limit_ns",
+    "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe",
 )
 
 _lib = None
@@ -59,6 +60,9 @@ def lib() -> ctypes.CDLL:
     L.ivf_debug_plan.argtypes = [i64, i32, i32, i32, i32, ctypes.POINTER(i64)]
     L.ivf_debug_span.argtypes = [i64, i32, i32, i32, i32, i32, ctypes.POINTER(i64)]
     L.ivf_debug_set_wait_limit_ns.argtypes = [i64]
+    L.ivf_debug_timing.argtypes = [i32]
+    L.ivf_debug_wait_probe.argtypes = [vp]
+    L.ivf_debug_timing_read.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
     for name in EXPORTS:
         if name not in ("ivf_last_error", "ivf_launch_count"):
             getattr(L, name).restype = i32
@@ -236,3 +240,28 @@ def ivf_debug_span(n: int, nlist: int, d: int, k: int, num_sms: int, cta: int):
 
 def ivf_debug_set_wait_limit_ns(ns: int) -> None:
     lib().ivf_debug_set_wait_limit_ns(ns)
+
+
+TIMING_FAMILIES = ("prep", "fused_argmin", "fused_topk", "merge", "update")
+
+
+def ivf_debug_timing(enable: bool) -> None:
+    lib().ivf_debug_timing(1 if enable else 0)
+
+
+def ivf_debug_timing_read() -> dict:
+    """{family: (milliseconds, launch groups)} since the last read; synchronises the device."""
+    ms = (ctypes.c_double * 5)()
+    cnt = (ctypes.c_int64 * 5)()
+    rc = lib().ivf_debug_timing_read(ms, cnt)
+    if rc != IVF_OK:
+        _raise(rc)
+    return {name: (float(ms[i]), int(cnt[i])) for i, name in enumerate(TIMING_FAMILIES)}
+
+
+def ivf_debug_wait_probe() -> None:
+    """Launches the orphaned-wait probe on the current stream (see the header)."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    rc = lib().ivf_debug_wait_probe(_stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)

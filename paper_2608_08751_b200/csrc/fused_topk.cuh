@@ -179,6 +179,24 @@ __device__ __noinline__ float warp_select_k(Entry* log, int c, int k, int* hist,
     return from_orderable(T);
 }
 
+// A wait on a barrier that nothing ever completes: exercises the bounded wait and the status word
+// without any copy or MMA in flight.
+__global__ void wait_probe_kernel(int* status, uint64_t limit_ns) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    WaitCtl ctl;
+    ctl.abort_flag = &abort_flag;
+    ctl.status = status;
+    ctl.limit_ns = limit_ns;
+    (void)mbar_wait(&bar, 0, ctl, 99);
+}
+
 __device__ __forceinline__ float min3f(float a, float b, float c) { return fminf(fminf(a, b), c); }
 
 __global__ void __launch_bounds__(kFusedThreads, 1)
@@ -197,7 +215,8 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     uint64_t* t_empty = bars + 4;   // [2]
     uint64_t* b_full = bars + 6;    // [kMaxStages]
     uint64_t* b_empty = bars + 6 + kMaxStages;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 6 + 2 * kMaxStages);
+    uint64_t* drain = bars + 6 + 2 * kMaxStages;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 7 + 2 * kMaxStages);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* hist_all = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(bars) + 256);
 
@@ -213,6 +232,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     if (threadIdx.x == 0) {
         mbar_init(a_full, 1);
         mbar_init(a_empty, 1);
+        mbar_init(drain, 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(&t_full[i], 1);
             mbar_init(&t_empty[i], kNumEpiWarps);
@@ -327,6 +347,13 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 if (ok) umma_commit(a_empty);
                 ++seg;
                 u = r * NT + t1;
+            }
+            if (!ok && it > 0) {
+                // gave up: wait (bounded) until the MMAs already issued have retired before TMEM is freed
+                umma_commit(drain);
+                const uint64_t t_start = global_timer_ns();
+                while (!mbar_try_wait(drain, 0) && global_timer_ns() - t_start < 2000000000ull) {
+                }
             }
         }
     } else {

@@ -14,6 +14,7 @@
 #include <mutex>
 #include <string>
 #include <type_traits>
+#include <vector>
 
 #include "fused_topk.cuh"
 #include "merge.cuh"
@@ -52,6 +53,32 @@ int fail(int code, const char* fmt, ...) {
         g_launches.fetch_add(1);          \
         CUDA_TRY(cudaGetLastError());     \
     } while (0)
+
+// ------------------------------------------------------------------ optional per-kernel timing
+// When enabled, launches of each kernel family are bracketed by CUDA events on the caller's stream.
+enum TimedKind { TK_PREP = 0, TK_FUSED_ARGMIN, TK_FUSED_TOPK, TK_MERGE, TK_UPDATE, TK_NUM };
+struct TimedLaunch {
+    cudaEvent_t a, b;
+    int kind;
+};
+std::vector<TimedLaunch> g_timed;
+bool g_timing = false;
+
+int timing_begin(int kind, cudaStream_t stream) {
+    if (!g_timing) return -1;
+    TimedLaunch t;
+    t.kind = kind;
+    if (cudaEventCreate(&t.a) != cudaSuccess || cudaEventCreate(&t.b) != cudaSuccess) return -1;
+    cudaEventRecord(t.a, stream);
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_timed.push_back(t);
+    return static_cast<int>(g_timed.size()) - 1;
+}
+void timing_end(int idx, cudaStream_t stream) {
+    if (idx < 0) return;
+    std::lock_guard<std::mutex> lk(g_mu);
+    cudaEventRecord(g_timed[idx].b, stream);
+}
 
 // ------------------------------------------------------------------ workspace
 enum WsSlot {
@@ -256,6 +283,7 @@ int prepare_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, 
     WS(WS_CN, static_cast<size_t>(padded) * sizeof(float), cp->cn);
     WS(WS_SCAL, 4 * sizeof(float), cp->scal);
     WS(WS_BITS, 2 * sizeof(unsigned int), cp->bits);
+    const int tk = timing_begin(TK_PREP, stream);
     CUDA_TRY(cudaMemsetAsync(cp->bits, 0, 2 * sizeof(unsigned int), stream));
     const int64_t count = static_cast<int64_t>(nlist) * d;
     int blocks = static_cast<int>((count + 256 * 8 - 1) / (256 * 8));
@@ -268,6 +296,7 @@ int prepare_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, 
     convert_rows_kernel<float><<<static_cast<unsigned>((threads + 255) / 256), 256, 0, stream>>>(
         centroids, nlist, padded, d, pl.kp, cp->scal, 1, cp->c16, cp->cn);
     LAUNCH_CHECK();
+    timing_end(tk, stream);
     return make_tmap(&cp->tmap_c, cp->c16, nlist, pl.kp, pl.block_n);
 }
 
@@ -287,6 +316,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     if (k > 1) WS(WS_PARTCNT, static_cast<size_t>(n) * pl.partials * sizeof(int), part_cnt);
 
     const int u8 = ptype == IVF_U8;
+    int tk = timing_begin(TK_PREP, stream);
     if (!u8) {
         CUDA_TRY(cudaMemsetAsync(cp.bits, 0, sizeof(unsigned int), stream));
         const int64_t count = n * d;
@@ -306,6 +336,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         convert_rows_kernel<float><<<cblocks, 256, 0, stream>>>(static_cast<const float*>(points), n, n, d, pl.kp,
                                                                 cp.scal, 0, x16, xn);
     LAUNCH_CHECK();
+    timing_end(tk, stream);
 
     CUtensorMap tmap_x;
     rc = make_tmap(&tmap_x, x16, n, pl.kp, kBlockM);
@@ -335,8 +366,10 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
                                       static_cast<int>(kSmemLimit)));
         ctx.smem_attr_set = true;
     }
+    tk = timing_begin(k == 1 ? TK_FUSED_ARGMIN : TK_FUSED_TOPK, stream);
     fused_topk_kernel<<<pl.ctas, kFusedThreads, pl.smem, stream>>>(tmap_x, cp.tmap_c, fp);
     LAUNCH_CHECK();
+    timing_end(tk, stream);
 
     MergeParams mp;
     mp.n = n;
@@ -351,12 +384,14 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     mp.xn = xn;
     mp.out_ids = out_ids;
     mp.out_dists = out_dists;
+    tk = timing_begin(TK_MERGE, stream);
     if (k == 1) {
         merge_argmin_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(mp);
     } else {
         merge_select_kernel<<<static_cast<unsigned>(n), kMergeThreads, 0, stream>>>(mp);
     }
     LAUNCH_CHECK();
+    timing_end(tk, stream);
     return IVF_OK;
 }
 
@@ -367,6 +402,7 @@ int update_device(DeviceCtx& ctx, const void* points, int ptype, const int32_t* 
     WS(WS_UOFF, (static_cast<size_t>(nlist) + 1) * sizeof(int), off);
     WS(WS_UCUR, static_cast<size_t>(nlist) * sizeof(int), cur);
     WS(WS_UPERM, static_cast<size_t>(n) * sizeof(int), perm);
+    const int tk = timing_begin(TK_UPDATE, stream);
     CUDA_TRY(cudaMemsetAsync(cnt, 0, static_cast<size_t>(nlist) * sizeof(int), stream));
     const unsigned rb = static_cast<unsigned>((n + 255) / 256);
     update_hist_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, cnt, ctx.status);
@@ -383,6 +419,7 @@ int update_device(DeviceCtx& ctx, const void* points, int ptype, const int32_t* 
         update_reduce_kernel<float><<<lb, 256, 0, stream>>>(static_cast<const float*>(points), perm, off, nlist, d,
                                                             sums, reinterpret_cast<long long*>(counts));
     LAUNCH_CHECK();
+    timing_end(tk, stream);
     return IVF_OK;
 }
 
@@ -592,6 +629,47 @@ int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int
     if (cta < 0 || cta >= pl.ctas) return fail(IVF_ERR_INVALID_ARG, "cta %d outside [0, %d)", cta, pl.ctas);
     out[0] = span_begin(pl.total_units, pl.ctas, cta);
     out[1] = span_begin(pl.total_units, pl.ctas, cta + 1);
+    return IVF_OK;
+}
+
+int ivf_debug_timing(int enable) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    for (TimedLaunch& t : g_timed) {
+        cudaEventDestroy(t.a);
+        cudaEventDestroy(t.b);
+    }
+    g_timed.clear();
+    g_timing = enable != 0;
+    return IVF_OK;
+}
+
+int ivf_debug_timing_read(double ms[5], int64_t launches[5]) {
+    if (!ms || !launches) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    CUDA_TRY(cudaDeviceSynchronize());
+    std::lock_guard<std::mutex> lk(g_mu);
+    for (int i = 0; i < TK_NUM; ++i) {
+        ms[i] = 0.0;
+        launches[i] = 0;
+    }
+    for (TimedLaunch& t : g_timed) {
+        float e = 0.f;
+        if (cudaEventElapsedTime(&e, t.a, t.b) == cudaSuccess) {
+            ms[t.kind] += e;
+            launches[t.kind] += 1;
+        }
+        cudaEventDestroy(t.a);
+        cudaEventDestroy(t.b);
+    }
+    g_timed.clear();
+    return IVF_OK;
+}
+
+int ivf_debug_wait_probe(void* stream) {
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != IVF_OK) return rc;
+    wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->status, g_wait_limit_ns.load());
+    LAUNCH_CHECK();
     return IVF_OK;
 }
 

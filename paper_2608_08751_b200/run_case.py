@@ -1,0 +1,77 @@
+"""Runs one call of the library on seeded synthetic input of a chosen size and prints its timing.
+
+A small driver for profilers and quick measurements:
+    python -m paper_2608_08751_b200.run_case --op assign --n 262144 --nlist 65536 --d 128 --dtype u8 --reps 3
+    python -m paper_2608_08751_b200.run_case --op route --n 10000 --nlist 65536 --k 64
+    python -m paper_2608_08751_b200.run_case --op update --n 1048576 --nlist 65536
+Inputs follow the SIFT-shaped (uint8, all-positive mixture) or DEEP-shaped (float32, unit norm)
+recipes of ``synth``.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import synth
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--op", default="assign", choices=["assign", "route", "update"])
+    ap.add_argument("--n", type=int, default=262144)
+    ap.add_argument("--nlist", type=int, default=65536)
+    ap.add_argument("--d", type=int, default=128)
+    ap.add_argument("--k", type=int, default=64)
+    ap.add_argument("--dtype", default="u8", choices=["u8", "f32"])
+    ap.add_argument("--reps", type=int, default=3)
+    args = ap.parse_args()
+
+    if args.dtype == "u8":
+        x = synth.sift_like_rows(0, rows=args.n, d=args.d)
+        c = synth.sift_like_centroids(args.nlist, args.d)
+    else:
+        x = synth.deep_like_rows(0, rows=args.n, d=args.d)
+        c = synth.deep_like_centroids(args.nlist, args.d)
+    xt, ct = torch.from_numpy(x).cuda(), torch.from_numpy(c).cuda()
+    k = 1 if args.op != "route" else args.k
+    ids = torch.empty((args.n, k) if k > 1 else (args.n,), dtype=torch.int32, device="cuda")
+    dists = torch.empty_like(ids, dtype=torch.float32)
+    sums = torch.zeros((args.nlist, args.d), dtype=torch.float32, device="cuda")
+    counts = torch.zeros((args.nlist,), dtype=torch.int64, device="cuda")
+    if args.op == "update":
+        ids = torch.from_numpy(np.random.default_rng(0).integers(0, args.nlist, args.n).astype(np.int32)).cuda()
+
+    def call():
+        if args.op == "assign":
+            B.ivf_assign(xt, ct, ids, dists)
+        elif args.op == "route":
+            B.ivf_route(xt, ct, k, ids, dists)
+        else:
+            B.ivf_centroid_update(xt, ids, sums, counts)
+
+    call()
+    B.ivf_check()
+    B.ivf_debug_timing(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.reps):
+        call()
+    e1.record()
+    fam = B.ivf_debug_timing_read()
+    B.ivf_check()
+    flops = 2.0 * args.n * args.nlist * args.d
+    out = {"op": args.op, "n": args.n, "nlist": args.nlist, "d": args.d, "k": k, "dtype": args.dtype,
+           "ms_per_call": e0.elapsed_time(e1) / args.reps,
+           "kernel_ms": {name: ms / max(cnt, 1) for name, (ms, cnt) in fam.items() if cnt}}
+    fused = out["kernel_ms"].get("fused_argmin") or out["kernel_ms"].get("fused_topk")
+    if fused:
+        out["fused_tflops"] = flops / (fused / 1e3) / 1e12
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,291 @@
+"""Parity of the CUDA path (through the C-ABI) with the CPU oracle, element by element on the same
+seeded inputs.  Distances within 1e-3 * (|x|^2 + |c|^2); id lists equal except inside that band;
+integer-exact inputs bit for bit; counts bit-exact, sums within 1e-5 relative (exact for uint8)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle
+from paper_2608_08751_b200 import binding as B
+from paper_2608_08751_b200 import synth
+
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def _cuda(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _route(x, c, k):
+    if k == 1:
+        ids, d = B.ivf_assign(_cuda(x), _cuda(c))
+    else:
+        ids, d = B.ivf_route(_cuda(x), _cuda(c), k)
+    B.ivf_check()
+    return ids.cpu().numpy(), d.cpu().numpy()
+
+
+def _rand(n, nlist, d, dtype, seed):
+    rng = np.random.default_rng(seed)
+    if dtype == "u8":
+        x = rng.integers(0, 256, (n, d)).astype(np.uint8)
+        c = (rng.standard_normal((nlist, d)) * 40 + 100).astype(np.float32)
+    else:
+        x = rng.standard_normal((n, d)).astype(np.float32)
+        c = rng.standard_normal((nlist, d)).astype(np.float32)
+    return x, c
+
+
+# several row tiles and centroid tiles, ragged tails on both, every supported K-slice count
+SMALL = [
+    (1, 1, 16, 1, "f32"), (1, 300, 128, 7, "f32"), (129, 257, 128, 1, "f32"), (300, 1000, 128, 1, "f32"),
+    (300, 1000, 96, 1, "f32"), (1000, 5000, 128, 1, "u8"), (300, 1000, 128, 16, "f32"), (300, 3000, 96, 64, "f32"),
+    (500, 20000, 128, 64, "u8"), (200, 700, 256, 8, "f32"), (200, 700, 192, 1, "u8"), (64, 40000, 16, 128, "f32"),
+    (700, 513, 64, 512, "f32"), (130, 2000, 48, 2, "u8"), (40000, 3000, 128, 1, "u8"), (257, 9000, 96, 256, "f32"),
+    (5, 600, 32, 600 - 88, "f32"),
+]
+
+
+@pytest.mark.parametrize("n,nlist,d,k,dtype", SMALL)
+def test_small_cases_match_oracle(n, nlist, d, k, dtype):
+    x, c = _rand(n, nlist, d, dtype, seed=n + nlist + d + k)
+    ids, dists = _route(x, c, k)
+    parity.check_route(x, c, k, ids, dists)
+
+
+def test_k_equals_nlist_returns_sorted_permutation():
+    x, c = _rand(50, 300, 64, "f32", 3)
+    ids, dists = _route(x, c, 300)
+    parity.check_route(x, c, 300, ids, dists)
+    assert (np.sort(ids, 1) == np.arange(300)).all()
+
+
+def test_config0_tiny_routing_full():
+    cfg = synth.C0
+    q, c = synth.routing_inputs(cfg)
+    ids, dists = _route(q, c, cfg.nprobe)
+    st = parity.check_route(q, c, cfg.nprobe, ids, dists)
+    assert st["rows"] == cfg.nq
+
+
+@pytest.mark.parametrize("n,nlist,d,k", [(300, 1500, 128, 1), (300, 1500, 128, 32), (260, 3000, 64, 100),
+                                         (1000, 700, 16, 5), (200, 600, 256, 64)])
+def test_integer_inputs_are_bit_exact_including_ties(n, nlist, d, k):
+    # uint8 points and integer-valued centroids: every product and sum is exact in fp16 -> fp32 and in
+    # fp64 alike, so ids (ties to the lower id) and distances must equal the oracle's bit for bit
+    hi = 256 if d <= 128 else 128
+    q, c = synth.integer_case(n, nlist, d, seed=d + k, hi=hi)
+    if d == 16:
+        q = (q % 4).astype(np.uint8)  # few distinct values: ties are plentiful
+        c = np.floor(c / 64).astype(np.float32)
+    ids, dists = _route(q, c, k)
+    st = parity.check_route(q, c, k, ids, dists, exact=True)
+    assert st["rows_identical"] == 1.0
+
+
+def test_duplicate_centroids_resolve_to_lower_id():
+    _, c = _rand(1, 700, 128, "f32", 9)
+    c[500] = c[20]
+    c[699] = c[20]
+    ids, dists = _route(c[[20, 500, 699, 3]], c, 4)
+    assert ids[0, :3].tolist() == [20, 500, 699] and ids[1, :3].tolist() == [20, 500, 699]
+    assert ids[3, 0] == 3 and (dists[:, 0] <= 1e-3 * 2 * (c[20] ** 2).sum()).all()
+
+
+def test_scaling_of_tiny_and_huge_magnitudes():
+    x, c = _rand(200, 900, 96, "f32", 4)
+    for s in (1e-6, 3e4):
+        ids, dists = _route((x * s).astype(np.float32), (c * s).astype(np.float32), 10)
+        parity.check_route((x * s).astype(np.float32), (c * s).astype(np.float32), 10, ids, dists)
+
+
+def test_run_to_run_determinism():
+    x, c = _rand(700, 6000, 128, "u8", 5)
+    a = _route(x, c, 40)
+    for _ in range(2):
+        b = _route(x, c, 40)
+        assert (a[0] == b[0]).all() and (a[1] == b[1]).all()
+
+
+def test_no_distances_requested():
+    x, c = _rand(200, 500, 64, "f32", 6)
+    ids, none = B.ivf_route(_cuda(x), _cuda(c), 5, want_dists=False)
+    B.ivf_check()
+    assert none is None
+    ids2, _ = _route(x, c, 5)
+    assert (ids.cpu().numpy() == ids2).all()
+
+
+# ---------------------------------------------------------------- full-size configurations, sampled rows
+def _sampled_full(cfg, sample):
+    q, c = synth.routing_inputs(cfg)
+    ids, dists = _route(q, c, cfg.nprobe)
+    rows = np.random.default_rng(cfg.index).choice(cfg.nq, sample, replace=False)
+    st = parity.check_route(q, c, cfg.nprobe, ids[rows], dists[rows], rows=rows)
+    # properties that hold at any size, for all rows
+    assert ((ids >= 0) & (ids < cfg.nlist)).all() and (np.diff(dists, axis=1) >= 0).all()
+    s = np.sort(ids, 1)
+    assert (s[:, 1:] != s[:, :-1]).all()
+    return st
+
+
+def test_config1_sift_shaped_full_size_sampled():
+    _sampled_full(synth.C1, 96)
+
+
+def test_config2_deep_shaped_full_size_sampled():
+    _sampled_full(synth.C2, 32)
+
+
+def test_config4_stress_full_size_sampled():
+    _sampled_full(synth.C4, 8)
+
+
+def test_config3_chunk_assignment_full_width_sampled():
+    x = synth.sift_like_rows(0)
+    c = synth.sift_like_centroids(synth.C3_NLIST)
+    ids, dists = _route(x, c, 1)
+    rows = np.random.default_rng(3).choice(x.shape[0], 96, replace=False)
+    parity.check_route(x, c, 1, ids[rows], dists[rows], rows=rows)
+    # every returned distance re-checked against the definition (n*d work)
+    D = oracle.pair_dists(x, c, np.arange(x.shape[0]), ids)
+    tol = 1e-3 * (oracle.sqnorms(x) + oracle.sqnorms(c)[ids])
+    assert (np.abs(dists - D) <= tol).all()
+
+
+# ---------------------------------------------------------------- Lloyd update
+@pytest.mark.parametrize("dtype,n,nlist,d", [("u8", 5000, 300, 128), ("f32", 5000, 300, 96), ("u8", 70000, 65536, 128),
+                                             ("f32", 3000, 7, 256), ("u8", 1, 5, 16), ("f32", 9000, 4097, 32)])
+def test_update_matches_oracle_and_accumulates(dtype, n, nlist, d):
+    rng = np.random.default_rng(n + nlist)
+    x = rng.integers(0, 256, (n, d)).astype(np.uint8) if dtype == "u8" else rng.standard_normal((n, d)).astype(np.float32)
+    ids = rng.integers(0, nlist, n).astype(np.int32)
+    if nlist > 10:
+        ids[ids == 3] = 4  # an empty list
+    sums = torch.zeros((nlist, d), dtype=torch.float32, device="cuda")
+    counts = torch.zeros((nlist,), dtype=torch.int64, device="cuda")
+    xt, it = _cuda(x), _cuda(ids)
+    h = n // 2
+    B.ivf_centroid_update(xt[:h].contiguous(), it[:h].contiguous(), sums, counts) if h else None
+    B.ivf_centroid_update(xt[h:].contiguous(), it[h:].contiguous(), sums, counts)
+    B.ivf_check()
+    parity.check_update(x, ids, nlist, sums.cpu().numpy(), counts.cpu().numpy())
+    assert counts.sum().item() == n
+
+
+def test_update_flags_and_skips_bad_ids():
+    x = np.arange(4 * 16, dtype=np.float32).reshape(4, 16)
+    ids = np.array([1, 9, -1, 0], np.int32)
+    sums = torch.zeros((3, 16), dtype=torch.float32, device="cuda")
+    counts = torch.zeros((3,), dtype=torch.int64, device="cuda")
+    B.ivf_centroid_update(_cuda(x), _cuda(ids), sums, counts)
+    with pytest.raises(B.IvfError) as e:
+        B.ivf_check()
+    assert e.value.code == B.IVF_ERR_BAD_ID
+    assert counts.cpu().tolist() == [1, 1, 0]
+    assert (sums.cpu().numpy()[1] == x[0]).all() and (sums.cpu().numpy()[0] == x[3]).all()
+    B.ivf_check()  # the status word was cleared
+
+
+def test_finalize_matches_oracle_and_keeps_empty_lists():
+    rng = np.random.default_rng(1)
+    sums = rng.standard_normal((50, 32)).astype(np.float32) * 100
+    counts = rng.integers(0, 5, 50).astype(np.int64)
+    old = rng.standard_normal((50, 32)).astype(np.float32)
+    ct = _cuda(old.copy())
+    B.ivf_centroid_finalize(_cuda(sums), _cuda(counts), ct)
+    want = oracle.finalize(sums.astype(np.float64), counts, old)
+    got = ct.cpu().numpy()
+    assert (got[counts == 0] == old[counts == 0]).all()
+    np.testing.assert_allclose(got, want, rtol=2e-7)  # fp32 divide vs fp64 divide then rounding: <= 1 ulp
+
+
+# ---------------------------------------------------------------- host streaming
+def test_route_from_pinned_host_memory():
+    x, c = _rand(3000, 2000, 128, "u8", 12)
+    xt = torch.from_numpy(x).pin_memory()
+    ids, dists = B.ivf_route(xt, _cuda(c), 8)
+    B.ivf_check()
+    ids2, d2 = _route(x, c, 8)
+    assert (ids.cpu().numpy() == ids2).all() and (dists.cpu().numpy() == d2).all()
+
+
+@pytest.mark.parametrize("host", [True, False])
+def test_assign_update_streamed_in_chunks(host):
+    n, nlist, d = 10500, 400, 128
+    x = synth.sift_like_rows(7, rows=n)
+    c = synth.sift_like_centroids(nlist)
+    xt = torch.from_numpy(x).pin_memory() if host else _cuda(x)
+    sums = torch.zeros((nlist, d), dtype=torch.float32, device="cuda")
+    counts = torch.zeros((nlist,), dtype=torch.int64, device="cuda")
+    ids = torch.empty((n,), dtype=torch.int32, device="cuda")
+    dists = torch.empty((n,), dtype=torch.float32, device="cuda")
+    B.ivf_assign_update(xt, _cuda(c), sums, counts, ids, dists, chunk_rows=2048)  # 6 chunks, ragged tail
+    B.ivf_check()
+    parity.check_route(x, c, 1, ids.cpu().numpy(), dists.cpu().numpy())
+    parity.check_update(x, ids.cpu().numpy(), nlist, sums.cpu().numpy(), counts.cpu().numpy())
+    # without id output
+    sums2, counts2 = torch.zeros_like(sums), torch.zeros_like(counts)
+    B.ivf_assign_update(xt, _cuda(c), sums2, counts2, chunk_rows=4096)
+    B.ivf_check()
+    assert (counts2 == counts).all() and (sums2 == sums).all()
+
+
+def test_pageable_host_memory_is_rejected():
+    x, c = _rand(100, 200, 64, "f32", 1)
+    xt = torch.from_numpy(x)
+    with pytest.raises((ValueError, B.IvfError)):
+        B.ivf_route(xt, _cuda(c), 4)
+    buf = np.zeros((100, 64), np.float32)
+    ids = torch.empty((100, 4), dtype=torch.int32, device="cuda")
+    rc = B.lib().ivf_route(buf.ctypes.data, 100, 64, 0, _cuda(c).data_ptr(), 200, 4, ids.data_ptr(), None, None)
+    assert rc in (B.IVF_ERR_INVALID_ARG, B.IVF_ERR_CUDA)
+
+
+# ---------------------------------------------------------------- Lloyd iterations, step-wise against the oracle
+def test_lloyd_twin_stepwise():
+    n, nlist, d, iters = 20000, 512, 128, 3
+    x = synth.sift_like_rows(1, rows=n)
+    init = x[synth.init_sample(n, nlist)].astype(np.float32)
+    xt = _cuda(x)
+    ct = _cuda(init.copy())
+    inertia = []
+    for _ in range(iters):
+        c_now = ct.cpu().numpy().copy()
+        sums = torch.zeros((nlist, d), dtype=torch.float32, device="cuda")
+        counts = torch.zeros((nlist,), dtype=torch.int64, device="cuda")
+        ids = torch.empty((n,), dtype=torch.int32, device="cuda")
+        dists = torch.empty((n,), dtype=torch.float32, device="cuda")
+        B.ivf_assign_update(xt, ct, sums, counts, ids, dists, chunk_rows=8192)
+        B.ivf_centroid_finalize(sums, counts, ct)
+        B.ivf_check()
+        g_ids = ids.cpu().numpy()
+        # the oracle is fed the GPU's current centroids, so a tolerated near-tie cannot compound
+        parity.check_route(x, c_now, 1, g_ids, dists.cpu().numpy())
+        parity.check_update(x, g_ids, nlist, sums.cpu().numpy(), counts.cpu().numpy())
+        want = oracle.finalize(sums.cpu().numpy().astype(np.float64), counts.cpu().numpy(), c_now)
+        np.testing.assert_allclose(ct.cpu().numpy(), want, rtol=2e-7)
+        inertia.append(float(dists.double().sum().item()))
+    assert all(b <= a * (1 + 1e-6) for a, b in zip(inertia, inertia[1:]))
+    _, _, o_inertia = oracle.lloyd(x, init, iters)
+    np.testing.assert_allclose(inertia, o_inertia, rtol=1e-3)
+
+
+# ---------------------------------------------------------------- bounded waits
+def test_expired_wait_is_reported_and_context_survives():
+    # a wait on a barrier that nothing completes runs out after the (shortened) limit; the kernel
+    # returns normally, the host reads the status, and the same context keeps computing correctly
+    x, c = _rand(300, 1000, 128, "f32", 2)
+    B.ivf_debug_set_wait_limit_ns(2_000_000)  # 2 ms
+    try:
+        B.ivf_debug_wait_probe()
+        with pytest.raises(B.IvfError) as e:
+            B.ivf_check()
+        assert e.value.code == B.IVF_ERR_DEVICE_TIMEOUT and "99" in str(e.value)
+    finally:
+        B.ivf_debug_set_wait_limit_ns(0)
+    B.ivf_check()
+    ids, dists = _route(x, c, 1)
+    parity.check_route(x, c, 1, ids, dists)
