@@ -172,6 +172,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2608_08751_b200 import binding as B
+    from paper_2608_08751_b200 import sharding
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
@@ -207,9 +208,7 @@ def main():
         sums.zero_()
         counts.zero_()
         B.ivf_assign_update(chunk, cent_lloyd, sums, counts, a_ids, a_dists)
-        if distributed:
-            dist.all_reduce(sums)
-            dist.all_reduce(counts)
+        sharding.allreduce_lloyd(sums, counts)  # the one exchange of a Lloyd iteration (no-op at N = 1)
         if ev:
             ev[2].record()
         B.ivf_centroid_finalize(sums, counts, cent_lloyd)
