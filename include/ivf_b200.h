@@ -134,17 +134,31 @@ int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[
 int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int64_t out[2]);
 int ivf_debug_set_wait_limit_ns(int64_t ns);
 int ivf_debug_wait_probe(void* stream);
+/* Test hook: when on, the merge of a k > 1 call declares every row's candidate set insufficient, so
+ * that all rows take the exact brute-force recomputation that normally only catches rare rows. */
+int ivf_debug_force_fallback(int on);
+/* Test hook (host only): which threshold rule a call with this nprobe and nlist uses -- out[0] =
+ * -1 (k = 1: argmin), 0 running (k <= 16), 1 given (threshold pass over every out[1]-th centroid),
+ * 2 bounded (sample too small). */
+int ivf_debug_rule(int k, int nlist, int out[2]);
 
 /*
  * Measurement hooks.  ivf_debug_timing(1) makes every later call bracket its kernels with CUDA
- * events on the caller's stream, grouped into five families: 0 operand preparation (norms,
+ * events on the caller's stream, grouped into six families: 0 operand preparation (norms,
  * fp16 copies), 1 fused distance+argmin (k = 1), 2 fused distance+top-k (k > 1), 3 merge of
- * partial results, 4 centroid update.  ivf_debug_timing_read synchronises the device, writes the
+ * partial results (and the brute-force recomputation of failed rows), 4 centroid update,
+ * 5 threshold pass of k > 16 calls (fused kernel over the centroid sample + its merge).  ivf_debug_timing_read synchronises the device, writes the
  * summed milliseconds and launch-group counts of each family since the last read, and clears
  * them.  ivf_debug_timing(0) switches the events off (the default).
  */
+/*
+ * ivf_debug_stats synchronises the device, writes three counters accumulated by k > 1 calls since
+ * the last read to out[3] (may be NULL) -- in-kernel log selections, candidate-log entries left for
+ * the merge, rows recomputed by brute force -- clears them, and switches the counting on or off.
+ */
+int ivf_debug_stats(int enable, int64_t out[3]);
 int ivf_debug_timing(int enable);
-int ivf_debug_timing_read(double ms[5], int64_t launches[5]);
+int ivf_debug_timing_read(double ms[6], int64_t launches[6]);
 
 #ifdef __cplusplus
 }

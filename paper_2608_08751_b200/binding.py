@@ -23,7 +23,7 @@ EXPORTS = (
     "ivf_route", "ivf_assign", "ivf_centroid_update", "ivf_centroid_finalize", "ivf_assign_update",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
     "ivf_debug_plan", "ivf_debug_span", "ivf_debug_set_wait_limit_ns",
-    "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe",
+    "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_stats",
 )
 
 _lib = None
@@ -62,6 +62,9 @@ def lib() -> ctypes.CDLL:
     L.ivf_debug_set_wait_limit_ns.argtypes = [i64]
     L.ivf_debug_timing.argtypes = [i32]
     L.ivf_debug_wait_probe.argtypes = [vp]
+    L.ivf_debug_force_fallback.argtypes = [i32]
+    L.ivf_debug_stats.argtypes = [i32, ctypes.POINTER(i64)]
+    L.ivf_debug_rule.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_int)]
     L.ivf_debug_timing_read.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
     for name in EXPORTS:
         if name not in ("ivf_last_error", "ivf_launch_count"):
@@ -242,7 +245,7 @@ def ivf_debug_set_wait_limit_ns(ns: int) -> None:
     lib().ivf_debug_set_wait_limit_ns(ns)
 
 
-TIMING_FAMILIES = ("prep", "fused_argmin", "fused_topk", "merge", "update")
+TIMING_FAMILIES = ("prep", "fused_argmin", "fused_topk", "merge", "update", "threshold_pass")
 
 
 def ivf_debug_timing(enable: bool) -> None:
@@ -251,8 +254,8 @@ def ivf_debug_timing(enable: bool) -> None:
 
 def ivf_debug_timing_read() -> dict:
     """{family: (milliseconds, launch groups)} since the last read; synchronises the device."""
-    ms = (ctypes.c_double * 5)()
-    cnt = (ctypes.c_int64 * 5)()
+    ms = (ctypes.c_double * 6)()
+    cnt = (ctypes.c_int64 * 6)()
     rc = lib().ivf_debug_timing_read(ms, cnt)
     if rc != IVF_OK:
         _raise(rc)
@@ -265,3 +268,25 @@ def ivf_debug_wait_probe() -> None:
     rc = lib().ivf_debug_wait_probe(_stream(dev))
     if rc != IVF_OK:
         _raise(rc)
+
+
+def ivf_debug_force_fallback(on: bool) -> None:
+    lib().ivf_debug_force_fallback(1 if on else 0)
+
+
+def ivf_debug_rule(k: int, nlist: int):
+    """(rule, sample stride): -1 argmin, 0 running, 1 given (threshold pass), 2 bounded."""
+    out = (ctypes.c_int * 2)()
+    rc = lib().ivf_debug_rule(k, nlist, out)
+    if rc != IVF_OK:
+        _raise(rc)
+    return int(out[0]), int(out[1])
+
+
+def ivf_debug_stats(enable: bool) -> dict:
+    """Counters of the k > 1 path since the last read (see the header); then switches counting on/off."""
+    out = (ctypes.c_int64 * 3)()
+    rc = lib().ivf_debug_stats(1 if enable else 0, out)
+    if rc != IVF_OK:
+        _raise(rc)
+    return {"selections": int(out[0]), "log_entries": int(out[1]), "fallback_rows": int(out[2])}

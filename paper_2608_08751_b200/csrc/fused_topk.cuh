@@ -1,19 +1,32 @@
 // Fused distance + per-row top-k kernel (Sec. 4.1: dense centroid evaluation by Eq. 3 and
 // on-device list selection; Sec. 3.1 / 5.5: assignment is the k = 1 case).
 //
+// The whole ranking key of Eq. 3 comes out of the tensor core: the operand copies carry 16 extra
+// K columns, so that  acc = sum_t x'_t c''_t + A (w_hi + w_mid + w_lo) = sx sc (|c|^2 - 2 x.c)
+// with x' = sx x, c'' = -2 sc c, w = sc^2 |c|^2 / 2^15 split into three fp16 parts and
+// A = 2^15 sx / sc (sx, sc exact powers of two).  The epilogue only compares.
+//
 // One persistent CTA per SM walks a contiguous span of (row tile, centroid tile) units.
 //   warp 0      TMA producer: the stationary 128-row point tile and a ring of centroid tiles
-//   warp 1      single-thread tcgen05.mma issuer; S = X * C^T accumulates in TMEM (fp32), two
-//               accumulator buffers so the next tile's MMAs overlap this tile's epilogue
-//   warps 2..5  epilogue: each thread owns one point row (= one TMEM lane), reads its 256
-//               accumulator columns with tcgen05.ld, forms the ranking key
-//               v = |c|^2 - 2 x.c  and keeps the row's candidates.  Nothing of the n x nlist
-//               matrix is written to memory.
-// k = 1 keeps (best key, id) in registers.  k > 1 appends every key below the row's threshold tau
-// to the row's candidate log; when a log fills up, its warp selects the k smallest in place (radix
-// select on the key bits, ties to the lower id) and tightens tau to the k-th.  A row tile whose
-// centroid sweep is shared by several CTAs yields one partial result per CTA; a second kernel
-// merges them (merge.cuh).
+//   warp 1      single-thread tcgen05.mma issuer; accumulators live in TMEM (fp32), two buffers,
+//               so the next tile's MMAs overlap this tile's epilogue
+//   warps 2..9  epilogue: TMEM lane = point row; the two warps that share a lane quadrant split
+//               each tile's columns in 64-column groups.  Nothing of the n x nlist matrix is
+//               written to memory.
+// k = 1 keeps (best key, id) in registers.  k > 1 appends every key <= the row's threshold tau to
+// a candidate log in global memory.  tau comes from one of three rules, fixed per launch:
+//   running   (k <= 16) tau = the 16th smallest group-of-8 minimum seen so far, kept in a sorted
+//             register network: at least 16 keys are <= tau, so the result is exact;
+//   given     tau is read per row from memory.  The host computes it with a first, small launch of
+//             this same kernel (sketch rule) over every S-th centroid, S = k / 4: the 16th smallest
+//             group minimum of that sample lets about 4k candidates through.  Whether tau was loose
+//             enough is checked exactly by the merge kernel (at least k candidates <= tau); a row
+//             that fails is recomputed by brute force;
+//   sketch    the threshold pass itself: nothing is appended; each thread only keeps its 16
+//             smallest group minima and leaves them as its partial result;
+//   bounded   (small problems) tau = +inf until the log fills, then the warp selects the k
+//             smallest in place (radix select on the key bits, ties to the lower id) and tau
+//             becomes the k-th.  The same in-place selection catches any log that fills up.
 #pragma once
 #include "ptx.cuh"
 
@@ -22,37 +35,41 @@ namespace ivf {
 constexpr int kBlockM = 128;         // point rows per tile = TMEM lanes
 constexpr int kTmemCols = 512;       // whole TMEM: two accumulator buffers of 256 columns
 constexpr int kAccStride = 256;      // TMEM columns between the two accumulator buffers
-constexpr int kNumEpiWarps = 4;
+constexpr int kEpiHalves = 2;        // epilogue warps per TMEM lane quadrant
+constexpr int kNumEpiWarps = 4 * kEpiHalves;
 constexpr int kFusedThreads = 32 * (2 + kNumEpiWarps);
 constexpr int kSliceK = 64;          // fp16 elements per 128-byte swizzled row
 constexpr int kSliceRowBytes = 128;
+constexpr int kAugK = 16;            // extra K columns that carry |c|^2
+constexpr int kAugRowBytes = 32;
 constexpr int kMaxStages = 8;
+constexpr int kSampleM = 16;         // order statistic of the sample that becomes tau
 
 struct Entry {
-    float v;  // ranking key  |c|^2 - 2 x.c
+    float v;  // ranking key  sx sc (|c|^2 - 2 x.c)
     int j;    // centroid id
 };
 
-enum { MODE_ARGMIN = 0, MODE_APPEND = 1 };
+enum { TAU_RUNNING = 0, TAU_GIVEN = 1, TAU_BOUNDED = 2, TAU_SKETCH = 3 };
 
 struct FusedParams {
     int64_t n;            // point rows
     int nlist;
     int k;
-    int mode;
-    int ksteps;           // MMA instructions per tile = ceil(d / 16)
+    int ksteps;           // data MMA instructions per tile = ceil(d / 16); one more for the norm columns
     int kslices;          // 64-wide K slices of the operand copies
     int block_n;          // centroids per tile: 256 or 128
     int nstage;           // centroid-tile ring depth
     int col_tiles;        // centroid tiles per sweep
     int64_t total_units;  // row tiles * col_tiles
-    int partials;         // partial-result slots per row
+    int partials;         // partial-result slots per row (CTAs sharing a row tile x kEpiHalves)
     int cap;              // candidate-log capacity per (row, slot), k > 1 only
-    const float* cn;      // |c|^2, padded with +inf to col_tiles * block_n
-    const float* scal;    // device scalars: scal[2] = -2 / (point scale * centroid scale)
+    int rule;             // k > 1: TAU_RUNNING, TAU_GIVEN or TAU_BOUNDED
+    const float* tau_in;  // given rule: threshold per row, in key units
     Entry* part;          // k = 1: [n][partials]; k > 1: [n][partials][cap]
-    int* part_cnt;        // k > 1: [n][partials] entries in each log
+    int2* part_meta;      // k > 1: [n][partials] {entries in the log, bits of the final tau}
     int* status;          // sticky device status word
+    unsigned long long* stats;  // optional counters: [0] in-kernel selections, [1] log entries written
     uint64_t wait_limit_ns;
 };
 
@@ -63,11 +80,11 @@ __host__ __device__ inline int cta_of_unit(int64_t T, int G, int64_t u) {
 }
 
 __host__ __device__ inline size_t fused_smem_bytes(int kslices, int block_n, int nstage) {
-    return 1024                                                    // alignment slack
-           + static_cast<size_t>(kslices) * kBlockM * kSliceRowBytes  // point tile
-           + static_cast<size_t>(nstage) * kslices * block_n * kSliceRowBytes
-           + 256                                                   // barriers, TMEM slot, abort flag
-           + kNumEpiWarps * 256 * sizeof(int);                     // radix histograms
+    return 1024                                                                        // alignment slack
+           + static_cast<size_t>(kBlockM) * (kslices * kSliceRowBytes + kAugRowBytes)  // point tile
+           + static_cast<size_t>(nstage) * block_n * (kslices * kSliceRowBytes + kAugRowBytes)
+           + 256                                                                       // barriers etc.
+           + kNumEpiWarps * 256 * sizeof(int);                                         // radix histograms
 }
 
 __device__ __forceinline__ uint32_t orderable(float v) {
@@ -197,15 +214,143 @@ __global__ void wait_probe_kernel(int* status, uint64_t limit_ns) {
     (void)mbar_wait(&bar, 0, ctl, 99);
 }
 
-__device__ __forceinline__ float min3f(float a, float b, float c) { return fminf(fminf(a, b), c); }
+__device__ __forceinline__ float min3f(float a, float b, float c) {
+    float r;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
 
+// smallest of 32 keys (NaN entries are ignored by min)
+__device__ __forceinline__ float min32(const uint32_t (&a)[32]) {
+    float m[11];
+#pragma unroll
+    for (int i = 0; i < 10; ++i)
+        m[i] = min3f(__uint_as_float(a[3 * i]), __uint_as_float(a[3 * i + 1]), __uint_as_float(a[3 * i + 2]));
+    m[10] = fminf(__uint_as_float(a[30]), __uint_as_float(a[31]));
+    m[0] = min3f(m[0], m[1], m[2]);
+    m[1] = min3f(m[3], m[4], m[5]);
+    m[2] = min3f(m[6], m[7], m[8]);
+    m[3] = fminf(m[9], m[10]);
+    return fminf(min3f(m[0], m[1], m[2]), m[3]);
+}
+
+// sorted insertion of v into a[0] <= a[1] <= ... <= a[15] (the largest falls out); branch-free
+__device__ __forceinline__ void network_insert(float (&a)[kSampleM], float v) {
+#pragma unroll
+    for (int i = kSampleM - 1; i >= 1; --i) a[i] = fminf(a[i], fmaxf(a[i - 1], v));
+    a[0] = fminf(a[0], v);
+}
+
+// Compile-time variants of the epilogue.
+enum { EPI_ARGMIN = 0, EPI_RUNNING = 1, EPI_FILTER = 2, EPI_SKETCH = 3 };
+
+template <int EPI>
+struct RowState;
+template <>
+struct RowState<EPI_ARGMIN> {
+    float tau;  // best key so far
+    int bestj;
+};
+template <>
+struct RowState<EPI_FILTER> {
+    float tau;  // threshold (given per row, or +inf until the first in-place selection)
+    int cnt;    // entries in the log
+    Entry* log;
+};
+template <>
+struct RowState<EPI_RUNNING> {
+    float tau;
+    int cnt;
+    Entry* log;
+    float net[kSampleM];  // the 16 smallest group-of-8 minima seen
+};
+template <>
+struct RowState<EPI_SKETCH> {
+    float tau;
+    float net[kSampleM];
+};
+
+__device__ __forceinline__ void mask_ragged(uint32_t (&acc)[32], int jbase, int nlist) {
+#pragma unroll
+    for (int c = 0; c < 32; ++c)
+        if (jbase + c >= nlist) acc[c] = 0x7fc00000u;  // NaN: never below any threshold, ignored by min
+}
+
+__device__ __forceinline__ float min8(const uint32_t (&acc)[32], int g) {
+    float m = min3f(__uint_as_float(acc[8 * g]), __uint_as_float(acc[8 * g + 1]), __uint_as_float(acc[8 * g + 2]));
+    m = min3f(m, __uint_as_float(acc[8 * g + 3]), __uint_as_float(acc[8 * g + 4]));
+    m = min3f(m, __uint_as_float(acc[8 * g + 5]), __uint_as_float(acc[8 * g + 6]));
+    return fminf(m, __uint_as_float(acc[8 * g + 7]));
+}
+
+// 32 accumulator columns of one row.
+template <int EPI>
+__device__ __forceinline__ void consume(uint32_t (&acc)[32], int jbase, RowState<EPI>& st) {
+    if constexpr (EPI == EPI_ARGMIN) {
+        const float m = min32(acc);
+        if (m < st.tau) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+                const float key = __uint_as_float(acc[c]);
+                if (key < st.tau) {
+                    st.tau = key;
+                    st.bestj = jbase + c;
+                }
+            }
+        }
+    } else if constexpr (EPI == EPI_FILTER) {
+        // Straight-line predicated code on purpose: hits are rare, but 32 rows share every branch,
+        // so a branch per column costs more in divergence than the predicated store it would skip.
+        Entry* wp = st.log + st.cnt;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t"
+                "setp.le.f32 p, %1, %2;\n\t"
+                "@p st.global.v2.b32 [%0], {%3, %4};\n\t"
+                "@p add.s64 %0, %0, 8;\n\t}"
+                : "+l"(wp)
+                : "f"(__uint_as_float(acc[c])), "f"(st.tau), "r"(acc[c]), "r"(jbase + c)
+                : "memory");
+        }
+        st.cnt = static_cast<int>(wp - st.log);
+    } else {
+        // the sample statistic is the minimum of each group of 8 keys: one network insertion per
+        // group.  tau = the 16th smallest group minimum, so at least 16 keys are <= tau.
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const float m = min8(acc, g);
+            if (__any_sync(0xFFFFFFFFu, m <= st.tau)) {
+                if constexpr (EPI == EPI_RUNNING) {
+#pragma unroll
+                    for (int c = 8 * g; c < 8 * g + 8; ++c) {
+                        if (__uint_as_float(acc[c]) <= st.tau) {
+                            *reinterpret_cast<uint2*>(&st.log[st.cnt]) =
+                                make_uint2(acc[c], static_cast<uint32_t>(jbase + c));
+                            ++st.cnt;
+                        }
+                    }
+                }
+                if (m < st.net[kSampleM - 1]) {
+                    network_insert(st.net, m);
+                    st.tau = fminf(st.tau, st.net[kSampleM - 1]);
+                }
+            }
+        }
+    }
+}
+
+template <int EPI>
 __global__ void __launch_bounds__(kFusedThreads, 1)
-fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_c,
+fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_xa,
+                  const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_ca,
                   const FusedParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int a_bytes = p.kslices * kBlockM * kSliceRowBytes;
-    const int stage_bytes = p.kslices * p.block_n * kSliceRowBytes;
+    const int a_data_bytes = p.kslices * kBlockM * kSliceRowBytes;
+    const int a_bytes = a_data_bytes + kBlockM * kAugRowBytes;
+    const int b_data_bytes = p.kslices * p.block_n * kSliceRowBytes;
+    const int stage_bytes = b_data_bytes + p.block_n * kAugRowBytes;
     uint8_t* smem_a = smem;
     uint8_t* smem_b = smem + a_bytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_b + static_cast<size_t>(p.nstage) * stage_bytes);
@@ -244,7 +389,9 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         *abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tmap_x);
+        tma_prefetch_desc(&tmap_xa);
         tma_prefetch_desc(&tmap_c);
+        tma_prefetch_desc(&tmap_ca);
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, kTmemCols);
@@ -259,6 +406,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     ctl.abort_flag = abort_flag;
     ctl.status = p.status;
     ctl.limit_ns = p.wait_limit_ns;
+    const int kd = p.kslices * kSliceK;  // K column where the norm columns start
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -276,6 +424,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 for (int s = 0; s < p.kslices; ++s)
                     tma_load_2d(smem_a + s * kBlockM * kSliceRowBytes, &tmap_x, a_full, s * kSliceK,
                                 static_cast<int>(r * kBlockM));
+                tma_load_2d(smem_a + a_data_bytes, &tmap_xa, a_full, kd, static_cast<int>(r * kBlockM));
                 for (int t = t0; t < t1; ++t) {
                     const int st = it % p.nstage;
                     const uint32_t ph = (it / p.nstage) & 1;
@@ -286,6 +435,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                     for (int s = 0; s < p.kslices; ++s)
                         tma_load_2d(dst + s * p.block_n * kSliceRowBytes, &tmap_c, &b_full[st], s * kSliceK,
                                     t * p.block_n);
+                    tma_load_2d(dst + b_data_bytes, &tmap_ca, &b_full[st], kd, t * p.block_n);
                     ++it;
                 }
                 ++seg;
@@ -332,14 +482,16 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                     if (!ok) break;
                     tc_fence_after_sync();
                     const uint32_t d_tmem = tmem_base + buf * kAccStride;
+                    const uint32_t b_stage = b_addr + st * stage_bytes;
                     for (int kk = 0; kk < p.ksteps; ++kk) {
                         const int slice = kk >> 2;
                         const uint32_t off = (kk & 3) * 32;  // 16 fp16 = 32 bytes inside the swizzled row
                         const uint64_t adesc = umma_desc_sw128(a_addr + slice * kBlockM * kSliceRowBytes + off);
-                        const uint64_t bdesc =
-                            umma_desc_sw128(b_addr + st * stage_bytes + slice * p.block_n * kSliceRowBytes + off);
+                        const uint64_t bdesc = umma_desc_sw128(b_stage + slice * p.block_n * kSliceRowBytes + off);
                         umma_f16(d_tmem, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
                     }
+                    umma_f16(d_tmem, umma_desc_sw32(a_addr + a_data_bytes), umma_desc_sw32(b_stage + b_data_bytes),
+                             idesc, 1u);
                     umma_commit(&b_empty[st]);
                     umma_commit(&t_full[buf]);
                     ++it;
@@ -358,11 +510,13 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         }
     } else {
         // ------------------------------------------------------------ epilogue warps
-        const int quad = warp & 3;  // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
+        const int quad = warp & 3;               // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
+        const int half = (warp - 2) >> 2;        // which 64-column groups of a tile this warp takes
         const int row_in_tile = quad * 32 + lane;
-        int* hist = hist_all + (warp - 2) * 256;
-        const float mult = p.scal[2];
+        [[maybe_unused]] int* hist = hist_all + (warp - 2) * 256;
         const float INF = __int_as_float(0x7f800000);
+        const int nq = p.block_n / 64;  // 32-column chunks per warp and tile: 4 or 2
+        constexpr bool kHasLog = (EPI == EPI_RUNNING || EPI == EPI_FILTER);
         int it = 0;
         bool ok = true;
         for (int64_t u = u0; u < u1 && ok;) {
@@ -371,15 +525,21 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             const int t1 = static_cast<int>((u1 - r * NT < NT) ? (u1 - r * NT) : NT);
             const int64_t row = r * kBlockM + row_in_tile;
             const bool valid = row < p.n;
-            const int slot = b - cta_of_unit(T, G, r * NT);
-            const int64_t warp_row0 = r * kBlockM + quad * 32;
+            const int slot = (b - cta_of_unit(T, G, r * NT)) * kEpiHalves + half;
+            [[maybe_unused]] const int64_t warp_row0 = r * kBlockM + quad * 32;
 
-            float best = valid ? INF : -INF;  // k = 1: best key; k > 1: threshold tau
-            int bestj = 0x7fffffff;
-            int cnt = 0;
-            Entry* log = nullptr;
-            if (p.mode == MODE_APPEND && valid)
-                log = p.part + (static_cast<size_t>(row) * p.partials + slot) * p.cap;
+            RowState<EPI> st;
+            st.tau = valid ? INF : -INF;  // invalid rows: a threshold nothing passes
+            if constexpr (EPI == EPI_ARGMIN) st.bestj = 0x7fffffff;
+            if constexpr (EPI == EPI_RUNNING || EPI == EPI_SKETCH) {
+#pragma unroll
+                for (int i = 0; i < kSampleM; ++i) st.net[i] = INF;
+            }
+            if constexpr (kHasLog) {
+                st.cnt = 0;
+                st.log = p.part + (static_cast<size_t>(valid ? row : 0) * p.partials + slot) * p.cap;
+                if (EPI == EPI_FILTER && p.rule == TAU_GIVEN && valid) st.tau = p.tau_in[row];
+            }
 
             for (int t = t0; t < t1; ++t) {
                 const int buf = it & 1;
@@ -388,63 +548,46 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + buf * kAccStride;
-                const int nchunks = p.block_n / 32;
-#pragma unroll 1
-                for (int ch = 0; ch < nchunks; ++ch) {
-                    uint32_t acc[32];
-                    tmem_ld_32x32b_x32(taddr + ch * 32, acc);
-                    const int jbase = t * p.block_n + ch * 32;
-                    const float4* cn4 = reinterpret_cast<const float4*>(p.cn + jbase);
-                    float key[32];
-                    float4 cnv[8];
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) cnv[q] = __ldg(cn4 + q);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        key[4 * q + 0] = fmaf(__uint_as_float(acc[4 * q + 0]), mult, cnv[q].x);
-                        key[4 * q + 1] = fmaf(__uint_as_float(acc[4 * q + 1]), mult, cnv[q].y);
-                        key[4 * q + 2] = fmaf(__uint_as_float(acc[4 * q + 2]), mult, cnv[q].z);
-                        key[4 * q + 3] = fmaf(__uint_as_float(acc[4 * q + 3]), mult, cnv[q].w);
-                    }
-                    if (p.mode == MODE_ARGMIN) {
-                        float m = key[0];
-#pragma unroll
-                        for (int c = 1; c < 31; c += 2) m = min3f(m, key[c], key[c + 1]);
-                        m = fminf(m, key[31]);
-                        if (m < best) {
-#pragma unroll
-                            for (int c = 0; c < 32; ++c) {
-                                if (key[c] < best) {
-                                    best = key[c];
-                                    bestj = jbase + c;
-                                }
-                            }
-                        }
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            if (key[c] < best) {
-                                *reinterpret_cast<uint2*>(&log[cnt]) =
-                                    make_uint2(__float_as_uint(key[c]), static_cast<uint32_t>(jbase + c));
-                                ++cnt;
-                            }
-                        }
-                        if (__any_sync(0xFFFFFFFFu, cnt > p.cap - 32)) {
+                const bool ragged = (t + 1) * p.block_n > p.nlist;
+                const int tile_j0 = t * p.block_n;
+
+                // chunk q of this warp starts at column ((q/2) * halves + half) * 64 + (q%2) * 32
+                auto col_of = [&](int q) { return ((q >> 1) * kEpiHalves + half) * 64 + (q & 1) * 32; };
+                auto after_chunk = [&]() {
+                    if constexpr (kHasLog) {
+                        if (__any_sync(0xFFFFFFFFu, st.cnt > p.cap - 32)) {
                             __syncwarp();
                             for (int rr = 0; rr < 32; ++rr) {
-                                const int c_r = __shfl_sync(0xFFFFFFFFu, cnt, rr);
+                                const int c_r = __shfl_sync(0xFFFFFFFFu, st.cnt, rr);
                                 if (c_r > p.cap - 32) {
-                                    Entry* lr = p.part +
-                                                (static_cast<size_t>(warp_row0 + rr) * p.partials + slot) * p.cap;
-                                    const float tau = warp_select_k(lr, c_r, p.k, hist, lane);
+                                    Entry* lr =
+                                        p.part + (static_cast<size_t>(warp_row0 + rr) * p.partials + slot) * p.cap;
+                                    const float tk = warp_select_k(lr, c_r, p.k, hist, lane);
+                                    if (p.stats && lane == 0) atomicAdd(&p.stats[0], 1ull);
                                     if (lane == rr) {
-                                        cnt = p.k;
-                                        best = tau;
+                                        st.cnt = p.k;
+                                        st.tau = fminf(st.tau, tk);
                                     }
                                 }
                             }
                         }
+                    }
+                };
+                uint32_t accA[32], accB[32];
+                tmem_ld_32x32b_x32(taddr + col_of(0), accA);
+#pragma unroll
+                for (int q = 0; q < 4; q += 2) {
+                    if (q < nq) {
+                        tmem_wait_ld_regs(accA);
+                        tmem_ld_32x32b_x32(taddr + col_of(q + 1), accB);  // in flight while accA is consumed
+                        if (ragged) mask_ragged(accA, tile_j0 + col_of(q), p.nlist);
+                        consume<EPI>(accA, tile_j0 + col_of(q), st);
+                        after_chunk();
+                        tmem_wait_ld_regs(accB);
+                        if (q + 2 < nq) tmem_ld_32x32b_x32(taddr + col_of(q + 2), accA);
+                        if (ragged) mask_ragged(accB, tile_j0 + col_of(q + 1), p.nlist);
+                        consume<EPI>(accB, tile_j0 + col_of(q + 1), st);
+                        after_chunk();
                     }
                 }
                 tc_fence_before_sync();
@@ -453,13 +596,22 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 ++it;
             }
             if (ok && valid) {
-                if (p.mode == MODE_ARGMIN) {
+                const size_t at = static_cast<size_t>(row) * p.partials + slot;
+                if constexpr (EPI == EPI_ARGMIN) {
                     Entry e;
-                    e.v = best;
-                    e.j = bestj;
-                    p.part[static_cast<size_t>(row) * p.partials + slot] = e;
+                    e.v = st.tau;
+                    e.j = st.bestj;
+                    p.part[at] = e;
+                } else if constexpr (EPI == EPI_SKETCH) {
+                    // the partial result of the threshold pass: the thread's 16 smallest group minima
+                    Entry* log = p.part + at * p.cap;
+#pragma unroll
+                    for (int i = 0; i < kSampleM; ++i)
+                        *reinterpret_cast<uint2*>(&log[i]) = make_uint2(__float_as_uint(st.net[i]), 0u);
+                    p.part_meta[at] = make_int2(kSampleM, __float_as_int(INF));
                 } else {
-                    p.part_cnt[static_cast<size_t>(row) * p.partials + slot] = cnt;
+                    p.part_meta[at] = make_int2(st.cnt, __float_as_int(st.tau));
+                    if (p.stats) atomicAdd(&p.stats[1], static_cast<unsigned long long>(st.cnt));
                 }
             }
             u = r * NT + t1;

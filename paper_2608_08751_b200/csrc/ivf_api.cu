@@ -56,7 +56,7 @@ int fail(int code, const char* fmt, ...) {
 
 // ------------------------------------------------------------------ optional per-kernel timing
 // When enabled, launches of each kernel family are bracketed by CUDA events on the caller's stream.
-enum TimedKind { TK_PREP = 0, TK_FUSED_ARGMIN, TK_FUSED_TOPK, TK_MERGE, TK_UPDATE, TK_NUM };
+enum TimedKind { TK_PREP = 0, TK_FUSED_ARGMIN, TK_FUSED_TOPK, TK_MERGE, TK_UPDATE, TK_THRESH, TK_NUM };
 struct TimedLaunch {
     cudaEvent_t a, b;
     int kind;
@@ -82,7 +82,7 @@ void timing_end(int idx, cudaStream_t stream) {
 
 // ------------------------------------------------------------------ workspace
 enum WsSlot {
-    WS_X16, WS_C16, WS_XN, WS_CN, WS_SCAL, WS_BITS, WS_PART, WS_PARTCNT,
+    WS_X16, WS_C16, WS_XN, WS_SCAL, WS_BITS, WS_PART, WS_PARTMETA, WS_FAIL, WS_FBKEYS, WS_TAU,
     WS_UCNT, WS_UOFF, WS_UCUR, WS_UPERM, WS_IDS, WS_CHUNK0, WS_CHUNK1, WS_NUM
 };
 struct Buf {
@@ -93,6 +93,7 @@ struct DeviceCtx {
     bool init = false;
     int num_sms = 0;
     int* status = nullptr;
+    unsigned long long* stats = nullptr;  // 4 counters, only written while g_stats is on
     Buf bufs[WS_NUM];
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_copied[2] = {nullptr, nullptr};
@@ -118,6 +119,8 @@ int get_ctx(DeviceCtx** out) {
         c.num_sms = prop.multiProcessorCount;
         CUDA_TRY(cudaMalloc(&c.status, 4 * sizeof(int)));
         CUDA_TRY(cudaMemset(c.status, 0, 4 * sizeof(int)));
+        CUDA_TRY(cudaMalloc(&c.stats, 4 * sizeof(unsigned long long)));
+        CUDA_TRY(cudaMemset(c.stats, 0, 4 * sizeof(unsigned long long)));
         CUDA_TRY(cudaStreamCreateWithFlags(&c.copy_stream, cudaStreamNonBlocking));
         for (int i = 0; i < 2; ++i) {
             CUDA_TRY(cudaEventCreateWithFlags(&c.ev_copied[i], cudaEventDisableTiming));
@@ -161,21 +164,40 @@ int ws_get(DeviceCtx& c, WsSlot slot, size_t bytes, cudaStream_t stream, void** 
 
 // ------------------------------------------------------------------ schedule
 struct Plan {
-    int kp, kslices, ksteps, block_n, nstage;
+    int kd, kp, kslices, ksteps, block_n, nstage;
     int64_t row_tiles;
     int col_tiles;
     int64_t total_units;
     int ctas;
-    int partials;
+    int partials;    // slots per row: CTAs that can share a row tile x epilogue halves
     int cap;
     size_t smem;
 };
 
 constexpr size_t kSmemLimit = 227 * 1024;
+constexpr int kFallbackCtas = 32;  // slow-path CTAs of the brute-force recomputation
+
+int log_capacity(int k) { return (k == 1) ? 1 : (4 * k > 512 ? 4 * k : 512); }
+
+// Threshold rule of a k > 1 call, and the centroid stride of the sample that the threshold pass
+// looks at (every S-th centroid, S = k / 4: the 16th smallest key of a 4/k sample lets about 4k
+// candidates through; P(fewer than k) is about 1e-3 and those rows are recomputed exactly).
+constexpr int kMinSampleRows = 512;
+int choose_rule(int k, int nlist, int* stride) {
+    *stride = 1;
+    if (k <= kSampleM) return TAU_RUNNING;
+    const int S = k / 4;
+    if ((nlist + S - 1) / S >= kMinSampleRows) {
+        *stride = S;
+        return TAU_GIVEN;
+    }
+    return TAU_BOUNDED;
+}
 
 int make_plan(int64_t n, int nlist, int d, int k, int num_sms, Plan* pl) {
-    pl->kp = (d + 63) / 64 * 64;
-    pl->kslices = pl->kp / 64;
+    pl->kd = (d + 63) / 64 * 64;
+    pl->kp = pl->kd + kAugK;
+    pl->kslices = pl->kd / 64;
     pl->ksteps = (d + 15) / 16;
     pl->block_n = pl->kslices <= 2 ? 256 : 128;
     int nstage = kMaxStages;
@@ -190,17 +212,16 @@ int make_plan(int64_t n, int nlist, int d, int k, int num_sms, Plan* pl) {
     const int64_t lmin = pl->total_units / pl->ctas;
     int64_t parts = (pl->col_tiles + lmin - 1) / lmin + 1;
     if (parts > pl->ctas) parts = pl->ctas;
-    pl->partials = static_cast<int>(parts);
-    pl->cap = (k == 1) ? 1 : (4 * k > 128 ? 4 * k : 128);
+    pl->partials = static_cast<int>(parts) * kEpiHalves;
+    pl->cap = log_capacity(k);
     return IVF_OK;
 }
 
 // rows per launch so that the per-launch scratch stays bounded
 int64_t rows_per_launch(int d, int k) {
-    const int kp = (d + 63) / 64 * 64;
-    const int cap = (k == 1) ? 1 : (4 * k > 128 ? 4 * k : 128);
-    const int64_t per_row = static_cast<int64_t>(kp) * 2 + 3ll * cap * 8;  // fp16 copy + ~3 partial logs
-    int64_t rows = (int64_t(2) << 30) / per_row;
+    const int kp = (d + 63) / 64 * 64 + kAugK;
+    const int64_t per_row = static_cast<int64_t>(kp) * 2 + 6ll * log_capacity(k) * 8 + (k > kSampleM ? 6ll * 512 * 8 : 0);
+    int64_t rows = (int64_t(3) << 30) / per_row;
     rows = rows / kBlockM * kBlockM;
     if (rows < kBlockM) rows = kBlockM;
     if (rows > (int64_t(4) << 20)) rows = int64_t(4) << 20;
@@ -224,14 +245,17 @@ int get_encode() {
     return IVF_OK;
 }
 
-// fp16 matrix [rows][kp] row-major; box = 64 columns x box_rows rows; 128-byte swizzle.
-int make_tmap(CUtensorMap* map, const void* base, int64_t rows, int kp, int box_rows) {
+// fp16 matrix [rows][kp] row-major.  Data map: box = 64 columns x box_rows, 128-byte swizzle.
+// Norm-column map: box = 16 columns x box_rows, 32-byte swizzle (read at column kd).
+// row_step > 1 maps every row_step-th row (rows = number of rows of that strided view).
+int make_tmap(CUtensorMap* map, const void* base, int64_t rows, int kp, int box_rows, bool aug, int row_step = 1) {
     cuuint64_t dims[2] = {static_cast<cuuint64_t>(kp), static_cast<cuuint64_t>(rows)};
-    cuuint64_t strides[1] = {static_cast<cuuint64_t>(kp) * 2};
-    cuuint32_t box[2] = {static_cast<cuuint32_t>(kSliceK), static_cast<cuuint32_t>(box_rows)};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(kp) * 2 * row_step};
+    cuuint32_t box[2] = {static_cast<cuuint32_t>(aug ? kAugK : kSliceK), static_cast<cuuint32_t>(box_rows)};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          aug ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(IVF_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
     return IVF_OK;
@@ -270,17 +294,19 @@ int classify_pointer(const void* p) {
 // ------------------------------------------------------------------ device-resident building blocks
 struct CentroidPrep {
     __half* c16;
-    float* cn;
     float* scal;
     unsigned int* bits;
-    CUtensorMap tmap_c;
+    CUtensorMap tmap_c, tmap_ca;    // all centroids
+    CUtensorMap tmap_cs, tmap_csa;  // every `stride`-th centroid (threshold pass), if rule == TAU_GIVEN
+    int rule, stride, sample_rows;
 };
 
-int prepare_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, const Plan& pl, cudaStream_t stream,
-                      CentroidPrep* cp) {
-    const int64_t padded = static_cast<int64_t>(pl.col_tiles) * pl.block_n;
+int g_force_fallback = 0;
+bool g_stats = false;
+
+int prepare_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, int k, const Plan& pl,
+                      cudaStream_t stream, CentroidPrep* cp) {
     WS(WS_C16, static_cast<size_t>(nlist) * pl.kp * sizeof(__half), cp->c16);
-    WS(WS_CN, static_cast<size_t>(padded) * sizeof(float), cp->cn);
     WS(WS_SCAL, 4 * sizeof(float), cp->scal);
     WS(WS_BITS, 2 * sizeof(unsigned int), cp->bits);
     const int tk = timing_begin(TK_PREP, stream);
@@ -292,28 +318,132 @@ int prepare_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, 
     LAUNCH_CHECK();
     scales_kernel<<<1, 1, 0, stream>>>(cp->bits, 1, cp->scal);
     LAUNCH_CHECK();
-    const int64_t threads = padded * 32;
-    convert_rows_kernel<float><<<static_cast<unsigned>((threads + 255) / 256), 256, 0, stream>>>(
-        centroids, nlist, padded, d, pl.kp, cp->scal, 1, cp->c16, cp->cn);
+    const int64_t threads = static_cast<int64_t>(nlist) * 32;
+    convert_rows_kernel<float, true><<<static_cast<unsigned>((threads + 255) / 256), 256, 0, stream>>>(
+        centroids, nlist, d, pl.kd, cp->scal, cp->c16, nullptr);
     LAUNCH_CHECK();
     timing_end(tk, stream);
-    return make_tmap(&cp->tmap_c, cp->c16, nlist, pl.kp, pl.block_n);
+    int rc = make_tmap(&cp->tmap_c, cp->c16, nlist, pl.kp, pl.block_n, false);
+    if (rc != IVF_OK) return rc;
+    rc = make_tmap(&cp->tmap_ca, cp->c16, nlist, pl.kp, pl.block_n, true);
+    if (rc != IVF_OK) return rc;
+    cp->rule = (k == 1) ? TAU_RUNNING : choose_rule(k, nlist, &cp->stride);
+    cp->sample_rows = 0;
+    if (k > 1 && cp->rule == TAU_GIVEN) {
+        cp->sample_rows = (nlist + cp->stride - 1) / cp->stride;
+        rc = make_tmap(&cp->tmap_cs, cp->c16, cp->sample_rows, pl.kp, pl.block_n, false, cp->stride);
+        if (rc != IVF_OK) return rc;
+        rc = make_tmap(&cp->tmap_csa, cp->c16, cp->sample_rows, pl.kp, pl.block_n, true, cp->stride);
+        if (rc != IVF_OK) return rc;
+    }
+    return IVF_OK;
 }
 
-// Routes `n` device-resident rows against prepared centroids (one fused launch + one merge).
-int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int ptype, int nlist, int k,
-                      const CentroidPrep& cp, int32_t* out_ids, float* out_dists, cudaStream_t stream) {
-    Plan pl;
-    int rc = make_plan(n, nlist, d, k, ctx.num_sms, &pl);
-    if (rc != IVF_OK) return rc;
+struct PointPrep {
     __half* x16;
     float* xn;
+    CUtensorMap tmap_x, tmap_xa;
+};
+
+int launch_fused(DeviceCtx& ctx, const Plan& pl, int64_t n, int nlist, int k, int rule, const float* tau_in,
+                 const PointPrep& pp, const CUtensorMap& tmap_c, const CUtensorMap& tmap_ca, Entry* part,
+                 int2* part_meta, int kind, cudaStream_t stream) {
+    FusedParams fp;
+    fp.n = n;
+    fp.nlist = nlist;
+    fp.k = k;
+    fp.ksteps = pl.ksteps;
+    fp.kslices = pl.kslices;
+    fp.block_n = pl.block_n;
+    fp.nstage = pl.nstage;
+    fp.col_tiles = pl.col_tiles;
+    fp.total_units = pl.total_units;
+    fp.partials = pl.partials;
+    fp.cap = pl.cap;
+    fp.rule = rule;
+    fp.tau_in = tau_in;
+    fp.part = part;
+    fp.part_meta = part_meta;
+    fp.status = ctx.status;
+    fp.stats = g_stats ? ctx.stats : nullptr;
+    fp.wait_limit_ns = g_wait_limit_ns.load();
+    if (!ctx.smem_attr_set) {
+        const int lim = static_cast<int>(kSmemLimit);
+        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_ARGMIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim));
+        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_RUNNING>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim));
+        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_FILTER>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim));
+        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_SKETCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim));
+        ctx.smem_attr_set = true;
+    }
+    const int tk = timing_begin(kind, stream);
+    if (k == 1)
+        fused_topk_kernel<EPI_ARGMIN><<<pl.ctas, kFusedThreads, pl.smem, stream>>>(pp.tmap_x, pp.tmap_xa, tmap_c, tmap_ca, fp);
+    else if (rule == TAU_RUNNING)
+        fused_topk_kernel<EPI_RUNNING><<<pl.ctas, kFusedThreads, pl.smem, stream>>>(pp.tmap_x, pp.tmap_xa, tmap_c, tmap_ca, fp);
+    else if (rule == TAU_SKETCH)
+        fused_topk_kernel<EPI_SKETCH><<<pl.ctas, kFusedThreads, pl.smem, stream>>>(pp.tmap_x, pp.tmap_xa, tmap_c, tmap_ca, fp);
+    else
+        fused_topk_kernel<EPI_FILTER><<<pl.ctas, kFusedThreads, pl.smem, stream>>>(pp.tmap_x, pp.tmap_xa, tmap_c, tmap_ca, fp);
+    LAUNCH_CHECK();
+    timing_end(tk, stream);
+    return IVF_OK;
+}
+
+MergeParams merge_params(const Plan& pl, int64_t n, int k, const Entry* part, const int2* part_meta,
+                         const PointPrep& pp, const float* scal) {
+    MergeParams mp;
+    mp.n = n;
+    mp.k = k;
+    mp.partials = pl.partials;
+    mp.cap = pl.cap;
+    mp.col_tiles = pl.col_tiles;
+    mp.total_units = pl.total_units;
+    mp.ctas = pl.ctas;
+    mp.part = part;
+    mp.part_meta = part_meta;
+    mp.xn = pp.xn;
+    mp.scal = scal;
+    mp.out_ids = nullptr;
+    mp.out_dists = nullptr;
+    mp.fail = nullptr;
+    mp.force_fail = 0;
+    mp.tau_out = nullptr;
+    mp.stats = nullptr;
+    return mp;
+}
+
+// Routes `n` device-resident rows against prepared centroids.
+int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int ptype, int nlist, int k,
+                      const CentroidPrep& cp, int32_t* out_ids, float* out_dists, cudaStream_t stream) {
+    Plan pl, pls;
+    int rc = make_plan(n, nlist, d, k, ctx.num_sms, &pl);
+    if (rc != IVF_OK) return rc;
+    const bool given = k > 1 && cp.rule == TAU_GIVEN;
+    size_t part_bytes = static_cast<size_t>(n) * pl.partials * pl.cap * sizeof(Entry);
+    size_t meta_bytes = static_cast<size_t>(n) * pl.partials * sizeof(int2);
+    if (given) {
+        rc = make_plan(n, cp.sample_rows, d, kSampleM, ctx.num_sms, &pls);
+        if (rc != IVF_OK) return rc;
+        const size_t pb = static_cast<size_t>(n) * pls.partials * pls.cap * sizeof(Entry);
+        const size_t mb = static_cast<size_t>(n) * pls.partials * sizeof(int2);
+        part_bytes = pb > part_bytes ? pb : part_bytes;
+        meta_bytes = mb > meta_bytes ? mb : meta_bytes;
+    }
+    PointPrep pp;
     Entry* part;
-    int* part_cnt = nullptr;
-    WS(WS_X16, static_cast<size_t>(n) * pl.kp * sizeof(__half), x16);
-    WS(WS_XN, static_cast<size_t>(n) * sizeof(float), xn);
-    WS(WS_PART, static_cast<size_t>(n) * pl.partials * pl.cap * sizeof(Entry), part);
-    if (k > 1) WS(WS_PARTCNT, static_cast<size_t>(n) * pl.partials * sizeof(int), part_cnt);
+    int2* part_meta = nullptr;
+    int* failbuf = nullptr;
+    float* fbkeys = nullptr;
+    float* tau = nullptr;
+    WS(WS_X16, static_cast<size_t>(n) * pl.kp * sizeof(__half), pp.x16);
+    WS(WS_XN, static_cast<size_t>(n) * sizeof(float), pp.xn);
+    WS(WS_PART, part_bytes, part);
+    if (k > 1) {
+        WS(WS_PARTMETA, meta_bytes, part_meta);
+        WS(WS_FAIL, (static_cast<size_t>(n) + 1) * sizeof(int), failbuf);
+        if (given || g_force_fallback) WS(WS_FBKEYS, static_cast<size_t>(kFallbackFastRows + kFallbackCtas) * nlist * sizeof(float), fbkeys);
+        if (given) WS(WS_TAU, static_cast<size_t>(n) * sizeof(float), tau);
+    }
 
     const int u8 = ptype == IVF_U8;
     int tk = timing_begin(TK_PREP, stream);
@@ -330,67 +460,70 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     const int64_t threads = n * 32;
     const unsigned cblocks = static_cast<unsigned>((threads + 255) / 256);
     if (u8)
-        convert_rows_kernel<uint8_t><<<cblocks, 256, 0, stream>>>(static_cast<const uint8_t*>(points), n, n, d, pl.kp,
-                                                                  cp.scal, 0, x16, xn);
+        convert_rows_kernel<uint8_t, false><<<cblocks, 256, 0, stream>>>(static_cast<const uint8_t*>(points), n, d,
+                                                                         pl.kd, cp.scal, pp.x16, pp.xn);
     else
-        convert_rows_kernel<float><<<cblocks, 256, 0, stream>>>(static_cast<const float*>(points), n, n, d, pl.kp,
-                                                                cp.scal, 0, x16, xn);
+        convert_rows_kernel<float, false><<<cblocks, 256, 0, stream>>>(static_cast<const float*>(points), n, d, pl.kd,
+                                                                       cp.scal, pp.x16, pp.xn);
     LAUNCH_CHECK();
     timing_end(tk, stream);
 
-    CUtensorMap tmap_x;
-    rc = make_tmap(&tmap_x, x16, n, pl.kp, kBlockM);
+    rc = make_tmap(&pp.tmap_x, pp.x16, n, pl.kp, kBlockM, false);
+    if (rc != IVF_OK) return rc;
+    rc = make_tmap(&pp.tmap_xa, pp.x16, n, pl.kp, kBlockM, true);
     if (rc != IVF_OK) return rc;
 
-    FusedParams fp;
-    fp.n = n;
-    fp.nlist = nlist;
-    fp.k = k;
-    fp.mode = (k == 1) ? MODE_ARGMIN : MODE_APPEND;
-    fp.ksteps = pl.ksteps;
-    fp.kslices = pl.kslices;
-    fp.block_n = pl.block_n;
-    fp.nstage = pl.nstage;
-    fp.col_tiles = pl.col_tiles;
-    fp.total_units = pl.total_units;
-    fp.partials = pl.partials;
-    fp.cap = pl.cap;
-    fp.cn = cp.cn;
-    fp.scal = cp.scal;
-    fp.part = part;
-    fp.part_cnt = part_cnt;
-    fp.status = ctx.status;
-    fp.wait_limit_ns = g_wait_limit_ns.load();
-    if (!ctx.smem_attr_set) {
-        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      static_cast<int>(kSmemLimit)));
-        ctx.smem_attr_set = true;
+    if (given) {
+        // threshold pass over every S-th centroid: the 16th smallest group minimum becomes the row's tau
+        rc = launch_fused(ctx, pls, n, cp.sample_rows, kSampleM, TAU_SKETCH, nullptr, pp, cp.tmap_cs, cp.tmap_csa, part,
+                          part_meta, TK_THRESH, stream);
+        if (rc != IVF_OK) return rc;
+        MergeParams ms = merge_params(pls, n, kSampleM, part, part_meta, pp, cp.scal);
+        ms.tau_out = tau;
+        tk = timing_begin(TK_THRESH, stream);
+        merge_select_kernel<<<static_cast<unsigned>(n), kMergeThreads, 0, stream>>>(ms);
+        LAUNCH_CHECK();
+        timing_end(tk, stream);
     }
-    tk = timing_begin(k == 1 ? TK_FUSED_ARGMIN : TK_FUSED_TOPK, stream);
-    fused_topk_kernel<<<pl.ctas, kFusedThreads, pl.smem, stream>>>(tmap_x, cp.tmap_c, fp);
-    LAUNCH_CHECK();
-    timing_end(tk, stream);
+    rc = launch_fused(ctx, pl, n, nlist, k, cp.rule, tau, pp, cp.tmap_c, cp.tmap_ca, part, part_meta,
+                      k == 1 ? TK_FUSED_ARGMIN : TK_FUSED_TOPK, stream);
+    if (rc != IVF_OK) return rc;
 
-    MergeParams mp;
-    mp.n = n;
-    mp.k = k;
-    mp.partials = pl.partials;
-    mp.cap = pl.cap;
-    mp.col_tiles = pl.col_tiles;
-    mp.total_units = pl.total_units;
-    mp.ctas = pl.ctas;
-    mp.part = part;
-    mp.part_cnt = part_cnt;
-    mp.xn = xn;
+    MergeParams mp = merge_params(pl, n, k, part, part_meta, pp, cp.scal);
     mp.out_ids = out_ids;
     mp.out_dists = out_dists;
+    mp.fail = failbuf;
+    mp.force_fail = g_force_fallback;
+    mp.stats = g_stats ? ctx.stats : nullptr;
     tk = timing_begin(TK_MERGE, stream);
     if (k == 1) {
         merge_argmin_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(mp);
+        LAUNCH_CHECK();
     } else {
+        CUDA_TRY(cudaMemsetAsync(failbuf, 0, sizeof(int), stream));
         merge_select_kernel<<<static_cast<unsigned>(n), kMergeThreads, 0, stream>>>(mp);
+        LAUNCH_CHECK();
+        if (given || g_force_fallback) {
+            FallbackParams fb;
+            fb.nlist = nlist;
+            fb.k = k;
+            fb.kp = pl.kp;
+            fb.x16 = pp.x16;
+            fb.c16 = cp.c16;
+            fb.xn = pp.xn;
+            fb.scal = cp.scal;
+            fb.fail = failbuf;
+            fb.keys = fbkeys;
+            fb.out_ids = out_ids;
+            fb.out_dists = out_dists;
+            fallback_keys_kernel<<<dim3(kFallbackKeyChunks, kFallbackFastRows), kFallbackThreads, 0, stream>>>(fb);
+            LAUNCH_CHECK();
+            fallback_select_kernel<<<kFallbackFastRows, kFallbackThreads, 0, stream>>>(fb);
+            LAUNCH_CHECK();
+            fallback_rows_kernel<<<kFallbackCtas, kFallbackThreads, 0, stream>>>(fb);
+            LAUNCH_CHECK();
+        }
     }
-    LAUNCH_CHECK();
     timing_end(tk, stream);
     return IVF_OK;
 }
@@ -450,7 +583,7 @@ int run_chunks(const void* points, int64_t n, int d, int ptype, const float* cen
     rc = make_plan(rows, nlist, d, k, ctx.num_sms, &pl0);
     if (rc != IVF_OK) return rc;
     CentroidPrep cp;
-    rc = prepare_centroids(ctx, centroids, nlist, d, pl0, stream, &cp);
+    rc = prepare_centroids(ctx, centroids, nlist, d, k, pl0, stream, &cp);
     if (rc != IVF_OK) return rc;
 
     uint8_t* stage[2] = {nullptr, nullptr};
@@ -643,7 +776,7 @@ int ivf_debug_timing(int enable) {
     return IVF_OK;
 }
 
-int ivf_debug_timing_read(double ms[5], int64_t launches[5]) {
+int ivf_debug_timing_read(double ms[6], int64_t launches[6]) {
     if (!ms || !launches) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
     CUDA_TRY(cudaDeviceSynchronize());
     std::lock_guard<std::mutex> lk(g_mu);
@@ -661,6 +794,33 @@ int ivf_debug_timing_read(double ms[5], int64_t launches[5]) {
         cudaEventDestroy(t.b);
     }
     g_timed.clear();
+    return IVF_OK;
+}
+
+int ivf_debug_stats(int enable, int64_t out[3]) {
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != IVF_OK) return rc;
+    CUDA_TRY(cudaDeviceSynchronize());
+    if (out) {
+        unsigned long long h[4];
+        CUDA_TRY(cudaMemcpy(h, ctx->stats, sizeof h, cudaMemcpyDeviceToHost));
+        for (int i = 0; i < 3; ++i) out[i] = static_cast<int64_t>(h[i]);
+    }
+    CUDA_TRY(cudaMemset(ctx->stats, 0, 4 * sizeof(unsigned long long)));
+    g_stats = enable != 0;
+    return IVF_OK;
+}
+
+int ivf_debug_rule(int k, int nlist, int out[2]) {
+    if (k < 1 || nlist < 1 || !out) return fail(IVF_ERR_INVALID_ARG, "bad arguments");
+    out[1] = 1;
+    out[0] = (k == 1) ? -1 : choose_rule(k, nlist, &out[1]);
+    return IVF_OK;
+}
+
+int ivf_debug_force_fallback(int on) {
+    g_force_fallback = on != 0;
     return IVF_OK;
 }
 

@@ -1,8 +1,15 @@
 // Second stage of the on-device list selection (Sec. 4.1: tile-local candidates are merged on the
-// device): the partial results that the CTAs sharing a row tile left behind are merged into the
-// final k ids per row, ascending by (distance, id), and the point norm is added back
-// (Eq. 3: |x-c|^2 = |x|^2 + (|c|^2 - 2 x.c)).
+// device): the partial results left by the CTAs (and epilogue warps) that shared a row are merged
+// into the final k ids per row, ascending by (distance, id); the key is rescaled and the point norm
+// added back (Eq. 3: |x-c|^2 = |x|^2 + (|c|^2 - 2 x.c)).
+//
+// For k > 16 the candidate logs were filled against per-partial thresholds tau_p.  Every element
+// with key < tau_p is in log p, and enough of the elements equal to tau_p, so the union of the logs
+// holds the true top-k whenever at least k candidates are <= min_p tau_p.  That test is exact; a
+// row that fails it is recomputed by fallback_rows_kernel (brute force over all centroids).
 #pragma once
+#include <cuda_fp16.h>
+
 #include "fused_topk.cuh"
 
 namespace ivf {
@@ -16,23 +23,28 @@ struct MergeParams {
     int64_t total_units;
     int ctas;              // grid size of the fused kernel (defines which slots exist)
     const Entry* part;
-    const int* part_cnt;
+    const int2* part_meta;
     const float* xn;       // |x|^2 per row
+    const float* scal;     // scal[2] = 1 / (sx sc)
     int32_t* out_ids;      // [n, k]
     float* out_dists;      // [n, k] or nullptr
+    int* fail;             // fail[0] = number of failed rows, fail[1..] = their indices
+    int force_fail;        // test hook: treat every row as failed
+    float* tau_out;        // if set: write only the 16th smallest key of every row here (threshold pass)
+    unsigned long long* stats;  // optional counters: [2] rows sent to the brute-force recomputation
 };
 
-__device__ __forceinline__ int slots_of_row_tile(const MergeParams& p, int64_t r) {
-    const int first = cta_of_unit(p.total_units, p.ctas, r * p.col_tiles);
-    const int last = cta_of_unit(p.total_units, p.ctas, (r + 1) * p.col_tiles - 1);
-    return last - first + 1;
+__device__ __forceinline__ int slots_of_row_tile(int64_t total_units, int ctas, int col_tiles, int64_t r) {
+    const int first = cta_of_unit(total_units, ctas, r * col_tiles);
+    const int last = cta_of_unit(total_units, ctas, (r + 1) * col_tiles - 1);
+    return (last - first + 1) * kEpiHalves;
 }
 
 // k = 1: one thread per row takes the lexicographic minimum over the row's partial results.
 __global__ void merge_argmin_kernel(const MergeParams p) {
     const int64_t row = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (row >= p.n) return;
-    const int ns = slots_of_row_tile(p, row / kBlockM);
+    const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / kBlockM);
     const Entry* e = p.part + static_cast<size_t>(row) * p.partials;
     float bv = e[0].v;
     int bj = e[0].j;
@@ -45,7 +57,7 @@ __global__ void merge_argmin_kernel(const MergeParams p) {
         }
     }
     p.out_ids[row] = bj;
-    if (p.out_dists) p.out_dists[row] = fmaxf(bv + p.xn[row], 0.0f);
+    if (p.out_dists) p.out_dists[row] = fmaxf(fmaf(bv, p.scal[2], p.xn[row]), 0.0f);
 }
 
 constexpr int kSortCap = 4096;
@@ -70,56 +82,240 @@ __device__ __forceinline__ void bitonic_sort_smem(uint64_t* keys, int m /* power
     __syncthreads();
 }
 
-// k > 1: one CTA per row sorts the row's candidates by the 64-bit key (orderable value, id) in
-// shared memory and writes the first k.  More than kSortCap candidates are folded in rounds.
+// k > 1: one CTA per row.  Candidates <= the row's smallest tau are sorted by the 64-bit key
+// (orderable value, id) in shared memory; more than kSortCap of them are folded in rounds.
 __global__ void __launch_bounds__(kMergeThreads) merge_select_kernel(const MergeParams p) {
     __shared__ uint64_t keys[kSortCap];
     __shared__ int s_fill;
     const int64_t row = blockIdx.x;
-    const int ns = slots_of_row_tile(p, row / kBlockM);
+    const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / kBlockM);
     const Entry* base = p.part + static_cast<size_t>(row) * p.partials * p.cap;
-    const int* cnts = p.part_cnt + static_cast<size_t>(row) * p.partials;
+    const int2* meta = p.part_meta + static_cast<size_t>(row) * p.partials;
 
-    int kept = 0;  // sorted keys carried at the front of keys[]
+    float tau_min = __int_as_float(0x7f800000);
+    for (int s = 0; s < ns; ++s) tau_min = fminf(tau_min, __int_as_float(meta[s].y));
+
+    int kept = 0;   // sorted keys carried at the front of keys[]
+    int total = 0;  // candidates <= tau_min seen so far
     int slot = 0, pos = 0;
-    bool more = ns > 0;
-    while (more) {
-        // fill keys[kept ..) from the remaining candidates, slot by slot
-        int fill = kept;
-        while (slot < ns && fill < kSortCap) {
-            const int c = min(cnts[slot], p.cap);
-            const int take = min(c - pos, kSortCap - fill);
+    if (threadIdx.x == 0) s_fill = 0;
+    __syncthreads();
+    while (true) {
+        // append the remaining candidates that pass the threshold, slot by slot, until keys[] is full
+        while (slot < ns) {
+            const int room = kSortCap - s_fill;
+            __syncthreads();  // everyone has read s_fill before anyone appends
+            if (room == 0) break;
+            const int c = min(meta[slot].x, p.cap);
+            const int take = min(c - pos, room);
             for (int i = threadIdx.x; i < take; i += blockDim.x) {
                 const Entry e = base[static_cast<size_t>(slot) * p.cap + pos + i];
-                keys[fill + i] = (static_cast<uint64_t>(orderable(e.v)) << 32) | static_cast<uint32_t>(e.j);
+                if (e.v <= tau_min)
+                    keys[atomicAdd(&s_fill, 1)] =
+                        (static_cast<uint64_t>(orderable(e.v)) << 32) | static_cast<uint32_t>(e.j);
             }
-            fill += take;
+            __syncthreads();
             pos += take;
             if (pos >= c) {
                 ++slot;
                 pos = 0;
             }
         }
-        more = slot < ns;
+        const int fill = s_fill;
+        total += fill - kept;
         int m = 2;
         while (m < fill) m <<= 1;
         for (int i = fill + threadIdx.x; i < m; i += blockDim.x) keys[i] = ~0ull;
         bitonic_sort_smem(keys, m);
         kept = min(fill, p.k);
-        if (kept == kSortCap) more = false;  // cannot happen for k <= 512; guards the loop
+        if (slot >= ns) break;
+        if (threadIdx.x == 0) s_fill = kept;
+        __syncthreads();
     }
-    (void)s_fill;
-    const float xn = p.xn[row];
-    for (int i = threadIdx.x; i < p.k; i += blockDim.x) {
-        int32_t id = -1;
-        float dist = __int_as_float(0x7f800000);
-        if (i < kept) {
-            const uint64_t key = keys[i];
-            id = static_cast<int32_t>(key & 0xFFFFFFFFull);
-            dist = fmaxf(from_orderable(static_cast<uint32_t>(key >> 32)) + xn, 0.0f);
+    if (p.tau_out) {
+        if (threadIdx.x == 0)
+            p.tau_out[row] = kept >= kSampleM ? from_orderable(static_cast<uint32_t>(keys[kSampleM - 1] >> 32))
+                                              : __int_as_float(0x7f800000);
+        return;
+    }
+    if (total < p.k || p.force_fail) {
+        if (threadIdx.x == 0) {
+            const int at = atomicAdd(&p.fail[0], 1);
+            p.fail[1 + at] = static_cast<int>(row);
+            if (p.stats) atomicAdd(&p.stats[2], 1ull);
         }
-        p.out_ids[row * p.k + i] = id;
-        if (p.out_dists) p.out_dists[row * p.k + i] = dist;
+        return;
+    }
+    const float xn = p.xn[row];
+    const float inv = p.scal[2];
+    for (int i = threadIdx.x; i < p.k; i += blockDim.x) {
+        const uint64_t key = keys[i];
+        p.out_ids[row * p.k + i] = static_cast<int32_t>(key & 0xFFFFFFFFull);
+        if (p.out_dists)
+            p.out_dists[row * p.k + i] = fmaxf(fmaf(from_orderable(static_cast<uint32_t>(key >> 32)), inv, xn), 0.0f);
+    }
+}
+
+// ------------------------------------------------------------------ brute-force recomputation
+struct FallbackParams {
+    int nlist;
+    int k;
+    int kp;                // pitch of the fp16 operand copies
+    const __half* x16;     // [n][kp]
+    const __half* c16;     // [nlist][kp]
+    const float* xn;
+    const float* scal;
+    const int* fail;       // fail[0] = count, fail[1..] = rows
+    float* keys;           // [kFallbackFastRows + slow-path CTAs][nlist] scratch
+    int32_t* out_ids;
+    float* out_dists;
+};
+
+constexpr int kFallbackThreads = 256;
+constexpr int kFallbackMaxK = 512;
+constexpr int kFallbackFastRows = 16;   // failed rows whose keys are computed by the whole grid
+constexpr int kFallbackKeyChunks = 128; // CTAs per row in that case
+
+// key of point row `xs` (fp32 copy of its fp16 operand row, in shared memory) against centroid j:
+// the same contraction as the MMA, in fp32 FMA.  One warp per centroid.
+__device__ __forceinline__ float fallback_key(const float* xs, const __half* cj, int kp, int lane) {
+    float acc = 0.0f;
+    for (int t = lane * 8; t < kp; t += 256) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(cj + t);
+        const __half2* h = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float2 f = __half22float2(h[q]);
+            acc = fmaf(xs[t + 2 * q], f.x, acc);
+            acc = fmaf(xs[t + 2 * q + 1], f.y, acc);
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+    return acc;
+}
+
+struct FallbackSmem {
+    float xs[288];
+    int hist[256];
+    int scan[kFallbackThreads];
+    uint64_t cand[kFallbackMaxK];
+    int cnt, digit, rank;
+};
+
+// Exact top-k of keys[0..nlist) by (key, id): 8-bit radix select for the k-th smallest key, ties to
+// the lower id, then a sort of the k winners; writes the row's outputs.  One CTA.
+__device__ void fallback_select_row(const FallbackParams& p, const float* keys, int64_t row, FallbackSmem& sm) {
+    uint32_t prefix = 0, mask = 0;
+    int rank = p.k;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) sm.hist[i] = 0;
+        __syncthreads();
+        for (int j = threadIdx.x; j < p.nlist; j += blockDim.x) {
+            const uint32_t u = orderable(keys[j]);
+            if ((u & mask) == prefix) atomicAdd(&sm.hist[(u >> shift) & 255u], 1);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int acc = 0, dgt = 255, r = rank;
+            for (int b = 0; b < 256; ++b) {
+                if (rank <= acc + sm.hist[b]) {
+                    dgt = b;
+                    r = rank - acc;
+                    break;
+                }
+                acc += sm.hist[b];
+            }
+            sm.digit = dgt;
+            sm.rank = r;
+        }
+        __syncthreads();
+        prefix |= static_cast<uint32_t>(sm.digit) << shift;
+        mask |= 255u << shift;
+        rank = sm.rank;
+        __syncthreads();
+    }
+    const uint32_t Tk = prefix;  // `rank` of the keys equal to Tk are wanted, lowest ids first
+    if (threadIdx.x == 0) sm.cnt = 0;
+    const int per = (p.nlist + blockDim.x - 1) / blockDim.x;
+    const int j0 = min(p.nlist, static_cast<int>(threadIdx.x) * per), j1 = min(p.nlist, j0 + per);
+    int eq = 0;
+    for (int j = j0; j < j1; ++j) eq += orderable(keys[j]) == Tk;
+    sm.scan[threadIdx.x] = eq;
+    __syncthreads();
+    int before = 0;
+    for (int t = 0; t < static_cast<int>(threadIdx.x); ++t) before += sm.scan[t];
+    for (int j = j0; j < j1; ++j) {
+        const uint32_t u = orderable(keys[j]);
+        bool take = u < Tk;
+        if (u == Tk) {
+            take = before < rank;
+            ++before;
+        }
+        if (take) sm.cand[atomicAdd(&sm.cnt, 1)] = (static_cast<uint64_t>(u) << 32) | static_cast<uint32_t>(j);
+    }
+    __syncthreads();
+    const int got = sm.cnt;  // == k
+    int m = 2;
+    while (m < got) m <<= 1;
+    for (int i = got + threadIdx.x; i < m; i += blockDim.x) sm.cand[i] = ~0ull;
+    bitonic_sort_smem(sm.cand, m);
+    const float xn = p.xn[row];
+    const float inv = p.scal[2];
+    for (int i = threadIdx.x; i < p.k; i += blockDim.x) {
+        const uint64_t key = sm.cand[i];
+        p.out_ids[row * p.k + i] = static_cast<int32_t>(key & 0xFFFFFFFFull);
+        if (p.out_dists)
+            p.out_dists[row * p.k + i] = fmaxf(fmaf(from_orderable(static_cast<uint32_t>(key >> 32)), inv, xn), 0.0f);
+    }
+    __syncthreads();
+}
+
+// The first kFallbackFastRows failed rows: grid (kFallbackKeyChunks, kFallbackFastRows); every CTA
+// computes one slice of one row's keys, so a single failed row still uses the whole GPU.
+__global__ void __launch_bounds__(kFallbackThreads) fallback_keys_kernel(const FallbackParams p) {
+    __shared__ float xs[288];
+    const int nfail = p.fail[0];
+    const int idx = blockIdx.y;
+    if (idx >= nfail) return;
+    const int64_t row = p.fail[1 + idx];
+    for (int t = threadIdx.x; t < p.kp; t += blockDim.x) xs[t] = __half2float(p.x16[row * p.kp + t]);
+    __syncthreads();
+    float* keys = p.keys + static_cast<size_t>(idx) * p.nlist;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int per = (p.nlist + gridDim.x - 1) / gridDim.x;
+    const int j0 = blockIdx.x * per, j1 = min(p.nlist, j0 + per);
+    for (int j = j0 + warp; j < j1; j += kFallbackThreads / 32) {
+        const float key = fallback_key(xs, p.c16 + static_cast<size_t>(j) * p.kp, p.kp, lane);
+        if (lane == 0) keys[j] = key;
+    }
+}
+
+__global__ void __launch_bounds__(kFallbackThreads) fallback_select_kernel(const FallbackParams p) {
+    __shared__ FallbackSmem sm;
+    const int nfail = p.fail[0];
+    const int idx = blockIdx.x;
+    if (idx >= nfail || idx >= kFallbackFastRows) return;
+    fallback_select_row(p, p.keys + static_cast<size_t>(idx) * p.nlist, p.fail[1 + idx], sm);
+}
+
+// Any further failed rows (none in practice): one CTA per row does both steps; slow and exact.
+__global__ void __launch_bounds__(kFallbackThreads) fallback_rows_kernel(const FallbackParams p) {
+    __shared__ FallbackSmem sm;
+    const int nfail = p.fail[0];
+    float* keys = p.keys + static_cast<size_t>(kFallbackFastRows + blockIdx.x) * p.nlist;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int idx = kFallbackFastRows + blockIdx.x; idx < nfail; idx += gridDim.x) {
+        const int64_t row = p.fail[1 + idx];
+        __syncthreads();
+        for (int t = threadIdx.x; t < p.kp; t += blockDim.x) sm.xs[t] = __half2float(p.x16[row * p.kp + t]);
+        __syncthreads();
+        for (int j = warp; j < p.nlist; j += kFallbackThreads / 32) {
+            const float key = fallback_key(sm.xs, p.c16 + static_cast<size_t>(j) * p.kp, p.kp, lane);
+            if (lane == 0) keys[j] = key;
+        }
+        __syncthreads();
+        fallback_select_row(p, keys, row, sm);
     }
 }
 

@@ -1,7 +1,12 @@
 // Operand preparation for the distance contraction (Sec. 4.1, Eq. 3: "inner products and
-// precomputed norms").  Norms are accumulated in fp32 from the unrounded inputs; the tensor-core
-// operands are fp16 copies scaled by an exact power of two chosen from the largest magnitude, so
-// nothing overflows and small-magnitude data keeps its 11 significant bits.  uint8 values are exact.
+// precomputed norms").  Norms are accumulated in fp32 from the unrounded inputs.  The tensor-core
+// operands are fp16 copies scaled by exact powers of two chosen from the largest magnitudes, so
+// nothing overflows and small-magnitude data keeps its 11 significant bits; uint8 values are exact.
+//
+// Row layouts (fp16, pitch kp = kd + 16, kd = d rounded up to 64):
+//   point     [ sx * x (d) | zeros to kd | A  A  A  0 ... 0 ]
+//   centroid  [ -2 sc * c (d) | zeros to kd | w_hi w_mid w_lo 0 ... 0 ],  w = sc^2 |c|^2 / 2^15
+// so that one K sweep of the MMA yields  sx sc (|c|^2 - 2 x.c)  with A = 2^15 sx / sc.
 #pragma once
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -29,44 +34,46 @@ __global__ void maxabs_kernel(const float* __restrict__ x, int64_t count, unsign
 }
 
 __device__ __forceinline__ float pow2_scale_for(float maxabs) {
-    // largest power of two s with s * maxabs < 2^14 (fp16 overflows at 65504); exponent clamped so
-    // that the product of two scales stays finite in fp32
+    // largest power of two s with s * maxabs < 2^11: the scaled squared norm of a row then stays
+    // below d * 2^22, and its 2^-15 multiple fits fp16.  Exponent clamped to keep products finite.
     if (!(maxabs > 0.0f) || isinf(maxabs)) return 1.0f;
     int e;
     frexpf(maxabs, &e);  // maxabs = f * 2^e, f in [0.5, 1)
-    int s = 14 - e;
-    s = s < -60 ? -60 : (s > 60 ? 60 : s);
+    int s = 11 - e;
+    s = s < -40 ? -40 : (s > 40 ? 40 : s);
     return ldexpf(1.0f, s);
 }
 
-// scal[0] = point scale, scal[1] = centroid scale, scal[2] = -2 / (scal[0] * scal[1]).
-// bits[0] = max |x| bits (ignored for uint8 points), bits[1] = max |c| bits.
+// scal[0] = sx (point scale), scal[1] = sc (centroid scale), scal[2] = 1 / (sx sc),
+// scal[3] = A = 2^15 sx / sc.  bits[0] = max |x| bits (unused for uint8 points), bits[1] = max |c|.
+// The point scale never exceeds the centroid scale (so A <= 2^15) and is at least sc * 2^-29
+// (so A stays a normal fp16 number).
 __global__ void scales_kernel(const unsigned int* bits, int points_are_u8, float* scal) {
-    const float sx = points_are_u8 ? 1.0f : pow2_scale_for(__uint_as_float(bits[0]));
     const float sc = pow2_scale_for(__uint_as_float(bits[1]));
+    float sx = points_are_u8 ? 8.0f : pow2_scale_for(__uint_as_float(bits[0]));
+    sx = fminf(sx, sc);
+    sx = fmaxf(sx, sc * 1.862645149230957e-09f);  // 2^-29
     scal[0] = sx;
     scal[1] = sc;
-    scal[2] = -2.0f / (sx * sc);
+    scal[2] = 1.0f / (sx * sc);
+    scal[3] = 32768.0f * sx / sc;
 }
 
-// One warp per row: writes the scaled fp16 copy (row pitch kp, zero padded beyond d) and the fp32
-// squared norm.  Rows in [rows, rows_padded) only get norm = +inf (their operand rows are never
-// read: the TMA zero-fills rows beyond the tensor).  Lane g handles columns [8g, 8g+8).
-template <typename T>
-__global__ void convert_rows_kernel(const T* __restrict__ x, int64_t rows, int64_t rows_padded, int d, int kp,
-                                    const float* __restrict__ scal, int which_scale, __half* __restrict__ out,
+// One warp per row.  Lane g converts columns [8g, 8g+8) of the data part; after the norm is reduced
+// lanes 0 and 1 write the 16 extra columns.
+template <typename T, bool CENTROID>
+__global__ void convert_rows_kernel(const T* __restrict__ x, int64_t rows, int d, int kd,
+                                    const float* __restrict__ scal, __half* __restrict__ out,
                                     float* __restrict__ norms) {
     const int lane = threadIdx.x & 31;
     const int64_t row = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
-    if (row >= rows_padded) return;
-    if (row >= rows) {
-        if (lane == 0) norms[row] = __int_as_float(0x7f800000);
-        return;
-    }
-    const float s = scal[which_scale];
+    if (row >= rows) return;
+    const int kp = kd + 16;
+    const float sc = scal[1];
+    const float s = CENTROID ? -2.0f * sc : scal[0];
     float acc = 0.0f;
     const int c0 = lane * 8;
-    if (c0 < kp) {
+    if (c0 < kd) {
         float v[8];
         if (c0 < d) {
             if constexpr (sizeof(T) == 1) {
@@ -95,7 +102,30 @@ __global__ void convert_rows_kernel(const T* __restrict__ x, int64_t rows, int64
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
-    if (lane == 0) norms[row] = acc;
+    if (lane < 2) {
+        __half a[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a[i] = __float2half_rn(0.0f);
+        if (lane == 0) {
+            if (CENTROID) {
+                const float w = sc * sc * acc * 3.0517578125e-05f;  // 2^-15; exact power-of-two scaling
+                const __half hi = __float2half_rn(w);
+                const float r1 = w - __half2float(hi);
+                const __half mid = __float2half_rn(r1);
+                const float r2 = r1 - __half2float(mid);
+                a[0] = hi;
+                a[1] = mid;
+                a[2] = __float2half_rn(r2);
+            } else {
+                const __half av = __float2half_rn(scal[3]);
+                a[0] = av;
+                a[1] = av;
+                a[2] = av;
+            }
+        }
+        *reinterpret_cast<uint4*>(out + row * kp + kd + lane * 8) = *reinterpret_cast<const uint4*>(a);
+    }
+    if (lane == 0 && norms != nullptr) norms[row] = acc;
 }
 
 }  // namespace ivf

@@ -55,6 +55,9 @@ def main():
 
     call()
     B.ivf_check()
+    B.ivf_debug_stats(True)
+    call()
+    stats = B.ivf_debug_stats(False)
     B.ivf_debug_timing(True)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
@@ -68,6 +71,8 @@ def main():
            "ms_per_call": e0.elapsed_time(e1) / args.reps,
            "kernel_ms": {name: ms / max(cnt, 1) for name, (ms, cnt) in fam.items() if cnt}}
     fused = out["kernel_ms"].get("fused_argmin") or out["kernel_ms"].get("fused_topk")
+    if k > 1:
+        out["stats_per_call"] = stats
     if fused:
         out["fused_tflops"] = flops / (fused / 1e3) / 1e12
     print(json.dumps(out))

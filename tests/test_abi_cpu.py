@@ -92,3 +92,13 @@ def test_schedule_covers_every_unit_once_and_bounds_partials(n, nlist, d, k, sms
             per_row_tile[r1] = per_row_tile.get(r1, 0) + 1
     assert prev_end == T
     assert max(per_row_tile.values()) <= pl["partials"]
+
+
+def test_threshold_rule_selection():
+    assert binding.ivf_debug_rule(1, 65536) == (-1, 1)
+    assert binding.ivf_debug_rule(16, 65536) == (0, 1)            # running: exact
+    assert binding.ivf_debug_rule(64, 65536) == (1, 16)           # threshold pass over every 16th centroid
+    assert binding.ivf_debug_rule(128, 262144) == (1, 32)
+    assert binding.ivf_debug_rule(256, 1 << 20) == (1, 64)
+    assert binding.ivf_debug_rule(512, 600)[0] == 2               # sample too small: bounded logs
+    assert binding.ivf_debug_rule(17, 2044)[0] == 2 and binding.ivf_debug_rule(17, 2045) == (1, 4)

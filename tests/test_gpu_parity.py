@@ -45,6 +45,8 @@ SMALL = [
     (500, 20000, 128, 64, "u8"), (200, 700, 256, 8, "f32"), (200, 700, 192, 1, "u8"), (64, 40000, 16, 128, "f32"),
     (700, 513, 64, 512, "f32"), (130, 2000, 48, 2, "u8"), (40000, 3000, 128, 1, "u8"), (257, 9000, 96, 256, "f32"),
     (5, 600, 32, 600 - 88, "f32"),
+    # long centroid sweeps per CTA: the sampled-threshold rule
+    (128, 500000, 64, 64, "f32"), (100, 300000, 128, 40, "u8"), (128, 500000, 64, 17, "f32"), (300, 400000, 96, 128, "f32"),
 ]
 
 
@@ -83,6 +85,25 @@ def test_integer_inputs_are_bit_exact_including_ties(n, nlist, d, k):
     ids, dists = _route(q, c, k)
     st = parity.check_route(q, c, k, ids, dists, exact=True)
     assert st["rows_identical"] == 1.0
+
+
+@pytest.mark.parametrize("n,nlist,d,k,dtype", [(300, 5000, 128, 40, "u8"), (130, 2000, 96, 17, "f32"), (64, 70000, 64, 200, "f32")])
+def test_brute_force_recomputation_of_failed_rows(n, nlist, d, k, dtype):
+    # every row is declared failed by the merge, so all results come from the exact fallback kernel
+    x, c = _rand(n, nlist, d, dtype, seed=7)
+    B.ivf_debug_force_fallback(True)
+    try:
+        ids, dists = _route(x, c, k)
+    finally:
+        B.ivf_debug_force_fallback(False)
+    parity.check_route(x, c, k, ids, dists)
+    q, ci = synth.integer_case(200, 3000, 64, seed=3)
+    B.ivf_debug_force_fallback(True)
+    try:
+        ids, dists = _route(q, ci, 50)
+    finally:
+        B.ivf_debug_force_fallback(False)
+    parity.check_route(q, ci, 50, ids, dists, exact=True)
 
 
 def test_duplicate_centroids_resolve_to_lower_id():
