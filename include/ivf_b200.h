@@ -87,6 +87,32 @@ int ivf_centroid_update(const void* points, ivf_dtype ptype, const int32_t* ids,
                         int nlist, float* sums, int64_t* counts, void* stream);
 
 /*
+ * The same accumulation for callers that must not allocate device memory when they call.
+ * (This entry point has no counterpart in the paper; it exists for how the library is deployed.)
+ * Think of an index-maintenance thread living beside a serving process that has already handed all
+ * free device memory to its own pool, where a cudaMalloc would fail or stall; or of a latency-bound
+ * loop that cannot afford the device-wide synchronisation a cudaMalloc or cudaFree implies.
+ * ivf_centroid_update grows the library workspace on demand; this variant never does.  It calls no
+ * cudaMalloc, cudaFree or other allocating routine: its scratch (list counts, offsets, cursors and
+ * the row permutation) is a fixed array of about 4.8 MB inside the library image, which every
+ * device that loads the library holds until the process exits.
+ *   Limits   n <= 1,048,576 rows and nlist <= 65,536 lists per call; anything larger returns
+ *            IVF_ERR_UNSUPPORTED with a message (split the rows over several calls: the
+ *            accumulation composes).  Other arguments, layouts and results are those of
+ *            ivf_centroid_update.
+ *   Set-up   the first call on each device looks up the array's device address (with that device
+ *            current); make that first call before starting any stream capture.
+ *   Sharing  all calls on a device use the one array, which still holds the previous call's
+ *            contents (the call clears what it needs cleared).  Two calls whose kernels overlap on
+ *            the GPU -- different streams without an ordering between them -- race on it: keep the
+ *            calls of a device in one stream or order them with events.
+ *   Bad ids  rows whose id is outside [0, nlist) are skipped; this variant does not report them
+ *            through ivf_check.
+ */
+int ivf_centroid_update_noalloc(const void* points, ivf_dtype ptype, const int32_t* ids, int64_t n, int d,
+                                int nlist, float* sums, int64_t* counts, void* stream);
+
+/*
  * Helper: new centroid = sums / counts per list (float32 divide); a list with count 0 keeps its
  * row of centroids_inout (the paper does not say what an empty list does).  All device pointers.
  */

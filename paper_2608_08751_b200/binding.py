@@ -20,7 +20,8 @@ IVF_ERR_INVALID_ARG, IVF_ERR_UNSUPPORTED, IVF_ERR_ALLOC = -1, -2, -3
 IVF_ERR_CUDA, IVF_ERR_DEVICE_TIMEOUT, IVF_ERR_BAD_ID = -4, -5, -6
 
 EXPORTS = (
-    "ivf_route", "ivf_assign", "ivf_centroid_update", "ivf_centroid_finalize", "ivf_assign_update",
+    "ivf_route", "ivf_assign", "ivf_centroid_update", "ivf_centroid_update_noalloc", "ivf_centroid_finalize",
+    "ivf_assign_update",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
     "ivf_debug_plan", "ivf_debug_span", "ivf_debug_set_wait_limit_ns",
     "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_stats",
@@ -52,6 +53,7 @@ def lib() -> ctypes.CDLL:
     L.ivf_route.argtypes = [vp, i64, i32, i32, vp, i32, i32, vp, vp, vp]
     L.ivf_assign.argtypes = [vp, i64, i32, i32, vp, i32, vp, vp, vp]
     L.ivf_centroid_update.argtypes = [vp, i32, vp, i64, i32, i32, vp, vp, vp]
+    L.ivf_centroid_update_noalloc.argtypes = [vp, i32, vp, i64, i32, i32, vp, vp, vp]
     L.ivf_centroid_finalize.argtypes = [vp, vp, i32, i32, vp, vp]
     L.ivf_assign_update.argtypes = [vp, i64, i32, i32, vp, i32, vp, vp, vp, vp, i64, vp]
     L.ivf_check.argtypes = [vp]
@@ -166,6 +168,29 @@ def ivf_centroid_update(points: torch.Tensor, ids: torch.Tensor, sums: torch.Ten
     with torch.cuda.device(dev):
         rc = lib().ivf_centroid_update(_ptr(points), _dtype_code(points), _ptr(ids), n, d, nlist,
                                        _ptr(sums), _ptr(counts), _stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
+
+
+def ivf_centroid_update_noalloc(points: torch.Tensor, ids: torch.Tensor, sums: torch.Tensor, counts: torch.Tensor):
+    """ivf_centroid_update for callers that must not allocate device memory at call time (for
+    instance beside a serving process whose pool already owns all free memory): the library's
+    built-in scratch is used, so at most 1,048,576 rows and 65,536 lists per call.  Calls on one
+    device share that scratch and must not overlap on the GPU."""
+    if not points.is_cuda:
+        raise ValueError("points must be a CUDA tensor")
+    _rows(points, "points")
+    _dev(ids, "ids", torch.int32)
+    _dev(sums, "sums", torch.float32)
+    _dev(counts, "counts", torch.int64)
+    n, d = points.shape
+    nlist = sums.shape[0]
+    if sums.shape != (nlist, d) or counts.shape != (nlist,) or ids.shape != (n,):
+        raise ValueError("shape mismatch between points, ids, sums and counts")
+    dev = points.device
+    with torch.cuda.device(dev):
+        rc = lib().ivf_centroid_update_noalloc(_ptr(points), _dtype_code(points), _ptr(ids), n, d, nlist,
+                                               _ptr(sums), _ptr(counts), _stream(dev))
     if rc != IVF_OK:
         _raise(rc)
 

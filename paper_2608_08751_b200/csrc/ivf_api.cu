@@ -839,3 +839,85 @@ int ivf_debug_set_wait_limit_ns(int64_t ns) {
 }
 
 }  // extern "C"
+
+// ====================================================================== allocation-free update
+// Scratch of ivf_centroid_update_noalloc: lives in the module image, so every device that loads
+// the library holds these ~4.8 MB until the process exits.  Layout (ints):
+//   [0, 8)                         header: [0] = "an id was out of range" flag of the last call
+//   [8, 8 + L)                     per-list member counts of the call        (L = kNoAllocMaxLists)
+//   [8 + L, 8 + 2L + 1)            exclusive offsets of the list segments
+//   [8 + 2L + 8, 8 + 3L + 8)       per-list fill cursors
+//   [8 + 3L + 8, ... + R)          row permutation sorted by list             (R = kNoAllocMaxRows)
+namespace {
+constexpr int kNoAllocMaxLists = 65536;
+constexpr int kNoAllocMaxRows = 1 << 20;
+constexpr size_t kNoAllocInts = 8 + 3 * static_cast<size_t>(kNoAllocMaxLists) + 8 + kNoAllocMaxRows;
+static __device__ __align__(256) int g_noalloc_scratch[kNoAllocInts];
+// device address of the array above, per device (the host-side symbol is not a device pointer)
+int* g_noalloc_ptr[kMaxDevices] = {};
+}  // namespace
+
+extern "C" int ivf_centroid_update_noalloc(const void* points, ivf_dtype ptype, const int32_t* ids, int64_t n, int d,
+                                           int nlist, float* sums, int64_t* counts, void* stream_) {
+    if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
+    if (ptype != IVF_F32 && ptype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
+    if (d < 16 || d > 256 || d % 16 != 0)
+        return fail(IVF_ERR_UNSUPPORTED, "d = %d: must be a multiple of 16 in [16, 256]", d);
+    if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
+    if (n > kNoAllocMaxRows)
+        return fail(IVF_ERR_UNSUPPORTED,
+                    "ivf_centroid_update_noalloc: n = %lld exceeds the built-in scratch (at most %d rows per call); "
+                    "split the rows or use ivf_centroid_update",
+                    (long long)n, kNoAllocMaxRows);
+    if (nlist > kNoAllocMaxLists)
+        return fail(IVF_ERR_UNSUPPORTED,
+                    "ivf_centroid_update_noalloc: nlist = %d exceeds the built-in scratch (at most %d lists); "
+                    "use ivf_centroid_update",
+                    nlist, kNoAllocMaxLists);
+    if (n == 0) return IVF_OK;
+    if (!points || !ids || !sums || !counts) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    if ((reinterpret_cast<uintptr_t>(points) & 15) || (reinterpret_cast<uintptr_t>(sums) & 15))
+        return fail(IVF_ERR_INVALID_ARG, "points and sums must be 16-byte aligned");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(IVF_ERR_CUDA, "device index %d out of range", dev);
+    int* base = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        if (!g_noalloc_ptr[dev]) {
+            // first call on this device: look the array's device address up (no allocation involved)
+            void* p = nullptr;
+            CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+            g_noalloc_ptr[dev] = static_cast<int*>(p);
+        }
+        base = g_noalloc_ptr[dev];
+    }
+    int* flag = base;
+    int* cnt = base + 8;
+    int* off = cnt + kNoAllocMaxLists;
+    int* cur = off + kNoAllocMaxLists + 8;
+    int* perm = cur + kNoAllocMaxLists;
+
+    // the array keeps the previous call's contents: the counts and the flag must start at zero
+    // (offsets, cursors and the permutation are fully rewritten by the kernels below)
+    CUDA_TRY(cudaMemsetAsync(flag, 0, 8 * sizeof(int), stream));
+    CUDA_TRY(cudaMemsetAsync(cnt, 0, static_cast<size_t>(nlist) * sizeof(int), stream));
+    const unsigned rb = static_cast<unsigned>((n + 255) / 256);
+    update_hist_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, cnt, flag);
+    LAUNCH_CHECK();
+    update_scan_kernel<<<1, 1024, 0, stream>>>(cnt, nlist, off, cur);
+    LAUNCH_CHECK();
+    update_fill_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, off, cur, perm);
+    LAUNCH_CHECK();
+    const unsigned lb = static_cast<unsigned>((static_cast<int64_t>(nlist) * 32 + 255) / 256);
+    if (ptype == IVF_U8)
+        update_reduce_kernel<uint8_t><<<lb, 256, 0, stream>>>(static_cast<const uint8_t*>(points), perm, off, nlist, d,
+                                                              sums, reinterpret_cast<long long*>(counts));
+    else
+        update_reduce_kernel<float><<<lb, 256, 0, stream>>>(static_cast<const float*>(points), perm, off, nlist, d,
+                                                            sums, reinterpret_cast<long long*>(counts));
+    LAUNCH_CHECK();
+    return IVF_OK;
+}
