@@ -147,8 +147,9 @@ int64_t ivf_launch_count(void);
 /*
  * Test hooks (host logic only; no kernel is launched).
  *   ivf_debug_plan   the persistent schedule of the fused kernel for a problem size on a device
- *                    with `num_sms` SMs: writes {row_tiles, col_tiles, ctas, max_partials_per_row_tile,
- *                    block_n, k_slices, stages, smem_bytes} to out[8].
+ *                    with `num_sms` SMs: writes {row_groups, col_tiles, ctas, max_partials_per_row,
+ *                    block_n, k_slices, stages, smem_bytes, row tiles of 128 points per row group}
+ *                    to out[9].
  *   ivf_debug_span   first unit and one-past-last unit of CTA `cta` in that schedule.
  *   ivf_debug_set_wait_limit_ns   time limit of every device-side wait (0 restores the default
  *                    of 2 s).
@@ -156,7 +157,7 @@ int64_t ivf_launch_count(void);
  *                    on a barrier nothing ever completes: after the limit it records
  *                    IVF_ERR_DEVICE_TIMEOUT (wait site 99) in the status word and returns normally.
  */
-int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[8]);
+int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[9]);
 int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int64_t out[2]);
 int ivf_debug_set_wait_limit_ns(int64_t ns);
 int ivf_debug_wait_probe(void* stream);

@@ -250,11 +250,11 @@ def ivf_release_workspace() -> None:
 
 
 def ivf_debug_plan(n: int, nlist: int, d: int, k: int, num_sms: int = 148) -> dict:
-    out = (ctypes.c_int64 * 8)()
+    out = (ctypes.c_int64 * 9)()
     rc = lib().ivf_debug_plan(n, nlist, d, k, num_sms, out)
     if rc != IVF_OK:
         _raise(rc)
-    keys = ("row_tiles", "col_tiles", "ctas", "partials", "block_n", "k_slices", "stages", "smem_bytes")
+    keys = ("row_tiles", "col_tiles", "ctas", "partials", "block_n", "k_slices", "stages", "smem_bytes", "mtiles")
     return dict(zip(keys, (int(v) for v in out)))
 
 

@@ -6,7 +6,10 @@
 // with x' = sx x, c'' = -2 sc c, w = sc^2 |c|^2 / 2^15 split into three fp16 parts and
 // A = 2^15 sx / sc (sx, sc exact powers of two).  The epilogue only compares.
 //
-// One persistent CTA per SM walks a contiguous span of (row tile, centroid tile) units.
+// One persistent CTA per SM walks a contiguous span of (row group, centroid tile) units.  A row
+// group is MT = 1 or 2 row tiles of 128 points that stay in shared memory; with MT = 2 every centroid
+// tile brought from L2 feeds two MMA sweeps (one TMEM accumulator buffer each), which halves the
+// L2 -> shared-memory traffic per FLOP.
 //   warp 0      TMA producer: the stationary 128-row point tile and a ring of centroid tiles
 //   warp 1      single-thread tcgen05.mma issuer; accumulators live in TMEM (fp32), two buffers,
 //               so the next tile's MMAs overlap this tile's epilogue
@@ -61,7 +64,7 @@ struct FusedParams {
     int block_n;          // centroids per tile: 256 or 128
     int nstage;           // centroid-tile ring depth
     int col_tiles;        // centroid tiles per sweep
-    int64_t total_units;  // row tiles * col_tiles
+    int64_t total_units;  // row groups * col_tiles
     int partials;         // partial-result slots per row (CTAs sharing a row tile x kEpiHalves)
     int cap;              // candidate-log capacity per (row, slot), k > 1 only
     int rule;             // k > 1: TAU_RUNNING, TAU_GIVEN or TAU_BOUNDED
@@ -79,9 +82,9 @@ __host__ __device__ inline int cta_of_unit(int64_t T, int G, int64_t u) {
     return static_cast<int>(((u + 1) * G - 1) / T);
 }
 
-__host__ __device__ inline size_t fused_smem_bytes(int kslices, int block_n, int nstage) {
+__host__ __device__ inline size_t fused_smem_bytes(int kslices, int block_n, int nstage, int mtiles) {
     return 1024                                                                        // alignment slack
-           + static_cast<size_t>(kBlockM) * (kslices * kSliceRowBytes + kAugRowBytes)  // point tile
+           + static_cast<size_t>(mtiles) * kBlockM * (kslices * kSliceRowBytes + kAugRowBytes)  // point tiles
            + static_cast<size_t>(nstage) * block_n * (kslices * kSliceRowBytes + kAugRowBytes)
            + 256                                                                       // barriers etc.
            + kNumEpiWarps * 256 * sizeof(int);                                         // radix histograms
@@ -340,7 +343,7 @@ __device__ __forceinline__ void consume(uint32_t (&acc)[32], int jbase, RowState
     }
 }
 
-template <int EPI>
+template <int EPI, int MT>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_xa,
                   const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_ca,
@@ -352,7 +355,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     const int b_data_bytes = p.kslices * p.block_n * kSliceRowBytes;
     const int stage_bytes = b_data_bytes + p.block_n * kAugRowBytes;
     uint8_t* smem_a = smem;
-    uint8_t* smem_b = smem + a_bytes;
+    uint8_t* smem_b = smem + MT * a_bytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_b + static_cast<size_t>(p.nstage) * stage_bytes);
     uint64_t* a_full = bars + 0;
     uint64_t* a_empty = bars + 1;
@@ -419,12 +422,15 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 const int t1 = static_cast<int>((u1 - r * NT < NT) ? (u1 - r * NT) : NT);
                 if (seg > 0) ok = mbar_wait(a_empty, (seg - 1) & 1, ctl, 1);
                 if (!ok) break;
-                mbar_arrive_expect_tx(a_full, a_bytes);
+                mbar_arrive_expect_tx(a_full, MT * a_bytes);
                 ++a_armed;
-                for (int s = 0; s < p.kslices; ++s)
-                    tma_load_2d(smem_a + s * kBlockM * kSliceRowBytes, &tmap_x, a_full, s * kSliceK,
-                                static_cast<int>(r * kBlockM));
-                tma_load_2d(smem_a + a_data_bytes, &tmap_xa, a_full, kd, static_cast<int>(r * kBlockM));
+                for (int h = 0; h < MT; ++h) {
+                    const int y = static_cast<int>((r * MT + h) * kBlockM);
+                    uint8_t* dst = smem_a + h * a_bytes;
+                    for (int s = 0; s < p.kslices; ++s)
+                        tma_load_2d(dst + s * kBlockM * kSliceRowBytes, &tmap_x, a_full, s * kSliceK, y);
+                    tma_load_2d(dst + a_data_bytes, &tmap_xa, a_full, kd, y);
+                }
                 for (int t = t0; t < t1; ++t) {
                     const int st = it % p.nstage;
                     const uint32_t ph = (it / p.nstage) & 1;
@@ -472,28 +478,35 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 const int t1 = static_cast<int>((u1 - r * NT < NT) ? (u1 - r * NT) : NT);
                 ok = mbar_wait(a_full, seg & 1, ctl, 3);
                 if (!ok) break;
-                for (int t = t0; t < t1; ++t) {
+                for (int t = t0; t < t1 && ok; ++t) {
                     const int st = it % p.nstage;
                     const uint32_t ph = (it / p.nstage) & 1;
-                    const int buf = it & 1;
-                    const uint32_t aph = (it >> 1) & 1;
                     ok = mbar_wait(&b_full[st], ph, ctl, 4);
-                    if (ok) ok = mbar_wait(&t_empty[buf], aph ^ 1u, ctl, 5);
                     if (!ok) break;
-                    tc_fence_after_sync();
-                    const uint32_t d_tmem = tmem_base + buf * kAccStride;
                     const uint32_t b_stage = b_addr + st * stage_bytes;
-                    for (int kk = 0; kk < p.ksteps; ++kk) {
-                        const int slice = kk >> 2;
-                        const uint32_t off = (kk & 3) * 32;  // 16 fp16 = 32 bytes inside the swizzled row
-                        const uint64_t adesc = umma_desc_sw128(a_addr + slice * kBlockM * kSliceRowBytes + off);
-                        const uint64_t bdesc = umma_desc_sw128(b_stage + slice * p.block_n * kSliceRowBytes + off);
-                        umma_f16(d_tmem, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
+                    for (int h = 0; h < MT; ++h) {
+                        const int su = it * MT + h;  // accumulator buffers alternate per (tile, row tile)
+                        const int buf = su & 1;
+                        const uint32_t aph = (su >> 1) & 1;
+                        ok = mbar_wait(&t_empty[buf], aph ^ 1u, ctl, 5);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        const uint32_t d_tmem = tmem_base + buf * kAccStride;
+                        const uint32_t a_tile = a_addr + h * a_bytes;
+                        for (int kk = 0; kk < p.ksteps; ++kk) {
+                            const int slice = kk >> 2;
+                            const uint32_t off = (kk & 3) * 32;  // 16 fp16 = 32 bytes inside the swizzled row
+                            const uint64_t adesc = umma_desc_sw128(a_tile + slice * kBlockM * kSliceRowBytes + off);
+                            const uint64_t bdesc =
+                                umma_desc_sw128(b_stage + slice * p.block_n * kSliceRowBytes + off);
+                            umma_f16(d_tmem, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
+                        }
+                        umma_f16(d_tmem, umma_desc_sw32(a_tile + a_data_bytes), umma_desc_sw32(b_stage + b_data_bytes),
+                                 idesc, 1u);
+                        umma_commit(&t_full[buf]);
                     }
-                    umma_f16(d_tmem, umma_desc_sw32(a_addr + a_data_bytes), umma_desc_sw32(b_stage + b_data_bytes),
-                             idesc, 1u);
+                    if (!ok) break;
                     umma_commit(&b_empty[st]);
-                    umma_commit(&t_full[buf]);
                     ++it;
                 }
                 if (ok) umma_commit(a_empty);
@@ -520,98 +533,116 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         int it = 0;
         bool ok = true;
         for (int64_t u = u0; u < u1 && ok;) {
-            const int64_t r = u / NT;
+            const int64_t r = u / NT;  // row group
             const int t0 = static_cast<int>(u - r * NT);
             const int t1 = static_cast<int>((u1 - r * NT < NT) ? (u1 - r * NT) : NT);
-            const int64_t row = r * kBlockM + row_in_tile;
-            const bool valid = row < p.n;
             const int slot = (b - cta_of_unit(T, G, r * NT)) * kEpiHalves + half;
-            [[maybe_unused]] const int64_t warp_row0 = r * kBlockM + quad * 32;
 
-            RowState<EPI> st;
-            st.tau = valid ? INF : -INF;  // invalid rows: a threshold nothing passes
-            if constexpr (EPI == EPI_ARGMIN) st.bestj = 0x7fffffff;
-            if constexpr (EPI == EPI_RUNNING || EPI == EPI_SKETCH) {
+            RowState<EPI> st[MT];
+            int64_t row[MT];
+            bool valid[MT];
 #pragma unroll
-                for (int i = 0; i < kSampleM; ++i) st.net[i] = INF;
-            }
-            if constexpr (kHasLog) {
-                st.cnt = 0;
-                st.log = p.part + (static_cast<size_t>(valid ? row : 0) * p.partials + slot) * p.cap;
-                if (EPI == EPI_FILTER && p.rule == TAU_GIVEN && valid) st.tau = p.tau_in[row];
+            for (int h = 0; h < MT; ++h) {
+                row[h] = (r * MT + h) * kBlockM + row_in_tile;
+                valid[h] = row[h] < p.n;
+                st[h].tau = valid[h] ? INF : -INF;  // invalid rows: a threshold nothing passes
+                if constexpr (EPI == EPI_ARGMIN) st[h].bestj = 0x7fffffff;
+                if constexpr (EPI == EPI_RUNNING || EPI == EPI_SKETCH) {
+#pragma unroll
+                    for (int i = 0; i < kSampleM; ++i) st[h].net[i] = INF;
+                }
+                if constexpr (kHasLog) {
+                    st[h].cnt = 0;
+                    st[h].log = p.part + (static_cast<size_t>(valid[h] ? row[h] : 0) * p.partials + slot) * p.cap;
+                    if (EPI == EPI_FILTER && p.rule == TAU_GIVEN && valid[h]) st[h].tau = p.tau_in[row[h]];
+                }
             }
 
-            for (int t = t0; t < t1; ++t) {
-                const int buf = it & 1;
-                const uint32_t aph = (it >> 1) & 1;
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(&t_full[buf], aph, ctl, 6));
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + buf * kAccStride;
+            for (int t = t0; t < t1 && ok; ++t) {
                 const bool ragged = (t + 1) * p.block_n > p.nlist;
                 const int tile_j0 = t * p.block_n;
+#pragma unroll
+                for (int h = 0; h < MT; ++h) {
+                    const int su = it * MT + h;
+                    const int buf = su & 1;
+                    const uint32_t aph = (su >> 1) & 1;
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(&t_full[buf], aph, ctl, 6));
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + buf * kAccStride;
+                    [[maybe_unused]] const int64_t warp_row0 = (r * MT + h) * kBlockM + quad * 32;
 
-                // chunk q of this warp starts at column ((q/2) * halves + half) * 64 + (q%2) * 32
-                auto col_of = [&](int q) { return ((q >> 1) * kEpiHalves + half) * 64 + (q & 1) * 32; };
-                auto after_chunk = [&]() {
-                    if constexpr (kHasLog) {
-                        if (__any_sync(0xFFFFFFFFu, st.cnt > p.cap - 32)) {
-                            __syncwarp();
-                            for (int rr = 0; rr < 32; ++rr) {
-                                const int c_r = __shfl_sync(0xFFFFFFFFu, st.cnt, rr);
-                                if (c_r > p.cap - 32) {
-                                    Entry* lr =
-                                        p.part + (static_cast<size_t>(warp_row0 + rr) * p.partials + slot) * p.cap;
-                                    const float tk = warp_select_k(lr, c_r, p.k, hist, lane);
-                                    if (p.stats && lane == 0) atomicAdd(&p.stats[0], 1ull);
-                                    if (lane == rr) {
-                                        st.cnt = p.k;
-                                        st.tau = fminf(st.tau, tk);
+                    // chunk q of this warp starts at column ((q/2) * halves + half) * 64 + (q%2) * 32
+                    auto col_of = [&](int q) { return ((q >> 1) * kEpiHalves + half) * 64 + (q & 1) * 32; };
+                    auto after_chunk = [&]() {
+                        if constexpr (kHasLog) {
+                            if (__any_sync(0xFFFFFFFFu, st[h].cnt > p.cap - 32)) {
+                                __syncwarp();
+                                for (int rr = 0; rr < 32; ++rr) {
+                                    const int c_r = __shfl_sync(0xFFFFFFFFu, st[h].cnt, rr);
+                                    if (c_r > p.cap - 32) {
+                                        Entry* lr = p.part +
+                                                    (static_cast<size_t>(warp_row0 + rr) * p.partials + slot) * p.cap;
+                                        const float tk = warp_select_k(lr, c_r, p.k, hist, lane);
+                                        if (p.stats && lane == 0) atomicAdd(&p.stats[0], 1ull);
+                                        if (lane == rr) {
+                                            st[h].cnt = p.k;
+                                            st[h].tau = fminf(st[h].tau, tk);
+                                        }
                                     }
                                 }
                             }
                         }
-                    }
-                };
-                uint32_t accA[32], accB[32];
-                tmem_ld_32x32b_x32(taddr + col_of(0), accA);
+                    };
+                    // TMEM -> register loads have a long latency and only one wait primitive
+                    // (it waits for all of the thread's loads), so each round trip fetches 64 columns
+                    // as two 32-column loads issued back to back; the other epilogue warp of the
+                    // scheduler computes meanwhile.
+                    uint32_t accA[32], accB[32];
 #pragma unroll
-                for (int q = 0; q < 4; q += 2) {
-                    if (q < nq) {
-                        tmem_wait_ld_regs(accA);
-                        tmem_ld_32x32b_x32(taddr + col_of(q + 1), accB);  // in flight while accA is consumed
-                        if (ragged) mask_ragged(accA, tile_j0 + col_of(q), p.nlist);
-                        consume<EPI>(accA, tile_j0 + col_of(q), st);
-                        after_chunk();
-                        tmem_wait_ld_regs(accB);
-                        if (q + 2 < nq) tmem_ld_32x32b_x32(taddr + col_of(q + 2), accA);
-                        if (ragged) mask_ragged(accB, tile_j0 + col_of(q + 1), p.nlist);
-                        consume<EPI>(accB, tile_j0 + col_of(q + 1), st);
-                        after_chunk();
+                    for (int q = 0; q < 4; q += 2) {
+                        if (q < nq) {
+                            tmem_ld_32x32b_x32(taddr + col_of(q), accA);
+                            tmem_ld_32x32b_x32(taddr + col_of(q + 1), accB);
+                            tmem_wait_ld_regs(accA);
+                            tmem_wait_ld_regs(accB);
+                            if (ragged) {
+                                mask_ragged(accA, tile_j0 + col_of(q), p.nlist);
+                                mask_ragged(accB, tile_j0 + col_of(q + 1), p.nlist);
+                            }
+                            consume<EPI>(accA, tile_j0 + col_of(q), st[h]);
+                            after_chunk();
+                            consume<EPI>(accB, tile_j0 + col_of(q + 1), st[h]);
+                            after_chunk();
+                        }
                     }
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&t_empty[buf]);
                 }
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&t_empty[buf]);
                 ++it;
             }
-            if (ok && valid) {
-                const size_t at = static_cast<size_t>(row) * p.partials + slot;
-                if constexpr (EPI == EPI_ARGMIN) {
-                    Entry e;
-                    e.v = st.tau;
-                    e.j = st.bestj;
-                    p.part[at] = e;
-                } else if constexpr (EPI == EPI_SKETCH) {
-                    // the partial result of the threshold pass: the thread's 16 smallest group minima
-                    Entry* log = p.part + at * p.cap;
+            if (ok) {
 #pragma unroll
-                    for (int i = 0; i < kSampleM; ++i)
-                        *reinterpret_cast<uint2*>(&log[i]) = make_uint2(__float_as_uint(st.net[i]), 0u);
-                    p.part_meta[at] = make_int2(kSampleM, __float_as_int(INF));
-                } else {
-                    p.part_meta[at] = make_int2(st.cnt, __float_as_int(st.tau));
-                    if (p.stats) atomicAdd(&p.stats[1], static_cast<unsigned long long>(st.cnt));
+                for (int h = 0; h < MT; ++h) {
+                    if (!valid[h]) continue;
+                    const size_t at = static_cast<size_t>(row[h]) * p.partials + slot;
+                    if constexpr (EPI == EPI_ARGMIN) {
+                        Entry e;
+                        e.v = st[h].tau;
+                        e.j = st[h].bestj;
+                        p.part[at] = e;
+                    } else if constexpr (EPI == EPI_SKETCH) {
+                        // the partial result of the threshold pass: the thread's 16 smallest group minima
+                        Entry* log = p.part + at * p.cap;
+#pragma unroll
+                        for (int i = 0; i < kSampleM; ++i)
+                            *reinterpret_cast<uint2*>(&log[i]) = make_uint2(__float_as_uint(st[h].net[i]), 0u);
+                        p.part_meta[at] = make_int2(kSampleM, __float_as_int(INF));
+                    } else {
+                        p.part_meta[at] = make_int2(st[h].cnt, __float_as_int(st[h].tau));
+                        if (p.stats) atomicAdd(&p.stats[1], static_cast<unsigned long long>(st[h].cnt));
+                    }
                 }
             }
             u = r * NT + t1;

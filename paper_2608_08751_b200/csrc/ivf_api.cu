@@ -165,7 +165,8 @@ int ws_get(DeviceCtx& c, WsSlot slot, size_t bytes, cudaStream_t stream, void** 
 // ------------------------------------------------------------------ schedule
 struct Plan {
     int kd, kp, kslices, ksteps, block_n, nstage;
-    int64_t row_tiles;
+    int mtiles;         // row tiles of 128 points per CTA unit (1 or 2)
+    int64_t row_tiles;  // row groups of mtiles * 128 points
     int col_tiles;
     int64_t total_units;
     int ctas;
@@ -194,18 +195,23 @@ int choose_rule(int k, int nlist, int* stride) {
     return TAU_BOUNDED;
 }
 
-int make_plan(int64_t n, int nlist, int d, int k, int num_sms, Plan* pl) {
+int make_plan(int64_t n, int nlist, int d, int k, int num_sms, Plan* pl, bool one_row_tile = false) {
     pl->kd = (d + 63) / 64 * 64;
     pl->kp = pl->kd + kAugK;
     pl->kslices = pl->kd / 64;
     pl->ksteps = (d + 15) / 16;
     pl->block_n = pl->kslices <= 2 ? 256 : 128;
+    // two row tiles per unit when they fit next to a two-stage ring (d <= 128) and there are at
+    // least two row tiles; the epilogues that keep a candidate log stay with one (they are bound by
+    // their own instruction count, not by the centroid traffic, and their per-row state is larger)
+    pl->mtiles = (!one_row_tile && n > kBlockM && fused_smem_bytes(pl->kslices, pl->block_n, 2, 2) <= kSmemLimit) ? 2 : 1;
     int nstage = kMaxStages;
-    while (nstage > 1 && fused_smem_bytes(pl->kslices, pl->block_n, nstage) > kSmemLimit) --nstage;
+    while (nstage > 1 && fused_smem_bytes(pl->kslices, pl->block_n, nstage, pl->mtiles) > kSmemLimit) --nstage;
     if (nstage < 2) return fail(IVF_ERR_UNSUPPORTED, "d = %d does not fit the shared-memory ring", d);
     pl->nstage = nstage;
-    pl->smem = fused_smem_bytes(pl->kslices, pl->block_n, nstage);
-    pl->row_tiles = (n + kBlockM - 1) / kBlockM;
+    pl->smem = fused_smem_bytes(pl->kslices, pl->block_n, nstage, pl->mtiles);
+    const int group_rows = kBlockM * pl->mtiles;
+    pl->row_tiles = (n + group_rows - 1) / group_rows;
     pl->col_tiles = (nlist + pl->block_n - 1) / pl->block_n;
     pl->total_units = pl->row_tiles * pl->col_tiles;
     pl->ctas = static_cast<int>(pl->total_units < num_sms ? pl->total_units : num_sms);
@@ -222,8 +228,8 @@ int64_t rows_per_launch(int d, int k) {
     const int kp = (d + 63) / 64 * 64 + kAugK;
     const int64_t per_row = static_cast<int64_t>(kp) * 2 + 6ll * log_capacity(k) * 8 + (k > kSampleM ? 6ll * 512 * 8 : 0);
     int64_t rows = (int64_t(3) << 30) / per_row;
-    rows = rows / kBlockM * kBlockM;
-    if (rows < kBlockM) rows = kBlockM;
+    rows = rows / (2 * kBlockM) * (2 * kBlockM);
+    if (rows < 2 * kBlockM) rows = 2 * kBlockM;
     if (rows > (int64_t(4) << 20)) rows = int64_t(4) << 20;
     return rows;
 }
@@ -369,21 +375,30 @@ int launch_fused(DeviceCtx& ctx, const Plan& pl, int64_t n, int nlist, int k, in
     fp.wait_limit_ns = g_wait_limit_ns.load();
     if (!ctx.smem_attr_set) {
         const int lim = static_cast<int>(kSmemLimit);
-        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_ARGMIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim));
-        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_RUNNING>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim));
-        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_FILTER>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim));
-        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_SKETCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim));
+        const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_ARGMIN, 1>, attr, lim));
+        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_ARGMIN, 2>, attr, lim));
+        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_RUNNING, 1>, attr, lim));
+        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_FILTER, 1>, attr, lim));
+        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_SKETCH, 1>, attr, lim));
+        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_SKETCH, 2>, attr, lim));
         ctx.smem_attr_set = true;
     }
     const int tk = timing_begin(kind, stream);
-    if (k == 1)
-        fused_topk_kernel<EPI_ARGMIN><<<pl.ctas, kFusedThreads, pl.smem, stream>>>(pp.tmap_x, pp.tmap_xa, tmap_c, tmap_ca, fp);
-    else if (rule == TAU_RUNNING)
-        fused_topk_kernel<EPI_RUNNING><<<pl.ctas, kFusedThreads, pl.smem, stream>>>(pp.tmap_x, pp.tmap_xa, tmap_c, tmap_ca, fp);
-    else if (rule == TAU_SKETCH)
-        fused_topk_kernel<EPI_SKETCH><<<pl.ctas, kFusedThreads, pl.smem, stream>>>(pp.tmap_x, pp.tmap_xa, tmap_c, tmap_ca, fp);
-    else
-        fused_topk_kernel<EPI_FILTER><<<pl.ctas, kFusedThreads, pl.smem, stream>>>(pp.tmap_x, pp.tmap_xa, tmap_c, tmap_ca, fp);
+    const dim3 grid(pl.ctas), block(kFusedThreads);
+#define IVF_LAUNCH(EPI, MT) \
+    fused_topk_kernel<EPI, MT><<<grid, block, pl.smem, stream>>>(pp.tmap_x, pp.tmap_xa, tmap_c, tmap_ca, fp)
+    const bool two = pl.mtiles == 2;
+    if (k == 1) {
+        if (two) IVF_LAUNCH(EPI_ARGMIN, 2); else IVF_LAUNCH(EPI_ARGMIN, 1);
+    } else if (rule == TAU_RUNNING) {
+        IVF_LAUNCH(EPI_RUNNING, 1);
+    } else if (rule == TAU_SKETCH) {
+        if (two) IVF_LAUNCH(EPI_SKETCH, 2); else IVF_LAUNCH(EPI_SKETCH, 1);
+    } else {
+        IVF_LAUNCH(EPI_FILTER, 1);
+    }
+#undef IVF_LAUNCH
     LAUNCH_CHECK();
     timing_end(tk, stream);
     return IVF_OK;
@@ -399,6 +414,7 @@ MergeParams merge_params(const Plan& pl, int64_t n, int k, const Entry* part, co
     mp.col_tiles = pl.col_tiles;
     mp.total_units = pl.total_units;
     mp.ctas = pl.ctas;
+    mp.group_rows = kBlockM * pl.mtiles;
     mp.part = part;
     mp.part_meta = part_meta;
     mp.xn = pp.xn;
@@ -416,7 +432,7 @@ MergeParams merge_params(const Plan& pl, int64_t n, int k, const Entry* part, co
 int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int ptype, int nlist, int k,
                       const CentroidPrep& cp, int32_t* out_ids, float* out_dists, cudaStream_t stream) {
     Plan pl, pls;
-    int rc = make_plan(n, nlist, d, k, ctx.num_sms, &pl);
+    int rc = make_plan(n, nlist, d, k, ctx.num_sms, &pl, k > 1);
     if (rc != IVF_OK) return rc;
     const bool given = k > 1 && cp.rule == TAU_GIVEN;
     size_t part_bytes = static_cast<size_t>(n) * pl.partials * pl.cap * sizeof(Entry);
@@ -481,7 +497,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         MergeParams ms = merge_params(pls, n, kSampleM, part, part_meta, pp, cp.scal);
         ms.tau_out = tau;
         tk = timing_begin(TK_THRESH, stream);
-        merge_select_kernel<<<static_cast<unsigned>(n), kMergeThreads, 0, stream>>>(ms);
+        merge_tau_kernel<<<static_cast<unsigned>((n * 32 + 255) / 256), 256, 0, stream>>>(ms);
         LAUNCH_CHECK();
         timing_end(tk, stream);
     }
@@ -737,11 +753,11 @@ int ivf_release_workspace(void) {
 
 int64_t ivf_launch_count(void) { return g_launches.load(); }
 
-int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[8]) {
+int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[9]) {
     if (n < 1 || nlist < 1 || num_sms < 1 || !out) return fail(IVF_ERR_INVALID_ARG, "bad plan arguments");
     if (d < 16 || d > 256 || d % 16 != 0) return fail(IVF_ERR_UNSUPPORTED, "d = %d", d);
     Plan pl;
-    int rc = make_plan(n, nlist, d, k, num_sms, &pl);
+    int rc = make_plan(n, nlist, d, k, num_sms, &pl, k > 1);
     if (rc != IVF_OK) return rc;
     out[0] = pl.row_tiles;
     out[1] = pl.col_tiles;
@@ -751,13 +767,14 @@ int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[
     out[5] = pl.kslices;
     out[6] = pl.nstage;
     out[7] = static_cast<int64_t>(pl.smem);
+    out[8] = pl.mtiles;
     return IVF_OK;
 }
 
 int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int64_t out[2]) {
     if (n < 1 || nlist < 1 || num_sms < 1 || !out) return fail(IVF_ERR_INVALID_ARG, "bad plan arguments");
     Plan pl;
-    int rc = make_plan(n, nlist, d, k, num_sms, &pl);
+    int rc = make_plan(n, nlist, d, k, num_sms, &pl, k > 1);
     if (rc != IVF_OK) return rc;
     if (cta < 0 || cta >= pl.ctas) return fail(IVF_ERR_INVALID_ARG, "cta %d outside [0, %d)", cta, pl.ctas);
     out[0] = span_begin(pl.total_units, pl.ctas, cta);

@@ -22,6 +22,7 @@ struct MergeParams {
     int col_tiles;
     int64_t total_units;
     int ctas;              // grid size of the fused kernel (defines which slots exist)
+    int group_rows;        // point rows per row group of the fused kernel (128 or 256)
     const Entry* part;
     const int2* part_meta;
     const float* xn;       // |x|^2 per row
@@ -44,7 +45,7 @@ __device__ __forceinline__ int slots_of_row_tile(int64_t total_units, int ctas, 
 __global__ void merge_argmin_kernel(const MergeParams p) {
     const int64_t row = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (row >= p.n) return;
-    const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / kBlockM);
+    const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows);
     const Entry* e = p.part + static_cast<size_t>(row) * p.partials;
     float bv = e[0].v;
     int bj = e[0].j;
@@ -82,45 +83,78 @@ __device__ __forceinline__ void bitonic_sort_smem(uint64_t* keys, int m /* power
     __syncthreads();
 }
 
-// k > 1: one CTA per row.  Candidates <= the row's smallest tau are sorted by the 64-bit key
-// (orderable value, id) in shared memory; more than kSortCap of them are folded in rounds.
+constexpr int kMaxSlots = 512;  // >= 2 * number of CTAs of the fused kernel
+
+// k > 1: one CTA per row.  The row's logs are read as one flattened array (all loads in flight
+// together); candidates <= the row's smallest tau are sorted by the 64-bit key (orderable value,
+// id) in shared memory; more than kSortCap raw entries are folded in rounds.
 __global__ void __launch_bounds__(kMergeThreads) merge_select_kernel(const MergeParams p) {
     __shared__ uint64_t keys[kSortCap];
+    __shared__ int pre[kMaxSlots + 1];  // exclusive prefix of the slots' entry counts
+    __shared__ float s_tau[kMergeThreads / 32];
     __shared__ int s_fill;
     const int64_t row = blockIdx.x;
-    const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / kBlockM);
+    const int ns = min(slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows), kMaxSlots);
     const Entry* base = p.part + static_cast<size_t>(row) * p.partials * p.cap;
     const int2* meta = p.part_meta + static_cast<size_t>(row) * p.partials;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
-    float tau_min = __int_as_float(0x7f800000);
-    for (int s = 0; s < ns; ++s) tau_min = fminf(tau_min, __int_as_float(meta[s].y));
+    // ---- per-slot counts, their prefix sums, and the smallest threshold
+    float tau = __int_as_float(0x7f800000);
+    for (int s0 = 0; s0 < ns; s0 += kMergeThreads) {
+        const int sidx = s0 + threadIdx.x;
+        if (sidx < ns) {
+            const int2 m = meta[sidx];
+            pre[sidx + 1] = min(m.x, p.cap);
+            tau = fminf(tau, __int_as_float(m.y));
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) tau = fminf(tau, __shfl_xor_sync(0xFFFFFFFFu, tau, off));
+    if (lane == 0) s_tau[warp] = tau;
+    if (threadIdx.x == 0) {
+        pre[0] = 0;
+        s_fill = 0;
+    }
+    __syncthreads();
+    if (warp == 0) {  // inclusive scan of pre[1..ns] by one warp, 32 slots at a time
+        int carry = 0;
+        for (int s0 = 0; s0 < ns; s0 += 32) {
+            const int sidx = s0 + lane;
+            int v = sidx < ns ? pre[sidx + 1] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int t = __shfl_up_sync(0xFFFFFFFFu, v, off);
+                if (lane >= off) v += t;
+            }
+            if (sidx < ns) pre[sidx + 1] = v + carry;
+            carry += __shfl_sync(0xFFFFFFFFu, v, 31);
+        }
+    }
+    __syncthreads();
+    float tau_min = s_tau[0];
+#pragma unroll
+    for (int w = 1; w < kMergeThreads / 32; ++w) tau_min = fminf(tau_min, s_tau[w]);
+    const int raw_total = pre[ns];
 
     int kept = 0;   // sorted keys carried at the front of keys[]
     int total = 0;  // candidates <= tau_min seen so far
-    int slot = 0, pos = 0;
-    if (threadIdx.x == 0) s_fill = 0;
-    __syncthreads();
-    while (true) {
-        // append the remaining candidates that pass the threshold, slot by slot, until keys[] is full
-        while (slot < ns) {
-            const int room = kSortCap - s_fill;
-            __syncthreads();  // everyone has read s_fill before anyone appends
-            if (room == 0) break;
-            const int c = min(meta[slot].x, p.cap);
-            const int take = min(c - pos, room);
-            for (int i = threadIdx.x; i < take; i += blockDim.x) {
-                const Entry e = base[static_cast<size_t>(slot) * p.cap + pos + i];
-                if (e.v <= tau_min)
-                    keys[atomicAdd(&s_fill, 1)] =
-                        (static_cast<uint64_t>(orderable(e.v)) << 32) | static_cast<uint32_t>(e.j);
+    for (int done = 0; done < raw_total || done == 0;) {
+        const int room = kSortCap - kept;
+        const int take = min(raw_total - done, room);
+        for (int i = threadIdx.x; i < take; i += blockDim.x) {
+            const int idx = done + i;
+            int lo = 0, hi = ns;  // slot with pre[slot] <= idx < pre[slot + 1]
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (pre[mid] <= idx) lo = mid; else hi = mid;
             }
-            __syncthreads();
-            pos += take;
-            if (pos >= c) {
-                ++slot;
-                pos = 0;
-            }
+            const Entry e = base[static_cast<size_t>(lo) * p.cap + (idx - pre[lo])];
+            if (e.v <= tau_min)
+                keys[atomicAdd(&s_fill, 1)] = (static_cast<uint64_t>(orderable(e.v)) << 32) | static_cast<uint32_t>(e.j);
         }
+        __syncthreads();
+        done += take;
         const int fill = s_fill;
         total += fill - kept;
         int m = 2;
@@ -128,7 +162,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_select_kernel(const Merge
         for (int i = fill + threadIdx.x; i < m; i += blockDim.x) keys[i] = ~0ull;
         bitonic_sort_smem(keys, m);
         kept = min(fill, p.k);
-        if (slot >= ns) break;
+        if (done >= raw_total) break;
         if (threadIdx.x == 0) s_fill = kept;
         __syncthreads();
     }
@@ -154,6 +188,42 @@ __global__ void __launch_bounds__(kMergeThreads) merge_select_kernel(const Merge
         if (p.out_dists)
             p.out_dists[row * p.k + i] = fmaxf(fmaf(from_orderable(static_cast<uint32_t>(key >> 32)), inv, xn), 0.0f);
     }
+}
+
+// Threshold pass: one warp per row reads the partial sketches (16 smallest group minima per
+// thread of the fused kernel) and writes the 16th smallest value overall.
+__global__ void __launch_bounds__(256) merge_tau_kernel(const MergeParams p) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    if (row >= p.n) return;
+    const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows);
+    const Entry* base = p.part + static_cast<size_t>(row) * p.partials * p.cap;
+    const int total = ns * kSampleM;
+    // every lane keeps the 16 smallest of its share; then 16 rounds of "extract the warp minimum"
+    float net[kSampleM];
+#pragma unroll
+    for (int i = 0; i < kSampleM; ++i) net[i] = __int_as_float(0x7f800000);
+    for (int idx = lane; idx < total; idx += 32) {
+        const float v = base[static_cast<size_t>(idx / kSampleM) * p.cap + (idx % kSampleM)].v;
+        if (v < net[kSampleM - 1]) network_insert(net, v);
+    }
+    float result = __int_as_float(0x7f800000);
+#pragma unroll 1
+    for (int round = 0; round < kSampleM; ++round) {
+        float m = net[0];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) m = fminf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+        result = m;
+        // the first lane holding m drops it (shift its sorted list down by one)
+        const uint32_t who = __ballot_sync(0xFFFFFFFFu, net[0] == m);
+        if (who == 0u) break;  // only infinities left
+        if (lane == __ffs(who) - 1) {
+#pragma unroll
+            for (int i = 0; i < kSampleM - 1; ++i) net[i] = net[i + 1];
+            net[kSampleM - 1] = __int_as_float(0x7f800000);
+        }
+    }
+    if (lane == 0) p.tau_out[row] = result;
 }
 
 // ------------------------------------------------------------------ brute-force recomputation

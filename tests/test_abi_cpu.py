@@ -77,7 +77,8 @@ def test_argument_errors_come_before_any_cuda_call():
 def test_schedule_covers_every_unit_once_and_bounds_partials(n, nlist, d, k, sms):
     pl = binding.ivf_debug_plan(n, nlist, d, k, sms)
     T = pl["row_tiles"] * pl["col_tiles"]
-    assert pl["row_tiles"] == -(-n // 128) and pl["col_tiles"] == -(-nlist // pl["block_n"])
+    assert pl["mtiles"] in (1, 2)
+    assert pl["row_tiles"] == -(-n // (128 * pl["mtiles"])) and pl["col_tiles"] == -(-nlist // pl["block_n"])
     assert pl["ctas"] == min(sms, T) and pl["stages"] >= 2 and pl["smem_bytes"] <= 227 * 1024
     prev_end = 0
     per_row_tile = {}
@@ -91,7 +92,7 @@ def test_schedule_covers_every_unit_once_and_bounds_partials(n, nlist, d, k, sms
         if r1 > r0 + 3:  # a CTA covering many whole row tiles: each of those has exactly one partial
             per_row_tile[r1] = per_row_tile.get(r1, 0) + 1
     assert prev_end == T
-    assert max(per_row_tile.values()) <= pl["partials"]
+    assert 2 * max(per_row_tile.values()) <= pl["partials"]  # two epilogue warps share every row
 
 
 def test_threshold_rule_selection():
