@@ -20,7 +20,9 @@
 // a candidate log in global memory.  tau comes from one of three rules, fixed per launch:
 //   running   (k <= 16) tau = the 16th smallest group-of-8 minimum seen so far, kept in a sorted
 //             register network: at least 16 keys are <= tau, so the result is exact;
-//   given     tau is read per row from memory.  The host computes it with a first, small launch of
+//   given     tau is read per row from memory, and the log holds whole groups of 8 keys: if the
+//             minimum of a group passes, the 8 raw keys are appended (two 16-byte stores, ~1.4
+//             instructions per key, no branch) and the merge kernel compares key by key.  The host computes it with a first, small launch of
 //             this same kernel (sketch rule) over every S-th centroid, S = k / 4: the 16th smallest
 //             group minimum of that sample lets about 4k candidates through.  Whether tau was loose
 //             enough is checked exactly by the merge kernel (at least k candidates <= tau); a row
@@ -69,8 +71,10 @@ struct FusedParams {
     int cap;              // candidate-log capacity per (row, slot), k > 1 only
     int rule;             // k > 1: TAU_RUNNING, TAU_GIVEN or TAU_BOUNDED
     const float* tau_in;  // given rule: threshold per row, in key units
-    Entry* part;          // k = 1: [n][partials]; k > 1: [n][partials][cap]
-    int2* part_meta;      // k > 1: [n][partials] {entries in the log, bits of the final tau}
+    Entry* part;          // k = 1: [n][partials]; k > 1: [n][partials][cap] entries, or 48-byte group
+                          // records for the given rule
+    int2* part_meta;      // k > 1: [n][partials] {entries (records) in the log or -1 if it overflowed,
+                          // bits of the final tau}
     int* status;          // sticky device status word
     unsigned long long* stats;  // optional counters: [0] in-kernel selections, [1] log entries written
     uint64_t wait_limit_ns;
@@ -245,7 +249,10 @@ __device__ __forceinline__ void network_insert(float (&a)[kSampleM], float v) {
 }
 
 // Compile-time variants of the epilogue.
-enum { EPI_ARGMIN = 0, EPI_RUNNING = 1, EPI_FILTER = 2, EPI_SKETCH = 3 };
+enum { EPI_ARGMIN = 0, EPI_RUNNING = 1, EPI_FILTER = 2, EPI_SKETCH = 3, EPI_GROUPS = 4 };
+
+// A record of the group log (EPI_GROUPS): 8 consecutive keys and the id of the first.
+constexpr int kRecordBytes = 48;
 
 template <int EPI>
 struct RowState;
@@ -266,6 +273,14 @@ struct RowState<EPI_RUNNING> {
     int cnt;
     Entry* log;
     float net[kSampleM];  // the 16 smallest group-of-8 minima seen
+};
+template <>
+struct RowState<EPI_GROUPS> {
+    float tau;       // threshold, given per row
+    char* wp;        // next record of the group log
+    char* base;      // first record
+    char* limit;     // wp beyond this after a chunk = the log is full
+    int overflow;
 };
 template <>
 struct RowState<EPI_SKETCH> {
@@ -300,6 +315,30 @@ __device__ __forceinline__ void consume(uint32_t (&acc)[32], int jbase, RowState
                     st.bestj = jbase + c;
                 }
             }
+        }
+    } else if constexpr (EPI == EPI_GROUPS) {
+        // One decision per group of 8 columns: if the group's minimum passes the threshold, the
+        // whole group (8 raw keys + the id of the first) is appended with two 16-byte stores; the
+        // merge kernel does the per-key comparison.  About 1.4 instructions per key, no branch.
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t.reg .f32 m;\n\t"
+                "min.f32 m, %2, %3, %4;\n\t"
+                "min.f32 m, m, %5, %6;\n\t"
+                "min.f32 m, m, %7, %8;\n\t"
+                "min.f32 m, m, %9;\n\t"
+                "setp.le.f32 p, m, %1;\n\t"
+                "@p st.global.v4.f32 [%0], {%2, %3, %4, %5};\n\t"
+                "@p st.global.v4.f32 [%0+16], {%6, %7, %8, %9};\n\t"
+                "@p st.global.b32 [%0+32], %10;\n\t"
+                "@p add.s64 %0, %0, 48;\n\t}"
+                : "+l"(st.wp)
+                : "f"(st.tau), "f"(__uint_as_float(acc[8 * g])), "f"(__uint_as_float(acc[8 * g + 1])),
+                  "f"(__uint_as_float(acc[8 * g + 2])), "f"(__uint_as_float(acc[8 * g + 3])),
+                  "f"(__uint_as_float(acc[8 * g + 4])), "f"(__uint_as_float(acc[8 * g + 5])),
+                  "f"(__uint_as_float(acc[8 * g + 6])), "f"(__uint_as_float(acc[8 * g + 7])), "r"(jbase + 8 * g)
+                : "memory");
         }
     } else if constexpr (EPI == EPI_FILTER) {
         // Straight-line predicated code on purpose: hits are rare, but 32 rows share every branch,
@@ -556,6 +595,14 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                     st[h].log = p.part + (static_cast<size_t>(valid[h] ? row[h] : 0) * p.partials + slot) * p.cap;
                     if (EPI == EPI_FILTER && p.rule == TAU_GIVEN && valid[h]) st[h].tau = p.tau_in[row[h]];
                 }
+                if constexpr (EPI == EPI_GROUPS) {
+                    st[h].base = reinterpret_cast<char*>(p.part) +
+                                 (static_cast<size_t>(valid[h] ? row[h] : 0) * p.partials + slot) * p.cap * kRecordBytes;
+                    st[h].wp = st[h].base;
+                    st[h].limit = st[h].base + static_cast<size_t>(p.cap - 4) * kRecordBytes;
+                    st[h].overflow = 0;
+                    if (valid[h]) st[h].tau = p.tau_in[row[h]];
+                }
             }
 
             for (int t = t0; t < t1 && ok; ++t) {
@@ -575,6 +622,14 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                     // chunk q of this warp starts at column ((q/2) * halves + half) * 64 + (q%2) * 32
                     auto col_of = [&](int q) { return ((q >> 1) * kEpiHalves + half) * 64 + (q & 1) * 32; };
                     auto after_chunk = [&]() {
+                        if constexpr (EPI == EPI_GROUPS) {
+                            // a full log cannot be compacted here (it holds raw groups): the row is
+                            // flagged and recomputed by brute force after the merge
+                            if (st[h].wp > st[h].limit) {
+                                st[h].overflow = 1;
+                                st[h].wp = st[h].base;
+                            }
+                        }
                         if constexpr (kHasLog) {
                             if (__any_sync(0xFFFFFFFFu, st[h].cnt > p.cap - 32)) {
                                 __syncwarp();
@@ -639,6 +694,10 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                         for (int i = 0; i < kSampleM; ++i)
                             *reinterpret_cast<uint2*>(&log[i]) = make_uint2(__float_as_uint(st[h].net[i]), 0u);
                         p.part_meta[at] = make_int2(kSampleM, __float_as_int(INF));
+                    } else if constexpr (EPI == EPI_GROUPS) {
+                        const int recs = static_cast<int>((st[h].wp - st[h].base) / kRecordBytes);
+                        p.part_meta[at] = make_int2(st[h].overflow ? -1 : recs, __float_as_int(st[h].tau));
+                        if (p.stats) atomicAdd(&p.stats[1], static_cast<unsigned long long>(recs));
                     } else {
                         p.part_meta[at] = make_int2(st[h].cnt, __float_as_int(st[h].tau));
                         if (p.stats) atomicAdd(&p.stats[1], static_cast<unsigned long long>(st[h].cnt));

@@ -100,6 +100,7 @@ struct DeviceCtx {
     cudaEvent_t ev_free[2] = {nullptr, nullptr};
     cudaEvent_t ev_ready = nullptr;
     bool smem_attr_set = false;
+    bool merge_attr_set = false;
 };
 constexpr int kMaxDevices = 64;
 DeviceCtx g_ctx[kMaxDevices];
@@ -226,7 +227,8 @@ int make_plan(int64_t n, int nlist, int d, int k, int num_sms, Plan* pl, bool on
 // rows per launch so that the per-launch scratch stays bounded
 int64_t rows_per_launch(int d, int k) {
     const int kp = (d + 63) / 64 * 64 + kAugK;
-    const int64_t per_row = static_cast<int64_t>(kp) * 2 + 6ll * log_capacity(k) * 8 + (k > kSampleM ? 6ll * 512 * 8 : 0);
+    const int64_t per_row = static_cast<int64_t>(kp) * 2 +
+                            (k > kSampleM ? 6ll * (4 * k + 4) * kRecordBytes + 6ll * 512 * 8 : 6ll * log_capacity(k) * 8);
     int64_t rows = (int64_t(3) << 30) / per_row;
     rows = rows / (2 * kBlockM) * (2 * kBlockM);
     if (rows < 2 * kBlockM) rows = 2 * kBlockM;
@@ -380,6 +382,8 @@ int launch_fused(DeviceCtx& ctx, const Plan& pl, int64_t n, int nlist, int k, in
         CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_ARGMIN, 2>, attr, lim));
         CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_RUNNING, 1>, attr, lim));
         CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_FILTER, 1>, attr, lim));
+        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_GROUPS, 1>, attr, lim));
+        CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_GROUPS, 2>, attr, lim));
         CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_SKETCH, 1>, attr, lim));
         CUDA_TRY(cudaFuncSetAttribute(fused_topk_kernel<EPI_SKETCH, 2>, attr, lim));
         ctx.smem_attr_set = true;
@@ -395,6 +399,8 @@ int launch_fused(DeviceCtx& ctx, const Plan& pl, int64_t n, int nlist, int k, in
         IVF_LAUNCH(EPI_RUNNING, 1);
     } else if (rule == TAU_SKETCH) {
         if (two) IVF_LAUNCH(EPI_SKETCH, 2); else IVF_LAUNCH(EPI_SKETCH, 1);
+    } else if (rule == TAU_GIVEN) {
+        if (two) IVF_LAUNCH(EPI_GROUPS, 2); else IVF_LAUNCH(EPI_GROUPS, 1);
     } else {
         IVF_LAUNCH(EPI_FILTER, 1);
     }
@@ -424,6 +430,8 @@ MergeParams merge_params(const Plan& pl, int64_t n, int k, const Entry* part, co
     mp.fail = nullptr;
     mp.force_fail = 0;
     mp.tau_out = nullptr;
+    mp.records = 0;
+    mp.big = nullptr;
     mp.stats = nullptr;
     return mp;
 }
@@ -432,10 +440,12 @@ MergeParams merge_params(const Plan& pl, int64_t n, int k, const Entry* part, co
 int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int ptype, int nlist, int k,
                       const CentroidPrep& cp, int32_t* out_ids, float* out_dists, cudaStream_t stream) {
     Plan pl, pls;
-    int rc = make_plan(n, nlist, d, k, ctx.num_sms, &pl, k > 1);
+    int rc = make_plan(n, nlist, d, k, ctx.num_sms, &pl, k > 1 && cp.rule != TAU_GIVEN);
     if (rc != IVF_OK) return rc;
     const bool given = k > 1 && cp.rule == TAU_GIVEN;
-    size_t part_bytes = static_cast<size_t>(n) * pl.partials * pl.cap * sizeof(Entry);
+    // given rule: the logs hold 48-byte group records, at most 4k + 4 per (row, slot)
+    if (given) pl.cap = 4 * k + 4;
+    size_t part_bytes = static_cast<size_t>(n) * pl.partials * pl.cap * (given ? kRecordBytes : sizeof(Entry));
     size_t meta_bytes = static_cast<size_t>(n) * pl.partials * sizeof(int2);
     if (given) {
         rc = make_plan(n, cp.sample_rows, d, kSampleM, ctx.num_sms, &pls);
@@ -456,7 +466,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     WS(WS_PART, part_bytes, part);
     if (k > 1) {
         WS(WS_PARTMETA, meta_bytes, part_meta);
-        WS(WS_FAIL, (static_cast<size_t>(n) + 1) * sizeof(int), failbuf);
+        WS(WS_FAIL, 2 * (static_cast<size_t>(n) + 1) * sizeof(int), failbuf);  // failed rows, then passed-on rows
         if (given || g_force_fallback) WS(WS_FBKEYS, static_cast<size_t>(kFallbackFastRows + kFallbackCtas) * nlist * sizeof(float), fbkeys);
         if (given) WS(WS_TAU, static_cast<size_t>(n) * sizeof(float), tau);
     }
@@ -510,15 +520,38 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     mp.out_dists = out_dists;
     mp.fail = failbuf;
     mp.force_fail = g_force_fallback;
+    mp.records = given ? 1 : 0;
     mp.stats = g_stats ? ctx.stats : nullptr;
     tk = timing_begin(TK_MERGE, stream);
     if (k == 1) {
         merge_argmin_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(mp);
         LAUNCH_CHECK();
     } else {
+        // warp-per-row fast path first; rows it passes on (many partial logs, many candidates or
+        // ties) are listed in `big` and merged by the general CTA-per-row kernel
+        mp.big = failbuf + n + 1;
         CUDA_TRY(cudaMemsetAsync(failbuf, 0, sizeof(int), stream));
-        merge_select_kernel<<<static_cast<unsigned>(n), kMergeThreads, 0, stream>>>(mp);
-        LAUNCH_CHECK();
+        CUDA_TRY(cudaMemsetAsync(mp.big, 0, sizeof(int), stream));
+        if (!ctx.merge_attr_set) {
+            CUDA_TRY(cudaFuncSetAttribute(merge_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(kMergeWarps * sizeof(MergeWarpSmem))));
+            ctx.merge_attr_set = true;
+        }
+        // about 4k candidates per row pass a given threshold: beyond k = 128 they do not fit the
+        // warp-level buffers, so everything goes to the general kernel directly
+        const bool try_warp = !(given && 5 * k > kWarpKeys);
+        if (try_warp) {
+            merge_warp_kernel<<<static_cast<unsigned>((n + kMergeWarps - 1) / kMergeWarps), 32 * kMergeWarps,
+                                kMergeWarps * sizeof(MergeWarpSmem), stream>>>(mp);
+            LAUNCH_CHECK();
+        } else {
+            mp.big = nullptr;
+        }
+        {
+            const int64_t grid = n < 8 * static_cast<int64_t>(ctx.num_sms) ? n : 8 * static_cast<int64_t>(ctx.num_sms);
+            merge_select_kernel<<<static_cast<unsigned>(grid), kMergeThreads, 0, stream>>>(mp);
+            LAUNCH_CHECK();
+        }
         if (given || g_force_fallback) {
             FallbackParams fb;
             fb.nlist = nlist;
@@ -757,7 +790,8 @@ int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[
     if (n < 1 || nlist < 1 || num_sms < 1 || !out) return fail(IVF_ERR_INVALID_ARG, "bad plan arguments");
     if (d < 16 || d > 256 || d % 16 != 0) return fail(IVF_ERR_UNSUPPORTED, "d = %d", d);
     Plan pl;
-    int rc = make_plan(n, nlist, d, k, num_sms, &pl, k > 1);
+    int stride = 1;
+    int rc = make_plan(n, nlist, d, k, num_sms, &pl, k > 1 && choose_rule(k, nlist, &stride) != TAU_GIVEN);
     if (rc != IVF_OK) return rc;
     out[0] = pl.row_tiles;
     out[1] = pl.col_tiles;
@@ -774,7 +808,8 @@ int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[
 int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int64_t out[2]) {
     if (n < 1 || nlist < 1 || num_sms < 1 || !out) return fail(IVF_ERR_INVALID_ARG, "bad plan arguments");
     Plan pl;
-    int rc = make_plan(n, nlist, d, k, num_sms, &pl, k > 1);
+    int stride = 1;
+    int rc = make_plan(n, nlist, d, k, num_sms, &pl, k > 1 && choose_rule(k, nlist, &stride) != TAU_GIVEN);
     if (rc != IVF_OK) return rc;
     if (cta < 0 || cta >= pl.ctas) return fail(IVF_ERR_INVALID_ARG, "cta %d outside [0, %d)", cta, pl.ctas);
     out[0] = span_begin(pl.total_units, pl.ctas, cta);

@@ -32,6 +32,8 @@ struct MergeParams {
     int* fail;             // fail[0] = number of failed rows, fail[1..] = their indices
     int force_fail;        // test hook: treat every row as failed
     float* tau_out;        // if set: write only the 16th smallest key of every row here (threshold pass)
+    int records;           // the logs hold 48-byte group records (8 keys + first id), not entries
+    int* big;              // big[0] = number of rows the warp-level merge passed on, big[1..] = the rows
     unsigned long long* stats;  // optional counters: [2] rows sent to the brute-force recomputation
 };
 
@@ -85,109 +87,396 @@ __device__ __forceinline__ void bitonic_sort_smem(uint64_t* keys, int m /* power
 
 constexpr int kMaxSlots = 512;  // >= 2 * number of CTAs of the fused kernel
 
-// k > 1: one CTA per row.  The row's logs are read as one flattened array (all loads in flight
-// together); candidates <= the row's smallest tau are sorted by the 64-bit key (orderable value,
-// id) in shared memory; more than kSortCap raw entries are folded in rounds.
-__global__ void __launch_bounds__(kMergeThreads) merge_select_kernel(const MergeParams p) {
-    __shared__ uint64_t keys[kSortCap];
-    __shared__ int pre[kMaxSlots + 1];  // exclusive prefix of the slots' entry counts
-    __shared__ float s_tau[kMergeThreads / 32];
-    __shared__ int s_fill;
-    const int64_t row = blockIdx.x;
-    const int ns = min(slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows), kMaxSlots);
-    const Entry* base = p.part + static_cast<size_t>(row) * p.partials * p.cap;
-    const int2* meta = p.part_meta + static_cast<size_t>(row) * p.partials;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-
-    // ---- per-slot counts, their prefix sums, and the smallest threshold
-    float tau = __int_as_float(0x7f800000);
-    for (int s0 = 0; s0 < ns; s0 += kMergeThreads) {
-        const int sidx = s0 + threadIdx.x;
-        if (sidx < ns) {
-            const int2 m = meta[sidx];
-            pre[sidx + 1] = min(m.x, p.cap);
-            tau = fminf(tau, __int_as_float(m.y));
-        }
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) tau = fminf(tau, __shfl_xor_sync(0xFFFFFFFFu, tau, off));
-    if (lane == 0) s_tau[warp] = tau;
-    if (threadIdx.x == 0) {
-        pre[0] = 0;
-        s_fill = 0;
-    }
-    __syncthreads();
-    if (warp == 0) {  // inclusive scan of pre[1..ns] by one warp, 32 slots at a time
-        int carry = 0;
-        for (int s0 = 0; s0 < ns; s0 += 32) {
-            const int sidx = s0 + lane;
-            int v = sidx < ns ? pre[sidx + 1] : 0;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int t = __shfl_up_sync(0xFFFFFFFFu, v, off);
-                if (lane >= off) v += t;
-            }
-            if (sidx < ns) pre[sidx + 1] = v + carry;
-            carry += __shfl_sync(0xFFFFFFFFu, v, 31);
-        }
-    }
-    __syncthreads();
-    float tau_min = s_tau[0];
-#pragma unroll
-    for (int w = 1; w < kMergeThreads / 32; ++w) tau_min = fminf(tau_min, s_tau[w]);
-    const int raw_total = pre[ns];
-
-    int kept = 0;   // sorted keys carried at the front of keys[]
-    int total = 0;  // candidates <= tau_min seen so far
-    for (int done = 0; done < raw_total || done == 0;) {
-        const int room = kSortCap - kept;
-        const int take = min(raw_total - done, room);
-        for (int i = threadIdx.x; i < take; i += blockDim.x) {
-            const int idx = done + i;
-            int lo = 0, hi = ns;  // slot with pre[slot] <= idx < pre[slot + 1]
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (pre[mid] <= idx) lo = mid; else hi = mid;
-            }
-            const Entry e = base[static_cast<size_t>(lo) * p.cap + (idx - pre[lo])];
-            if (e.v <= tau_min)
-                keys[atomicAdd(&s_fill, 1)] = (static_cast<uint64_t>(orderable(e.v)) << 32) | static_cast<uint32_t>(e.j);
-        }
-        __syncthreads();
-        done += take;
-        const int fill = s_fill;
-        total += fill - kept;
-        int m = 2;
-        while (m < fill) m <<= 1;
-        for (int i = fill + threadIdx.x; i < m; i += blockDim.x) keys[i] = ~0ull;
-        bitonic_sort_smem(keys, m);
-        kept = min(fill, p.k);
-        if (done >= raw_total) break;
-        if (threadIdx.x == 0) s_fill = kept;
-        __syncthreads();
-    }
-    if (p.tau_out) {
-        if (threadIdx.x == 0)
-            p.tau_out[row] = kept >= kSampleM ? from_orderable(static_cast<uint32_t>(keys[kSampleM - 1] >> 32))
-                                              : __int_as_float(0x7f800000);
-        return;
-    }
-    if (total < p.k || p.force_fail) {
-        if (threadIdx.x == 0) {
-            const int at = atomicAdd(&p.fail[0], 1);
-            p.fail[1 + at] = static_cast<int>(row);
-            if (p.stats) atomicAdd(&p.stats[2], 1ull);
-        }
-        return;
-    }
+// Writes the first k sorted keys of a row (or hands the row to the brute-force path).
+__device__ __forceinline__ void merge_write_row(const MergeParams& p, int64_t row, const uint64_t* keys, int i0,
+                                                int istep) {
     const float xn = p.xn[row];
     const float inv = p.scal[2];
-    for (int i = threadIdx.x; i < p.k; i += blockDim.x) {
+    for (int i = i0; i < p.k; i += istep) {
         const uint64_t key = keys[i];
         p.out_ids[row * p.k + i] = static_cast<int32_t>(key & 0xFFFFFFFFull);
         if (p.out_dists)
             p.out_dists[row * p.k + i] = fmaxf(fmaf(from_orderable(static_cast<uint32_t>(key >> 32)), inv, xn), 0.0f);
     }
+}
+__device__ __forceinline__ void merge_fail_row(const MergeParams& p, int64_t row) {
+    const int at = atomicAdd(&p.fail[0], 1);
+    p.fail[1 + at] = static_cast<int>(row);
+    if (p.stats) atomicAdd(&p.stats[2], 1ull);
+}
+
+// k > 1, general path: one CTA per row.  The row's logs are read as one flattened array (all loads
+// in flight together); candidates <= the row's smallest tau are sorted by the 64-bit key (orderable
+// value, id) in shared memory; more than kSortCap raw entries are folded in rounds.  If p.big is
+// set the CTAs walk that list of rows (the rows the warp-level kernel passed on) instead of all.
+__global__ void __launch_bounds__(kMergeThreads) merge_select_kernel(const MergeParams p) {
+    __shared__ uint64_t keys[kSortCap];
+    __shared__ int pre[kMaxSlots + 1];  // exclusive prefix of the slots' entry counts
+    __shared__ float s_tau[kMergeThreads / 32];
+    __shared__ int hist[256];
+    __shared__ int s_wcnt[kMergeThreads / 32];
+    __shared__ int s_sel[2];
+    __shared__ int s_fill;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t nrows = p.big ? p.big[0] : p.n;
+    for (int64_t item = blockIdx.x; item < nrows; item += gridDim.x) {
+        const int64_t row = p.big ? p.big[1 + item] : item;
+        const int ns = min(slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows), kMaxSlots);
+        const Entry* base = p.part + static_cast<size_t>(row) * p.partials * p.cap;
+        const int2* meta = p.part_meta + static_cast<size_t>(row) * p.partials;
+        __syncthreads();  // the previous row of this CTA is finished with the shared arrays
+
+        // ---- per-slot counts, their prefix sums, and the smallest threshold
+        float tau = __int_as_float(0x7f800000);
+        int overflowed = 0;
+        for (int s0 = 0; s0 < ns; s0 += kMergeThreads) {
+            const int sidx = s0 + threadIdx.x;
+            if (sidx < ns) {
+                const int2 m = meta[sidx];
+                if (m.x < 0) overflowed = 1;  // a group log filled up: the row goes to the brute-force path
+                pre[sidx + 1] = max(0, min(m.x, p.cap));
+                tau = fminf(tau, __int_as_float(m.y));
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) tau = fminf(tau, __shfl_xor_sync(0xFFFFFFFFu, tau, off));
+        if (lane == 0) s_tau[warp] = tau;
+        if (threadIdx.x == 0) {
+            pre[0] = 0;
+            s_fill = 0;
+        }
+        __syncthreads();
+        if (warp == 0) {  // inclusive scan of pre[1..ns] by one warp, 32 slots at a time
+            int carry = 0;
+            for (int s0 = 0; s0 < ns; s0 += 32) {
+                const int sidx = s0 + lane;
+                int v = sidx < ns ? pre[sidx + 1] : 0;
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const int t = __shfl_up_sync(0xFFFFFFFFu, v, off);
+                    if (lane >= off) v += t;
+                }
+                if (sidx < ns) pre[sidx + 1] = v + carry;
+                carry += __shfl_sync(0xFFFFFFFFu, v, 31);
+            }
+        }
+        overflowed = __syncthreads_or(overflowed);
+        float tau_min = s_tau[0];
+#pragma unroll
+        for (int w = 1; w < kMergeThreads / 32; ++w) tau_min = fminf(tau_min, s_tau[w]);
+        const int raw_total = pre[ns];
+
+        int kept = 0;   // sorted keys carried at the front of keys[]
+        int total = 0;  // candidates <= tau_min seen so far
+        for (int done = 0; done < raw_total || done == 0;) {
+            // a record yields 8 candidates at most but about one in practice: take half as many
+            // records as there is room for keys; should a round still overflow, the row fails
+            const int room = (kSortCap - kept) / (p.records ? 2 : 1);
+            const int take = min(raw_total - done, room);
+            for (int i0 = 0; i0 < take; i0 += blockDim.x) {  // uniform trip count: ballots inside
+                const int i = i0 + threadIdx.x;
+                float v[8];
+                uint32_t j0 = 0;
+                int nv = 0;
+                if (i < take) {
+                    const int idx = done + i;
+                    int lo = 0, hi = ns;  // slot with pre[slot] <= idx < pre[slot + 1]
+                    while (hi - lo > 1) {
+                        const int mid = (lo + hi) >> 1;
+                        if (pre[mid] <= idx) lo = mid; else hi = mid;
+                    }
+                    if (p.records) {
+                        const char* rec = reinterpret_cast<const char*>(p.part) +
+                                          ((static_cast<size_t>(row) * p.partials + lo) * p.cap + (idx - pre[lo])) *
+                                              kRecordBytes;
+                        const float4 a = *reinterpret_cast<const float4*>(rec);
+                        const float4 b = *reinterpret_cast<const float4*>(rec + 16);
+                        j0 = *reinterpret_cast<const uint32_t*>(rec + 32);
+                        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+                        v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+                        nv = 8;
+                    } else {
+                        const Entry e = base[static_cast<size_t>(lo) * p.cap + (idx - pre[lo])];
+                        v[0] = e.v;
+                        j0 = static_cast<uint32_t>(e.j);
+                        nv = 1;
+                    }
+                }
+                // one shared-memory atomic per warp and column instead of one per candidate
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const bool hit = q < nv && v[q] <= tau_min;
+                    const uint32_t bal = __ballot_sync(0xFFFFFFFFu, hit);
+                    if (bal) {
+                        int at0 = 0;
+                        if (lane == 0) at0 = atomicAdd(&s_fill, __popc(bal));
+                        at0 = __shfl_sync(0xFFFFFFFFu, at0, 0);
+                        const int at = at0 + __popc(bal & ((1u << lane) - 1u));
+                        if (hit) {
+                            if (at < kSortCap) keys[at] = (static_cast<uint64_t>(orderable(v[q])) << 32) | (j0 + q);
+                            else overflowed = 1;
+                        }
+                    }
+                    if (!p.records) break;
+                }
+            }
+            __syncthreads();
+            done += take;
+            int fill = min(s_fill, kSortCap);
+            total += fill - kept;
+            if (fill > 2 * p.k) {
+                // only the k smallest matter: find the k-th smallest value (8-bit radix select over the
+                // keys' upper halves) and keep what is <= it, so that the sort below is short
+                uint32_t prefix = 0, mask = 0;
+                int rank = p.k;
+                for (int shift = 24; shift >= 0; shift -= 8) {
+                    for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+                    __syncthreads();
+                    for (int i = threadIdx.x; i < fill; i += blockDim.x) {
+                        const uint32_t u = static_cast<uint32_t>(keys[i] >> 32);
+                        if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & 255u], 1);
+                    }
+                    __syncthreads();
+                    if (warp == 0) {
+                        int r = rank, eq = 0;
+                        const int digit = radix_pick_digit(hist, lane, r, eq);
+                        if (lane == 0) {
+                            s_sel[0] = digit;
+                            s_sel[1] = r;
+                        }
+                    }
+                    __syncthreads();
+                    prefix |= static_cast<uint32_t>(s_sel[0]) << shift;
+                    mask |= 255u << shift;
+                    rank = s_sel[1];
+                }
+                // stable in-place compaction, 256 keys at a time
+                int outp = 0;
+                for (int i0 = 0; i0 < fill; i0 += blockDim.x) {
+                    const int i = i0 + threadIdx.x;
+                    uint64_t key = 0;
+                    bool keep = false;
+                    if (i < fill) {
+                        key = keys[i];
+                        keep = static_cast<uint32_t>(key >> 32) <= prefix;
+                    }
+                    const uint32_t bal = __ballot_sync(0xFFFFFFFFu, keep);
+                    if (lane == 0) s_wcnt[warp] = __popc(bal);
+                    __syncthreads();
+                    int before = 0, all = 0;
+#pragma unroll
+                    for (int w = 0; w < kMergeThreads / 32; ++w) {
+                        const int c = s_wcnt[w];
+                        if (w < warp) before += c;
+                        all += c;
+                    }
+                    if (keep) keys[outp + before + __popc(bal & ((1u << lane) - 1u))] = key;
+                    outp += all;
+                    __syncthreads();
+                }
+                fill = outp;
+            }
+            int m = 2;
+            while (m < fill) m <<= 1;
+            for (int i = fill + threadIdx.x; i < m; i += blockDim.x) keys[i] = ~0ull;
+            bitonic_sort_smem(keys, m);
+            kept = min(fill, p.k);
+            if (done >= raw_total) break;
+            if (threadIdx.x == 0) s_fill = kept;
+            __syncthreads();
+        }
+        overflowed = __syncthreads_or(overflowed);
+        if (p.tau_out) {
+            if (threadIdx.x == 0)
+                p.tau_out[row] = kept >= kSampleM ? from_orderable(static_cast<uint32_t>(keys[kSampleM - 1] >> 32))
+                                                  : __int_as_float(0x7f800000);
+            continue;
+        }
+        if (total < p.k || p.force_fail || overflowed) {
+            if (threadIdx.x == 0) merge_fail_row(p, row);
+            continue;
+        }
+        merge_write_row(p, row, keys, threadIdx.x, blockDim.x);
+    }
+}
+
+// k > 1, fast path: one WARP per row, no block-wide barriers.  Serves rows with at most kWarpSlots
+// partial logs and at most kWarpKeys candidates <= tau: the candidates go to the warp's slice of
+// shared memory, an 8-bit radix select on the key's value finds the k-th smallest, and only the
+// keys up to it are sorted.  Other rows are appended to p.big for merge_select_kernel.
+constexpr int kWarpKeys = 1024;
+constexpr int kWarpSlots = 64;
+constexpr int kWarpSort = 512;
+constexpr int kMergeWarps = 8;
+
+struct MergeWarpSmem {
+    uint64_t keys[kWarpKeys];
+    int hist[256];
+    int pre[kWarpSlots + 1];
+};
+
+__device__ __forceinline__ void warp_bitonic_sort(uint64_t* keys, int m, int lane) {
+    for (int size = 2; size <= m; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            __syncwarp();
+            for (int t = lane; t < (m >> 1); t += 32) {
+                const int lo = 2 * t - (t & (stride - 1));
+                const int hi = lo + stride;
+                const bool up = (lo & size) == 0;
+                const uint64_t a = keys[lo], b = keys[hi];
+                if ((a > b) == up) {
+                    keys[lo] = b;
+                    keys[hi] = a;
+                }
+            }
+        }
+    }
+    __syncwarp();
+}
+
+__global__ void __launch_bounds__(32 * kMergeWarps) merge_warp_kernel(const MergeParams p) {
+    extern __shared__ __align__(16) uint8_t merge_smem_raw[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    MergeWarpSmem& sm = reinterpret_cast<MergeWarpSmem*>(merge_smem_raw)[warp];
+    const int64_t row = static_cast<int64_t>(blockIdx.x) * kMergeWarps + warp;
+    if (row >= p.n) return;
+    const uint32_t FULL = 0xFFFFFFFFu;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows);
+    const int2* meta = p.part_meta + static_cast<size_t>(row) * p.partials;
+    bool pass_on = ns > kWarpSlots || p.force_fail;
+
+    // ---- slot counts, prefix sums, smallest threshold
+    float tau_min = __int_as_float(0x7f800000);
+    int raw_total = 0;
+    if (!pass_on) {
+        int carry = 0;
+        for (int s0 = 0; s0 < ns; s0 += 32) {
+            const int sidx = s0 + lane;
+            int c = 0;
+            if (sidx < ns) {
+                const int2 m = meta[sidx];
+                if (m.x < 0) pass_on = true;
+                c = max(0, min(m.x, p.cap));
+                tau_min = fminf(tau_min, __int_as_float(m.y));
+            }
+            int v = c;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int t = __shfl_up_sync(FULL, v, off);
+                if (lane >= off) v += t;
+            }
+            if (sidx < ns) sm.pre[sidx + 1] = v + carry;
+            carry += __shfl_sync(FULL, v, 31);
+        }
+        if (lane == 0) sm.pre[0] = 0;
+        raw_total = carry;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) tau_min = fminf(tau_min, __shfl_xor_sync(FULL, tau_min, off));
+        pass_on = __any_sync(FULL, pass_on);
+        __syncwarp();
+    }
+
+    // ---- gather the candidates <= tau_min into the warp's key buffer
+    int fill = 0;
+    if (!pass_on) {
+        for (int i0 = 0; i0 < raw_total && !pass_on; i0 += 32) {
+            const int idx = i0 + lane;
+            float v[8];
+            uint32_t j0 = 0;
+            int nv = 0;
+            if (idx < raw_total) {
+                int lo = 0, hi = ns;
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (sm.pre[mid] <= idx) lo = mid; else hi = mid;
+                }
+                const size_t at = (static_cast<size_t>(row) * p.partials + lo) * p.cap + (idx - sm.pre[lo]);
+                if (p.records) {
+                    const char* rec = reinterpret_cast<const char*>(p.part) + at * kRecordBytes;
+                    const float4 a = *reinterpret_cast<const float4*>(rec);
+                    const float4 b = *reinterpret_cast<const float4*>(rec + 16);
+                    j0 = *reinterpret_cast<const uint32_t*>(rec + 32);
+                    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+                    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+                    nv = 8;
+                } else {
+                    const Entry e = p.part[at];
+                    v[0] = e.v;
+                    j0 = static_cast<uint32_t>(e.j);
+                    nv = 1;
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const bool hit = q < nv && v[q] <= tau_min;
+                const uint32_t bal = __ballot_sync(FULL, hit);
+                if (bal) {
+                    const int at = fill + __popc(bal & lt_mask);
+                    if (hit && at < kWarpKeys) sm.keys[at] = (static_cast<uint64_t>(orderable(v[q])) << 32) | (j0 + q);
+                    fill += __popc(bal);
+                }
+                if (!p.records) break;
+            }
+            if (fill > kWarpKeys) pass_on = true;
+        }
+        __syncwarp();
+    }
+    if (!pass_on && fill < p.k) {  // too few candidates: the threshold was too tight for this row
+        if (lane == 0) merge_fail_row(p, row);
+        return;
+    }
+
+    // ---- k-th smallest value by radix select, then keep everything up to it
+    int kept = fill;
+    if (!pass_on && fill > 2 * p.k) {
+        uint32_t prefix = 0, mask = 0;
+        int r = p.k, eq = 0;
+#pragma unroll 1
+        for (int shift = 24; shift >= 0; shift -= 8) {
+            for (int i = lane; i < 256; i += 32) sm.hist[i] = 0;
+            __syncwarp();
+            for (int i = lane; i < fill; i += 32) {
+                const uint32_t u = static_cast<uint32_t>(sm.keys[i] >> 32);
+                if ((u & mask) == prefix) atomicAdd(&sm.hist[(u >> shift) & 255u], 1);
+            }
+            __syncwarp();
+            const int digit = radix_pick_digit(sm.hist, lane, r, eq);
+            prefix |= static_cast<uint32_t>(digit) << shift;
+            mask |= 255u << shift;
+            __syncwarp();
+        }
+        // compact the keys whose value is <= the k-th smallest to the front (ties all stay)
+        int outp = 0;
+        for (int i0 = 0; i0 < fill; i0 += 32) {
+            const int i = i0 + lane;
+            uint64_t key = 0;
+            bool keep = false;
+            if (i < fill) {
+                key = sm.keys[i];
+                keep = static_cast<uint32_t>(key >> 32) <= prefix;
+            }
+            const uint32_t bal = __ballot_sync(FULL, keep);
+            __syncwarp();
+            if (keep) sm.keys[outp + __popc(bal & lt_mask)] = key;
+            outp += __popc(bal);
+        }
+        __syncwarp();
+        kept = outp;
+    }
+    if (!pass_on && kept > kWarpSort) pass_on = true;  // very many ties: let the general path sort
+    if (pass_on) {
+        if (lane == 0) {
+            const int at = atomicAdd(&p.big[0], 1);
+            p.big[1 + at] = static_cast<int>(row);
+        }
+        return;
+    }
+    int m = 2;
+    while (m < kept) m <<= 1;
+    for (int i = kept + lane; i < m; i += 32) sm.keys[i] = ~0ull;
+    warp_bitonic_sort(sm.keys, m, lane);
+    merge_write_row(p, row, sm.keys, lane, 32);
 }
 
 // Threshold pass: one warp per row reads the partial sketches (16 smallest group minima per
