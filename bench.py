@@ -39,10 +39,12 @@ WORKLOAD = ("C1 SIFT-shaped routing (10000 u8 queries x 65536 f32 centroids, d=1
 METRIC = "routed queries/s"
 UNIT = "queries/s"
 
-# DRAM bytes (read + write) per launch of the dominant kernel from the ncu capture summarised in
-# profiles/; None until a capture exists.
-TRAFFIC_FUSED_ARGMIN_BYTES = None
-TRAFFIC_FUSED_TOPK_BYTES = None
+# DRAM bytes (read + write) per launch from the ncu captures summarised in profiles/.
+# k = 1 kernel: captured at 262,144 rows (115.6 MB, profiles/fused_argmin_262144x65536x128.md) and
+# scaled by 4 to the bench's 1,048,576-row launch (an upper bound: the centroid copy does not grow).
+TRAFFIC_FUSED_ARGMIN_BYTES = 4 * (107.677952e6 + 7.954176e6)
+# k = 64 kernel: captured at the bench's own size (profiles/fused_groups_routing_c1_c2.md).
+TRAFFIC_FUSED_TOPK_BYTES = 96.510720e6 + 104.337664e6
 
 
 def peaks():
@@ -271,6 +273,28 @@ def main():
     t_e2e = float(t_e2e.cpu()[0])
     B.ivf_check(dev)
 
+    # ---- the same for the assignment chunk: rows streamed from page-locked host memory, ids read back
+    chunk_host = torch.from_numpy(chunk_np).pin_memory()
+    a_ids_host = torch.empty((CHUNK,), dtype=torch.int32).pin_memory()
+    ea0, ea1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sums.zero_()
+    counts.zero_()
+    B.ivf_assign_update(chunk_host, cent_route, sums, counts, a_ids, None)
+    barrier()
+    ea0.record()
+    for _ in range(args.steps):
+        sums.zero_()
+        counts.zero_()
+        B.ivf_assign_update(chunk_host, cent_route, sums, counts, a_ids, None)
+        a_ids_host.copy_(a_ids, non_blocking=True)
+    ea1.record()
+    barrier()
+    t_e2e_a = torch.tensor([ea0.elapsed_time(ea1)], dtype=torch.float64, device=dev)
+    if distributed:
+        dist.all_reduce(t_e2e_a, op=dist.ReduceOp.MAX)
+    t_e2e_a = float(t_e2e_a.cpu()[0])
+    B.ivf_check(dev)
+
     if rank != 0:
         if distributed:
             dist.destroy_process_group()
@@ -318,6 +342,9 @@ def main():
                             "traffic": None, "peak_source": pk["source"]},
         "e2e": {"value": world * NQ * K / (t_e2e / 1e3), "unit": UNIT, "h2d_bytes_per_step": NQ * D,
                 "d2h_bytes_per_step": NQ * NPROBE * 8},
+        "e2e_assign": {"value": world * CHUNK * K / (t_e2e_a / 1e3), "unit": "vectors/s",
+                       "h2d_bytes_per_step": CHUNK * D, "d2h_bytes_per_step": CHUNK * 4,
+                       "host_link_GBps": CHUNK * D * K / (t_e2e_a / 1e3) / 1e9},
         "gpu_launches": int(launches),
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                    "samples": clocks["samples"]},
@@ -327,7 +354,12 @@ def main():
     if not args.no_cpu_baseline and world == 1:
         from oracle import oracle
         cores = oracle.num_threads()
-        rows = max(64, 48 * cores)
+        # size the sample for about 15 s of CPU work from a short probe
+        probe = np.ascontiguousarray(queries_np[:8 * cores])
+        t0 = time.perf_counter()
+        oracle.route(probe, cent_np, NPROBE)
+        rate = probe.shape[0] / (time.perf_counter() - t0)
+        rows = int(min(NQ, max(64, rate * 15.0)))
         sel = np.random.default_rng(1).choice(NQ, rows, replace=False)
         sample = np.ascontiguousarray(queries_np[sel])
         t0 = time.perf_counter()

@@ -581,7 +581,9 @@ int update_device(DeviceCtx& ctx, const void* points, int ptype, const int32_t* 
                   float* sums, int64_t* counts, cudaStream_t stream) {
     int *cnt, *off, *cur, *perm;
     WS(WS_UCNT, static_cast<size_t>(nlist) * sizeof(int), cnt);
-    WS(WS_UOFF, (static_cast<size_t>(nlist) + 1) * sizeof(int), off);
+    const int scan_blocks = (nlist + kScanBlock - 1) / kScanBlock;
+    WS(WS_UOFF, (static_cast<size_t>(nlist) + 1 + scan_blocks) * sizeof(int), off);
+    int* block_sums = off + nlist + 1;
     WS(WS_UCUR, static_cast<size_t>(nlist) * sizeof(int), cur);
     WS(WS_UPERM, static_cast<size_t>(n) * sizeof(int), perm);
     const int tk = timing_begin(TK_UPDATE, stream);
@@ -589,7 +591,9 @@ int update_device(DeviceCtx& ctx, const void* points, int ptype, const int32_t* 
     const unsigned rb = static_cast<unsigned>((n + 255) / 256);
     update_hist_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, cnt, ctx.status);
     LAUNCH_CHECK();
-    update_scan_kernel<<<1, 1024, 0, stream>>>(cnt, nlist, off, cur);
+    update_scan_local_kernel<<<scan_blocks, 1024, 0, stream>>>(cnt, nlist, off, block_sums);
+    LAUNCH_CHECK();
+    update_scan_fix_kernel<<<scan_blocks, 1024, 0, stream>>>(nlist, off, block_sums, cur);
     LAUNCH_CHECK();
     update_fill_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, off, cur, perm);
     LAUNCH_CHECK();
@@ -898,12 +902,14 @@ int ivf_debug_set_wait_limit_ns(int64_t ns) {
 //   [0, 8)                         header: [0] = "an id was out of range" flag of the last call
 //   [8, 8 + L)                     per-list member counts of the call        (L = kNoAllocMaxLists)
 //   [8 + L, 8 + 2L + 1)            exclusive offsets of the list segments
-//   [8 + 2L + 8, 8 + 3L + 8)       per-list fill cursors
-//   [8 + 3L + 8, ... + R)          row permutation sorted by list             (R = kNoAllocMaxRows)
+//   [8 + 2L + 8, 8 + 2L + 40)      partial totals of the offset scan (one per 4096 lists)
+//   [8 + 2L + 40, 8 + 3L + 40)     per-list fill cursors
+//   [8 + 3L + 40, ... + R)         row permutation sorted by list             (R = kNoAllocMaxRows)
 namespace {
 constexpr int kNoAllocMaxLists = 65536;
 constexpr int kNoAllocMaxRows = 1 << 20;
-constexpr size_t kNoAllocInts = 8 + 3 * static_cast<size_t>(kNoAllocMaxLists) + 8 + kNoAllocMaxRows;
+constexpr size_t kNoAllocInts = 8 + 3 * static_cast<size_t>(kNoAllocMaxLists) + 40 + kNoAllocMaxRows;
+static_assert(kNoAllocMaxLists / kScanBlock <= 32, "scan totals must fit their slot");
 static __device__ __align__(256) int g_noalloc_scratch[kNoAllocInts];
 // device address of the array above, per device (the host-side symbol is not a device pointer)
 int* g_noalloc_ptr[kMaxDevices] = {};
@@ -949,7 +955,8 @@ extern "C" int ivf_centroid_update_noalloc(const void* points, ivf_dtype ptype, 
     int* flag = base;
     int* cnt = base + 8;
     int* off = cnt + kNoAllocMaxLists;
-    int* cur = off + kNoAllocMaxLists + 8;
+    int* block_sums = off + kNoAllocMaxLists + 8;
+    int* cur = block_sums + 32;
     int* perm = cur + kNoAllocMaxLists;
 
     // the array keeps the previous call's contents: the counts and the flag must start at zero
@@ -959,7 +966,10 @@ extern "C" int ivf_centroid_update_noalloc(const void* points, ivf_dtype ptype, 
     const unsigned rb = static_cast<unsigned>((n + 255) / 256);
     update_hist_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, cnt, flag);
     LAUNCH_CHECK();
-    update_scan_kernel<<<1, 1024, 0, stream>>>(cnt, nlist, off, cur);
+    const int scan_blocks = (nlist + kScanBlock - 1) / kScanBlock;
+    update_scan_local_kernel<<<scan_blocks, 1024, 0, stream>>>(cnt, nlist, off, block_sums);
+    LAUNCH_CHECK();
+    update_scan_fix_kernel<<<scan_blocks, 1024, 0, stream>>>(nlist, off, block_sums, cur);
     LAUNCH_CHECK();
     update_fill_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, off, cur, perm);
     LAUNCH_CHECK();

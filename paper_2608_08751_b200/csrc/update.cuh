@@ -22,58 +22,74 @@ __global__ void update_hist_kernel(const int32_t* __restrict__ ids, int64_t n, i
     atomicAdd(&cnt[l], 1);
 }
 
-// Exclusive scan of cnt[0..nlist) into off[0..nlist]; single CTA of 1024 threads walking the array
-// in blocks of 4096 with a running carry.  Also clears cursor[].
-__global__ void __launch_bounds__(1024) update_scan_kernel(const int* __restrict__ cnt, int nlist,
-                                                           int* __restrict__ off, int* __restrict__ cursor) {
+// Exclusive scan of cnt[0..nlist) into off[0..nlist] in two small kernels.  First every CTA scans
+// its own 4096 counts and publishes their total; then every CTA adds the totals of the CTAs before
+// it (at most a few hundred values) to its slice, and clears the fill cursors.
+constexpr int kScanBlock = 4096;
+
+__global__ void __launch_bounds__(1024) update_scan_local_kernel(const int* __restrict__ cnt, int nlist,
+                                                                 int* __restrict__ off, int* __restrict__ block_sums) {
     __shared__ int warp_sums[32];
-    __shared__ int carry_s;
-    if (threadIdx.x == 0) carry_s = 0;
-    __syncthreads();
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    for (int base = 0; base < nlist; base += 4096) {
-        const int i0 = base + threadIdx.x * 4;
-        int v[4];
-        int tsum = 0;
+    const int i0 = blockIdx.x * kScanBlock + threadIdx.x * 4;
+    int v[4];
+    int tsum = 0;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            v[q] = (i0 + q < nlist) ? cnt[i0 + q] : 0;
-            tsum += v[q];
-        }
-        int incl = tsum;
+    for (int q = 0; q < 4; ++q) {
+        v[q] = (i0 + q < nlist) ? cnt[i0 + q] : 0;
+        tsum += v[q];
+    }
+    int incl = tsum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) warp_sums[w] = incl;
+    __syncthreads();
+    if (w == 0) {
+        const int ws = warp_sums[lane];
+        int wi = ws;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-            if (lane >= o) incl += t;
+            const int t = __shfl_up_sync(0xFFFFFFFFu, wi, o);
+            if (lane >= o) wi += t;
         }
-        if (lane == 31) warp_sums[w] = incl;
-        __syncthreads();
-        if (w == 0) {
-            int ws = warp_sums[lane];
-            int wi = ws;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int t = __shfl_up_sync(0xFFFFFFFFu, wi, o);
-                if (lane >= o) wi += t;
-            }
-            warp_sums[lane] = wi - ws;  // exclusive prefix of the warp sums
-        }
-        __syncthreads();
-        const int carry = carry_s;
-        int run = carry + warp_sums[w] + (incl - tsum);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            if (i0 + q < nlist) {
-                off[i0 + q] = run;
-                cursor[i0 + q] = 0;
-            }
-            run += v[q];
-        }
-        __syncthreads();
-        if (threadIdx.x == 1023) carry_s = run;  // last thread's running total = carry for the next block
-        __syncthreads();
+        warp_sums[lane] = wi - ws;  // exclusive prefix of the warp sums
+        if (lane == 31) block_sums[blockIdx.x] = wi;
     }
-    if (threadIdx.x == 0) off[nlist] = carry_s;
+    __syncthreads();
+    int run = warp_sums[w] + (incl - tsum);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        if (i0 + q < nlist) off[i0 + q] = run;
+        run += v[q];
+    }
+}
+
+__global__ void __launch_bounds__(1024) update_scan_fix_kernel(int nlist, int* __restrict__ off,
+                                                               const int* __restrict__ block_sums,
+                                                               int* __restrict__ cursor) {
+    __shared__ int s_part[32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int acc = 0;
+    for (int b = threadIdx.x; b < static_cast<int>(blockIdx.x); b += blockDim.x) acc += block_sums[b];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    if (lane == 0) s_part[w] = acc;
+    __syncthreads();
+    int before = 0;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) before += s_part[i];
+    const int i0 = blockIdx.x * kScanBlock + threadIdx.x * 4;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        if (i0 + q < nlist) {
+            off[i0 + q] += before;
+            cursor[i0 + q] = 0;
+        }
+    }
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) off[nlist] = before + block_sums[blockIdx.x];
 }
 
 __global__ void update_fill_kernel(const int32_t* __restrict__ ids, int64_t n, int nlist,
@@ -100,24 +116,39 @@ __global__ void update_reduce_kernel(const T* __restrict__ x, const int* __restr
     for (int m0 = beg; m0 < end; m0 += 32) {
         const int mine = (m0 + lane < end) ? perm[m0 + lane] : -1;
         const int cntm = min(32, end - m0);
-        for (int m = 0; m < cntm; ++m) {
-            const int64_t row = __shfl_sync(0xFFFFFFFFu, mine, m);
+        for (int m = 0; m < cntm; m += 4) {  // four member rows in flight
+            int64_t rows[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) rows[u] = __shfl_sync(0xFFFFFFFFu, mine, (m + u) & 31);
 #pragma unroll
             for (int blk = 0; blk < 2; ++blk) {
                 const int c0 = 128 * blk + 4 * lane;
                 if (c0 < d) {
                     if constexpr (sizeof(T) == 1) {
-                        const uint32_t w = *reinterpret_cast<const uint32_t*>(x + row * d + c0);
-                        acc[blk][0] += static_cast<float>(w & 0xFFu);
-                        acc[blk][1] += static_cast<float>((w >> 8) & 0xFFu);
-                        acc[blk][2] += static_cast<float>((w >> 16) & 0xFFu);
-                        acc[blk][3] += static_cast<float>(w >> 24);
+                        uint32_t wv[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            wv[u] = (m + u < cntm) ? *reinterpret_cast<const uint32_t*>(x + rows[u] * d + c0) : 0u;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            acc[blk][0] += static_cast<float>(wv[u] & 0xFFu);
+                            acc[blk][1] += static_cast<float>((wv[u] >> 8) & 0xFFu);
+                            acc[blk][2] += static_cast<float>((wv[u] >> 16) & 0xFFu);
+                            acc[blk][3] += static_cast<float>(wv[u] >> 24);
+                        }
                     } else {
-                        const float4 v = *reinterpret_cast<const float4*>(x + row * d + c0);
-                        acc[blk][0] += v.x;
-                        acc[blk][1] += v.y;
-                        acc[blk][2] += v.z;
-                        acc[blk][3] += v.w;
+                        float4 fv[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            fv[u] = (m + u < cntm) ? *reinterpret_cast<const float4*>(x + rows[u] * d + c0)
+                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            acc[blk][0] += fv[u].x;
+                            acc[blk][1] += fv[u].y;
+                            acc[blk][2] += fv[u].z;
+                            acc[blk][3] += fv[u].w;
+                        }
                     }
                 }
             }

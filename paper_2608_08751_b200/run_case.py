@@ -4,6 +4,9 @@ A small driver for profilers and quick measurements:
     python -m paper_2608_08751_b200.run_case --op assign --n 262144 --nlist 65536 --d 128 --dtype u8 --reps 3
     python -m paper_2608_08751_b200.run_case --op route --n 10000 --nlist 65536 --k 64
     python -m paper_2608_08751_b200.run_case --op update --n 1048576 --nlist 65536
+    python -m paper_2608_08751_b200.run_case --op stream --n 8388608 --nlist 65536 --iters 2
+"stream" is the IVF-build configuration in small: rows in page-locked host memory, streamed in
+1,048,576-row chunks through assign + update, then the finalize, per Lloyd iteration.
 Inputs follow the SIFT-shaped (uint8, all-positive mixture) or DEEP-shaped (float32, unit norm)
 recipes of ``synth``.
 """
@@ -19,9 +22,52 @@ from . import binding as B
 from . import synth
 
 
+def stream_case(args):
+    chunk = synth.CHUNK_ROWS
+    nchunks = -(-args.n // chunk)
+    host = torch.empty((args.n, args.d), dtype=torch.uint8 if args.dtype == "u8" else torch.float32).pin_memory()
+    for c in range(nchunks):  # the same seeded chunk recipe as the full configuration
+        rows = min(chunk, args.n - c * chunk)
+        if args.dtype == "u8":
+            blk = synth.sift_like_rows(c, rows=rows, d=args.d)
+        else:
+            blk = synth.deep_like_rows(c, rows=rows, d=args.d)
+        host[c * chunk:c * chunk + rows] = torch.from_numpy(blk)
+    init = synth.init_sample(args.n, args.nlist)
+    cent = host[torch.from_numpy(init)].to(torch.float32).cuda()
+    sums = torch.zeros((args.nlist, args.d), dtype=torch.float32, device="cuda")
+    counts = torch.zeros((args.nlist,), dtype=torch.int64, device="cuda")
+    ids = torch.empty((args.n,), dtype=torch.int32, device="cuda")
+    dists = torch.empty((args.n,), dtype=torch.float32, device="cuda")
+
+    def iteration():
+        sums.zero_()
+        counts.zero_()
+        B.ivf_assign_update(host, cent, sums, counts, ids, dists)
+        B.ivf_centroid_finalize(sums, counts, cent)
+
+    iteration()  # warm-up (workspace growth)
+    B.ivf_check()
+    inertia = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.iters):
+        iteration()
+        inertia.append(float(dists.double().sum().item()))
+    e1.record()
+    B.ivf_check()
+    ms = e0.elapsed_time(e1) / args.iters
+    esize = 1 if args.dtype == "u8" else 4
+    print(json.dumps({"op": "stream", "n": args.n, "nlist": args.nlist, "d": args.d, "dtype": args.dtype,
+                      "chunks": nchunks, "ms_per_iteration": ms, "vectors_per_s": args.n / (ms / 1e3),
+                      "host_link_GBps": args.n * args.d * esize / (ms / 1e3) / 1e9,
+                      "tflops": 2.0 * args.n * args.nlist * args.d / (ms / 1e3) / 1e12, "inertia": inertia}))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="assign", choices=["assign", "route", "update"])
+    ap.add_argument("--op", default="assign", choices=["assign", "route", "update", "stream"])
+    ap.add_argument("--iters", type=int, default=1, help="Lloyd iterations of --op stream")
     ap.add_argument("--n", type=int, default=262144)
     ap.add_argument("--nlist", type=int, default=65536)
     ap.add_argument("--d", type=int, default=128)
@@ -30,6 +76,8 @@ def main():
     ap.add_argument("--reps", type=int, default=3)
     args = ap.parse_args()
 
+    if args.op == "stream":
+        return stream_case(args)
     if args.dtype == "u8":
         x = synth.sift_like_rows(0, rows=args.n, d=args.d)
         c = synth.sift_like_centroids(args.nlist, args.d)
