@@ -120,6 +120,21 @@ int ivf_centroid_finalize(const float* sums, const int64_t* counts, int nlist, i
                           float* centroids_inout, void* stream);
 
 /*
+ * Cluster-major layout (Sec. 3.1 index layout: the vectors of a list are stored contiguously, with
+ * per-list offset, length and ids), the step right after the final assignment of an index build.
+ *   points       [n, d] (ptype), ids [n] int32: device
+ *   out_offsets  [nlist + 1] int64, device: list l occupies rows [out_offsets[l], out_offsets[l+1])
+ *   out_order    [n] int32, device: out_order[p] = source row stored at position p
+ *   out_points   [n, d] (ptype), device: row p = points[out_order[p]]
+ * The order of the rows inside a list is unspecified (every order is a valid layout; out_order tells
+ * which one was taken).  A row whose id is outside [0, nlist) is dropped from the layout and flags
+ * IVF_ERR_BAD_ID in the status word.  At most 2^31 - 1 rows per call.
+ */
+int ivf_cluster_major_reorder(const void* points, ivf_dtype ptype, const int32_t* ids, int64_t n, int d,
+                              int nlist, void* out_points, int64_t* out_offsets, int32_t* out_order,
+                              void* stream);
+
+/*
  * Helper: one pass of a Lloyd iteration over a point set that may exceed device memory
  * (Table 3: assignment in batches of 1,048,576 vectors; Table 1: the host link is the scarce
  * resource).  For each chunk of `chunk_rows` rows: copy to the device if `points` is page-locked

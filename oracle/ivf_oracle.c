@@ -25,7 +25,7 @@
  * Pins (tests/test_oracle_pins.py): hand-computed tiny cases, one-hot closed form,
  * unit-norm identity, scipy cdist, brute force over all k-subsets, lexsort,
  * permutation / translation / scaling invariants, bincount cross-check, Lloyd
- * monotonicity and toy clusters.  No function here is unpinned.
+ * monotonicity and toy clusters, numpy stable argsort for the reorder.  No function here is unpinned.
  */
 #include <math.h>
 #include <stdint.h>
@@ -155,6 +155,28 @@ int oracle_update(const void *x, int xtype, const int32_t *ids, int64_t n, int d
         counts[l] += 1;
     }
     return bad ? -1 : 0;
+}
+
+/*
+ * Cluster-major layout (Sec. 3.1 index layout: the vectors of one list are stored contiguously,
+ * with per-list offset / length / ids).  Stable counting sort written out:
+ *   offsets[l]  = number of rows whose id is smaller than l          (offsets[nlist] = n)
+ *   order[p]    = source row stored at position p; within a list the rows keep their input order
+ * Returns -1 if an id is out of range.
+ */
+int oracle_reorder(const int32_t *ids, int64_t n, int32_t nlist, int64_t *offsets, int64_t *order) {
+    for (int32_t l = 0; l <= nlist; ++l) offsets[l] = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (ids[i] < 0 || ids[i] >= nlist) return -1;
+        offsets[ids[i] + 1] += 1;
+    }
+    for (int32_t l = 0; l < nlist; ++l) offsets[l + 1] += offsets[l];
+    int64_t *cursor = (int64_t *)malloc(sizeof(int64_t) * (size_t)(nlist > 0 ? nlist : 1));
+    if (!cursor) return -1;
+    for (int32_t l = 0; l < nlist; ++l) cursor[l] = offsets[l];
+    for (int64_t i = 0; i < n; ++i) order[cursor[ids[i]]++] = i;
+    free(cursor);
+    return 0;
 }
 
 /* Mean per list, rounded once to float; an empty list keeps its previous centroid. */

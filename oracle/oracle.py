@@ -41,6 +41,7 @@ def _load():
         _lib.oracle_sqnorms.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, vp]
         _lib.oracle_update.argtypes = [vp, ctypes.c_int, vp, i64, ctypes.c_int, i32, vp, vp]
         _lib.oracle_finalize.argtypes = [vp, vp, i32, ctypes.c_int, vp]
+        _lib.oracle_reorder.argtypes = [vp, i64, i32, vp, vp]
         _lib.oracle_lloyd.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, i32, ctypes.c_int, vp, vp, vp]
         _lib.oracle_num_threads.restype = ctypes.c_int
     return _lib
@@ -131,6 +132,17 @@ def update(x: np.ndarray, ids: np.ndarray, nlist: int, sums: np.ndarray | None =
     assert sums.dtype == np.float64 and counts.dtype == np.int64 and sums.flags.c_contiguous
     rc = _load().oracle_update(_p(x), xt, _p(ids), n, d, nlist, _p(sums), _p(counts))
     return sums, counts, rc == 0
+
+
+def reorder(ids: np.ndarray, nlist: int):
+    """(offsets int64 [nlist+1], order int64 [n]): cluster-major layout, input order kept inside a list."""
+    ids = np.ascontiguousarray(ids, np.int32)
+    offsets = np.empty((nlist + 1,), np.int64)
+    order = np.empty((ids.shape[0],), np.int64)
+    rc = _load().oracle_reorder(_p(ids), ids.shape[0], nlist, _p(offsets), _p(order))
+    if rc != 0:
+        raise ValueError("oracle_reorder: id out of range")
+    return offsets, order
 
 
 def finalize(sums: np.ndarray, counts: np.ndarray, centroids: np.ndarray) -> np.ndarray:

@@ -21,7 +21,7 @@ IVF_ERR_CUDA, IVF_ERR_DEVICE_TIMEOUT, IVF_ERR_BAD_ID = -4, -5, -6
 
 EXPORTS = (
     "ivf_route", "ivf_assign", "ivf_centroid_update", "ivf_centroid_update_noalloc", "ivf_centroid_finalize",
-    "ivf_assign_update",
+    "ivf_assign_update", "ivf_cluster_major_reorder",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
     "ivf_debug_plan", "ivf_debug_span", "ivf_debug_set_wait_limit_ns",
     "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_stats",
@@ -55,6 +55,7 @@ def lib() -> ctypes.CDLL:
     L.ivf_centroid_update.argtypes = [vp, i32, vp, i64, i32, i32, vp, vp, vp]
     L.ivf_centroid_update_noalloc.argtypes = [vp, i32, vp, i64, i32, i32, vp, vp, vp]
     L.ivf_centroid_finalize.argtypes = [vp, vp, i32, i32, vp, vp]
+    L.ivf_cluster_major_reorder.argtypes = [vp, i32, vp, i64, i32, i32, vp, vp, vp, vp]
     L.ivf_assign_update.argtypes = [vp, i64, i32, i32, vp, i32, vp, vp, vp, vp, i64, vp]
     L.ivf_check.argtypes = [vp]
     L.ivf_last_error.restype = ctypes.c_char_p
@@ -193,6 +194,26 @@ def ivf_centroid_update_noalloc(points: torch.Tensor, ids: torch.Tensor, sums: t
                                                _ptr(sums), _ptr(counts), _stream(dev))
     if rc != IVF_OK:
         _raise(rc)
+
+
+def ivf_cluster_major_reorder(points: torch.Tensor, ids: torch.Tensor, nlist: int):
+    """(out_points [n,d], out_offsets int64 [nlist+1], out_order int32 [n]): the rows regrouped so that
+    every list is contiguous; the order inside a list is unspecified."""
+    if not points.is_cuda:
+        raise ValueError("points must be a CUDA tensor")
+    _rows(points, "points")
+    _dev(ids, "ids", torch.int32)
+    n, d = points.shape
+    dev = points.device
+    out_points = torch.empty_like(points)
+    out_offsets = torch.empty((nlist + 1,), dtype=torch.int64, device=dev)
+    out_order = torch.empty((n,), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib().ivf_cluster_major_reorder(_ptr(points), _dtype_code(points), _ptr(ids), n, d, nlist,
+                                             _ptr(out_points), _ptr(out_offsets), _ptr(out_order), _stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
+    return out_points, out_offsets, out_order
 
 
 def ivf_centroid_finalize(sums: torch.Tensor, counts: torch.Tensor, centroids: torch.Tensor):

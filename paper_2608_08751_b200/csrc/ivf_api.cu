@@ -732,6 +732,55 @@ int ivf_centroid_update(const void* points, ivf_dtype ptype, const int32_t* ids,
     return update_device(*ctx, points, ptype, ids, n, d, nlist, sums, counts, static_cast<cudaStream_t>(stream));
 }
 
+int ivf_cluster_major_reorder(const void* points, ivf_dtype ptype, const int32_t* ids, int64_t n, int d, int nlist,
+                              void* out_points, int64_t* out_offsets, int32_t* out_order, void* stream_) {
+    if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
+    if (ptype != IVF_F32 && ptype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
+    if (d < 16 || d > 256 || d % 16 != 0)
+        return fail(IVF_ERR_UNSUPPORTED, "d = %d: must be a multiple of 16 in [16, 256]", d);
+    if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
+    if (n >= (int64_t(1) << 31)) return fail(IVF_ERR_UNSUPPORTED, "n = %lld: at most 2^31 - 1 rows per call", (long long)n);
+    if (!out_offsets || !out_order) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    if (n > 0 && (!points || !ids || !out_points)) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    if ((reinterpret_cast<uintptr_t>(points) & 15) || (reinterpret_cast<uintptr_t>(out_points) & 15))
+        return fail(IVF_ERR_INVALID_ARG, "points and out_points must be 16-byte aligned");
+    DeviceCtx* pctx = nullptr;
+    int rc = get_ctx(&pctx);
+    if (rc != IVF_OK) return rc;
+    DeviceCtx& ctx = *pctx;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int *cnt, *off, *cur;
+    const int scan_blocks = (nlist + kScanBlock - 1) / kScanBlock;
+    WS(WS_UCNT, static_cast<size_t>(nlist) * sizeof(int), cnt);
+    WS(WS_UOFF, (static_cast<size_t>(nlist) + 1 + scan_blocks) * sizeof(int), off);
+    WS(WS_UCUR, static_cast<size_t>(nlist) * sizeof(int), cur);
+    int* block_sums = off + nlist + 1;
+    const int tk = timing_begin(TK_UPDATE, stream);
+    CUDA_TRY(cudaMemsetAsync(cnt, 0, static_cast<size_t>(nlist) * sizeof(int), stream));
+    const unsigned rb = static_cast<unsigned>((n + 255) / 256);
+    if (n > 0) {
+        update_hist_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, cnt, ctx.status);
+        LAUNCH_CHECK();
+    }
+    update_scan_local_kernel<<<scan_blocks, 1024, 0, stream>>>(cnt, nlist, off, block_sums);
+    LAUNCH_CHECK();
+    update_scan_fix_kernel<<<scan_blocks, 1024, 0, stream>>>(nlist, off, block_sums, cur);
+    LAUNCH_CHECK();
+    widen_offsets_kernel<<<(nlist + 256) / 256, 256, 0, stream>>>(off, nlist, reinterpret_cast<long long*>(out_offsets));
+    LAUNCH_CHECK();
+    if (n > 0) {
+        update_fill_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, off, cur, out_order);
+        LAUNCH_CHECK();
+        const int row_chunks = d * (ptype == IVF_U8 ? 1 : 4) / 16;
+        const int64_t pieces = n * row_chunks;
+        reorder_gather_kernel<<<static_cast<unsigned>((pieces + 255) / 256), 256, 0, stream>>>(
+            static_cast<const uint4*>(points), out_order, n, row_chunks, static_cast<uint4*>(out_points));
+        LAUNCH_CHECK();
+    }
+    timing_end(tk, stream);
+    return IVF_OK;
+}
+
 int ivf_centroid_finalize(const float* sums, const int64_t* counts, int nlist, int d, float* centroids_inout,
                           void* stream) {
     if (nlist < 1 || d < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d, d = %d", nlist, d);

@@ -170,6 +170,22 @@ __global__ void update_reduce_kernel(const T* __restrict__ x, const int* __restr
     if (lane == 0) counts[l] += static_cast<long long>(end - beg);
 }
 
+// Cluster-major copy (Sec. 3.1 index layout): destination row p receives source row order[p];
+// one thread per 16-byte piece of a row.  Also widens the list offsets to 64 bits.
+__global__ void reorder_gather_kernel(const uint4* __restrict__ src, const int* __restrict__ order, int64_t n,
+                                      int row_chunks, uint4* __restrict__ dst) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n * row_chunks) return;
+    const int64_t p = i / row_chunks;
+    const int c = static_cast<int>(i - p * row_chunks);
+    dst[i] = src[static_cast<int64_t>(order[p]) * row_chunks + c];
+}
+
+__global__ void widen_offsets_kernel(const int* __restrict__ off, int nlist, long long* __restrict__ out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i <= nlist) out[i] = off[i];
+}
+
 __global__ void finalize_kernel(const float* __restrict__ sums, const long long* __restrict__ counts, int nlist,
                                 int d, float* __restrict__ centroids) {
     const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;

@@ -223,6 +223,27 @@ def test_finalize_matches_oracle_and_keeps_empty_lists():
     np.testing.assert_allclose(got, want, rtol=2e-7)  # fp32 divide vs fp64 divide then rounding: <= 1 ulp
 
 
+# ---------------------------------------------------------------- cluster-major reorder
+@pytest.mark.parametrize("dtype,n,nlist,d", [("u8", 20000, 700, 128), ("f32", 5000, 4097, 96), ("u8", 300, 5, 16),
+                                             ("f32", 1, 3, 32)])
+def test_cluster_major_reorder(dtype, n, nlist, d):
+    rng = np.random.default_rng(n)
+    x = rng.integers(0, 256, (n, d)).astype(np.uint8) if dtype == "u8" else rng.standard_normal((n, d)).astype(np.float32)
+    ids = rng.integers(0, nlist, n).astype(np.int32)
+    if nlist > 10:
+        ids[ids == 2] = 3  # an empty list
+    out, offsets, order = B.ivf_cluster_major_reorder(_cuda(x), _cuda(ids), nlist)
+    B.ivf_check()
+    out, offsets, order = out.cpu().numpy(), offsets.cpu().numpy(), order.cpu().numpy()
+    o_off, o_order = oracle.reorder(ids, nlist)
+    assert (offsets == o_off).all()                       # unique: where every list starts and ends
+    assert (np.sort(order) == np.arange(n)).all()         # a permutation of the rows
+    assert (ids[order] == np.repeat(np.arange(nlist), np.diff(o_off))).all()  # list-major
+    for l in (0, nlist // 2, nlist - 1):                  # inside a list any order is valid: compare the sets
+        assert sorted(order[o_off[l]:o_off[l + 1]].tolist()) == o_order[o_off[l]:o_off[l + 1]].tolist()
+    assert (out == x[order]).all()
+
+
 # ---------------------------------------------------------------- host streaming
 def test_route_from_pinned_host_memory():
     x, c = _rand(3000, 2000, 128, "u8", 12)

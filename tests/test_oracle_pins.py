@@ -240,3 +240,18 @@ def test_lloyd_every_row_its_own_list():
     x = rng.permutation(200)[:40, None].astype(np.float32) * np.ones((1, 3), np.float32)  # distinct rows
     c, ids, inertia = oracle.lloyd(x, x.copy(), 2)
     assert (inertia == 0).all() and ids.tolist() == list(range(40)) and (c == x).all()
+
+
+# ---------------------------------------------------------------- cluster-major reorder
+def test_reorder_hand_case_and_stable_argsort():
+    ids = np.array([2, 0, 2, 1, 0, 2], np.int32)
+    offsets, order = oracle.reorder(ids, 4)
+    assert offsets.tolist() == [0, 2, 3, 6, 6]        # list 3 is empty
+    assert order.tolist() == [1, 4, 3, 0, 2, 5]       # input order kept inside each list
+    rng = np.random.default_rng(6)
+    ids = rng.integers(0, 37, 5000).astype(np.int32)
+    offsets, order = oracle.reorder(ids, 37)
+    assert (order == np.argsort(ids, kind="stable")).all()
+    assert (np.diff(offsets) == np.bincount(ids, minlength=37)).all() and offsets[-1] == 5000
+    with pytest.raises(ValueError):
+        oracle.reorder(np.array([0, 5], np.int32), 5)
