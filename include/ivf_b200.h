@@ -66,6 +66,24 @@ int ivf_route(const void* queries, int64_t nq, int d, ivf_dtype qtype,
               int32_t* out_ids, float* out_dists, void* stream);
 
 /*
+ * Routing against a centroid table that stays resident on the device (Sec. 3.1 / 4.1: the centroid
+ * matrix is GPU-resident routing state; only the query batch changes per call).  ivf_route prepares
+ * the tensor-core copy of the centroids on every call, which is right while they change (Lloyd
+ * iterations) and wasteful when they do not (serving).  ivf_centroids_create does that preparation
+ * once -- it enqueues its work on `stream` and allocates the prepared copy (nlist * (d rounded up
+ * to 64, + 16) * 2 bytes) stream-ordered; the float32 `centroids` may be freed after that work is
+ * done.  ivf_route_prepared is ivf_route without the centroid preparation; outputs are identical.
+ * A handle belongs to the device that was current at creation and must be used by one stream at a
+ * time (every call updates per-batch scale factors stored with it).  ivf_centroids_destroy frees it
+ * stream-ordered.
+ */
+typedef struct ivf_centroids ivf_centroids;
+int ivf_centroids_create(const float* centroids, int nlist, int d, ivf_centroids** out, void* stream);
+int ivf_centroids_destroy(ivf_centroids* handle, void* stream);
+int ivf_route_prepared(const ivf_centroids* handle, const void* queries, int64_t nq, ivf_dtype qtype,
+                       int nprobe, int32_t* out_ids, float* out_dists, void* stream);
+
+/*
  * Assignment to the nearest centroid (Sec. 3.1 index layout; Sec. 5.5 full-mode construction).
  * Same as ivf_route with nprobe = 1: out_ids [n] int32, out_dists [n] float32 (may be NULL).
  * `points` may be device or page-locked host memory as for ivf_route.

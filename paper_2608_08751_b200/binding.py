@@ -21,7 +21,8 @@ IVF_ERR_CUDA, IVF_ERR_DEVICE_TIMEOUT, IVF_ERR_BAD_ID = -4, -5, -6
 
 EXPORTS = (
     "ivf_route", "ivf_assign", "ivf_centroid_update", "ivf_centroid_update_noalloc", "ivf_centroid_finalize",
-    "ivf_assign_update", "ivf_cluster_major_reorder",
+    "ivf_assign_update", "ivf_cluster_major_reorder", "ivf_centroids_create", "ivf_centroids_destroy",
+    "ivf_route_prepared",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
     "ivf_debug_plan", "ivf_debug_span", "ivf_debug_set_wait_limit_ns",
     "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_stats",
@@ -56,6 +57,9 @@ def lib() -> ctypes.CDLL:
     L.ivf_centroid_update_noalloc.argtypes = [vp, i32, vp, i64, i32, i32, vp, vp, vp]
     L.ivf_centroid_finalize.argtypes = [vp, vp, i32, i32, vp, vp]
     L.ivf_cluster_major_reorder.argtypes = [vp, i32, vp, i64, i32, i32, vp, vp, vp, vp]
+    L.ivf_centroids_create.argtypes = [vp, i32, i32, ctypes.POINTER(vp), vp]
+    L.ivf_centroids_destroy.argtypes = [vp, vp]
+    L.ivf_route_prepared.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp]
     L.ivf_assign_update.argtypes = [vp, i64, i32, i32, vp, i32, vp, vp, vp, vp, i64, vp]
     L.ivf_check.argtypes = [vp]
     L.ivf_last_error.restype = ctypes.c_char_p
@@ -128,6 +132,54 @@ def ivf_route(queries: torch.Tensor, centroids: torch.Tensor, nprobe: int,
         rc = lib().ivf_route(_ptr(queries), nq, d, _dtype_code(queries), _ptr(centroids), nlist, nprobe,
                              _ptr(_dev(out_ids, "out_ids", torch.int32)),
                              _ptr(out_dists), _stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
+    return out_ids, out_dists
+
+
+class PreparedCentroids:
+    """Handle of a device-resident prepared centroid table (ivf_centroids_create / _destroy)."""
+
+    def __init__(self, centroids: torch.Tensor):
+        _dev(centroids, "centroids", torch.float32)
+        self.nlist, self.d = centroids.shape
+        self.device = centroids.device
+        self._h = ctypes.c_void_p()
+        with torch.cuda.device(self.device):
+            rc = lib().ivf_centroids_create(_ptr(centroids), self.nlist, self.d, ctypes.byref(self._h),
+                                            _stream(self.device))
+        if rc != IVF_OK:
+            _raise(rc)
+
+    def close(self):
+        if self._h:
+            with torch.cuda.device(self.device):
+                lib().ivf_centroids_destroy(self._h, _stream(self.device))
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def ivf_route_prepared(handle: PreparedCentroids, queries: torch.Tensor, nprobe: int,
+                       out_ids: torch.Tensor | None = None, out_dists: torch.Tensor | None = None,
+                       want_dists: bool = True):
+    """ivf_route against a prepared, device-resident centroid table."""
+    _rows(queries, "queries")
+    nq, d = queries.shape
+    if d != handle.d:
+        raise ValueError("dimension mismatch between queries and the prepared centroids")
+    dev = handle.device
+    if out_ids is None:
+        out_ids = torch.empty((nq, nprobe), dtype=torch.int32, device=dev)
+    if out_dists is None and want_dists:
+        out_dists = torch.empty((nq, nprobe), dtype=torch.float32, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib().ivf_route_prepared(handle._h, _ptr(queries), nq, _dtype_code(queries), nprobe,
+                                      _ptr(_dev(out_ids, "out_ids", torch.int32)), _ptr(out_dists), _stream(dev))
     if rc != IVF_OK:
         _raise(rc)
     return out_ids, out_dists

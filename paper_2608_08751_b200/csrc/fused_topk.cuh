@@ -75,6 +75,8 @@ struct FusedParams {
                           // records for the given rule
     int2* part_meta;      // k > 1: [n][partials] {entries (records) in the log or -1 if it overflowed,
                           // bits of the final tau}
+    int* clear0;          // two optional words that block 0 sets to zero (list counters of the merge)
+    int* clear1;
     int* status;          // sticky device status word
     unsigned long long* stats;  // optional counters: [0] in-kernel selections, [1] log entries written
     uint64_t wait_limit_ns;
@@ -429,6 +431,10 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             mbar_init(&b_empty[i], 1);
         }
         *abort_flag = 0;
+        if (blockIdx.x == 0) {
+            if (p.clear0) *p.clear0 = 0;
+            if (p.clear1) *p.clear1 = 0;
+        }
         fence_mbar_init();
         tma_prefetch_desc(&tmap_x);
         tma_prefetch_desc(&tmap_xa);

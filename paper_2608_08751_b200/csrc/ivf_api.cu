@@ -62,15 +62,29 @@ struct TimedLaunch {
     int kind;
 };
 std::vector<TimedLaunch> g_timed;
+std::vector<cudaEvent_t> g_event_pool;  // events are recycled: creating one per launch would make the host the bottleneck
 bool g_timing = false;
+
+cudaEvent_t pooled_event() {
+    if (!g_event_pool.empty()) {
+        cudaEvent_t e = g_event_pool.back();
+        g_event_pool.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+    return e;
+}
 
 int timing_begin(int kind, cudaStream_t stream) {
     if (!g_timing) return -1;
+    std::lock_guard<std::mutex> lk(g_mu);
     TimedLaunch t;
     t.kind = kind;
-    if (cudaEventCreate(&t.a) != cudaSuccess || cudaEventCreate(&t.b) != cudaSuccess) return -1;
+    t.a = pooled_event();
+    t.b = pooled_event();
+    if (!t.a || !t.b) return -1;
     cudaEventRecord(t.a, stream);
-    std::lock_guard<std::mutex> lk(g_mu);
     g_timed.push_back(t);
     return static_cast<int>(g_timed.size()) - 1;
 }
@@ -187,13 +201,14 @@ int log_capacity(int k) { return (k == 1) ? 1 : (4 * k > 512 ? 4 * k : 512); }
 constexpr int kMinSampleRows = 512;
 int choose_rule(int k, int nlist, int* stride) {
     *stride = 1;
-    if (k <= kSampleM) return TAU_RUNNING;
-    const int S = k / 4;
+    // k <= 16: the 16 sample keys that define tau are themselves candidates, so the given rule can
+    // never come up short; a sample of every 16th centroid lets about 256 candidates through
+    const int S = k <= kSampleM ? 16 : k / 4;
     if ((nlist + S - 1) / S >= kMinSampleRows) {
         *stride = S;
         return TAU_GIVEN;
     }
-    return TAU_BOUNDED;
+    return k <= kSampleM ? TAU_RUNNING : TAU_BOUNDED;
 }
 
 int make_plan(int64_t n, int nlist, int d, int k, int num_sms, Plan* pl, bool one_row_tile = false) {
@@ -228,7 +243,7 @@ int make_plan(int64_t n, int nlist, int d, int k, int num_sms, Plan* pl, bool on
 int64_t rows_per_launch(int d, int k) {
     const int kp = (d + 63) / 64 * 64 + kAugK;
     const int64_t per_row = static_cast<int64_t>(kp) * 2 +
-                            (k > kSampleM ? 6ll * (4 * k + 4) * kRecordBytes + 6ll * 512 * 8 : 6ll * log_capacity(k) * 8);
+                            (k > 1 ? 6ll * (4 * (k < 96 ? 96 : k) + 4) * kRecordBytes + 6ll * 512 * 8 : 6ll * 8);
     int64_t rows = (int64_t(3) << 30) / per_row;
     rows = rows / (2 * kBlockM) * (2 * kBlockM);
     if (rows < 2 * kBlockM) rows = 2 * kBlockM;
@@ -312,11 +327,10 @@ struct CentroidPrep {
 int g_force_fallback = 0;
 bool g_stats = false;
 
-int prepare_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, int k, const Plan& pl,
-                      cudaStream_t stream, CentroidPrep* cp) {
-    WS(WS_C16, static_cast<size_t>(nlist) * pl.kp * sizeof(__half), cp->c16);
-    WS(WS_SCAL, 4 * sizeof(float), cp->scal);
-    WS(WS_BITS, 2 * sizeof(unsigned int), cp->bits);
+// Converts the centroids into cp->c16 (already allocated) and computes their scale; cp->scal and
+// cp->bits must point to 4 floats / 2 uints of device memory.
+int convert_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, const Plan& pl, cudaStream_t stream,
+                      CentroidPrep* cp) {
     const int tk = timing_begin(TK_PREP, stream);
     CUDA_TRY(cudaMemsetAsync(cp->bits, 0, 2 * sizeof(unsigned int), stream));
     const int64_t count = static_cast<int64_t>(nlist) * d;
@@ -328,9 +342,14 @@ int prepare_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, 
     LAUNCH_CHECK();
     const int64_t threads = static_cast<int64_t>(nlist) * 32;
     convert_rows_kernel<float, true><<<static_cast<unsigned>((threads + 255) / 256), 256, 0, stream>>>(
-        centroids, nlist, d, pl.kd, cp->scal, cp->c16, nullptr);
+        centroids, nlist, d, pl.kd, cp->scal, cp->c16, nullptr, nullptr, 0);
     LAUNCH_CHECK();
     timing_end(tk, stream);
+    return IVF_OK;
+}
+
+// Tensor maps over cp->c16 and the threshold rule for nprobe = k.
+int map_centroids(int nlist, int k, const Plan& pl, CentroidPrep* cp) {
     int rc = make_tmap(&cp->tmap_c, cp->c16, nlist, pl.kp, pl.block_n, false);
     if (rc != IVF_OK) return rc;
     rc = make_tmap(&cp->tmap_ca, cp->c16, nlist, pl.kp, pl.block_n, true);
@@ -347,6 +366,16 @@ int prepare_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, 
     return IVF_OK;
 }
 
+int prepare_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, int k, const Plan& pl,
+                      cudaStream_t stream, CentroidPrep* cp) {
+    WS(WS_C16, static_cast<size_t>(nlist) * pl.kp * sizeof(__half), cp->c16);
+    WS(WS_SCAL, 4 * sizeof(float), cp->scal);
+    WS(WS_BITS, 2 * sizeof(unsigned int), cp->bits);
+    int rc = convert_centroids(ctx, centroids, nlist, d, pl, stream, cp);
+    if (rc != IVF_OK) return rc;
+    return map_centroids(nlist, k, pl, cp);
+}
+
 struct PointPrep {
     __half* x16;
     float* xn;
@@ -355,8 +384,10 @@ struct PointPrep {
 
 int launch_fused(DeviceCtx& ctx, const Plan& pl, int64_t n, int nlist, int k, int rule, const float* tau_in,
                  const PointPrep& pp, const CUtensorMap& tmap_c, const CUtensorMap& tmap_ca, Entry* part,
-                 int2* part_meta, int kind, cudaStream_t stream) {
+                 int2* part_meta, int kind, cudaStream_t stream, int* clear0 = nullptr, int* clear1 = nullptr) {
     FusedParams fp;
+    fp.clear0 = clear0;
+    fp.clear1 = clear1;
     fp.n = n;
     fp.nlist = nlist;
     fp.k = k;
@@ -444,7 +475,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     if (rc != IVF_OK) return rc;
     const bool given = k > 1 && cp.rule == TAU_GIVEN;
     // given rule: the logs hold 48-byte group records, at most 4k + 4 per (row, slot)
-    if (given) pl.cap = 4 * k + 4;
+    if (given) pl.cap = (k <= kSampleM ? 384 : 4 * k) + 4;
     size_t part_bytes = static_cast<size_t>(n) * pl.partials * pl.cap * (given ? kRecordBytes : sizeof(Entry));
     size_t meta_bytes = static_cast<size_t>(n) * pl.partials * sizeof(int2);
     if (given) {
@@ -466,7 +497,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     WS(WS_PART, part_bytes, part);
     if (k > 1) {
         WS(WS_PARTMETA, meta_bytes, part_meta);
-        WS(WS_FAIL, 2 * (static_cast<size_t>(n) + 1) * sizeof(int), failbuf);  // failed rows, then passed-on rows
+        WS(WS_FAIL, 2 * (static_cast<size_t>(n) + 2) * sizeof(int), failbuf);  // failed rows and passed-on rows
         if (given || g_force_fallback) WS(WS_FBKEYS, static_cast<size_t>(kFallbackFastRows + kFallbackCtas) * nlist * sizeof(float), fbkeys);
         if (given) WS(WS_TAU, static_cast<size_t>(n) * sizeof(float), tau);
     }
@@ -481,16 +512,15 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         maxabs_kernel<<<blocks, 256, 0, stream>>>(static_cast<const float*>(points), count, cp.bits);
         LAUNCH_CHECK();
     }
-    scales_kernel<<<1, 1, 0, stream>>>(cp.bits, u8, cp.scal);
-    LAUNCH_CHECK();
+    // the point conversion derives the scales of this chunk itself (and publishes them in cp.scal)
     const int64_t threads = n * 32;
     const unsigned cblocks = static_cast<unsigned>((threads + 255) / 256);
     if (u8)
         convert_rows_kernel<uint8_t, false><<<cblocks, 256, 0, stream>>>(static_cast<const uint8_t*>(points), n, d,
-                                                                         pl.kd, cp.scal, pp.x16, pp.xn);
+                                                                         pl.kd, cp.scal, pp.x16, pp.xn, cp.bits, 1);
     else
         convert_rows_kernel<float, false><<<cblocks, 256, 0, stream>>>(static_cast<const float*>(points), n, d, pl.kd,
-                                                                       cp.scal, pp.x16, pp.xn);
+                                                                       cp.scal, pp.x16, pp.xn, cp.bits, 0);
     LAUNCH_CHECK();
     timing_end(tk, stream);
 
@@ -507,12 +537,17 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         MergeParams ms = merge_params(pls, n, kSampleM, part, part_meta, pp, cp.scal);
         ms.tau_out = tau;
         tk = timing_begin(TK_THRESH, stream);
-        merge_tau_kernel<<<static_cast<unsigned>((n * 32 + 255) / 256), 256, 0, stream>>>(ms);
+        if (pls.partials <= 32)
+            merge_tau_warp_kernel<<<static_cast<unsigned>((n * 32 + 255) / 256), 256, 0, stream>>>(ms);
+        else {
+            const int threads = pls.partials >= kTauThreads ? kTauThreads : (pls.partials + 31) / 32 * 32;
+            merge_tau_kernel<<<static_cast<unsigned>(n), threads, 0, stream>>>(ms);
+        }
         LAUNCH_CHECK();
         timing_end(tk, stream);
     }
     rc = launch_fused(ctx, pl, n, nlist, k, cp.rule, tau, pp, cp.tmap_c, cp.tmap_ca, part, part_meta,
-                      k == 1 ? TK_FUSED_ARGMIN : TK_FUSED_TOPK, stream);
+                      k == 1 ? TK_FUSED_ARGMIN : TK_FUSED_TOPK, stream, failbuf, failbuf ? failbuf + n + 2 : nullptr);
     if (rc != IVF_OK) return rc;
 
     MergeParams mp = merge_params(pl, n, k, part, part_meta, pp, cp.scal);
@@ -529,9 +564,8 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     } else {
         // warp-per-row fast path first; rows it passes on (many partial logs, many candidates or
         // ties) are listed in `big` and merged by the general CTA-per-row kernel
-        mp.big = failbuf + n + 1;
-        CUDA_TRY(cudaMemsetAsync(failbuf, 0, sizeof(int), stream));
-        CUDA_TRY(cudaMemsetAsync(mp.big, 0, sizeof(int), stream));
+        // (both list counters were cleared by the fused kernel that just ran)
+        mp.big = failbuf + n + 2;
         if (!ctx.merge_attr_set) {
             CUDA_TRY(cudaFuncSetAttribute(merge_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(kMergeWarps * sizeof(MergeWarpSmem))));
@@ -539,7 +573,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         }
         // about 4k candidates per row pass a given threshold: beyond k = 128 they do not fit the
         // warp-level buffers, so everything goes to the general kernel directly
-        const bool try_warp = !(given && 5 * k > kWarpKeys);
+        const bool try_warp = !(given && 5 * k > kWarpKeys);  // (k <= 16 lets ~256 through: fits)
         if (try_warp) {
             merge_warp_kernel<<<static_cast<unsigned>((n + kMergeWarps - 1) / kMergeWarps), 32 * kMergeWarps,
                                 kMergeWarps * sizeof(MergeWarpSmem), stream>>>(mp);
@@ -567,9 +601,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
             fb.out_dists = out_dists;
             fallback_keys_kernel<<<dim3(kFallbackKeyChunks, kFallbackFastRows), kFallbackThreads, 0, stream>>>(fb);
             LAUNCH_CHECK();
-            fallback_select_kernel<<<kFallbackFastRows, kFallbackThreads, 0, stream>>>(fb);
-            LAUNCH_CHECK();
-            fallback_rows_kernel<<<kFallbackCtas, kFallbackThreads, 0, stream>>>(fb);
+            fallback_select_kernel<<<kFallbackFastRows + kFallbackCtas, kFallbackThreads, 0, stream>>>(fb);
             LAUNCH_CHECK();
         }
     }
@@ -612,9 +644,17 @@ int update_device(DeviceCtx& ctx, const void* points, int ptype, const int32_t* 
 // ------------------------------------------------------------------ the chunk pipeline
 // Walks the rows in chunks; a host-resident chunk is staged through one of two device buffers on
 // the copy stream.  `with_update` adds the Lloyd accumulation of each chunk.
+struct ivf_centroids_impl {
+    int device;
+    int nlist, d;
+    __half* c16;     // fp16 operand copy with the norm columns
+    float* scal;     // 4 floats: point scale, centroid scale, 1 / product, A
+    unsigned* bits;  // 2 uints: max |x| of the current chunk, max |c|
+};
+
 int run_chunks(const void* points, int64_t n, int d, int ptype, const float* centroids, int nlist, int k,
                int32_t* out_ids, float* out_dists, bool with_update, float* sums, int64_t* counts,
-               int64_t chunk_rows, cudaStream_t stream) {
+               int64_t chunk_rows, cudaStream_t stream, const ivf_centroids_impl* prepared = nullptr) {
     DeviceCtx* pctx = nullptr;
     int rc = get_ctx(&pctx);
     if (rc != IVF_OK) return rc;
@@ -636,7 +676,14 @@ int run_chunks(const void* points, int64_t n, int d, int ptype, const float* cen
     rc = make_plan(rows, nlist, d, k, ctx.num_sms, &pl0);
     if (rc != IVF_OK) return rc;
     CentroidPrep cp;
-    rc = prepare_centroids(ctx, centroids, nlist, d, k, pl0, stream, &cp);
+    if (prepared) {
+        cp.c16 = prepared->c16;
+        cp.scal = prepared->scal;
+        cp.bits = prepared->bits;
+        rc = map_centroids(nlist, k, pl0, &cp);
+    } else {
+        rc = prepare_centroids(ctx, centroids, nlist, d, k, pl0, stream, &cp);
+    }
     if (rc != IVF_OK) return rc;
 
     uint8_t* stage[2] = {nullptr, nullptr};
@@ -704,6 +751,72 @@ int ivf_route(const void* queries, int64_t nq, int d, ivf_dtype qtype, const flo
     if (rc != IVF_OK || nq == 0) return rc;
     return run_chunks(queries, nq, d, qtype, centroids, nlist, nprobe, out_ids, out_dists, false, nullptr, nullptr, 0,
                       static_cast<cudaStream_t>(stream));
+}
+
+int ivf_centroids_create(const float* centroids, int nlist, int d, ivf_centroids** out, void* stream_) {
+    if (!out) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    *out = nullptr;
+    if (d < 16 || d > 256 || d % 16 != 0)
+        return fail(IVF_ERR_UNSUPPORTED, "d = %d: must be a multiple of 16 in [16, 256]", d);
+    if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
+    if (!centroids) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    if (reinterpret_cast<uintptr_t>(centroids) & 15) return fail(IVF_ERR_INVALID_ARG, "centroids must be 16-byte aligned");
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != IVF_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    Plan pl;
+    rc = make_plan(kBlockM, nlist, d, 1, ctx->num_sms, &pl);
+    if (rc != IVF_OK) return rc;
+    ivf_centroids_impl* h = new ivf_centroids_impl();
+    CUDA_TRY(cudaGetDevice(&h->device));
+    h->nlist = nlist;
+    h->d = d;
+    void* mem = nullptr;
+    const size_t c16_bytes = (static_cast<size_t>(nlist) * pl.kp * sizeof(__half) + 255) & ~size_t(255);
+    cudaError_t e = cudaMallocAsync(&mem, c16_bytes + 256, stream);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        delete h;
+        return fail(IVF_ERR_ALLOC, "allocation of %zu bytes for the prepared centroids failed: %s", c16_bytes + 256,
+                    cudaGetErrorString(e));
+    }
+    h->c16 = static_cast<__half*>(mem);
+    h->scal = reinterpret_cast<float*>(static_cast<uint8_t*>(mem) + c16_bytes);
+    h->bits = reinterpret_cast<unsigned*>(h->scal + 4);
+    CentroidPrep cp;
+    cp.c16 = h->c16;
+    cp.scal = h->scal;
+    cp.bits = h->bits;
+    rc = convert_centroids(*ctx, centroids, nlist, d, pl, stream, &cp);
+    if (rc != IVF_OK) {
+        cudaFreeAsync(mem, stream);
+        delete h;
+        return rc;
+    }
+    *out = reinterpret_cast<ivf_centroids*>(h);
+    return IVF_OK;
+}
+
+int ivf_centroids_destroy(ivf_centroids* handle, void* stream) {
+    if (!handle) return IVF_OK;
+    ivf_centroids_impl* h = reinterpret_cast<ivf_centroids_impl*>(handle);
+    CUDA_TRY(cudaFreeAsync(h->c16, static_cast<cudaStream_t>(stream)));
+    delete h;
+    return IVF_OK;
+}
+
+int ivf_route_prepared(const ivf_centroids* handle, const void* queries, int64_t nq, ivf_dtype qtype, int nprobe,
+                       int32_t* out_ids, float* out_dists, void* stream) {
+    if (!handle) return fail(IVF_ERR_INVALID_ARG, "null centroid handle");
+    const ivf_centroids_impl* h = reinterpret_cast<const ivf_centroids_impl*>(handle);
+    int rc = check_common(queries, nq, h->d, qtype, reinterpret_cast<const float*>(h->c16), h->nlist, nprobe, out_ids);
+    if (rc != IVF_OK || nq == 0) return rc;
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != h->device) return fail(IVF_ERR_INVALID_ARG, "the centroid handle belongs to device %d, current is %d", h->device, dev);
+    return run_chunks(queries, nq, h->d, qtype, nullptr, h->nlist, nprobe, out_ids, out_dists, false, nullptr, nullptr, 0,
+                      static_cast<cudaStream_t>(stream), h);
 }
 
 int ivf_assign(const void* points, int64_t n, int d, ivf_dtype ptype, const float* centroids, int nlist,
@@ -873,8 +986,8 @@ int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int
 int ivf_debug_timing(int enable) {
     std::lock_guard<std::mutex> lk(g_mu);
     for (TimedLaunch& t : g_timed) {
-        cudaEventDestroy(t.a);
-        cudaEventDestroy(t.b);
+        g_event_pool.push_back(t.a);
+        g_event_pool.push_back(t.b);
     }
     g_timed.clear();
     g_timing = enable != 0;
@@ -895,8 +1008,8 @@ int ivf_debug_timing_read(double ms[6], int64_t launches[6]) {
             ms[t.kind] += e;
             launches[t.kind] += 1;
         }
-        cudaEventDestroy(t.a);
-        cudaEventDestroy(t.b);
+        g_event_pool.push_back(t.a);
+        g_event_pool.push_back(t.b);
     }
     g_timed.clear();
     return IVF_OK;

@@ -479,39 +479,77 @@ __global__ void __launch_bounds__(32 * kMergeWarps) merge_warp_kernel(const Merg
     merge_write_row(p, row, sm.keys, lane, 32);
 }
 
-// Threshold pass: one warp per row reads the partial sketches (16 smallest group minima per
-// thread of the fused kernel) and writes the 16th smallest value overall.
-__global__ void __launch_bounds__(256) merge_tau_kernel(const MergeParams p) {
+// Threshold pass: per row, the 16th smallest of all the sketch values its partial results hold.
+// Every partial sketch is 16 values in ascending order, so a lane that holds one sketch only ever
+// offers its head: 16 rounds of "take the smallest head, advance that lane" give the 16 smallest of
+// up to 32 sketches.  One CTA per row; each warp reduces 32 sketches at a time to a sorted list of
+// 16 in shared memory, and warp 0 reduces those lists the same way.
+constexpr int kTauThreads = 256;
+
+__device__ __forceinline__ void take16(float (&v)[kSampleM], int lane, float* out /* 16 ascending, may be null */,
+                                       float& last) {
+    const float INF = __int_as_float(0x7f800000);
+#pragma unroll 1
+    for (int round = 0; round < kSampleM; ++round) {
+        float m = v[0];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) m = fminf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+        last = m;
+        if (out != nullptr && lane == 0) out[round] = m;
+        const uint32_t who = __ballot_sync(0xFFFFFFFFu, v[0] == m);
+        if (lane == __ffs(who) - 1) {  // the first lane holding m advances its sorted list
+#pragma unroll
+            for (int i = 0; i < kSampleM - 1; ++i) v[i] = v[i + 1];
+            v[kSampleM - 1] = INF;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kTauThreads) merge_tau_kernel(const MergeParams p) {
+    __shared__ float lists[kTauThreads / 32 + 1][kSampleM];  // one per warp, plus the running result
+    const float INF = __int_as_float(0x7f800000);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row = blockIdx.x;
+    const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows);
+    const Entry* base = p.part + static_cast<size_t>(row) * p.partials * p.cap;
+    if (threadIdx.x < kSampleM) lists[kTauThreads / 32][threadIdx.x] = INF;
+    float result = INF;
+    const int nw = blockDim.x >> 5;  // the launch sizes the CTA to the number of partial sketches
+    for (int s0 = 0; s0 < ns; s0 += blockDim.x) {
+        __syncthreads();
+        float v[kSampleM];
+        const int slot = s0 + threadIdx.x;
+#pragma unroll
+        for (int i = 0; i < kSampleM; ++i) v[i] = slot < ns ? base[static_cast<size_t>(slot) * p.cap + i].v : INF;
+        float last;
+        take16(v, lane, lists[warp], last);
+        __syncthreads();
+        if (warp == 0) {
+            // lanes 0..8 hold the lists of the 8 warps and the running result
+#pragma unroll
+            for (int i = 0; i < kSampleM; ++i)
+                v[i] = lane < nw ? lists[lane][i] : (lane == nw ? lists[kTauThreads / 32][i] : INF);
+            __syncwarp();
+            take16(v, lane, lists[kTauThreads / 32], result);
+        }
+    }
+    if (threadIdx.x == 0) p.tau_out[row] = result;
+}
+
+// The same with one warp per row, for rows with at most 32 partial sketches (large batches, where
+// few CTAs share a row): lane = sketch.
+__global__ void __launch_bounds__(256) merge_tau_warp_kernel(const MergeParams p) {
+    const float INF = __int_as_float(0x7f800000);
     const int lane = threadIdx.x & 31;
     const int64_t row = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
     if (row >= p.n) return;
     const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows);
     const Entry* base = p.part + static_cast<size_t>(row) * p.partials * p.cap;
-    const int total = ns * kSampleM;
-    // every lane keeps the 16 smallest of its share; then 16 rounds of "extract the warp minimum"
-    float net[kSampleM];
+    float v[kSampleM];
 #pragma unroll
-    for (int i = 0; i < kSampleM; ++i) net[i] = __int_as_float(0x7f800000);
-    for (int idx = lane; idx < total; idx += 32) {
-        const float v = base[static_cast<size_t>(idx / kSampleM) * p.cap + (idx % kSampleM)].v;
-        if (v < net[kSampleM - 1]) network_insert(net, v);
-    }
-    float result = __int_as_float(0x7f800000);
-#pragma unroll 1
-    for (int round = 0; round < kSampleM; ++round) {
-        float m = net[0];
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) m = fminf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
-        result = m;
-        // the first lane holding m drops it (shift its sorted list down by one)
-        const uint32_t who = __ballot_sync(0xFFFFFFFFu, net[0] == m);
-        if (who == 0u) break;  // only infinities left
-        if (lane == __ffs(who) - 1) {
-#pragma unroll
-            for (int i = 0; i < kSampleM - 1; ++i) net[i] = net[i + 1];
-            net[kSampleM - 1] = __int_as_float(0x7f800000);
-        }
-    }
+    for (int i = 0; i < kSampleM; ++i) v[i] = lane < ns ? base[static_cast<size_t>(lane) * p.cap + i].v : INF;
+    float result;
+    take16(v, lane, nullptr, result);
     if (lane == 0) p.tau_out[row] = result;
 }
 
@@ -650,21 +688,21 @@ __global__ void __launch_bounds__(kFallbackThreads) fallback_keys_kernel(const F
     }
 }
 
+// Blocks [0, kFallbackFastRows) select from the keys that fallback_keys_kernel prepared.  The other
+// blocks take any further failed rows (none in practice), one CTA per row doing both steps: slow
+// and exact.
 __global__ void __launch_bounds__(kFallbackThreads) fallback_select_kernel(const FallbackParams p) {
     __shared__ FallbackSmem sm;
     const int nfail = p.fail[0];
-    const int idx = blockIdx.x;
-    if (idx >= nfail || idx >= kFallbackFastRows) return;
-    fallback_select_row(p, p.keys + static_cast<size_t>(idx) * p.nlist, p.fail[1 + idx], sm);
-}
-
-// Any further failed rows (none in practice): one CTA per row does both steps; slow and exact.
-__global__ void __launch_bounds__(kFallbackThreads) fallback_rows_kernel(const FallbackParams p) {
-    __shared__ FallbackSmem sm;
-    const int nfail = p.fail[0];
-    float* keys = p.keys + static_cast<size_t>(kFallbackFastRows + blockIdx.x) * p.nlist;
+    if (blockIdx.x < kFallbackFastRows) {
+        const int idx = blockIdx.x;
+        if (idx < nfail) fallback_select_row(p, p.keys + static_cast<size_t>(idx) * p.nlist, p.fail[1 + idx], sm);
+        return;
+    }
+    const int slow = blockIdx.x - kFallbackFastRows, nslow = gridDim.x - kFallbackFastRows;
+    float* keys = p.keys + static_cast<size_t>(kFallbackFastRows + slow) * p.nlist;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int idx = kFallbackFastRows + blockIdx.x; idx < nfail; idx += gridDim.x) {
+    for (int idx = kFallbackFastRows + slow; idx < nfail; idx += nslow) {
         const int64_t row = p.fail[1 + idx];
         __syncthreads();
         for (int t = threadIdx.x; t < p.kp; t += blockDim.x) sm.xs[t] = __half2float(p.x16[row * p.kp + t]);

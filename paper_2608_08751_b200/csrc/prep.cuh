@@ -48,29 +48,48 @@ __device__ __forceinline__ float pow2_scale_for(float maxabs) {
 // scal[3] = A = 2^15 sx / sc.  bits[0] = max |x| bits (unused for uint8 points), bits[1] = max |c|.
 // The point scale never exceeds the centroid scale (so A <= 2^15) and is at least sc * 2^-29
 // (so A stays a normal fp16 number).
-__global__ void scales_kernel(const unsigned int* bits, int points_are_u8, float* scal) {
+__device__ __forceinline__ void compute_scales(const unsigned int* bits, int points_are_u8, float (&out)[4]) {
     const float sc = pow2_scale_for(__uint_as_float(bits[1]));
     float sx = points_are_u8 ? 8.0f : pow2_scale_for(__uint_as_float(bits[0]));
     sx = fminf(sx, sc);
     sx = fmaxf(sx, sc * 1.862645149230957e-09f);  // 2^-29
-    scal[0] = sx;
-    scal[1] = sc;
-    scal[2] = 1.0f / (sx * sc);
-    scal[3] = 32768.0f * sx / sc;
+    out[0] = sx;
+    out[1] = sc;
+    out[2] = 1.0f / (sx * sc);
+    out[3] = 32768.0f * sx / sc;
+}
+__global__ void scales_kernel(const unsigned int* bits, int points_are_u8, float* scal) {
+    float v[4];
+    compute_scales(bits, points_are_u8, v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) scal[i] = v[i];
 }
 
 // One warp per row.  Lane g converts columns [8g, 8g+8) of the data part; after the norm is reduced
-// lanes 0 and 1 write the 16 extra columns.
+// lanes 0 and 1 write the 16 extra columns.  If `bits` is given (point rows), the scales are derived
+// here from the magnitude words instead of being read, and the first thread publishes them in `scal`
+// for the kernels that follow.
 template <typename T, bool CENTROID>
-__global__ void convert_rows_kernel(const T* __restrict__ x, int64_t rows, int d, int kd,
-                                    const float* __restrict__ scal, __half* __restrict__ out,
-                                    float* __restrict__ norms) {
+__global__ void convert_rows_kernel(const T* __restrict__ x, int64_t rows, int d, int kd, float* scal,
+                                    __half* __restrict__ out, float* __restrict__ norms,
+                                    const unsigned int* __restrict__ bits, int points_are_u8) {
     const int lane = threadIdx.x & 31;
     const int64_t row = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
     if (row >= rows) return;
     const int kp = kd + 16;
-    const float sc = scal[1];
-    const float s = CENTROID ? -2.0f * sc : scal[0];
+    float sv[4];
+    if (bits != nullptr) {
+        compute_scales(bits, points_are_u8, sv);
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) scal[i] = sv[i];
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) sv[i] = scal[i];
+    }
+    const float sc = sv[1];
+    const float s = CENTROID ? -2.0f * sc : sv[0];
     float acc = 0.0f;
     const int c0 = lane * 8;
     if (c0 < kd) {
@@ -117,7 +136,7 @@ __global__ void convert_rows_kernel(const T* __restrict__ x, int64_t rows, int d
                 a[1] = mid;
                 a[2] = __float2half_rn(r2);
             } else {
-                const __half av = __float2half_rn(scal[3]);
+                const __half av = __float2half_rn(sv[3]);
                 a[0] = av;
                 a[1] = av;
                 a[2] = av;

@@ -5,6 +5,9 @@ A small driver for profilers and quick measurements:
     python -m paper_2608_08751_b200.run_case --op route --n 10000 --nlist 65536 --k 64
     python -m paper_2608_08751_b200.run_case --op update --n 1048576 --nlist 65536
     python -m paper_2608_08751_b200.run_case --op stream --n 8388608 --nlist 65536 --iters 2
+    python -m paper_2608_08751_b200.run_case --op serve --nlist 524288 --k 64 --batches 8,32,256,2048
+"serve" routes small query batches against a prepared, device-resident centroid table (the paper's
+serving setting: N_list = 0.5M, batch sizes 8 to 2048) and reports the time per batch.
 "stream" is the IVF-build configuration in small: rows in page-locked host memory, streamed in
 1,048,576-row chunks through assign + update, then the finalize, per Lloyd iteration.
 Inputs follow the SIFT-shaped (uint8, all-positive mixture) or DEEP-shaped (float32, unit norm)
@@ -64,9 +67,40 @@ def stream_case(args):
                       "tflops": 2.0 * args.n * args.nlist * args.d / (ms / 1e3) / 1e12, "inertia": inertia}))
 
 
+def serve_case(args):
+    if args.dtype == "u8":
+        c = synth.sift_like_centroids(args.nlist, args.d)
+        q_all = synth.sift_like_queries(max(int(v) for v in args.batches.split(",")), args.d)
+    else:
+        c = synth.deep_like_centroids(args.nlist, args.d)
+        q_all = synth.deep_like_queries(max(int(v) for v in args.batches.split(",")), args.d)
+    ct = torch.from_numpy(c).cuda()
+    handle = B.PreparedCentroids(ct)
+    out = {"op": "serve", "nlist": args.nlist, "d": args.d, "k": args.k, "dtype": args.dtype, "batches": {}}
+    for bs in [int(v) for v in args.batches.split(",")]:
+        q = torch.from_numpy(q_all[:bs]).cuda()
+        ids = torch.empty((bs, args.k), dtype=torch.int32, device="cuda")
+        dists = torch.empty((bs, args.k), dtype=torch.float32, device="cuda")
+        for _ in range(3):
+            B.ivf_route_prepared(handle, q, args.k, ids, dists)
+        B.ivf_check()
+        reps = max(args.reps, 20)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            B.ivf_route_prepared(handle, q, args.k, ids, dists)
+        e1.record()
+        B.ivf_check()
+        us = e0.elapsed_time(e1) / reps * 1e3
+        out["batches"][str(bs)] = {"us_per_batch": us, "queries_per_s": bs / (us / 1e6)}
+    handle.close()
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="assign", choices=["assign", "route", "update", "stream"])
+    ap.add_argument("--op", default="assign", choices=["assign", "route", "update", "stream", "serve"])
+    ap.add_argument("--batches", default="8,32,256,2048", help="query batch sizes of --op serve")
     ap.add_argument("--iters", type=int, default=1, help="Lloyd iterations of --op stream")
     ap.add_argument("--n", type=int, default=262144)
     ap.add_argument("--nlist", type=int, default=65536)
@@ -78,6 +112,8 @@ def main():
 
     if args.op == "stream":
         return stream_case(args)
+    if args.op == "serve":
+        return serve_case(args)
     if args.dtype == "u8":
         x = synth.sift_like_rows(0, rows=args.n, d=args.d)
         c = synth.sift_like_centroids(args.nlist, args.d)

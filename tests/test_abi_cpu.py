@@ -97,7 +97,8 @@ def test_schedule_covers_every_unit_once_and_bounds_partials(n, nlist, d, k, sms
 
 def test_threshold_rule_selection():
     assert binding.ivf_debug_rule(1, 65536) == (-1, 1)
-    assert binding.ivf_debug_rule(16, 65536) == (0, 1)            # running: exact
+    assert binding.ivf_debug_rule(16, 65536) == (1, 16)           # threshold pass, can never come up short
+    assert binding.ivf_debug_rule(16, 1024) == (0, 1)             # small table: running rule, exact
     assert binding.ivf_debug_rule(64, 65536) == (1, 16)           # threshold pass over every 16th centroid
     assert binding.ivf_debug_rule(128, 262144) == (1, 32)
     assert binding.ivf_debug_rule(256, 1 << 20) == (1, 64)

@@ -130,6 +130,21 @@ def test_run_to_run_determinism():
         assert (a[0] == b[0]).all() and (a[1] == b[1]).all()
 
 
+@pytest.mark.parametrize("n,nlist,d,k,dtype", [(8, 30000, 128, 64, "u8"), (300, 5000, 96, 10, "f32"), (2048, 9000, 128, 1, "u8")])
+def test_prepared_centroids_give_identical_results(n, nlist, d, k, dtype):
+    x, c = _rand(n, nlist, d, dtype, seed=n + k)
+    h = B.PreparedCentroids(_cuda(c))
+    for rep in range(2):  # the handle is reused across batches
+        xs = x if rep == 0 else np.ascontiguousarray(x[::-1])
+        ids_p, d_p = B.ivf_route_prepared(h, _cuda(xs), k)
+        B.ivf_check()
+        ids, dists = B.ivf_route(_cuda(xs), _cuda(c), k)
+        B.ivf_check()
+        assert (ids_p == ids).all() and (d_p == dists).all()
+        parity.check_route(xs, c, k, ids_p.cpu().numpy(), d_p.cpu().numpy())
+    h.close()
+
+
 def test_no_distances_requested():
     x, c = _rand(200, 500, 64, "f32", 6)
     ids, none = B.ivf_route(_cuda(x), _cuda(c), 5, want_dists=False)
