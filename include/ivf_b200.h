@@ -197,6 +197,9 @@ int ivf_debug_wait_probe(void* stream);
 /* Test hook: when on, the merge of a k > 1 call declares every row's candidate set insufficient, so
  * that all rows take the exact brute-force recomputation that normally only catches rare rows. */
 int ivf_debug_force_fallback(int on);
+/* Test hook: rows per fused-kernel launch (0 restores the size derived from the scratch budget), so
+ * that the row-chunk loop of large calls can be exercised on small inputs. */
+int ivf_debug_set_row_chunk(int64_t rows);
 /* Test hook (host only): which threshold rule a call with this nprobe and nlist uses -- out[0] =
  * -1 (k = 1: argmin), 0 running (k <= 16), 1 given (threshold pass over every out[1]-th centroid),
  * 2 bounded (sample too small). */

@@ -25,7 +25,7 @@ EXPORTS = (
     "ivf_route_prepared",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
     "ivf_debug_plan", "ivf_debug_span", "ivf_debug_set_wait_limit_ns",
-    "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_stats",
+    "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_set_row_chunk", "ivf_debug_stats",
 )
 
 _lib = None
@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
     L.ivf_debug_timing.argtypes = [i32]
     L.ivf_debug_wait_probe.argtypes = [vp]
     L.ivf_debug_force_fallback.argtypes = [i32]
+    L.ivf_debug_set_row_chunk.argtypes = [i64]
     L.ivf_debug_stats.argtypes = [i32, ctypes.POINTER(i64)]
     L.ivf_debug_rule.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_int)]
     L.ivf_debug_timing_read.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
@@ -388,3 +389,7 @@ def ivf_debug_stats(enable: bool) -> dict:
     if rc != IVF_OK:
         _raise(rc)
     return {"selections": int(out[0]), "log_entries": int(out[1]), "fallback_rows": int(out[2])}
+
+
+def ivf_debug_set_row_chunk(rows: int) -> None:
+    lib().ivf_debug_set_row_chunk(rows)

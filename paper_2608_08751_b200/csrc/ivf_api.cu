@@ -326,6 +326,7 @@ struct CentroidPrep {
 
 int g_force_fallback = 0;
 bool g_stats = false;
+std::atomic<int64_t> g_row_chunk_override{0};  // test hook: rows per fused launch
 
 // Converts the centroids into cp->c16 (already allocated) and computes their scale; cp->scal and
 // cp->bits must point to 4 floats / 2 uints of device memory.
@@ -667,6 +668,7 @@ int run_chunks(const void* points, int64_t n, int d, int ptype, const float* cen
     const size_t esize = ptype == IVF_U8 ? 1 : 4;
 
     int64_t rows = rows_per_launch(d, k);
+    if (g_row_chunk_override.load() > 0) rows = g_row_chunk_override.load();
     if (chunk_rows <= 0) chunk_rows = int64_t(1) << 20;
     if ((host || with_update) && rows > chunk_rows) rows = chunk_rows;
     if (rows > n) rows = n;
@@ -1034,6 +1036,11 @@ int ivf_debug_rule(int k, int nlist, int out[2]) {
     if (k < 1 || nlist < 1 || !out) return fail(IVF_ERR_INVALID_ARG, "bad arguments");
     out[1] = 1;
     out[0] = (k == 1) ? -1 : choose_rule(k, nlist, &out[1]);
+    return IVF_OK;
+}
+
+int ivf_debug_set_row_chunk(int64_t rows) {
+    g_row_chunk_override.store(rows > 0 ? rows : 0);
     return IVF_OK;
 }
 

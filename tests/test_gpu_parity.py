@@ -106,6 +106,33 @@ def test_brute_force_recomputation_of_failed_rows(n, nlist, d, k, dtype):
     parity.check_route(q, ci, 50, ids, dists, exact=True)
 
 
+@pytest.mark.parametrize("k", [1, 8, 40])
+def test_row_chunk_loop_of_large_calls(k):
+    # big calls are split into row chunks that share the prepared centroids and the workspace;
+    # force small chunks (ragged last one) and compare with the unsplit call and the oracle
+    x, c = _rand(1000, 9000, 128, "u8", seed=31 + k)
+    want = _route(x, c, k)
+    B.ivf_debug_set_row_chunk(384)
+    try:
+        got = _route(x, c, k)
+    finally:
+        B.ivf_debug_set_row_chunk(0)
+    assert (got[0] == want[0]).all() and (got[1] == want[1]).all()
+    parity.check_route(x, c, k, got[0], got[1])
+
+
+def test_sampled_threshold_rarely_needs_the_exact_recomputation():
+    # the threshold pass lets about 4k candidates through; fewer than k should be a rare event
+    q, c = synth.routing_inputs(synth.C1, nq=4096)
+    B.ivf_debug_stats(True)
+    ids, dists = _route(q, c, 64)
+    st = B.ivf_debug_stats(False)
+    assert st["fallback_rows"] <= 0.005 * 4096
+    assert 64 <= st["log_entries"] / 4096 <= 6 * 64  # group records per row: near 4k, not the whole table
+    rows = np.arange(0, 4096, 128)
+    parity.check_route(q, c, 64, ids[rows], dists[rows], rows=rows)
+
+
 def test_duplicate_centroids_resolve_to_lower_id():
     _, c = _rand(1, 700, 128, "f32", 9)
     c[500] = c[20]
