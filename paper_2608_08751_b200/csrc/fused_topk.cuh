@@ -10,7 +10,10 @@
 // group is MT = 1 or 2 row tiles of 128 points that stay in shared memory; with MT = 2 every centroid
 // tile brought from L2 feeds two MMA sweeps (one TMEM accumulator buffer each), which halves the
 // L2 -> shared-memory traffic per FLOP.
-//   warp 0      TMA producer: the stationary 128-row point tile and a ring of centroid tiles
+//   warp 0      producer: TMA loads of the stationary 128-row point tile(s) and of a ring of centroid
+//               tiles.  uint8 points need no fp16 copy in HBM: at the start of a row group every
+//               epilogue thread reads its own raw row, widens it to fp16 (exact) and writes it into
+//               the swizzled operand tile in shared memory, along with |x|^2.
 //   warp 1      single-thread tcgen05.mma issuer; accumulators live in TMEM (fp32), two buffers,
 //               so the next tile's MMAs overlap this tile's epilogue
 //   warps 2..9  epilogue: TMEM lane = point row; the two warps that share a lane quadrant split
@@ -33,7 +36,10 @@
 //             smallest in place (radix select on the key bits, ties to the lower id) and tau
 //             becomes the k-th.  The same in-place selection catches any log that fills up.
 #pragma once
+#include <cuda_fp16.h>
+
 #include "ptx.cuh"
+#include "scales.cuh"
 
 namespace ivf {
 
@@ -75,6 +81,11 @@ struct FusedParams {
                           // records for the given rule
     int2* part_meta;      // k > 1: [n][partials] {entries (records) in the log or -1 if it overflowed,
                           // bits of the final tau}
+    const uint8_t* x_raw; // uint8 points [n][d], widened in shared memory (nullptr: fp16 copy via TMA)
+    int d;                // columns of x_raw
+    const unsigned int* bits;  // x_raw mode: magnitude words the scales are derived from
+    float* scal_out;      // x_raw mode: the four scale factors, published by block 0
+    float* xn_out;        // x_raw mode: |x|^2 per row
     int* clear0;          // two optional words that block 0 sets to zero (list counters of the merge)
     int* clear1;
     int* status;          // sticky device status word
@@ -384,6 +395,55 @@ __device__ __forceinline__ void consume(uint32_t (&acc)[32], int jbase, RowState
     }
 }
 
+// One thread widens one uint8 point row into the fp16 operand tile in shared memory: 16-byte
+// chunks of 8 values at the positions the 128-byte swizzle (data) and the 32-byte swizzle (norm
+// columns) give them, exactly as a TMA load of the fp16 copy would have placed them.  Returns |x|^2.
+__device__ __forceinline__ unsigned int widen_row_u8(const uint8_t* __restrict__ src, bool valid, int d, int kd,
+                                                     uint8_t* tile, int a_data_bytes, int row, float sx, float A) {
+    const __half2 k1024 = __floats2half2_rn(1024.0f, 1024.0f);
+    const __half2 sx2 = __floats2half2_rn(sx, sx);
+    // two bytes -> two fp16: 0x6400 | b is the half 1024 + b; subtract 1024, scale (all exact)
+    auto cvt2 = [&](uint32_t w, uint32_t sel) {
+        uint32_t q = __byte_perm(w, 0x64646464u, sel);
+        const __half2 t2 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&q), k1024), sx2);
+        return *reinterpret_cast<const uint32_t*>(&t2);
+    };
+    unsigned int sumsq = 0;
+#pragma unroll 1
+    for (int c0 = 0; c0 < kd / 8; c0 += 16) {  // 16 chunks (128 columns) in flight
+        uint2 w[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int c = c0 + i;
+            w[i] = make_uint2(0u, 0u);
+            if (valid && c * 8 < d) w[i] = *reinterpret_cast<const uint2*>(src + c * 8);
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int c = c0 + i;
+            if (c < kd / 8) {
+                sumsq = __dp4a(w[i].x, w[i].x, sumsq);
+                sumsq = __dp4a(w[i].y, w[i].y, sumsq);
+                uint4 o;
+                o.x = cvt2(w[i].x, 0x5140u);
+                o.y = cvt2(w[i].x, 0x5342u);
+                o.z = cvt2(w[i].y, 0x5140u);
+                o.w = cvt2(w[i].y, 0x5342u);
+                const int slice = c >> 3, j = c & 7;  // chunk j of the row goes to position j ^ (row % 8)
+                *reinterpret_cast<uint4*>(tile + slice * kBlockM * kSliceRowBytes + row * kSliceRowBytes +
+                                          ((j ^ (row & 7)) << 4)) = o;
+            }
+        }
+    }
+    // norm columns: A A A 0 ... 0; chunk j of the row goes to position j ^ ((row / 4) % 2)
+    const uint32_t a16 = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(A)));
+    const uint4 aug0 = valid ? make_uint4(a16 | (a16 << 16), a16, 0u, 0u) : make_uint4(0u, 0u, 0u, 0u);
+    const int sw = (row >> 2) & 1;
+    *reinterpret_cast<uint4*>(tile + a_data_bytes + row * kAugRowBytes + ((0 ^ sw) << 4)) = aug0;
+    *reinterpret_cast<uint4*>(tile + a_data_bytes + row * kAugRowBytes + ((1 ^ sw) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+    return sumsq;
+}
+
 template <int EPI, int MT>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_xa,
@@ -419,7 +479,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     const int64_t u1 = span_begin(T, G, b + 1);
 
     if (threadIdx.x == 0) {
-        mbar_init(a_full, 1);
+        mbar_init(a_full, p.x_raw != nullptr ? 4 * MT : 1);  // TMA bytes, or one arrival per widening warp
         mbar_init(a_empty, 1);
         mbar_init(drain, 1);
         for (int i = 0; i < 2; ++i) {
@@ -457,16 +517,32 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     const int kd = p.kslices * kSliceK;  // K column where the norm columns start
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            int it = 0, seg = 0, a_armed = 0;
-            bool ok = true;
-            for (int64_t u = u0; u < u1 && ok;) {
-                const int64_t r = u / NT;
-                const int t0 = static_cast<int>(u - r * NT);
-                const int t1 = static_cast<int>((u1 - r * NT < NT) ? (u1 - r * NT) : NT);
-                if (seg > 0) ok = mbar_wait(a_empty, (seg - 1) & 1, ctl, 1);
-                if (!ok) break;
+        // ------------------------------------------------------------ producer
+        // (uint8 points: the epilogue warps build the point tiles themselves, see below)
+        const bool raw = p.x_raw != nullptr;
+        int it = 0, seg = 0, a_armed = 0;
+        bool ok = true;
+        auto load_b = [&](int t) -> bool {  // lane 0: one centroid tile into the next ring stage
+            const int st = it % p.nstage;
+            const uint32_t ph = (it / p.nstage) & 1;
+            if (!mbar_wait(&b_empty[st], ph ^ 1u, ctl, 2)) return false;
+            mbar_arrive_expect_tx(&b_full[st], stage_bytes);
+            uint8_t* dst = smem_b + static_cast<size_t>(st) * stage_bytes;
+            for (int s = 0; s < p.kslices; ++s)
+                tma_load_2d(dst + s * p.block_n * kSliceRowBytes, &tmap_c, &b_full[st], s * kSliceK, t * p.block_n);
+            tma_load_2d(dst + b_data_bytes, &tmap_ca, &b_full[st], kd, t * p.block_n);
+            ++it;
+            return true;
+        };
+        for (int64_t u = u0; u < u1 && ok;) {
+            const int64_t r = u / NT;
+            const int t0 = static_cast<int>(u - r * NT);
+            const int t1 = static_cast<int>((u1 - r * NT < NT) ? (u1 - r * NT) : NT);
+            if (lane == 0 && seg > 0) ok = mbar_wait(a_empty, (seg - 1) & 1, ctl, 1);
+            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            int t = t0;
+            if (!raw && lane == 0) {
                 mbar_arrive_expect_tx(a_full, MT * a_bytes);
                 ++a_armed;
                 for (int h = 0; h < MT; ++h) {
@@ -476,36 +552,26 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                         tma_load_2d(dst + s * kBlockM * kSliceRowBytes, &tmap_x, a_full, s * kSliceK, y);
                     tma_load_2d(dst + a_data_bytes, &tmap_xa, a_full, kd, y);
                 }
-                for (int t = t0; t < t1; ++t) {
-                    const int st = it % p.nstage;
-                    const uint32_t ph = (it / p.nstage) & 1;
-                    ok = mbar_wait(&b_empty[st], ph ^ 1u, ctl, 2);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(&b_full[st], stage_bytes);
-                    uint8_t* dst = smem_b + static_cast<size_t>(st) * stage_bytes;
-                    for (int s = 0; s < p.kslices; ++s)
-                        tma_load_2d(dst + s * p.block_n * kSliceRowBytes, &tmap_c, &b_full[st], s * kSliceK,
-                                    t * p.block_n);
-                    tma_load_2d(dst + b_data_bytes, &tmap_ca, &b_full[st], kd, t * p.block_n);
-                    ++it;
-                }
-                ++seg;
-                u = r * NT + t1;
             }
-            if (!ok) {
-                // gave up: let the copies already issued land before the CTA goes away (bounded)
-                const uint64_t t_start = global_timer_ns();
-                const int first = it > p.nstage ? it - p.nstage : 0;
-                for (int i = first; i < it; ++i) {
-                    const int st = i % p.nstage;
-                    const uint32_t ph = (i / p.nstage) & 1;
-                    while (!mbar_try_wait(&b_full[st], ph) && global_timer_ns() - t_start < 2000000000ull) {
-                    }
+            if (lane == 0) {
+                for (; t < t1 && ok; ++t) ok = load_b(t);
+            }
+            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+            ++seg;
+            u = r * NT + t1;
+        }
+        if (lane == 0 && !ok) {
+            // gave up: let the copies already issued land before the CTA goes away (bounded)
+            const uint64_t t_start = global_timer_ns();
+            const int first = it > p.nstage ? it - p.nstage : 0;
+            for (int i = first; i < it; ++i) {
+                const int st = i % p.nstage;
+                const uint32_t ph = (i / p.nstage) & 1;
+                while (!mbar_try_wait(&b_full[st], ph) && global_timer_ns() - t_start < 2000000000ull) {
                 }
-                if (a_armed > 0) {
-                    while (!mbar_try_wait(a_full, (a_armed - 1) & 1) &&
-                           global_timer_ns() - t_start < 2000000000ull) {
-                    }
+            }
+            if (a_armed > 0) {
+                while (!mbar_try_wait(a_full, (a_armed - 1) & 1) && global_timer_ns() - t_start < 2000000000ull) {
                 }
             }
         }
@@ -575,6 +641,14 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         const float INF = __int_as_float(0x7f800000);
         const int nq = p.block_n / 64;  // 32-column chunks per warp and tile: 4 or 2
         constexpr bool kHasLog = (EPI == EPI_RUNNING || EPI == EPI_FILTER);
+        float raw_scales[4] = {1.f, 1.f, 1.f, 1.f};
+        if (p.x_raw != nullptr) {
+            compute_scales(p.bits, 1, raw_scales);
+            if (b == 0 && warp == 2 && lane == 0) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) p.scal_out[i] = raw_scales[i];
+            }
+        }
         int it = 0;
         bool ok = true;
         for (int64_t u = u0; u < u1 && ok;) {
@@ -582,6 +656,21 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             const int t0 = static_cast<int>(u - r * NT);
             const int t1 = static_cast<int>((u1 - r * NT < NT) ? (u1 - r * NT) : NT);
             const int slot = (b - cta_of_unit(T, G, r * NT)) * kEpiHalves + half;
+
+            if (p.x_raw != nullptr && half < MT) {
+                // uint8 points: this thread widens its own row of point tile `half`.  The tile is free:
+                // the last accumulator of the previous row group could only be read after every MMA
+                // that used the old tile had completed.
+                const int64_t grow = (r * MT + half) * kBlockM + row_in_tile;
+                const bool v = grow < p.n;
+                const unsigned int sumsq =
+                    widen_row_u8(p.x_raw + static_cast<size_t>(v ? grow : 0) * p.d, v, p.d, kd, smem_a + half * a_bytes,
+                                 a_data_bytes, row_in_tile, raw_scales[0], raw_scales[3]);
+                if (v) p.xn_out[grow] = static_cast<float>(sumsq);
+                fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(a_full);
+            }
 
             RowState<EPI> st[MT];
             int64_t row[MT];

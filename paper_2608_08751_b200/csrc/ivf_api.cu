@@ -378,17 +378,25 @@ int prepare_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, 
 }
 
 struct PointPrep {
-    __half* x16;
+    __half* x16;           // fp16 operand copy (float points), or nullptr
+    const uint8_t* x_raw;  // raw uint8 points, widened inside the fused kernel
+    int d;
     float* xn;
     CUtensorMap tmap_x, tmap_xa;
 };
 
 int launch_fused(DeviceCtx& ctx, const Plan& pl, int64_t n, int nlist, int k, int rule, const float* tau_in,
                  const PointPrep& pp, const CUtensorMap& tmap_c, const CUtensorMap& tmap_ca, Entry* part,
-                 int2* part_meta, int kind, cudaStream_t stream, int* clear0 = nullptr, int* clear1 = nullptr) {
+                 int2* part_meta, int kind, cudaStream_t stream, const unsigned int* bits, float* scal,
+                 int* clear0 = nullptr, int* clear1 = nullptr) {
     FusedParams fp;
     fp.clear0 = clear0;
     fp.clear1 = clear1;
+    fp.x_raw = pp.x_raw;
+    fp.d = pp.d;
+    fp.bits = bits;
+    fp.scal_out = scal;
+    fp.xn_out = pp.xn;
     fp.n = n;
     fp.nlist = nlist;
     fp.k = k;
@@ -493,7 +501,11 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     int* failbuf = nullptr;
     float* fbkeys = nullptr;
     float* tau = nullptr;
-    WS(WS_X16, static_cast<size_t>(n) * pl.kp * sizeof(__half), pp.x16);
+    const int u8 = ptype == IVF_U8;
+    pp.x16 = nullptr;
+    pp.x_raw = u8 ? static_cast<const uint8_t*>(points) : nullptr;
+    pp.d = d;
+    if (!u8) WS(WS_X16, static_cast<size_t>(n) * pl.kp * sizeof(__half), pp.x16);
     WS(WS_XN, static_cast<size_t>(n) * sizeof(float), pp.xn);
     WS(WS_PART, part_bytes, part);
     if (k > 1) {
@@ -503,37 +515,36 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         if (given) WS(WS_TAU, static_cast<size_t>(n) * sizeof(float), tau);
     }
 
-    const int u8 = ptype == IVF_U8;
-    int tk = timing_begin(TK_PREP, stream);
+    int tk = -1;
     if (!u8) {
+        // float points: magnitude, scales and the fp16 operand copy (uint8 points are widened inside
+        // the fused kernel, which also derives the scales and writes |x|^2)
+        tk = timing_begin(TK_PREP, stream);
         CUDA_TRY(cudaMemsetAsync(cp.bits, 0, sizeof(unsigned int), stream));
         const int64_t count = n * d;
         int blocks = static_cast<int>((count + 256 * 8 - 1) / (256 * 8));
         if (blocks > ctx.num_sms * 8) blocks = ctx.num_sms * 8;
         maxabs_kernel<<<blocks, 256, 0, stream>>>(static_cast<const float*>(points), count, cp.bits);
         LAUNCH_CHECK();
-    }
-    // the point conversion derives the scales of this chunk itself (and publishes them in cp.scal)
-    const int64_t threads = n * 32;
-    const unsigned cblocks = static_cast<unsigned>((threads + 255) / 256);
-    if (u8)
-        convert_rows_kernel<uint8_t, false><<<cblocks, 256, 0, stream>>>(static_cast<const uint8_t*>(points), n, d,
-                                                                         pl.kd, cp.scal, pp.x16, pp.xn, cp.bits, 1);
-    else
+        const int64_t threads = n * 32;
+        const unsigned cblocks = static_cast<unsigned>((threads + 255) / 256);
         convert_rows_kernel<float, false><<<cblocks, 256, 0, stream>>>(static_cast<const float*>(points), n, d, pl.kd,
                                                                        cp.scal, pp.x16, pp.xn, cp.bits, 0);
-    LAUNCH_CHECK();
-    timing_end(tk, stream);
-
-    rc = make_tmap(&pp.tmap_x, pp.x16, n, pl.kp, kBlockM, false);
-    if (rc != IVF_OK) return rc;
-    rc = make_tmap(&pp.tmap_xa, pp.x16, n, pl.kp, kBlockM, true);
-    if (rc != IVF_OK) return rc;
+        LAUNCH_CHECK();
+        timing_end(tk, stream);
+        rc = make_tmap(&pp.tmap_x, pp.x16, n, pl.kp, kBlockM, false);
+        if (rc != IVF_OK) return rc;
+        rc = make_tmap(&pp.tmap_xa, pp.x16, n, pl.kp, kBlockM, true);
+        if (rc != IVF_OK) return rc;
+    } else {
+        pp.tmap_x = cp.tmap_c;  // unused in this mode; the kernel parameters must still be valid maps
+        pp.tmap_xa = cp.tmap_ca;
+    }
 
     if (given) {
         // threshold pass over every S-th centroid: the 16th smallest group minimum becomes the row's tau
         rc = launch_fused(ctx, pls, n, cp.sample_rows, kSampleM, TAU_SKETCH, nullptr, pp, cp.tmap_cs, cp.tmap_csa, part,
-                          part_meta, TK_THRESH, stream);
+                          part_meta, TK_THRESH, stream, cp.bits, cp.scal);
         if (rc != IVF_OK) return rc;
         MergeParams ms = merge_params(pls, n, kSampleM, part, part_meta, pp, cp.scal);
         ms.tau_out = tau;
@@ -548,7 +559,8 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         timing_end(tk, stream);
     }
     rc = launch_fused(ctx, pl, n, nlist, k, cp.rule, tau, pp, cp.tmap_c, cp.tmap_ca, part, part_meta,
-                      k == 1 ? TK_FUSED_ARGMIN : TK_FUSED_TOPK, stream, failbuf, failbuf ? failbuf + n + 2 : nullptr);
+                      k == 1 ? TK_FUSED_ARGMIN : TK_FUSED_TOPK, stream, cp.bits, cp.scal, failbuf,
+                      failbuf ? failbuf + n + 2 : nullptr);
     if (rc != IVF_OK) return rc;
 
     MergeParams mp = merge_params(pl, n, k, part, part_meta, pp, cp.scal);
@@ -593,6 +605,9 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
             fb.k = k;
             fb.kp = pl.kp;
             fb.x16 = pp.x16;
+            fb.x_raw = pp.x_raw;
+            fb.d = d;
+            fb.kd = pl.kd;
             fb.c16 = cp.c16;
             fb.xn = pp.xn;
             fb.scal = cp.scal;

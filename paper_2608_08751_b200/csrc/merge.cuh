@@ -558,7 +558,9 @@ struct FallbackParams {
     int nlist;
     int k;
     int kp;                // pitch of the fp16 operand copies
-    const __half* x16;     // [n][kp]
+    const __half* x16;     // [n][kp], or nullptr when the points are raw uint8 rows
+    const uint8_t* x_raw;  // [n][d] uint8 (widened on the fly with the same scales)
+    int d, kd;
     const __half* c16;     // [nlist][kp]
     const float* xn;
     const float* scal;
@@ -590,6 +592,21 @@ __device__ __forceinline__ float fallback_key(const float* xs, const __half* cj,
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
     return acc;
+}
+
+// fp32 copy of one point's operand row (data columns, zero padding, the three norm columns)
+__device__ __forceinline__ void fallback_load_point(const FallbackParams& p, int64_t row, float* xs) {
+    for (int t = threadIdx.x; t < p.kp; t += blockDim.x) {
+        float v;
+        if (p.x16 != nullptr) {
+            v = __half2float(p.x16[row * p.kp + t]);
+        } else {
+            v = 0.0f;
+            if (t < p.d) v = p.scal[0] * static_cast<float>(p.x_raw[row * p.d + t]);
+            else if (t >= p.kd && t < p.kd + 3) v = __half2float(__float2half_rn(p.scal[3]));
+        }
+        xs[t] = v;
+    }
 }
 
 struct FallbackSmem {
@@ -676,7 +693,7 @@ __global__ void __launch_bounds__(kFallbackThreads) fallback_keys_kernel(const F
     const int idx = blockIdx.y;
     if (idx >= nfail) return;
     const int64_t row = p.fail[1 + idx];
-    for (int t = threadIdx.x; t < p.kp; t += blockDim.x) xs[t] = __half2float(p.x16[row * p.kp + t]);
+    fallback_load_point(p, row, xs);
     __syncthreads();
     float* keys = p.keys + static_cast<size_t>(idx) * p.nlist;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -705,7 +722,7 @@ __global__ void __launch_bounds__(kFallbackThreads) fallback_select_kernel(const
     for (int idx = kFallbackFastRows + slow; idx < nfail; idx += nslow) {
         const int64_t row = p.fail[1 + idx];
         __syncthreads();
-        for (int t = threadIdx.x; t < p.kp; t += blockDim.x) sm.xs[t] = __half2float(p.x16[row * p.kp + t]);
+        fallback_load_point(p, row, sm.xs);
         __syncthreads();
         for (int j = warp; j < p.nlist; j += kFallbackThreads / 32) {
             const float key = fallback_key(sm.xs, p.c16 + static_cast<size_t>(j) * p.kp, p.kp, lane);
