@@ -192,6 +192,7 @@ struct Plan {
 
 constexpr size_t kSmemLimit = 227 * 1024;
 constexpr int kFallbackCtas = 32;  // slow-path CTAs of the brute-force recomputation
+inline int fallback_slices(int nlist) { return (nlist + kFallbackSlice - 1) / kFallbackSlice; }
 
 int log_capacity(int k) { return (k == 1) ? 1 : (4 * k > 512 ? 4 * k : 512); }
 
@@ -499,7 +500,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     Entry* part;
     int2* part_meta = nullptr;
     int* failbuf = nullptr;
-    float* fbkeys = nullptr;
+    uint64_t* fbkeys = nullptr;
     float* tau = nullptr;
     const int u8 = ptype == IVF_U8;
     pp.x16 = nullptr;
@@ -511,7 +512,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     if (k > 1) {
         WS(WS_PARTMETA, meta_bytes, part_meta);
         WS(WS_FAIL, 2 * (static_cast<size_t>(n) + 2) * sizeof(int), failbuf);  // failed rows and passed-on rows
-        if (given || g_force_fallback) WS(WS_FBKEYS, static_cast<size_t>(kFallbackFastRows + kFallbackCtas) * nlist * sizeof(float), fbkeys);
+        if (given || g_force_fallback) WS(WS_FBKEYS, static_cast<size_t>(kFallbackFastRows + kFallbackCtas) * fallback_slices(nlist) * k * sizeof(uint64_t), fbkeys);
         if (given) WS(WS_TAU, static_cast<size_t>(n) * sizeof(float), tau);
     }
 
@@ -579,17 +580,23 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         // ties) are listed in `big` and merged by the general CTA-per-row kernel
         // (both list counters were cleared by the fused kernel that just ran)
         mp.big = failbuf + n + 2;
+        // two sizes of the warp-level kernel: up to 1024 candidates / 512 sorted (k <= 128 under the given
+        // rule), up to 2048 / 1024 (k <= 320); beyond that everything goes to the general kernel
+        const int expect = given ? 5 * k : 2 * k;
         if (!ctx.merge_attr_set) {
-            CUDA_TRY(cudaFuncSetAttribute(merge_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          static_cast<int>(kMergeWarps * sizeof(MergeWarpSmem))));
+            CUDA_TRY(cudaFuncSetAttribute(merge_warp_kernel<1024, 512, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(8 * sizeof(MergeWarpSmem<1024>))));
+            CUDA_TRY(cudaFuncSetAttribute(merge_warp_kernel<2048, 1024, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(4 * sizeof(MergeWarpSmem<2048>))));
             ctx.merge_attr_set = true;
         }
-        // about 4k candidates per row pass a given threshold: beyond k = 128 they do not fit the
-        // warp-level buffers, so everything goes to the general kernel directly
-        const bool try_warp = !(given && 5 * k > kWarpKeys);  // (k <= 16 lets ~256 through: fits)
-        if (try_warp) {
-            merge_warp_kernel<<<static_cast<unsigned>((n + kMergeWarps - 1) / kMergeWarps), 32 * kMergeWarps,
-                                kMergeWarps * sizeof(MergeWarpSmem), stream>>>(mp);
+        if (expect <= 700) {
+            merge_warp_kernel<1024, 512, 8><<<static_cast<unsigned>((n + 7) / 8), 256, 8 * sizeof(MergeWarpSmem<1024>),
+                                              stream>>>(mp);
+            LAUNCH_CHECK();
+        } else if (expect <= 1700) {
+            merge_warp_kernel<2048, 1024, 4><<<static_cast<unsigned>((n + 3) / 4), 128, 4 * sizeof(MergeWarpSmem<2048>),
+                                               stream>>>(mp);
             LAUNCH_CHECK();
         } else {
             mp.big = nullptr;
@@ -612,10 +619,11 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
             fb.xn = pp.xn;
             fb.scal = cp.scal;
             fb.fail = failbuf;
-            fb.keys = fbkeys;
+            fb.cand = fbkeys;
+            fb.slices = fallback_slices(nlist);
             fb.out_ids = out_ids;
             fb.out_dists = out_dists;
-            fallback_keys_kernel<<<dim3(kFallbackKeyChunks, kFallbackFastRows), kFallbackThreads, 0, stream>>>(fb);
+            fallback_keys_kernel<<<dim3(static_cast<unsigned>(fb.slices), kFallbackFastRows), kFallbackThreads, 0, stream>>>(fb);
             LAUNCH_CHECK();
             fallback_select_kernel<<<kFallbackFastRows + kFallbackCtas, kFallbackThreads, 0, stream>>>(fb);
             LAUNCH_CHECK();

@@ -304,13 +304,12 @@ __global__ void __launch_bounds__(kMergeThreads) merge_select_kernel(const Merge
 // partial logs and at most kWarpKeys candidates <= tau: the candidates go to the warp's slice of
 // shared memory, an 8-bit radix select on the key's value finds the k-th smallest, and only the
 // keys up to it are sorted.  Other rows are appended to p.big for merge_select_kernel.
-constexpr int kWarpKeys = 1024;
 constexpr int kWarpSlots = 64;
-constexpr int kWarpSort = 512;
-constexpr int kMergeWarps = 8;
 
+// Two sizes: KEYS candidates per row at most, SORT keys sorted at most, WARPS rows per CTA.
+template <int KEYS>
 struct MergeWarpSmem {
-    uint64_t keys[kWarpKeys];
+    uint64_t keys[KEYS];
     int hist[256];
     int pre[kWarpSlots + 1];
 };
@@ -334,11 +333,13 @@ __device__ __forceinline__ void warp_bitonic_sort(uint64_t* keys, int m, int lan
     __syncwarp();
 }
 
-__global__ void __launch_bounds__(32 * kMergeWarps) merge_warp_kernel(const MergeParams p) {
+template <int KEYS, int SORT, int WARPS>
+__global__ void __launch_bounds__(32 * WARPS) merge_warp_kernel(const MergeParams p) {
     extern __shared__ __align__(16) uint8_t merge_smem_raw[];
+    constexpr int kWarpKeys = KEYS, kWarpSort = SORT;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    MergeWarpSmem& sm = reinterpret_cast<MergeWarpSmem*>(merge_smem_raw)[warp];
-    const int64_t row = static_cast<int64_t>(blockIdx.x) * kMergeWarps + warp;
+    MergeWarpSmem<KEYS>& sm = reinterpret_cast<MergeWarpSmem<KEYS>*>(merge_smem_raw)[warp];
+    const int64_t row = static_cast<int64_t>(blockIdx.x) * WARPS + warp;
     if (row >= p.n) return;
     const uint32_t FULL = 0xFFFFFFFFu;
     const uint32_t lt_mask = (1u << lane) - 1u;
@@ -554,6 +555,11 @@ __global__ void __launch_bounds__(256) merge_tau_warp_kernel(const MergeParams p
 }
 
 // ------------------------------------------------------------------ brute-force recomputation
+// A row whose threshold admitted fewer than k candidates (or that was forced here by a test hook) is
+// recomputed exactly: all nlist keys with the MMA's own contraction in fp32 FMA, then the k smallest
+// by (key, id).  Two stages so that one failed row still uses many SMs: every CTA takes a slice of
+// kFallbackSlice centroids, keeps the slice's keys in shared memory and emits the slice's k smallest
+// (key, id) pairs; a second CTA selects the k smallest of those candidates and sorts them.
 struct FallbackParams {
     int nlist;
     int k;
@@ -565,34 +571,24 @@ struct FallbackParams {
     const float* xn;
     const float* scal;
     const int* fail;       // fail[0] = count, fail[1..] = rows
-    float* keys;           // [kFallbackFastRows + slow-path CTAs][nlist] scratch
+    uint64_t* cand;        // [kFallbackFastRows + slow-path CTAs][slices * k] candidate pairs
+    int slices;            // ceil(nlist / kFallbackSlice)
     int32_t* out_ids;
     float* out_dists;
 };
 
 constexpr int kFallbackThreads = 256;
 constexpr int kFallbackMaxK = 512;
-constexpr int kFallbackFastRows = 16;   // failed rows whose keys are computed by the whole grid
-constexpr int kFallbackKeyChunks = 128; // CTAs per row in that case
+constexpr int kFallbackFastRows = 16;  // failed rows whose slices are spread over the grid
+constexpr int kFallbackSlice = 8192;   // centroids per slice
 
-// key of point row `xs` (fp32 copy of its fp16 operand row, in shared memory) against centroid j:
-// the same contraction as the MMA, in fp32 FMA.  One warp per centroid.
-__device__ __forceinline__ float fallback_key(const float* xs, const __half* cj, int kp, int lane) {
-    float acc = 0.0f;
-    for (int t = lane * 8; t < kp; t += 256) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(cj + t);
-        const __half2* h = reinterpret_cast<const __half2*>(&raw);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const float2 f = __half22float2(h[q]);
-            acc = fmaf(xs[t + 2 * q], f.x, acc);
-            acc = fmaf(xs[t + 2 * q + 1], f.y, acc);
-        }
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
-    return acc;
-}
+struct FallbackSmem {
+    float xs[288];
+    float keys[kFallbackSlice];
+    uint64_t top[kFallbackMaxK];
+    int hist[256];
+    int cnt, digit, rank, eq;
+};
 
 // fp32 copy of one point's operand row (data columns, zero padding, the three norm columns)
 __device__ __forceinline__ void fallback_load_point(const FallbackParams& p, int64_t row, float* xs) {
@@ -609,75 +605,138 @@ __device__ __forceinline__ void fallback_load_point(const FallbackParams& p, int
     }
 }
 
-struct FallbackSmem {
-    float xs[288];
-    int hist[256];
-    int scan[kFallbackThreads];
-    uint64_t cand[kFallbackMaxK];
-    int cnt, digit, rank;
-};
+// Keys of centroids [j0, j1) against the point row in xs, into keys[0 .. j1-j0).  One warp per
+// centroid, four centroids in flight per warp.
+__device__ __forceinline__ void fallback_slice_keys(const FallbackParams& p, const float* xs, int j0, int j1,
+                                                    float* keys) {
+    constexpr int kInFlight = 4;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nwarps = blockDim.x >> 5;
+    for (int jb = j0 + warp * kInFlight; jb < j1; jb += nwarps * kInFlight) {
+        float acc[kInFlight];
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) acc[u] = 0.0f;
+        for (int t = lane * 8; t < p.kp; t += 256) {
+            uint4 raw[kInFlight];
+#pragma unroll
+            for (int u = 0; u < kInFlight; ++u) {
+                const int j = min(jb + u, j1 - 1);
+                raw[u] = *reinterpret_cast<const uint4*>(p.c16 + static_cast<size_t>(j) * p.kp + t);
+            }
+#pragma unroll
+            for (int u = 0; u < kInFlight; ++u) {
+                const __half2* h = reinterpret_cast<const __half2*>(&raw[u]);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float2 f = __half22float2(h[q]);
+                    acc[u] = fmaf(xs[t + 2 * q], f.x, acc[u]);
+                    acc[u] = fmaf(xs[t + 2 * q + 1], f.y, acc[u]);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) acc[u] += __shfl_xor_sync(0xFFFFFFFFu, acc[u], off);
+            if (lane == 0 && jb + u < j1) keys[jb + u - j0] = acc[u];
+        }
+    }
+}
 
-// Exact top-k of keys[0..nlist) by (key, id): 8-bit radix select for the k-th smallest key, ties to
-// the lower id, then a sort of the k winners; writes the row's outputs.  One CTA.
-__device__ void fallback_select_row(const FallbackParams& p, const float* keys, int64_t row, FallbackSmem& sm) {
-    uint32_t prefix = 0, mask = 0;
-    int rank = p.k;
-    for (int shift = 24; shift >= 0; shift -= 8) {
+// Block-wide selection of the k smallest of `count` distinct 64-bit items (get(i), i < count): radix
+// select from the top byte down, stopping as soon as the digit that holds rank k is wanted whole;
+// returns the largest admitted item (every item <= it is among the k smallest, and there are
+// exactly min(k, count) of those).  Histogram increments are combined per warp, because the keys of
+// one row share their leading bytes.
+template <typename Get>
+__device__ __forceinline__ uint64_t fallback_select_bound(Get get, int count, int k, FallbackSmem& sm) {
+    if (count <= k) return ~0ull;
+    const int lane = threadIdx.x & 31;
+    uint64_t prefix = 0, mask = 0;
+    int rank = k;
+    const int rounded = (count + 31) & ~31;
+    for (int shift = 56; shift >= 0; shift -= 8) {
         for (int i = threadIdx.x; i < 256; i += blockDim.x) sm.hist[i] = 0;
         __syncthreads();
-        for (int j = threadIdx.x; j < p.nlist; j += blockDim.x) {
-            const uint32_t u = orderable(keys[j]);
-            if ((u & mask) == prefix) atomicAdd(&sm.hist[(u >> shift) & 255u], 1);
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            int acc = 0, dgt = 255, r = rank;
-            for (int b = 0; b < 256; ++b) {
-                if (rank <= acc + sm.hist[b]) {
-                    dgt = b;
-                    r = rank - acc;
-                    break;
-                }
-                acc += sm.hist[b];
+        for (int i = threadIdx.x; i < rounded; i += blockDim.x) {
+            uint32_t dg = 0xFFFFFFFFu;
+            if (i < count) {
+                const uint64_t v = get(i);
+                if ((v & mask) == prefix) dg = static_cast<uint32_t>(v >> shift) & 255u;
             }
-            sm.digit = dgt;
-            sm.rank = r;
+            const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dg);
+            if (dg != 0xFFFFFFFFu && lane == __ffs(peers) - 1) atomicAdd(&sm.hist[dg], __popc(peers));
         }
         __syncthreads();
-        prefix |= static_cast<uint32_t>(sm.digit) << shift;
-        mask |= 255u << shift;
+        if (threadIdx.x < 32) {
+            int r = rank, eq = 0;
+            const int digit = radix_pick_digit(sm.hist, lane, r, eq);
+            if (lane == 0) {
+                sm.digit = digit;
+                sm.rank = r;
+                sm.eq = eq;
+            }
+        }
+        __syncthreads();
+        prefix |= static_cast<uint64_t>(sm.digit) << shift;
+        mask |= 255ull << shift;
         rank = sm.rank;
+        const bool whole = sm.eq == rank;
         __syncthreads();
+        if (whole) return prefix | ~mask;
     }
-    const uint32_t Tk = prefix;  // `rank` of the keys equal to Tk are wanted, lowest ids first
+    return prefix;
+}
+
+__device__ __forceinline__ int fallback_slice_len(const FallbackParams& p, int slice) {
+    return min(kFallbackSlice, p.nlist - slice * kFallbackSlice);
+}
+
+// Stage 1 for one slice: keys into shared memory, the slice's min(k, len) smallest (key, id) pairs
+// into out[0 .. min(k, len)) in no particular order.
+__device__ __forceinline__ void fallback_slice(const FallbackParams& p, int slice, uint64_t* out, FallbackSmem& sm) {
+    const int j0 = slice * kFallbackSlice, len = fallback_slice_len(p, slice);
+    fallback_slice_keys(p, sm.xs, j0, j0 + len, sm.keys);
     if (threadIdx.x == 0) sm.cnt = 0;
-    const int per = (p.nlist + blockDim.x - 1) / blockDim.x;
-    const int j0 = min(p.nlist, static_cast<int>(threadIdx.x) * per), j1 = min(p.nlist, j0 + per);
-    int eq = 0;
-    for (int j = j0; j < j1; ++j) eq += orderable(keys[j]) == Tk;
-    sm.scan[threadIdx.x] = eq;
     __syncthreads();
-    int before = 0;
-    for (int t = 0; t < static_cast<int>(threadIdx.x); ++t) before += sm.scan[t];
-    for (int j = j0; j < j1; ++j) {
-        const uint32_t u = orderable(keys[j]);
-        bool take = u < Tk;
-        if (u == Tk) {
-            take = before < rank;
-            ++before;
-        }
-        if (take) sm.cand[atomicAdd(&sm.cnt, 1)] = (static_cast<uint64_t>(u) << 32) | static_cast<uint32_t>(j);
+    auto get = [&](int i) { return (static_cast<uint64_t>(orderable(sm.keys[i])) << 32) | static_cast<uint32_t>(j0 + i); };
+    const uint64_t bound = fallback_select_bound(get, len, p.k, sm);
+    for (int i = threadIdx.x; i < len; i += blockDim.x) {
+        const uint64_t v = get(i);
+        if (v <= bound) out[atomicAdd(&sm.cnt, 1)] = v;
     }
     __syncthreads();
-    const int got = sm.cnt;  // == k
+}
+
+// Stage 2: the k smallest of a row's candidates (slot s of k per slice, the first min(k, len_s) of
+// each filled), sorted, to the row's outputs.
+__device__ __forceinline__ void fallback_finish_row(const FallbackParams& p, const uint64_t* cand, int64_t row,
+                                                    FallbackSmem& sm) {
+    const int total = p.slices * p.k;
+    auto get = [&](int i) {
+        const int s = i / p.k, r = i - s * p.k;
+        return r < fallback_slice_len(p, s) ? __ldcg(cand + i) : ~0ull;
+    };
+    const uint64_t bound = fallback_select_bound(get, total, p.k, sm);
+    if (threadIdx.x == 0) sm.cnt = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < total; i += blockDim.x) {
+        const uint64_t v = get(i);
+        if (v <= bound && v != ~0ull) {
+            const int at = atomicAdd(&sm.cnt, 1);
+            if (at < kFallbackMaxK) sm.top[at] = v;
+        }
+    }
+    __syncthreads();
+    const int got = min(sm.cnt, kFallbackMaxK);  // == k
     int m = 2;
     while (m < got) m <<= 1;
-    for (int i = got + threadIdx.x; i < m; i += blockDim.x) sm.cand[i] = ~0ull;
-    bitonic_sort_smem(sm.cand, m);
+    for (int i = got + threadIdx.x; i < m; i += blockDim.x) sm.top[i] = ~0ull;
+    bitonic_sort_smem(sm.top, m);
     const float xn = p.xn[row];
     const float inv = p.scal[2];
     for (int i = threadIdx.x; i < p.k; i += blockDim.x) {
-        const uint64_t key = sm.cand[i];
+        const uint64_t key = sm.top[i];
         p.out_ids[row * p.k + i] = static_cast<int32_t>(key & 0xFFFFFFFFull);
         if (p.out_dists)
             p.out_dists[row * p.k + i] = fmaxf(fmaf(from_orderable(static_cast<uint32_t>(key >> 32)), inv, xn), 0.0f);
@@ -685,51 +744,36 @@ __device__ void fallback_select_row(const FallbackParams& p, const float* keys, 
     __syncthreads();
 }
 
-// The first kFallbackFastRows failed rows: grid (kFallbackKeyChunks, kFallbackFastRows); every CTA
-// computes one slice of one row's keys, so a single failed row still uses the whole GPU.
+// The first kFallbackFastRows failed rows: grid (slices, kFallbackFastRows), one slice of one row per CTA.
 __global__ void __launch_bounds__(kFallbackThreads) fallback_keys_kernel(const FallbackParams p) {
-    __shared__ float xs[288];
+    __shared__ FallbackSmem sm;
     const int nfail = p.fail[0];
     const int idx = blockIdx.y;
     if (idx >= nfail) return;
-    const int64_t row = p.fail[1 + idx];
-    fallback_load_point(p, row, xs);
+    fallback_load_point(p, p.fail[1 + idx], sm.xs);
     __syncthreads();
-    float* keys = p.keys + static_cast<size_t>(idx) * p.nlist;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int per = (p.nlist + gridDim.x - 1) / gridDim.x;
-    const int j0 = blockIdx.x * per, j1 = min(p.nlist, j0 + per);
-    for (int j = j0 + warp; j < j1; j += kFallbackThreads / 32) {
-        const float key = fallback_key(xs, p.c16 + static_cast<size_t>(j) * p.kp, p.kp, lane);
-        if (lane == 0) keys[j] = key;
-    }
+    fallback_slice(p, blockIdx.x, p.cand + (static_cast<size_t>(idx) * p.slices + blockIdx.x) * p.k, sm);
 }
 
-// Blocks [0, kFallbackFastRows) select from the keys that fallback_keys_kernel prepared.  The other
-// blocks take any further failed rows (none in practice), one CTA per row doing both steps: slow
-// and exact.
+// Blocks [0, kFallbackFastRows) finish the rows whose candidates fallback_keys_kernel prepared.  The
+// other blocks take any further failed rows (none in practice), one CTA per row doing both stages.
 __global__ void __launch_bounds__(kFallbackThreads) fallback_select_kernel(const FallbackParams p) {
     __shared__ FallbackSmem sm;
     const int nfail = p.fail[0];
     if (blockIdx.x < kFallbackFastRows) {
         const int idx = blockIdx.x;
-        if (idx < nfail) fallback_select_row(p, p.keys + static_cast<size_t>(idx) * p.nlist, p.fail[1 + idx], sm);
+        if (idx < nfail) fallback_finish_row(p, p.cand + static_cast<size_t>(idx) * p.slices * p.k, p.fail[1 + idx], sm);
         return;
     }
     const int slow = blockIdx.x - kFallbackFastRows, nslow = gridDim.x - kFallbackFastRows;
-    float* keys = p.keys + static_cast<size_t>(kFallbackFastRows + slow) * p.nlist;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint64_t* cand = p.cand + static_cast<size_t>(kFallbackFastRows + slow) * p.slices * p.k;
     for (int idx = kFallbackFastRows + slow; idx < nfail; idx += nslow) {
         const int64_t row = p.fail[1 + idx];
         __syncthreads();
         fallback_load_point(p, row, sm.xs);
         __syncthreads();
-        for (int j = warp; j < p.nlist; j += kFallbackThreads / 32) {
-            const float key = fallback_key(sm.xs, p.c16 + static_cast<size_t>(j) * p.kp, p.kp, lane);
-            if (lane == 0) keys[j] = key;
-        }
-        __syncthreads();
-        fallback_select_row(p, keys, row, sm);
+        for (int s = 0; s < p.slices; ++s) fallback_slice(p, s, cand + static_cast<size_t>(s) * p.k, sm);
+        fallback_finish_row(p, cand, row, sm);
     }
 }
 

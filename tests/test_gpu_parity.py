@@ -106,6 +106,18 @@ def test_brute_force_recomputation_of_failed_rows(n, nlist, d, k, dtype):
     parity.check_route(q, ci, 50, ids, dists, exact=True)
 
 
+def test_brute_force_recomputation_with_ties_across_slices():
+    # integer data (many equal distances), several centroid slices with a ragged last one, the
+    # largest k: the (distance, id) order must survive both selection stages
+    q, ci = synth.integer_case(40, 20000, 64, seed=5)
+    B.ivf_debug_force_fallback(True)
+    try:
+        ids, dists = _route(q, ci, 512)
+    finally:
+        B.ivf_debug_force_fallback(False)
+    parity.check_route(q, ci, 512, ids, dists, exact=True)
+
+
 @pytest.mark.parametrize("k", [1, 8, 40])
 def test_row_chunk_loop_of_large_calls(k):
     # big calls are split into row chunks that share the prepared centroids and the workspace;
