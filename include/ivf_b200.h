@@ -5,7 +5,7 @@
  * point matrix to every centroid, with the k smallest per row kept on the device:
  *   - coarse search (Eq. 1): the P nearest lists of each query, P = nprobe;
  *   - distances come from inner products and precomputed norms,
- *     |x-c|^2 = |x|^2 + |c|^2 - 2 x.c  (Sec. 4.1, Eq. 3), as a dense tensor-core contraction;
+ *     |x-c|^2 = |x|^2 + |c|^2 - 2 x.c  (Sec. 4.1, Eq. 6), as a dense tensor-core contraction;
  *   - only ids and optional distances, O(B*P), leave the kernel (Sec. 4.1, on-device list
  *     selection); the B x N_list distance matrix is never written to memory;
  *   - index construction assigns every vector to its nearest centroid (Sec. 3.1, Sec. 5.5) -- the

@@ -9,7 +9,7 @@
  * Everything is fp64, written from the definitions:
  *   - coarse search (Eq. 1): the P-subset of lists minimising the summed distance to
  *     the query, i.e. the P nearest centroids;
- *   - the distance is squared L2.  Sec. 4.1 (Eq. 3) expands it as
+ *   - the distance is squared L2.  Sec. 4.1 (Eq. 6, the norm expansion) writes it as
  *     |q|^2 + |c|^2 - 2 q.c, an algebraic identity; the oracle deliberately uses the
  *     direct difference form sum_t (x_t - c_t)^2 instead;
  *   - selection is a full sort on (distance, id), ties broken by the lower id;

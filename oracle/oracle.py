@@ -14,6 +14,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "ivf_oracle.c")
+_SRC_PQ = os.path.join(_HERE, "pq_oracle.c")
 _LIB = os.path.join(_HERE, "libivf_oracle.so")
 
 F32, U8 = 0, 1
@@ -22,10 +23,11 @@ _lib = None
 
 def build(force: bool = False) -> str:
     """Compile the oracle's C file into a shared object next to it."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    newest = max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_PQ))
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest:
         tmp = _LIB + f".{os.getpid()}.tmp"
         subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared",
-                               "-ffp-contract=off", _SRC, "-o", tmp, "-lm"])
+                               "-ffp-contract=off", _SRC, _SRC_PQ, "-o", tmp, "-lm"])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -44,6 +46,13 @@ def _load():
         _lib.oracle_reorder.argtypes = [vp, i64, i32, vp, vp]
         _lib.oracle_lloyd.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, i32, ctypes.c_int, vp, vp, vp]
         _lib.oracle_num_threads.restype = ctypes.c_int
+        _lib.oracle_pq_lut.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, vp]
+        _lib.oracle_pq_lut.restype = None
+        _lib.oracle_pq_adc.argtypes = [vp, ctypes.c_int, vp, i64, i64, vp]
+        _lib.oracle_pq_adc.restype = None
+        _lib.oracle_pq_encode.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, vp, vp, i32, vp, ctypes.c_int, vp]
+        _lib.oracle_pq_search.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, vp, i32, vp, ctypes.c_int, vp, vp,
+                                          vp, ctypes.c_int, ctypes.c_int, vp, vp, vp]
     return _lib
 
 
@@ -165,3 +174,65 @@ def lloyd(x: np.ndarray, init_centroids: np.ndarray, iters: int):
     if rc != 0:
         raise ValueError("oracle_lloyd failed")
     return c, ids, inertia
+
+
+# ---------------------------------------------------------------- residual-PQ candidate reduction
+def _codebooks(cb: np.ndarray, d: int):
+    """codebooks [pq_m, 256, d // pq_m] float32"""
+    if cb.dtype != np.float32 or cb.ndim != 3 or cb.shape[1] != 256 or cb.shape[0] * cb.shape[2] != d:
+        raise TypeError("codebooks must be float32 [pq_m, 256, d / pq_m]")
+    return np.ascontiguousarray(cb), cb.shape[0]
+
+
+def pq_lut(r: np.ndarray, codebooks: np.ndarray) -> np.ndarray:
+    """float32 [pq_m, 256] table of one residual r [d] (float32)."""
+    r = np.ascontiguousarray(r, np.float32)
+    cb, m = _codebooks(codebooks, r.shape[0])
+    lut = np.empty((m, 256), np.float32)
+    _load().oracle_pq_lut(_p(r), r.shape[0], m, _p(cb), _p(lut))
+    return lut
+
+
+def pq_adc(lut: np.ndarray, codes: np.ndarray) -> np.ndarray:
+    """float32 ADC estimates of codes [n, pq_m] (uint8) with one table."""
+    lut = np.ascontiguousarray(lut, np.float32)
+    codes = np.ascontiguousarray(codes, np.uint8)
+    est = np.empty((codes.shape[0],), np.float32)
+    _load().oracle_pq_adc(_p(lut), lut.shape[0], _p(codes), 0, codes.shape[0], _p(est))
+    return est
+
+
+def pq_encode(x: np.ndarray, ids: np.ndarray, c: np.ndarray, codebooks: np.ndarray) -> np.ndarray:
+    """uint8 [n, pq_m]: residual-PQ codes of the rows of x, row i assigned to list ids[i]."""
+    x, xt = _rows(x)
+    c = _cent(c)
+    n, d = x.shape
+    cb, m = _codebooks(codebooks, d)
+    ids = np.ascontiguousarray(ids, np.int32)
+    codes = np.empty((n, m), np.uint8)
+    rc = _load().oracle_pq_encode(_p(x), xt, n, d, _p(ids), _p(c), c.shape[0], _p(cb), m, _p(codes))
+    if rc != 0:
+        raise ValueError("oracle_pq_encode: bad arguments")
+    return codes
+
+
+def pq_search(q: np.ndarray, c: np.ndarray, probes: np.ndarray, offsets: np.ndarray, codes: np.ndarray,
+              codebooks: np.ndarray, n_rerank: int):
+    """(pos int64 [nq, n_rerank], est float32 [nq, n_rerank], count int64 [nq]): the n_rerank smallest
+    ADC estimates over the codes of every query's probed lists, ascending (estimate, position)."""
+    q, qt = _rows(q)
+    c = _cent(c)
+    nq, d = q.shape
+    cb, m = _codebooks(codebooks, d)
+    probes = np.ascontiguousarray(probes, np.int32)
+    offsets = np.ascontiguousarray(offsets, np.int64)
+    codes = np.ascontiguousarray(codes, np.uint8)
+    assert probes.shape[0] == nq and offsets.shape[0] == c.shape[0] + 1 and codes.shape[1] == m
+    pos = np.empty((nq, n_rerank), np.int64)
+    est = np.empty((nq, n_rerank), np.float32)
+    count = np.empty((nq,), np.int64)
+    rc = _load().oracle_pq_search(_p(q), qt, nq, d, _p(c), c.shape[0], _p(probes), probes.shape[1], _p(offsets),
+                                  _p(codes), _p(cb), m, n_rerank, _p(pos), _p(est), _p(count))
+    if rc != 0:
+        raise ValueError("oracle_pq_search: bad arguments")
+    return pos, est, count

@@ -1,7 +1,7 @@
-// Fused distance + per-row top-k kernel (Sec. 4.1: dense centroid evaluation by Eq. 3 and
+// Fused distance + per-row top-k kernel (Sec. 4.1: dense centroid evaluation by Eq. 6 and
 // on-device list selection; Sec. 3.1 / 5.5: assignment is the k = 1 case).
 //
-// The whole ranking key of Eq. 3 comes out of the tensor core: the operand copies carry 16 extra
+// The whole ranking key of Eq. 6 comes out of the tensor core: the operand copies carry 16 extra
 // K columns, so that  acc = sum_t x'_t c''_t + A (w_hi + w_mid + w_lo) = sx sc (|c|^2 - 2 x.c)
 // with x' = sx x, c'' = -2 sc c, w = sc^2 |c|^2 / 2^15 split into three fp16 parts and
 // A = 2^15 sx / sc (sx, sc exact powers of two).  The epilogue only compares.

@@ -1,7 +1,7 @@
 // Second stage of the on-device list selection (Sec. 4.1: tile-local candidates are merged on the
 // device): the partial results left by the CTAs (and epilogue warps) that shared a row are merged
 // into the final k ids per row, ascending by (distance, id); the key is rescaled and the point norm
-// added back (Eq. 3: |x-c|^2 = |x|^2 + (|c|^2 - 2 x.c)).
+// added back (Eq. 6: |x-c|^2 = |x|^2 + (|c|^2 - 2 x.c)).
 //
 // For k > 16 the candidate logs were filled against per-partial thresholds tau_p.  Every element
 // with key < tau_p is in log p, and enough of the elements equal to tau_p, so the union of the logs

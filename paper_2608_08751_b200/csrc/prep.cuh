@@ -1,5 +1,5 @@
-// Operand preparation for the distance contraction (Sec. 4.1, Eq. 3: "inner products and
-// precomputed norms").  Norms are accumulated in fp32 from the unrounded inputs.  The tensor-core
+// Operand preparation for the distance contraction (Sec. 4.1, Eq. 6: the distance is
+// assembled from an inner product and norms computed beforehand).  Norms are accumulated in fp32 from the unrounded inputs.  The tensor-core
 // operands are fp16 copies scaled by exact powers of two chosen from the largest magnitudes, so
 // nothing overflows and small-magnitude data keeps its 11 significant bits; uint8 values are exact.
 //

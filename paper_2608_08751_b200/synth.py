@@ -153,3 +153,42 @@ def integer_case(nq: int, nlist: int, d: int, seed: int, hi: int = 256):
     q = rng.integers(0, hi, size=(nq, d)).astype(np.uint8)
     c = rng.integers(0, hi, size=(nlist, d)).astype(np.float32)
     return q, c
+
+
+# ------------------------------------------------------------------ residual-PQ inputs (stream ids 5-8)
+def pq_codebooks(pq_m: int, dsub: int, scale: float, seed: int, integer: bool = False) -> np.ndarray:
+    """float32 [pq_m, 256, dsub] codebooks: i.i.d. N(0, scale^2) entries (rounded to integers on
+    request).  A stand-in for trained codebooks with the spread of the residuals they quantise."""
+    cb = _rng(5, seed).normal(0.0, scale, size=(pq_m, 256, dsub))
+    if integer:
+        cb = np.rint(cb)
+    return cb.astype(np.float32)
+
+
+def skewed_list_ids(n: int, nlist: int, seed: int, sigma: float = 1.0):
+    """(ids int32 [n] in list-major (sorted) order, offsets int64 [nlist + 1]): list lengths drawn
+    from a multinomial with log-normal weights, so they vary by more than an order of magnitude
+    and some lists may be empty, as inverted lists do."""
+    rng = _rng(6, seed)
+    w = rng.lognormal(0.0, sigma, size=nlist)
+    counts = rng.multinomial(n, w / w.sum())
+    offsets = np.zeros(nlist + 1, np.int64)
+    np.cumsum(counts, out=offsets[1:])
+    ids = np.repeat(np.arange(nlist, dtype=np.int32), counts)
+    return ids, offsets
+
+
+def rows_near(c: np.ndarray, ids: np.ndarray, noise_std: float, seed: int, dtype: str = "f32") -> np.ndarray:
+    """Rows drawn around given centroid rows: c[ids] + N(0, noise_std^2); 'u8' rounds and clips."""
+    rng = _rng(7, seed)
+    x = c[ids] + rng.normal(0.0, noise_std, size=(len(ids), c.shape[1])).astype(np.float32)
+    return _to_u8(x) if dtype == "u8" else x.astype(np.float32)
+
+
+def distinct_probes(nq: int, nlist: int, nprobe: int, seed: int) -> np.ndarray:
+    """int32 [nq, nprobe]: nprobe distinct list ids per query, uniformly drawn, in random order."""
+    rng = _rng(8, seed)
+    out = np.empty((nq, nprobe), np.int32)
+    for b in range(nq):
+        out[b] = rng.choice(nlist, size=nprobe, replace=False)
+    return out
