@@ -207,10 +207,10 @@ int ivf_debug_rule(int k, int nlist, int out[2]);
 
 /*
  * Measurement hooks.  ivf_debug_timing(1) makes every later call bracket its kernels with CUDA
- * events on the caller's stream, grouped into six families: 0 operand preparation (norms,
+ * events on the caller's stream, grouped into nine families: 0 operand preparation (norms,
  * fp16 copies), 1 fused distance+argmin (k = 1), 2 fused distance+top-k (k > 1), 3 merge of
  * partial results (and the brute-force recomputation of failed rows), 4 centroid update,
- * 5 threshold pass of k > 16 calls (fused kernel over the centroid sample + its merge).  ivf_debug_timing_read synchronises the device, writes the
+ * 5 threshold pass of k > 16 calls (fused kernel over the centroid sample + its merge), 6 PQ encoding, 7 PQ set-up + scan, 8 PQ group merge.  ivf_debug_timing_read synchronises the device, writes the
  * summed milliseconds and launch-group counts of each family since the last read, and clears
  * them.  ivf_debug_timing(0) switches the events off (the default).
  */
@@ -221,7 +221,44 @@ int ivf_debug_rule(int k, int nlist, int out[2]);
  */
 int ivf_debug_stats(int enable, int64_t out[3]);
 int ivf_debug_timing(int enable);
-int ivf_debug_timing_read(double ms[6], int64_t launches[6]);
+int ivf_debug_timing_read(double ms[9], int64_t launches[9]);
+
+/*
+ * Residual-PQ candidate reduction (Sec. 2.2 Eq. 3-5; Sec. 4.3; Sec. 4.4).  K = 256 codewords per
+ * subspace, one byte per sub-code, fp32 lookup tables (the paper's setting).  All pointers are
+ * DEVICE pointers owned by the caller; calls enqueue on `stream` and return.
+ *
+ * Arithmetic (fp32, every operation rounded once, in this order, so codes and kept candidates are
+ * reproducible bit for bit):
+ *     r_t = float(x_t) - c_t;   LUT_m[j]: acc = 0, for t ascending: diff = r_t - p_m[j][t],
+ *     acc = fma(diff, diff, acc);   estimate: acc = 0, for m ascending: acc = acc + LUT_m[a_m].
+ *
+ * codebooks  [pq_m][256][d / pq_m] float32, row-major.  pq_m must divide d, and
+ *            1024 * (d + pq_m) + 4 * d + 17,472 bytes of shared memory must fit one SM's 227 KB
+ *            (d = 128 with pq_m = 32 does; d = 256 does not) -> IVF_ERR_UNSUPPORTED otherwise.
+ *
+ * ivf_pq_encode: out_codes[i][m] = arg-min over j of the table of x_i - centroids[ids[i]]
+ *            (Eq. 3 on the residual; ties to the lower j).  An id outside [0, nlist) writes zero
+ *            codes for that row and sets the sticky status IVF_ERR_BAD_ID.
+ *
+ * ivf_pq_search: for every query the codes of its nprobe probed lists (list l = positions
+ *            [list_offsets[l], list_offsets[l+1]) of the list-major `codes` array, n_codes rows in
+ *            all, n_codes < 2^32) are scored with the (query, list) table (Eq. 4 on q - c_l, Eq. 5) and
+ *            the n_rerank (<= 1024) smallest estimates are kept: out_ids [nq][n_rerank] = position
+ *            (or vec_ids[position] when vec_ids is given), out_est [nq][n_rerank] ascending by
+ *            (estimate, position); unused slots hold -1 and +inf.  out_counts [nq] (may be NULL) =
+ *            codes scanned for the query.  A list must not appear twice among a query's probes;
+ *            probe ids outside [0, nlist) are skipped and set IVF_ERR_BAD_ID.  `codes` must be
+ *            16-byte aligned.  Chunk and group descriptors are built on the device (no host
+ *            synchronisation); the workspace is the library's grow-only one.
+ */
+int ivf_pq_encode(const void* points, int64_t n, int d, ivf_dtype ptype, const int32_t* ids,
+                  const float* centroids, int nlist, const float* codebooks, int pq_m,
+                  uint8_t* out_codes, void* stream);
+int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const float* centroids, int nlist,
+                  const int32_t* probe_ids, int nprobe, const int64_t* list_offsets, const uint8_t* codes,
+                  int64_t n_codes, const float* codebooks, int pq_m, int n_rerank, const int64_t* vec_ids,
+                  int64_t* out_ids, float* out_est, int64_t* out_counts, void* stream);
 
 #ifdef __cplusplus
 }

@@ -23,6 +23,7 @@ EXPORTS = (
     "ivf_route", "ivf_assign", "ivf_centroid_update", "ivf_centroid_update_noalloc", "ivf_centroid_finalize",
     "ivf_assign_update", "ivf_cluster_major_reorder", "ivf_centroids_create", "ivf_centroids_destroy",
     "ivf_route_prepared",
+    "ivf_pq_encode", "ivf_pq_search",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
     "ivf_debug_plan", "ivf_debug_span", "ivf_debug_set_wait_limit_ns",
     "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_set_row_chunk", "ivf_debug_stats",
@@ -73,6 +74,8 @@ def lib() -> ctypes.CDLL:
     L.ivf_debug_set_row_chunk.argtypes = [i64]
     L.ivf_debug_stats.argtypes = [i32, ctypes.POINTER(i64)]
     L.ivf_debug_rule.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_int)]
+    L.ivf_pq_encode.argtypes = [vp, i64, i32, i32, vp, vp, i32, vp, i32, vp, vp]
+    L.ivf_pq_search.argtypes = [vp, i64, i32, i32, vp, i32, vp, i32, vp, vp, i64, vp, i32, i32, vp, vp, vp, vp, vp]
     L.ivf_debug_timing_read.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
     for name in EXPORTS:
         if name not in ("ivf_last_error", "ivf_launch_count"):
@@ -269,6 +272,68 @@ def ivf_cluster_major_reorder(points: torch.Tensor, ids: torch.Tensor, nlist: in
     return out_points, out_offsets, out_order
 
 
+def _codebooks(codebooks: torch.Tensor, d: int) -> int:
+    _dev(codebooks, "codebooks", torch.float32)
+    if codebooks.dim() != 3 or codebooks.shape[1] != 256 or codebooks.shape[0] * codebooks.shape[2] != d:
+        raise ValueError("codebooks must be [pq_m, 256, d / pq_m]")
+    return codebooks.shape[0]
+
+
+def ivf_pq_encode(points: torch.Tensor, ids: torch.Tensor, centroids: torch.Tensor, codebooks: torch.Tensor):
+    """uint8 [n, pq_m] residual-PQ codes of the rows of points, row i assigned to list ids[i]."""
+    if not points.is_cuda:
+        raise ValueError("points must be a CUDA tensor")
+    _rows(points, "points")
+    _dev(ids, "ids", torch.int32)
+    _dev(centroids, "centroids", torch.float32)
+    n, d = points.shape
+    pq_m = _codebooks(codebooks, d)
+    dev = points.device
+    codes = torch.empty((n, pq_m), dtype=torch.uint8, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib().ivf_pq_encode(_ptr(points), n, d, _dtype_code(points), _ptr(ids), _ptr(centroids),
+                                 centroids.shape[0], _ptr(codebooks), pq_m, _ptr(codes), _stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
+    return codes
+
+
+def ivf_pq_search(queries: torch.Tensor, centroids: torch.Tensor, probe_ids: torch.Tensor, list_offsets: torch.Tensor,
+                  codes: torch.Tensor, codebooks: torch.Tensor, n_rerank: int, vec_ids: torch.Tensor | None = None,
+                  want_counts: bool = True):
+    """(ids int64 [nq, n_rerank], estimates float32 [nq, n_rerank], counts int64 [nq] or None): the
+    n_rerank smallest ADC estimates over the codes of every query's probed lists, ascending."""
+    if not queries.is_cuda:
+        raise ValueError("queries must be a CUDA tensor")
+    _rows(queries, "queries")
+    _dev(centroids, "centroids", torch.float32)
+    _dev(probe_ids, "probe_ids", torch.int32)
+    _dev(list_offsets, "list_offsets", torch.int64)
+    _dev(codes, "codes", torch.uint8)
+    if vec_ids is not None:
+        _dev(vec_ids, "vec_ids", torch.int64)
+    nq, d = queries.shape
+    pq_m = _codebooks(codebooks, d)
+    if codes.dim() != 2 or codes.shape[1] != pq_m:
+        raise ValueError("codes must be [n_codes, pq_m]")
+    if probe_ids.dim() != 2 or probe_ids.shape[0] != nq:
+        raise ValueError("probe_ids must be [nq, nprobe]")
+    if list_offsets.numel() != centroids.shape[0] + 1:
+        raise ValueError("list_offsets must have nlist + 1 entries")
+    dev = queries.device
+    out_ids = torch.empty((nq, n_rerank), dtype=torch.int64, device=dev)
+    out_est = torch.empty((nq, n_rerank), dtype=torch.float32, device=dev)
+    counts = torch.empty((nq,), dtype=torch.int64, device=dev) if want_counts else None
+    with torch.cuda.device(dev):
+        rc = lib().ivf_pq_search(_ptr(queries), nq, d, _dtype_code(queries), _ptr(centroids), centroids.shape[0],
+                                 _ptr(probe_ids), probe_ids.shape[1], _ptr(list_offsets), _ptr(codes), codes.shape[0],
+                                 _ptr(codebooks), pq_m, n_rerank, _ptr(vec_ids), _ptr(out_ids), _ptr(out_est),
+                                 _ptr(counts), _stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
+    return out_ids, out_est, counts
+
+
 def ivf_centroid_finalize(sums: torch.Tensor, counts: torch.Tensor, centroids: torch.Tensor):
     """centroids[l] = sums[l] / counts[l] in place; lists with count 0 keep their row."""
     _dev(sums, "sums", torch.float32)
@@ -344,7 +409,8 @@ def ivf_debug_set_wait_limit_ns(ns: int) -> None:
     lib().ivf_debug_set_wait_limit_ns(ns)
 
 
-TIMING_FAMILIES = ("prep", "fused_argmin", "fused_topk", "merge", "update", "threshold_pass")
+TIMING_FAMILIES = ("prep", "fused_argmin", "fused_topk", "merge", "update", "threshold_pass",
+                   "pq_encode", "pq_scan", "pq_merge")
 
 
 def ivf_debug_timing(enable: bool) -> None:
@@ -353,8 +419,8 @@ def ivf_debug_timing(enable: bool) -> None:
 
 def ivf_debug_timing_read() -> dict:
     """{family: (milliseconds, launch groups)} since the last read; synchronises the device."""
-    ms = (ctypes.c_double * 6)()
-    cnt = (ctypes.c_int64 * 6)()
+    ms = (ctypes.c_double * len(TIMING_FAMILIES))()
+    cnt = (ctypes.c_int64 * len(TIMING_FAMILIES))()
     rc = lib().ivf_debug_timing_read(ms, cnt)
     if rc != IVF_OK:
         _raise(rc)

@@ -18,6 +18,7 @@
 
 #include "fused_topk.cuh"
 #include "merge.cuh"
+#include "pq.cuh"
 #include "prep.cuh"
 #include "update.cuh"
 
@@ -56,7 +57,7 @@ int fail(int code, const char* fmt, ...) {
 
 // ------------------------------------------------------------------ optional per-kernel timing
 // When enabled, launches of each kernel family are bracketed by CUDA events on the caller's stream.
-enum TimedKind { TK_PREP = 0, TK_FUSED_ARGMIN, TK_FUSED_TOPK, TK_MERGE, TK_UPDATE, TK_THRESH, TK_NUM };
+enum TimedKind { TK_PREP = 0, TK_FUSED_ARGMIN, TK_FUSED_TOPK, TK_MERGE, TK_UPDATE, TK_THRESH, TK_PQ_ENCODE, TK_PQ_SCAN, TK_PQ_MERGE, TK_NUM };
 struct TimedLaunch {
     cudaEvent_t a, b;
     int kind;
@@ -97,7 +98,7 @@ void timing_end(int idx, cudaStream_t stream) {
 // ------------------------------------------------------------------ workspace
 enum WsSlot {
     WS_X16, WS_C16, WS_XN, WS_SCAL, WS_BITS, WS_PART, WS_PARTMETA, WS_FAIL, WS_FBKEYS, WS_TAU,
-    WS_UCNT, WS_UOFF, WS_UCUR, WS_UPERM, WS_IDS, WS_CHUNK0, WS_CHUNK1, WS_NUM
+    WS_UCNT, WS_UOFF, WS_UCUR, WS_UPERM, WS_IDS, WS_CHUNK0, WS_CHUNK1, WS_PQ_CHUNKS, WS_PQ_GCAND, WS_PQ_GCOUNT, WS_NUM
 };
 struct Buf {
     void* p = nullptr;
@@ -115,6 +116,7 @@ struct DeviceCtx {
     cudaEvent_t ev_ready = nullptr;
     bool smem_attr_set = false;
     bool merge_attr_set = false;
+    bool pq_attr_set = false;
 };
 constexpr int kMaxDevices = 64;
 DeviceCtx g_ctx[kMaxDevices];
@@ -942,6 +944,147 @@ int ivf_assign_update(const void* points, int64_t n, int d, ivf_dtype ptype, con
                       static_cast<cudaStream_t>(stream));
 }
 
+// ------------------------------------------------------------------ residual-PQ candidate reduction
+namespace {
+int pq_check_shape(int d, int pq_m, const float* codebooks) {
+    if (d < 1 || pq_m < 1 || d % pq_m != 0)
+        return fail(IVF_ERR_INVALID_ARG, "d = %d, pq_m = %d: pq_m must divide d", d, pq_m);
+    if (!codebooks) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    if (pq_smem_bytes(d, pq_m) > kSmemLimit)
+        return fail(IVF_ERR_UNSUPPORTED, "d = %d, pq_m = %d: codebook + lookup table need %zu bytes of shared memory (limit %zu)",
+                    d, pq_m, pq_smem_bytes(d, pq_m), static_cast<size_t>(kSmemLimit));
+    return IVF_OK;
+}
+int pq_set_attrs(DeviceCtx& ctx) {
+    if (!ctx.pq_attr_set) {
+        CUDA_TRY(cudaFuncSetAttribute(pq_encode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      static_cast<int>(kSmemLimit)));
+        CUDA_TRY(cudaFuncSetAttribute(pq_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      static_cast<int>(kSmemLimit)));
+        ctx.pq_attr_set = true;
+    }
+    return IVF_OK;
+}
+}  // namespace
+
+int ivf_pq_encode(const void* points, int64_t n, int d, ivf_dtype ptype, const int32_t* ids, const float* centroids,
+                  int nlist, const float* codebooks, int pq_m, uint8_t* out_codes, void* stream_) {
+    if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
+    if (ptype != IVF_F32 && ptype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
+    if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
+    int rc = pq_check_shape(d, pq_m, codebooks);
+    if (rc != IVF_OK) return rc;
+    if (n == 0) return IVF_OK;
+    if (!points || !ids || !centroids || !out_codes) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    DeviceCtx* pctx = nullptr;
+    rc = get_ctx(&pctx);
+    if (rc != IVF_OK) return rc;
+    DeviceCtx& ctx = *pctx;
+    rc = pq_set_attrs(ctx);
+    if (rc != IVF_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    PqEncodeParams p;
+    p.x = points;
+    p.x_is_u8 = ptype == IVF_U8;
+    p.n = n;
+    p.d = d;
+    p.pq_m = pq_m;
+    p.nlist = nlist;
+    p.ids = ids;
+    p.centroids = centroids;
+    p.codebooks = codebooks;
+    p.codes = out_codes;
+    p.status = ctx.status;
+    const int tk = timing_begin(TK_PQ_ENCODE, stream);
+    const unsigned grid = static_cast<unsigned>(n < ctx.num_sms ? n : ctx.num_sms);
+    pq_encode_kernel<<<grid, kPqThreads, pq_smem_bytes(d, pq_m), stream>>>(p);
+    LAUNCH_CHECK();
+    timing_end(tk, stream);
+    return IVF_OK;
+}
+
+int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const float* centroids, int nlist,
+                  const int32_t* probe_ids, int nprobe, const int64_t* list_offsets, const uint8_t* codes,
+                  int64_t n_codes, const float* codebooks, int pq_m, int n_rerank, const int64_t* vec_ids,
+                  int64_t* out_ids, float* out_est, int64_t* out_counts, void* stream_) {
+    if (nq < 0) return fail(IVF_ERR_INVALID_ARG, "negative query count %lld", (long long)nq);
+    if (qtype != IVF_F32 && qtype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)qtype);
+    if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
+    if (nprobe < 1 || nprobe > nlist) return fail(IVF_ERR_INVALID_ARG, "nprobe = %d with nlist = %d", nprobe, nlist);
+    if (nprobe > 4096) return fail(IVF_ERR_UNSUPPORTED, "nprobe = %d: at most 4096", nprobe);
+    if (n_rerank < 1 || n_rerank > kPqMaxRerank)
+        return fail(IVF_ERR_UNSUPPORTED, "n_rerank = %d: must be in [1, %d]", n_rerank, kPqMaxRerank);
+    if (n_codes < 0 || n_codes >= (int64_t(1) << 32))
+        return fail(IVF_ERR_UNSUPPORTED, "n_codes = %lld: positions must fit 32 bits", (long long)n_codes);
+    if (nq >= (int64_t(1) << 24)) return fail(IVF_ERR_UNSUPPORTED, "nq = %lld: at most 2^24 - 1 queries per call", (long long)nq);
+    int rc = pq_check_shape(d, pq_m, codebooks);
+    if (rc != IVF_OK) return rc;
+    if (nq == 0) return IVF_OK;
+    if (!queries || !centroids || !probe_ids || !list_offsets || !out_ids || !out_est || (n_codes > 0 && !codes))
+        return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    if (reinterpret_cast<uintptr_t>(codes) & 15) return fail(IVF_ERR_INVALID_ARG, "codes must be 16-byte aligned");
+    DeviceCtx* pctx = nullptr;
+    rc = get_ctx(&pctx);
+    if (rc != IVF_OK) return rc;
+    DeviceCtx& ctx = *pctx;
+    rc = pq_set_attrs(ctx);
+    if (rc != IVF_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    // groups per query: enough CTAs of work for every SM even at serving-size batches
+    int ngroups = static_cast<int>((8 * static_cast<int64_t>(ctx.num_sms) + nq - 1) / nq);
+    if (ngroups < 1) ngroups = 1;
+    if (ngroups > 256) ngroups = 256;
+    const int64_t total_groups = nq * ngroups;
+    int* chunk_start;
+    uint64_t* gcand;
+    int* gcount;
+    WS(WS_PQ_CHUNKS, static_cast<size_t>(nq) * (nprobe + 1) * sizeof(int), chunk_start);
+    WS(WS_PQ_GCAND, static_cast<size_t>(total_groups) * n_rerank * sizeof(uint64_t), gcand);
+    WS(WS_PQ_GCOUNT, static_cast<size_t>(total_groups) * sizeof(int), gcount);
+    int tk = timing_begin(TK_PQ_SCAN, stream);
+    pq_setup_query_kernel<<<static_cast<unsigned>(nq), 128, 0, stream>>>(
+        probe_ids, nprobe, nlist, reinterpret_cast<const long long*>(list_offsets), chunk_start,
+        reinterpret_cast<long long*>(out_counts), ctx.status);
+    LAUNCH_CHECK();
+    PqScanParams sp;
+    sp.q = queries;
+    sp.q_is_u8 = qtype == IVF_U8;
+    sp.nq = nq;
+    sp.d = d;
+    sp.pq_m = pq_m;
+    sp.nlist = nlist;
+    sp.nprobe = nprobe;
+    sp.n_rerank = n_rerank;
+    sp.ngroups = ngroups;
+    sp.centroids = centroids;
+    sp.codebooks = codebooks;
+    sp.probes = probe_ids;
+    sp.offsets = reinterpret_cast<const long long*>(list_offsets);
+    sp.codes = codes;
+    sp.chunk_start = chunk_start;
+    sp.gcand = gcand;
+    sp.gcand_count = gcount;
+    sp.status = ctx.status;
+    const unsigned grid = static_cast<unsigned>(total_groups < ctx.num_sms ? total_groups : ctx.num_sms);
+    pq_scan_kernel<<<grid, kPqThreads, pq_smem_bytes(d, pq_m), stream>>>(sp);
+    LAUNCH_CHECK();
+    timing_end(tk, stream);
+    tk = timing_begin(TK_PQ_MERGE, stream);
+    PqMergeParams mp;
+    mp.nq = nq;
+    mp.n_rerank = n_rerank;
+    mp.ngroups = ngroups;
+    mp.gcand = gcand;
+    mp.gcand_count = gcount;
+    mp.vec_ids = reinterpret_cast<const long long*>(vec_ids);
+    mp.out_pos = reinterpret_cast<long long*>(out_ids);
+    mp.out_est = out_est;
+    pq_merge_kernel<<<static_cast<unsigned>(nq), kPqThreads, 0, stream>>>(mp);
+    LAUNCH_CHECK();
+    timing_end(tk, stream);
+    return IVF_OK;
+}
+
 int ivf_check(void* stream) {
     DeviceCtx* ctx = nullptr;
     int rc = get_ctx(&ctx);
@@ -1019,7 +1162,7 @@ int ivf_debug_timing(int enable) {
     return IVF_OK;
 }
 
-int ivf_debug_timing_read(double ms[6], int64_t launches[6]) {
+int ivf_debug_timing_read(double ms[9], int64_t launches[9]) {
     if (!ms || !launches) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
     CUDA_TRY(cudaDeviceSynchronize());
     std::lock_guard<std::mutex> lk(g_mu);

@@ -1,0 +1,475 @@
+// Residual-PQ candidate reduction on the GPU (Sec. 2.2 Eq. 3-5; Sec. 4.3 residual encoding and
+// lookup tables; Sec. 4.4: compact codes resident in GPU memory, task set-up on the device by
+// prefix scans, chunked ADC scan with a bounded local candidate set, chunk -> group -> query
+// merging, and the scan fused with the first merge level).
+//
+// Arithmetic, in fp32 with one fixed order so that every byte and every kept candidate is
+// reproducible (the paper fixes fp32 lookup tables):
+//     r_t = float(x_t) - c_t
+//     LUT_m[j] : acc = 0; for t in order: diff = r_t - p_m[j][t]; acc = fma(diff, diff, acc)
+//     ADC      : acc = 0; for m in order: acc = acc + LUT_m[a_m]
+// Encoding is the arg-min over j of the vector's own table (ties to the lower j).
+//
+// Design: a persistent CTA keeps the whole codebook (256 * d floats, transposed so that the 256
+// codewords of one coordinate are contiguous) in shared memory next to one lookup table, so a
+// table costs d/PQ_M fused multiply-adds per entry and no global traffic.  A group of chunks of one
+// query is scanned by one CTA; candidates that beat the running bound go to a shared-memory buffer
+// that is cut back to the N_rerank smallest by a 64-bit radix select when it fills, and only the
+// group's survivors are written out.  A last kernel selects and sorts per query.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fused_topk.cuh"  // orderable(), radix_pick_digit()
+
+namespace ivf {
+
+constexpr int kPqK = 256;          // codewords per subspace (one byte per sub-code)
+constexpr int kPqThreads = 512;
+constexpr int kPqChunk = 512;      // codes per chunk = one code per thread
+constexpr int kPqBufKeys = 2048;   // candidate buffer of a group
+constexpr int kPqMaxRerank = 1024;
+constexpr int kPqStatusBadId = -6;
+
+__host__ __device__ inline size_t pq_smem_bytes(int d, int pq_m) {
+    return static_cast<size_t>(d) * kPqK * 4 + static_cast<size_t>(pq_m) * kPqK * 4 + static_cast<size_t>(d) * 4 +
+           static_cast<size_t>(kPqBufKeys) * 8 + 256 * 4 + 64;
+}
+
+struct PqSmem {
+    float* cbt;     // [d][256]: coordinate-major codebook
+    float* lut;     // [pq_m][256]
+    float* r;       // [d]
+    uint64_t* buf;  // [kPqBufKeys]
+    int* hist;      // [256]
+    int* misc;      // [16]: 0 count, 1 digit, 2 rank, 3 eq
+};
+
+__device__ __forceinline__ PqSmem pq_carve(uint8_t* raw, int d, int pq_m) {
+    PqSmem s;
+    s.buf = reinterpret_cast<uint64_t*>(raw);
+    raw += static_cast<size_t>(kPqBufKeys) * 8;
+    s.cbt = reinterpret_cast<float*>(raw);
+    raw += static_cast<size_t>(d) * kPqK * 4;
+    s.lut = reinterpret_cast<float*>(raw);
+    raw += static_cast<size_t>(pq_m) * kPqK * 4;
+    s.r = reinterpret_cast<float*>(raw);
+    raw += static_cast<size_t>(d) * 4;
+    s.hist = reinterpret_cast<int*>(raw);
+    raw += 256 * 4;
+    s.misc = reinterpret_cast<int*>(raw);
+    return s;
+}
+
+// codebooks [pq_m][256][dsub] in global memory -> cbt[(m * dsub + t) * 256 + j]
+__device__ __forceinline__ void pq_load_codebooks(const float* __restrict__ codebooks, int d, int dsub, float* cbt) {
+    const int total = d * kPqK;
+    for (int i = threadIdx.x; i < total; i += blockDim.x) {
+        // i walks the global layout: i = (m * 256 + j) * dsub + t
+        const int t = i % dsub;
+        const int mj = i / dsub;
+        const int j = mj & (kPqK - 1), m = mj >> 8;
+        cbt[(m * dsub + t) * kPqK + j] = codebooks[i];
+    }
+}
+
+// lut[m * 256 + j] for the residual in s.r.  Thread -> codeword j = tid & 255; the 256-thread
+// halves of the CTA take alternate subspaces.
+__device__ __forceinline__ void pq_build_lut(const PqSmem& s, int pq_m, int dsub) {
+    const int j = threadIdx.x & (kPqK - 1);
+    const int step = blockDim.x >> 8;
+    for (int m = threadIdx.x >> 8; m < pq_m; m += step) {
+        const float* col = s.cbt + static_cast<size_t>(m) * dsub * kPqK + j;
+        const float* r = s.r + m * dsub;
+        float acc = 0.0f;
+        for (int t = 0; t < dsub; ++t) {
+            const float diff = __fsub_rn(r[t], col[t * kPqK]);
+            acc = __fmaf_rn(diff, diff, acc);
+        }
+        s.lut[m * kPqK + j] = acc;
+    }
+}
+
+template <typename T>
+__device__ __forceinline__ float pq_elem(const T* x, int64_t idx) {
+    return static_cast<float>(x[idx]);
+}
+
+// ------------------------------------------------------------------ residual encoding (Eq. 3 on x - c(x))
+struct PqEncodeParams {
+    const void* x;
+    int x_is_u8;
+    int64_t n;
+    int d, pq_m, nlist;
+    const int32_t* ids;
+    const float* centroids;
+    const float* codebooks;
+    uint8_t* codes;  // [n][pq_m]
+    int* status;
+};
+
+__global__ void __launch_bounds__(kPqThreads, 1) pq_encode_kernel(const PqEncodeParams p) {
+    extern __shared__ __align__(16) uint8_t pq_smem_raw[];
+    const PqSmem s = pq_carve(pq_smem_raw, p.d, p.pq_m);
+    const int dsub = p.d / p.pq_m;
+    pq_load_codebooks(p.codebooks, p.d, dsub, s.cbt);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    for (int64_t i = blockIdx.x; i < p.n; i += gridDim.x) {
+        const int32_t l = p.ids[i];
+        const bool ok = l >= 0 && l < p.nlist;
+        __syncthreads();  // the previous row's table has been consumed (and the codebook is in place)
+        if (!ok) {
+            if (threadIdx.x == 0) atomicCAS(p.status, 0, kPqStatusBadId);
+            for (int m = threadIdx.x; m < p.pq_m; m += blockDim.x) p.codes[i * p.pq_m + m] = 0;
+            continue;
+        }
+        for (int t = threadIdx.x; t < p.d; t += blockDim.x) {
+            const float xv = p.x_is_u8 ? pq_elem(static_cast<const uint8_t*>(p.x), i * p.d + t)
+                                       : pq_elem(static_cast<const float*>(p.x), i * p.d + t);
+            s.r[t] = __fsub_rn(xv, p.centroids[static_cast<int64_t>(l) * p.d + t]);
+        }
+        __syncthreads();
+        pq_build_lut(s, p.pq_m, dsub);
+        __syncthreads();
+        for (int m = warp; m < p.pq_m; m += nwarps) {
+            const float* row = s.lut + m * kPqK;
+            float best = row[lane];
+            int bj = lane;
+#pragma unroll
+            for (int q = 1; q < kPqK / 32; ++q) {
+                const float v = row[lane + 32 * q];
+                if (v < best) {
+                    best = v;
+                    bj = lane + 32 * q;
+                }
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xFFFFFFFFu, best, off);
+                const int oj = __shfl_xor_sync(0xFFFFFFFFu, bj, off);
+                if (ov < best || (ov == best && oj < bj)) {
+                    best = ov;
+                    bj = oj;
+                }
+            }
+            if (lane == 0) p.codes[i * p.pq_m + m] = static_cast<uint8_t>(bj);
+        }
+    }
+}
+
+// ------------------------------------------------------------------ task set-up (prefix scans on the device)
+// Per query: chunk_start[b][p] = chunks of the probes before p (a probed list of length L has
+// ceil(L / kPqChunk) chunks), chunk_start[b][nprobe] = the query's chunks; cand_count[b] = the codes
+// it will scan.  Every query's chunks are then dealt to a fixed number of groups, so the output
+// offset of a group follows from its index alone.
+__global__ void __launch_bounds__(128) pq_setup_query_kernel(const int32_t* __restrict__ probes, int nprobe, int nlist,
+                                                             const long long* __restrict__ offsets,
+                                                             int* __restrict__ chunk_start,
+                                                             long long* __restrict__ cand_count, int* status) {
+    __shared__ int wsum[4];
+    __shared__ long long wlen[4];
+    __shared__ int carry_s;
+    __shared__ long long total_len_s;
+    const int b = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        carry_s = 0;
+        total_len_s = 0;
+    }
+    __syncthreads();
+    int* cs = chunk_start + static_cast<size_t>(b) * (nprobe + 1);
+    for (int p0 = 0; p0 < nprobe; p0 += blockDim.x) {
+        const int p = p0 + threadIdx.x;
+        int nch = 0;
+        long long len = 0;
+        if (p < nprobe) {
+            const int l = probes[static_cast<size_t>(b) * nprobe + p];
+            if (l >= 0 && l < nlist) {
+                len = offsets[l + 1] - offsets[l];
+                if (len < 0) len = 0;
+                nch = static_cast<int>((len + kPqChunk - 1) / kPqChunk);
+            } else {
+                atomicCAS(status, 0, kPqStatusBadId);
+            }
+        }
+        int v = nch;
+        long long lv = len;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, v, off);
+            if (lane >= off) v += t;
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) lv += __shfl_xor_sync(0xFFFFFFFFu, lv, off);
+        if (lane == 31) wsum[warp] = v;
+        if (lane == 0) wlen[warp] = lv;
+        __syncthreads();
+        int before = carry_s;
+        for (int w = 0; w < warp; ++w) before += wsum[w];
+        if (p < nprobe) cs[p] = before + v - nch;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            carry_s += wsum[0] + wsum[1] + wsum[2] + wsum[3];
+            total_len_s += wlen[0] + wlen[1] + wlen[2] + wlen[3];
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        cs[nprobe] = carry_s;
+        if (cand_count) cand_count[b] = total_len_s;
+    }
+}
+
+// ------------------------------------------------------------------ block-wide selection of the k smallest keys
+// Largest admitted key among `count` distinct 64-bit keys in shared memory (count > k): radix
+// select from the top byte down, stopping once the digit that holds rank k is wanted whole.
+__device__ __forceinline__ uint64_t pq_select_bound(const uint64_t* keys, int count, int k, int* hist, int* misc) {
+    const int lane = threadIdx.x & 31;
+    uint64_t prefix = 0, mask = 0;
+    int rank = k;
+    const int rounded = (count + 31) & ~31;
+    for (int shift = 56; shift >= 0; shift -= 8) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+        __syncthreads();
+        for (int i = threadIdx.x; i < rounded; i += blockDim.x) {
+            uint32_t dg = 0xFFFFFFFFu;
+            if (i < count) {
+                const uint64_t v = keys[i];
+                if ((v & mask) == prefix) dg = static_cast<uint32_t>(v >> shift) & 255u;
+            }
+            const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dg);
+            if (dg != 0xFFFFFFFFu && lane == __ffs(peers) - 1) atomicAdd(&hist[dg], __popc(peers));
+        }
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            int r = rank, eq = 0;
+            const int digit = radix_pick_digit(hist, lane, r, eq);
+            if (lane == 0) {
+                misc[1] = digit;
+                misc[2] = r;
+                misc[3] = eq;
+            }
+        }
+        __syncthreads();
+        prefix |= static_cast<uint64_t>(misc[1]) << shift;
+        mask |= 255ull << shift;
+        rank = misc[2];
+        const bool whole = misc[3] == rank;
+        __syncthreads();
+        if (whole) return prefix | ~mask;
+    }
+    return prefix;
+}
+
+// Cuts the buffer back to its k smallest keys (in no particular order); returns the bound, i.e.
+// the largest key kept.  count > k on entry; on exit misc[0] == k.
+__device__ __forceinline__ uint64_t pq_cut_buffer(uint64_t* buf, int count, int k, int* hist, int* misc) {
+    const uint64_t bound = pq_select_bound(buf, count, k, hist, misc);
+    constexpr int kPer = kPqBufKeys / kPqThreads;
+    uint64_t mine[kPer];
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+        const int i = threadIdx.x + q * kPqThreads;
+        mine[q] = i < count ? buf[i] : ~0ull;
+    }
+    if (threadIdx.x == 0) misc[0] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < kPer; ++q)
+        if (mine[q] <= bound && mine[q] != ~0ull) buf[atomicAdd(&misc[0], 1)] = mine[q];
+    __syncthreads();
+    return bound;
+}
+
+// ------------------------------------------------------------------ chunked ADC scan fused with the group merge
+struct PqScanParams {
+    const void* q;
+    int q_is_u8;
+    int64_t nq;
+    int d, pq_m, nlist, nprobe, n_rerank;
+    int ngroups;             // groups per query
+    const float* centroids;
+    const float* codebooks;
+    const int32_t* probes;
+    const long long* offsets;
+    const uint8_t* codes;
+    const int* chunk_start;  // [nq][nprobe + 1]
+    uint64_t* gcand;         // [nq * ngroups][n_rerank] keys: (estimate bits << 32) | position
+    int* gcand_count;        // [nq * ngroups]
+    int* status;
+};
+
+__device__ __forceinline__ float pq_adc_code(const float* lut, const uint8_t* code, int pq_m) {
+    float acc = 0.0f;
+    if ((pq_m & 15) == 0) {
+        for (int m0 = 0; m0 < pq_m; m0 += 16) {
+            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(code + m0));
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+            for (int q = 0; q < 16; ++q)
+                acc = __fadd_rn(acc, lut[(m0 + q) * kPqK + ((w[q >> 2] >> (8 * (q & 3))) & 255u)]);
+        }
+    } else if ((pq_m & 3) == 0) {
+        for (int m0 = 0; m0 < pq_m; m0 += 4) {
+            const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(code + m0));
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc = __fadd_rn(acc, lut[(m0 + q) * kPqK + ((w >> (8 * q)) & 255u)]);
+        }
+    } else {
+        for (int m = 0; m < pq_m; ++m) acc = __fadd_rn(acc, lut[m * kPqK + __ldg(code + m)]);
+    }
+    return acc;
+}
+
+__global__ void __launch_bounds__(kPqThreads, 1) pq_scan_kernel(const PqScanParams p) {
+    extern __shared__ __align__(16) uint8_t pq_smem_raw[];
+    const PqSmem s = pq_carve(pq_smem_raw, p.d, p.pq_m);
+    const int dsub = p.d / p.pq_m;
+    const int64_t total_groups = p.nq * p.ngroups;
+    if (static_cast<int64_t>(blockIdx.x) >= total_groups) return;
+    pq_load_codebooks(p.codebooks, p.d, dsub, s.cbt);
+    const int lane = threadIdx.x & 31;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+
+    for (int64_t g = blockIdx.x; g < total_groups; g += gridDim.x) {
+        const int64_t b = g / p.ngroups;
+        const int gi = static_cast<int>(g - b * p.ngroups);
+        const int* cs = p.chunk_start + static_cast<size_t>(b) * (p.nprobe + 1);
+        const int group_chunks = (cs[p.nprobe] + p.ngroups - 1) / p.ngroups;
+        const int chunk0 = min(cs[p.nprobe], gi * group_chunks);
+        const int chunk1 = min(cs[p.nprobe], chunk0 + group_chunks);
+        __syncthreads();
+        if (threadIdx.x == 0) s.misc[0] = 0;
+        uint64_t bound = ~0ull;  // a candidate must be below this key to matter
+        int cur_probe = -1;
+        long long list_begin = 0, list_len = 0;
+        for (int ch = chunk0; ch < chunk1; ++ch) {
+            // probe that owns chunk ch: the last pr with cs[pr] <= ch (empty lists own no chunk)
+            int plo = max(cur_probe, 0), phi = p.nprobe;
+            while (phi - plo > 1) {
+                const int mid = (plo + phi) >> 1;
+                if (cs[mid] <= ch) plo = mid; else phi = mid;
+            }
+            if (plo != cur_probe) {
+                cur_probe = plo;
+                const int l = p.probes[static_cast<size_t>(b) * p.nprobe + plo];
+                list_begin = p.offsets[l];
+                list_len = p.offsets[l + 1] - list_begin;
+                __syncthreads();  // the previous table is no longer read
+                for (int t = threadIdx.x; t < p.d; t += blockDim.x) {
+                    const float qv = p.q_is_u8 ? pq_elem(static_cast<const uint8_t*>(p.q), b * p.d + t)
+                                               : pq_elem(static_cast<const float*>(p.q), b * p.d + t);
+                    s.r[t] = __fsub_rn(qv, p.centroids[static_cast<int64_t>(l) * p.d + t]);
+                }
+                __syncthreads();
+                pq_build_lut(s, p.pq_m, dsub);
+                __syncthreads();
+            }
+            const long long in_list = static_cast<long long>(ch - cs[cur_probe]) * kPqChunk + threadIdx.x;
+            bool hit = false;
+            uint64_t key = 0;
+            if (in_list < list_len) {
+                const long long pos = list_begin + in_list;
+                const float est = pq_adc_code(s.lut, p.codes + pos * p.pq_m, p.pq_m);
+                key = (static_cast<uint64_t>(orderable(est)) << 32) | static_cast<uint32_t>(pos);
+                hit = key < bound;
+            }
+            const uint32_t bal = __ballot_sync(0xFFFFFFFFu, hit);
+            if (bal) {
+                int base = 0;
+                if (lane == 0) base = atomicAdd(&s.misc[0], __popc(bal));
+                base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                if (hit) s.buf[base + __popc(bal & lt_mask)] = key;
+            }
+            __syncthreads();
+            const int count = s.misc[0];
+            if (count > kPqBufKeys - kPqChunk) bound = pq_cut_buffer(s.buf, count, p.n_rerank, s.hist, s.misc);
+        }
+        __syncthreads();
+        int count = s.misc[0];
+        if (count > p.n_rerank) {
+            pq_cut_buffer(s.buf, count, p.n_rerank, s.hist, s.misc);
+            count = p.n_rerank;
+        }
+        uint64_t* out = p.gcand + static_cast<size_t>(g) * p.n_rerank;
+        for (int i = threadIdx.x; i < count; i += blockDim.x) out[i] = s.buf[i];
+        if (threadIdx.x == 0) p.gcand_count[g] = count;
+    }
+}
+
+// ------------------------------------------------------------------ group -> query merge
+struct PqMergeParams {
+    int64_t nq;
+    int n_rerank;
+    int ngroups;
+    const uint64_t* gcand;
+    const int* gcand_count;
+    const long long* vec_ids;  // optional: position -> caller's identifier
+    long long* out_pos;        // [nq][n_rerank]
+    float* out_est;            // [nq][n_rerank]
+};
+
+// One CTA per query.  The query's group candidates are cut to the n_rerank smallest in rounds
+// through the same shared-memory buffer, sorted, and written in ascending (estimate, position) order.
+__global__ void __launch_bounds__(kPqThreads) pq_merge_kernel(const PqMergeParams p) {
+    __shared__ uint64_t buf[kPqBufKeys];
+    __shared__ int hist[256];
+    __shared__ int misc[16];
+    const int64_t b = blockIdx.x;
+    const int64_t g0 = b * p.ngroups, g1 = g0 + p.ngroups;
+    int count = 0;
+    for (int64_t g = g0; g < g1; ++g) {
+        const int c = p.gcand_count[g];
+        __syncthreads();
+        if (count + c > kPqBufKeys) {
+            if (threadIdx.x == 0) misc[0] = count;
+            __syncthreads();
+            pq_cut_buffer(buf, count, p.n_rerank, hist, misc);
+            count = p.n_rerank;
+        }
+        const uint64_t* src = p.gcand + static_cast<size_t>(g) * p.n_rerank;
+        for (int i = threadIdx.x; i < c; i += blockDim.x) buf[count + i] = src[i];
+        count += c;
+    }
+    __syncthreads();
+    if (count > p.n_rerank) {
+        if (threadIdx.x == 0) misc[0] = count;
+        __syncthreads();
+        pq_cut_buffer(buf, count, p.n_rerank, hist, misc);
+        count = p.n_rerank;
+    }
+    int m = 2;
+    while (m < count) m <<= 1;
+    for (int i = count + threadIdx.x; i < m; i += blockDim.x) buf[i] = ~0ull;
+    // bitonic sort of buf[0 .. m)
+    for (int size = 2; size <= m; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            __syncthreads();
+            for (int t = threadIdx.x; t < (m >> 1); t += blockDim.x) {
+                const int lo = 2 * t - (t & (stride - 1));
+                const int hi = lo + stride;
+                const bool up = (lo & size) == 0;
+                const uint64_t a = buf[lo], c = buf[hi];
+                if ((a > c) == up) {
+                    buf[lo] = c;
+                    buf[hi] = a;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < p.n_rerank; i += blockDim.x) {
+        long long pos = -1;
+        float est = __int_as_float(0x7f800000);
+        if (i < count) {
+            const uint64_t key = buf[i];
+            pos = static_cast<long long>(key & 0xFFFFFFFFull);
+            if (p.vec_ids) pos = p.vec_ids[pos];
+            est = from_orderable(static_cast<uint32_t>(key >> 32));
+        }
+        p.out_pos[b * p.n_rerank + i] = pos;
+        p.out_est[b * p.n_rerank + i] = est;
+    }
+}
+
+}  // namespace ivf

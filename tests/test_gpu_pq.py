@@ -1,0 +1,145 @@
+"""GPU parity of the residual-PQ chain (encode, set-up, chunked ADC scan, group and query merge)
+against the CPU oracle, through the C-ABI binding.  The oracle computes in the paper's fp32 with a
+stated operation order, so codes, kept positions and estimates must match bit for bit.  Every
+oracle input comes from the seeded generators or from the oracle itself, never from the GPU."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2608_08751_b200 import binding as B
+from paper_2608_08751_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _t(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def _problem(seed, n, nlist, d, pq_m, dtype, nq, nprobe, sigma=1.0, integer=False):
+    rng = np.random.default_rng(1000 + seed)
+    dsub = d // pq_m
+    if dtype == "u8":
+        c = rng.uniform(20, 230, (nlist, d)).astype(np.float32)
+        if integer:
+            c = np.rint(c)
+        scale = 20.0
+        q = rng.integers(0, 256, (nq, d)).astype(np.uint8)
+    else:
+        c = rng.normal(0, 1, (nlist, d)).astype(np.float32)
+        scale = 0.3
+        q = (c[rng.integers(0, nlist, nq)] + rng.normal(0, 0.4, (nq, d))).astype(np.float32)
+    cb = synth.pq_codebooks(pq_m, dsub, scale, seed, integer=integer)
+    ids, offsets = synth.skewed_list_ids(n, nlist, seed, sigma)
+    x = synth.rows_near(c, ids, scale, seed, dtype)
+    probes = synth.distinct_probes(nq, nlist, nprobe, seed)
+    return q, c, cb, ids, offsets, x, probes
+
+
+SHAPES = [
+    # n, nlist, d, pq_m, dtype
+    (3000, 40, 128, 32, "u8"),    # SIFT-shaped, 100M-scale code size (Table 2)
+    (3000, 40, 128, 16, "u8"),    # SIFT-shaped, 1B-scale code size
+    (2500, 30, 96, 32, "f32"),    # DEEP-shaped, sub-vectors of 3
+    (2500, 30, 96, 16, "f32"),    # DEEP-shaped, sub-vectors of 6
+    (2000, 25, 100, 20, "f32"),   # SPACEV-shaped width, 4-byte code path
+    (2000, 25, 100, 50, "f32"),   # SPACEV-shaped width, byte code path
+    (500, 7, 8, 8, "f32"),        # one coordinate per subspace
+    (500, 7, 16, 1, "u8"),        # a single subspace
+]
+
+
+@pytest.mark.parametrize("n,nlist,d,pq_m,dtype", SHAPES)
+def test_encode_is_bit_identical(n, nlist, d, pq_m, dtype):
+    q, c, cb, ids, offsets, x, probes = _problem(1, n, nlist, d, pq_m, dtype, 4, 2)
+    want = O.pq_encode(x, ids, c, cb)
+    got = B.ivf_pq_encode(_t(x), _t(ids), _t(c), _t(cb))
+    B.ivf_check()
+    assert (got.cpu().numpy() == want).all()
+
+
+def _check_search(q, c, cb, offsets, codes, probes, n_rerank, vec_ids=None):
+    want_pos, want_est, want_cnt = O.pq_search(q, c, probes, offsets, codes, cb, n_rerank)
+    got_pos, got_est, got_cnt = B.ivf_pq_search(_t(q), _t(c), _t(probes), _t(offsets), _t(codes), _t(cb), n_rerank,
+                                                vec_ids=None if vec_ids is None else _t(vec_ids))
+    B.ivf_check()
+    got_pos, got_est, got_cnt = got_pos.cpu().numpy(), got_est.cpu().numpy(), got_cnt.cpu().numpy()
+    assert (got_cnt == want_cnt).all()
+    if vec_ids is not None:
+        want_pos = np.where(want_pos >= 0, vec_ids[np.maximum(want_pos, 0)], -1)
+    assert (got_pos == want_pos).all()
+    assert (got_est.view(np.uint32) == want_est.view(np.uint32)).all()
+
+
+@pytest.mark.parametrize("n,nlist,d,pq_m,dtype", SHAPES)
+@pytest.mark.parametrize("nq,nprobe,n_rerank", [(1, 1, 16), (9, 5, 64), (37, 7, 512)])
+def test_search_is_bit_identical(n, nlist, d, pq_m, dtype, nq, nprobe, n_rerank):
+    nprobe = min(nprobe, nlist)
+    q, c, cb, ids, offsets, x, probes = _problem(2, n, nlist, d, pq_m, dtype, nq, nprobe)
+    codes = O.pq_encode(x, ids, c, cb)
+    _check_search(q, c, cb, offsets, codes, probes, n_rerank)
+
+
+@pytest.mark.parametrize("n_rerank", [1, 100, 512, 1024])
+def test_long_lists_many_buffer_cuts_and_ties(n_rerank):
+    # a few very long lists (many chunks per group, the buffer is cut back again and again) and
+    # integer data, where equal estimates are plentiful: the (estimate, position) order must hold
+    q, c, cb, ids, offsets, x, probes = _problem(3, 60000, 12, 32, 8, "u8", 5, 6, sigma=1.5, integer=True)
+    codes = O.pq_encode(x, ids, c, cb)
+    assert (offsets[1:] - offsets[:-1]).max() > 8 * 512
+    _check_search(q, c, cb, offsets, codes, probes, n_rerank)
+
+
+def test_batches_that_split_queries_into_many_groups_and_into_one():
+    q, c, cb, ids, offsets, x, probes = _problem(4, 40000, 300, 64, 16, "f32", 3000, 16)
+    codes = O.pq_encode(x, ids, c, cb)
+    _check_search(q[:2], c, cb, offsets, codes, probes[:2], 256)      # 256 groups per query
+    _check_search(q[:300], c, cb, offsets, codes, probes[:300], 128)  # 4 groups per query
+    _check_search(q, c, cb, offsets, codes, probes, 64)               # 1 group per query
+
+
+def test_fewer_candidates_than_slots_empty_lists_and_identifier_map():
+    q, c, cb, ids, offsets, x, probes = _problem(5, 400, 60, 32, 8, "f32", 20, 3, sigma=2.0)
+    lens = offsets[1:] - offsets[:-1]
+    assert (lens == 0).any()
+    probes[0, :] = np.flatnonzero(lens == 0)[:1].tolist() + np.flatnonzero(lens > 0)[:2].tolist()
+    probes[1, :] = np.argsort(lens)[:3]  # the three shortest lists
+    codes = O.pq_encode(x, ids, c, cb)
+    vec_ids = np.random.default_rng(0).permutation(len(x)).astype(np.int64) + 10 ** 10
+    _check_search(q, c, cb, offsets, codes, probes, 512)
+    _check_search(q, c, cb, offsets, codes, probes, 512, vec_ids=vec_ids)
+
+
+def test_bad_ids_are_flagged_not_followed():
+    q, c, cb, ids, offsets, x, probes = _problem(6, 300, 10, 32, 8, "f32", 4, 2)
+    bad = ids.copy()
+    bad[5] = 10
+    codes = B.ivf_pq_encode(_t(x), _t(bad), _t(c), _t(cb))
+    with pytest.raises(B.IvfError) as e:
+        B.ivf_check()
+    assert e.value.code == B.IVF_ERR_BAD_ID
+    assert (codes[5].cpu().numpy() == 0).all()
+    good = O.pq_encode(x, ids, c, cb)
+    badp = probes.copy()
+    badp[0, 0] = -3
+    pos, est, cnt = B.ivf_pq_search(_t(q), _t(c), _t(badp), _t(offsets), _t(good), _t(cb), 8)
+    with pytest.raises(B.IvfError):
+        B.ivf_check()
+    # the query simply loses that probe
+    l = badp[0, 1]
+    assert cnt[0].item() == offsets[l + 1] - offsets[l]
+
+
+def test_argument_checks():
+    q, c, cb, ids, offsets, x, probes = _problem(7, 100, 5, 32, 8, "f32", 2, 2)
+    codes = _t(O.pq_encode(x, ids, c, cb))
+    with pytest.raises(B.IvfError) as e:
+        B.ivf_pq_search(_t(q), _t(c), _t(probes), _t(offsets), codes, _t(cb), 2000)
+    assert e.value.code == B.IVF_ERR_UNSUPPORTED
+    big = torch.zeros((64, 256, 4), dtype=torch.float32, device=DEV)  # d = 256: codebook does not fit
+    with pytest.raises(B.IvfError) as e:
+        B.ivf_pq_encode(torch.zeros((4, 256), device=DEV), torch.zeros(4, dtype=torch.int32, device=DEV),
+                        torch.zeros((2, 256), device=DEV), big)
+    assert e.value.code == B.IVF_ERR_UNSUPPORTED
