@@ -220,6 +220,8 @@ int ivf_debug_rule(int k, int nlist, int out[2]);
  * the merge, rows recomputed by brute force -- clears them, and switches the counting on or off.
  */
 int ivf_debug_stats(int enable, int64_t out[3]);
+/* Test hook: groups per query used by ivf_pq_search (clamped to [1, 256]); 0 = chosen from the sizes. */
+int ivf_debug_set_pq_groups(int groups);
 int ivf_debug_timing(int enable);
 int ivf_debug_timing_read(double ms[9], int64_t launches[9]);
 
@@ -234,14 +236,14 @@ int ivf_debug_timing_read(double ms[9], int64_t launches[9]);
  *     acc = fma(diff, diff, acc);   estimate: acc = 0, for m ascending: acc = acc + LUT_m[a_m].
  *
  * codebooks  [pq_m][256][d / pq_m] float32, row-major.  pq_m must divide d, and
- *            1024 * (d + pq_m) + 4 * d + 17,472 bytes of shared memory must fit one SM's 227 KB
+ *            1024 * (d + pq_m) + 4 * d + 29,776 bytes of shared memory must fit one SM's 227 KB
  *            (d = 128 with pq_m = 32 does; d = 256 does not) -> IVF_ERR_UNSUPPORTED otherwise.
  *
  * ivf_pq_encode: out_codes[i][m] = arg-min over j of the table of x_i - centroids[ids[i]]
  *            (Eq. 3 on the residual; ties to the lower j).  An id outside [0, nlist) writes zero
  *            codes for that row and sets the sticky status IVF_ERR_BAD_ID.
  *
- * ivf_pq_search: for every query the codes of its nprobe probed lists (list l = positions
+ * ivf_pq_search: for every query the codes of its nprobe (<= 512) probed lists (list l = positions
  *            [list_offsets[l], list_offsets[l+1]) of the list-major `codes` array, n_codes rows in
  *            all, n_codes < 2^32) are scored with the (query, list) table (Eq. 4 on q - c_l, Eq. 5) and
  *            the n_rerank (<= 1024) smallest estimates are kept: out_ids [nq][n_rerank] = position

@@ -70,28 +70,31 @@ static void residual(const void *x, int xtype, int64_t row, const float *c, int6
 int oracle_pq_encode(const void *x, int xtype, int64_t n, int d, const int32_t *ids, const float *c,
                      int32_t nlist, const float *codebooks, int pq_m, uint8_t *codes) {
     if (n < 0 || d <= 0 || pq_m <= 0 || d % pq_m != 0) return -1;
-    float *r = (float *)malloc(sizeof(float) * (size_t)d);
-    float *lut = (float *)malloc(sizeof(float) * (size_t)pq_m * PQ_K);
-    if (!r || !lut) {
-        free(r); free(lut);
-        return -1;
-    }
     int rc = 0;
-    for (int64_t i = 0; i < n && rc == 0; ++i) {
-        if (ids[i] < 0 || ids[i] >= nlist) {
+    for (int64_t i = 0; i < n; ++i)
+        if (ids[i] < 0 || ids[i] >= nlist) return -1;
+#pragma omp parallel
+    {
+        float *r = (float *)malloc(sizeof(float) * (size_t)d);
+        float *lut = (float *)malloc(sizeof(float) * (size_t)pq_m * PQ_K);
+        if (!r || !lut) {
+#pragma omp atomic write
             rc = -1;
-            break;
         }
-        residual(x, xtype, i, c, ids[i], d, r);
-        oracle_pq_lut(r, d, pq_m, codebooks, lut);
-        for (int m = 0; m < pq_m; ++m) {
-            int best = 0;
-            for (int j = 1; j < PQ_K; ++j)
-                if (lut[m * PQ_K + j] < lut[m * PQ_K + best]) best = j;  /* strict: ties keep the lower j */
-            codes[i * pq_m + m] = (uint8_t)best;
+#pragma omp for schedule(static)
+        for (int64_t i = 0; i < n; ++i) {
+            if (!r || !lut) continue;
+            residual(x, xtype, i, c, ids[i], d, r);
+            oracle_pq_lut(r, d, pq_m, codebooks, lut);
+            for (int m = 0; m < pq_m; ++m) {
+                int best = 0;
+                for (int j = 1; j < PQ_K; ++j)
+                    if (lut[m * PQ_K + j] < lut[m * PQ_K + best]) best = j;  /* strict: ties keep the lower j */
+                codes[i * pq_m + m] = (uint8_t)best;
+            }
         }
+        free(r); free(lut);
     }
-    free(r); free(lut);
     return rc;
 }
 
@@ -116,6 +119,46 @@ void oracle_pq_adc(const float *lut, int pq_m, const uint8_t *codes, int64_t p0,
     }
 }
 
+static int search_one(const void *q, int qtype, int64_t b, int d, const float *c, int32_t nlist,
+                      const int32_t *probes, int nprobe, const int64_t *offsets, const uint8_t *codes,
+                      const float *codebooks, int pq_m, int n_rerank, int64_t *out_pos, float *out_est,
+                      int64_t *out_count) {
+    int64_t total = 0;
+    for (int p = 0; p < nprobe; ++p) {
+        const int32_t l = probes[b * nprobe + p];
+        if (l < 0 || l >= nlist) return -1;
+        total += offsets[l + 1] - offsets[l];
+    }
+    float *r = (float *)malloc(sizeof(float) * (size_t)d);
+    float *lut = (float *)malloc(sizeof(float) * (size_t)pq_m * PQ_K);
+    cand_t *cand = (cand_t *)malloc(sizeof(cand_t) * (size_t)(total > 0 ? total : 1));
+    float *est = (float *)malloc(sizeof(float) * (size_t)(total > 0 ? total : 1));
+    if (!r || !lut || !cand || !est) {
+        free(r); free(lut); free(cand); free(est);
+        return -1;
+    }
+    int64_t at = 0;
+    for (int p = 0; p < nprobe; ++p) {
+        const int32_t l = probes[b * nprobe + p];
+        residual(q, qtype, b, c, l, d, r);
+        oracle_pq_lut(r, d, pq_m, codebooks, lut);
+        oracle_pq_adc(lut, pq_m, codes, offsets[l], offsets[l + 1], est);
+        for (int64_t i = 0; i < offsets[l + 1] - offsets[l]; ++i) {
+            cand[at].est = est[i];
+            cand[at].pos = offsets[l] + i;
+            ++at;
+        }
+    }
+    qsort(cand, (size_t)total, sizeof(cand_t), cand_cmp);
+    for (int s = 0; s < n_rerank; ++s) {
+        out_pos[b * n_rerank + s] = s < total ? cand[s].pos : -1;
+        out_est[b * n_rerank + s] = s < total ? cand[s].est : INFINITY;
+    }
+    if (out_count) out_count[b] = total;
+    free(r); free(lut); free(cand); free(est);
+    return 0;
+}
+
 /*
  * Candidate reduction.  For every query: the codes of its nprobe probed lists (list l occupies
  * positions [offsets[l], offsets[l+1]) of the list-major code array) are scored by ADC with that
@@ -130,51 +173,14 @@ int oracle_pq_search(const void *q, int qtype, int64_t nq, int d, const float *c
                      const float *codebooks, int pq_m, int n_rerank, int64_t *out_pos, float *out_est,
                      int64_t *out_count) {
     if (nq < 0 || d <= 0 || pq_m <= 0 || d % pq_m != 0 || nprobe <= 0 || n_rerank <= 0) return -1;
-    float *r = (float *)malloc(sizeof(float) * (size_t)d);
-    float *lut = (float *)malloc(sizeof(float) * (size_t)pq_m * PQ_K);
-    if (!r || !lut) {
-        free(r); free(lut);
-        return -1;
-    }
     int rc = 0;
-    for (int64_t b = 0; b < nq && rc == 0; ++b) {
-        int64_t total = 0;
-        for (int p = 0; p < nprobe; ++p) {
-            const int32_t l = probes[b * nprobe + p];
-            if (l < 0 || l >= nlist) {
-                rc = -1;
-                break;
-            }
-            total += offsets[l + 1] - offsets[l];
-        }
-        if (rc) break;
-        cand_t *cand = (cand_t *)malloc(sizeof(cand_t) * (size_t)(total > 0 ? total : 1));
-        float *est = (float *)malloc(sizeof(float) * (size_t)(total > 0 ? total : 1));
-        if (!cand || !est) {
-            free(cand); free(est);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t b = 0; b < nq; ++b) {
+        if (search_one(q, qtype, b, d, c, nlist, probes, nprobe, offsets, codes, codebooks, pq_m, n_rerank, out_pos,
+                       out_est, out_count) != 0) {
+#pragma omp atomic write
             rc = -1;
-            break;
         }
-        int64_t at = 0;
-        for (int p = 0; p < nprobe; ++p) {
-            const int32_t l = probes[b * nprobe + p];
-            residual(q, qtype, b, c, l, d, r);
-            oracle_pq_lut(r, d, pq_m, codebooks, lut);
-            oracle_pq_adc(lut, pq_m, codes, offsets[l], offsets[l + 1], est);
-            for (int64_t i = 0; i < offsets[l + 1] - offsets[l]; ++i) {
-                cand[at].est = est[i];
-                cand[at].pos = offsets[l] + i;
-                ++at;
-            }
-        }
-        qsort(cand, (size_t)total, sizeof(cand_t), cand_cmp);
-        for (int s = 0; s < n_rerank; ++s) {
-            out_pos[b * n_rerank + s] = s < total ? cand[s].pos : -1;
-            out_est[b * n_rerank + s] = s < total ? cand[s].est : INFINITY;
-        }
-        if (out_count) out_count[b] = total;
-        free(cand); free(est);
     }
-    free(r); free(lut);
     return rc;
 }

@@ -328,6 +328,7 @@ struct CentroidPrep {
 };
 
 int g_force_fallback = 0;
+int g_pq_groups = 0;  // test hook: groups per query of ivf_pq_search (0 = chosen from the sizes)
 bool g_stats = false;
 std::atomic<int64_t> g_row_chunk_override{0};  // test hook: rows per fused launch
 
@@ -1011,7 +1012,7 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     if (qtype != IVF_F32 && qtype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)qtype);
     if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
     if (nprobe < 1 || nprobe > nlist) return fail(IVF_ERR_INVALID_ARG, "nprobe = %d with nlist = %d", nprobe, nlist);
-    if (nprobe > 4096) return fail(IVF_ERR_UNSUPPORTED, "nprobe = %d: at most 4096", nprobe);
+    if (nprobe > kPqMaxProbes) return fail(IVF_ERR_UNSUPPORTED, "nprobe = %d: at most %d", nprobe, kPqMaxProbes);
     if (n_rerank < 1 || n_rerank > kPqMaxRerank)
         return fail(IVF_ERR_UNSUPPORTED, "n_rerank = %d: must be in [1, %d]", n_rerank, kPqMaxRerank);
     if (n_codes < 0 || n_codes >= (int64_t(1) << 32))
@@ -1031,7 +1032,13 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     if (rc != IVF_OK) return rc;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     // groups per query: enough CTAs of work for every SM even at serving-size batches
+    // (but no more than one per ~4 chunks of the codes a query is expected to scan: a group hands
+    // on up to n_rerank candidates however little it scanned)
     int ngroups = static_cast<int>((8 * static_cast<int64_t>(ctx.num_sms) + nq - 1) / nq);
+    const int64_t expect_codes = static_cast<int64_t>(nprobe) * (n_codes / nlist + 1);
+    const int64_t by_work = expect_codes / (4 * kPqChunk);
+    if (ngroups > by_work) ngroups = static_cast<int>(by_work);
+    if (g_pq_groups > 0) ngroups = g_pq_groups;
     if (ngroups < 1) ngroups = 1;
     if (ngroups > 256) ngroups = 256;
     const int64_t total_groups = nq * ngroups;
@@ -1207,6 +1214,11 @@ int ivf_debug_rule(int k, int nlist, int out[2]) {
 
 int ivf_debug_set_row_chunk(int64_t rows) {
     g_row_chunk_override.store(rows > 0 ? rows : 0);
+    return IVF_OK;
+}
+
+int ivf_debug_set_pq_groups(int groups) {
+    g_pq_groups = groups < 0 ? 0 : groups;
     return IVF_OK;
 }
 

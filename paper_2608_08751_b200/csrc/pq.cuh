@@ -25,15 +25,17 @@
 namespace ivf {
 
 constexpr int kPqK = 256;          // codewords per subspace (one byte per sub-code)
-constexpr int kPqThreads = 512;
-constexpr int kPqChunk = 512;      // codes per chunk = one code per thread
+constexpr int kPqThreads = 1024;
+constexpr int kPqChunk = 1024;     // codes per chunk = one code per thread
 constexpr int kPqBufKeys = 2048;   // candidate buffer of a group
 constexpr int kPqMaxRerank = 1024;
+constexpr int kPqMaxProbes = 512;   // lists per query (the paper sweeps the probe count up to 512)
 constexpr int kPqStatusBadId = -6;
 
 __host__ __device__ inline size_t pq_smem_bytes(int d, int pq_m) {
     return static_cast<size_t>(d) * kPqK * 4 + static_cast<size_t>(pq_m) * kPqK * 4 + static_cast<size_t>(d) * 4 +
-           static_cast<size_t>(kPqBufKeys) * 8 + 256 * 4 + 64;
+           static_cast<size_t>(kPqBufKeys) * 8 + 256 * 4 + 64 +
+           static_cast<size_t>(kPqMaxProbes) * 24 + 16;  // probe descriptors
 }
 
 struct PqSmem {
@@ -43,12 +45,20 @@ struct PqSmem {
     uint64_t* buf;  // [kPqBufKeys]
     int* hist;      // [256]
     int* misc;      // [16]: 0 count, 1 digit, 2 rank, 3 eq
+    long long* list_begin;  // [kPqMaxProbes] first position of each probed list
+    long long* list_len;    // [kPqMaxProbes]
+    int* list_id;           // [kPqMaxProbes]
+    int* cs;                // [kPqMaxProbes + 1] chunk prefix of the query
 };
 
 __device__ __forceinline__ PqSmem pq_carve(uint8_t* raw, int d, int pq_m) {
     PqSmem s;
     s.buf = reinterpret_cast<uint64_t*>(raw);
     raw += static_cast<size_t>(kPqBufKeys) * 8;
+    s.list_begin = reinterpret_cast<long long*>(raw);
+    raw += static_cast<size_t>(kPqMaxProbes) * 8;
+    s.list_len = reinterpret_cast<long long*>(raw);
+    raw += static_cast<size_t>(kPqMaxProbes) * 8;
     s.cbt = reinterpret_cast<float*>(raw);
     raw += static_cast<size_t>(d) * kPqK * 4;
     s.lut = reinterpret_cast<float*>(raw);
@@ -58,6 +68,10 @@ __device__ __forceinline__ PqSmem pq_carve(uint8_t* raw, int d, int pq_m) {
     s.hist = reinterpret_cast<int*>(raw);
     raw += 256 * 4;
     s.misc = reinterpret_cast<int*>(raw);
+    raw += 64;
+    s.list_id = reinterpret_cast<int*>(raw);
+    raw += static_cast<size_t>(kPqMaxProbes) * 4;
+    s.cs = reinterpret_cast<int*>(raw);
     return s;
 }
 
@@ -78,6 +92,29 @@ __device__ __forceinline__ void pq_load_codebooks(const float* __restrict__ code
 __device__ __forceinline__ void pq_build_lut(const PqSmem& s, int pq_m, int dsub) {
     const int j = threadIdx.x & (kPqK - 1);
     const int step = blockDim.x >> 8;
+    if ((dsub & 3) == 0) {
+        // the residual's sub-vector comes in with 16-byte broadcast loads; same operation order
+        for (int m = threadIdx.x >> 8; m < pq_m; m += step) {
+            const float* col = s.cbt + static_cast<size_t>(m) * dsub * kPqK + j;
+            const float4* r4 = reinterpret_cast<const float4*>(s.r + m * dsub);
+            float acc = 0.0f;
+            for (int t4 = 0; t4 < (dsub >> 2); ++t4) {
+                const float4 rv = r4[t4];
+                const float c0 = col[(4 * t4 + 0) * kPqK], c1 = col[(4 * t4 + 1) * kPqK];
+                const float c2 = col[(4 * t4 + 2) * kPqK], c3 = col[(4 * t4 + 3) * kPqK];
+                float diff = __fsub_rn(rv.x, c0);
+                acc = __fmaf_rn(diff, diff, acc);
+                diff = __fsub_rn(rv.y, c1);
+                acc = __fmaf_rn(diff, diff, acc);
+                diff = __fsub_rn(rv.z, c2);
+                acc = __fmaf_rn(diff, diff, acc);
+                diff = __fsub_rn(rv.w, c3);
+                acc = __fmaf_rn(diff, diff, acc);
+            }
+            s.lut[m * kPqK + j] = acc;
+        }
+        return;
+    }
     for (int m = threadIdx.x >> 8; m < pq_m; m += step) {
         const float* col = s.cbt + static_cast<size_t>(m) * dsub * kPqK + j;
         const float* r = s.r + m * dsub;
@@ -221,9 +258,11 @@ __global__ void __launch_bounds__(128) pq_setup_query_kernel(const int32_t* __re
 }
 
 // ------------------------------------------------------------------ block-wide selection of the k smallest keys
-// Largest admitted key among `count` distinct 64-bit keys in shared memory (count > k): radix
+// Largest admitted key among the `count` distinct 64-bit keys get(0 .. count) (count > k; keys that
+// read as all-ones are padding and must number fewer than count - k): radix
 // select from the top byte down, stopping once the digit that holds rank k is wanted whole.
-__device__ __forceinline__ uint64_t pq_select_bound(const uint64_t* keys, int count, int k, int* hist, int* misc) {
+template <typename Get>
+__device__ __forceinline__ uint64_t pq_select_bound(Get get, int count, int k, int* hist, int* misc) {
     const int lane = threadIdx.x & 31;
     uint64_t prefix = 0, mask = 0;
     int rank = k;
@@ -234,7 +273,7 @@ __device__ __forceinline__ uint64_t pq_select_bound(const uint64_t* keys, int co
         for (int i = threadIdx.x; i < rounded; i += blockDim.x) {
             uint32_t dg = 0xFFFFFFFFu;
             if (i < count) {
-                const uint64_t v = keys[i];
+                const uint64_t v = get(i);
                 if ((v & mask) == prefix) dg = static_cast<uint32_t>(v >> shift) & 255u;
             }
             const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dg);
@@ -264,7 +303,7 @@ __device__ __forceinline__ uint64_t pq_select_bound(const uint64_t* keys, int co
 // Cuts the buffer back to its k smallest keys (in no particular order); returns the bound, i.e.
 // the largest key kept.  count > k on entry; on exit misc[0] == k.
 __device__ __forceinline__ uint64_t pq_cut_buffer(uint64_t* buf, int count, int k, int* hist, int* misc) {
-    const uint64_t bound = pq_select_bound(buf, count, k, hist, misc);
+    const uint64_t bound = pq_select_bound([buf](int i) { return buf[i]; }, count, k, hist, misc);
     constexpr int kPer = kPqBufKeys / kPqThreads;
     uint64_t mine[kPer];
 #pragma unroll
@@ -299,6 +338,31 @@ struct PqScanParams {
     int* status;
 };
 
+// The code bytes of one stored vector, held in registers so that the next chunk's bytes can be
+// fetched while the current chunk is being scored (sub-code counts that are a multiple of 16, up
+// to 32, take this path; others are read byte-wise while scoring).
+struct PqCodeRegs {
+    uint4 w[2];
+};
+__device__ __forceinline__ bool pq_codes_in_regs(int pq_m) { return pq_m == 16 || pq_m == 32; }
+__device__ __forceinline__ void pq_fetch_code(PqCodeRegs& c, const uint8_t* code, int pq_m) {
+    c.w[0] = __ldg(reinterpret_cast<const uint4*>(code));
+    if (pq_m == 32) c.w[1] = __ldg(reinterpret_cast<const uint4*>(code + 16));
+}
+__device__ __forceinline__ float pq_adc_regs(const float* lut, const PqCodeRegs& c, int pq_m) {
+    float acc = 0.0f;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        if (h * 16 < pq_m) {
+            const uint32_t w[4] = {c.w[h].x, c.w[h].y, c.w[h].z, c.w[h].w};
+#pragma unroll
+            for (int q = 0; q < 16; ++q)
+                acc = __fadd_rn(acc, lut[(h * 16 + q) * kPqK + ((w[q >> 2] >> (8 * (q & 3))) & 255u)]);
+        }
+    }
+    return acc;
+}
+
 __device__ __forceinline__ float pq_adc_code(const float* lut, const uint8_t* code, int pq_m) {
     float acc = 0.0f;
     if ((pq_m & 15) == 0) {
@@ -330,60 +394,106 @@ __global__ void __launch_bounds__(kPqThreads, 1) pq_scan_kernel(const PqScanPara
     pq_load_codebooks(p.codebooks, p.d, dsub, s.cbt);
     const int lane = threadIdx.x & 31;
     const uint32_t lt_mask = (1u << lane) - 1u;
+    const bool in_regs = pq_codes_in_regs(p.pq_m);
 
     for (int64_t g = blockIdx.x; g < total_groups; g += gridDim.x) {
         const int64_t b = g / p.ngroups;
         const int gi = static_cast<int>(g - b * p.ngroups);
-        const int* cs = p.chunk_start + static_cast<size_t>(b) * (p.nprobe + 1);
-        const int group_chunks = (cs[p.nprobe] + p.ngroups - 1) / p.ngroups;
-        const int chunk0 = min(cs[p.nprobe], gi * group_chunks);
-        const int chunk1 = min(cs[p.nprobe], chunk0 + group_chunks);
-        __syncthreads();
-        if (threadIdx.x == 0) s.misc[0] = 0;
-        uint64_t bound = ~0ull;  // a candidate must be below this key to matter
-        int cur_probe = -1;
-        long long list_begin = 0, list_len = 0;
-        for (int ch = chunk0; ch < chunk1; ++ch) {
-            // probe that owns chunk ch: the last pr with cs[pr] <= ch (empty lists own no chunk)
-            int plo = max(cur_probe, 0), phi = p.nprobe;
-            while (phi - plo > 1) {
-                const int mid = (plo + phi) >> 1;
-                if (cs[mid] <= ch) plo = mid; else phi = mid;
+        const int* cs_g = p.chunk_start + static_cast<size_t>(b) * (p.nprobe + 1);
+        __syncthreads();  // the previous group's descriptors, table and buffer are no longer in use
+        // the query's probe descriptors, once per group: chunk prefix, list begin, list length
+        for (int pr = threadIdx.x; pr <= p.nprobe; pr += blockDim.x) {
+            s.cs[pr] = cs_g[pr];
+            if (pr < p.nprobe) {
+                const int l = p.probes[static_cast<size_t>(b) * p.nprobe + pr];
+                long long begin = 0, len = 0;
+                if (l >= 0 && l < p.nlist) {
+                    begin = p.offsets[l];
+                    len = p.offsets[l + 1] - begin;
+                }
+                s.list_id[pr] = l;
+                s.list_begin[pr] = begin;
+                s.list_len[pr] = len;
             }
-            if (plo != cur_probe) {
-                cur_probe = plo;
-                const int l = p.probes[static_cast<size_t>(b) * p.nprobe + plo];
-                list_begin = p.offsets[l];
-                list_len = p.offsets[l + 1] - list_begin;
-                __syncthreads();  // the previous table is no longer read
-                for (int t = threadIdx.x; t < p.d; t += blockDim.x) {
-                    const float qv = p.q_is_u8 ? pq_elem(static_cast<const uint8_t*>(p.q), b * p.d + t)
-                                               : pq_elem(static_cast<const float*>(p.q), b * p.d + t);
-                    s.r[t] = __fsub_rn(qv, p.centroids[static_cast<int64_t>(l) * p.d + t]);
+        }
+        if (threadIdx.x == 0) s.misc[0] = 0;
+        __syncthreads();
+        const int nchunks = s.cs[p.nprobe];
+        const int group_chunks = (nchunks + p.ngroups - 1) / p.ngroups;
+        const int chunk0 = min(nchunks, gi * group_chunks);
+        const int chunk1 = min(nchunks, chunk0 + group_chunks);
+        uint64_t bound = ~0ull;  // a candidate must be below this key to matter
+        if (chunk0 < chunk1) {
+            // owner of chunk0: the last probe pr with cs[pr] <= chunk0 (empty lists own no chunk)
+            int pr = 0;
+            {
+                int hi = p.nprobe;
+                while (hi - pr > 1) {
+                    const int mid = (pr + hi) >> 1;
+                    if (s.cs[mid] <= chunk0) pr = mid; else hi = mid;
+                }
+            }
+            float qv = 0.0f, cnext = 0.0f;  // thread t < d: its query coordinate, the coming list's centroid coordinate
+            if (threadIdx.x < p.d) {
+                qv = p.q_is_u8 ? pq_elem(static_cast<const uint8_t*>(p.q), b * p.d + threadIdx.x)
+                               : pq_elem(static_cast<const float*>(p.q), b * p.d + threadIdx.x);
+                cnext = p.centroids[static_cast<int64_t>(s.list_id[pr]) * p.d + threadIdx.x];
+            }
+            int built = -1;
+            // the code of the first chunk
+            PqCodeRegs nxt;
+            nxt.w[0] = nxt.w[1] = make_uint4(0, 0, 0, 0);
+            long long nxt_pos = -1;
+            {
+                const long long in_list = static_cast<long long>(chunk0 - s.cs[pr]) * kPqChunk + threadIdx.x;
+                if (in_list < s.list_len[pr]) nxt_pos = s.list_begin[pr] + in_list;
+                if (in_regs && nxt_pos >= 0) pq_fetch_code(nxt, p.codes + nxt_pos * p.pq_m, p.pq_m);
+            }
+            int npr = pr;  // owner of the chunk whose code is in `nxt`
+            for (int ch = chunk0; ch < chunk1; ++ch) {
+                pr = npr;
+                if (pr != built) {
+                    __syncthreads();  // the previous table is no longer read
+                    if (threadIdx.x < p.d) s.r[threadIdx.x] = __fsub_rn(qv, cnext);
+                    // fetch the centroid of the next list that owns a chunk of this group
+                    int later = pr + 1;
+                    while (later < p.nprobe && s.cs[later + 1] == s.cs[later]) ++later;
+                    if (later < p.nprobe && s.cs[later] < chunk1 && threadIdx.x < p.d)
+                        cnext = p.centroids[static_cast<int64_t>(s.list_id[later]) * p.d + threadIdx.x];
+                    __syncthreads();
+                    pq_build_lut(s, p.pq_m, dsub);
+                    __syncthreads();
+                    built = pr;
+                }
+                const long long pos = nxt_pos;
+                const PqCodeRegs cur = nxt;
+                // fetch the next chunk's code while this one is scored
+                nxt_pos = -1;
+                if (ch + 1 < chunk1) {
+                    while (s.cs[npr + 1] <= ch + 1) ++npr;
+                    const long long in_list = static_cast<long long>(ch + 1 - s.cs[npr]) * kPqChunk + threadIdx.x;
+                    if (in_list < s.list_len[npr]) nxt_pos = s.list_begin[npr] + in_list;
+                    if (in_regs && nxt_pos >= 0) pq_fetch_code(nxt, p.codes + nxt_pos * p.pq_m, p.pq_m);
+                }
+                bool hit = false;
+                uint64_t key = 0;
+                if (pos >= 0) {
+                    const float est = in_regs ? pq_adc_regs(s.lut, cur, p.pq_m)
+                                              : pq_adc_code(s.lut, p.codes + pos * p.pq_m, p.pq_m);
+                    key = (static_cast<uint64_t>(orderable(est)) << 32) | static_cast<uint32_t>(pos);
+                    hit = key < bound;
+                }
+                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, hit);
+                if (bal) {
+                    int base = 0;
+                    if (lane == 0) base = atomicAdd(&s.misc[0], __popc(bal));
+                    base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                    if (hit) s.buf[base + __popc(bal & lt_mask)] = key;
                 }
                 __syncthreads();
-                pq_build_lut(s, p.pq_m, dsub);
-                __syncthreads();
+                const int count = s.misc[0];
+                if (count > kPqBufKeys - kPqChunk) bound = pq_cut_buffer(s.buf, count, p.n_rerank, s.hist, s.misc);
             }
-            const long long in_list = static_cast<long long>(ch - cs[cur_probe]) * kPqChunk + threadIdx.x;
-            bool hit = false;
-            uint64_t key = 0;
-            if (in_list < list_len) {
-                const long long pos = list_begin + in_list;
-                const float est = pq_adc_code(s.lut, p.codes + pos * p.pq_m, p.pq_m);
-                key = (static_cast<uint64_t>(orderable(est)) << 32) | static_cast<uint32_t>(pos);
-                hit = key < bound;
-            }
-            const uint32_t bal = __ballot_sync(0xFFFFFFFFu, hit);
-            if (bal) {
-                int base = 0;
-                if (lane == 0) base = atomicAdd(&s.misc[0], __popc(bal));
-                base = __shfl_sync(0xFFFFFFFFu, base, 0);
-                if (hit) s.buf[base + __popc(bal & lt_mask)] = key;
-            }
-            __syncthreads();
-            const int count = s.misc[0];
-            if (count > kPqBufKeys - kPqChunk) bound = pq_cut_buffer(s.buf, count, p.n_rerank, s.hist, s.misc);
         }
         __syncthreads();
         int count = s.misc[0];
@@ -409,31 +519,39 @@ struct PqMergeParams {
     float* out_est;            // [nq][n_rerank]
 };
 
-// One CTA per query.  The query's group candidates are cut to the n_rerank smallest in rounds
-// through the same shared-memory buffer, sorted, and written in ascending (estimate, position) order.
+// One CTA per query.  The n_rerank smallest of the query's group candidates are selected (in shared
+// memory when they all fit, else by a radix select over the group outputs in place), sorted, and
+// written in ascending (estimate, position) order.
 __global__ void __launch_bounds__(kPqThreads) pq_merge_kernel(const PqMergeParams p) {
     __shared__ uint64_t buf[kPqBufKeys];
     __shared__ int hist[256];
     __shared__ int misc[16];
     const int64_t b = blockIdx.x;
-    const int64_t g0 = b * p.ngroups, g1 = g0 + p.ngroups;
-    int count = 0;
-    for (int64_t g = g0; g < g1; ++g) {
-        const int c = p.gcand_count[g];
-        __syncthreads();
-        if (count + c > kPqBufKeys) {
-            if (threadIdx.x == 0) misc[0] = count;
-            __syncthreads();
-            pq_cut_buffer(buf, count, p.n_rerank, hist, misc);
-            count = p.n_rerank;
-        }
-        const uint64_t* src = p.gcand + static_cast<size_t>(g) * p.n_rerank;
-        for (int i = threadIdx.x; i < c; i += blockDim.x) buf[count + i] = src[i];
-        count += c;
+    const uint64_t* cand = p.gcand + static_cast<size_t>(b) * p.ngroups * p.n_rerank;
+    const int* cnt = p.gcand_count + b * p.ngroups;
+    const int slots = p.ngroups * p.n_rerank;
+    auto get = [&](int i) {
+        const int g = i / p.n_rerank;
+        return (i - g * p.n_rerank) < cnt[g] ? __ldcg(cand + i) : ~0ull;
+    };
+    if (threadIdx.x == 0) misc[4] = 0;
+    __syncthreads();
+    int mine = 0;
+    for (int g = threadIdx.x; g < p.ngroups; g += blockDim.x) mine += cnt[g];
+    if (mine) atomicAdd(&misc[4], mine);
+    __syncthreads();
+    const int total = misc[4];
+    uint64_t bound = ~0ull;
+    if (total > kPqBufKeys) bound = pq_select_bound(get, slots, p.n_rerank, hist, misc);
+    if (threadIdx.x == 0) misc[0] = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < slots; i += blockDim.x) {
+        const uint64_t v = get(i);
+        if (v != ~0ull && v <= bound) buf[atomicAdd(&misc[0], 1)] = v;
     }
     __syncthreads();
+    int count = misc[0];
     if (count > p.n_rerank) {
-        if (threadIdx.x == 0) misc[0] = count;
         __syncthreads();
         pq_cut_buffer(buf, count, p.n_rerank, hist, misc);
         count = p.n_rerank;

@@ -97,9 +97,88 @@ def serve_case(args):
     print(json.dumps(out))
 
 
+def pq_case(args):
+    """The PQ pipeline on the library's own calls: assign -> list-major reorder -> residual encoding
+    (timed once), then per batch: routing (prepared table) -> candidate reduction (timed)."""
+    d, nlist, pq_m = args.d, args.nlist, args.pq_m
+    dsub = d // pq_m
+    if args.dtype == "u8":
+        c = synth.sift_like_centroids(nlist, d)
+        scale = 20.0
+    else:
+        c = synth.deep_like_centroids(nlist, d)
+        scale = 0.05
+    ct = torch.from_numpy(c).cuda()
+    cb = torch.from_numpy(synth.pq_codebooks(pq_m, dsub, scale, seed=1)).cuda()
+    rows = []
+    done = 0
+    chunk = 0
+    while done < args.n:
+        take = min(synth.CHUNK_ROWS, args.n - done)
+        x = synth.sift_like_rows(chunk, rows=take, d=d) if args.dtype == "u8" else synth.deep_like_rows(chunk, take, d)
+        rows.append(torch.from_numpy(x).cuda())
+        done += take
+        chunk += 1
+    xt = torch.cat(rows)
+    del rows
+    ids, _ = B.ivf_assign(xt, ct)
+    xr, offsets, order = B.ivf_cluster_major_reorder(xt, ids, nlist)
+    ids_sorted = ids[order.long()]
+    del xt
+    B.ivf_pq_encode(xr[:1024], ids_sorted[:1024], ct, cb)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    codes = B.ivf_pq_encode(xr, ids_sorted, ct, cb)
+    e1.record()
+    B.ivf_check()
+    enc_ms = e0.elapsed_time(e1)
+    lens = (offsets[1:] - offsets[:-1]).float()
+    out = {"op": "pq", "n": args.n, "nlist": nlist, "d": d, "pq_m": pq_m, "dtype": args.dtype, "nprobe": args.k,
+           "n_rerank": args.n_rerank, "encode_ms": enc_ms, "encode_vectors_per_s": args.n / (enc_ms / 1e3),
+           "list_len": {"mean": lens.mean().item(), "max": lens.max().item(), "empty": int((lens == 0).sum().item())},
+           "batches": {}}
+    bmax = max(int(v) for v in args.batches.split(","))
+    q_all = synth.sift_like_queries(bmax, d) if args.dtype == "u8" else synth.deep_like_queries(bmax, d)
+    handle = B.PreparedCentroids(ct)
+    for bs in [int(v) for v in args.batches.split(",")]:
+        q = torch.from_numpy(q_all[:bs]).cuda()
+        probes = torch.empty((bs, args.k), dtype=torch.int32, device="cuda")
+        B.ivf_route_prepared(handle, q, args.k, probes, None, want_dists=False)
+        for _ in range(3):
+            pos, est, cnt = B.ivf_pq_search(q, ct, probes, offsets, codes, cb, args.n_rerank)
+        B.ivf_check()
+        reps = max(args.reps, 10)
+        B.ivf_debug_timing(True)
+        e0.record()
+        for _ in range(reps):
+            B.ivf_pq_search(q, ct, probes, offsets, codes, cb, args.n_rerank)
+        e1.record()
+        fam = B.ivf_debug_timing_read()
+        B.ivf_debug_timing(False)
+        us = e0.elapsed_time(e1) / reps * 1e3
+        e0.record()
+        for _ in range(reps):
+            B.ivf_route_prepared(handle, q, args.k, probes, None, want_dists=False)
+            B.ivf_pq_search(q, ct, probes, offsets, codes, cb, args.n_rerank)
+        e1.record()
+        B.ivf_check()
+        both_us = e0.elapsed_time(e1) / reps * 1e3
+        scanned = int(cnt.sum().item())
+        out["batches"][str(bs)] = {
+            "search_us": us, "route_plus_search_us": both_us, "queries_per_s": bs / (both_us / 1e6),
+            "codes_scanned": scanned, "codes_per_s": scanned / (us / 1e6),
+            "lookups_per_s": scanned * pq_m / (us / 1e6), "code_GBps": scanned * pq_m / (us / 1e6) / 1e9,
+            "kernel_us": {k: v[0] / max(v[1], 1) * 1e3 for k, v in fam.items() if v[1]}}
+    handle.close()
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="assign", choices=["assign", "route", "update", "stream", "serve"])
+    ap.add_argument("--op", default="assign", choices=["assign", "route", "update", "stream", "serve", "pq"])
+    ap.add_argument("--pq-m", type=int, default=32, dest="pq_m")
+    ap.add_argument("--n-rerank", type=int, default=512, dest="n_rerank")
     ap.add_argument("--batches", default="8,32,256,2048", help="query batch sizes of --op serve")
     ap.add_argument("--iters", type=int, default=1, help="Lloyd iterations of --op stream")
     ap.add_argument("--n", type=int, default=262144)
@@ -114,6 +193,8 @@ def main():
         return stream_case(args)
     if args.op == "serve":
         return serve_case(args)
+    if args.op == "pq":
+        return pq_case(args)
     if args.dtype == "u8":
         x = synth.sift_like_rows(0, rows=args.n, d=args.d)
         c = synth.sift_like_centroids(args.nlist, args.d)

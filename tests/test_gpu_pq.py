@@ -88,16 +88,28 @@ def test_long_lists_many_buffer_cuts_and_ties(n_rerank):
     # integer data, where equal estimates are plentiful: the (estimate, position) order must hold
     q, c, cb, ids, offsets, x, probes = _problem(3, 60000, 12, 32, 8, "u8", 5, 6, sigma=1.5, integer=True)
     codes = O.pq_encode(x, ids, c, cb)
-    assert (offsets[1:] - offsets[:-1]).max() > 8 * 512
+    assert (offsets[1:] - offsets[:-1]).max() > 8 * 1024
     _check_search(q, c, cb, offsets, codes, probes, n_rerank)
 
 
-def test_batches_that_split_queries_into_many_groups_and_into_one():
-    q, c, cb, ids, offsets, x, probes = _problem(4, 40000, 300, 64, 16, "f32", 3000, 16)
+@pytest.mark.parametrize("groups", [1, 2, 7, 256])
+def test_every_group_count_gives_the_same_result(groups):
+    # the chunks of a query are dealt to `groups` CTAs whose survivors the query merge combines:
+    # in shared memory when they fit, by a select over the group outputs when they do not
+    q, c, cb, ids, offsets, x, probes = _problem(4, 150000, 60, 64, 16, "f32", 6, 16, sigma=1.2)
     codes = O.pq_encode(x, ids, c, cb)
-    _check_search(q[:2], c, cb, offsets, codes, probes[:2], 256)      # 256 groups per query
-    _check_search(q[:300], c, cb, offsets, codes, probes[:300], 128)  # 4 groups per query
-    _check_search(q, c, cb, offsets, codes, probes, 64)               # 1 group per query
+    B.ivf_debug_set_pq_groups(groups)
+    try:
+        _check_search(q, c, cb, offsets, codes, probes, 200)
+        _check_search(q[:2], c, cb, offsets, codes, probes[:2], 1024)
+    finally:
+        B.ivf_debug_set_pq_groups(0)
+
+
+def test_large_batch_one_group_per_query():
+    q, c, cb, ids, offsets, x, probes = _problem(8, 40000, 300, 64, 16, "f32", 3000, 16)
+    codes = O.pq_encode(x, ids, c, cb)
+    _check_search(q, c, cb, offsets, codes, probes, 64)
 
 
 def test_fewer_candidates_than_slots_empty_lists_and_identifier_map():
@@ -143,3 +155,28 @@ def test_argument_checks():
         B.ivf_pq_encode(torch.zeros((4, 256), device=DEV), torch.zeros(4, dtype=torch.int32, device=DEV),
                         torch.zeros((2, 256), device=DEV), big)
     assert e.value.code == B.IVF_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("dtype,d,pq_m", [("u8", 128, 32), ("f32", 96, 16)])
+def test_full_size_batch_in_the_measured_configuration(dtype, d, pq_m):
+    # the launch configuration the timing harness uses (2,048 queries, 64 probes chosen by the
+    # oracle's own routing, N_rerank = 512, lists of about a thousand codes with a skewed length
+    # distribution); every query is compared with the oracle bit for bit
+    n, nlist, nq, nprobe, n_rerank = 1 << 20, 1024, 2048, 64, 512
+    if dtype == "u8":
+        c = synth.sift_like_centroids(nlist, d)
+        q = synth.sift_like_queries(nq, d)
+        scale = 20.0
+    else:
+        c = synth.deep_like_centroids(nlist, d)
+        q = synth.deep_like_queries(nq, d)
+        scale = 0.05
+    cb = synth.pq_codebooks(pq_m, d // pq_m, scale, seed=11)
+    ids, offsets = synth.skewed_list_ids(n, nlist, seed=11, sigma=0.7)
+    x = synth.rows_near(c, ids, scale, 11, dtype)
+    probes, _, _ = O.route(q, c, nprobe)
+    want_codes = O.pq_encode(x, ids, c, cb)
+    got_codes = B.ivf_pq_encode(_t(x), _t(ids), _t(c), _t(cb))
+    B.ivf_check()
+    assert (got_codes.cpu().numpy() == want_codes).all()
+    _check_search(q, c, cb, offsets, want_codes, probes, n_rerank)
