@@ -235,9 +235,10 @@ int ivf_debug_timing_read(double ms[9], int64_t launches[9]);
  *     r_t = float(x_t) - c_t;   LUT_m[j]: acc = 0, for t ascending: diff = r_t - p_m[j][t],
  *     acc = fma(diff, diff, acc);   estimate: acc = 0, for m ascending: acc = acc + LUT_m[a_m].
  *
- * codebooks  [pq_m][256][d / pq_m] float32, row-major.  pq_m must divide d, and
- *            1024 * (d + pq_m) + 4 * d + 29,776 bytes of shared memory must fit one SM's 227 KB
- *            (d = 128 with pq_m = 32 does; d = 256 does not) -> IVF_ERR_UNSUPPORTED otherwise.
+ * codebooks  [pq_m][256][d / pq_m] float32, row-major.  pq_m must divide d.  Encoding keeps the
+ *            codebook in shared memory: 1024 * (d + pq_m) + 4 * d + 29,776 bytes must fit one SM's
+ *            227 KB (d = 128 with pq_m = 32 does; d = 256 does not); searching needs
+ *            1024 * pq_m + 4 * d + 25,680 bytes and d <= 512 -> IVF_ERR_UNSUPPORTED otherwise.
  *
  * ivf_pq_encode: out_codes[i][m] = arg-min over j of the table of x_i - centroids[ids[i]]
  *            (Eq. 3 on the residual; ties to the lower j).  An id outside [0, nlist) writes zero

@@ -98,7 +98,7 @@ void timing_end(int idx, cudaStream_t stream) {
 // ------------------------------------------------------------------ workspace
 enum WsSlot {
     WS_X16, WS_C16, WS_XN, WS_SCAL, WS_BITS, WS_PART, WS_PARTMETA, WS_FAIL, WS_FBKEYS, WS_TAU,
-    WS_UCNT, WS_UOFF, WS_UCUR, WS_UPERM, WS_IDS, WS_CHUNK0, WS_CHUNK1, WS_PQ_CHUNKS, WS_PQ_GCAND, WS_PQ_GCOUNT, WS_NUM
+    WS_UCNT, WS_UOFF, WS_UCUR, WS_UPERM, WS_IDS, WS_CHUNK0, WS_CHUNK1, WS_PQ_CHUNKS, WS_PQ_GCAND, WS_PQ_GCOUNT, WS_PQ_CBT, WS_NUM
 };
 struct Buf {
     void* p = nullptr;
@@ -947,13 +947,14 @@ int ivf_assign_update(const void* points, int64_t n, int d, ivf_dtype ptype, con
 
 // ------------------------------------------------------------------ residual-PQ candidate reduction
 namespace {
-int pq_check_shape(int d, int pq_m, const float* codebooks) {
+int pq_check_shape(int d, int pq_m, const float* codebooks, bool encode) {
     if (d < 1 || pq_m < 1 || d % pq_m != 0)
         return fail(IVF_ERR_INVALID_ARG, "d = %d, pq_m = %d: pq_m must divide d", d, pq_m);
     if (!codebooks) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
-    if (pq_smem_bytes(d, pq_m) > kSmemLimit)
-        return fail(IVF_ERR_UNSUPPORTED, "d = %d, pq_m = %d: codebook + lookup table need %zu bytes of shared memory (limit %zu)",
-                    d, pq_m, pq_smem_bytes(d, pq_m), static_cast<size_t>(kSmemLimit));
+    const size_t need = encode ? pq_smem_bytes(d, pq_m) : pq_scan_smem_bytes(d, pq_m);
+    if (need > kSmemLimit || d > kPqScanThreads)
+        return fail(IVF_ERR_UNSUPPORTED, "d = %d, pq_m = %d: %zu bytes of shared memory needed (limit %zu), d at most %d", d,
+                    pq_m, need, static_cast<size_t>(kSmemLimit), kPqScanThreads);
     return IVF_OK;
 }
 int pq_set_attrs(DeviceCtx& ctx) {
@@ -973,7 +974,7 @@ int ivf_pq_encode(const void* points, int64_t n, int d, ivf_dtype ptype, const i
     if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
     if (ptype != IVF_F32 && ptype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
     if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
-    int rc = pq_check_shape(d, pq_m, codebooks);
+    int rc = pq_check_shape(d, pq_m, codebooks, true);
     if (rc != IVF_OK) return rc;
     if (n == 0) return IVF_OK;
     if (!points || !ids || !centroids || !out_codes) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
@@ -1018,7 +1019,7 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     if (n_codes < 0 || n_codes >= (int64_t(1) << 32))
         return fail(IVF_ERR_UNSUPPORTED, "n_codes = %lld: positions must fit 32 bits", (long long)n_codes);
     if (nq >= (int64_t(1) << 24)) return fail(IVF_ERR_UNSUPPORTED, "nq = %lld: at most 2^24 - 1 queries per call", (long long)nq);
-    int rc = pq_check_shape(d, pq_m, codebooks);
+    int rc = pq_check_shape(d, pq_m, codebooks, false);
     if (rc != IVF_OK) return rc;
     if (nq == 0) return IVF_OK;
     if (!queries || !centroids || !probe_ids || !list_offsets || !out_ids || !out_est || (n_codes > 0 && !codes))
@@ -1048,7 +1049,11 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     WS(WS_PQ_CHUNKS, static_cast<size_t>(nq) * (nprobe + 1) * sizeof(int), chunk_start);
     WS(WS_PQ_GCAND, static_cast<size_t>(total_groups) * n_rerank * sizeof(uint64_t), gcand);
     WS(WS_PQ_GCOUNT, static_cast<size_t>(total_groups) * sizeof(int), gcount);
+    float* cbt;
+    WS(WS_PQ_CBT, static_cast<size_t>(d) * kPqK * sizeof(float), cbt);
     int tk = timing_begin(TK_PQ_SCAN, stream);
+    pq_transpose_codebooks_kernel<<<(d * kPqK + 255) / 256, 256, 0, stream>>>(codebooks, d, d / pq_m, cbt);
+    LAUNCH_CHECK();
     pq_setup_query_kernel<<<static_cast<unsigned>(nq), 128, 0, stream>>>(
         probe_ids, nprobe, nlist, reinterpret_cast<const long long*>(list_offsets), chunk_start,
         reinterpret_cast<long long*>(out_counts), ctx.status);
@@ -1064,7 +1069,7 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     sp.n_rerank = n_rerank;
     sp.ngroups = ngroups;
     sp.centroids = centroids;
-    sp.codebooks = codebooks;
+    sp.cbt = cbt;
     sp.probes = probe_ids;
     sp.offsets = reinterpret_cast<const long long*>(list_offsets);
     sp.codes = codes;
@@ -1072,8 +1077,9 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     sp.gcand = gcand;
     sp.gcand_count = gcount;
     sp.status = ctx.status;
-    const unsigned grid = static_cast<unsigned>(total_groups < ctx.num_sms ? total_groups : ctx.num_sms);
-    pq_scan_kernel<<<grid, kPqThreads, pq_smem_bytes(d, pq_m), stream>>>(sp);
+    const int64_t resident = 2 * static_cast<int64_t>(ctx.num_sms);
+    const unsigned grid = static_cast<unsigned>(total_groups < resident ? total_groups : resident);
+    pq_scan_kernel<<<grid, kPqScanThreads, pq_scan_smem_bytes(d, pq_m), stream>>>(sp);
     LAUNCH_CHECK();
     timing_end(tk, stream);
     tk = timing_begin(TK_PQ_MERGE, stream);

@@ -25,9 +25,11 @@
 namespace ivf {
 
 constexpr int kPqK = 256;          // codewords per subspace (one byte per sub-code)
-constexpr int kPqThreads = 1024;
-constexpr int kPqChunk = 1024;     // codes per chunk = one code per thread
-constexpr int kPqBufKeys = 2048;   // candidate buffer of a group
+constexpr int kPqThreads = 1024;       // encode and query-merge kernels
+constexpr int kPqScanThreads = 512;    // scan kernel: two CTAs per SM, so one scores while the other builds a table
+constexpr int kPqChunk = kPqScanThreads;  // codes per chunk = one code per thread
+constexpr int kPqBufKeys = 2048;       // candidate buffer of the query merge
+constexpr int kPqScanBufKeys = 1536;   // candidate buffer of a group: a chunk on top of kPqMaxRerank
 constexpr int kPqMaxRerank = 1024;
 constexpr int kPqMaxProbes = 512;   // lists per query (the paper sweeps the probe count up to 512)
 constexpr int kPqStatusBadId = -6;
@@ -36,6 +38,11 @@ __host__ __device__ inline size_t pq_smem_bytes(int d, int pq_m) {
     return static_cast<size_t>(d) * kPqK * 4 + static_cast<size_t>(pq_m) * kPqK * 4 + static_cast<size_t>(d) * 4 +
            static_cast<size_t>(kPqBufKeys) * 8 + 256 * 4 + 64 +
            static_cast<size_t>(kPqMaxProbes) * 24 + 16;  // probe descriptors
+}
+
+__host__ __device__ inline size_t pq_scan_smem_bytes(int d, int pq_m) {
+    return static_cast<size_t>(pq_m) * kPqK * 4 + static_cast<size_t>(d) * 4 + static_cast<size_t>(kPqScanBufKeys) * 8 +
+           256 * 4 + 64 + static_cast<size_t>(512) * 24 + 16;
 }
 
 struct PqSmem {
@@ -51,16 +58,18 @@ struct PqSmem {
     int* cs;                // [kPqMaxProbes + 1] chunk prefix of the query
 };
 
-__device__ __forceinline__ PqSmem pq_carve(uint8_t* raw, int d, int pq_m) {
+// with_codebook: the encode kernel keeps the codebook in shared memory; the scan kernel reads its
+// transposed copy through L1 and carves none.
+__device__ __forceinline__ PqSmem pq_carve(uint8_t* raw, int d, int pq_m, bool with_codebook, int buf_keys) {
     PqSmem s;
     s.buf = reinterpret_cast<uint64_t*>(raw);
-    raw += static_cast<size_t>(kPqBufKeys) * 8;
+    raw += static_cast<size_t>(buf_keys) * 8;
     s.list_begin = reinterpret_cast<long long*>(raw);
     raw += static_cast<size_t>(kPqMaxProbes) * 8;
     s.list_len = reinterpret_cast<long long*>(raw);
     raw += static_cast<size_t>(kPqMaxProbes) * 8;
     s.cbt = reinterpret_cast<float*>(raw);
-    raw += static_cast<size_t>(d) * kPqK * 4;
+    if (with_codebook) raw += static_cast<size_t>(d) * kPqK * 4;
     s.lut = reinterpret_cast<float*>(raw);
     raw += static_cast<size_t>(pq_m) * kPqK * 4;
     s.r = reinterpret_cast<float*>(raw);
@@ -87,43 +96,78 @@ __device__ __forceinline__ void pq_load_codebooks(const float* __restrict__ code
     }
 }
 
-// lut[m * 256 + j] for the residual in s.r.  Thread -> codeword j = tid & 255; the 256-thread
-// halves of the CTA take alternate subspaces.
-__device__ __forceinline__ void pq_build_lut(const PqSmem& s, int pq_m, int dsub) {
+// Lookup-table build.  Thread -> codeword j = tid & 255; the 256-thread slices of the CTA take
+// alternate subspaces.
+template <bool kGlobal>
+__device__ __forceinline__ float pq_cb(const float* p) {
+    if constexpr (kGlobal) return __ldg(p);
+    else return *p;
+}
+
+// One sub-vector width: all strides are compile-time constants, so every load takes an immediate
+// offset from three running pointers; four subspaces per trip give four independent chains.
+template <bool kGlobal, int DSUB>
+__device__ __forceinline__ void pq_build_lut_fixed(const float* __restrict__ r, const float* __restrict__ cbt,
+                                                   float* __restrict__ lut, int pq_m) {
     const int j = threadIdx.x & (kPqK - 1);
+    const int first = threadIdx.x >> 8;
     const int step = blockDim.x >> 8;
-    if ((dsub & 3) == 0) {
-        // the residual's sub-vector comes in with 16-byte broadcast loads; same operation order
-        for (int m = threadIdx.x >> 8; m < pq_m; m += step) {
-            const float* col = s.cbt + static_cast<size_t>(m) * dsub * kPqK + j;
-            const float4* r4 = reinterpret_cast<const float4*>(s.r + m * dsub);
-            float acc = 0.0f;
-            for (int t4 = 0; t4 < (dsub >> 2); ++t4) {
-                const float4 rv = r4[t4];
-                const float c0 = col[(4 * t4 + 0) * kPqK], c1 = col[(4 * t4 + 1) * kPqK];
-                const float c2 = col[(4 * t4 + 2) * kPqK], c3 = col[(4 * t4 + 3) * kPqK];
-                float diff = __fsub_rn(rv.x, c0);
-                acc = __fmaf_rn(diff, diff, acc);
-                diff = __fsub_rn(rv.y, c1);
-                acc = __fmaf_rn(diff, diff, acc);
-                diff = __fsub_rn(rv.z, c2);
-                acc = __fmaf_rn(diff, diff, acc);
-                diff = __fsub_rn(rv.w, c3);
-                acc = __fmaf_rn(diff, diff, acc);
+    const float* col = cbt + first * (DSUB * kPqK) + j;
+    const float* rp = r + first * DSUB;
+    float* out = lut + first * kPqK + j;
+    const int col_step = step * DSUB * kPqK, r_step = step * DSUB, out_step = step * kPqK;
+#pragma unroll 4
+    for (int m = first; m < pq_m; m += step) {
+        float rv[DSUB];
+        if constexpr ((DSUB & 3) == 0) {
+#pragma unroll
+            for (int t4 = 0; t4 < DSUB / 4; ++t4) {
+                const float4 v = reinterpret_cast<const float4*>(rp)[t4];
+                rv[4 * t4] = v.x; rv[4 * t4 + 1] = v.y; rv[4 * t4 + 2] = v.z; rv[4 * t4 + 3] = v.w;
             }
-            s.lut[m * kPqK + j] = acc;
+        } else {
+#pragma unroll
+            for (int t = 0; t < DSUB; ++t) rv[t] = rp[t];
         }
-        return;
-    }
-    for (int m = threadIdx.x >> 8; m < pq_m; m += step) {
-        const float* col = s.cbt + static_cast<size_t>(m) * dsub * kPqK + j;
-        const float* r = s.r + m * dsub;
+        float cv[DSUB];
+#pragma unroll
+        for (int t = 0; t < DSUB; ++t) cv[t] = pq_cb<kGlobal>(col + t * kPqK);
         float acc = 0.0f;
-        for (int t = 0; t < dsub; ++t) {
-            const float diff = __fsub_rn(r[t], col[t * kPqK]);
+#pragma unroll
+        for (int t = 0; t < DSUB; ++t) {
+            const float diff = __fsub_rn(rv[t], cv[t]);
             acc = __fmaf_rn(diff, diff, acc);
         }
-        s.lut[m * kPqK + j] = acc;
+        *out = acc;
+        col += col_step;
+        rp += r_step;
+        out += out_step;
+    }
+}
+
+// lut[m * 256 + j] for the residual r.  kGlobal: cbt points to the transposed codebook in global
+// memory (read through L1); otherwise to the copy in shared memory.
+template <bool kGlobal>
+__device__ __forceinline__ void pq_build_lut(const float* r, const float* cbt, float* lut, int pq_m, int dsub) {
+    switch (dsub) {
+        case 2: return pq_build_lut_fixed<kGlobal, 2>(r, cbt, lut, pq_m);
+        case 3: return pq_build_lut_fixed<kGlobal, 3>(r, cbt, lut, pq_m);
+        case 4: return pq_build_lut_fixed<kGlobal, 4>(r, cbt, lut, pq_m);
+        case 6: return pq_build_lut_fixed<kGlobal, 6>(r, cbt, lut, pq_m);
+        case 8: return pq_build_lut_fixed<kGlobal, 8>(r, cbt, lut, pq_m);
+        default: break;
+    }
+    const int j = threadIdx.x & (kPqK - 1);
+    const int step = blockDim.x >> 8;
+    for (int m = threadIdx.x >> 8; m < pq_m; m += step) {
+        const float* col = cbt + static_cast<size_t>(m) * dsub * kPqK + j;
+        const float* rm = r + m * dsub;
+        float acc = 0.0f;
+        for (int t = 0; t < dsub; ++t) {
+            const float diff = __fsub_rn(rm[t], pq_cb<kGlobal>(col + t * kPqK));
+            acc = __fmaf_rn(diff, diff, acc);
+        }
+        lut[m * kPqK + j] = acc;
     }
 }
 
@@ -147,7 +191,7 @@ struct PqEncodeParams {
 
 __global__ void __launch_bounds__(kPqThreads, 1) pq_encode_kernel(const PqEncodeParams p) {
     extern __shared__ __align__(16) uint8_t pq_smem_raw[];
-    const PqSmem s = pq_carve(pq_smem_raw, p.d, p.pq_m);
+    const PqSmem s = pq_carve(pq_smem_raw, p.d, p.pq_m, true, kPqBufKeys);
     const int dsub = p.d / p.pq_m;
     pq_load_codebooks(p.codebooks, p.d, dsub, s.cbt);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
@@ -166,7 +210,7 @@ __global__ void __launch_bounds__(kPqThreads, 1) pq_encode_kernel(const PqEncode
             s.r[t] = __fsub_rn(xv, p.centroids[static_cast<int64_t>(l) * p.d + t]);
         }
         __syncthreads();
-        pq_build_lut(s, p.pq_m, dsub);
+        pq_build_lut<false>(s.r, s.cbt, s.lut, p.pq_m, dsub);
         __syncthreads();
         for (int m = warp; m < p.pq_m; m += nwarps) {
             const float* row = s.lut + m * kPqK;
@@ -192,6 +236,16 @@ __global__ void __launch_bounds__(kPqThreads, 1) pq_encode_kernel(const PqEncode
             if (lane == 0) p.codes[i * p.pq_m + m] = static_cast<uint8_t>(bj);
         }
     }
+}
+
+// codebooks [pq_m][256][dsub] -> out[(m * dsub + t) * 256 + j] (coordinate-major), for the scan kernel
+__global__ void pq_transpose_codebooks_kernel(const float* __restrict__ codebooks, int d, int dsub, float* __restrict__ out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;  // index in the output
+    if (i >= d * kPqK) return;
+    const int j = i & (kPqK - 1);
+    const int mt = i >> 8;  // m * dsub + t
+    const int m = mt / dsub, t = mt - m * dsub;
+    out[i] = codebooks[(static_cast<size_t>(m) * kPqK + j) * dsub + t];
 }
 
 // ------------------------------------------------------------------ task set-up (prefix scans on the device)
@@ -302,13 +356,15 @@ __device__ __forceinline__ uint64_t pq_select_bound(Get get, int count, int k, i
 
 // Cuts the buffer back to its k smallest keys (in no particular order); returns the bound, i.e.
 // the largest key kept.  count > k on entry; on exit misc[0] == k.
+template <int NT, int CAP>
 __device__ __forceinline__ uint64_t pq_cut_buffer(uint64_t* buf, int count, int k, int* hist, int* misc) {
     const uint64_t bound = pq_select_bound([buf](int i) { return buf[i]; }, count, k, hist, misc);
-    constexpr int kPer = kPqBufKeys / kPqThreads;
+    constexpr int kPer = CAP / NT;
+    static_assert(CAP % NT == 0, "buffer capacity must be a multiple of the thread count");
     uint64_t mine[kPer];
 #pragma unroll
     for (int q = 0; q < kPer; ++q) {
-        const int i = threadIdx.x + q * kPqThreads;
+        const int i = threadIdx.x + q * NT;
         mine[q] = i < count ? buf[i] : ~0ull;
     }
     if (threadIdx.x == 0) misc[0] = 0;
@@ -328,7 +384,7 @@ struct PqScanParams {
     int d, pq_m, nlist, nprobe, n_rerank;
     int ngroups;             // groups per query
     const float* centroids;
-    const float* codebooks;
+    const float* cbt;        // transposed codebook [d][256] in global memory
     const int32_t* probes;
     const long long* offsets;
     const uint8_t* codes;
@@ -345,23 +401,46 @@ struct PqCodeRegs {
     uint4 w[2];
 };
 __device__ __forceinline__ bool pq_codes_in_regs(int pq_m) { return pq_m == 16 || pq_m == 32; }
-__device__ __forceinline__ void pq_fetch_code(PqCodeRegs& c, const uint8_t* code, int pq_m) {
-    c.w[0] = __ldg(reinterpret_cast<const uint4*>(code));
-    if (pq_m == 32) c.w[1] = __ldg(reinterpret_cast<const uint4*>(code + 16));
+// streamed once: read-only path, not kept in L1 (which holds the codebook)
+__device__ __forceinline__ uint4 pq_ld_stream(const uint8_t* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
 }
-__device__ __forceinline__ float pq_adc_regs(const float* lut, const PqCodeRegs& c, int pq_m) {
+__device__ __forceinline__ void pq_fetch_code(PqCodeRegs& c, const uint8_t* code, int pq_m) {
+    c.w[0] = pq_ld_stream(code);
+    if (pq_m == 32) c.w[1] = pq_ld_stream(code + 16);
+}
+// ADC estimate from code bytes held in registers.  Every table entry is fetched with a
+// shared-space load whose row offset is an immediate: per sub-code one shift, one mask, one load,
+// one add.  lut_s = shared-space address of the table.
+#define PQ_ADC_STEP(WORD, Q, M)                                                                          \
+    {                                                                                                    \
+        const uint32_t scaled = ((Q) == 0 ? ((WORD) << 2) : ((WORD) >> (8 * (Q) - 2))) & 0x3FCu;       \
+        float v;                                                                                         \
+        asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(lut_s + scaled), "n"((M) * kPqK * 4)); \
+        acc = __fadd_rn(acc, v);                                                                         \
+    }
+#define PQ_ADC_WORD(WORD, M0) \
+    PQ_ADC_STEP(WORD, 0, (M0)) PQ_ADC_STEP(WORD, 1, (M0) + 1) PQ_ADC_STEP(WORD, 2, (M0) + 2) PQ_ADC_STEP(WORD, 3, (M0) + 3)
+__device__ __forceinline__ float pq_adc_regs(uint32_t lut_s, const PqCodeRegs& c, int pq_m) {
     float acc = 0.0f;
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        if (h * 16 < pq_m) {
-            const uint32_t w[4] = {c.w[h].x, c.w[h].y, c.w[h].z, c.w[h].w};
-#pragma unroll
-            for (int q = 0; q < 16; ++q)
-                acc = __fadd_rn(acc, lut[(h * 16 + q) * kPqK + ((w[q >> 2] >> (8 * (q & 3))) & 255u)]);
-        }
+    PQ_ADC_WORD(c.w[0].x, 0)
+    PQ_ADC_WORD(c.w[0].y, 4)
+    PQ_ADC_WORD(c.w[0].z, 8)
+    PQ_ADC_WORD(c.w[0].w, 12)
+    if (pq_m == 32) {
+        PQ_ADC_WORD(c.w[1].x, 16)
+        PQ_ADC_WORD(c.w[1].y, 20)
+        PQ_ADC_WORD(c.w[1].z, 24)
+        PQ_ADC_WORD(c.w[1].w, 28)
     }
     return acc;
 }
+#undef PQ_ADC_WORD
+#undef PQ_ADC_STEP
 
 __device__ __forceinline__ float pq_adc_code(const float* lut, const uint8_t* code, int pq_m) {
     float acc = 0.0f;
@@ -385,16 +464,16 @@ __device__ __forceinline__ float pq_adc_code(const float* lut, const uint8_t* co
     return acc;
 }
 
-__global__ void __launch_bounds__(kPqThreads, 1) pq_scan_kernel(const PqScanParams p) {
+__global__ void __launch_bounds__(kPqScanThreads, 2) pq_scan_kernel(const PqScanParams p) {
     extern __shared__ __align__(16) uint8_t pq_smem_raw[];
-    const PqSmem s = pq_carve(pq_smem_raw, p.d, p.pq_m);
+    const PqSmem s = pq_carve(pq_smem_raw, p.d, p.pq_m, false, kPqScanBufKeys);
     const int dsub = p.d / p.pq_m;
     const int64_t total_groups = p.nq * p.ngroups;
     if (static_cast<int64_t>(blockIdx.x) >= total_groups) return;
-    pq_load_codebooks(p.codebooks, p.d, dsub, s.cbt);
     const int lane = threadIdx.x & 31;
     const uint32_t lt_mask = (1u << lane) - 1u;
     const bool in_regs = pq_codes_in_regs(p.pq_m);
+    const uint32_t lut_s = static_cast<uint32_t>(__cvta_generic_to_shared(s.lut));
 
     for (int64_t g = blockIdx.x; g < total_groups; g += gridDim.x) {
         const int64_t b = g / p.ngroups;
@@ -461,7 +540,7 @@ __global__ void __launch_bounds__(kPqThreads, 1) pq_scan_kernel(const PqScanPara
                     if (later < p.nprobe && s.cs[later] < chunk1 && threadIdx.x < p.d)
                         cnext = p.centroids[static_cast<int64_t>(s.list_id[later]) * p.d + threadIdx.x];
                     __syncthreads();
-                    pq_build_lut(s, p.pq_m, dsub);
+                    pq_build_lut<true>(s.r, p.cbt, s.lut, p.pq_m, dsub);
                     __syncthreads();
                     built = pr;
                 }
@@ -478,7 +557,7 @@ __global__ void __launch_bounds__(kPqThreads, 1) pq_scan_kernel(const PqScanPara
                 bool hit = false;
                 uint64_t key = 0;
                 if (pos >= 0) {
-                    const float est = in_regs ? pq_adc_regs(s.lut, cur, p.pq_m)
+                    const float est = in_regs ? pq_adc_regs(lut_s, cur, p.pq_m)
                                               : pq_adc_code(s.lut, p.codes + pos * p.pq_m, p.pq_m);
                     key = (static_cast<uint64_t>(orderable(est)) << 32) | static_cast<uint32_t>(pos);
                     hit = key < bound;
@@ -492,13 +571,14 @@ __global__ void __launch_bounds__(kPqThreads, 1) pq_scan_kernel(const PqScanPara
                 }
                 __syncthreads();
                 const int count = s.misc[0];
-                if (count > kPqBufKeys - kPqChunk) bound = pq_cut_buffer(s.buf, count, p.n_rerank, s.hist, s.misc);
+                if (count > kPqScanBufKeys - kPqChunk)
+                    bound = pq_cut_buffer<kPqScanThreads, kPqScanBufKeys>(s.buf, count, p.n_rerank, s.hist, s.misc);
             }
         }
         __syncthreads();
         int count = s.misc[0];
         if (count > p.n_rerank) {
-            pq_cut_buffer(s.buf, count, p.n_rerank, s.hist, s.misc);
+            pq_cut_buffer<kPqScanThreads, kPqScanBufKeys>(s.buf, count, p.n_rerank, s.hist, s.misc);
             count = p.n_rerank;
         }
         uint64_t* out = p.gcand + static_cast<size_t>(g) * p.n_rerank;
@@ -553,7 +633,7 @@ __global__ void __launch_bounds__(kPqThreads) pq_merge_kernel(const PqMergeParam
     int count = misc[0];
     if (count > p.n_rerank) {
         __syncthreads();
-        pq_cut_buffer(buf, count, p.n_rerank, hist, misc);
+        pq_cut_buffer<kPqThreads, kPqBufKeys>(buf, count, p.n_rerank, hist, misc);
         count = p.n_rerank;
     }
     int m = 2;
