@@ -354,6 +354,47 @@ __device__ __forceinline__ uint64_t pq_select_bound(Get get, int count, int k, i
     return prefix;
 }
 
+// The same selection over keys that every thread holds in registers (PER per thread; all-ones =
+// padding), so that the passes touch no memory but the histogram.
+template <int PER>
+__device__ __forceinline__ uint64_t pq_select_bound_regs(const uint64_t (&mine)[PER], int k, int* hist, int* misc) {
+    const int lane = threadIdx.x & 31;
+    uint64_t prefix = 0, mask = 0;
+    int rank = k;
+    for (int shift = 56; shift >= 0; shift -= 8) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < PER; ++q) {
+            const uint64_t v = mine[q];
+            uint32_t dg = 0xFFFFFFFFu;
+            if (v != ~0ull && (v & mask) == prefix) dg = static_cast<uint32_t>(v >> shift) & 255u;
+            if (__any_sync(0xFFFFFFFFu, dg != 0xFFFFFFFFu)) {
+                const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dg);
+                if (dg != 0xFFFFFFFFu && lane == __ffs(peers) - 1) atomicAdd(&hist[dg], __popc(peers));
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            int r = rank, eq = 0;
+            const int digit = radix_pick_digit(hist, lane, r, eq);
+            if (lane == 0) {
+                misc[1] = digit;
+                misc[2] = r;
+                misc[3] = eq;
+            }
+        }
+        __syncthreads();
+        prefix |= static_cast<uint64_t>(misc[1]) << shift;
+        mask |= 255ull << shift;
+        rank = misc[2];
+        const bool whole = misc[3] == rank;
+        __syncthreads();
+        if (whole) return prefix | ~mask;
+    }
+    return prefix;
+}
+
 // Cuts the buffer back to its k smallest keys (in no particular order); returns the bound, i.e.
 // the largest key kept.  count > k on entry; on exit misc[0] == k.
 template <int NT, int CAP>
@@ -621,13 +662,37 @@ __global__ void __launch_bounds__(kPqThreads) pq_merge_kernel(const PqMergeParam
     if (mine) atomicAdd(&misc[4], mine);
     __syncthreads();
     const int total = misc[4];
-    uint64_t bound = ~0ull;
-    if (total > kPqBufKeys) bound = pq_select_bound(get, slots, p.n_rerank, hist, misc);
     if (threadIdx.x == 0) misc[0] = 0;
     __syncthreads();
-    for (int i = threadIdx.x; i < slots; i += blockDim.x) {
-        const uint64_t v = get(i);
-        if (v != ~0ull && v <= bound) buf[atomicAdd(&misc[0], 1)] = v;
+    constexpr int kRegKeys = 16;
+    if (slots <= kRegKeys * kPqThreads) {
+        // every slot is read once into registers; selection and gathering work from there
+        uint64_t mine[kRegKeys];
+#pragma unroll
+        for (int q = 0; q < kRegKeys; ++q) {
+            const int i = threadIdx.x + q * kPqThreads;
+            mine[q] = i < slots ? get(i) : ~0ull;
+        }
+        uint64_t bound = ~0ull;
+        if (total > kPqBufKeys) {
+            bound = pq_select_bound_regs<kRegKeys>(mine, p.n_rerank, hist, misc);
+            if (threadIdx.x == 0) misc[0] = 0;
+            __syncthreads();
+        }
+#pragma unroll
+        for (int q = 0; q < kRegKeys; ++q)
+            if (mine[q] != ~0ull && mine[q] <= bound) buf[atomicAdd(&misc[0], 1)] = mine[q];
+    } else {
+        uint64_t bound = ~0ull;
+        if (total > kPqBufKeys) {
+            bound = pq_select_bound(get, slots, p.n_rerank, hist, misc);
+            if (threadIdx.x == 0) misc[0] = 0;
+            __syncthreads();
+        }
+        for (int i = threadIdx.x; i < slots; i += blockDim.x) {
+            const uint64_t v = get(i);
+            if (v != ~0ull && v <= bound) buf[atomicAdd(&misc[0], 1)] = v;
+        }
     }
     __syncthreads();
     int count = misc[0];
