@@ -153,6 +153,68 @@ def run_reference(args, rank: int, world: int):
     print(json.dumps(line), flush=True)
 
 
+def pq_side_measurement(dev, pk, sm_max_mhz):
+    """Residual-PQ candidate reduction (the step after routing in the PQ variant), outside the
+    headline: a 2,097,152-vector SIFT-shaped index with 2,048 lists is assigned, regrouped and
+    encoded with the library's own calls, then a 2,048-query batch (64 probes, N_rerank 512, 32
+    sub-codes) is routed and reduced.  The scan is bound by shared-memory table lookups: the
+    ceiling quoted is one lookup per bank and clock on every SM."""
+    import torch
+    from paper_2608_08751_b200 import binding as B
+    from paper_2608_08751_b200 import synth
+    n, nlist, pq_m, nq, nprobe, n_rerank, reps = 2 * synth.CHUNK_ROWS, 2048, 32, 2048, 64, 512, 10
+    cent = torch.from_numpy(synth.sift_like_centroids(nlist, D)).to(dev)
+    cb = torch.from_numpy(synth.pq_codebooks(pq_m, D // pq_m, 20.0, seed=1)).to(dev)
+    x = torch.cat([torch.from_numpy(synth.sift_like_rows(c, rows=synth.CHUNK_ROWS, d=D)).to(dev) for c in range(2)])
+    ids, _ = B.ivf_assign(x, cent)
+    xr, offsets, order = B.ivf_cluster_major_reorder(x, ids, nlist)
+    ids_sorted = ids[order.long()]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    B.ivf_pq_encode(xr[:4096], ids_sorted[:4096], cent, cb)
+    e0.record()
+    codes = B.ivf_pq_encode(xr, ids_sorted, cent, cb)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    enc_ms = e0.elapsed_time(e1)
+    q = torch.from_numpy(synth.sift_like_queries(nq, D)).to(dev)
+    handle = B.PreparedCentroids(cent)
+    probes = torch.empty((nq, nprobe), dtype=torch.int32, device=dev)
+    for _ in range(3):
+        B.ivf_route_prepared(handle, q, nprobe, probes, None, want_dists=False)
+        pos, est, cnt = B.ivf_pq_search(q, cent, probes, offsets, codes, cb, n_rerank)
+    l0 = B.ivf_launch_count()
+    e0.record()
+    for _ in range(reps):
+        B.ivf_route_prepared(handle, q, nprobe, probes, None, want_dists=False)
+        B.ivf_pq_search(q, cent, probes, offsets, codes, cb, n_rerank)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    both_ms = e0.elapsed_time(e1) / reps
+    launches = (B.ivf_launch_count() - l0) // reps
+    B.ivf_debug_timing(True)
+    for _ in range(reps):
+        B.ivf_pq_search(q, cent, probes, offsets, codes, cb, n_rerank)
+    fam = B.ivf_debug_timing_read()
+    B.ivf_debug_timing(False)
+    B.ivf_check(dev)
+    handle.close()
+    scan_ms = fam["pq_scan"][0] / max(fam["pq_scan"][1], 1)
+    merge_ms = fam["pq_merge"][0] / max(fam["pq_merge"][1], 1)
+    scanned = int(cnt.sum().item())
+    lookups = scanned * pq_m / (scan_ms / 1e3)
+    peak = 148 * 32 * sm_max_mhz * 1e6  # one 4-byte lookup per bank and clock on every SM
+    return {
+        "workload": f"{n} uint8 vectors x {D}, {nlist} lists, {pq_m} sub-codes; batch {nq}, {nprobe} probes, N_rerank {n_rerank}",
+        "encode_vectors_per_s": n / (enc_ms / 1e3), "route_plus_reduce_ms": both_ms,
+        "queries_per_s": nq / (both_ms / 1e3), "scan_ms": scan_ms, "merge_ms": merge_ms,
+        "codes_scanned_per_batch": scanned, "codes_per_s": scanned / (scan_ms / 1e3),
+        "code_bytes_GBps": scanned * pq_m / (scan_ms / 1e3) / 1e9, "launches_per_batch": int(launches),
+        "roofline": {"kernel": "pq_scan_kernel", "bound": "alu", "achieved": lookups / 1e12, "peak": peak / 1e12,
+                     "unit": "T lookups/s", "frac": lookups / peak, "traffic": None,
+                     "peak_source": "derived: 148 SMs x 32 shared-memory banks x max SM clock"},
+    }
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -160,6 +222,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-pq", action="store_true", help="skip the residual-PQ candidate-reduction side measurement")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else max(args.warmup, 0)
 
@@ -359,6 +422,9 @@ def main():
                    "samples": clocks["samples"]},
         "wall_s_timed_region": t_wall,
     }
+
+    if not args.no_pq and world == 1:
+        line["pq"] = pq_side_measurement(dev, pk, clocks["sm_max_mhz"])
 
     if not args.no_cpu_baseline and world == 1:
         from oracle import oracle
