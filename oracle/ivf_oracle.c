@@ -25,7 +25,9 @@
  * Pins (tests/test_oracle_pins.py): hand-computed tiny cases, one-hot closed form,
  * unit-norm identity, scipy cdist, brute force over all k-subsets, lexsort,
  * permutation / translation / scaling invariants, bincount cross-check, Lloyd
- * monotonicity and toy clusters, numpy stable argsort for the reorder.  No function here is unpinned.
+ * monotonicity and toy clusters, numpy stable argsort for the reorder; the candidate-restricted
+ * assignment against the full assignment, numpy arg-min over the gathered rows and a hand case.
+ * No function here is unpinned.
  */
 #include <math.h>
 #include <stdint.h>
@@ -220,4 +222,37 @@ int oracle_lloyd(const void *x, int xtype, int64_t n, int d, int32_t nlist, int 
     }
     free(dist); free(sums); free(counts);
     return rc;
+}
+
+/*
+ * Assignment within given candidates (Appendix "Fast index building": a graph search proposes a
+ * small candidate-centroid set per vector -- 8 in the fast mode, 2 in the ultra-fast one, Table 3 --
+ * and the exact distance is evaluated within that set only).  The candidate generator is not part
+ * of this path; candidates are an input.
+ *   cand [n*m] int32: m candidate centroid ids per row (repeats allowed; every id must be in range)
+ *   out_ids [n], out_dists [n]: the candidate with the smallest squared L2 distance, ties to the
+ *   lower centroid id.
+ * Returns -1 on bad arguments or an id out of range.
+ */
+int oracle_assign_candidates(const void *x, int xtype, int64_t n, int d, const float *c, int32_t nlist,
+                             const int32_t *cand, int m, int32_t *out_ids, double *out_dists) {
+    if (n < 0 || d <= 0 || nlist <= 0 || m <= 0) return -1;
+    for (int64_t i = 0; i < n * m; ++i)
+        if (cand[i] < 0 || cand[i] >= nlist) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i) {
+        double best = INFINITY;
+        int32_t best_id = -1;
+        for (int p = 0; p < m; ++p) {
+            const int32_t j = cand[i * m + p];
+            const double dist = sqdist(x, xtype, i, c, j, d);
+            if (dist < best || (dist == best && j < best_id)) {
+                best = dist;
+                best_id = j;
+            }
+        }
+        out_ids[i] = best_id;
+        out_dists[i] = best;
+    }
+    return 0;
 }

@@ -46,6 +46,7 @@ def _load():
         _lib.oracle_reorder.argtypes = [vp, i64, i32, vp, vp]
         _lib.oracle_lloyd.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, i32, ctypes.c_int, vp, vp, vp]
         _lib.oracle_num_threads.restype = ctypes.c_int
+        _lib.oracle_assign_candidates.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, vp, i32, vp, ctypes.c_int, vp, vp]
         _lib.oracle_pq_lut.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, vp]
         _lib.oracle_pq_lut.restype = None
         _lib.oracle_pq_adc.argtypes = [vp, ctypes.c_int, vp, i64, i64, vp]
@@ -106,6 +107,21 @@ def assign(x: np.ndarray, c: np.ndarray):
     rc = _load().oracle_assign(_p(x), xt, n, d, _p(c), c.shape[0], _p(ids), _p(dists))
     if rc != 0:
         raise ValueError("oracle_assign: bad arguments")
+    return ids, dists
+
+
+def assign_candidates(x: np.ndarray, c: np.ndarray, cand: np.ndarray):
+    """(ids [n] int32, dists [n] float64): the nearest centroid among each row's candidates cand [n, m]."""
+    x, xt = _rows(x)
+    c = _cent(c)
+    cand = np.ascontiguousarray(cand, np.int32)
+    n, d = x.shape
+    assert cand.shape[0] == n
+    ids = np.empty((n,), np.int32)
+    dists = np.empty((n,), np.float64)
+    rc = _load().oracle_assign_candidates(_p(x), xt, n, d, _p(c), c.shape[0], _p(cand), cand.shape[1], _p(ids), _p(dists))
+    if rc != 0:
+        raise ValueError("oracle_assign_candidates: bad arguments")
     return ids, dists
 
 

@@ -255,3 +255,43 @@ def test_reorder_hand_case_and_stable_argsort():
     assert (np.diff(offsets) == np.bincount(ids, minlength=37)).all() and offsets[-1] == 5000
     with pytest.raises(ValueError):
         oracle.reorder(np.array([0, 5], np.int32), 5)
+
+
+# ---------------------------------------------------------------- assignment within given candidates
+def test_candidate_assignment_hand_case_and_ties():
+    # points on a line; candidates given explicitly.  x = 5: candidates {0 at 0, 2 at 9, 3 at 1} ->
+    # distances 25, 16, 16: tie between ids 2 and 3 -> id 2.  x = 0 with candidates {3, 3}: id 3, 1.
+    c = np.array([[0.0], [100.0], [9.0], [1.0]], np.float32)
+    x = np.array([[5.0], [0.0]], np.float32)
+    cand = np.array([[0, 2, 3], [3, 3, 3]], np.int32)
+    ids, d = oracle.assign_candidates(x, c, cand)
+    assert ids.tolist() == [2, 3] and d.tolist() == [16.0, 1.0]
+    # order of the candidates does not matter, nor do repeats
+    ids2, d2 = oracle.assign_candidates(x, c, np.array([[3, 0, 2], [3, 3, 3]], np.int32))
+    assert ids2.tolist() == [2, 3] and d2.tolist() == [16.0, 1.0]
+
+
+def test_candidate_assignment_against_numpy_and_full_assignment():
+    rng = np.random.default_rng(21)
+    n, nlist, d, m = 400, 300, 24, 8
+    x = rng.integers(0, 256, (n, d)).astype(np.uint8)
+    c = rng.normal(120, 40, (nlist, d)).astype(np.float32)
+    cand = rng.integers(0, nlist, (n, m)).astype(np.int32)
+    ids, dist = oracle.assign_candidates(x, c, cand)
+    gathered = c[cand].astype(np.float64)                         # [n, m, d]
+    ref = ((x.astype(np.float64)[:, None, :] - gathered) ** 2).sum(-1)
+    pick = np.array([min(range(m), key=lambda p: (ref[i, p], cand[i, p])) for i in range(n)])
+    assert (ids == cand[np.arange(n), pick]).all()
+    assert np.allclose(dist, ref[np.arange(n), pick], rtol=1e-12)
+    # if the true nearest centroid is among the candidates the result is the full assignment
+    full_ids, full_d = oracle.assign(x, c)
+    cand[:, 3] = full_ids
+    ids, dist = oracle.assign_candidates(x, c, cand)
+    assert (ids == full_ids).all() and (dist == full_d).all()
+    # all centroids as candidates: the same again
+    every = np.tile(np.arange(nlist, dtype=np.int32), (n, 1))
+    ids, dist = oracle.assign_candidates(x, c, every)
+    assert (ids == full_ids).all() and (dist == full_d).all()
+    bad = cand.copy(); bad[0, 0] = nlist
+    with pytest.raises(ValueError):
+        oracle.assign_candidates(x, c, bad)
