@@ -226,6 +226,20 @@ int ivf_debug_timing(int enable);
 int ivf_debug_timing_read(double ms[9], int64_t launches[9]);
 
 /*
+ * Assignment within given candidates (appendix on fast index building; Table 3 lists 8 and 2
+ * candidate centroids per vector).  cand_ids [n][m] int32 (device) holds m candidate centroid ids
+ * per row, produced by whatever search the caller runs (the paper uses a graph over the centroid
+ * table, which is not part of this library); repeats are allowed.  out_ids[i] = the candidate with
+ * the smallest squared L2 distance to row i (ties to the lower id), out_dists[i] (may be NULL) that
+ * distance, computed in fp32 from the differences (no norm expansion).  All pointers are device
+ * pointers; points and centroids 16-byte aligned; d a multiple of 4, at most 256.  A candidate id
+ * outside [0, nlist) is skipped and sets the sticky status IVF_ERR_BAD_ID (a row whose candidates
+ * are all invalid gets id -1 and +inf).
+ */
+int ivf_assign_candidates(const void* points, int64_t n, int d, ivf_dtype ptype, const float* centroids, int nlist,
+                          const int32_t* cand_ids, int m, int32_t* out_ids, float* out_dists, void* stream);
+
+/*
  * Residual-PQ candidate reduction (Sec. 2.2 Eq. 3-5; Sec. 4.3; Sec. 4.4).  K = 256 codewords per
  * subspace, one byte per sub-code, fp32 lookup tables (the paper's setting).  All pointers are
  * DEVICE pointers owned by the caller; calls enqueue on `stream` and return.

@@ -23,7 +23,7 @@ EXPORTS = (
     "ivf_route", "ivf_assign", "ivf_centroid_update", "ivf_centroid_update_noalloc", "ivf_centroid_finalize",
     "ivf_assign_update", "ivf_cluster_major_reorder", "ivf_centroids_create", "ivf_centroids_destroy",
     "ivf_route_prepared",
-    "ivf_pq_encode", "ivf_pq_search",
+    "ivf_pq_encode", "ivf_pq_search", "ivf_assign_candidates",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
     "ivf_debug_plan", "ivf_debug_span", "ivf_debug_set_wait_limit_ns",
     "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_set_row_chunk", "ivf_debug_stats", "ivf_debug_set_pq_groups",
@@ -74,6 +74,7 @@ def lib() -> ctypes.CDLL:
     L.ivf_debug_set_row_chunk.argtypes = [i64]
     L.ivf_debug_stats.argtypes = [i32, ctypes.POINTER(i64)]
     L.ivf_debug_rule.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_int)]
+    L.ivf_assign_candidates.argtypes = [vp, i64, i32, i32, vp, i32, vp, i32, vp, vp, vp]
     L.ivf_pq_encode.argtypes = [vp, i64, i32, i32, vp, vp, i32, vp, i32, vp, vp]
     L.ivf_pq_search.argtypes = [vp, i64, i32, i32, vp, i32, vp, i32, vp, vp, i64, vp, i32, i32, vp, vp, vp, vp, vp]
     L.ivf_debug_set_pq_groups.argtypes = [i32]
@@ -271,6 +272,29 @@ def ivf_cluster_major_reorder(points: torch.Tensor, ids: torch.Tensor, nlist: in
     if rc != IVF_OK:
         _raise(rc)
     return out_points, out_offsets, out_order
+
+
+def ivf_assign_candidates(points: torch.Tensor, centroids: torch.Tensor, cand_ids: torch.Tensor,
+                          want_dists: bool = True):
+    """(ids int32 [n], dists float32 [n] or None): for every row the nearest centroid among its
+    candidates cand_ids [n, m] (exact squared L2 within the set)."""
+    if not points.is_cuda:
+        raise ValueError("points must be a CUDA tensor")
+    _rows(points, "points")
+    _dev(centroids, "centroids", torch.float32)
+    _dev(cand_ids, "cand_ids", torch.int32)
+    n, d = points.shape
+    if cand_ids.dim() != 2 or cand_ids.shape[0] != n:
+        raise ValueError("cand_ids must be [n, m]")
+    dev = points.device
+    out_ids = torch.empty((n,), dtype=torch.int32, device=dev)
+    out_dists = torch.empty((n,), dtype=torch.float32, device=dev) if want_dists else None
+    with torch.cuda.device(dev):
+        rc = lib().ivf_assign_candidates(_ptr(points), n, d, _dtype_code(points), _ptr(centroids), centroids.shape[0],
+                                         _ptr(cand_ids), cand_ids.shape[1], _ptr(out_ids), _ptr(out_dists), _stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
+    return out_ids, out_dists
 
 
 def _codebooks(codebooks: torch.Tensor, d: int) -> int:

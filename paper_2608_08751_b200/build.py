@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libivf_b200.so")
 _SOURCES = ["ivf_api.cu"]
-_HEADERS = ["ptx.cuh", "scales.cuh", "fused_topk.cuh", "merge.cuh", "prep.cuh", "update.cuh", "pq.cuh"]
+_HEADERS = ["ptx.cuh", "scales.cuh", "fused_topk.cuh", "merge.cuh", "prep.cuh", "update.cuh", "pq.cuh", "candidates.cuh"]
 
 
 def _nvcc() -> str:

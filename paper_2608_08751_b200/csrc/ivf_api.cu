@@ -18,6 +18,7 @@
 
 #include "fused_topk.cuh"
 #include "merge.cuh"
+#include "candidates.cuh"
 #include "pq.cuh"
 #include "prep.cuh"
 #include "update.cuh"
@@ -943,6 +944,34 @@ int ivf_assign_update(const void* points, int64_t n, int d, ivf_dtype ptype, con
     if (reinterpret_cast<uintptr_t>(sums) & 15) return fail(IVF_ERR_INVALID_ARG, "sums must be 16-byte aligned");
     return run_chunks(points, n, d, ptype, centroids, nlist, 1, out_ids, out_dists, true, sums, counts, chunk_rows,
                       static_cast<cudaStream_t>(stream));
+}
+
+int ivf_assign_candidates(const void* points, int64_t n, int d, ivf_dtype ptype, const float* centroids, int nlist,
+                          const int32_t* cand_ids, int m, int32_t* out_ids, float* out_dists, void* stream_) {
+    if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
+    if (ptype != IVF_F32 && ptype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
+    if (d < 4 || d > kCandMaxD || d % 4 != 0)
+        return fail(IVF_ERR_UNSUPPORTED, "d = %d: must be a multiple of 4 in [4, %d]", d, kCandMaxD);
+    if (nlist < 1 || m < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d, candidates per row = %d", nlist, m);
+    if (n == 0) return IVF_OK;
+    if (!points || !centroids || !cand_ids || !out_ids) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    if ((reinterpret_cast<uintptr_t>(points) & 15) || (reinterpret_cast<uintptr_t>(centroids) & 15))
+        return fail(IVF_ERR_INVALID_ARG, "points and centroids must be 16-byte aligned");
+    DeviceCtx* pctx = nullptr;
+    int rc = get_ctx(&pctx);
+    if (rc != IVF_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int tk = timing_begin(TK_FUSED_ARGMIN, stream);
+    const unsigned grid = static_cast<unsigned>((n * 32 + 255) / 256);
+    if (ptype == IVF_U8)
+        assign_candidates_kernel<uint8_t><<<grid, 256, 0, stream>>>(static_cast<const uint8_t*>(points), n, d, centroids, nlist,
+                                                                    cand_ids, m, out_ids, out_dists, pctx->status);
+    else
+        assign_candidates_kernel<float><<<grid, 256, 0, stream>>>(static_cast<const float*>(points), n, d, centroids, nlist,
+                                                                  cand_ids, m, out_ids, out_dists, pctx->status);
+    LAUNCH_CHECK();
+    timing_end(tk, stream);
+    return IVF_OK;
 }
 
 // ------------------------------------------------------------------ residual-PQ candidate reduction

@@ -174,9 +174,33 @@ def pq_case(args):
     print(json.dumps(out))
 
 
+def candidates_case(args):
+    """Assignment within --k given candidates per row (random candidates: the gather is what costs)."""
+    x = synth.sift_like_rows(0, rows=args.n, d=args.d) if args.dtype == "u8" else synth.deep_like_rows(0, args.n, args.d)
+    c = synth.sift_like_centroids(args.nlist, args.d) if args.dtype == "u8" else synth.deep_like_centroids(args.nlist, args.d)
+    xt, ct = torch.from_numpy(x).cuda(), torch.from_numpy(c).cuda()
+    cand = torch.randint(0, args.nlist, (args.n, args.k), dtype=torch.int32, device="cuda",
+                         generator=torch.Generator(device="cuda").manual_seed(1))
+    for _ in range(3):
+        B.ivf_assign_candidates(xt, ct, cand)
+    B.ivf_check()
+    reps = max(args.reps, 10)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        B.ivf_assign_candidates(xt, ct, cand)
+    e1.record()
+    B.ivf_check()
+    ms = e0.elapsed_time(e1) / reps
+    esize = 1 if args.dtype == "u8" else 4
+    nbytes = args.n * (args.d * esize + args.k * 4 + args.k * args.d * 4 + 8)
+    print(json.dumps({"op": "candidates", "n": args.n, "nlist": args.nlist, "d": args.d, "m": args.k, "dtype": args.dtype,
+                      "ms_per_call": ms, "vectors_per_s": args.n / (ms / 1e3), "algorithmic_GBps": nbytes / (ms / 1e3) / 1e9}))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="assign", choices=["assign", "route", "update", "stream", "serve", "pq"])
+    ap.add_argument("--op", default="assign", choices=["assign", "route", "update", "stream", "serve", "pq", "candidates"])
     ap.add_argument("--pq-m", type=int, default=32, dest="pq_m")
     ap.add_argument("--n-rerank", type=int, default=512, dest="n_rerank")
     ap.add_argument("--batches", default="8,32,256,2048", help="query batch sizes of --op serve")
@@ -195,6 +219,8 @@ def main():
         return serve_case(args)
     if args.op == "pq":
         return pq_case(args)
+    if args.op == "candidates":
+        return candidates_case(args)
     if args.dtype == "u8":
         x = synth.sift_like_rows(0, rows=args.n, d=args.d)
         c = synth.sift_like_centroids(args.nlist, args.d)
