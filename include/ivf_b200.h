@@ -24,7 +24,8 @@
  *   Errors     every call returns IVF_OK or a negative ivf_status.  Argument errors are detected
  *              before anything is enqueued.  Device-side problems (a bounded wait that expired, an
  *              id out of range) set a sticky per-device status word that ivf_check reads.
- *   Limits     d must be a multiple of 16, 16 <= d <= 256.  1 <= nprobe <= min(nlist, 512).
+ *   Limits     d must be a multiple of 4, 4 <= d <= 256 (d = 100 is padded to the next multiple of 16 inside the operand copies;
+ *              uint8 rows with d a multiple of 16 take the fastest path: no fp16 copy in HBM).  1 <= nprobe <= min(nlist, 512).
  *              nlist < 2^31.  n == 0 is IVF_OK and enqueues nothing.
  *   Non-finite inputs give unspecified (but memory-safe) results.
  *
@@ -40,7 +41,7 @@
 extern "C" {
 #endif
 
-typedef enum { IVF_F32 = 0, IVF_U8 = 1 } ivf_dtype;
+typedef enum { IVF_F32 = 0, IVF_U8 = 1, IVF_I8 = 2 } ivf_dtype;  /* IVF_I8: signed bytes (SPACEV-shaped data, Table 2) */
 
 typedef enum {
     IVF_OK = 0,

@@ -37,7 +37,7 @@
 #include <omp.h>
 #endif
 
-enum { ORACLE_F32 = 0, ORACLE_U8 = 1 };
+enum { ORACLE_F32 = 0, ORACLE_U8 = 1, ORACLE_I8 = 2 };
 
 typedef struct {
     double dist;
@@ -52,7 +52,9 @@ static int pair_cmp(const void *pa, const void *pb) {
 }
 
 static inline double elem(const void *x, int xtype, int64_t idx) {
-    return xtype == ORACLE_U8 ? (double)((const uint8_t *)x)[idx] : (double)((const float *)x)[idx];
+    if (xtype == ORACLE_U8) return (double)((const uint8_t *)x)[idx];
+    if (xtype == ORACLE_I8) return (double)((const int8_t *)x)[idx];
+    return (double)((const float *)x)[idx];
 }
 
 /* squared L2 distance between row i of x and row j of c, direct difference form */

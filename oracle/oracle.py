@@ -17,7 +17,7 @@ _SRC = os.path.join(_HERE, "ivf_oracle.c")
 _SRC_PQ = os.path.join(_HERE, "pq_oracle.c")
 _LIB = os.path.join(_HERE, "libivf_oracle.so")
 
-F32, U8 = 0, 1
+F32, U8, I8 = 0, 1, 2
 _lib = None
 
 
@@ -58,12 +58,14 @@ def _load():
 
 
 def _rows(x: np.ndarray):
-    """(contiguous array, dtype code) for a float32 or uint8 row matrix."""
+    """(contiguous array, dtype code) for a float32, uint8 or int8 row matrix."""
     if x.dtype == np.uint8:
         return np.ascontiguousarray(x), U8
+    if x.dtype == np.int8:
+        return np.ascontiguousarray(x), I8
     if x.dtype == np.float32:
         return np.ascontiguousarray(x), F32
-    raise TypeError(f"oracle takes float32 or uint8 rows, got {x.dtype}")
+    raise TypeError(f"oracle takes float32, uint8 or int8 rows, got {x.dtype}")
 
 
 def _cent(c: np.ndarray) -> np.ndarray:

@@ -36,11 +36,13 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { PQ_F32 = 0, PQ_U8 = 1 };
+enum { PQ_F32 = 0, PQ_U8 = 1, PQ_I8 = 2 };
 enum { PQ_K = 256 };
 
 static inline float elem_f(const void *x, int xtype, int64_t idx) {
-    return xtype == PQ_U8 ? (float)((const uint8_t *)x)[idx] : ((const float *)x)[idx];
+    if (xtype == PQ_U8) return (float)((const uint8_t *)x)[idx];
+    if (xtype == PQ_I8) return (float)((const int8_t *)x)[idx];
+    return ((const float *)x)[idx];
 }
 
 /* lut[m*256 + j] = |r^(m) - p_m[j]|^2 for a residual r of d floats; codebooks [pq_m][256][dsub] */

@@ -14,7 +14,7 @@ import torch
 
 from . import build as _build
 
-IVF_F32, IVF_U8 = 0, 1
+IVF_F32, IVF_U8, IVF_I8 = 0, 1, 2
 IVF_OK = 0
 IVF_ERR_INVALID_ARG, IVF_ERR_UNSUPPORTED, IVF_ERR_ALLOC = -1, -2, -3
 IVF_ERR_CUDA, IVF_ERR_DEVICE_TIMEOUT, IVF_ERR_BAD_ID = -4, -5, -6
@@ -95,7 +95,9 @@ def _dtype_code(t: torch.Tensor) -> int:
         return IVF_F32
     if t.dtype == torch.uint8:
         return IVF_U8
-    raise TypeError(f"points must be float32 or uint8, got {t.dtype}")
+    if t.dtype == torch.int8:
+        return IVF_I8
+    raise TypeError(f"points must be float32, uint8 or int8, got {t.dtype}")
 
 
 def _rows(t: torch.Tensor, name: str) -> torch.Tensor:

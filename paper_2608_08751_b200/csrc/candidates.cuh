@@ -9,6 +9,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 namespace ivf {
 
 constexpr int kCandStatusBadId = -6;
@@ -18,10 +20,18 @@ template <typename T>
 __device__ __forceinline__ void cand_load_piece(const T* row, int t, float (&v)[4]) {
     if constexpr (sizeof(T) == 1) {
         const uint32_t w = *reinterpret_cast<const uint32_t*>(row + t);
-        v[0] = static_cast<float>(w & 255u);
-        v[1] = static_cast<float>((w >> 8) & 255u);
-        v[2] = static_cast<float>((w >> 16) & 255u);
-        v[3] = static_cast<float>(w >> 24);
+        if constexpr (std::is_signed<T>::value) {
+            const int sv = static_cast<int>(w);
+            v[0] = static_cast<float>((sv << 24) >> 24);
+            v[1] = static_cast<float>((sv << 16) >> 24);
+            v[2] = static_cast<float>((sv << 8) >> 24);
+            v[3] = static_cast<float>(sv >> 24);
+        } else {
+            v[0] = static_cast<float>(w & 255u);
+            v[1] = static_cast<float>((w >> 8) & 255u);
+            v[2] = static_cast<float>((w >> 16) & 255u);
+            v[3] = static_cast<float>(w >> 24);
+        }
     } else {
         const float4 f = *reinterpret_cast<const float4*>(row + t);
         v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;

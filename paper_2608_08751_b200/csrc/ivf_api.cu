@@ -289,12 +289,19 @@ int make_tmap(CUtensorMap* map, const void* base, int64_t rows, int kp, int box_
 }
 
 // ------------------------------------------------------------------ argument checks (no CUDA calls)
+inline bool valid_dtype(int t) { return t == IVF_F32 || t == IVF_U8 || t == IVF_I8; }
+inline size_t dtype_size(int t) { return t == IVF_F32 ? 4 : 1; }
+int check_d(int d) {
+    if (d < 4 || d > 256 || d % 4 != 0)
+        return fail(IVF_ERR_UNSUPPORTED, "d = %d: must be a multiple of 4 in [4, 256]", d);
+    return IVF_OK;
+}
+
 int check_common(const void* points, int64_t n, int d, int ptype, const float* centroids, int nlist, int k,
                  const int32_t* out_ids) {
     if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
-    if (ptype != IVF_F32 && ptype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", ptype);
-    if (d < 16 || d > 256 || d % 16 != 0)
-        return fail(IVF_ERR_UNSUPPORTED, "d = %d: must be a multiple of 16 in [16, 256]", d);
+    if (!valid_dtype(ptype)) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", ptype);
+    if (check_d(d) != IVF_OK) return IVF_ERR_UNSUPPORTED;
     if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
     if (k < 1 || k > nlist || k > 512)
         return fail(IVF_ERR_UNSUPPORTED, "nprobe = %d: must be in [1, min(nlist, 512)] (nlist = %d)", k, nlist);
@@ -506,7 +513,9 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     int* failbuf = nullptr;
     uint64_t* fbkeys = nullptr;
     float* tau = nullptr;
-    const int u8 = ptype == IVF_U8;
+    // uint8 rows whose length is a multiple of 16 are widened inside the fused kernel (no copy in HBM);
+    // every other input goes through an fp16 operand copy
+    const bool u8 = ptype == IVF_U8 && d % 16 == 0;
     pp.x16 = nullptr;
     pp.x_raw = u8 ? static_cast<const uint8_t*>(points) : nullptr;
     pp.d = d;
@@ -522,19 +531,27 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
 
     int tk = -1;
     if (!u8) {
-        // float points: magnitude, scales and the fp16 operand copy (uint8 points are widened inside
-        // the fused kernel, which also derives the scales and writes |x|^2)
+        // magnitude (float points only: byte types have a fixed bound), scales and the fp16 operand
+        // copy with |x|^2
         tk = timing_begin(TK_PREP, stream);
-        CUDA_TRY(cudaMemsetAsync(cp.bits, 0, sizeof(unsigned int), stream));
-        const int64_t count = n * d;
-        int blocks = static_cast<int>((count + 256 * 8 - 1) / (256 * 8));
-        if (blocks > ctx.num_sms * 8) blocks = ctx.num_sms * 8;
-        maxabs_kernel<<<blocks, 256, 0, stream>>>(static_cast<const float*>(points), count, cp.bits);
-        LAUNCH_CHECK();
         const int64_t threads = n * 32;
         const unsigned cblocks = static_cast<unsigned>((threads + 255) / 256);
-        convert_rows_kernel<float, false><<<cblocks, 256, 0, stream>>>(static_cast<const float*>(points), n, d, pl.kd,
-                                                                       cp.scal, pp.x16, pp.xn, cp.bits, 0);
+        if (ptype == IVF_F32) {
+            CUDA_TRY(cudaMemsetAsync(cp.bits, 0, sizeof(unsigned int), stream));
+            const int64_t count = n * d;
+            int blocks = static_cast<int>((count + 256 * 8 - 1) / (256 * 8));
+            if (blocks > ctx.num_sms * 8) blocks = ctx.num_sms * 8;
+            maxabs_kernel<<<blocks, 256, 0, stream>>>(static_cast<const float*>(points), count, cp.bits);
+            LAUNCH_CHECK();
+            convert_rows_kernel<float, false><<<cblocks, 256, 0, stream>>>(static_cast<const float*>(points), n, d, pl.kd,
+                                                                           cp.scal, pp.x16, pp.xn, cp.bits, 0);
+        } else if (ptype == IVF_U8) {
+            convert_rows_kernel<uint8_t, false><<<cblocks, 256, 0, stream>>>(static_cast<const uint8_t*>(points), n, d,
+                                                                             pl.kd, cp.scal, pp.x16, pp.xn, cp.bits, 1);
+        } else {
+            convert_rows_kernel<int8_t, false><<<cblocks, 256, 0, stream>>>(static_cast<const int8_t*>(points), n, d,
+                                                                            pl.kd, cp.scal, pp.x16, pp.xn, cp.bits, 1);
+        }
         LAUNCH_CHECK();
         timing_end(tk, stream);
         rc = make_tmap(&pp.tmap_x, pp.x16, n, pl.kp, kBlockM, false);
@@ -661,6 +678,9 @@ int update_device(DeviceCtx& ctx, const void* points, int ptype, const int32_t* 
     if (ptype == IVF_U8)
         update_reduce_kernel<uint8_t><<<lb, 256, 0, stream>>>(static_cast<const uint8_t*>(points), perm, off, nlist, d,
                                                               sums, reinterpret_cast<long long*>(counts));
+    else if (ptype == IVF_I8)
+        update_reduce_kernel<int8_t><<<lb, 256, 0, stream>>>(static_cast<const int8_t*>(points), perm, off, nlist, d,
+                                                             sums, reinterpret_cast<long long*>(counts));
     else
         update_reduce_kernel<float><<<lb, 256, 0, stream>>>(static_cast<const float*>(points), perm, off, nlist, d,
                                                             sums, reinterpret_cast<long long*>(counts));
@@ -692,7 +712,7 @@ int run_chunks(const void* points, int64_t n, int d, int ptype, const float* cen
     const int where = classify_pointer(points);
     if (where < 0) return where;
     const bool host = where == 1;
-    const size_t esize = ptype == IVF_U8 ? 1 : 4;
+    const size_t esize = dtype_size(ptype);
 
     int64_t rows = rows_per_launch(d, k);
     if (g_row_chunk_override.load() > 0) rows = g_row_chunk_override.load();
@@ -785,8 +805,7 @@ int ivf_route(const void* queries, int64_t nq, int d, ivf_dtype qtype, const flo
 int ivf_centroids_create(const float* centroids, int nlist, int d, ivf_centroids** out, void* stream_) {
     if (!out) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
     *out = nullptr;
-    if (d < 16 || d > 256 || d % 16 != 0)
-        return fail(IVF_ERR_UNSUPPORTED, "d = %d: must be a multiple of 16 in [16, 256]", d);
+    if (check_d(d) != IVF_OK) return IVF_ERR_UNSUPPORTED;
     if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
     if (!centroids) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
     if (reinterpret_cast<uintptr_t>(centroids) & 15) return fail(IVF_ERR_INVALID_ARG, "centroids must be 16-byte aligned");
@@ -859,9 +878,8 @@ int ivf_assign(const void* points, int64_t n, int d, ivf_dtype ptype, const floa
 int ivf_centroid_update(const void* points, ivf_dtype ptype, const int32_t* ids, int64_t n, int d, int nlist,
                         float* sums, int64_t* counts, void* stream) {
     if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
-    if (ptype != IVF_F32 && ptype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
-    if (d < 16 || d > 256 || d % 16 != 0)
-        return fail(IVF_ERR_UNSUPPORTED, "d = %d: must be a multiple of 16 in [16, 256]", d);
+    if (!valid_dtype(ptype)) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
+    if (check_d(d) != IVF_OK) return IVF_ERR_UNSUPPORTED;
     if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
     if (n >= (int64_t(1) << 31)) return fail(IVF_ERR_UNSUPPORTED, "n = %lld: at most 2^31 - 1 rows per call", (long long)n);
     if (n == 0) return IVF_OK;
@@ -877,9 +895,8 @@ int ivf_centroid_update(const void* points, ivf_dtype ptype, const int32_t* ids,
 int ivf_cluster_major_reorder(const void* points, ivf_dtype ptype, const int32_t* ids, int64_t n, int d, int nlist,
                               void* out_points, int64_t* out_offsets, int32_t* out_order, void* stream_) {
     if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
-    if (ptype != IVF_F32 && ptype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
-    if (d < 16 || d > 256 || d % 16 != 0)
-        return fail(IVF_ERR_UNSUPPORTED, "d = %d: must be a multiple of 16 in [16, 256]", d);
+    if (!valid_dtype(ptype)) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
+    if (check_d(d) != IVF_OK) return IVF_ERR_UNSUPPORTED;
     if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
     if (n >= (int64_t(1) << 31)) return fail(IVF_ERR_UNSUPPORTED, "n = %lld: at most 2^31 - 1 rows per call", (long long)n);
     if (!out_offsets || !out_order) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
@@ -913,10 +930,18 @@ int ivf_cluster_major_reorder(const void* points, ivf_dtype ptype, const int32_t
     if (n > 0) {
         update_fill_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, off, cur, out_order);
         LAUNCH_CHECK();
-        const int row_chunks = d * (ptype == IVF_U8 ? 1 : 4) / 16;
-        const int64_t pieces = n * row_chunks;
-        reorder_gather_kernel<<<static_cast<unsigned>((pieces + 255) / 256), 256, 0, stream>>>(
-            static_cast<const uint4*>(points), out_order, n, row_chunks, static_cast<uint4*>(out_points));
+        const int row_bytes = d * static_cast<int>(dtype_size(ptype));
+        if (row_bytes % 16 == 0) {
+            const int row_chunks = row_bytes / 16;
+            const int64_t pieces = n * row_chunks;
+            reorder_gather_kernel<uint4><<<static_cast<unsigned>((pieces + 255) / 256), 256, 0, stream>>>(
+                static_cast<const uint4*>(points), out_order, n, row_chunks, static_cast<uint4*>(out_points));
+        } else {
+            const int row_chunks = row_bytes / 4;
+            const int64_t pieces = n * row_chunks;
+            reorder_gather_kernel<uint32_t><<<static_cast<unsigned>((pieces + 255) / 256), 256, 0, stream>>>(
+                static_cast<const uint32_t*>(points), out_order, n, row_chunks, static_cast<uint32_t*>(out_points));
+        }
         LAUNCH_CHECK();
     }
     timing_end(tk, stream);
@@ -949,7 +974,7 @@ int ivf_assign_update(const void* points, int64_t n, int d, ivf_dtype ptype, con
 int ivf_assign_candidates(const void* points, int64_t n, int d, ivf_dtype ptype, const float* centroids, int nlist,
                           const int32_t* cand_ids, int m, int32_t* out_ids, float* out_dists, void* stream_) {
     if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
-    if (ptype != IVF_F32 && ptype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
+    if (!valid_dtype(ptype)) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
     if (d < 4 || d > kCandMaxD || d % 4 != 0)
         return fail(IVF_ERR_UNSUPPORTED, "d = %d: must be a multiple of 4 in [4, %d]", d, kCandMaxD);
     if (nlist < 1 || m < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d, candidates per row = %d", nlist, m);
@@ -966,6 +991,9 @@ int ivf_assign_candidates(const void* points, int64_t n, int d, ivf_dtype ptype,
     if (ptype == IVF_U8)
         assign_candidates_kernel<uint8_t><<<grid, 256, 0, stream>>>(static_cast<const uint8_t*>(points), n, d, centroids, nlist,
                                                                     cand_ids, m, out_ids, out_dists, pctx->status);
+    else if (ptype == IVF_I8)
+        assign_candidates_kernel<int8_t><<<grid, 256, 0, stream>>>(static_cast<const int8_t*>(points), n, d, centroids, nlist,
+                                                                   cand_ids, m, out_ids, out_dists, pctx->status);
     else
         assign_candidates_kernel<float><<<grid, 256, 0, stream>>>(static_cast<const float*>(points), n, d, centroids, nlist,
                                                                   cand_ids, m, out_ids, out_dists, pctx->status);
@@ -1001,7 +1029,7 @@ int pq_set_attrs(DeviceCtx& ctx) {
 int ivf_pq_encode(const void* points, int64_t n, int d, ivf_dtype ptype, const int32_t* ids, const float* centroids,
                   int nlist, const float* codebooks, int pq_m, uint8_t* out_codes, void* stream_) {
     if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
-    if (ptype != IVF_F32 && ptype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
+    if (!valid_dtype(ptype)) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
     if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
     int rc = pq_check_shape(d, pq_m, codebooks, true);
     if (rc != IVF_OK) return rc;
@@ -1016,7 +1044,7 @@ int ivf_pq_encode(const void* points, int64_t n, int d, ivf_dtype ptype, const i
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     PqEncodeParams p;
     p.x = points;
-    p.x_is_u8 = ptype == IVF_U8;
+    p.x_type = ptype;
     p.n = n;
     p.d = d;
     p.pq_m = pq_m;
@@ -1039,7 +1067,7 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
                   int64_t n_codes, const float* codebooks, int pq_m, int n_rerank, const int64_t* vec_ids,
                   int64_t* out_ids, float* out_est, int64_t* out_counts, void* stream_) {
     if (nq < 0) return fail(IVF_ERR_INVALID_ARG, "negative query count %lld", (long long)nq);
-    if (qtype != IVF_F32 && qtype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)qtype);
+    if (!valid_dtype(qtype)) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)qtype);
     if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
     if (nprobe < 1 || nprobe > nlist) return fail(IVF_ERR_INVALID_ARG, "nprobe = %d with nlist = %d", nprobe, nlist);
     if (nprobe > kPqMaxProbes) return fail(IVF_ERR_UNSUPPORTED, "nprobe = %d: at most %d", nprobe, kPqMaxProbes);
@@ -1089,7 +1117,7 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     LAUNCH_CHECK();
     PqScanParams sp;
     sp.q = queries;
-    sp.q_is_u8 = qtype == IVF_U8;
+    sp.q_type = qtype;
     sp.nq = nq;
     sp.d = d;
     sp.pq_m = pq_m;
@@ -1164,7 +1192,7 @@ int64_t ivf_launch_count(void) { return g_launches.load(); }
 
 int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[9]) {
     if (n < 1 || nlist < 1 || num_sms < 1 || !out) return fail(IVF_ERR_INVALID_ARG, "bad plan arguments");
-    if (d < 16 || d > 256 || d % 16 != 0) return fail(IVF_ERR_UNSUPPORTED, "d = %d", d);
+    if (check_d(d) != IVF_OK) return IVF_ERR_UNSUPPORTED;
     Plan pl;
     int stride = 1;
     int rc = make_plan(n, nlist, d, k, num_sms, &pl, k > 1 && choose_rule(k, nlist, &stride) != TAU_GIVEN);
@@ -1300,9 +1328,8 @@ int* g_noalloc_ptr[kMaxDevices] = {};
 extern "C" int ivf_centroid_update_noalloc(const void* points, ivf_dtype ptype, const int32_t* ids, int64_t n, int d,
                                            int nlist, float* sums, int64_t* counts, void* stream_) {
     if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
-    if (ptype != IVF_F32 && ptype != IVF_U8) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
-    if (d < 16 || d > 256 || d % 16 != 0)
-        return fail(IVF_ERR_UNSUPPORTED, "d = %d: must be a multiple of 16 in [16, 256]", d);
+    if (!valid_dtype(ptype)) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
+    if (check_d(d) != IVF_OK) return IVF_ERR_UNSUPPORTED;
     if (nlist < 1) return fail(IVF_ERR_INVALID_ARG, "nlist = %d", nlist);
     if (n > kNoAllocMaxRows)
         return fail(IVF_ERR_UNSUPPORTED,
@@ -1359,6 +1386,9 @@ extern "C" int ivf_centroid_update_noalloc(const void* points, ivf_dtype ptype, 
     if (ptype == IVF_U8)
         update_reduce_kernel<uint8_t><<<lb, 256, 0, stream>>>(static_cast<const uint8_t*>(points), perm, off, nlist, d,
                                                               sums, reinterpret_cast<long long*>(counts));
+    else if (ptype == IVF_I8)
+        update_reduce_kernel<int8_t><<<lb, 256, 0, stream>>>(static_cast<const int8_t*>(points), perm, off, nlist, d,
+                                                             sums, reinterpret_cast<long long*>(counts));
     else
         update_reduce_kernel<float><<<lb, 256, 0, stream>>>(static_cast<const float*>(points), perm, off, nlist, d,
                                                             sums, reinterpret_cast<long long*>(counts));

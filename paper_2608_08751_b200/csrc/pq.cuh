@@ -171,15 +171,17 @@ __device__ __forceinline__ void pq_build_lut(const float* r, const float* cbt, f
     }
 }
 
-template <typename T>
-__device__ __forceinline__ float pq_elem(const T* x, int64_t idx) {
-    return static_cast<float>(x[idx]);
+// element idx of a row matrix of the given type code (0 float, 1 uint8, 2 int8), as a float
+__device__ __forceinline__ float pq_elem(const void* x, int type, int64_t idx) {
+    if (type == 1) return static_cast<float>(static_cast<const uint8_t*>(x)[idx]);
+    if (type == 2) return static_cast<float>(static_cast<const int8_t*>(x)[idx]);
+    return static_cast<const float*>(x)[idx];
 }
 
 // ------------------------------------------------------------------ residual encoding (Eq. 3 on x - c(x))
 struct PqEncodeParams {
     const void* x;
-    int x_is_u8;
+    int x_type;  // 0 float, 1 uint8, 2 int8
     int64_t n;
     int d, pq_m, nlist;
     const int32_t* ids;
@@ -205,8 +207,7 @@ __global__ void __launch_bounds__(kPqThreads, 1) pq_encode_kernel(const PqEncode
             continue;
         }
         for (int t = threadIdx.x; t < p.d; t += blockDim.x) {
-            const float xv = p.x_is_u8 ? pq_elem(static_cast<const uint8_t*>(p.x), i * p.d + t)
-                                       : pq_elem(static_cast<const float*>(p.x), i * p.d + t);
+            const float xv = pq_elem(p.x, p.x_type, i * p.d + t);
             s.r[t] = __fsub_rn(xv, p.centroids[static_cast<int64_t>(l) * p.d + t]);
         }
         __syncthreads();
@@ -420,7 +421,7 @@ __device__ __forceinline__ uint64_t pq_cut_buffer(uint64_t* buf, int count, int 
 // ------------------------------------------------------------------ chunked ADC scan fused with the group merge
 struct PqScanParams {
     const void* q;
-    int q_is_u8;
+    int q_type;  // 0 float, 1 uint8, 2 int8
     int64_t nq;
     int d, pq_m, nlist, nprobe, n_rerank;
     int ngroups;             // groups per query
@@ -555,8 +556,7 @@ __global__ void __launch_bounds__(kPqScanThreads, 2) pq_scan_kernel(const PqScan
             }
             float qv = 0.0f, cnext = 0.0f;  // thread t < d: its query coordinate, the coming list's centroid coordinate
             if (threadIdx.x < p.d) {
-                qv = p.q_is_u8 ? pq_elem(static_cast<const uint8_t*>(p.q), b * p.d + threadIdx.x)
-                               : pq_elem(static_cast<const float*>(p.q), b * p.d + threadIdx.x);
+                qv = pq_elem(p.q, p.q_type, b * p.d + threadIdx.x);
                 cnext = p.centroids[static_cast<int64_t>(s.list_id[pr]) * p.d + threadIdx.x];
             }
             int built = -1;

@@ -12,6 +12,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "scales.cuh"
 
 namespace ivf {
@@ -70,22 +72,30 @@ __global__ void convert_rows_kernel(const T* __restrict__ x, int64_t rows, int d
     float acc = 0.0f;
     const int c0 = lane * 8;
     if (c0 < kd) {
+        // two 4-element pieces per lane, each present or absent as a whole (d is a multiple of 4)
         float v[8];
-        if (c0 < d) {
-            if constexpr (sizeof(T) == 1) {
-                const uint2 raw = *reinterpret_cast<const uint2*>(x + row * d + c0);
-                const uint32_t w[2] = {raw.x, raw.y};
 #pragma unroll
-                for (int i = 0; i < 8; ++i) v[i] = static_cast<float>((w[i >> 2] >> (8 * (i & 3))) & 0xFFu);
+        for (int half = 0; half < 2; ++half) {
+            const int t = c0 + 4 * half;
+            if (t < d) {
+                if constexpr (sizeof(T) == 1) {
+                    const uint32_t w = *reinterpret_cast<const uint32_t*>(x + row * d + t);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t b = (w >> (8 * i)) & 0xFFu;
+                        if constexpr (std::is_signed<T>::value)
+                            v[4 * half + i] = static_cast<float>(static_cast<int>(static_cast<int8_t>(b)));
+                        else
+                            v[4 * half + i] = static_cast<float>(b);
+                    }
+                } else {
+                    const float4 a = *reinterpret_cast<const float4*>(x + row * d + t);
+                    v[4 * half] = a.x; v[4 * half + 1] = a.y; v[4 * half + 2] = a.z; v[4 * half + 3] = a.w;
+                }
             } else {
-                const float4 a = *reinterpret_cast<const float4*>(x + row * d + c0);
-                const float4 b = *reinterpret_cast<const float4*>(x + row * d + c0 + 4);
-                v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
-                v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-            }
-        } else {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = 0.0f;
+                for (int i = 0; i < 4; ++i) v[4 * half + i] = 0.0f;
+            }
         }
         __half2 h[4];
 #pragma unroll

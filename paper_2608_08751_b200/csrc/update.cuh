@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 namespace ivf {
 
 constexpr int kStatusBadId = -6;
@@ -131,10 +133,18 @@ __global__ void update_reduce_kernel(const T* __restrict__ x, const int* __restr
                             wv[u] = (m + u < cntm) ? *reinterpret_cast<const uint32_t*>(x + rows[u] * d + c0) : 0u;
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
-                            acc[blk][0] += static_cast<float>(wv[u] & 0xFFu);
-                            acc[blk][1] += static_cast<float>((wv[u] >> 8) & 0xFFu);
-                            acc[blk][2] += static_cast<float>((wv[u] >> 16) & 0xFFu);
-                            acc[blk][3] += static_cast<float>(wv[u] >> 24);
+                            if constexpr (std::is_signed<T>::value) {
+                                const int sv = static_cast<int>(wv[u]);  // arithmetic shifts sign-extend each byte
+                                acc[blk][0] += static_cast<float>((sv << 24) >> 24);
+                                acc[blk][1] += static_cast<float>((sv << 16) >> 24);
+                                acc[blk][2] += static_cast<float>((sv << 8) >> 24);
+                                acc[blk][3] += static_cast<float>(sv >> 24);
+                            } else {
+                                acc[blk][0] += static_cast<float>(wv[u] & 0xFFu);
+                                acc[blk][1] += static_cast<float>((wv[u] >> 8) & 0xFFu);
+                                acc[blk][2] += static_cast<float>((wv[u] >> 16) & 0xFFu);
+                                acc[blk][3] += static_cast<float>(wv[u] >> 24);
+                            }
                         }
                     } else {
                         float4 fv[4];
@@ -171,9 +181,10 @@ __global__ void update_reduce_kernel(const T* __restrict__ x, const int* __restr
 }
 
 // Cluster-major copy (Sec. 3.1 index layout): destination row p receives source row order[p];
-// one thread per 16-byte piece of a row.  Also widens the list offsets to 64 bits.
-__global__ void reorder_gather_kernel(const uint4* __restrict__ src, const int* __restrict__ order, int64_t n,
-                                      int row_chunks, uint4* __restrict__ dst) {
+// one thread per 16-byte piece of a row (4-byte pieces when a row is not a multiple of 16 bytes).  Also widens the list offsets to 64 bits.
+template <typename Piece>
+__global__ void reorder_gather_kernel(const Piece* __restrict__ src, const int* __restrict__ order, int64_t n,
+                                      int row_chunks, Piece* __restrict__ dst) {
     const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (i >= n * row_chunks) return;
     const int64_t p = i / row_chunks;

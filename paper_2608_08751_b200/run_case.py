@@ -67,6 +67,52 @@ def stream_case(args):
                       "tflops": 2.0 * args.n * args.nlist * args.d / (ms / 1e3) / 1e12, "inertia": inertia}))
 
 
+def build_case(args):
+    """Index construction in the accelerated style (appendix on fast index building): the centroids
+    are trained by Lloyd iterations on a SAMPLE of the base set (--train-rows), then every base
+    vector is assigned once, regrouped list-major and residual-encoded.  Assignment is exact brute
+    force here (no graph); everything streams from page-locked host memory."""
+    chunk = synth.CHUNK_ROWS
+    nchunks = -(-args.n // chunk)
+    host = torch.empty((args.n, args.d), dtype=torch.uint8 if args.dtype == "u8" else torch.float32).pin_memory()
+    for c in range(nchunks):
+        rows = min(chunk, args.n - c * chunk)
+        blk = synth.sift_like_rows(c, rows=rows, d=args.d) if args.dtype == "u8" else synth.deep_like_rows(c, rows, args.d)
+        host[c * chunk:c * chunk + rows] = torch.from_numpy(blk)
+    train_rows = min(args.train_rows, args.n)
+    train = host[:train_rows]
+    init = synth.init_sample(train_rows, args.nlist)
+    cent = train[torch.from_numpy(init)].to(torch.float32).cuda()
+    sums = torch.zeros((args.nlist, args.d), dtype=torch.float32, device="cuda")
+    counts = torch.zeros((args.nlist,), dtype=torch.int64, device="cuda")
+    ids = torch.empty((args.n,), dtype=torch.int32, device="cuda")
+    cb = torch.from_numpy(synth.pq_codebooks(args.pq_m, args.d // args.pq_m, 20.0 if args.dtype == "u8" else 0.05, seed=1)).cuda()
+    B.ivf_assign_update(train[:4096], cent, sums, counts, None, None)  # warm-up (workspace growth)
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    ev[0].record()
+    for _ in range(args.iters):
+        sums.zero_()
+        counts.zero_()
+        B.ivf_assign_update(train, cent, sums, counts, None, None)
+        B.ivf_centroid_finalize(sums, counts, cent)
+    ev[1].record()
+    B.ivf_assign(host, cent, ids, None, want_dists=False)
+    ev[2].record()
+    dev_rows = host.cuda()
+    xr, offsets, order = B.ivf_cluster_major_reorder(dev_rows, ids, args.nlist)
+    codes = B.ivf_pq_encode(xr, ids[order.long()], cent, cb)
+    ev[3].record()
+    B.ivf_check()
+    t = [ev[i].elapsed_time(ev[i + 1]) for i in range(3)]
+    lens = (offsets[1:] - offsets[:-1])
+    print(json.dumps({"op": "build", "n": args.n, "train_rows": train_rows, "nlist": args.nlist, "d": args.d,
+                      "dtype": args.dtype, "iters": args.iters, "train_ms": t[0], "assign_all_ms": t[1],
+                      "reorder_encode_ms": t[2], "total_ms": sum(t), "vectors_per_s": args.n / (sum(t) / 1e3),
+                      "empty_lists": int((lens == 0).sum().item()), "max_list": int(lens.max().item()),
+                      "codes_bytes": int(codes.numel())}))
+
+
 def serve_case(args):
     if args.dtype == "u8":
         c = synth.sift_like_centroids(args.nlist, args.d)
@@ -200,7 +246,8 @@ def candidates_case(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="assign", choices=["assign", "route", "update", "stream", "serve", "pq", "candidates"])
+    ap.add_argument("--op", default="assign", choices=["assign", "route", "update", "stream", "serve", "pq", "candidates", "build"])
+    ap.add_argument("--train-rows", type=int, default=1 << 20, dest="train_rows", help="sample size of --op build")
     ap.add_argument("--pq-m", type=int, default=32, dest="pq_m")
     ap.add_argument("--n-rerank", type=int, default=512, dest="n_rerank")
     ap.add_argument("--batches", default="8,32,256,2048", help="query batch sizes of --op serve")
@@ -209,7 +256,7 @@ def main():
     ap.add_argument("--nlist", type=int, default=65536)
     ap.add_argument("--d", type=int, default=128)
     ap.add_argument("--k", type=int, default=64)
-    ap.add_argument("--dtype", default="u8", choices=["u8", "f32"])
+    ap.add_argument("--dtype", default="u8", choices=["u8", "f32", "i8"])
     ap.add_argument("--reps", type=int, default=3)
     args = ap.parse_args()
 
@@ -221,7 +268,11 @@ def main():
         return pq_case(args)
     if args.op == "candidates":
         return candidates_case(args)
-    if args.dtype == "u8":
+    if args.op == "build":
+        return build_case(args)
+    if args.dtype == "i8":
+        x, c = synth.spacev_like(args.n, args.nlist, seed=0, d=args.d)
+    elif args.dtype == "u8":
         x = synth.sift_like_rows(0, rows=args.n, d=args.d)
         c = synth.sift_like_centroids(args.nlist, args.d)
     else:

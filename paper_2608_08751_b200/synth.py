@@ -192,3 +192,15 @@ def distinct_probes(nq: int, nlist: int, nprobe: int, seed: int) -> np.ndarray:
     for b in range(nq):
         out[b] = rng.choice(nlist, size=nprobe, replace=False)
     return out
+
+
+# ------------------------------------------------------------------ SPACEV-shaped inputs (Table 2: int8, d = 100)
+def spacev_like(rows: int, nlist: int, seed: int, d: int = 100):
+    """(points int8 [rows, d], centroids float32 [nlist, d]): a 1,000-component mixture (means
+    N(0, 30^2), std 12) rounded and clipped to signed bytes; centroids are fresh mixture samples
+    with N(0, 1) noise, unrounded."""
+    rng = _rng(9, seed)
+    means = rng.normal(0.0, 30.0, size=(N_COMPONENTS, d)).astype(np.float32)
+    x = _mixture_rows(rng, means, rows, 12.0)
+    c = _mixture_rows(rng, means, nlist, 12.0) + rng.normal(0.0, 1.0, size=(nlist, d)).astype(np.float32)
+    return np.clip(np.rint(x), -128, 127).astype(np.int8), c.astype(np.float32)

@@ -63,8 +63,8 @@ def check_update(x, ids, nlist, gpu_sums, gpu_counts, base_sums=None, base_count
         sums = sums + base_sums
     assert (np.asarray(gpu_counts) == counts).all(), "counts differ"
     gs = np.asarray(gpu_sums, dtype=np.float64)
-    if x.dtype == np.uint8 and sums.max() < 2 ** 24:
-        assert (gs == sums).all(), "uint8 sums must be exact"
+    if x.dtype in (np.uint8, np.int8) and np.abs(sums).max() < 2 ** 24:
+        assert (gs == sums).all(), "byte-typed sums must be exact"
         return 0.0
     mag = np.zeros_like(sums)
     np.add.at(mag, ids, np.abs(x.astype(np.float64)))

@@ -45,7 +45,7 @@ def test_argument_errors_come_before_any_cuda_call():
     p = ctypes.addressof(buf)
     p = (p + 255) & ~255
     assert _route(L, p, -1, 128, 0, p, 10, 1, p) == binding.IVF_ERR_INVALID_ARG
-    assert _route(L, p, 4, 100, 0, p, 10, 1, p) == binding.IVF_ERR_UNSUPPORTED      # d % 16
+    assert _route(L, p, 4, 102, 0, p, 10, 1, p) == binding.IVF_ERR_UNSUPPORTED      # d % 4
     assert _route(L, p, 4, 272, 0, p, 10, 1, p) == binding.IVF_ERR_UNSUPPORTED      # d > 256
     assert _route(L, p, 4, 128, 7, p, 10, 1, p) == binding.IVF_ERR_INVALID_ARG      # dtype
     assert _route(L, p, 4, 128, 0, p, 10, 11, p) == binding.IVF_ERR_UNSUPPORTED     # nprobe > nlist
@@ -61,7 +61,7 @@ def test_argument_errors_come_before_any_cuda_call():
     assert L.ivf_assign(None, 0, 96, 0, None, 5, None, None, None) == binding.IVF_OK
     assert L.ivf_assign(p, 3, 96, 0, None, 5, p, None, None) == binding.IVF_ERR_INVALID_ARG
     assert L.ivf_centroid_update(p, 0, p, -2, 128, 10, p, p, None) == binding.IVF_ERR_INVALID_ARG
-    assert L.ivf_centroid_update(p, 0, p, 5, 20, 10, p, p, None) == binding.IVF_ERR_UNSUPPORTED
+    assert L.ivf_centroid_update(p, 0, p, 5, 22, 10, p, p, None) == binding.IVF_ERR_UNSUPPORTED
     assert L.ivf_centroid_update(p, 0, None, 5, 32, 10, p, p, None) == binding.IVF_ERR_INVALID_ARG
     assert L.ivf_centroid_update(None, 0, None, 0, 32, 10, None, None, None) == binding.IVF_OK
     assert L.ivf_assign_update(p, 5, 32, 0, p, 10, None, None, None, p, 0, None) == binding.IVF_ERR_INVALID_ARG
