@@ -223,6 +223,10 @@ int ivf_debug_rule(int k, int nlist, int out[2]);
 int ivf_debug_stats(int enable, int64_t out[3]);
 /* Test hook: groups per query used by ivf_pq_search (clamped to [1, 256]); 0 = chosen from the sizes. */
 int ivf_debug_set_pq_groups(int groups);
+/* Test hook: mask of the kernel families of the routing path that may start while their predecessor
+ * drains (programmatic dependent launch): 1 operand preparation, 2 fused kernel, 4 threshold merge,
+ * 8 merge, 16 merge of passed-on rows, 32 recomputation.  0 = ordinary stream launches; default 57. */
+int ivf_debug_set_dependent_launch(int mask);
 int ivf_debug_timing(int enable);
 int ivf_debug_timing_read(double ms[9], int64_t launches[9]);
 

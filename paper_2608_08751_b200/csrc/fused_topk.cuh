@@ -342,9 +342,9 @@ __device__ __forceinline__ void consume(uint32_t (&acc)[32], int jbase, RowState
                 "min.f32 m, m, %7, %8;\n\t"
                 "min.f32 m, m, %9;\n\t"
                 "setp.le.f32 p, m, %1;\n\t"
-                "@p st.global.v4.f32 [%0], {%2, %3, %4, %5};\n\t"
-                "@p st.global.v4.f32 [%0+16], {%6, %7, %8, %9};\n\t"
-                "@p st.global.b32 [%0+32], %10;\n\t"
+                "@p st.global.cs.v4.f32 [%0], {%2, %3, %4, %5};\n\t"
+                "@p st.global.cs.v4.f32 [%0+16], {%6, %7, %8, %9};\n\t"
+                "@p st.global.cs.b32 [%0+32], %10;\n\t"
                 "@p add.s64 %0, %0, 48;\n\t}"
                 : "+l"(st.wp)
                 : "f"(st.tau), "f"(__uint_as_float(acc[8 * g])), "f"(__uint_as_float(acc[8 * g + 1])),
@@ -491,10 +491,6 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             mbar_init(&b_empty[i], 1);
         }
         *abort_flag = 0;
-        if (blockIdx.x == 0) {
-            if (p.clear0) *p.clear0 = 0;
-            if (p.clear1) *p.clear1 = 0;
-        }
         fence_mbar_init();
         tma_prefetch_desc(&tmap_x);
         tma_prefetch_desc(&tmap_xa);
@@ -509,6 +505,13 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // the set-up above touched no global memory; from here on the predecessor's results are needed
+    pdl_wait();
+    pdl_trigger();
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        if (p.clear0) *p.clear0 = 0;
+        if (p.clear1) *p.clear1 = 0;
+    }
 
     WaitCtl ctl;
     ctl.abort_flag = abort_flag;

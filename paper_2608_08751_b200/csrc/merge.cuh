@@ -45,6 +45,8 @@ __device__ __forceinline__ int slots_of_row_tile(int64_t total_units, int ctas, 
 
 // k = 1: one thread per row takes the lexicographic minimum over the row's partial results.
 __global__ void merge_argmin_kernel(const MergeParams p) {
+    pdl_wait();
+    pdl_trigger();
     const int64_t row = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (row >= p.n) return;
     const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows);
@@ -110,6 +112,8 @@ __device__ __forceinline__ void merge_fail_row(const MergeParams& p, int64_t row
 // value, id) in shared memory; more than kSortCap raw entries are folded in rounds.  If p.big is
 // set the CTAs walk that list of rows (the rows the warp-level kernel passed on) instead of all.
 __global__ void __launch_bounds__(kMergeThreads) merge_select_kernel(const MergeParams p) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ uint64_t keys[kSortCap];
     __shared__ int pre[kMaxSlots + 1];  // exclusive prefix of the slots' entry counts
     __shared__ float s_tau[kMergeThreads / 32];
@@ -335,6 +339,8 @@ __device__ __forceinline__ void warp_bitonic_sort(uint64_t* keys, int m, int lan
 
 template <int KEYS, int SORT, int WARPS>
 __global__ void __launch_bounds__(32 * WARPS) merge_warp_kernel(const MergeParams p) {
+    pdl_wait();
+    pdl_trigger();
     extern __shared__ __align__(16) uint8_t merge_smem_raw[];
     constexpr int kWarpKeys = KEYS, kWarpSort = SORT;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -507,6 +513,8 @@ __device__ __forceinline__ void take16(float (&v)[kSampleM], int lane, float* ou
 }
 
 __global__ void __launch_bounds__(kTauThreads) merge_tau_kernel(const MergeParams p) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ float lists[kTauThreads / 32 + 1][kSampleM];  // one per warp, plus the running result
     const float INF = __int_as_float(0x7f800000);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -540,6 +548,8 @@ __global__ void __launch_bounds__(kTauThreads) merge_tau_kernel(const MergeParam
 // The same with one warp per row, for rows with at most 32 partial sketches (large batches, where
 // few CTAs share a row): lane = sketch.
 __global__ void __launch_bounds__(256) merge_tau_warp_kernel(const MergeParams p) {
+    pdl_wait();
+    pdl_trigger();
     const float INF = __int_as_float(0x7f800000);
     const int lane = threadIdx.x & 31;
     const int64_t row = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
@@ -746,6 +756,8 @@ __device__ __forceinline__ void fallback_finish_row(const FallbackParams& p, con
 
 // The first kFallbackFastRows failed rows: grid (slices, kFallbackFastRows), one slice of one row per CTA.
 __global__ void __launch_bounds__(kFallbackThreads) fallback_keys_kernel(const FallbackParams p) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ FallbackSmem sm;
     const int nfail = p.fail[0];
     const int idx = blockIdx.y;
@@ -758,6 +770,8 @@ __global__ void __launch_bounds__(kFallbackThreads) fallback_keys_kernel(const F
 // Blocks [0, kFallbackFastRows) finish the rows whose candidates fallback_keys_kernel prepared.  The
 // other blocks take any further failed rows (none in practice), one CTA per row doing both stages.
 __global__ void __launch_bounds__(kFallbackThreads) fallback_select_kernel(const FallbackParams p) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ FallbackSmem sm;
     const int nfail = p.fail[0];
     if (blockIdx.x < kFallbackFastRows) {

@@ -14,12 +14,15 @@
 
 #include <type_traits>
 
+#include "ptx.cuh"
 #include "scales.cuh"
 
 namespace ivf {
 
 // max |x| over a float array, as the bit pattern of a non-negative float (atomicMax on uint).
 __global__ void maxabs_kernel(const float* __restrict__ x, int64_t count, unsigned int* out_bits) {
+    pdl_wait();
+    pdl_trigger();
     float m = 0.0f;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
     for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < count; i += stride)
@@ -38,6 +41,8 @@ __global__ void maxabs_kernel(const float* __restrict__ x, int64_t count, unsign
 }
 
 __global__ void scales_kernel(const unsigned int* bits, int points_are_u8, float* scal) {
+    pdl_wait();
+    pdl_trigger();
     float v[4];
     compute_scales(bits, points_are_u8, v);
 #pragma unroll
@@ -52,6 +57,8 @@ template <typename T, bool CENTROID>
 __global__ void convert_rows_kernel(const T* __restrict__ x, int64_t rows, int d, int kd, float* scal,
                                     __half* __restrict__ out, float* __restrict__ norms,
                                     const unsigned int* __restrict__ bits, int points_are_u8) {
+    pdl_wait();
+    pdl_trigger();
     const int lane = threadIdx.x & 31;
     const int64_t row = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
     if (row >= rows) return;

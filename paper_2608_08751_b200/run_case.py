@@ -258,7 +258,10 @@ def main():
     ap.add_argument("--k", type=int, default=64)
     ap.add_argument("--dtype", default="u8", choices=["u8", "f32", "i8"])
     ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--dependent-launch", type=int, default=-1, help="kernel-family mask of dependent launches (0 = none)")
     args = ap.parse_args()
+    if args.dependent_launch >= 0:
+        B.ivf_debug_set_dependent_launch(args.dependent_launch)
 
     if args.op == "stream":
         return stream_case(args)
