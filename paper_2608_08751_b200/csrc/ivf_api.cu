@@ -379,10 +379,11 @@ int convert_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, 
     int blocks = static_cast<int>((count + 256 * 8 - 1) / (256 * 8));
     if (blocks > ctx.num_sms * 8) blocks = ctx.num_sms * 8;
     LAUNCH_DEP(1, maxabs_kernel, blocks, 256, 0, stream, centroids, count, cp->bits + 1);
-    LAUNCH_DEP(1, scales_kernel, 1, 1, 0, stream, cp->bits, 1, cp->scal);
+    // the conversion derives the centroid scale from the magnitude word itself and publishes the scale
+    // vector (with the byte-type point scale as a placeholder until the points are known)
     const int64_t threads = static_cast<int64_t>(nlist) * 32;
-    LAUNCH_DEP(1, (convert_rows_kernel<float, true>), static_cast<unsigned>((threads + 255) / 256), 256, 0, stream, 
-        centroids, nlist, d, pl.kd, cp->scal, cp->c16, nullptr, nullptr, 0);
+    LAUNCH_DEP(1, (convert_rows_kernel<float, true>), static_cast<unsigned>((threads + 255) / 256), 256, 0, stream,
+               centroids, nlist, d, pl.kd, cp->scal, cp->c16, nullptr, cp->bits, 1);
     timing_end(tk, stream);
     return IVF_OK;
 }
@@ -624,17 +625,22 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         // ties) are listed in `big` and merged by the general CTA-per-row kernel
         // (both list counters were cleared by the fused kernel that just ran)
         mp.big = failbuf + n + 2;
-        // two sizes of the warp-level kernel: up to 1024 candidates / 512 sorted (k <= 128 under the given
-        // rule), up to 2048 / 1024 (k <= 320); beyond that everything goes to the general kernel
+        // three sizes of the warp-level kernel (the smaller the key buffer, the more warps per SM): up to
+        // 512 candidates / 256 sorted (k <= 68 under the given rule), 1024 / 512 (k <= 140), 2048 / 1024
+        // (k <= 340); beyond that everything goes to the general kernel
         const int expect = given ? 5 * k : 2 * k;
         if (!ctx.merge_attr_set) {
+            CUDA_TRY(cudaFuncSetAttribute(merge_warp_kernel<512, 256, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(8 * sizeof(MergeWarpSmem<512>))));
             CUDA_TRY(cudaFuncSetAttribute(merge_warp_kernel<1024, 512, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(8 * sizeof(MergeWarpSmem<1024>))));
             CUDA_TRY(cudaFuncSetAttribute(merge_warp_kernel<2048, 1024, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(4 * sizeof(MergeWarpSmem<2048>))));
             ctx.merge_attr_set = true;
         }
-        if (expect <= 700) {
+        if (expect <= 340) {
+            LAUNCH_DEP(8, (merge_warp_kernel<512, 256, 8>), static_cast<unsigned>((n + 7) / 8), 256, 8 * sizeof(MergeWarpSmem<512>), stream, mp);
+        } else if (expect <= 700) {
             LAUNCH_DEP(8, (merge_warp_kernel<1024, 512, 8>), static_cast<unsigned>((n + 7) / 8), 256, 8 * sizeof(MergeWarpSmem<1024>), stream, mp);
         } else if (expect <= 1700) {
             LAUNCH_DEP(8, (merge_warp_kernel<2048, 1024, 4>), static_cast<unsigned>((n + 3) / 4), 128, 4 * sizeof(MergeWarpSmem<2048>), stream, mp);

@@ -40,15 +40,6 @@ __global__ void maxabs_kernel(const float* __restrict__ x, int64_t count, unsign
     }
 }
 
-__global__ void scales_kernel(const unsigned int* bits, int points_are_u8, float* scal) {
-    pdl_wait();
-    pdl_trigger();
-    float v[4];
-    compute_scales(bits, points_are_u8, v);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) scal[i] = v[i];
-}
-
 // One warp per row.  Lane g converts columns [8g, 8g+8) of the data part; after the norm is reduced
 // lanes 0 and 1 write the 16 extra columns.  If `bits` is given (point rows), the scales are derived
 // here from the magnitude words instead of being read, and the first thread publishes them in `scal`
