@@ -221,7 +221,9 @@ int ivf_debug_rule(int k, int nlist, int out[2]);
  * the merge, rows recomputed by brute force -- clears them, and switches the counting on or off.
  */
 int ivf_debug_stats(int enable, int64_t out[3]);
-/* Test hook: groups per query used by ivf_pq_search (clamped to [1, 256]); 0 = chosen from the sizes. */
+/* Test hook: groups per query used by ivf_pq_search (clamped to [1, 256]); 0 = chosen from the sizes.
+ * A negative value -(g + 1) asks for g groups and for the scan kernel variant that reads the codebook
+ * through L1 (otherwise the two-team shared-memory variant is used whenever it fits). */
 int ivf_debug_set_pq_groups(int groups);
 /* Test hook: mask of the kernel families of the routing path that may start while their predecessor
  * drains (programmatic dependent launch): 1 operand preparation, 2 fused kernel, 4 threshold merge,
@@ -257,7 +259,7 @@ int ivf_assign_candidates(const void* points, int64_t n, int d, ivf_dtype ptype,
  * codebooks  [pq_m][256][d / pq_m] float32, row-major.  pq_m must divide d.  Encoding keeps the
  *            codebook in shared memory: 1024 * (d + pq_m) + 4 * d + 29,776 bytes must fit one SM's
  *            227 KB (d = 128 with pq_m = 32 does; d = 256 does not); searching needs
- *            1024 * pq_m + 4 * d + 25,680 bytes and d <= 512 -> IVF_ERR_UNSUPPORTED otherwise.
+ *            1024 * pq_m + 21,584 bytes and d <= 256 -> IVF_ERR_UNSUPPORTED otherwise.
  *
  * ivf_pq_encode: out_codes[i][m] = arg-min over j of the table of x_i - centroids[ids[i]]
  *            (Eq. 3 on the residual; ties to the lower j).  An id outside [0, nlist) writes zero

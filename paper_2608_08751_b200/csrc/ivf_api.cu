@@ -365,6 +365,7 @@ struct CentroidPrep {
 };
 
 int g_force_fallback = 0;
+int g_pq_kernel = 0;  // test hook: 1 forces the scan kernel that reads the codebook through L1
 int g_pq_groups = 0;  // test hook: groups per query of ivf_pq_search (0 = chosen from the sizes)
 bool g_stats = false;
 std::atomic<int64_t> g_row_chunk_override{0};  // test hook: rows per fused launch
@@ -1026,9 +1027,9 @@ int pq_check_shape(int d, int pq_m, const float* codebooks, bool encode) {
         return fail(IVF_ERR_INVALID_ARG, "d = %d, pq_m = %d: pq_m must divide d", d, pq_m);
     if (!codebooks) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
     const size_t need = encode ? pq_smem_bytes(d, pq_m) : pq_scan_smem_bytes(d, pq_m);
-    if (need > kSmemLimit || d > kPqScanThreads)
-        return fail(IVF_ERR_UNSUPPORTED, "d = %d, pq_m = %d: %zu bytes of shared memory needed (limit %zu), d at most %d", d,
-                    pq_m, need, static_cast<size_t>(kSmemLimit), kPqScanThreads);
+    if (need > kSmemLimit || d > 256)
+        return fail(IVF_ERR_UNSUPPORTED, "d = %d, pq_m = %d: %zu bytes of shared memory needed (limit %zu), d at most 256", d,
+                    pq_m, need, static_cast<size_t>(kSmemLimit));
     return IVF_OK;
 }
 int pq_set_attrs(DeviceCtx& ctx) {
@@ -1036,6 +1037,8 @@ int pq_set_attrs(DeviceCtx& ctx) {
         CUDA_TRY(cudaFuncSetAttribute(pq_encode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       static_cast<int>(kSmemLimit)));
         CUDA_TRY(cudaFuncSetAttribute(pq_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      static_cast<int>(kSmemLimit)));
+        CUDA_TRY(cudaFuncSetAttribute(pq_scan_teams_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       static_cast<int>(kSmemLimit)));
         ctx.pq_attr_set = true;
     }
@@ -1151,9 +1154,18 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     sp.gcand = gcand;
     sp.gcand_count = gcount;
     sp.status = ctx.status;
-    const int64_t resident = 2 * static_cast<int64_t>(ctx.num_sms);
-    const unsigned grid = static_cast<unsigned>(total_groups < resident ? total_groups : resident);
-    pq_scan_kernel<<<grid, kPqScanThreads, pq_scan_smem_bytes(d, pq_m), stream>>>(sp);
+    // two teams per CTA around one shared-memory codebook when that fits; otherwise (or when asked by
+    // the test hook) two single-team CTAs per SM that read the codebook through L1
+    const bool teams = g_pq_kernel != 1 && nprobe <= kPqTeamProbes && pq_teams_smem_bytes(d, pq_m) <= kSmemLimit;
+    if (teams) {
+        const int64_t pairs = (total_groups + 1) / 2;
+        const unsigned grid = static_cast<unsigned>(pairs < ctx.num_sms ? pairs : ctx.num_sms);
+        pq_scan_teams_kernel<<<grid, 2 * kPqScanThreads, pq_teams_smem_bytes(d, pq_m), stream>>>(sp);
+    } else {
+        const int64_t resident = 2 * static_cast<int64_t>(ctx.num_sms);
+        const unsigned grid = static_cast<unsigned>(total_groups < resident ? total_groups : resident);
+        pq_scan_kernel<<<grid, kPqScanThreads, pq_scan_smem_bytes(d, pq_m), stream>>>(sp);
+    }
     LAUNCH_CHECK();
     timing_end(tk, stream);
     tk = timing_begin(TK_PQ_MERGE, stream);
@@ -1166,7 +1178,11 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     mp.vec_ids = reinterpret_cast<const long long*>(vec_ids);
     mp.out_pos = reinterpret_cast<long long*>(out_ids);
     mp.out_est = out_est;
-    pq_merge_kernel<<<static_cast<unsigned>(nq), kPqThreads, 0, stream>>>(mp);
+    const int64_t slots = static_cast<int64_t>(ngroups) * n_rerank;
+    if (slots > kPqBufKeys && slots <= static_cast<int64_t>(kPqMergeRegKeys) * kPqThreads)
+        pq_merge_kernel<true><<<static_cast<unsigned>(nq), kPqThreads, 0, stream>>>(mp);
+    else
+        pq_merge_kernel<false><<<static_cast<unsigned>(nq), kPqThreads, 0, stream>>>(mp);
     LAUNCH_CHECK();
     timing_end(tk, stream);
     return IVF_OK;
@@ -1303,6 +1319,8 @@ int ivf_debug_set_dependent_launch(int on) {
 }
 
 int ivf_debug_set_pq_groups(int groups) {
+    g_pq_kernel = groups < 0 ? 1 : 0;  // a negative count also selects the single-team kernel
+    if (groups < 0) groups = -groups - 1;
     g_pq_groups = groups < 0 ? 0 : groups;
     return IVF_OK;
 }

@@ -40,11 +40,6 @@ __host__ __device__ inline size_t pq_smem_bytes(int d, int pq_m) {
            static_cast<size_t>(kPqMaxProbes) * 24 + 16;  // probe descriptors
 }
 
-__host__ __device__ inline size_t pq_scan_smem_bytes(int d, int pq_m) {
-    return static_cast<size_t>(pq_m) * kPqK * 4 + static_cast<size_t>(d) * 4 + static_cast<size_t>(kPqScanBufKeys) * 8 +
-           256 * 4 + 64 + static_cast<size_t>(512) * 24 + 16;
-}
-
 struct PqSmem {
     float* cbt;     // [d][256]: coordinate-major codebook
     float* lut;     // [pq_m][256]
@@ -84,6 +79,14 @@ __device__ __forceinline__ PqSmem pq_carve(uint8_t* raw, int d, int pq_m, bool w
     return s;
 }
 
+// A thread group: NT threads numbered tid that synchronise on hardware barrier BAR (BAR = 0 with
+// NT = the CTA size is __syncthreads).  The scan kernels run one or two such groups per CTA.
+template <int BAR, int NT>
+__device__ __forceinline__ void pq_group_sync() {
+    if constexpr (BAR == 0) __syncthreads();
+    else asm volatile("bar.sync %0, %1;" ::"n"(BAR), "n"(NT) : "memory");
+}
+
 // codebooks [pq_m][256][dsub] in global memory -> cbt[(m * dsub + t) * 256 + j]
 __device__ __forceinline__ void pq_load_codebooks(const float* __restrict__ codebooks, int d, int dsub, float* cbt) {
     const int total = d * kPqK;
@@ -108,10 +111,10 @@ __device__ __forceinline__ float pq_cb(const float* p) {
 // offset from three running pointers; four subspaces per trip give four independent chains.
 template <bool kGlobal, int DSUB>
 __device__ __forceinline__ void pq_build_lut_fixed(const float* __restrict__ r, const float* __restrict__ cbt,
-                                                   float* __restrict__ lut, int pq_m) {
-    const int j = threadIdx.x & (kPqK - 1);
-    const int first = threadIdx.x >> 8;
-    const int step = blockDim.x >> 8;
+                                                   float* __restrict__ lut, int pq_m, int tid, int nthreads) {
+    const int j = tid & (kPqK - 1);
+    const int first = tid >> 8;
+    const int step = nthreads >> 8;
     const float* col = cbt + first * (DSUB * kPqK) + j;
     const float* rp = r + first * DSUB;
     float* out = lut + first * kPqK + j;
@@ -148,18 +151,19 @@ __device__ __forceinline__ void pq_build_lut_fixed(const float* __restrict__ r, 
 // lut[m * 256 + j] for the residual r.  kGlobal: cbt points to the transposed codebook in global
 // memory (read through L1); otherwise to the copy in shared memory.
 template <bool kGlobal>
-__device__ __forceinline__ void pq_build_lut(const float* r, const float* cbt, float* lut, int pq_m, int dsub) {
+__device__ __forceinline__ void pq_build_lut(const float* r, const float* cbt, float* lut, int pq_m, int dsub, int tid,
+                                             int nthreads) {
     switch (dsub) {
-        case 2: return pq_build_lut_fixed<kGlobal, 2>(r, cbt, lut, pq_m);
-        case 3: return pq_build_lut_fixed<kGlobal, 3>(r, cbt, lut, pq_m);
-        case 4: return pq_build_lut_fixed<kGlobal, 4>(r, cbt, lut, pq_m);
-        case 6: return pq_build_lut_fixed<kGlobal, 6>(r, cbt, lut, pq_m);
-        case 8: return pq_build_lut_fixed<kGlobal, 8>(r, cbt, lut, pq_m);
+        case 2: return pq_build_lut_fixed<kGlobal, 2>(r, cbt, lut, pq_m, tid, nthreads);
+        case 3: return pq_build_lut_fixed<kGlobal, 3>(r, cbt, lut, pq_m, tid, nthreads);
+        case 4: return pq_build_lut_fixed<kGlobal, 4>(r, cbt, lut, pq_m, tid, nthreads);
+        case 6: return pq_build_lut_fixed<kGlobal, 6>(r, cbt, lut, pq_m, tid, nthreads);
+        case 8: return pq_build_lut_fixed<kGlobal, 8>(r, cbt, lut, pq_m, tid, nthreads);
         default: break;
     }
-    const int j = threadIdx.x & (kPqK - 1);
-    const int step = blockDim.x >> 8;
-    for (int m = threadIdx.x >> 8; m < pq_m; m += step) {
+    const int j = tid & (kPqK - 1);
+    const int step = nthreads >> 8;
+    for (int m = tid >> 8; m < pq_m; m += step) {
         const float* col = cbt + static_cast<size_t>(m) * dsub * kPqK + j;
         const float* rm = r + m * dsub;
         float acc = 0.0f;
@@ -211,7 +215,7 @@ __global__ void __launch_bounds__(kPqThreads, 1) pq_encode_kernel(const PqEncode
             s.r[t] = __fsub_rn(xv, p.centroids[static_cast<int64_t>(l) * p.d + t]);
         }
         __syncthreads();
-        pq_build_lut<false>(s.r, s.cbt, s.lut, p.pq_m, dsub);
+        pq_build_lut<false>(s.r, s.cbt, s.lut, p.pq_m, dsub, threadIdx.x, blockDim.x);
         __syncthreads();
         for (int m = warp; m < p.pq_m; m += nwarps) {
             const float* row = s.lut + m * kPqK;
@@ -312,20 +316,20 @@ __global__ void __launch_bounds__(128) pq_setup_query_kernel(const int32_t* __re
     }
 }
 
-// ------------------------------------------------------------------ block-wide selection of the k smallest keys
+// ------------------------------------------------------------------ selection of the k smallest keys by a thread group
 // Largest admitted key among the `count` distinct 64-bit keys get(0 .. count) (count > k; keys that
-// read as all-ones are padding and must number fewer than count - k): radix
-// select from the top byte down, stopping once the digit that holds rank k is wanted whole.
-template <typename Get>
-__device__ __forceinline__ uint64_t pq_select_bound(Get get, int count, int k, int* hist, int* misc) {
-    const int lane = threadIdx.x & 31;
+// read as all-ones are padding and must number fewer than count - k): radix select from the top
+// byte down, stopping once the digit that holds rank k is wanted whole.
+template <int BAR, int NT, typename Get>
+__device__ __forceinline__ uint64_t pq_select_bound(Get get, int count, int k, int* hist, int* misc, int tid) {
+    const int lane = tid & 31;
     uint64_t prefix = 0, mask = 0;
     int rank = k;
     const int rounded = (count + 31) & ~31;
     for (int shift = 56; shift >= 0; shift -= 8) {
-        for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
-        __syncthreads();
-        for (int i = threadIdx.x; i < rounded; i += blockDim.x) {
+        for (int i = tid; i < 256; i += NT) hist[i] = 0;
+        pq_group_sync<BAR, NT>();
+        for (int i = tid; i < rounded; i += NT) {
             uint32_t dg = 0xFFFFFFFFu;
             if (i < count) {
                 const uint64_t v = get(i);
@@ -334,8 +338,8 @@ __device__ __forceinline__ uint64_t pq_select_bound(Get get, int count, int k, i
             const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dg);
             if (dg != 0xFFFFFFFFu && lane == __ffs(peers) - 1) atomicAdd(&hist[dg], __popc(peers));
         }
-        __syncthreads();
-        if (threadIdx.x < 32) {
+        pq_group_sync<BAR, NT>();
+        if (tid < 32) {
             int r = rank, eq = 0;
             const int digit = radix_pick_digit(hist, lane, r, eq);
             if (lane == 0) {
@@ -344,12 +348,12 @@ __device__ __forceinline__ uint64_t pq_select_bound(Get get, int count, int k, i
                 misc[3] = eq;
             }
         }
-        __syncthreads();
+        pq_group_sync<BAR, NT>();
         prefix |= static_cast<uint64_t>(misc[1]) << shift;
         mask |= 255ull << shift;
         rank = misc[2];
         const bool whole = misc[3] == rank;
-        __syncthreads();
+        pq_group_sync<BAR, NT>();
         if (whole) return prefix | ~mask;
     }
     return prefix;
@@ -357,14 +361,15 @@ __device__ __forceinline__ uint64_t pq_select_bound(Get get, int count, int k, i
 
 // The same selection over keys that every thread holds in registers (PER per thread; all-ones =
 // padding), so that the passes touch no memory but the histogram.
-template <int PER>
-__device__ __forceinline__ uint64_t pq_select_bound_regs(const uint64_t (&mine)[PER], int k, int* hist, int* misc) {
-    const int lane = threadIdx.x & 31;
+template <int BAR, int NT, int PER>
+__device__ __forceinline__ uint64_t pq_select_bound_regs(const uint64_t (&mine)[PER], int k, int* hist, int* misc,
+                                                         int tid) {
+    const int lane = tid & 31;
     uint64_t prefix = 0, mask = 0;
     int rank = k;
     for (int shift = 56; shift >= 0; shift -= 8) {
-        for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
-        __syncthreads();
+        for (int i = tid; i < 256; i += NT) hist[i] = 0;
+        pq_group_sync<BAR, NT>();
 #pragma unroll
         for (int q = 0; q < PER; ++q) {
             const uint64_t v = mine[q];
@@ -375,8 +380,8 @@ __device__ __forceinline__ uint64_t pq_select_bound_regs(const uint64_t (&mine)[
                 if (dg != 0xFFFFFFFFu && lane == __ffs(peers) - 1) atomicAdd(&hist[dg], __popc(peers));
             }
         }
-        __syncthreads();
-        if (threadIdx.x < 32) {
+        pq_group_sync<BAR, NT>();
+        if (tid < 32) {
             int r = rank, eq = 0;
             const int digit = radix_pick_digit(hist, lane, r, eq);
             if (lane == 0) {
@@ -385,36 +390,36 @@ __device__ __forceinline__ uint64_t pq_select_bound_regs(const uint64_t (&mine)[
                 misc[3] = eq;
             }
         }
-        __syncthreads();
+        pq_group_sync<BAR, NT>();
         prefix |= static_cast<uint64_t>(misc[1]) << shift;
         mask |= 255ull << shift;
         rank = misc[2];
         const bool whole = misc[3] == rank;
-        __syncthreads();
+        pq_group_sync<BAR, NT>();
         if (whole) return prefix | ~mask;
     }
     return prefix;
 }
 
-// Cuts the buffer back to its k smallest keys (in no particular order); returns the bound, i.e.
-// the largest key kept.  count > k on entry; on exit misc[0] == k.
-template <int NT, int CAP>
-__device__ __forceinline__ uint64_t pq_cut_buffer(uint64_t* buf, int count, int k, int* hist, int* misc) {
-    const uint64_t bound = pq_select_bound([buf](int i) { return buf[i]; }, count, k, hist, misc);
+// Cuts the buffer (capacity CAP) back to its k smallest keys (in no particular order); returns the
+// bound, i.e. the largest key kept.  count > k on entry; on exit misc[0] == k.
+template <int BAR, int NT, int CAP>
+__device__ __forceinline__ uint64_t pq_cut_buffer(uint64_t* buf, int count, int k, int* hist, int* misc, int tid) {
+    const uint64_t bound = pq_select_bound<BAR, NT>([buf](int i) { return buf[i]; }, count, k, hist, misc, tid);
     constexpr int kPer = CAP / NT;
     static_assert(CAP % NT == 0, "buffer capacity must be a multiple of the thread count");
     uint64_t mine[kPer];
 #pragma unroll
     for (int q = 0; q < kPer; ++q) {
-        const int i = threadIdx.x + q * NT;
+        const int i = tid + q * NT;
         mine[q] = i < count ? buf[i] : ~0ull;
     }
-    if (threadIdx.x == 0) misc[0] = 0;
-    __syncthreads();
+    if (tid == 0) misc[0] = 0;
+    pq_group_sync<BAR, NT>();
 #pragma unroll
     for (int q = 0; q < kPer; ++q)
         if (mine[q] <= bound && mine[q] != ~0ull) buf[atomicAdd(&misc[0], 1)] = mine[q];
-    __syncthreads();
+    pq_group_sync<BAR, NT>();
     return bound;
 }
 
@@ -426,7 +431,7 @@ struct PqScanParams {
     int d, pq_m, nlist, nprobe, n_rerank;
     int ngroups;             // groups per query
     const float* centroids;
-    const float* cbt;        // transposed codebook [d][256] in global memory
+    const float* cbt;        // transposed codebook [d][256] in global memory (read through L1, or copied to shared memory)
     const int32_t* probes;
     const long long* offsets;
     const uint8_t* codes;
@@ -435,6 +440,50 @@ struct PqScanParams {
     int* gcand_count;        // [nq * ngroups]
     int* status;
 };
+
+// Working set of one scanning team (kPqScanThreads threads) in shared memory.  r and hist share a
+// region: the residual is dead once the table is built, the histogram lives only inside a buffer cut.
+struct PqTeamSmem {
+    float* lut;            // [pq_m][256]
+    float* r;              // [d], d <= 256
+    uint64_t* buf;         // [kPqScanBufKeys]
+    int* hist;             // [256]
+    int* misc;             // [16]
+    uint32_t* list_begin;  // [maxp] first position of each probed list
+    int* list_len;         // [maxp]
+    int* list_id;          // [maxp]
+    int* cs;               // [maxp + 1] chunk prefix of the query
+};
+__host__ __device__ inline size_t pq_team_bytes(int pq_m, int maxp) {
+    return static_cast<size_t>(pq_m) * kPqK * 4 + static_cast<size_t>(kPqScanBufKeys) * 8 + 1024 + 64 +
+           static_cast<size_t>(maxp) * 12 + ((static_cast<size_t>(maxp) + 1) * 4 + 15) / 16 * 16;
+}
+__device__ __forceinline__ PqTeamSmem pq_team_carve(uint8_t* raw, int pq_m, int maxp) {
+    PqTeamSmem s;
+    s.buf = reinterpret_cast<uint64_t*>(raw);
+    raw += static_cast<size_t>(kPqScanBufKeys) * 8;
+    s.lut = reinterpret_cast<float*>(raw);
+    raw += static_cast<size_t>(pq_m) * kPqK * 4;
+    s.hist = reinterpret_cast<int*>(raw);
+    s.r = reinterpret_cast<float*>(raw);
+    raw += 1024;
+    s.misc = reinterpret_cast<int*>(raw);
+    raw += 64;
+    s.list_begin = reinterpret_cast<uint32_t*>(raw);
+    raw += static_cast<size_t>(maxp) * 4;
+    s.list_len = reinterpret_cast<int*>(raw);
+    raw += static_cast<size_t>(maxp) * 4;
+    s.list_id = reinterpret_cast<int*>(raw);
+    raw += static_cast<size_t>(maxp) * 4;
+    s.cs = reinterpret_cast<int*>(raw);
+    return s;
+}
+// shared memory of the two scan kernels
+__host__ __device__ inline size_t pq_scan_smem_bytes(int d, int pq_m) { return pq_team_bytes(pq_m, kPqMaxProbes); }
+constexpr int kPqTeamProbes = 256;  // probes per query that the two-team kernel stages
+__host__ __device__ inline size_t pq_teams_smem_bytes(int d, int pq_m) {
+    return static_cast<size_t>(d) * kPqK * 4 + 2 * pq_team_bytes(pq_m, kPqTeamProbes);
+}
 
 // The code bytes of one stored vector, held in registers so that the next chunk's bytes can be
 // fetched while the current chunk is being scored (sub-code counts that are a multiple of 16, up
@@ -506,24 +555,27 @@ __device__ __forceinline__ float pq_adc_code(const float* lut, const uint8_t* co
     return acc;
 }
 
-__global__ void __launch_bounds__(kPqScanThreads, 2) pq_scan_kernel(const PqScanParams p) {
-    extern __shared__ __align__(16) uint8_t pq_smem_raw[];
-    const PqSmem s = pq_carve(pq_smem_raw, p.d, p.pq_m, false, kPqScanBufKeys);
+// The groups g_first, g_first + g_step, ... scanned by one team: thread tid of kPqScanThreads,
+// synchronising on barrier BAR.  kGlobalCb: cbt is the transposed codebook in global memory (read
+// through L1), otherwise the copy in shared memory.
+template <bool kGlobalCb, int BAR>
+__device__ __forceinline__ void pq_scan_groups(const PqScanParams& p, const PqTeamSmem& s, const float* cbt,
+                                               int64_t g_first, int64_t g_step, int tid) {
+    constexpr int NT = kPqScanThreads;
     const int dsub = p.d / p.pq_m;
     const int64_t total_groups = p.nq * p.ngroups;
-    if (static_cast<int64_t>(blockIdx.x) >= total_groups) return;
-    const int lane = threadIdx.x & 31;
+    const int lane = tid & 31;
     const uint32_t lt_mask = (1u << lane) - 1u;
     const bool in_regs = pq_codes_in_regs(p.pq_m);
     const uint32_t lut_s = static_cast<uint32_t>(__cvta_generic_to_shared(s.lut));
 
-    for (int64_t g = blockIdx.x; g < total_groups; g += gridDim.x) {
+    for (int64_t g = g_first; g < total_groups; g += g_step) {
         const int64_t b = g / p.ngroups;
         const int gi = static_cast<int>(g - b * p.ngroups);
         const int* cs_g = p.chunk_start + static_cast<size_t>(b) * (p.nprobe + 1);
-        __syncthreads();  // the previous group's descriptors, table and buffer are no longer in use
+        pq_group_sync<BAR, NT>();  // the previous group's descriptors, table and buffer are no longer in use
         // the query's probe descriptors, once per group: chunk prefix, list begin, list length
-        for (int pr = threadIdx.x; pr <= p.nprobe; pr += blockDim.x) {
+        for (int pr = tid; pr <= p.nprobe; pr += NT) {
             s.cs[pr] = cs_g[pr];
             if (pr < p.nprobe) {
                 const int l = p.probes[static_cast<size_t>(b) * p.nprobe + pr];
@@ -533,12 +585,12 @@ __global__ void __launch_bounds__(kPqScanThreads, 2) pq_scan_kernel(const PqScan
                     len = p.offsets[l + 1] - begin;
                 }
                 s.list_id[pr] = l;
-                s.list_begin[pr] = begin;
-                s.list_len[pr] = len;
+                s.list_begin[pr] = static_cast<uint32_t>(begin);
+                s.list_len[pr] = static_cast<int>(len < 0 ? 0 : (len > 0x7fffffffLL ? 0x7fffffffLL : len));
             }
         }
-        if (threadIdx.x == 0) s.misc[0] = 0;
-        __syncthreads();
+        if (tid == 0) s.misc[0] = 0;
+        pq_group_sync<BAR, NT>();
         const int nchunks = s.cs[p.nprobe];
         const int group_chunks = (nchunks + p.ngroups - 1) / p.ngroups;
         const int chunk0 = min(nchunks, gi * group_chunks);
@@ -555,9 +607,9 @@ __global__ void __launch_bounds__(kPqScanThreads, 2) pq_scan_kernel(const PqScan
                 }
             }
             float qv = 0.0f, cnext = 0.0f;  // thread t < d: its query coordinate, the coming list's centroid coordinate
-            if (threadIdx.x < p.d) {
-                qv = pq_elem(p.q, p.q_type, b * p.d + threadIdx.x);
-                cnext = p.centroids[static_cast<int64_t>(s.list_id[pr]) * p.d + threadIdx.x];
+            if (tid < p.d) {
+                qv = pq_elem(p.q, p.q_type, b * p.d + tid);
+                cnext = p.centroids[static_cast<int64_t>(s.list_id[pr]) * p.d + tid];
             }
             int built = -1;
             // the code of the first chunk
@@ -565,24 +617,24 @@ __global__ void __launch_bounds__(kPqScanThreads, 2) pq_scan_kernel(const PqScan
             nxt.w[0] = nxt.w[1] = make_uint4(0, 0, 0, 0);
             long long nxt_pos = -1;
             {
-                const long long in_list = static_cast<long long>(chunk0 - s.cs[pr]) * kPqChunk + threadIdx.x;
-                if (in_list < s.list_len[pr]) nxt_pos = s.list_begin[pr] + in_list;
+                const int in_list = (chunk0 - s.cs[pr]) * kPqChunk + tid;
+                if (in_list < s.list_len[pr]) nxt_pos = static_cast<long long>(s.list_begin[pr]) + in_list;
                 if (in_regs && nxt_pos >= 0) pq_fetch_code(nxt, p.codes + nxt_pos * p.pq_m, p.pq_m);
             }
             int npr = pr;  // owner of the chunk whose code is in `nxt`
             for (int ch = chunk0; ch < chunk1; ++ch) {
                 pr = npr;
                 if (pr != built) {
-                    __syncthreads();  // the previous table is no longer read
-                    if (threadIdx.x < p.d) s.r[threadIdx.x] = __fsub_rn(qv, cnext);
+                    pq_group_sync<BAR, NT>();  // the previous table is no longer read (nor the histogram, which r overlays)
+                    if (tid < p.d) s.r[tid] = __fsub_rn(qv, cnext);
                     // fetch the centroid of the next list that owns a chunk of this group
                     int later = pr + 1;
                     while (later < p.nprobe && s.cs[later + 1] == s.cs[later]) ++later;
-                    if (later < p.nprobe && s.cs[later] < chunk1 && threadIdx.x < p.d)
-                        cnext = p.centroids[static_cast<int64_t>(s.list_id[later]) * p.d + threadIdx.x];
-                    __syncthreads();
-                    pq_build_lut<true>(s.r, p.cbt, s.lut, p.pq_m, dsub);
-                    __syncthreads();
+                    if (later < p.nprobe && s.cs[later] < chunk1 && tid < p.d)
+                        cnext = p.centroids[static_cast<int64_t>(s.list_id[later]) * p.d + tid];
+                    pq_group_sync<BAR, NT>();
+                    pq_build_lut<kGlobalCb>(s.r, cbt, s.lut, p.pq_m, dsub, tid, NT);
+                    pq_group_sync<BAR, NT>();
                     built = pr;
                 }
                 const long long pos = nxt_pos;
@@ -591,8 +643,8 @@ __global__ void __launch_bounds__(kPqScanThreads, 2) pq_scan_kernel(const PqScan
                 nxt_pos = -1;
                 if (ch + 1 < chunk1) {
                     while (s.cs[npr + 1] <= ch + 1) ++npr;
-                    const long long in_list = static_cast<long long>(ch + 1 - s.cs[npr]) * kPqChunk + threadIdx.x;
-                    if (in_list < s.list_len[npr]) nxt_pos = s.list_begin[npr] + in_list;
+                    const int in_list = (ch + 1 - s.cs[npr]) * kPqChunk + tid;
+                    if (in_list < s.list_len[npr]) nxt_pos = static_cast<long long>(s.list_begin[npr]) + in_list;
                     if (in_regs && nxt_pos >= 0) pq_fetch_code(nxt, p.codes + nxt_pos * p.pq_m, p.pq_m);
                 }
                 bool hit = false;
@@ -610,22 +662,52 @@ __global__ void __launch_bounds__(kPqScanThreads, 2) pq_scan_kernel(const PqScan
                     base = __shfl_sync(0xFFFFFFFFu, base, 0);
                     if (hit) s.buf[base + __popc(bal & lt_mask)] = key;
                 }
-                __syncthreads();
+                pq_group_sync<BAR, NT>();
                 const int count = s.misc[0];
                 if (count > kPqScanBufKeys - kPqChunk)
-                    bound = pq_cut_buffer<kPqScanThreads, kPqScanBufKeys>(s.buf, count, p.n_rerank, s.hist, s.misc);
+                    bound = pq_cut_buffer<BAR, NT, kPqScanBufKeys>(s.buf, count, p.n_rerank, s.hist, s.misc, tid);
             }
         }
-        __syncthreads();
+        pq_group_sync<BAR, NT>();
         int count = s.misc[0];
         if (count > p.n_rerank) {
-            pq_cut_buffer<kPqScanThreads, kPqScanBufKeys>(s.buf, count, p.n_rerank, s.hist, s.misc);
+            pq_cut_buffer<BAR, NT, kPqScanBufKeys>(s.buf, count, p.n_rerank, s.hist, s.misc, tid);
             count = p.n_rerank;
         }
         uint64_t* out = p.gcand + static_cast<size_t>(g) * p.n_rerank;
-        for (int i = threadIdx.x; i < count; i += blockDim.x) out[i] = s.buf[i];
-        if (threadIdx.x == 0) p.gcand_count[g] = count;
+        for (int i = tid; i < count; i += NT) out[i] = s.buf[i];
+        if (tid == 0) p.gcand_count[g] = count;
     }
+}
+
+// One team per CTA, two CTAs per SM; the codebook is read through L1 from its transposed copy.
+// Serves every shape (up to kPqMaxProbes probes) with little shared memory.
+__global__ void __launch_bounds__(kPqScanThreads, 2) pq_scan_kernel(const PqScanParams p) {
+    extern __shared__ __align__(16) uint8_t pq_smem_raw[];
+    if (static_cast<int64_t>(blockIdx.x) >= p.nq * p.ngroups) return;
+    const PqTeamSmem s = pq_team_carve(pq_smem_raw, p.pq_m, kPqMaxProbes);
+    pq_scan_groups<true, 0>(p, s, p.cbt, blockIdx.x, gridDim.x, threadIdx.x);
+}
+
+// Two teams per CTA, one CTA per SM: both teams read the codebook from one transposed copy in shared
+// memory and otherwise work on different groups with their own table, buffer and barrier, so one
+// team's table build (arithmetic) runs under the other's scan (shared-memory lookups).
+__global__ void __launch_bounds__(2 * kPqScanThreads, 1) pq_scan_teams_kernel(const PqScanParams p) {
+    extern __shared__ __align__(16) uint8_t pq_smem_raw[];
+    if (2 * static_cast<int64_t>(blockIdx.x) >= p.nq * p.ngroups) return;
+    float* cbt = reinterpret_cast<float*>(pq_smem_raw);
+    {   // straight copy of the transposed codebook (d * 256 floats, 16-byte pieces)
+        const float4* src = reinterpret_cast<const float4*>(p.cbt);
+        float4* dst = reinterpret_cast<float4*>(cbt);
+        for (int i = threadIdx.x; i < p.d * (kPqK / 4); i += blockDim.x) dst[i] = __ldg(src + i);
+    }
+    __syncthreads();
+    uint8_t* teams = pq_smem_raw + static_cast<size_t>(p.d) * kPqK * 4;
+    const int team = threadIdx.x / kPqScanThreads;
+    const int tid = threadIdx.x - team * kPqScanThreads;
+    const PqTeamSmem s = pq_team_carve(teams + team * pq_team_bytes(p.pq_m, kPqTeamProbes), p.pq_m, kPqTeamProbes);
+    if (team == 0) pq_scan_groups<false, 1>(p, s, cbt, 2 * static_cast<int64_t>(blockIdx.x), 2 * static_cast<int64_t>(gridDim.x), tid);
+    else pq_scan_groups<false, 2>(p, s, cbt, 2 * static_cast<int64_t>(blockIdx.x) + 1, 2 * static_cast<int64_t>(gridDim.x), tid);
 }
 
 // ------------------------------------------------------------------ group -> query merge
@@ -643,7 +725,12 @@ struct PqMergeParams {
 // One CTA per query.  The n_rerank smallest of the query's group candidates are selected (in shared
 // memory when they all fit, else by a radix select over the group outputs in place), sorted, and
 // written in ascending (estimate, position) order.
-__global__ void __launch_bounds__(kPqThreads) pq_merge_kernel(const PqMergeParams p) {
+// kRegs: the variant for group outputs of more than kPqBufKeys and at most 16 keys per thread, which
+// holds them in registers during the selection (one CTA per SM); the other variant keeps two CTAs
+// per SM for large batches.
+constexpr int kPqMergeRegKeys = 16;
+template <bool kRegs>
+__global__ void __launch_bounds__(kPqThreads, kRegs ? 1 : 2) pq_merge_kernel(const PqMergeParams p) {
     __shared__ uint64_t buf[kPqBufKeys];
     __shared__ int hist[256];
     __shared__ int misc[16];
@@ -657,15 +744,15 @@ __global__ void __launch_bounds__(kPqThreads) pq_merge_kernel(const PqMergeParam
     };
     if (threadIdx.x == 0) misc[4] = 0;
     __syncthreads();
-    int mine = 0;
-    for (int g = threadIdx.x; g < p.ngroups; g += blockDim.x) mine += cnt[g];
-    if (mine) atomicAdd(&misc[4], mine);
+    int own = 0;
+    for (int g = threadIdx.x; g < p.ngroups; g += blockDim.x) own += cnt[g];
+    if (own) atomicAdd(&misc[4], own);
     __syncthreads();
     const int total = misc[4];
     if (threadIdx.x == 0) misc[0] = 0;
     __syncthreads();
-    constexpr int kRegKeys = 16;
-    if (slots <= kRegKeys * kPqThreads) {
+    constexpr int kRegKeys = kPqMergeRegKeys;
+    if constexpr (kRegs) {
         // every slot is read once into registers; selection and gathering work from there
         uint64_t mine[kRegKeys];
 #pragma unroll
@@ -675,7 +762,7 @@ __global__ void __launch_bounds__(kPqThreads) pq_merge_kernel(const PqMergeParam
         }
         uint64_t bound = ~0ull;
         if (total > kPqBufKeys) {
-            bound = pq_select_bound_regs<kRegKeys>(mine, p.n_rerank, hist, misc);
+            bound = pq_select_bound_regs<0, kPqThreads, kRegKeys>(mine, p.n_rerank, hist, misc, threadIdx.x);
             if (threadIdx.x == 0) misc[0] = 0;
             __syncthreads();
         }
@@ -685,7 +772,7 @@ __global__ void __launch_bounds__(kPqThreads) pq_merge_kernel(const PqMergeParam
     } else {
         uint64_t bound = ~0ull;
         if (total > kPqBufKeys) {
-            bound = pq_select_bound(get, slots, p.n_rerank, hist, misc);
+            bound = pq_select_bound<0, kPqThreads>(get, slots, p.n_rerank, hist, misc, threadIdx.x);
             if (threadIdx.x == 0) misc[0] = 0;
             __syncthreads();
         }
@@ -698,7 +785,7 @@ __global__ void __launch_bounds__(kPqThreads) pq_merge_kernel(const PqMergeParam
     int count = misc[0];
     if (count > p.n_rerank) {
         __syncthreads();
-        pq_cut_buffer<kPqThreads, kPqBufKeys>(buf, count, p.n_rerank, hist, misc);
+        pq_cut_buffer<0, kPqThreads, kPqBufKeys>(buf, count, p.n_rerank, hist, misc, threadIdx.x);
         count = p.n_rerank;
     }
     int m = 2;

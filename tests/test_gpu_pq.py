@@ -92,7 +92,7 @@ def test_long_lists_many_buffer_cuts_and_ties(n_rerank):
     _check_search(q, c, cb, offsets, codes, probes, n_rerank)
 
 
-@pytest.mark.parametrize("groups", [1, 2, 7, 256])
+@pytest.mark.parametrize("groups", [1, 2, 7, 256, -2, -8])  # negative: the scan kernel that reads the codebook through L1
 def test_every_group_count_gives_the_same_result(groups):
     # the chunks of a query are dealt to `groups` CTAs whose survivors the query merge combines:
     # in shared memory when they fit, by a select over the group outputs when they do not
