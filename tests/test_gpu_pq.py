@@ -180,3 +180,15 @@ def test_full_size_batch_in_the_measured_configuration(dtype, d, pq_m):
     B.ivf_check()
     assert (got_codes.cpu().numpy() == want_codes).all()
     _check_search(q, c, cb, offsets, want_codes, probes, n_rerank)
+
+
+@pytest.mark.parametrize("nprobe", [257, 512])
+def test_many_probes_take_the_single_team_kernel(nprobe):
+    # more than 256 probes per query do not fit the two-team kernel's descriptor tables; 512 is the
+    # largest probe count of the paper's sweep and of this library
+    q, c, cb, ids, offsets, x, probes = _problem(9, 30000, 600, 64, 16, "f32", 5, nprobe, sigma=1.0)
+    codes = O.pq_encode(x, ids, c, cb)
+    _check_search(q, c, cb, offsets, codes, probes, 300)
+    with pytest.raises(B.IvfError) as e:
+        B.ivf_pq_search(_t(q), _t(c), _t(np.tile(probes, (1, 2))[:, :513].copy()), _t(offsets), _t(codes), _t(cb), 8)
+    assert e.value.code in (B.IVF_ERR_UNSUPPORTED, B.IVF_ERR_INVALID_ARG)
