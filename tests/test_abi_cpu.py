@@ -104,3 +104,35 @@ def test_threshold_rule_selection():
     assert binding.ivf_debug_rule(256, 1 << 20) == (1, 64)
     assert binding.ivf_debug_rule(512, 600)[0] == 2               # sample too small: bounded logs
     assert binding.ivf_debug_rule(17, 2044)[0] == 2 and binding.ivf_debug_rule(17, 2045) == (1, 4)
+
+
+def test_pq_and_candidate_entry_points_check_arguments_first():
+    L = binding.lib()
+    i64, i32, vp = ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p
+    L.ivf_pq_encode.argtypes = [vp, i64, i32, i32, vp, vp, i32, vp, i32, vp, vp]
+    L.ivf_pq_search.argtypes = [vp, i64, i32, i32, vp, i32, vp, i32, vp, vp, i64, vp, i32, i32, vp, vp, vp, vp, vp]
+    L.ivf_assign_candidates.argtypes = [vp, i64, i32, i32, vp, i32, vp, i32, vp, vp, vp]
+    buf = (ctypes.c_char * 4096)()
+    p = (ctypes.addressof(buf) + 255) & ~255
+    UNS, INV, OK = binding.IVF_ERR_UNSUPPORTED, binding.IVF_ERR_INVALID_ARG, binding.IVF_OK
+    # encode: pq_m must divide d; the codebook must fit shared memory; empty input is fine
+    assert L.ivf_pq_encode(p, 4, 128, 0, p, p, 10, p, 24, p, None) == INV
+    assert L.ivf_pq_encode(p, 4, 256, 0, p, p, 10, p, 64, p, None) == UNS
+    assert L.ivf_pq_encode(p, 4, 128, 5, p, p, 10, p, 32, p, None) == INV           # dtype
+    assert L.ivf_pq_encode(None, 0, 128, 0, None, None, 10, p, 32, None, None) == OK
+    # search: probe count, N_rerank, position width, alignment of the code array
+    def search(nq=4, d=128, qt=1, nlist=100, nprobe=8, n_codes=1000, pq_m=32, n_rerank=64, codes=p, q=p):
+        return L.ivf_pq_search(q, nq, d, qt, p, nlist, p, nprobe, p, codes, n_codes, p, pq_m, n_rerank, None, p, p, None, None)
+    assert search(nprobe=0) == INV and search(nprobe=101) == INV
+    assert search(nlist=1000, nprobe=513) == UNS
+    assert search(n_rerank=0) == UNS and search(n_rerank=1025) == UNS
+    assert search(n_codes=1 << 32) == UNS
+    assert search(pq_m=48) == INV
+    assert search(codes=p + 8) == INV
+    assert search(nq=-1) == INV
+    assert search(nq=0, q=None) == OK
+    # candidates: d a multiple of 4 up to 256, at least one candidate per row
+    assert L.ivf_assign_candidates(p, 4, 130, 0, p, 10, p, 8, p, None, None) == UNS
+    assert L.ivf_assign_candidates(p, 4, 128, 0, p, 10, p, 0, p, None, None) == INV
+    assert L.ivf_assign_candidates(p, 4, 128, 0, None, 10, p, 8, p, None, None) == INV
+    assert L.ivf_assign_candidates(None, 0, 128, 0, None, 10, None, 8, None, None, None) == OK
