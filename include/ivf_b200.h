@@ -184,7 +184,9 @@ int64_t ivf_launch_count(void);
  *                    with `num_sms` SMs: writes {row_groups, col_tiles, ctas, max_partials_per_row,
  *                    block_n, k_slices, stages, smem_bytes, row tiles of 128 points per row group}
  *                    to out[9].
- *   ivf_debug_span   first unit and one-past-last unit of CTA `cta` in that schedule.
+ *   ivf_debug_span   out[0], out[1]: first unit and one-past-last unit of CTA `cta` in that schedule;
+ *                    out[2], out[3]: the CTA that the kernels' unit-to-CTA mapping gives for the first and
+ *                    the last unit of the span (both must equal `cta`).
  *   ivf_debug_set_wait_limit_ns   time limit of every device-side wait (0 restores the default
  *                    of 2 s).
  *   ivf_debug_wait_probe   launches a one-warp kernel that waits, with the library's bounded wait,
@@ -192,7 +194,7 @@ int64_t ivf_launch_count(void);
  *                    IVF_ERR_DEVICE_TIMEOUT (wait site 99) in the status word and returns normally.
  */
 int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[9]);
-int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int64_t out[2]);
+int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int64_t out[4]);
 int ivf_debug_set_wait_limit_ns(int64_t ns);
 int ivf_debug_wait_probe(void* stream);
 /* Test hook: when on, the merge of a k > 1 call declares every row's candidate set insufficient, so
@@ -225,6 +227,10 @@ int ivf_debug_stats(int enable, int64_t out[3]);
  * A negative value -(g + 1) asks for g groups and for the scan kernel variant that reads the codebook
  * through L1 (otherwise the two-team shared-memory variant is used whenever it fits). */
 int ivf_debug_set_pq_groups(int groups);
+/* Test hook: the cost, in units of one (row group, centroid tile) step, that the persistent schedule
+ * charges a CTA for changing row group in the middle of its span (0 = equal unit counts; negative =
+ * the default: 8 for the k = 1 kernel, 4 otherwise). */
+int ivf_debug_set_crossing_cost(int units);
 /* Test hook: mask of the kernel families of the routing path that may start while their predecessor
  * drains (programmatic dependent launch): 1 operand preparation, 2 fused kernel, 4 threshold merge,
  * 8 merge, 16 merge of passed-on rows, 32 recomputation.  0 = ordinary stream launches; default 57. */

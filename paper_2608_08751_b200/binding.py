@@ -26,7 +26,7 @@ EXPORTS = (
     "ivf_pq_encode", "ivf_pq_search", "ivf_assign_candidates",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
     "ivf_debug_plan", "ivf_debug_span", "ivf_debug_set_wait_limit_ns",
-    "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_set_row_chunk", "ivf_debug_stats", "ivf_debug_set_pq_groups", "ivf_debug_set_dependent_launch",
+    "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_set_row_chunk", "ivf_debug_stats", "ivf_debug_set_pq_groups", "ivf_debug_set_dependent_launch", "ivf_debug_set_crossing_cost",
 )
 
 _lib = None
@@ -78,6 +78,7 @@ def lib() -> ctypes.CDLL:
     L.ivf_pq_encode.argtypes = [vp, i64, i32, i32, vp, vp, i32, vp, i32, vp, vp]
     L.ivf_pq_search.argtypes = [vp, i64, i32, i32, vp, i32, vp, i32, vp, vp, i64, vp, i32, i32, vp, vp, vp, vp, vp]
     L.ivf_debug_set_pq_groups.argtypes = [i32]
+    L.ivf_debug_set_crossing_cost.argtypes = [i32]
     L.ivf_debug_set_dependent_launch.argtypes = [i32]
     L.ivf_debug_timing_read.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
     for name in EXPORTS:
@@ -426,10 +427,12 @@ def ivf_debug_plan(n: int, nlist: int, d: int, k: int, num_sms: int = 148) -> di
 
 
 def ivf_debug_span(n: int, nlist: int, d: int, k: int, num_sms: int, cta: int):
-    out = (ctypes.c_int64 * 2)()
+    out = (ctypes.c_int64 * 4)()
     rc = lib().ivf_debug_span(n, nlist, d, k, num_sms, cta, out)
     if rc != IVF_OK:
         _raise(rc)
+    if int(out[2]) != cta or int(out[3]) != cta:
+        raise AssertionError(f"unit-to-CTA mapping disagrees with the span of CTA {cta}: {list(out)}")
     return int(out[0]), int(out[1])
 
 
@@ -439,6 +442,10 @@ def ivf_debug_set_wait_limit_ns(ns: int) -> None:
 
 TIMING_FAMILIES = ("prep", "fused_argmin", "fused_topk", "merge", "update", "threshold_pass",
                    "pq_encode", "pq_scan", "pq_merge")
+
+
+def ivf_debug_set_crossing_cost(units: int) -> None:
+    lib().ivf_debug_set_crossing_cost(int(units))
 
 
 def ivf_debug_set_dependent_launch(on: bool) -> None:

@@ -73,6 +73,7 @@ struct FusedParams {
     int nstage;           // centroid-tile ring depth
     int col_tiles;        // centroid tiles per sweep
     int64_t total_units;  // row groups * col_tiles
+    int cross;            // cost of a mid-span row-group crossing in units (span partition)
     int partials;         // partial-result slots per row (CTAs sharing a row tile x kEpiHalves)
     int cap;              // candidate-log capacity per (row, slot), k > 1 only
     int rule;             // k > 1: TAU_RUNNING, TAU_GIVEN or TAU_BOUNDED
@@ -94,9 +95,26 @@ struct FusedParams {
 };
 
 // ---- persistent schedule: CTA b of G owns units [T*b/G, T*(b+1)/G) of the row-major unit grid
-__host__ __device__ inline int64_t span_begin(int64_t T, int G, int b) { return (T * b) / G; }
-__host__ __device__ inline int cta_of_unit(int64_t T, int G, int64_t u) {
-    return static_cast<int>(((u + 1) * G - 1) / T);
+// The T = R * NT units are dealt to G CTAs by cost, not by count: a CTA that crosses from one row
+// group to the next in mid-span idles its tensor core while the last accumulators are read and the
+// next point tile is fetched, which costs about as much as `cross` units.  In cost space every row
+// group is a block of `cross` cost units followed by its NT unit slots; CTA b starts at cost
+// C * b / G (C = R * (NT + cross)), and a start that falls inside a crossing block is moved to the row
+// group's first unit.  cross = 0 is the plain equal-count split.
+__host__ __device__ inline int64_t span_begin(int64_t T, int G, int NT, int cross, int b) {
+    const int64_t w = NT + cross;
+    const int64_t C = (T / NT) * w;
+    const int64_t c = (C * b) / G;
+    const int64_t r = c / w, o = c - r * w;
+    return r * NT + (o > cross ? o - cross : 0);
+}
+// the CTA whose span holds unit u: the largest b with span_begin(b) <= u
+__host__ __device__ inline int cta_of_unit(int64_t T, int G, int NT, int cross, int64_t u) {
+    const int64_t w = NT + cross;
+    const int64_t C = (T / NT) * w;
+    const int64_t r = u / NT;
+    const int64_t cu = r * w + cross + (u - r * NT);  // cost coordinate of the unit's slot
+    return static_cast<int>(((cu + 1) * G - 1) / C);
 }
 
 __host__ __device__ inline size_t fused_smem_bytes(int kslices, int block_n, int nstage, int mtiles) {
@@ -475,8 +493,8 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     const int b = blockIdx.x;
     const int64_t T = p.total_units;
     const int NT = p.col_tiles;
-    const int64_t u0 = span_begin(T, G, b);
-    const int64_t u1 = span_begin(T, G, b + 1);
+    const int64_t u0 = span_begin(T, G, NT, p.cross, b);
+    const int64_t u1 = span_begin(T, G, NT, p.cross, b + 1);
 
     if (threadIdx.x == 0) {
         mbar_init(a_full, p.x_raw != nullptr ? 4 * MT : 1);  // TMA bytes, or one arrival per widening warp
@@ -658,7 +676,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             const int64_t r = u / NT;  // row group
             const int t0 = static_cast<int>(u - r * NT);
             const int t1 = static_cast<int>((u1 - r * NT < NT) ? (u1 - r * NT) : NT);
-            const int slot = (b - cta_of_unit(T, G, r * NT)) * kEpiHalves + half;
+            const int slot = (b - cta_of_unit(T, G, NT, p.cross, r * NT)) * kEpiHalves + half;
 
             if (p.x_raw != nullptr && half < MT) {
                 // uint8 points: this thread widens its own row of point tile `half`.  The tile is free:

@@ -216,6 +216,7 @@ struct Plan {
     int64_t row_tiles;  // row groups of mtiles * 128 points
     int col_tiles;
     int64_t total_units;
+    int cross;  // crossing cost of the span partition, in units
     int ctas;
     int partials;    // slots per row: CTAs that can share a row tile x epilogue halves
     int cap;
@@ -244,6 +245,8 @@ int choose_rule(int k, int nlist, int* stride) {
     return k <= kSampleM ? TAU_RUNNING : TAU_BOUNDED;
 }
 
+int g_cross = -1;  // crossing cost used by the span partition; -1 = by kernel variant (test hook: ivf_debug_set_crossing_cost)
+
 int make_plan(int64_t n, int nlist, int d, int k, int num_sms, Plan* pl, bool one_row_tile = false) {
     pl->kd = (d + 63) / 64 * 64;
     pl->kp = pl->kd + kAugK;
@@ -264,7 +267,17 @@ int make_plan(int64_t n, int nlist, int d, int k, int num_sms, Plan* pl, bool on
     pl->col_tiles = (nlist + pl->block_n - 1) / pl->block_n;
     pl->total_units = pl->row_tiles * pl->col_tiles;
     pl->ctas = static_cast<int>(pl->total_units < num_sms ? pl->total_units : num_sms);
-    const int64_t lmin = pl->total_units / pl->ctas;
+    // a CTA that changes row group in mid-span loses about g_cross units of time; charge it in the
+    // partition when spans are long enough for that to be a correction (and there is more than one
+    // row group to cross into)
+    // measured: 8 units for the k = 1 kernel (10,240 rows: 163 -> 153 us), about 4 for the others
+    int cross = pl->row_tiles > 1 ? (g_cross >= 0 ? g_cross : (k == 1 ? 8 : 4)) : 0;
+    const int64_t per_cta = pl->total_units / pl->ctas;
+    if (cross > per_cta / 4) cross = static_cast<int>(per_cta / 4);
+    if (cross > pl->col_tiles / 2) cross = pl->col_tiles / 2;
+    pl->cross = cross;
+    int64_t lmin = (pl->row_tiles * static_cast<int64_t>(pl->col_tiles + cross)) / pl->ctas - cross;  // shortest span
+    if (lmin < 1) lmin = 1;
     int64_t parts = (pl->col_tiles + lmin - 1) / lmin + 1;
     if (parts > pl->ctas) parts = pl->ctas;
     pl->partials = static_cast<int>(parts) * kEpiHalves;
@@ -446,6 +459,7 @@ int launch_fused(DeviceCtx& ctx, const Plan& pl, int64_t n, int nlist, int k, in
     fp.nstage = pl.nstage;
     fp.col_tiles = pl.col_tiles;
     fp.total_units = pl.total_units;
+    fp.cross = pl.cross;
     fp.partials = pl.partials;
     fp.cap = pl.cap;
     fp.rule = rule;
@@ -498,6 +512,7 @@ MergeParams merge_params(const Plan& pl, int64_t n, int k, const Entry* part, co
     mp.cap = pl.cap;
     mp.col_tiles = pl.col_tiles;
     mp.total_units = pl.total_units;
+    mp.cross = pl.cross;
     mp.ctas = pl.ctas;
     mp.group_rows = kBlockM * pl.mtiles;
     mp.part = part;
@@ -1242,15 +1257,18 @@ int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[
     return IVF_OK;
 }
 
-int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int64_t out[2]) {
+int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int64_t out[4]) {
     if (n < 1 || nlist < 1 || num_sms < 1 || !out) return fail(IVF_ERR_INVALID_ARG, "bad plan arguments");
     Plan pl;
     int stride = 1;
     int rc = make_plan(n, nlist, d, k, num_sms, &pl, k > 1 && choose_rule(k, nlist, &stride) != TAU_GIVEN);
     if (rc != IVF_OK) return rc;
     if (cta < 0 || cta >= pl.ctas) return fail(IVF_ERR_INVALID_ARG, "cta %d outside [0, %d)", cta, pl.ctas);
-    out[0] = span_begin(pl.total_units, pl.ctas, cta);
-    out[1] = span_begin(pl.total_units, pl.ctas, cta + 1);
+    out[0] = span_begin(pl.total_units, pl.ctas, pl.col_tiles, pl.cross, cta);
+    out[1] = span_begin(pl.total_units, pl.ctas, pl.col_tiles, pl.cross, cta + 1);
+    // the inverse mapping the kernels use to number a row group's partial slots
+    out[2] = cta_of_unit(pl.total_units, pl.ctas, pl.col_tiles, pl.cross, out[0]);
+    out[3] = cta_of_unit(pl.total_units, pl.ctas, pl.col_tiles, pl.cross, out[1] - 1);
     return IVF_OK;
 }
 
@@ -1315,6 +1333,11 @@ int ivf_debug_set_row_chunk(int64_t rows) {
 
 int ivf_debug_set_dependent_launch(int on) {
     g_pdl = on;
+    return IVF_OK;
+}
+
+int ivf_debug_set_crossing_cost(int units) {
+    g_cross = units;  // negative: chosen by kernel variant
     return IVF_OK;
 }
 

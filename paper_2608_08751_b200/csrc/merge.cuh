@@ -21,6 +21,7 @@ struct MergeParams {
     int cap;
     int col_tiles;
     int64_t total_units;
+    int cross;             // crossing cost of the fused kernel's span partition
     int ctas;              // grid size of the fused kernel (defines which slots exist)
     int group_rows;        // point rows per row group of the fused kernel (128 or 256)
     const Entry* part;
@@ -37,9 +38,9 @@ struct MergeParams {
     unsigned long long* stats;  // optional counters: [2] rows sent to the brute-force recomputation
 };
 
-__device__ __forceinline__ int slots_of_row_tile(int64_t total_units, int ctas, int col_tiles, int64_t r) {
-    const int first = cta_of_unit(total_units, ctas, r * col_tiles);
-    const int last = cta_of_unit(total_units, ctas, (r + 1) * col_tiles - 1);
+__device__ __forceinline__ int slots_of_row_tile(const MergeParams& p, int64_t r) {
+    const int first = cta_of_unit(p.total_units, p.ctas, p.col_tiles, p.cross, r * p.col_tiles);
+    const int last = cta_of_unit(p.total_units, p.ctas, p.col_tiles, p.cross, (r + 1) * p.col_tiles - 1);
     return (last - first + 1) * kEpiHalves;
 }
 
@@ -49,7 +50,7 @@ __global__ void merge_argmin_kernel(const MergeParams p) {
     pdl_trigger();
     const int64_t row = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (row >= p.n) return;
-    const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows);
+    const int ns = slots_of_row_tile(p, row / p.group_rows);
     const Entry* e = p.part + static_cast<size_t>(row) * p.partials;
     float bv = e[0].v;
     int bj = e[0].j;
@@ -125,7 +126,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_select_kernel(const Merge
     const int64_t nrows = p.big ? p.big[0] : p.n;
     for (int64_t item = blockIdx.x; item < nrows; item += gridDim.x) {
         const int64_t row = p.big ? p.big[1 + item] : item;
-        const int ns = min(slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows), kMaxSlots);
+        const int ns = min(slots_of_row_tile(p, row / p.group_rows), kMaxSlots);
         const Entry* base = p.part + static_cast<size_t>(row) * p.partials * p.cap;
         const int2* meta = p.part_meta + static_cast<size_t>(row) * p.partials;
         __syncthreads();  // the previous row of this CTA is finished with the shared arrays
@@ -349,7 +350,7 @@ __global__ void __launch_bounds__(32 * WARPS) merge_warp_kernel(const MergeParam
     if (row >= p.n) return;
     const uint32_t FULL = 0xFFFFFFFFu;
     const uint32_t lt_mask = (1u << lane) - 1u;
-    const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows);
+    const int ns = slots_of_row_tile(p, row / p.group_rows);
     const int2* meta = p.part_meta + static_cast<size_t>(row) * p.partials;
     bool pass_on = ns > kWarpSlots || p.force_fail;
 
@@ -519,7 +520,7 @@ __global__ void __launch_bounds__(kTauThreads) merge_tau_kernel(const MergeParam
     const float INF = __int_as_float(0x7f800000);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t row = blockIdx.x;
-    const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows);
+    const int ns = slots_of_row_tile(p, row / p.group_rows);
     const Entry* base = p.part + static_cast<size_t>(row) * p.partials * p.cap;
     if (threadIdx.x < kSampleM) lists[kTauThreads / 32][threadIdx.x] = INF;
     float result = INF;
@@ -554,7 +555,7 @@ __global__ void __launch_bounds__(256) merge_tau_warp_kernel(const MergeParams p
     const int lane = threadIdx.x & 31;
     const int64_t row = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
     if (row >= p.n) return;
-    const int ns = slots_of_row_tile(p.total_units, p.ctas, p.col_tiles, row / p.group_rows);
+    const int ns = slots_of_row_tile(p, row / p.group_rows);
     const Entry* base = p.part + static_cast<size_t>(row) * p.partials * p.cap;
     float v[kSampleM];
 #pragma unroll

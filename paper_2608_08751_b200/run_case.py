@@ -259,7 +259,10 @@ def main():
     ap.add_argument("--dtype", default="u8", choices=["u8", "f32", "i8"])
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--dependent-launch", type=int, default=-1, help="kernel-family mask of dependent launches (0 = none)")
+    ap.add_argument("--crossing-cost", type=int, default=-1, help="span-partition crossing cost in units (0 = equal counts)")
     args = ap.parse_args()
+    if args.crossing_cost >= 0:
+        B.ivf_debug_set_crossing_cost(args.crossing_cost)
     if args.dependent_launch >= 0:
         B.ivf_debug_set_dependent_launch(args.dependent_launch)
 

@@ -74,7 +74,16 @@ def test_argument_errors_come_before_any_cuda_call():
     (1 << 20, 65536, 128, 1, 148), (100000, 1 << 20, 96, 256, 148), (1, 1, 16, 1, 148),
     (5, 100000, 64, 8, 148), (129, 257, 256, 2, 148), (300, 1000, 192, 5, 7), (128 * 148, 256, 128, 1, 148),
 ])
-def test_schedule_covers_every_unit_once_and_bounds_partials(n, nlist, d, k, sms):
+@pytest.mark.parametrize("cross", [-1, 0, 3, 8, 40])
+def test_schedule_covers_every_unit_once_and_bounds_partials(n, nlist, d, k, sms, cross):
+    binding.ivf_debug_set_crossing_cost(cross)
+    try:
+        _check_schedule(n, nlist, d, k, sms)
+    finally:
+        binding.ivf_debug_set_crossing_cost(-1)
+
+
+def _check_schedule(n, nlist, d, k, sms):
     pl = binding.ivf_debug_plan(n, nlist, d, k, sms)
     T = pl["row_tiles"] * pl["col_tiles"]
     assert pl["mtiles"] in (1, 2)
