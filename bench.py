@@ -209,7 +209,7 @@ def pq_side_measurement(dev, pk, sm_max_mhz):
         "queries_per_s": nq / (both_ms / 1e3), "scan_ms": scan_ms, "merge_ms": merge_ms,
         "codes_scanned_per_batch": scanned, "codes_per_s": scanned / (scan_ms / 1e3),
         "code_bytes_GBps": scanned * pq_m / (scan_ms / 1e3) / 1e9, "launches_per_batch": int(launches),
-        "roofline": {"kernel": "pq_scan_kernel", "bound": "alu", "achieved": lookups / 1e12, "peak": peak / 1e12,
+        "roofline": {"kernel": "pq_scan_teams_kernel", "bound": "alu", "achieved": lookups / 1e12, "peak": peak / 1e12,
                      "unit": "T lookups/s", "frac": lookups / peak, "traffic": None,
                      "peak_source": "derived: 148 SMs x 32 shared-memory banks x max SM clock"},
     }
