@@ -752,6 +752,12 @@ int run_chunks(const void* points, int64_t n, int d, int ptype, const float* cen
     if (chunk_rows <= 0) chunk_rows = int64_t(1) << 20;
     if ((host || with_update) && rows > chunk_rows) rows = chunk_rows;
     if (rows > n) rows = n;
+    // host-resident input in fewer than four chunks: cut it in four, so that only a quarter of the
+    // copy is exposed before the first kernel can start (the rest runs under the kernels)
+    if (host && g_row_chunk_override.load() <= 0 && (n + rows - 1) / rows < 4 && n >= 4 * 65536) {
+        const int64_t quarter = ((n + 3) / 4 + 255) / 256 * 256;
+        if (quarter < rows) rows = quarter;
+    }
     const int64_t nchunks = (n + rows - 1) / rows;
 
     Plan pl0;
