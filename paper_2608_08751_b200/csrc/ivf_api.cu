@@ -763,17 +763,6 @@ int run_chunks(const void* points, int64_t n, int d, int ptype, const float* cen
     Plan pl0;
     rc = make_plan(rows, nlist, d, k, ctx.num_sms, &pl0);
     if (rc != IVF_OK) return rc;
-    CentroidPrep cp;
-    if (prepared) {
-        cp.c16 = prepared->c16;
-        cp.scal = prepared->scal;
-        cp.bits = prepared->bits;
-        rc = map_centroids(nlist, k, pl0, &cp);
-    } else {
-        rc = prepare_centroids(ctx, centroids, nlist, d, k, pl0, stream, &cp);
-    }
-    if (rc != IVF_OK) return rc;
-
     uint8_t* stage[2] = {nullptr, nullptr};
     int32_t* tmp_ids = nullptr;
     if (host) {
@@ -800,6 +789,17 @@ int run_chunks(const void* points, int64_t n, int d, int ptype, const float* cen
         rc = issue_copy(0);
         if (rc != IVF_OK) return rc;
     }
+    // the centroid preparation is enqueued after the first copy was issued, so the two overlap
+    CentroidPrep cp;
+    if (prepared) {
+        cp.c16 = prepared->c16;
+        cp.scal = prepared->scal;
+        cp.bits = prepared->bits;
+        rc = map_centroids(nlist, k, pl0, &cp);
+    } else {
+        rc = prepare_centroids(ctx, centroids, nlist, d, k, pl0, stream, &cp);
+    }
+    if (rc != IVF_OK) return rc;
     for (int64_t c = 0; c < nchunks; ++c) {
         const int64_t r0 = c * rows;
         const int64_t nr = (n - r0 < rows) ? (n - r0) : rows;
