@@ -1,0 +1,132 @@
+"""Seeded random sweeps over shapes, element types and k for every entry point, each case compared
+with the CPU oracle: the fixed parity cases pick the sizes someone thought of, these pick the rest."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2608_08751_b200 import binding as B
+from paper_2608_08751_b200 import synth
+
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def _t(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _points(rng, dtype, n, d, integer):
+    if dtype == "u8":
+        return rng.integers(0, 16 if integer else 256, (n, d)).astype(np.uint8)
+    if dtype == "i8":
+        return rng.integers(-8 if integer else -128, 8 if integer else 128, (n, d)).astype(np.int8)
+    return (rng.standard_normal((n, d)) * rng.choice([1e-3, 1.0, 50.0])).astype(np.float32)
+
+
+def _centroids(rng, dtype, nlist, d, integer):
+    if integer:
+        lo, hi = (0, 16) if dtype == "u8" else (-8, 8)
+        return rng.integers(lo, hi, (nlist, d)).astype(np.float32)
+    if dtype == "u8":
+        return (rng.standard_normal((nlist, d)) * 40 + 100).astype(np.float32)
+    if dtype == "i8":
+        return (rng.standard_normal((nlist, d)) * 40).astype(np.float32)
+    return (rng.standard_normal((nlist, d))).astype(np.float32)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_route_random_shapes(seed):
+    rng = np.random.default_rng(5000 + seed)
+    dtype = rng.choice(["u8", "i8", "f32"])
+    integer = dtype != "f32" and rng.random() < 0.4
+    d = int(rng.choice([4, 8, 16, 20, 32, 48, 64, 96, 100, 128, 160, 192, 256]))
+    n = int(rng.choice([1, 2, 31, 127, 128, 129, 255, 257, 500, 1000, 1500]))
+    nlist = int(rng.choice([1, 2, 7, 64, 255, 256, 257, 1000, 4096, 9000, 20000, 70000]))
+    k = int(min(nlist, rng.choice([1, 1, 2, 3, 10, 16, 17, 50, 64, 100, 200, 512])))
+    if n * nlist * d > 3e9:  # keep the oracle quick
+        n = max(1, int(3e9 / (nlist * d)))
+    x = _points(rng, dtype, n, d, integer)
+    c = _centroids(rng, dtype, nlist, d, integer)
+    if k == 1 and rng.random() < 0.5:
+        ids, dists = B.ivf_assign(_t(x), _t(c))
+    else:
+        ids, dists = B.ivf_route(_t(x), _t(c), k)
+    B.ivf_check()
+    parity.check_route(x, c, k, ids.cpu().numpy(), dists.cpu().numpy(), exact=bool(integer))
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_update_and_reorder_random_shapes(seed):
+    rng = np.random.default_rng(6000 + seed)
+    dtype = rng.choice(["u8", "i8", "f32"])
+    d = int(rng.choice([4, 16, 36, 100, 128, 256]))
+    n = int(rng.choice([1, 100, 5000, 40000]))
+    nlist = int(rng.choice([1, 3, 300, 5000, 70000]))
+    x = _points(rng, dtype, n, d, False)
+    ids = rng.integers(0, nlist, n).astype(np.int32)
+    # accumulation on top of earlier sums: integers for byte-typed points (the result stays exact)
+    base = rng.integers(-50, 50, (nlist, d)) if dtype != "f32" else rng.standard_normal((nlist, d))
+    sums = torch.from_numpy(base.astype(np.float32)).cuda()
+    counts = torch.from_numpy(rng.integers(0, 5, nlist).astype(np.int64)).cuda()
+    base_s, base_c = sums.cpu().numpy().astype(np.float64), counts.cpu().numpy().copy()
+    B.ivf_centroid_update(_t(x), _t(ids), sums, counts)
+    B.ivf_check()
+    parity.check_update(x, ids, nlist, sums.cpu().numpy(), counts.cpu().numpy(), base_s, base_c)
+    xr, offsets, order = B.ivf_cluster_major_reorder(_t(x), _t(ids), nlist)
+    B.ivf_check()
+    want_off, _ = O.reorder(ids, nlist)
+    order = order.cpu().numpy()
+    assert (offsets.cpu().numpy() == want_off).all()
+    assert (np.sort(order) == np.arange(n)).all() and (np.diff(ids[order]) >= 0).all()
+    assert (xr.cpu().numpy() == x[order]).all()
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_pq_random_shapes(seed):
+    rng = np.random.default_rng(7000 + seed)
+    dtype = rng.choice(["u8", "i8", "f32"])
+    pq_m, dsub = [(32, 4), (16, 8), (32, 3), (16, 6), (20, 5), (50, 2), (8, 1), (1, 16), (64, 2), (4, 7)][seed % 10]
+    d = pq_m * dsub
+    nlist = int(rng.choice([3, 40, 400]))
+    n = int(rng.choice([200, 5000, 30000]))
+    nq = int(rng.choice([1, 7, 40]))
+    nprobe = int(min(nlist, rng.choice([1, 3, 16, 64])))
+    n_rerank = int(rng.choice([1, 10, 100, 512, 1024]))
+    c = _centroids(rng, dtype, nlist, d, False)
+    ids, offsets = synth.skewed_list_ids(n, nlist, seed=seed, sigma=float(rng.choice([0.3, 1.0, 2.0])))
+    x = _points(rng, dtype, n, d, False)
+    cb = synth.pq_codebooks(pq_m, dsub, 20.0 if dtype != "f32" else 0.5, seed=seed, integer=bool(rng.random() < 0.3))
+    q = _points(rng, dtype, nq, d, False)
+    probes = synth.distinct_probes(nq, nlist, nprobe, seed=seed)
+    want_codes = O.pq_encode(x, ids, c, cb)
+    got_codes = B.ivf_pq_encode(_t(x), _t(ids), _t(c), _t(cb))
+    B.ivf_check()
+    assert (got_codes.cpu().numpy() == want_codes).all()
+    want = O.pq_search(q, c, probes, offsets, want_codes, cb, n_rerank)
+    got = B.ivf_pq_search(_t(q), _t(c), _t(probes), _t(offsets), _t(want_codes), _t(cb), n_rerank)
+    B.ivf_check()
+    assert (got[0].cpu().numpy() == want[0]).all() and (got[2].cpu().numpy() == want[2]).all()
+    assert (got[1].cpu().numpy().view(np.uint32) == want[1].view(np.uint32)).all()
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_candidates_random_shapes(seed):
+    rng = np.random.default_rng(8000 + seed)
+    dtype = rng.choice(["u8", "i8", "f32"])
+    d = int(rng.choice([4, 36, 100, 128, 256]))
+    n, nlist, m = int(rng.choice([1, 333, 4000])), int(rng.choice([1, 50, 3000])), int(rng.choice([1, 2, 3, 8, 11]))
+    x = _points(rng, dtype, n, d, True)
+    c = _centroids(rng, dtype, nlist, d, True)
+    cand = rng.integers(0, nlist, (n, m)).astype(np.int32)
+    ids, dist = B.ivf_assign_candidates(_t(x), _t(c), _t(cand))
+    B.ivf_check()
+    want_ids, want_d = O.assign_candidates(x, c, cand)
+    ids, dist = ids.cpu().numpy(), dist.cpu().numpy().astype(np.float64)
+    if dtype != "f32":  # integer data: exact
+        assert (ids == want_ids).all() and (dist == want_d).all()
+    else:
+        true_d = O.pair_dists(x, c, np.arange(n), ids)
+        assert np.allclose(dist, true_d, rtol=1e-5, atol=1e-30)
+        assert (true_d <= want_d * (1 + 1e-5) + 1e-30).all()
