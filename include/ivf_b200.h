@@ -26,6 +26,10 @@
  *              id out of range) set a sticky per-device status word that ivf_check reads.
  *   Limits     d must be a multiple of 4, 4 <= d <= 256 (d = 100 is padded to the next multiple of 16 inside the operand copies;
  *              uint8 rows with d a multiple of 16 take the fastest path: no fp16 copy in HBM).  1 <= nprobe <= min(nlist, 512).
+ *              Float inputs are scaled by an exact power of two (exponent clamped to +-40) before they are
+ *              rounded to fp16: finite values with magnitude between about 1e-12 and 1e12 keep the stated
+ *              tolerance (tested); beyond 2^51 the operands overflow and the results are undefined,
+ *              as they are for non-finite inputs (always memory-safe).
  *              nlist < 2^31.  n == 0 is IVF_OK and enqueues nothing.
  *   Non-finite inputs give unspecified (but memory-safe) results.
  *

@@ -130,3 +130,28 @@ def test_candidates_random_shapes(seed):
         true_d = O.pair_dists(x, c, np.arange(n), ids)
         assert np.allclose(dist, true_d, rtol=1e-5, atol=1e-30)
         assert (true_d <= want_d * (1 + 1e-5) + 1e-30).all()
+
+
+@pytest.mark.parametrize("scale", [1e-12, 1e-6, 1e6, 1e12])
+@pytest.mark.parametrize("k", [1, 20])
+def test_route_extreme_magnitudes(scale, k):
+    # the power-of-two operand scaling must keep small and large inputs inside fp16's range and the
+    # returned distances inside the tolerance, which is relative to the norms
+    rng = np.random.default_rng(int(abs(np.log10(scale))) + k)
+    x = (rng.standard_normal((300, 64)) * scale).astype(np.float32)
+    c = (rng.standard_normal((2500, 64)) * scale).astype(np.float32)
+    ids, dists = (B.ivf_assign if k == 1 else lambda a, b: B.ivf_route(a, b, k))(_t(x), _t(c))
+    B.ivf_check()
+    parity.check_route(x, c, k, ids.cpu().numpy(), dists.cpu().numpy())
+
+
+def test_route_mixed_magnitudes_between_points_and_centroids():
+    # points much smaller than centroids and the other way round (the point scale is capped by the
+    # centroid scale and floored 2^29 below it)
+    rng = np.random.default_rng(77)
+    for sx, sc in [(1e-4, 10.0), (300.0, 1e-2), (1.0, 1e5)]:
+        x = (rng.standard_normal((200, 32)) * sx).astype(np.float32)
+        c = (rng.standard_normal((1500, 32)) * sc).astype(np.float32)
+        ids, dists = B.ivf_route(_t(x), _t(c), 12)
+        B.ivf_check()
+        parity.check_route(x, c, 12, ids.cpu().numpy(), dists.cpu().numpy())
