@@ -777,6 +777,13 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                             tmem_ld_32x32b_x32(taddr + col_of(q + 1), accB);
                             tmem_wait_ld_regs(accA);
                             tmem_wait_ld_regs(accB);
+                            if (q + 2 >= nq) {
+                                // the warp's last columns of this accumulator are in registers: hand the
+                                // buffer back to the MMA warp before working on them
+                                tc_fence_before_sync();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(&t_empty[buf]);
+                            }
                             if (ragged) {
                                 mask_ragged(accA, tile_j0 + col_of(q), p.nlist);
                                 mask_ragged(accB, tile_j0 + col_of(q + 1), p.nlist);
@@ -787,9 +794,6 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                             after_chunk();
                         }
                     }
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&t_empty[buf]);
                 }
                 ++it;
             }
