@@ -559,6 +559,16 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             const int64_t r = u / NT;
             const int t0 = static_cast<int>(u - r * NT);
             const int t1 = static_cast<int>((u1 - r * NT < NT) ? (u1 - r * NT) : NT);
+            if (raw && u1 > (r + 1) * NT) {
+                // this CTA will move on to the next row group: pull its raw rows into L2 now, so that
+                // the widening at the crossing does not wait for HBM
+                const int64_t first_row = (r + 1) * MT * kBlockM;
+                const int64_t last_row = (first_row + MT * kBlockM < p.n) ? first_row + MT * kBlockM : p.n;
+                const char* base = reinterpret_cast<const char*>(p.x_raw) + first_row * p.d;
+                const int64_t bytes = (last_row - first_row) * p.d;
+                for (int64_t off = static_cast<int64_t>(lane) * 128; off < bytes; off += 32 * 128)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
+            }
             if (lane == 0 && seg > 0) ok = mbar_wait(a_empty, (seg - 1) & 1, ctl, 1);
             ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
