@@ -267,7 +267,7 @@ int ivf_assign_candidates(const void* points, int64_t n, int d, ivf_dtype ptype,
  *     acc = fma(diff, diff, acc);   estimate: acc = 0, for m ascending: acc = acc + LUT_m[a_m].
  *
  * codebooks  [pq_m][256][d / pq_m] float32, row-major.  pq_m must divide d.  Encoding keeps the
- *            codebook in shared memory: 1024 * (d + pq_m) + 4 * d + 29,776 bytes must fit one SM's
+ *            codebook in shared memory: 1024 * (d + pq_m) + 4 * d bytes must fit one SM's
  *            227 KB (d = 128 with pq_m = 32 does; d = 256 does not); searching needs
  *            1024 * pq_m + 21,584 bytes and d <= 256 -> IVF_ERR_UNSUPPORTED otherwise.
  *

@@ -34,48 +34,24 @@ constexpr int kPqMaxRerank = 1024;
 constexpr int kPqMaxProbes = 512;   // lists per query (the paper sweeps the probe count up to 512)
 constexpr int kPqStatusBadId = -6;
 
+// shared memory of the encode kernel: the transposed codebook, one lookup table, one residual
 __host__ __device__ inline size_t pq_smem_bytes(int d, int pq_m) {
-    return static_cast<size_t>(d) * kPqK * 4 + static_cast<size_t>(pq_m) * kPqK * 4 + static_cast<size_t>(d) * 4 +
-           static_cast<size_t>(kPqBufKeys) * 8 + 256 * 4 + 64 +
-           static_cast<size_t>(kPqMaxProbes) * 24 + 16;  // probe descriptors
+    return static_cast<size_t>(d) * kPqK * 4 + static_cast<size_t>(pq_m) * kPqK * 4 + static_cast<size_t>(d) * 4;
 }
 
 struct PqSmem {
-    float* cbt;     // [d][256]: coordinate-major codebook
-    float* lut;     // [pq_m][256]
-    float* r;       // [d]
-    uint64_t* buf;  // [kPqBufKeys]
-    int* hist;      // [256]
-    int* misc;      // [16]: 0 count, 1 digit, 2 rank, 3 eq
-    long long* list_begin;  // [kPqMaxProbes] first position of each probed list
-    long long* list_len;    // [kPqMaxProbes]
-    int* list_id;           // [kPqMaxProbes]
-    int* cs;                // [kPqMaxProbes + 1] chunk prefix of the query
+    float* cbt;  // [d][256]: coordinate-major codebook
+    float* lut;  // [pq_m][256]
+    float* r;    // [d]
 };
 
-// with_codebook: the encode kernel keeps the codebook in shared memory; the scan kernel reads its
-// transposed copy through L1 and carves none.
-__device__ __forceinline__ PqSmem pq_carve(uint8_t* raw, int d, int pq_m, bool with_codebook, int buf_keys) {
+__device__ __forceinline__ PqSmem pq_carve(uint8_t* raw, int d, int pq_m) {
     PqSmem s;
-    s.buf = reinterpret_cast<uint64_t*>(raw);
-    raw += static_cast<size_t>(buf_keys) * 8;
-    s.list_begin = reinterpret_cast<long long*>(raw);
-    raw += static_cast<size_t>(kPqMaxProbes) * 8;
-    s.list_len = reinterpret_cast<long long*>(raw);
-    raw += static_cast<size_t>(kPqMaxProbes) * 8;
     s.cbt = reinterpret_cast<float*>(raw);
-    if (with_codebook) raw += static_cast<size_t>(d) * kPqK * 4;
+    raw += static_cast<size_t>(d) * kPqK * 4;
     s.lut = reinterpret_cast<float*>(raw);
     raw += static_cast<size_t>(pq_m) * kPqK * 4;
     s.r = reinterpret_cast<float*>(raw);
-    raw += static_cast<size_t>(d) * 4;
-    s.hist = reinterpret_cast<int*>(raw);
-    raw += 256 * 4;
-    s.misc = reinterpret_cast<int*>(raw);
-    raw += 64;
-    s.list_id = reinterpret_cast<int*>(raw);
-    raw += static_cast<size_t>(kPqMaxProbes) * 4;
-    s.cs = reinterpret_cast<int*>(raw);
     return s;
 }
 
@@ -197,7 +173,7 @@ struct PqEncodeParams {
 
 __global__ void __launch_bounds__(kPqThreads, 1) pq_encode_kernel(const PqEncodeParams p) {
     extern __shared__ __align__(16) uint8_t pq_smem_raw[];
-    const PqSmem s = pq_carve(pq_smem_raw, p.d, p.pq_m, true, kPqBufKeys);
+    const PqSmem s = pq_carve(pq_smem_raw, p.d, p.pq_m);
     const int dsub = p.d / p.pq_m;
     pq_load_codebooks(p.codebooks, p.d, dsub, s.cbt);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
