@@ -409,8 +409,8 @@ def main():
     line = {
         "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
         "ms_per_step": t_step / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f16 operands (uint8 exact), f32 accumulate", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "l2": "256 MB buffer rewritten between timed steps, outside the per-step events",
+        "dtype": "f16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "arithmetic": "fp16 tensor-core operands (uint8 values exact), fp32 accumulation, fp32 norms", "l2": "256 MB buffer rewritten between timed steps, outside the per-step events",
                    "kernel_timing": "per-kernel CUDA events in a second pass of the same K steps",
                    "exchange": "all-reduce of sums/counts per step" if distributed else "none (1 GPU)"},
         "assigned_vectors_per_s": vps,
