@@ -286,6 +286,12 @@ int ivf_assign_candidates(const void* points, int64_t n, int d, ivf_dtype ptype,
  *            16-byte aligned.  Chunk and group descriptors are built on the device (no host
  *            synchronisation); the workspace is the library's grow-only one.
  */
+/* out_residuals[i][t] = float(points[i][t]) - centroids[ids[i]][t] (fp32 [n][d], device): the vectors
+ * the PQ codebooks are trained on (Sec. 4.3).  Training itself is k-means per subspace and is composed
+ * from ivf_assign_update / ivf_centroid_finalize on the sub-vector columns (256 lists, d / pq_m wide).
+ * An id outside [0, nlist) gives a zero row and sets IVF_ERR_BAD_ID. */
+int ivf_pq_residuals(const void* points, int64_t n, int d, ivf_dtype ptype, const int32_t* ids,
+                     const float* centroids, int nlist, float* out_residuals, void* stream);
 int ivf_pq_encode(const void* points, int64_t n, int d, ivf_dtype ptype, const int32_t* ids,
                   const float* centroids, int nlist, const float* codebooks, int pq_m,
                   uint8_t* out_codes, void* stream);

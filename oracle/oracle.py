@@ -51,6 +51,7 @@ def _load():
         _lib.oracle_pq_lut.restype = None
         _lib.oracle_pq_adc.argtypes = [vp, ctypes.c_int, vp, i64, i64, vp]
         _lib.oracle_pq_adc.restype = None
+        _lib.oracle_residuals.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, vp, vp, i32, vp]
         _lib.oracle_pq_encode.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, vp, vp, i32, vp, ctypes.c_int, vp]
         _lib.oracle_pq_search.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, vp, i32, vp, ctypes.c_int, vp, vp,
                                           vp, ctypes.c_int, ctypes.c_int, vp, vp, vp]
@@ -254,3 +255,15 @@ def pq_search(q: np.ndarray, c: np.ndarray, probes: np.ndarray, offsets: np.ndar
     if rc != 0:
         raise ValueError("oracle_pq_search: bad arguments")
     return pos, est, count
+
+
+def residuals(x: np.ndarray, ids: np.ndarray, c: np.ndarray) -> np.ndarray:
+    """float32 [n, d]: x - c[ids], one rounded fp32 subtraction per coordinate."""
+    x, xt = _rows(x)
+    c = _cent(c)
+    ids = np.ascontiguousarray(ids, np.int32)
+    out = np.empty(x.shape, np.float32)
+    rc = _load().oracle_residuals(_p(x), xt, x.shape[0], x.shape[1], _p(ids), _p(c), c.shape[0], _p(out))
+    if rc != 0:
+        raise ValueError("oracle_residuals: id out of range")
+    return out

@@ -186,3 +186,16 @@ int oracle_pq_search(const void *q, int qtype, int64_t nq, int d, const float *c
     }
     return rc;
 }
+
+/*
+ * Residuals x - c(x) (Sec. 4.3: the vectors that the PQ codebooks are trained on and that are
+ * encoded), in fp32 as one rounded subtraction per coordinate.  out [n][d] float.
+ * Returns -1 on an id out of range.
+ */
+int oracle_residuals(const void *x, int xtype, int64_t n, int d, const int32_t *ids, const float *c, int32_t nlist,
+                     float *out) {
+    for (int64_t i = 0; i < n; ++i)
+        if (ids[i] < 0 || ids[i] >= nlist) return -1;
+    for (int64_t i = 0; i < n; ++i) residual(x, xtype, i, c, ids[i], d, out + i * d);
+    return 0;
+}

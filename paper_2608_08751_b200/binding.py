@@ -23,7 +23,7 @@ EXPORTS = (
     "ivf_route", "ivf_assign", "ivf_centroid_update", "ivf_centroid_update_noalloc", "ivf_centroid_finalize",
     "ivf_assign_update", "ivf_cluster_major_reorder", "ivf_centroids_create", "ivf_centroids_destroy",
     "ivf_route_prepared",
-    "ivf_pq_encode", "ivf_pq_search", "ivf_assign_candidates",
+    "ivf_pq_encode", "ivf_pq_search", "ivf_pq_residuals", "ivf_assign_candidates",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
     "ivf_debug_plan", "ivf_debug_span", "ivf_debug_set_wait_limit_ns",
     "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_set_row_chunk", "ivf_debug_stats", "ivf_debug_set_pq_groups", "ivf_debug_set_dependent_launch", "ivf_debug_set_crossing_cost",
@@ -75,6 +75,7 @@ def lib() -> ctypes.CDLL:
     L.ivf_debug_stats.argtypes = [i32, ctypes.POINTER(i64)]
     L.ivf_debug_rule.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_int)]
     L.ivf_assign_candidates.argtypes = [vp, i64, i32, i32, vp, i32, vp, i32, vp, vp, vp]
+    L.ivf_pq_residuals.argtypes = [vp, i64, i32, i32, vp, vp, i32, vp, vp]
     L.ivf_pq_encode.argtypes = [vp, i64, i32, i32, vp, vp, i32, vp, i32, vp, vp]
     L.ivf_pq_search.argtypes = [vp, i64, i32, i32, vp, i32, vp, i32, vp, vp, i64, vp, i32, i32, vp, vp, vp, vp, vp]
     L.ivf_debug_set_pq_groups.argtypes = [i32]
@@ -306,6 +307,23 @@ def _codebooks(codebooks: torch.Tensor, d: int) -> int:
     if codebooks.dim() != 3 or codebooks.shape[1] != 256 or codebooks.shape[0] * codebooks.shape[2] != d:
         raise ValueError("codebooks must be [pq_m, 256, d / pq_m]")
     return codebooks.shape[0]
+
+
+def ivf_pq_residuals(points: torch.Tensor, ids: torch.Tensor, centroids: torch.Tensor) -> torch.Tensor:
+    """float32 [n, d]: points - centroids[ids], the training vectors of the PQ codebooks."""
+    if not points.is_cuda:
+        raise ValueError("points must be a CUDA tensor")
+    _rows(points, "points")
+    _dev(ids, "ids", torch.int32)
+    _dev(centroids, "centroids", torch.float32)
+    n, d = points.shape
+    out = torch.empty((n, d), dtype=torch.float32, device=points.device)
+    with torch.cuda.device(points.device):
+        rc = lib().ivf_pq_residuals(_ptr(points), n, d, _dtype_code(points), _ptr(ids), _ptr(centroids),
+                                    centroids.shape[0], _ptr(out), _stream(points.device))
+    if rc != IVF_OK:
+        _raise(rc)
+    return out
 
 
 def ivf_pq_encode(points: torch.Tensor, ids: torch.Tensor, centroids: torch.Tensor, codebooks: torch.Tensor):

@@ -1067,6 +1067,25 @@ int pq_set_attrs(DeviceCtx& ctx) {
 }
 }  // namespace
 
+int ivf_pq_residuals(const void* points, int64_t n, int d, ivf_dtype ptype, const int32_t* ids, const float* centroids,
+                     int nlist, float* out_residuals, void* stream_) {
+    if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
+    if (!valid_dtype(ptype)) return fail(IVF_ERR_INVALID_ARG, "unknown element type %d", (int)ptype);
+    if (d < 1 || nlist < 1) return fail(IVF_ERR_INVALID_ARG, "d = %d, nlist = %d", d, nlist);
+    if (n == 0) return IVF_OK;
+    if (!points || !ids || !centroids || !out_residuals) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    DeviceCtx* pctx = nullptr;
+    int rc = get_ctx(&pctx);
+    if (rc != IVF_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int64_t total = n * d;
+    pq_residuals_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, stream>>>(points, static_cast<int>(ptype), n, d, ids,
+                                                                                     centroids, nlist, out_residuals,
+                                                                                     pctx->status);
+    LAUNCH_CHECK();
+    return IVF_OK;
+}
+
 int ivf_pq_encode(const void* points, int64_t n, int d, ivf_dtype ptype, const int32_t* ids, const float* centroids,
                   int nlist, const float* codebooks, int pq_m, uint8_t* out_codes, void* stream_) {
     if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);

@@ -219,6 +219,24 @@ __global__ void __launch_bounds__(kPqThreads, 1) pq_encode_kernel(const PqEncode
     }
 }
 
+// Residuals x - c(x) as fp32 rows (the training set of the codebooks, Sec. 4.3): one rounded
+// subtraction per coordinate, exactly what the encoder and the oracle compute.
+__global__ void pq_residuals_kernel(const void* __restrict__ x, int x_type, int64_t n, int d,
+                                    const int32_t* __restrict__ ids, const float* __restrict__ centroids, int nlist,
+                                    float* __restrict__ out, int* status) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n * d) return;
+    const int64_t row = i / d;
+    const int t = static_cast<int>(i - row * d);
+    const int32_t l = ids[row];
+    if (l < 0 || l >= nlist) {
+        if (t == 0) atomicCAS(status, 0, kPqStatusBadId);
+        out[i] = 0.0f;
+        return;
+    }
+    out[i] = __fsub_rn(pq_elem(x, x_type, i), centroids[static_cast<int64_t>(l) * d + t]);
+}
+
 // codebooks [pq_m][256][dsub] -> out[(m * dsub + t) * 256 + j] (coordinate-major), for the scan kernel
 __global__ void pq_transpose_codebooks_kernel(const float* __restrict__ codebooks, int d, int dsub, float* __restrict__ out) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;  // index in the output

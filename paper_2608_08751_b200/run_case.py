@@ -86,7 +86,6 @@ def build_case(args):
     sums = torch.zeros((args.nlist, args.d), dtype=torch.float32, device="cuda")
     counts = torch.zeros((args.nlist,), dtype=torch.int64, device="cuda")
     ids = torch.empty((args.n,), dtype=torch.int32, device="cuda")
-    cb = torch.from_numpy(synth.pq_codebooks(args.pq_m, args.d // args.pq_m, 20.0 if args.dtype == "u8" else 0.05, seed=1)).cuda()
     B.ivf_assign_update(train[:4096], cent, sums, counts, None, None)  # warm-up (workspace growth)
     torch.cuda.synchronize()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
@@ -101,14 +100,24 @@ def build_case(args):
     ev[2].record()
     dev_rows = host.cuda()
     xr, offsets, order = B.ivf_cluster_major_reorder(dev_rows, ids, args.nlist)
-    codes = B.ivf_pq_encode(xr, ids[order.long()], cent, cb)
+    ids_sorted = ids[order.long()]
+    ev.append(torch.cuda.Event(enable_timing=True))
     ev[3].record()
+    from . import pq_train
+    cb, _ = pq_train.train_codebooks(xr, ids_sorted, cent, args.pq_m, iters=args.iters, seed=1,
+                                     sample_rows=min(args.n, 1 << 20))
+    ev.append(torch.cuda.Event(enable_timing=True))
+    ev[4].record()
+    codes = B.ivf_pq_encode(xr, ids_sorted, cent, cb)
+    ev.append(torch.cuda.Event(enable_timing=True))
+    ev[5].record()
     B.ivf_check()
-    t = [ev[i].elapsed_time(ev[i + 1]) for i in range(3)]
+    t = [ev[i].elapsed_time(ev[i + 1]) for i in range(5)]
     lens = (offsets[1:] - offsets[:-1])
     print(json.dumps({"op": "build", "n": args.n, "train_rows": train_rows, "nlist": args.nlist, "d": args.d,
                       "dtype": args.dtype, "iters": args.iters, "train_ms": t[0], "assign_all_ms": t[1],
-                      "reorder_encode_ms": t[2], "total_ms": sum(t), "vectors_per_s": args.n / (sum(t) / 1e3),
+                      "copy_reorder_ms": t[2], "pq_train_ms": t[3], "pq_encode_ms": t[4], "total_ms": sum(t),
+                      "vectors_per_s": args.n / (sum(t) / 1e3),
                       "empty_lists": int((lens == 0).sum().item()), "max_list": int(lens.max().item()),
                       "codes_bytes": int(codes.numel())}))
 

@@ -192,3 +192,46 @@ def test_many_probes_take_the_single_team_kernel(nprobe):
     with pytest.raises(B.IvfError) as e:
         B.ivf_pq_search(_t(q), _t(c), _t(np.tile(probes, (1, 2))[:, :513].copy()), _t(offsets), _t(codes), _t(cb), 8)
     assert e.value.code in (B.IVF_ERR_UNSUPPORTED, B.IVF_ERR_INVALID_ARG)
+
+
+def test_residuals_and_codebook_training_step_by_step():
+    # residuals bit-identical; then every Lloyd step of the per-subspace training is compared with
+    # the oracle fed the GPU's current codebook (so a tolerated near-tie cannot compound)
+    from paper_2608_08751_b200 import pq_train
+    import parity
+    rng = np.random.default_rng(41)
+    n, nlist, d, pq_m = 6000, 30, 32, 8
+    dsub = d // pq_m
+    c = rng.normal(0, 1, (nlist, d)).astype(np.float32)
+    ids, _ = synth.skewed_list_ids(n, nlist, seed=41)
+    x = synth.rows_near(c, ids, 0.3, 41)
+    res = B.ivf_pq_residuals(_t(x), _t(ids), _t(c))
+    B.ivf_check()
+    want = O.residuals(x, ids, c)
+    assert (res.cpu().numpy().view(np.uint32) == want.view(np.uint32)).all()
+    codebooks, inertia = pq_train.train_codebooks(_t(x), _t(ids), _t(c), pq_m, iters=4, seed=1)
+    B.ivf_check()
+    assert codebooks.shape == (pq_m, 256, dsub)
+    assert (np.diff(inertia.numpy(), axis=1) <= 1e-6 * inertia.numpy()[:, :-1]).all()  # Lloyd never gets worse
+    # one more step on subspace 3, checked against the oracle: assignment inside the tolerance band,
+    # sums and counts for the GPU's ids, means
+    sub = np.ascontiguousarray(want[:, 3 * dsub:4 * dsub])
+    cb = codebooks[3].clone()
+    sums = torch.zeros((256, dsub), dtype=torch.float32, device="cuda")
+    counts = torch.zeros((256,), dtype=torch.int64, device="cuda")
+    a_ids = torch.empty((n,), dtype=torch.int32, device="cuda")
+    a_d = torch.empty((n,), dtype=torch.float32, device="cuda")
+    B.ivf_assign_update(_t(sub), cb, sums, counts, a_ids, a_d)
+    B.ivf_check()
+    g = a_ids.cpu().numpy()
+    parity.check_route(sub, codebooks[3].cpu().numpy(), 1, g, a_d.cpu().numpy())
+    parity.check_update(sub, g, 256, sums.cpu().numpy(), counts.cpu().numpy())
+    # the trained codebooks quantise better than the synthetic Gaussian ones the other tests use
+    codes = B.ivf_pq_encode(_t(x), _t(ids), _t(c), codebooks)
+    rand_cb = _t(synth.pq_codebooks(pq_m, dsub, 0.3, seed=41))
+    codes_r = B.ivf_pq_encode(_t(x), _t(ids), _t(c), rand_cb)
+    def err(cb_t, cd):
+        cbn, cdn = cb_t.cpu().numpy(), cd.cpu().numpy()
+        dec = np.concatenate([cbn[m, cdn[:, m]] for m in range(pq_m)], axis=1)
+        return ((want - dec) ** 2).sum(1).mean()
+    assert err(codebooks, codes) < 0.8 * err(rand_cb, codes_r)

@@ -209,3 +209,18 @@ def test_bad_arguments_are_refused():
     badp = probes.copy(); badp[0, 0] = -1
     with pytest.raises(ValueError):
         O.pq_search(q, c, badp, offsets, codes, cb, 4)
+
+
+def test_residuals_against_numpy():
+    rng = np.random.default_rng(31)
+    c = rng.normal(0, 3, (9, 12)).astype(np.float32)
+    ids = rng.integers(0, 9, 50).astype(np.int32)
+    for x in (rng.integers(0, 256, (50, 12)).astype(np.uint8), rng.integers(-128, 128, (50, 12)).astype(np.int8),
+              rng.normal(0, 3, (50, 12)).astype(np.float32)):
+        r = O.residuals(x, ids, c)
+        assert r.dtype == np.float32 and (r == (x.astype(np.float32) - c[ids])).all()
+    # a point equal to its centroid has a zero residual; the encoder then picks the codeword nearest 0
+    x = c[ids].copy()
+    assert (O.residuals(x, ids, c) == 0).all()
+    with pytest.raises(ValueError):
+        O.residuals(x, np.full(50, 9, np.int32), c)
