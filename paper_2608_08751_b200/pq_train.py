@@ -19,9 +19,10 @@ def train_codebooks(points: torch.Tensor, ids: torch.Tensor, centroids: torch.Te
     """(codebooks float32 [pq_m, 256, d // pq_m], inertia [pq_m, iters]): k-means per subspace on the
     residuals of `points` (row i assigned to list ids[i]).  `sample_rows` trains on a seeded sample."""
     n, d = points.shape
-    if d % pq_m != 0 or (d // pq_m) % 4 != 0:
-        raise ValueError("the sub-vector width d / pq_m must be a multiple of 4 (the assignment kernel's limit)")
+    if d % pq_m != 0:
+        raise ValueError("pq_m must divide d")
     dsub = d // pq_m
+    wide = (dsub + 3) // 4 * 4  # the assignment kernel takes rows of 4k floats: zero columns change no distance
     dev = points.device
     gen = torch.Generator(device="cpu").manual_seed(seed)
     if sample_rows is not None and sample_rows < n:
@@ -34,12 +35,13 @@ def train_codebooks(points: torch.Tensor, ids: torch.Tensor, centroids: torch.Te
     init = torch.randperm(n, generator=gen)[:256].sort().values.to(dev)
     codebooks = torch.empty((pq_m, 256, dsub), dtype=torch.float32, device=dev)
     inertia = torch.zeros((pq_m, iters), dtype=torch.float64)
-    sums = torch.empty((256, dsub), dtype=torch.float32, device=dev)
+    sums = torch.empty((256, wide), dtype=torch.float32, device=dev)
     counts = torch.empty((256,), dtype=torch.int64, device=dev)
     a_ids = torch.empty((n,), dtype=torch.int32, device=dev)
     a_d = torch.empty((n,), dtype=torch.float32, device=dev)
     for m in range(pq_m):
-        sub = res[:, m * dsub:(m + 1) * dsub].contiguous()
+        sub = torch.zeros((n, wide), dtype=torch.float32, device=dev)
+        sub[:, :dsub] = res[:, m * dsub:(m + 1) * dsub]
         cb = sub[init].clone()
         for it in range(iters):
             sums.zero_()
@@ -47,5 +49,5 @@ def train_codebooks(points: torch.Tensor, ids: torch.Tensor, centroids: torch.Te
             B.ivf_assign_update(sub, cb, sums, counts, a_ids, a_d)
             B.ivf_centroid_finalize(sums, counts, cb)
             inertia[m, it] = float(a_d.double().sum().item())
-        codebooks[m] = cb
+        codebooks[m] = cb[:, :dsub]
     return codebooks, inertia

@@ -235,3 +235,21 @@ def test_residuals_and_codebook_training_step_by_step():
         dec = np.concatenate([cbn[m, cdn[:, m]] for m in range(pq_m)], axis=1)
         return ((want - dec) ** 2).sum(1).mean()
     assert err(codebooks, codes) < 0.8 * err(rand_cb, codes_r)
+
+
+def test_codebook_training_with_sub_vectors_of_three():
+    # DEEP-shaped width: 96 / 32 = 3 coordinates per subspace (padded to 4 inside the training helper)
+    from paper_2608_08751_b200 import pq_train
+    rng = np.random.default_rng(43)
+    n, nlist, d, pq_m = 3000, 10, 24, 8
+    c = rng.normal(0, 1, (nlist, d)).astype(np.float32)
+    ids, _ = synth.skewed_list_ids(n, nlist, seed=43)
+    x = synth.rows_near(c, ids, 0.3, 43)
+    codebooks, inertia = pq_train.train_codebooks(_t(x), _t(ids), _t(c), pq_m, iters=3, seed=2)
+    B.ivf_check()
+    assert codebooks.shape == (pq_m, 256, 3) and torch.isfinite(codebooks).all()
+    assert (np.diff(inertia.numpy(), axis=1) <= 1e-6 * inertia.numpy()[:, :-1]).all()
+    want = O.pq_encode(x, ids, c, codebooks.cpu().numpy())
+    got = B.ivf_pq_encode(_t(x), _t(ids), _t(c), codebooks.contiguous())
+    B.ivf_check()
+    assert (got.cpu().numpy() == want).all()
