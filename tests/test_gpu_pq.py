@@ -209,7 +209,7 @@ def test_residuals_and_codebook_training_step_by_step():
     B.ivf_check()
     want = O.residuals(x, ids, c)
     assert (res.cpu().numpy().view(np.uint32) == want.view(np.uint32)).all()
-    codebooks, inertia = pq_train.train_codebooks(_t(x), _t(ids), _t(c), pq_m, iters=4, seed=1)
+    codebooks, inertia = pq_train.train_codebooks(_t(x), _t(ids), _t(c), pq_m, iters=4, seed=1, method="assign")
     B.ivf_check()
     assert codebooks.shape == (pq_m, 256, dsub)
     assert (np.diff(inertia.numpy(), axis=1) <= 1e-6 * inertia.numpy()[:, :-1]).all()  # Lloyd never gets worse
@@ -245,7 +245,7 @@ def test_codebook_training_with_sub_vectors_of_three():
     c = rng.normal(0, 1, (nlist, d)).astype(np.float32)
     ids, _ = synth.skewed_list_ids(n, nlist, seed=43)
     x = synth.rows_near(c, ids, 0.3, 43)
-    codebooks, inertia = pq_train.train_codebooks(_t(x), _t(ids), _t(c), pq_m, iters=3, seed=2)
+    codebooks, inertia = pq_train.train_codebooks(_t(x), _t(ids), _t(c), pq_m, iters=3, seed=2, method="assign")
     B.ivf_check()
     assert codebooks.shape == (pq_m, 256, 3) and torch.isfinite(codebooks).all()
     assert (np.diff(inertia.numpy(), axis=1) <= 1e-6 * inertia.numpy()[:, :-1]).all()
@@ -253,3 +253,41 @@ def test_codebook_training_with_sub_vectors_of_three():
     got = B.ivf_pq_encode(_t(x), _t(ids), _t(c), codebooks.contiguous())
     B.ivf_check()
     assert (got.cpu().numpy() == want).all()
+
+
+@pytest.mark.parametrize("d,pq_m", [(32, 8), (24, 8)])
+def test_codebook_training_through_the_encoder(d, pq_m):
+    # the default training method: assignment = the encoder over all subspaces, update = the sum/count
+    # kernel with the code bytes as list ids.  Every iteration is checked against the oracle: the codes
+    # it used (bit-identical) and the means it produced; the quantisation error never increases.
+    from paper_2608_08751_b200 import pq_train
+    rng = np.random.default_rng(47)
+    n, nlist = 5000, 12
+    dsub = d // pq_m
+    c = rng.normal(0, 1, (nlist, d)).astype(np.float32)
+    ids, _ = synth.skewed_list_ids(n, nlist, seed=47)
+    x = synth.rows_near(c, ids, 0.3, 47)
+    res = O.residuals(x, ids, c)
+
+    def err(cb):
+        codes = O.pq_encode(x, ids, c, cb)
+        dec = np.concatenate([cb[m, codes[:, m]] for m in range(pq_m)], axis=1)
+        return float(((res.astype(np.float64) - dec) ** 2).sum())
+
+    prev_cb, prev_err = None, None
+    for iters in (1, 2, 3):
+        cb, inertia = pq_train.train_codebooks(_t(x), _t(ids), _t(c), pq_m, iters=iters, seed=5)
+        B.ivf_check()
+        cb = cb.cpu().numpy()
+        assert inertia is None and cb.shape == (pq_m, 256, dsub)
+        if prev_cb is not None:
+            # one oracle Lloyd step from the previous codebooks reproduces this iteration
+            codes = O.pq_encode(x, ids, c, prev_cb)
+            for m in range(pq_m):
+                sub = np.ascontiguousarray(res[:, m * dsub:(m + 1) * dsub])
+                sums, counts, ok = O.update(sub, codes[:, m].astype(np.int32), 256)
+                want = O.finalize(sums, counts, prev_cb[m])
+                assert np.allclose(cb[m], want, rtol=2e-6, atol=1e-7)
+        e = err(cb)
+        assert prev_err is None or e <= prev_err * (1 + 1e-9)
+        prev_cb, prev_err = cb, e
