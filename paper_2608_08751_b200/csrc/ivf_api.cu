@@ -128,7 +128,7 @@ void timing_end(int idx, cudaStream_t stream) {
 // ------------------------------------------------------------------ workspace
 enum WsSlot {
     WS_X16, WS_C16, WS_XN, WS_SCAL, WS_BITS, WS_PART, WS_PARTMETA, WS_FAIL, WS_FBKEYS, WS_TAU,
-    WS_UCNT, WS_UOFF, WS_UCUR, WS_UPERM, WS_IDS, WS_CHUNK0, WS_CHUNK1, WS_PQ_CHUNKS, WS_PQ_GCAND, WS_PQ_GCOUNT, WS_PQ_CBT, WS_NUM
+    WS_UCNT, WS_UOFF, WS_UCUR, WS_UPERM, WS_IDS, WS_CHUNK0, WS_CHUNK1, WS_PQ_CHUNKS, WS_PQ_GCAND, WS_PQ_GCOUNT, WS_PQ_CBT, WS_UPARTS, WS_NUM
 };
 struct Buf {
     void* p = nullptr;
@@ -708,6 +708,28 @@ int update_device(DeviceCtx& ctx, const void* points, int ptype, const int32_t* 
     update_scan_local_kernel<<<scan_blocks, 1024, 0, stream>>>(cnt, nlist, off, block_sums);
     update_scan_fix_kernel<<<scan_blocks, 1024, 0, stream>>>(nlist, off, block_sums, cur);
     update_fill_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, off, cur, perm);
+    // few long lists: cut every list into pieces, one warp each, and add the pieces up in order
+    const int64_t avg = n / nlist;
+    int parts = avg >= 4096 ? static_cast<int>((avg + 2047) / 2048) : 1;
+    if (parts > 1024) parts = 1024;
+    if (parts > 1) {
+        float* scratch;
+        WS(WS_UPARTS, static_cast<size_t>(nlist) * parts * d * sizeof(float), scratch);
+        const unsigned pb = static_cast<unsigned>((static_cast<int64_t>(nlist) * parts * 32 + 255) / 256);
+        if (ptype == IVF_U8)
+            update_reduce_parts_kernel<uint8_t><<<pb, 256, 0, stream>>>(static_cast<const uint8_t*>(points), perm, off, nlist, d, parts, scratch);
+        else if (ptype == IVF_I8)
+            update_reduce_parts_kernel<int8_t><<<pb, 256, 0, stream>>>(static_cast<const int8_t*>(points), perm, off, nlist, d, parts, scratch);
+        else
+            update_reduce_parts_kernel<float><<<pb, 256, 0, stream>>>(static_cast<const float*>(points), perm, off, nlist, d, parts, scratch);
+        LAUNCH_CHECK();
+        const int64_t cells = static_cast<int64_t>(nlist) * d;
+        update_combine_parts_kernel<<<static_cast<unsigned>((cells + 255) / 256), 256, 0, stream>>>(
+            scratch, off, nlist, d, parts, sums, reinterpret_cast<long long*>(counts));
+        LAUNCH_CHECK();
+        timing_end(tk, stream);
+        return IVF_OK;
+    }
     const unsigned lb = static_cast<unsigned>((static_cast<int64_t>(nlist) * 32 + 255) / 256);
     if (ptype == IVF_U8)
         update_reduce_kernel<uint8_t><<<lb, 256, 0, stream>>>(static_cast<const uint8_t*>(points), perm, off, nlist, d,

@@ -104,17 +104,11 @@ __global__ void update_fill_kernel(const int32_t* __restrict__ ids, int64_t n, i
     perm[pos] = static_cast<int>(i);
 }
 
-// One warp per list.  Lane q owns columns [128*blk + 4*q, +4) for blk = 0, 1 (d <= 256).
+// Sum of the member rows perm[beg .. end) for one warp: lane q owns columns [128*blk + 4*q, +4) for
+// blk = 0, 1 (d <= 256), four member rows in flight.
 template <typename T>
-__global__ void update_reduce_kernel(const T* __restrict__ x, const int* __restrict__ perm,
-                                     const int* __restrict__ off, int nlist, int d, float* __restrict__ sums,
-                                     long long* __restrict__ counts) {
-    const int lane = threadIdx.x & 31;
-    const int l = static_cast<int>((static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5);
-    if (l >= nlist) return;
-    const int beg = off[l], end = off[l + 1];
-    if (beg == end) return;
-    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+__device__ __forceinline__ void reduce_members(const T* __restrict__ x, const int* __restrict__ perm, int beg, int end, int d,
+                                               int lane, float (&acc)[2][4]) {
     for (int m0 = beg; m0 < end; m0 += 32) {
         const int mine = (m0 + lane < end) ? perm[m0 + lane] : -1;
         const int cntm = min(32, end - m0);
@@ -164,6 +158,20 @@ __global__ void update_reduce_kernel(const T* __restrict__ x, const int* __restr
             }
         }
     }
+}
+
+// One warp per list.
+template <typename T>
+__global__ void update_reduce_kernel(const T* __restrict__ x, const int* __restrict__ perm,
+                                     const int* __restrict__ off, int nlist, int d, float* __restrict__ sums,
+                                     long long* __restrict__ counts) {
+    const int lane = threadIdx.x & 31;
+    const int l = static_cast<int>((static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5);
+    if (l >= nlist) return;
+    const int beg = off[l], end = off[l + 1];
+    if (beg == end) return;
+    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    reduce_members(x, perm, beg, end, d, lane, acc);
 #pragma unroll
     for (int blk = 0; blk < 2; ++blk) {
         const int c0 = 128 * blk + 4 * lane;
@@ -178,6 +186,42 @@ __global__ void update_reduce_kernel(const T* __restrict__ x, const int* __restr
         }
     }
     if (lane == 0) counts[l] += static_cast<long long>(end - beg);
+}
+
+// Few long lists (k-means with a handful of clusters, PQ codebook training with 256): every list is
+// cut into `parts` equal pieces, one warp per piece writes its partial sum to scratch[l][part][d],
+// and update_combine_parts_kernel adds a list's partial sums in piece order (so the result does not
+// depend on scheduling).
+template <typename T>
+__global__ void update_reduce_parts_kernel(const T* __restrict__ x, const int* __restrict__ perm,
+                                           const int* __restrict__ off, int nlist, int d, int parts,
+                                           float* __restrict__ scratch) {
+    const int lane = threadIdx.x & 31;
+    const int64_t w = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    if (w >= static_cast<int64_t>(nlist) * parts) return;
+    const int l = static_cast<int>(w / parts), j = static_cast<int>(w - static_cast<int64_t>(l) * parts);
+    const int beg = off[l], len = off[l + 1] - beg;
+    const int b0 = beg + static_cast<int>(static_cast<int64_t>(len) * j / parts);
+    const int b1 = beg + static_cast<int>(static_cast<int64_t>(len) * (j + 1) / parts);
+    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    reduce_members(x, perm, b0, b1, d, lane, acc);
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk) {
+        const int c0 = 128 * blk + 4 * lane;
+        if (c0 < d)
+            *reinterpret_cast<float4*>(scratch + w * d + c0) = make_float4(acc[blk][0], acc[blk][1], acc[blk][2], acc[blk][3]);
+    }
+}
+
+__global__ void update_combine_parts_kernel(const float* __restrict__ scratch, const int* __restrict__ off, int nlist, int d,
+                                            int parts, float* __restrict__ sums, long long* __restrict__ counts) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= static_cast<int64_t>(nlist) * d) return;
+    const int l = static_cast<int>(i / d), t = static_cast<int>(i - static_cast<int64_t>(l) * d);
+    float partial = 0.0f;
+    for (int j = 0; j < parts; ++j) partial += scratch[(static_cast<int64_t>(l) * parts + j) * d + t];
+    sums[i] += partial;
+    if (t == 0) counts[l] += static_cast<long long>(off[l + 1] - off[l]);
 }
 
 // Cluster-major copy (Sec. 3.1 index layout): destination row p receives source row order[p];

@@ -385,3 +385,24 @@ def test_expired_wait_is_reported_and_context_survives():
     B.ivf_check()
     ids, dists = _route(x, c, 1)
     parity.check_route(x, c, 1, ids, dists)
+
+
+@pytest.mark.parametrize("dtype,n,nlist,d", [("u8", 300000, 3, 128), ("f32", 200000, 1, 96), ("u8", 1 << 20, 256, 4),
+                                              ("f32", 500000, 17, 36), ("u8", 70000, 16, 256)])
+def test_update_with_few_long_lists(dtype, n, nlist, d):
+    # lists of thousands of members are cut into pieces (one warp each) whose partial sums are added
+    # in piece order; uint8 sums stay exact, float sums inside the tolerance, counts exact; the sums
+    # accumulate on top of what is there
+    rng = np.random.default_rng(n % 1000 + nlist)
+    if dtype == "u8":
+        x = rng.integers(0, 16, (n, d)).astype(np.uint8)  # small values: list sums stay below 2^24
+    else:
+        x = rng.standard_normal((n, d)).astype(np.float32)
+    ids = rng.integers(0, nlist, n).astype(np.int32)
+    ids[: n // 3] = 0  # one list much longer than the others
+    base = rng.integers(0, 9, (nlist, d)).astype(np.float32)
+    sums = torch.from_numpy(base.copy()).cuda()
+    counts = torch.full((nlist,), 5, dtype=torch.int64, device="cuda")
+    B.ivf_centroid_update(_cuda(x), _cuda(ids), sums, counts)
+    B.ivf_check()
+    parity.check_update(x, ids, nlist, sums.cpu().numpy(), counts.cpu().numpy(), base.astype(np.float64), np.full(nlist, 5, np.int64))
