@@ -336,41 +336,74 @@ __device__ __forceinline__ float min8(const uint32_t (&acc)[32], int g) {
 template <int EPI>
 __device__ __forceinline__ void consume(uint32_t (&acc)[32], int jbase, RowState<EPI>& st) {
     if constexpr (EPI == EPI_ARGMIN) {
-        const float m = min32(acc);
+        // The chunk's minimum first; only a thread whose minimum beats its best looks for the column.
+        // That search is kept short (the threads of a warp wait for each other on this branch): the
+        // first group of 8 that holds the minimum, then the first column of that group that equals it,
+        // which is the lowest id among equal keys.
+        const float m0 = min8(acc, 0), m1 = min8(acc, 1), m2 = min8(acc, 2), m3 = min8(acc, 3);
+        const float m = fminf(fminf(m0, m1), fminf(m2, m3));
         if (m < st.tau) {
+            st.tau = m;
+            const bool in0 = (m0 == m), in1 = (m1 == m), in2 = (m2 == m);
+            const int g = in0 ? 0 : (in1 ? 1 : (in2 ? 2 : 3));
+            int idx = 7;
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-                const float key = __uint_as_float(acc[c]);
-                if (key < st.tau) {
-                    st.tau = key;
-                    st.bestj = jbase + c;
-                }
+            for (int i = 6; i >= 0; --i) {
+                const float v = __uint_as_float(in0 ? acc[i] : (in1 ? acc[8 + i] : (in2 ? acc[16 + i] : acc[24 + i])));
+                if (v == m) idx = i;
             }
+            st.bestj = jbase + 8 * g + idx;
         }
     } else if constexpr (EPI == EPI_GROUPS) {
         // One decision per group of 8 columns: if the group's minimum passes the threshold, the
         // whole group (8 raw keys + the id of the first) is appended with two 16-byte stores; the
-        // merge kernel does the per-key comparison.  About 1.4 instructions per key, no branch.
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            asm volatile(
-                "{\n\t.reg .pred p;\n\t.reg .f32 m;\n\t"
-                "min.f32 m, %2, %3, %4;\n\t"
-                "min.f32 m, m, %5, %6;\n\t"
-                "min.f32 m, m, %7, %8;\n\t"
-                "min.f32 m, m, %9;\n\t"
-                "setp.le.f32 p, m, %1;\n\t"
-                "@p st.global.cs.v4.f32 [%0], {%2, %3, %4, %5};\n\t"
-                "@p st.global.cs.v4.f32 [%0+16], {%6, %7, %8, %9};\n\t"
-                "@p st.global.cs.b32 [%0+32], %10;\n\t"
-                "@p add.s64 %0, %0, 48;\n\t}"
-                : "+l"(st.wp)
-                : "f"(st.tau), "f"(__uint_as_float(acc[8 * g])), "f"(__uint_as_float(acc[8 * g + 1])),
-                  "f"(__uint_as_float(acc[8 * g + 2])), "f"(__uint_as_float(acc[8 * g + 3])),
-                  "f"(__uint_as_float(acc[8 * g + 4])), "f"(__uint_as_float(acc[8 * g + 5])),
-                  "f"(__uint_as_float(acc[8 * g + 6])), "f"(__uint_as_float(acc[8 * g + 7])), "r"(jbase + 8 * g)
-                : "memory");
-        }
+        // merge kernel does the per-key comparison.  About 1.2 instructions per key, no branch.  The
+        // four groups of a chunk are written as one block with their minimum chains interleaved:
+        // with two warps per scheduler a chain of dependent instructions is paid in full latency, and
+        // four separate blocks (each waiting for the write pointer of the one before) ran 2.5x slower.
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p0, p1, p2, p3;\n\t.reg .f32 m0, m1, m2, m3;\n\t.reg .b64 w1, w2, w3;\n\t"
+            "min.f32 m0, %2, %3, %4;\n\t"
+            "min.f32 m1, %10, %11, %12;\n\t"
+            "min.f32 m2, %18, %19, %20;\n\t"
+            "min.f32 m3, %26, %27, %28;\n\t"
+            "min.f32 m0, m0, %5, %6;\n\t"
+            "min.f32 m1, m1, %13, %14;\n\t"
+            "min.f32 m2, m2, %21, %22;\n\t"
+            "min.f32 m3, m3, %29, %30;\n\t"
+            "min.f32 m0, m0, %7, %8;\n\t"
+            "min.f32 m1, m1, %15, %16;\n\t"
+            "min.f32 m2, m2, %23, %24;\n\t"
+            "min.f32 m3, m3, %31, %32;\n\t"
+            "min.f32 m0, m0, %9;\n\t"
+            "min.f32 m1, m1, %17;\n\t"
+            "min.f32 m2, m2, %25;\n\t"
+            "min.f32 m3, m3, %33;\n\t"
+            "setp.le.f32 p0, m0, %1;\n\t"
+            "setp.le.f32 p1, m1, %1;\n\t"
+            "setp.le.f32 p2, m2, %1;\n\t"
+            "setp.le.f32 p3, m3, %1;\n\t"
+            "mov.b64 w1, %0;\n\t@p0 add.s64 w1, %0, 48;\n\t"
+            "mov.b64 w2, w1;\n\t@p1 add.s64 w2, w1, 48;\n\t"
+            "mov.b64 w3, w2;\n\t@p2 add.s64 w3, w2, 48;\n\t"
+            "@p0 st.global.cs.v4.f32 [%0], {%2, %3, %4, %5};\n\t"
+            "@p0 st.global.cs.v4.f32 [%0+16], {%6, %7, %8, %9};\n\t"
+            "@p0 st.global.cs.b32 [%0+32], %34;\n\t"
+            "@p1 st.global.cs.v4.f32 [w1], {%10, %11, %12, %13};\n\t"
+            "@p1 st.global.cs.v4.f32 [w1+16], {%14, %15, %16, %17};\n\t"
+            "@p1 st.global.cs.b32 [w1+32], %35;\n\t"
+            "@p2 st.global.cs.v4.f32 [w2], {%18, %19, %20, %21};\n\t"
+            "@p2 st.global.cs.v4.f32 [w2+16], {%22, %23, %24, %25};\n\t"
+            "@p2 st.global.cs.b32 [w2+32], %36;\n\t"
+            "@p3 st.global.cs.v4.f32 [w3], {%26, %27, %28, %29};\n\t"
+            "@p3 st.global.cs.v4.f32 [w3+16], {%30, %31, %32, %33};\n\t"
+            "@p3 st.global.cs.b32 [w3+32], %37;\n\t"
+            "mov.b64 %0, w3;\n\t@p3 add.s64 %0, w3, 48;\n\t}"
+            : "+l"(st.wp)
+            : "f"(st.tau), "f"(__uint_as_float(acc[0])), "f"(__uint_as_float(acc[1])), "f"(__uint_as_float(acc[2])), "f"(__uint_as_float(acc[3])), "f"(__uint_as_float(acc[4])), "f"(__uint_as_float(acc[5])), "f"(__uint_as_float(acc[6])), "f"(__uint_as_float(acc[7])), "f"(__uint_as_float(acc[8])), "f"(__uint_as_float(acc[9])), "f"(__uint_as_float(acc[10])), "f"(__uint_as_float(acc[11])), "f"(__uint_as_float(acc[12])), "f"(__uint_as_float(acc[13])), "f"(__uint_as_float(acc[14])), "f"(__uint_as_float(acc[15])), "f"(__uint_as_float(acc[16])), "f"(__uint_as_float(acc[17])), "f"(__uint_as_float(acc[18])), "f"(__uint_as_float(acc[19])), "f"(__uint_as_float(acc[20])), "f"(__uint_as_float(acc[21])), "f"(__uint_as_float(acc[22])), "f"(__uint_as_float(acc[23])), "f"(__uint_as_float(acc[24])), "f"(__uint_as_float(acc[25])), "f"(__uint_as_float(acc[26])), "f"(__uint_as_float(acc[27])), "f"(__uint_as_float(acc[28])), "f"(__uint_as_float(acc[29])), "f"(__uint_as_float(acc[30])), "f"(__uint_as_float(acc[31])),
+              "r"(jbase), "r"(jbase + 8), "r"(jbase + 16), "r"(jbase + 24)
+            : "memory");
     } else if constexpr (EPI == EPI_FILTER) {
         // Straight-line predicated code on purpose: hits are rare, but 32 rows share every branch,
         // so a branch per column costs more in divergence than the predicated store it would skip.
