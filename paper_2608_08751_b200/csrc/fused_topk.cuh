@@ -645,6 +645,8 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             const uint32_t idesc = umma_idesc_f16(kBlockM, p.block_n);
             const uint32_t a_addr = smem_u32(smem_a);
             const uint32_t b_addr = smem_u32(smem_b);
+            const uint32_t a_slice_step = (kBlockM * kSliceRowBytes) >> 4;
+            const uint32_t b_slice_step = static_cast<uint32_t>(p.block_n * kSliceRowBytes) >> 4;
             int it = 0, seg = 0;
             bool ok = true;
             for (int64_t u = u0; u < u1 && ok;) {
@@ -668,16 +670,21 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                         tc_fence_after_sync();
                         const uint32_t d_tmem = tmem_base + buf * kAccStride;
                         const uint32_t a_tile = a_addr + h * a_bytes;
+                        // The descriptors of consecutive K steps differ only in the start-address field
+                        // (16-byte units, low word): +2 inside a 64-column slice, then on to the next
+                        // slice.  Stepping the low words keeps this thread's work per MMA to a few
+                        // instructions; building each descriptor from scratch took about as long as the
+                        // tensor core needs for the MMA itself.
+                        uint32_t a_lo = umma_desc_lo(a_tile), b_lo = umma_desc_lo(b_stage);
                         for (int kk = 0; kk < p.ksteps; ++kk) {
-                            const int slice = kk >> 2;
-                            const uint32_t off = (kk & 3) * 32;  // 16 fp16 = 32 bytes inside the swizzled row
-                            const uint64_t adesc = umma_desc_sw128(a_tile + slice * kBlockM * kSliceRowBytes + off);
-                            const uint64_t bdesc =
-                                umma_desc_sw128(b_stage + slice * p.block_n * kSliceRowBytes + off);
-                            umma_f16(d_tmem, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
+                            umma_f16(d_tmem, umma_desc_join(a_lo, kDescHiSw128), umma_desc_join(b_lo, kDescHiSw128), idesc,
+                                     kk > 0 ? 1u : 0u);
+                            const bool last_of_slice = (kk & 3) == 3;
+                            a_lo += last_of_slice ? a_slice_step - 6u : 2u;
+                            b_lo += last_of_slice ? b_slice_step - 6u : 2u;
                         }
-                        umma_f16(d_tmem, umma_desc_sw32(a_tile + a_data_bytes), umma_desc_sw32(b_stage + b_data_bytes),
-                                 idesc, 1u);
+                        umma_f16(d_tmem, umma_desc_join(umma_desc_lo(a_tile + a_data_bytes), kDescHiSw32),
+                                 umma_desc_join(umma_desc_lo(b_stage + b_data_bytes), kDescHiSw32), idesc, 1u);
                         umma_commit(&t_full[buf]);
                     }
                     if (!ok) break;

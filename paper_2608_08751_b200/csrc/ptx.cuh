@@ -219,6 +219,17 @@ __device__ __forceinline__ uint64_t umma_desc_sw32(uint32_t smem_addr) {
     return d;
 }
 
+// The two halves of those descriptors: the low word holds the start address (16-byte units) and the
+// unused leading byte offset; the high word is the same for every tile of a layout.
+constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << (46 - 32)) | (2u << (61 - 32));
+constexpr uint32_t kDescHiSw32 = (256u >> 4) | (1u << (46 - 32)) | (6u << (61 - 32));
+__device__ __forceinline__ uint32_t umma_desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ uint64_t umma_desc_join(uint32_t lo, uint32_t hi) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+    return d;
+}
+
 // Instruction descriptor: fp16 A and B, both K-major, fp32 accumulator, tile M x N.
 __host__ __device__ constexpr uint32_t umma_idesc_f16(int M, int N) {
     return (1u << 4)                               // D format fp32
