@@ -385,36 +385,39 @@ __global__ void __launch_bounds__(32 * WARPS) merge_warp_kernel(const MergeParam
         __syncwarp();
     }
 
-    // ---- gather the candidates <= tau_min into the warp's key buffer
+    // ---- gather the candidates <= tau_min into the warp's key buffer.  The loads of the next 32
+    // log entries are issued before the current ones are filtered, so that a row's entries arrive in
+    // one memory round trip after another without the filtering in between.
     int fill = 0;
     if (!pass_on) {
+        float4 na = make_float4(0.f, 0.f, 0.f, 0.f), nb = na;
+        uint32_t nj0 = 0;
+        auto fetch = [&](int idx) {
+            if (idx >= raw_total) return;
+            int lo = 0, hi = ns;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (sm.pre[mid] <= idx) lo = mid; else hi = mid;
+            }
+            const size_t at = (static_cast<size_t>(row) * p.partials + lo) * p.cap + (idx - sm.pre[lo]);
+            if (p.records) {
+                const char* rec = reinterpret_cast<const char*>(p.part) + at * kRecordBytes;
+                na = *reinterpret_cast<const float4*>(rec);
+                nb = *reinterpret_cast<const float4*>(rec + 16);
+                nj0 = *reinterpret_cast<const uint32_t*>(rec + 32);
+            } else {
+                const Entry e = p.part[at];
+                na.x = e.v;
+                nj0 = static_cast<uint32_t>(e.j);
+            }
+        };
+        fetch(lane);
         for (int i0 = 0; i0 < raw_total && !pass_on; i0 += 32) {
             const int idx = i0 + lane;
-            float v[8];
-            uint32_t j0 = 0;
-            int nv = 0;
-            if (idx < raw_total) {
-                int lo = 0, hi = ns;
-                while (hi - lo > 1) {
-                    const int mid = (lo + hi) >> 1;
-                    if (sm.pre[mid] <= idx) lo = mid; else hi = mid;
-                }
-                const size_t at = (static_cast<size_t>(row) * p.partials + lo) * p.cap + (idx - sm.pre[lo]);
-                if (p.records) {
-                    const char* rec = reinterpret_cast<const char*>(p.part) + at * kRecordBytes;
-                    const float4 a = *reinterpret_cast<const float4*>(rec);
-                    const float4 b = *reinterpret_cast<const float4*>(rec + 16);
-                    j0 = *reinterpret_cast<const uint32_t*>(rec + 32);
-                    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
-                    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-                    nv = 8;
-                } else {
-                    const Entry e = p.part[at];
-                    v[0] = e.v;
-                    j0 = static_cast<uint32_t>(e.j);
-                    nv = 1;
-                }
-            }
+            const float v[8] = {na.x, na.y, na.z, na.w, nb.x, nb.y, nb.z, nb.w};
+            const uint32_t j0 = nj0;
+            const int nv = (idx < raw_total) ? (p.records ? 8 : 1) : 0;
+            fetch(idx + 32);
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
                 const bool hit = q < nv && v[q] <= tau_min;
