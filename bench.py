@@ -461,9 +461,24 @@ def main():
         o_ids, o_d, _ = oracle.route(sample, cent_np, NPROBE)
         dt = time.perf_counter() - t0
         g_ids = out_ids.cpu().numpy()[sel]
+        # agreement with the oracle by the stated rule (outside the timed part): an id list may differ
+        # from the oracle's only where the true distances involved lie within 1e-3 (|x|^2 + |c|^2)
+        xn, cn = oracle.sqnorms(sample), oracle.sqnorms(cent_np)
+        rr = np.repeat(np.arange(rows, dtype=np.int64), NPROBE)
+        d_true = oracle.pair_dists(sample, cent_np, rr, g_ids.ravel().astype(np.int64)).reshape(rows, NPROBE)
+        tol_g = 1e-3 * (xn[:, None] + cn[g_ids])
+        tol_o = 1e-3 * (xn[:, None] + cn[o_ids])
+        dk = o_d[:, -1]
+        must = o_d < (dk[:, None] - tol_o)
+        present = (o_ids[:, :, None] == g_ids[:, None, :]).any(-1)
+        differs = g_ids != o_ids
+        row_ok = ((present | ~must).all(axis=1) & (d_true <= dk[:, None] + tol_g).all(axis=1)
+                  & ((np.abs(d_true - o_d) < np.maximum(tol_g, tol_o)) | ~differs).all(axis=1))
         line["cpu_baseline"] = {"value": rows / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"{rows} seeded rows of the C1 routing batch, full centroid width, {dt:.1f} s",
-                                "ids_identical_to_gpu": float((g_ids == o_ids).all(axis=1).mean())}
+                                "rows_matching_oracle_by_tolerance_rule": float(row_ok.mean()),
+                                "rows_with_identical_id_lists": float((~differs).all(axis=1).mean()),
+                                "top_k_set_overlap": float(present.mean())}
     print(json.dumps(line), flush=True)
     if distributed:
         dist.destroy_process_group()
