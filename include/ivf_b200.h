@@ -21,6 +21,10 @@
  *              stream-ordered allocation on `stream`.  Calls that share a device must therefore be
  *              issued in stream order with respect to each other (one stream, or streams the
  *              caller has ordered with events).
+ *   Graphs     a call whose buffers are all device memory enqueues only kernels and memsets once the
+ *              workspace has been sized by an earlier call of the same shape, so it may be captured
+ *              in a CUDA graph by the caller (tested for ivf_assign and ivf_route_prepared); calls
+ *              with page-locked host buffers wait on internal events and are not meant for capture.
  *   Errors     every call returns IVF_OK or a negative ivf_status.  Argument errors are detected
  *              before anything is enqueued.  Device-side problems (a bounded wait that expired, an
  *              id out of range) set a sticky per-device status word that ivf_check reads.

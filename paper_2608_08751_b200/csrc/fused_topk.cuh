@@ -284,6 +284,8 @@ enum { EPI_ARGMIN = 0, EPI_RUNNING = 1, EPI_FILTER = 2, EPI_SKETCH = 3, EPI_GROU
 
 // A record of the group log (EPI_GROUPS): 8 consecutive keys and the id of the first.
 constexpr int kRecordBytes = 48;
+// Records one thread can append between two checks of its log's fill level (one tile: 4 chunks of 4 groups).
+constexpr int kGroupLogMargin = 16;
 
 template <int EPI>
 struct RowState;
@@ -765,7 +767,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                     st[h].base = reinterpret_cast<char*>(p.part) +
                                  (static_cast<size_t>(valid[h] ? row[h] : 0) * p.partials + slot) * p.cap * kRecordBytes;
                     st[h].wp = st[h].base;
-                    st[h].limit = st[h].base + static_cast<size_t>(p.cap - 4) * kRecordBytes;
+                    st[h].limit = st[h].base + static_cast<size_t>(p.cap - kGroupLogMargin) * kRecordBytes;
                     st[h].overflow = 0;
                     if (valid[h]) st[h].tau = p.tau_in[row[h]];
                 }
@@ -788,14 +790,6 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                     // chunk q of this warp starts at column ((q/2) * halves + half) * 64 + (q%2) * 32
                     auto col_of = [&](int q) { return ((q >> 1) * kEpiHalves + half) * 64 + (q & 1) * 32; };
                     auto after_chunk = [&]() {
-                        if constexpr (EPI == EPI_GROUPS) {
-                            // a full log cannot be compacted here (it holds raw groups): the row is
-                            // flagged and recomputed by brute force after the merge
-                            if (st[h].wp > st[h].limit) {
-                                st[h].overflow = 1;
-                                st[h].wp = st[h].base;
-                            }
-                        }
                         if constexpr (kHasLog) {
                             if (__any_sync(0xFFFFFFFFu, st[h].cnt > p.cap - 32)) {
                                 __syncwarp();
@@ -842,6 +836,15 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                             after_chunk();
                             consume<EPI>(accB, tile_j0 + col_of(q + 1), st[h]);
                             after_chunk();
+                        }
+                    }
+                    if constexpr (EPI == EPI_GROUPS) {
+                        // checked once per tile (a tile appends at most 16 records per thread).  A full
+                        // log cannot be compacted here (it holds raw groups): the row is flagged and
+                        // recomputed by brute force after the merge
+                        if (st[h].wp > st[h].limit) {
+                            st[h].overflow = 1;
+                            st[h].wp = st[h].base;
                         }
                     }
                 }

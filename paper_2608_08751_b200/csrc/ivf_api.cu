@@ -538,7 +538,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     if (rc != IVF_OK) return rc;
     const bool given = k > 1 && cp.rule == TAU_GIVEN;
     // given rule: the logs hold 48-byte group records, at most 4k + 4 per (row, slot)
-    if (given) pl.cap = (k <= kSampleM ? 384 : 4 * k) + 4;
+    if (given) pl.cap = (k <= kSampleM ? 384 : 4 * k) + kGroupLogMargin;
     size_t part_bytes = static_cast<size_t>(n) * pl.partials * pl.cap * (given ? kRecordBytes : sizeof(Entry));
     size_t meta_bytes = static_cast<size_t>(n) * pl.partials * sizeof(int2);
     if (given) {

@@ -125,3 +125,44 @@ def test_candidates_and_pq_with_signed_bytes():
     B.ivf_check()
     assert (got[0].cpu().numpy() == want[0]).all() and (got[2].cpu().numpy() == want[2]).all()
     assert (got[1].cpu().numpy().view(np.uint32) == want[1].view(np.uint32)).all()
+
+
+@pytest.mark.parametrize("nq,nlist,k", [(8, 40000, 64), (700, 9000, 1), (300, 3000, 12)])
+def test_calls_can_be_captured_in_a_cuda_graph(nq, nlist, k):
+    """Once the workspace has been sized by a first call of the same shape, a call enqueues only
+    kernels and memsets, so a caller may capture it in a CUDA graph; the replay must give the
+    results of the plain call (and those match the oracle)."""
+    rng = np.random.default_rng(nq + nlist)
+    x = rng.integers(0, 256, (nq, 64)).astype(np.uint8)
+    c = (rng.standard_normal((nlist, 64)) * 30 + 110).astype(np.float32)
+    xt, ct = _t(x), _t(c)
+    h = B.PreparedCentroids(ct)
+    ids = torch.empty((nq, k), dtype=torch.int32, device="cuda")
+    ds = torch.empty((nq, k), dtype=torch.float32, device="cuda")
+
+    def call():
+        if k == 1:
+            B.ivf_assign(xt, ct, ids.view(-1), ds.view(-1))
+        else:
+            B.ivf_route_prepared(h, xt, k, ids, ds)
+
+    call()
+    B.ivf_check()
+    want_ids, want_d = ids.clone(), ds.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        call()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            call()
+    for _ in range(3):
+        ids.zero_()
+        ds.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(ids, want_ids) and torch.equal(ds, want_d)
+    B.ivf_check()
+    parity.check_route(x, c, k, ids.cpu().numpy(), ds.cpu().numpy())
+    h.close()
