@@ -360,9 +360,8 @@ __device__ __forceinline__ void consume(uint32_t (&acc)[32], int jbase, RowState
         // One decision per group of 8 columns: if the group's minimum passes the threshold, the
         // whole group (8 raw keys + the id of the first) is appended with two 16-byte stores; the
         // merge kernel does the per-key comparison.  About 1.2 instructions per key, no branch.  The
-        // four groups of a chunk are written as one block with their minimum chains interleaved:
-        // with two warps per scheduler a chain of dependent instructions is paid in full latency, and
-        // four separate blocks (each waiting for the write pointer of the one before) ran 2.5x slower.
+        // four groups of a chunk are one block: their minimum chains are interleaved and every group
+        // stores through its own pointer (w1..w3 = the write pointer advanced by the groups before).
         asm volatile(
             "{\n\t"
             ".reg .pred p0, p1, p2, p3;\n\t.reg .f32 m0, m1, m2, m3;\n\t.reg .b64 w1, w2, w3;\n\t"
@@ -403,7 +402,15 @@ __device__ __forceinline__ void consume(uint32_t (&acc)[32], int jbase, RowState
             "@p3 st.global.cs.b32 [w3+32], %37;\n\t"
             "mov.b64 %0, w3;\n\t@p3 add.s64 %0, w3, 48;\n\t}"
             : "+l"(st.wp)
-            : "f"(st.tau), "f"(__uint_as_float(acc[0])), "f"(__uint_as_float(acc[1])), "f"(__uint_as_float(acc[2])), "f"(__uint_as_float(acc[3])), "f"(__uint_as_float(acc[4])), "f"(__uint_as_float(acc[5])), "f"(__uint_as_float(acc[6])), "f"(__uint_as_float(acc[7])), "f"(__uint_as_float(acc[8])), "f"(__uint_as_float(acc[9])), "f"(__uint_as_float(acc[10])), "f"(__uint_as_float(acc[11])), "f"(__uint_as_float(acc[12])), "f"(__uint_as_float(acc[13])), "f"(__uint_as_float(acc[14])), "f"(__uint_as_float(acc[15])), "f"(__uint_as_float(acc[16])), "f"(__uint_as_float(acc[17])), "f"(__uint_as_float(acc[18])), "f"(__uint_as_float(acc[19])), "f"(__uint_as_float(acc[20])), "f"(__uint_as_float(acc[21])), "f"(__uint_as_float(acc[22])), "f"(__uint_as_float(acc[23])), "f"(__uint_as_float(acc[24])), "f"(__uint_as_float(acc[25])), "f"(__uint_as_float(acc[26])), "f"(__uint_as_float(acc[27])), "f"(__uint_as_float(acc[28])), "f"(__uint_as_float(acc[29])), "f"(__uint_as_float(acc[30])), "f"(__uint_as_float(acc[31])),
+            : "f"(st.tau),
+              "f"(__uint_as_float(acc[0])), "f"(__uint_as_float(acc[1])), "f"(__uint_as_float(acc[2])), "f"(__uint_as_float(acc[3])),
+              "f"(__uint_as_float(acc[4])), "f"(__uint_as_float(acc[5])), "f"(__uint_as_float(acc[6])), "f"(__uint_as_float(acc[7])),
+              "f"(__uint_as_float(acc[8])), "f"(__uint_as_float(acc[9])), "f"(__uint_as_float(acc[10])), "f"(__uint_as_float(acc[11])),
+              "f"(__uint_as_float(acc[12])), "f"(__uint_as_float(acc[13])), "f"(__uint_as_float(acc[14])), "f"(__uint_as_float(acc[15])),
+              "f"(__uint_as_float(acc[16])), "f"(__uint_as_float(acc[17])), "f"(__uint_as_float(acc[18])), "f"(__uint_as_float(acc[19])),
+              "f"(__uint_as_float(acc[20])), "f"(__uint_as_float(acc[21])), "f"(__uint_as_float(acc[22])), "f"(__uint_as_float(acc[23])),
+              "f"(__uint_as_float(acc[24])), "f"(__uint_as_float(acc[25])), "f"(__uint_as_float(acc[26])), "f"(__uint_as_float(acc[27])),
+              "f"(__uint_as_float(acc[28])), "f"(__uint_as_float(acc[29])), "f"(__uint_as_float(acc[30])), "f"(__uint_as_float(acc[31])),
               "r"(jbase), "r"(jbase + 8), "r"(jbase + 16), "r"(jbase + 24)
             : "memory");
     } else if constexpr (EPI == EPI_FILTER) {
