@@ -721,6 +721,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         const float INF = __int_as_float(0x7f800000);
         const int nq = p.block_n / 64;  // 32-column chunks per warp and tile: 4 or 2
         constexpr bool kHasLog = (EPI == EPI_RUNNING || EPI == EPI_FILTER);
+        constexpr bool kWideLoads = (EPI == EPI_ARGMIN);
         float raw_scales[4] = {1.f, 1.f, 1.f, 1.f};
         if (p.x_raw != nullptr) {
             compute_scales(p.bits, 1, raw_scales);
@@ -821,6 +822,38 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                     // as two 32-column loads issued back to back; the other epilogue warp of the
                     // scheduler computes meanwhile.
                     uint32_t accA[32], accB[32];
+                    if (kWideLoads && nq == 4) {
+                        // All 128 columns of this warp in one round trip, so that the accumulator goes
+                        // back to the MMA warp one load latency after it was filled: the MMA-issuing
+                        // thread cannot run far ahead of the tensor core, and every cycle it waits for a
+                        // free accumulator is a cycle the tensor core idles.
+                        uint32_t accC[32], accD[32];
+                        tmem_ld_32x32b_x32(taddr + col_of(0), accA);
+                        tmem_ld_32x32b_x32(taddr + col_of(1), accB);
+                        tmem_ld_32x32b_x32(taddr + col_of(2), accC);
+                        tmem_ld_32x32b_x32(taddr + col_of(3), accD);
+                        tmem_wait_ld_regs(accA);
+                        tmem_wait_ld_regs(accB);
+                        tmem_wait_ld_regs(accC);
+                        tmem_wait_ld_regs(accD);
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&t_empty[buf]);
+                        if (ragged) {
+                            mask_ragged(accA, tile_j0 + col_of(0), p.nlist);
+                            mask_ragged(accB, tile_j0 + col_of(1), p.nlist);
+                            mask_ragged(accC, tile_j0 + col_of(2), p.nlist);
+                            mask_ragged(accD, tile_j0 + col_of(3), p.nlist);
+                        }
+                        consume<EPI>(accA, tile_j0 + col_of(0), st[h]);
+                        after_chunk();
+                        consume<EPI>(accB, tile_j0 + col_of(1), st[h]);
+                        after_chunk();
+                        consume<EPI>(accC, tile_j0 + col_of(2), st[h]);
+                        after_chunk();
+                        consume<EPI>(accD, tile_j0 + col_of(3), st[h]);
+                        after_chunk();
+                    } else {
 #pragma unroll
                     for (int q = 0; q < 4; q += 2) {
                         if (q < nq) {
@@ -844,6 +877,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                             consume<EPI>(accB, tile_j0 + col_of(q + 1), st[h]);
                             after_chunk();
                         }
+                    }
                     }
                     if constexpr (EPI == EPI_GROUPS) {
                         // checked once per tile (a tile appends at most 16 records per thread).  A full
