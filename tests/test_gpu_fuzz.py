@@ -155,3 +155,24 @@ def test_route_mixed_magnitudes_between_points_and_centroids():
         ids, dists = B.ivf_route(_t(x), _t(c), 12)
         B.ivf_check()
         parity.check_route(x, c, 12, ids.cpu().numpy(), dists.cpu().numpy())
+
+
+@pytest.mark.parametrize("dtype,n,nlist,d,k", [
+    ("u8", 2500, 4096, 32, 1), ("i8", 5000, 9000, 64, 1), ("u8", 1000, 40000, 16, 1),
+    ("u8", 700, 4096, 128, 64), ("i8", 300, 1000, 100, 20),
+])
+def test_duplicate_centroids_lower_id_wins(dtype, n, nlist, d, k):
+    """A third of the centroids are copies of other centroids, on integer data whose distances are
+    exact: every tie between a centroid and its copy (in the same 8-column group, in another group of
+    the same accumulator chunk, in another chunk, tile or CTA) must go to the lower id, as in the
+    oracle's sort."""
+    rng = np.random.default_rng(n + nlist + d + k)
+    x = _points(rng, dtype, n, d, True)
+    c = _centroids(rng, dtype, nlist, d, True)
+    c[rng.integers(0, nlist, nlist // 3)] = c[rng.integers(0, nlist, nlist // 3)]
+    if k == 1:
+        ids, dists = B.ivf_assign(_t(x), _t(c))
+    else:
+        ids, dists = B.ivf_route(_t(x), _t(c), k)
+    B.ivf_check()
+    parity.check_route(x, c, k, ids.cpu().numpy(), dists.cpu().numpy(), exact=True)
