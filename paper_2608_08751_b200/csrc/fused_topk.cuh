@@ -429,6 +429,13 @@ __device__ __forceinline__ void consume(uint32_t (&acc)[32], int jbase, RowState
                 : "memory");
         }
         st.cnt = static_cast<int>(wp - st.log);
+    } else if constexpr (EPI == EPI_SKETCH) {
+        // Threshold pass: the statistic is the minimum of each chunk of 32 keys, one network
+        // insertion per chunk; tau will be the 16th smallest chunk minimum of the row, so at least 16
+        // sampled keys are <= tau.  (With one insertion per group of 8 this epilogue cost four times
+        // the group-record one, because some row of the warp needs nearly every insertion.)
+        const float m = fminf(fminf(min8(acc, 0), min8(acc, 1)), fminf(min8(acc, 2), min8(acc, 3)));
+        if (__any_sync(0xFFFFFFFFu, m < st.net[kSampleM - 1])) network_insert(st.net, m);
     } else {
         // the sample statistic is the minimum of each group of 8 keys: one network insertion per
         // group.  tau = the 16th smallest group minimum, so at least 16 keys are <= tau.
