@@ -89,6 +89,7 @@ struct FusedParams {
     float* xn_out;        // x_raw mode: |x|^2 per row
     int* clear0;          // two optional words that block 0 sets to zero (list counters of the merge)
     int* clear1;
+    int* clear32;         // optional: 32 more words for block 0 to clear (work counters of the call's tail kernel)
     int* status;          // sticky device status word
     unsigned long long* stats;  // optional counters: [0] in-kernel selections, [1] log entries written
     uint64_t wait_limit_ns;
@@ -579,6 +580,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         if (p.clear0) *p.clear0 = 0;
         if (p.clear1) *p.clear1 = 0;
     }
+    if (threadIdx.x < 32 && blockIdx.x == 0 && p.clear32) p.clear32[threadIdx.x] = 0;
 
     WaitCtl ctl;
     ctl.abort_flag = abort_flag;

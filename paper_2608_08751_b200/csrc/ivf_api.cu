@@ -61,8 +61,8 @@ int fail(int code, const char* fmt, ...) {
 // Kernels of the routing path begin with griddepcontrol.wait, so they may be launched with the
 // programmatic-serialization attribute: the launch latency and the kernel's own set-up then overlap
 // the end of the kernel before it.  g_pdl = 0 falls back to ordinary launches (test hook).
-// Bit per kernel family: 1 prep, 2 fused, 4 threshold merge, 8 merge, 16 merge of passed-on rows,
-// 32 recomputation.  Measured: letting the fused kernel or the threshold merge start early costs time
+// Bit per kernel family: 1 prep, 2 fused, 4 threshold merge, 8 merge, 16 tail kernel (passed-on rows
+// and recomputation; 32 unused).  Measured: letting the fused kernel or the threshold merge start early costs time
 // (their waiting warps sit next to the running kernel), the other families gain 6-9 us per call.
 int g_pdl = 57;
 template <typename... KArgs, typename... Args>
@@ -224,7 +224,6 @@ struct Plan {
 };
 
 constexpr size_t kSmemLimit = 227 * 1024;
-constexpr int kFallbackCtas = 32;  // slow-path CTAs of the brute-force recomputation
 inline int fallback_slices(int nlist) { return (nlist + kFallbackSlice - 1) / kFallbackSlice; }
 
 int log_capacity(int k) { return (k == 1) ? 1 : (4 * k > 512 ? 4 * k : 512); }
@@ -441,10 +440,11 @@ struct PointPrep {
 int launch_fused(DeviceCtx& ctx, const Plan& pl, int64_t n, int nlist, int k, int rule, const float* tau_in,
                  const PointPrep& pp, const CUtensorMap& tmap_c, const CUtensorMap& tmap_ca, Entry* part,
                  int2* part_meta, int kind, cudaStream_t stream, const unsigned int* bits, float* scal,
-                 int* clear0 = nullptr, int* clear1 = nullptr) {
+                 int* clear0 = nullptr, int* clear1 = nullptr, int* clear32 = nullptr) {
     FusedParams fp;
     fp.clear0 = clear0;
     fp.clear1 = clear1;
+    fp.clear32 = clear32;
     fp.x_raw = pp.x_raw;
     fp.d = pp.d;
     fp.bits = bits;
@@ -566,7 +566,8 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     WS(WS_PART, part_bytes, part);
     if (k > 1) {
         WS(WS_PARTMETA, meta_bytes, part_meta);
-        WS(WS_FAIL, 2 * (static_cast<size_t>(n) + 2) * sizeof(int), failbuf);  // failed rows and passed-on rows
+        // failed rows, passed-on rows, and the work counters of the tail kernel
+        WS(WS_FAIL, (2 * (static_cast<size_t>(n) + 2) + kTailSyncWords) * sizeof(int), failbuf);
         if (given || g_force_fallback) WS(WS_FBKEYS, static_cast<size_t>(kFallbackFastRows + kFallbackCtas) * fallback_slices(nlist) * k * sizeof(uint64_t), fbkeys);
         if (given) WS(WS_TAU, static_cast<size_t>(n) * sizeof(float), tau);
     }
@@ -623,7 +624,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     }
     rc = launch_fused(ctx, pl, n, nlist, k, cp.rule, tau, pp, cp.tmap_c, cp.tmap_ca, part, part_meta,
                       k == 1 ? TK_FUSED_ARGMIN : TK_FUSED_TOPK, stream, cp.bits, cp.scal, failbuf,
-                      failbuf ? failbuf + n + 2 : nullptr);
+                      failbuf ? failbuf + n + 2 : nullptr, failbuf ? failbuf + 2 * (n + 2) : nullptr);
     if (rc != IVF_OK) return rc;
 
     MergeParams mp = merge_params(pl, n, k, part, part_meta, pp, cp.scal);
@@ -654,7 +655,11 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
                                           static_cast<int>(4 * sizeof(MergeWarpSmem<2048>))));
             ctx.merge_attr_set = true;
         }
-        if (expect <= 340) {
+        if (pl.partials > kWarpSlots) {
+            // (small batches: every CTA of the fused kernel shared the one row group, so every row has
+            // more partial logs than the warp-level kernel takes -- all rows go to the tail kernel)
+            mp.big = nullptr;
+        } else if (expect <= 340) {
             LAUNCH_DEP(8, (merge_warp_kernel<512, 256, 8>), static_cast<unsigned>((n + 7) / 8), 256, 8 * sizeof(MergeWarpSmem<512>), stream, mp);
         } else if (expect <= 700) {
             LAUNCH_DEP(8, (merge_warp_kernel<1024, 512, 8>), static_cast<unsigned>((n + 7) / 8), 256, 8 * sizeof(MergeWarpSmem<1024>), stream, mp);
@@ -664,11 +669,14 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
             mp.big = nullptr;
         }
         {
-            const int64_t grid = n < 8 * static_cast<int64_t>(ctx.num_sms) ? n : 8 * static_cast<int64_t>(ctx.num_sms);
-            LAUNCH_DEP(16, merge_select_kernel, static_cast<unsigned>(grid), kMergeThreads, 0, stream, mp);
-        }
-        if (given || g_force_fallback) {
-            FallbackParams fb;
+            // one launch for everything that is rarely needed: rows the warp-level kernel passed on,
+            // then the brute-force recomputation of rows whose threshold admitted too few candidates
+            TailParams tp;
+            tp.mp = mp;
+            tp.sync = failbuf + 2 * (n + 2);
+            tp.status = ctx.status;
+            tp.fallback = (given || g_force_fallback) ? 1 : 0;
+            FallbackParams& fb = tp.fb;
             fb.nlist = nlist;
             fb.k = k;
             fb.kp = pl.kp;
@@ -684,8 +692,10 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
             fb.slices = fallback_slices(nlist);
             fb.out_ids = out_ids;
             fb.out_dists = out_dists;
-            LAUNCH_DEP(32, fallback_keys_kernel, dim3(static_cast<unsigned>(fb.slices), kFallbackFastRows), kFallbackThreads, 0, stream, fb);
-            LAUNCH_DEP(32, fallback_select_kernel, kFallbackFastRows + kFallbackCtas, kFallbackThreads, 0, stream, fb);
+            const int64_t most = (mp.big ? 2 : 8) * static_cast<int64_t>(ctx.num_sms);
+            int64_t grid = mp.big ? most : (n < most ? n : most);
+            if (grid < kFallbackCtas) grid = kFallbackCtas;
+            LAUNCH_DEP(16, route_tail_kernel, static_cast<unsigned>(grid), kMergeThreads, 0, stream, tp);
         }
     }
     timing_end(tk, stream);

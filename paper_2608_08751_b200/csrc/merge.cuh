@@ -108,24 +108,30 @@ __device__ __forceinline__ void merge_fail_row(const MergeParams& p, int64_t row
     if (p.stats) atomicAdd(&p.stats[2], 1ull);
 }
 
-// k > 1, general path: one CTA per row.  The row's logs are read as one flattened array (all loads
-// in flight together); candidates <= the row's smallest tau are sorted by the 64-bit key (orderable
-// value, id) in shared memory; more than kSortCap raw entries are folded in rounds.  If p.big is
-// set the CTAs walk that list of rows (the rows the warp-level kernel passed on) instead of all.
-__global__ void __launch_bounds__(kMergeThreads) merge_select_kernel(const MergeParams p) {
-    pdl_wait();
-    pdl_trigger();
-    __shared__ uint64_t keys[kSortCap];
-    __shared__ int pre[kMaxSlots + 1];  // exclusive prefix of the slots' entry counts
-    __shared__ float s_tau[kMergeThreads / 32];
-    __shared__ int hist[256];
-    __shared__ int s_wcnt[kMergeThreads / 32];
-    __shared__ int s_sel[2];
-    __shared__ int s_fill;
+// k > 1, general path: one CTA per row (a device function of route_tail_kernel).  The row's logs are
+// read as one flattened array (all loads in flight together); candidates <= the row's smallest tau
+// are sorted by the 64-bit key (orderable value, id) in shared memory; more than kSortCap raw entries
+// are folded in rounds.
+struct SelectSmem {
+    uint64_t keys[kSortCap];
+    int pre[kMaxSlots + 1];  // exclusive prefix of the slots' entry counts
+    float s_tau[kMergeThreads / 32];
+    int hist[256];
+    int s_wcnt[kMergeThreads / 32];
+    int s_sel[2];
+    int s_fill;
+};
+
+__device__ __forceinline__ void merge_select_row(const MergeParams& p, int64_t row, SelectSmem& sm) {
+    uint64_t* const keys = sm.keys;
+    int* const pre = sm.pre;
+    float* const s_tau = sm.s_tau;
+    int* const hist = sm.hist;
+    int* const s_wcnt = sm.s_wcnt;
+    int* const s_sel = sm.s_sel;
+    int& s_fill = sm.s_fill;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t nrows = p.big ? p.big[0] : p.n;
-    for (int64_t item = blockIdx.x; item < nrows; item += gridDim.x) {
-        const int64_t row = p.big ? p.big[1 + item] : item;
+    {
         const int ns = min(slots_of_row_tile(p, row / p.group_rows), kMaxSlots);
         const Entry* base = p.part + static_cast<size_t>(row) * p.partials * p.cap;
         const int2* meta = p.part_meta + static_cast<size_t>(row) * p.partials;
@@ -291,15 +297,9 @@ __global__ void __launch_bounds__(kMergeThreads) merge_select_kernel(const Merge
             __syncthreads();
         }
         overflowed = __syncthreads_or(overflowed);
-        if (p.tau_out) {
-            if (threadIdx.x == 0)
-                p.tau_out[row] = kept >= kSampleM ? from_orderable(static_cast<uint32_t>(keys[kSampleM - 1] >> 32))
-                                                  : __int_as_float(0x7f800000);
-            continue;
-        }
         if (total < p.k || p.force_fail || overflowed) {
             if (threadIdx.x == 0) merge_fail_row(p, row);
-            continue;
+            return;
         }
         merge_write_row(p, row, keys, threadIdx.x, blockDim.x);
     }
@@ -308,7 +308,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_select_kernel(const Merge
 // k > 1, fast path: one WARP per row, no block-wide barriers.  Serves rows with at most kWarpSlots
 // partial logs and at most kWarpKeys candidates <= tau: the candidates go to the warp's slice of
 // shared memory, an 8-bit radix select on the key's value finds the k-th smallest, and only the
-// keys up to it are sorted.  Other rows are appended to p.big for merge_select_kernel.
+// keys up to it are sorted.  Other rows are appended to p.big for route_tail_kernel.
 constexpr int kWarpSlots = 64;
 
 // Two sizes: KEYS candidates per row at most, SORT keys sorted at most, WARPS rows per CTA.
@@ -385,10 +385,51 @@ __global__ void __launch_bounds__(32 * WARPS) merge_warp_kernel(const MergeParam
         __syncwarp();
     }
 
+    // ---- k-th smallest value of keys[0 .. fill) by radix select, then everything up to it moved to
+    // the front (ties all stay); returns how many were kept.  Used when the buffer fills up during
+    // the gather and once at the end.
+    auto keep_k_smallest = [&](int fill) -> int {
+        uint32_t prefix = 0, mask = 0;
+        int r = p.k, eq = 0;
+#pragma unroll 1
+        for (int shift = 24; shift >= 0; shift -= 8) {
+            for (int i = lane; i < 256; i += 32) sm.hist[i] = 0;
+            __syncwarp();
+            for (int i = lane; i < fill; i += 32) {
+                const uint32_t u = static_cast<uint32_t>(sm.keys[i] >> 32);
+                if ((u & mask) == prefix) atomicAdd(&sm.hist[(u >> shift) & 255u], 1);
+            }
+            __syncwarp();
+            const int digit = radix_pick_digit(sm.hist, lane, r, eq);
+            prefix |= static_cast<uint32_t>(digit) << shift;
+            mask |= 255u << shift;
+            __syncwarp();
+        }
+        int outp = 0;
+        for (int i0 = 0; i0 < fill; i0 += 32) {
+            const int i = i0 + lane;
+            uint64_t key = 0;
+            bool keep = false;
+            if (i < fill) {
+                key = sm.keys[i];
+                keep = static_cast<uint32_t>(key >> 32) <= prefix;
+            }
+            const uint32_t bal = __ballot_sync(FULL, keep);
+            __syncwarp();
+            if (keep) sm.keys[outp + __popc(bal & lt_mask)] = key;
+            outp += __popc(bal);
+        }
+        __syncwarp();
+        return outp;
+    };
+
     // ---- gather the candidates <= tau_min into the warp's key buffer.  The loads of the next 32
     // log entries are issued before the current ones are filtered, so that a row's entries arrive in
-    // one memory round trip after another without the filtering in between.
-    int fill = 0;
+    // one memory round trip after another without the filtering in between.  A batch that does not fit
+    // (a row with several times the usual number of candidates) is filtered again after the buffer
+    // has been cut down to the k smallest so far; only a row whose ties fill the buffer is passed on.
+    int fill = 0;    // keys in the buffer
+    int total = 0;   // candidates <= tau_min seen (the exactness test needs at least k)
     if (!pass_on) {
         float4 na = make_float4(0.f, 0.f, 0.f, 0.f), nb = na;
         uint32_t nj0 = 0;
@@ -418,63 +459,45 @@ __global__ void __launch_bounds__(32 * WARPS) merge_warp_kernel(const MergeParam
             const uint32_t j0 = nj0;
             const int nv = (idx < raw_total) ? (p.records ? 8 : 1) : 0;
             fetch(idx + 32);
+            for (int attempt = 0; attempt < 2; ++attempt) {
+                int f = fill;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                const bool hit = q < nv && v[q] <= tau_min;
-                const uint32_t bal = __ballot_sync(FULL, hit);
-                if (bal) {
-                    const int at = fill + __popc(bal & lt_mask);
-                    if (hit && at < kWarpKeys) sm.keys[at] = (static_cast<uint64_t>(orderable(v[q])) << 32) | (j0 + q);
-                    fill += __popc(bal);
+                for (int q = 0; q < 8; ++q) {
+                    const bool hit = q < nv && v[q] <= tau_min;
+                    const uint32_t bal = __ballot_sync(FULL, hit);
+                    if (bal) {
+                        const int at = f + __popc(bal & lt_mask);
+                        if (hit && at < kWarpKeys) sm.keys[at] = (static_cast<uint64_t>(orderable(v[q])) << 32) | (j0 + q);
+                        f += __popc(bal);
+                    }
+                    if (!p.records) break;
                 }
-                if (!p.records) break;
+                if (f <= kWarpKeys) {
+                    total += f - fill;
+                    fill = f;
+                    break;
+                }
+                // the batch did not fit: cut the buffer down (the batch's keys written so far are
+                // dropped with it) and filter the batch once more
+                __syncwarp();
+                if (attempt == 1 || fill <= p.k) {
+                    pass_on = true;
+                    break;
+                }
+                fill = keep_k_smallest(fill);
+                if (fill + 256 > kWarpKeys) pass_on = true;  // ties: no room for a worst-case batch
+                if (pass_on) break;
             }
-            if (fill > kWarpKeys) pass_on = true;
         }
         __syncwarp();
     }
-    if (!pass_on && fill < p.k) {  // too few candidates: the threshold was too tight for this row
+    if (!pass_on && total < p.k) {  // too few candidates: the threshold was too tight for this row
         if (lane == 0) merge_fail_row(p, row);
         return;
     }
 
-    // ---- k-th smallest value by radix select, then keep everything up to it
     int kept = fill;
-    if (!pass_on && fill > 2 * p.k) {
-        uint32_t prefix = 0, mask = 0;
-        int r = p.k, eq = 0;
-#pragma unroll 1
-        for (int shift = 24; shift >= 0; shift -= 8) {
-            for (int i = lane; i < 256; i += 32) sm.hist[i] = 0;
-            __syncwarp();
-            for (int i = lane; i < fill; i += 32) {
-                const uint32_t u = static_cast<uint32_t>(sm.keys[i] >> 32);
-                if ((u & mask) == prefix) atomicAdd(&sm.hist[(u >> shift) & 255u], 1);
-            }
-            __syncwarp();
-            const int digit = radix_pick_digit(sm.hist, lane, r, eq);
-            prefix |= static_cast<uint32_t>(digit) << shift;
-            mask |= 255u << shift;
-            __syncwarp();
-        }
-        // compact the keys whose value is <= the k-th smallest to the front (ties all stay)
-        int outp = 0;
-        for (int i0 = 0; i0 < fill; i0 += 32) {
-            const int i = i0 + lane;
-            uint64_t key = 0;
-            bool keep = false;
-            if (i < fill) {
-                key = sm.keys[i];
-                keep = static_cast<uint32_t>(key >> 32) <= prefix;
-            }
-            const uint32_t bal = __ballot_sync(FULL, keep);
-            __syncwarp();
-            if (keep) sm.keys[outp + __popc(bal & lt_mask)] = key;
-            outp += __popc(bal);
-        }
-        __syncwarp();
-        kept = outp;
-    }
+    if (!pass_on && fill > 2 * p.k) kept = keep_k_smallest(fill);
     if (!pass_on && kept > kWarpSort) pass_on = true;  // very many ties: let the general path sort
     if (pass_on) {
         if (lane == 0) {
@@ -758,40 +781,127 @@ __device__ __forceinline__ void fallback_finish_row(const FallbackParams& p, con
     __syncthreads();
 }
 
-// The first kFallbackFastRows failed rows: grid (slices, kFallbackFastRows), one slice of one row per CTA.
-__global__ void __launch_bounds__(kFallbackThreads) fallback_keys_kernel(const FallbackParams p) {
-    pdl_wait();
-    pdl_trigger();
-    __shared__ FallbackSmem sm;
-    const int nfail = p.fail[0];
-    const int idx = blockIdx.y;
-    if (idx >= nfail) return;
-    fallback_load_point(p, p.fail[1 + idx], sm.xs);
-    __syncthreads();
-    fallback_slice(p, blockIdx.x, p.cand + (static_cast<size_t>(idx) * p.slices + blockIdx.x) * p.k, sm);
+// ------------------------------------------------------------------ tail of a routing call
+// Everything that is rarely needed after the warp-level merge, as ONE launch (three launches that
+// found nothing to do cost 19 us per call, a quarter of a small serving batch):
+//   A. rows the warp-level kernel passed on (many partial logs, many candidates or ties) are merged
+//      by one CTA each (merge_select_row); with p.big == nullptr every row goes this way;
+//   B. rows whose threshold admitted fewer than k candidates (found by the warp-level kernel or in A)
+//      are recomputed by brute force: the first kFallbackFastRows of them slice by slice over the
+//      whole grid, the CTA that finishes a row's last slice also finishes the row; any further rows
+//      by one CTA each (blocks below kFallbackCtas).
+// Work is dealt through counters in global memory (`sync`, cleared by the fused kernel): [0] next
+// item of A, [1] items of A done, [2] next (row, slice) item of B, [3] next whole-row item of B,
+// [4 + i] slices of fast row i done.  B may only start when every item of A is done (A appends to the
+// list of failed rows); a CTA that finds no item of A left waits for that -- for CTAs that are
+// running, never for CTAs yet to be scheduled -- with a time limit, after which it records a timeout
+// in the status word and returns.  When both lists are empty a CTA reads two words and exits.
+constexpr int kTailSyncWords = 32;
+constexpr int kFallbackCtas = 32;  // CTAs that take whole rows beyond the fast ones
+
+struct TailParams {
+    MergeParams mp;
+    FallbackParams fb;
+    int* sync;
+    int* status;
+    int fallback;  // 0: the logs are exact by construction (no recomputation stage)
+};
+
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
 
-// Blocks [0, kFallbackFastRows) finish the rows whose candidates fallback_keys_kernel prepared.  The
-// other blocks take any further failed rows (none in practice), one CTA per row doing both stages.
-__global__ void __launch_bounds__(kFallbackThreads) fallback_select_kernel(const FallbackParams p) {
+__global__ void __launch_bounds__(kMergeThreads) route_tail_kernel(const TailParams t) {
     pdl_wait();
     pdl_trigger();
-    __shared__ FallbackSmem sm;
-    const int nfail = p.fail[0];
-    if (blockIdx.x < kFallbackFastRows) {
-        const int idx = blockIdx.x;
-        if (idx < nfail) fallback_finish_row(p, p.cand + static_cast<size_t>(idx) * p.slices * p.k, p.fail[1 + idx], sm);
-        return;
+    static_assert(kMergeThreads == kFallbackThreads, "one block size for both stages");
+    constexpr size_t kSmem = sizeof(SelectSmem) > sizeof(FallbackSmem) ? sizeof(SelectSmem) : sizeof(FallbackSmem);
+    __shared__ __align__(16) unsigned char raw[kSmem];
+    __shared__ int s_item, s_flag;
+    auto next_item = [&](int* ctr) {
+        __syncthreads();
+        if (threadIdx.x == 0) s_item = atomicAdd(ctr, 1);
+        __syncthreads();
+        return s_item;
+    };
+
+    // ---- A
+    const MergeParams& p = t.mp;
+    const int64_t nbig = p.big ? __ldcg(p.big) : p.n;
+    if (nbig > 0) {
+        SelectSmem& sel = *reinterpret_cast<SelectSmem*>(raw);
+        for (;;) {
+            const int64_t item = next_item(&t.sync[0]);
+            if (item >= nbig) break;
+            merge_select_row(p, p.big ? __ldcg(p.big + 1 + item) : item, sel);
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) atomicAdd(&t.sync[1], 1);
+        }
+        if (t.fallback) {
+            if (threadIdx.x == 0) {
+                const uint64_t t_start = global_timer_ns();
+                int ok = 1;
+                while (ld_acquire_gpu(&t.sync[1]) < nbig) {
+                    if (global_timer_ns() - t_start > 4000000000ull) {
+                        ok = 0;
+                        break;
+                    }
+                    __nanosleep(200);
+                }
+                if (!ok && atomicCAS(t.status, 0, kStatusTimeout) == 0) {
+                    t.status[1] = 20;
+                    t.status[2] = static_cast<int>(blockIdx.x);
+                }
+                s_flag = ok;
+            }
+            __syncthreads();
+            if (!s_flag) return;
+        }
     }
-    const int slow = blockIdx.x - kFallbackFastRows, nslow = gridDim.x - kFallbackFastRows;
-    uint64_t* cand = p.cand + static_cast<size_t>(kFallbackFastRows + slow) * p.slices * p.k;
-    for (int idx = kFallbackFastRows + slow; idx < nfail; idx += nslow) {
-        const int64_t row = p.fail[1 + idx];
+    if (!t.fallback) return;
+
+    // ---- B
+    const FallbackParams& f = t.fb;
+    const int nfail = ld_acquire_gpu(f.fail);
+    if (nfail == 0) return;
+    FallbackSmem& sm = *reinterpret_cast<FallbackSmem*>(raw);
+    const int nfast = min(nfail, kFallbackFastRows);
+    const int items = nfast * f.slices;
+    int loaded = -1;
+    for (;;) {
+        const int item = next_item(&t.sync[2]);
+        if (item >= items) break;
+        const int idx = item / f.slices, slice = item - idx * f.slices;
+        const int64_t row = __ldcg(f.fail + 1 + idx);
+        if (idx != loaded) {
+            fallback_load_point(f, row, sm.xs);
+            loaded = idx;
+            __syncthreads();
+        }
+        fallback_slice(f, slice, f.cand + (static_cast<size_t>(idx) * f.slices + slice) * f.k, sm);
+        __threadfence();
         __syncthreads();
-        fallback_load_point(p, row, sm.xs);
+        if (threadIdx.x == 0) s_flag = atomicAdd(&t.sync[4 + idx], 1) == f.slices - 1;
         __syncthreads();
-        for (int s = 0; s < p.slices; ++s) fallback_slice(p, s, cand + static_cast<size_t>(s) * p.k, sm);
-        fallback_finish_row(p, cand, row, sm);
+        if (s_flag) {  // this CTA finished the row's last slice: every slice's candidates are visible now
+            __threadfence();
+            fallback_finish_row(f, f.cand + static_cast<size_t>(idx) * f.slices * f.k, row, sm);
+        }
+    }
+    if (nfail > kFallbackFastRows && blockIdx.x < kFallbackCtas) {
+        uint64_t* cand = f.cand + static_cast<size_t>(kFallbackFastRows + blockIdx.x) * f.slices * f.k;
+        for (;;) {
+            const int idx = kFallbackFastRows + next_item(&t.sync[3]);
+            if (idx >= nfail) break;
+            const int64_t row = __ldcg(f.fail + 1 + idx);
+            fallback_load_point(f, row, sm.xs);
+            __syncthreads();
+            for (int s2 = 0; s2 < f.slices; ++s2) fallback_slice(f, s2, cand + static_cast<size_t>(s2) * f.k, sm);
+            fallback_finish_row(f, cand, row, sm);
+        }
     }
 }
 

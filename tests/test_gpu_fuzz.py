@@ -176,3 +176,24 @@ def test_duplicate_centroids_lower_id_wins(dtype, n, nlist, d, k):
         ids, dists = B.ivf_route(_t(x), _t(c), k)
     B.ivf_check()
     parity.check_route(x, c, k, ids.cpu().numpy(), dists.cpu().numpy(), exact=True)
+
+
+@pytest.mark.parametrize("cluster,k", [(700, 64), (1500, 64), (3000, 128), (300, 20)])
+def test_rows_with_many_times_the_usual_candidates(cluster, k):
+    """A tight cluster of centroids sits next to some of the queries, at positions the threshold
+    pass does not sample (it looks at every S-th centroid), so those rows' thresholds admit the whole
+    cluster: several times the usual number of candidates reach the merge, which has to cut its
+    buffer down in mid-gather (or hand the row to the general path) and still return the exact lists."""
+    rng = np.random.default_rng(cluster + k)
+    nlist, d, n = 32768, 32, 600
+    c = (rng.standard_normal((nlist, d)) * 30 + 100).astype(np.float32)
+    x = rng.integers(0, 256, (n, d)).astype(np.uint8)
+    centre = x[0].astype(np.float32)
+    stride = 64 if cluster <= nlist // 64 else 8
+    where = np.flatnonzero(np.arange(nlist) % stride == 5)[:cluster]
+    c[where] = centre + rng.standard_normal((where.size, d)).astype(np.float32) * 2.0
+    x[:200] = np.clip(centre + rng.standard_normal((200, d)) * 3.0, 0, 255).astype(np.uint8)
+    ids, dists = B.ivf_route(_t(x), _t(c), k)
+    B.ivf_check()
+    stats = parity.check_route(x, c, k, ids.cpu().numpy(), dists.cpu().numpy())
+    assert stats["rows"] == n
