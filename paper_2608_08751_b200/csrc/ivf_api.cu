@@ -643,8 +643,10 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         // (both list counters were cleared by the fused kernel that just ran)
         mp.big = failbuf + n + 2;
         // three sizes of the warp-level kernel (the smaller the key buffer, the more warps per SM): up to
-        // 512 candidates / 256 sorted (k <= 68 under the given rule), 1024 / 512 (k <= 140), 2048 / 1024
-        // (k <= 340); beyond that everything goes to the general kernel
+        // 512 candidates in the buffer / 256 sorted (k <= 68 under the given rule), 1024 / 512 (k <= 280;
+        // a row with more candidates than fit is cut down to its k smallest in mid-gather, which for
+        // k = 256 costs less than the lower occupancy of the next size: C4 chunk 0.52 -> 0.40 ms),
+        // 2048 / 1024 (k <= 340); beyond that everything goes to the general path of the tail kernel
         const int expect = given ? 5 * k : 2 * k;
         if (!ctx.merge_attr_set) {
             CUDA_TRY(cudaFuncSetAttribute(merge_warp_kernel<512, 256, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -661,7 +663,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
             mp.big = nullptr;
         } else if (expect <= 340) {
             LAUNCH_DEP(8, (merge_warp_kernel<512, 256, 8>), static_cast<unsigned>((n + 7) / 8), 256, 8 * sizeof(MergeWarpSmem<512>), stream, mp);
-        } else if (expect <= 700) {
+        } else if (expect <= 1400) {
             LAUNCH_DEP(8, (merge_warp_kernel<1024, 512, 8>), static_cast<unsigned>((n + 7) / 8), 256, 8 * sizeof(MergeWarpSmem<1024>), stream, mp);
         } else if (expect <= 1700) {
             LAUNCH_DEP(8, (merge_warp_kernel<2048, 1024, 4>), static_cast<unsigned>((n + 3) / 4), 128, 4 * sizeof(MergeWarpSmem<2048>), stream, mp);
