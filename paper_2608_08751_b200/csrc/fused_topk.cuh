@@ -27,11 +27,11 @@
 //             minimum of a group passes, the 8 raw keys are appended (two 16-byte stores, ~1.4
 //             instructions per key, no branch) and the merge kernel compares key by key.  The host computes it with a first, small launch of
 //             this same kernel (sketch rule) over every S-th centroid, S = k / 4: the 16th smallest
-//             group minimum of that sample lets about 4k candidates through.  Whether tau was loose
+//             32-key-chunk minimum of that sample lets about 4k candidates through.  Whether tau was loose
 //             enough is checked exactly by the merge kernel (at least k candidates <= tau); a row
 //             that fails is recomputed by brute force;
 //   sketch    the threshold pass itself: nothing is appended; each thread only keeps its 16
-//             smallest group minima and leaves them as its partial result;
+//             smallest chunk minima (one per 32 keys) and leaves them as its partial result;
 //   bounded   (small problems) tau = +inf until the log fills, then the warp selects the k
 //             smallest in place (radix select on the key bits, ties to the lower id) and tau
 //             becomes the k-th.  The same in-place selection catches any log that fills up.
