@@ -288,7 +288,7 @@ int make_plan(int64_t n, int nlist, int d, int k, int num_sms, Plan* pl, bool on
 int64_t rows_per_launch(int d, int k) {
     const int kp = (d + 63) / 64 * 64 + kAugK;
     const int64_t per_row = static_cast<int64_t>(kp) * 2 +
-                            (k > 1 ? 6ll * (4 * (k < 96 ? 96 : k) + 4) * kRecordBytes + 6ll * 512 * 8 : 6ll * 8);
+                            (k > 1 ? 6ll * (4 * (k < 96 ? 96 : k) + kGroupLogMargin) * kRecordBytes + 6ll * 512 * 8 : 6ll * 8);
     int64_t rows = (int64_t(3) << 30) / per_row;
     rows = rows / (2 * kBlockM) * (2 * kBlockM);
     if (rows < 2 * kBlockM) rows = 2 * kBlockM;
