@@ -472,8 +472,9 @@ def main():
         must = o_d < (dk[:, None] - tol_o)
         present = (o_ids[:, :, None] == g_ids[:, None, :]).any(-1)
         differs = g_ids != o_ids
+        lower = np.maximum.accumulate(d_true - tol_g, axis=1)
         row_ok = ((present | ~must).all(axis=1) & (d_true <= dk[:, None] + tol_g).all(axis=1)
-                  & ((np.abs(d_true - o_d) < np.maximum(tol_g, tol_o)) | ~differs).all(axis=1))
+                  & (lower[:, :-1] <= (d_true + tol_g)[:, 1:]).all(axis=1))
         line["cpu_baseline"] = {"value": rows / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"{rows} seeded rows of the C1 routing batch, full centroid width, {dt:.1f} s",
                                 "rows_matching_oracle_by_tolerance_rule": float(row_ok.mean()),

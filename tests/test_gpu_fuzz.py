@@ -197,3 +197,17 @@ def test_rows_with_many_times_the_usual_candidates(cluster, k):
     B.ivf_check()
     stats = parity.check_route(x, c, k, ids.cpu().numpy(), dists.cpu().numpy())
     assert stats["rows"] == n
+
+
+def test_low_dimension_mixed_norms_order_within_tolerance():
+    """d = 4, float rows, k = 256 of 1,000: centroid norms differ by an order of magnitude, so the
+    tolerance differs from id to id; an id with a large norm may be ranked a few places off while the
+    small-norm ids between keep their exact order (the case a random sweep found)."""
+    rng = np.random.default_rng(770397)
+    x = rng.standard_normal((5000, 4)).astype(np.float32)
+    c = rng.standard_normal((1000, 4)).astype(np.float32)
+    c[::7] *= 3.0
+    ids, dists = B.ivf_route(_t(x), _t(c), 256)
+    B.ivf_check()
+    stats = parity.check_route(x, c, 256, ids.cpu().numpy(), dists.cpu().numpy())
+    assert stats["max_err_over_tol"] <= 1.0
