@@ -593,10 +593,10 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         // (uint8 points: the epilogue warps build the point tiles themselves, see below)
         const bool raw = p.x_raw != nullptr;
         int it = 0, seg = 0, a_armed = 0;
+        int st = 0;        // ring stage of tile `it` and the parity of its use, stepped instead of
+        uint32_t ph = 0;   // divided out of `it` (the stage count is a run-time value)
         bool ok = true;
         auto load_b = [&](int t) -> bool {  // lane 0: one centroid tile into the next ring stage
-            const int st = it % p.nstage;
-            const uint32_t ph = (it / p.nstage) & 1;
             if (!mbar_wait(&b_empty[st], ph ^ 1u, ctl, 2)) return false;
             mbar_arrive_expect_tx(&b_full[st], stage_bytes);
             uint8_t* dst = smem_b + static_cast<size_t>(st) * stage_bytes;
@@ -604,6 +604,10 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 tma_load_2d(dst + s * p.block_n * kSliceRowBytes, &tmap_c, &b_full[st], s * kSliceK, t * p.block_n);
             tma_load_2d(dst + b_data_bytes, &tmap_ca, &b_full[st], kd, t * p.block_n);
             ++it;
+            if (++st == p.nstage) {
+                st = 0;
+                ph ^= 1u;
+            }
             return true;
         };
         for (int64_t u = u0; u < u1 && ok;) {
@@ -666,6 +670,8 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             const uint32_t a_slice_step = (kBlockM * kSliceRowBytes) >> 4;
             const uint32_t b_slice_step = static_cast<uint32_t>(p.block_n * kSliceRowBytes) >> 4;
             int it = 0, seg = 0;
+            int st = 0;       // ring stage and use parity of tile `it`, stepped
+            uint32_t ph = 0;
             bool ok = true;
             for (int64_t u = u0; u < u1 && ok;) {
                 const int64_t r = u / NT;
@@ -674,8 +680,6 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 ok = mbar_wait(a_full, seg & 1, ctl, 3);
                 if (!ok) break;
                 for (int t = t0; t < t1 && ok; ++t) {
-                    const int st = it % p.nstage;
-                    const uint32_t ph = (it / p.nstage) & 1;
                     ok = mbar_wait(&b_full[st], ph, ctl, 4);
                     if (!ok) break;
                     const uint32_t b_stage = b_addr + st * stage_bytes;
@@ -708,6 +712,10 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                     if (!ok) break;
                     umma_commit(&b_empty[st]);
                     ++it;
+                    if (++st == p.nstage) {
+                        st = 0;
+                        ph ^= 1u;
+                    }
                 }
                 if (ok) umma_commit(a_empty);
                 ++seg;
