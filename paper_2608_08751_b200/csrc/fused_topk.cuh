@@ -672,6 +672,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             int it = 0, seg = 0;
             int st = 0;       // ring stage and use parity of tile `it`, stepped
             uint32_t ph = 0;
+            bool acc_ready = false, b_ready = false;  // barriers of the next tile already seen complete
             bool ok = true;
             for (int64_t u = u0; u < u1 && ok;) {
                 const int64_t r = u / NT;
@@ -680,15 +681,17 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 ok = mbar_wait(a_full, seg & 1, ctl, 3);
                 if (!ok) break;
                 for (int t = t0; t < t1 && ok; ++t) {
-                    ok = mbar_wait(&b_full[st], ph, ctl, 4);
+                    if (!b_ready) ok = mbar_wait(&b_full[st], ph, ctl, 4);
                     if (!ok) break;
+                    b_ready = false;
                     const uint32_t b_stage = b_addr + st * stage_bytes;
                     for (int h = 0; h < MT; ++h) {
                         const int su = it * MT + h;  // accumulator buffers alternate per (tile, row tile)
                         const int buf = su & 1;
                         const uint32_t aph = (su >> 1) & 1;
-                        ok = mbar_wait(&t_empty[buf], aph ^ 1u, ctl, 5);
+                        if (!acc_ready) ok = mbar_wait(&t_empty[buf], aph ^ 1u, ctl, 5);
                         if (!ok) break;
+                        acc_ready = false;
                         tc_fence_after_sync();
                         const uint32_t d_tmem = tmem_base + buf * kAccStride;
                         const uint32_t a_tile = a_addr + h * a_bytes;
@@ -704,6 +707,17 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                             const bool last_of_slice = (kk & 3) == 3;
                             a_lo += last_of_slice ? a_slice_step - 6u : 2u;
                             b_lo += last_of_slice ? b_slice_step - 6u : 2u;
+                        }
+                        // While the tensor core works through those, look at the barriers the next tile
+                        // will need: a wait costs this thread 50-100 cycles even when the phase has long
+                        // completed, and the tensor core's queue runs dry meanwhile.
+                        {
+                            const int nsu = su + 1;
+                            acc_ready = mbar_test_wait(&t_empty[nsu & 1], ((nsu >> 1) & 1u) ^ 1u);
+                            if (h == MT - 1) {
+                                const bool wrap = st + 1 == p.nstage;
+                                b_ready = mbar_test_wait(&b_full[wrap ? 0 : st + 1], wrap ? ph ^ 1u : ph);
+                            }
                         }
                         umma_f16(d_tmem, umma_desc_join(umma_desc_lo(a_tile + a_data_bytes), kDescHiSw32),
                                  umma_desc_join(umma_desc_lo(b_stage + b_data_bytes), kDescHiSw32), idesc, 1u);
