@@ -669,6 +669,16 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             const uint32_t b_addr = smem_u32(smem_b);
             const uint32_t a_slice_step = (kBlockM * kSliceRowBytes) >> 4;
             const uint32_t b_slice_step = static_cast<uint32_t>(p.block_n * kSliceRowBytes) >> 4;
+            // descriptor low words that never change: the point tiles (data and norm columns) and stage 0
+            // of the ring; a stage's words follow by adding its offset in 16-byte units
+            uint32_t a_lo_data[MT], a_lo_norm[MT];
+#pragma unroll
+            for (int h = 0; h < MT; ++h) {
+                a_lo_data[h] = umma_desc_lo(a_addr + h * a_bytes);
+                a_lo_norm[h] = umma_desc_lo(a_addr + h * a_bytes + a_data_bytes);
+            }
+            const uint32_t b_lo_data0 = umma_desc_lo(b_addr), b_lo_norm0 = umma_desc_lo(b_addr + b_data_bytes);
+            const uint32_t stage_step = static_cast<uint32_t>(stage_bytes) >> 4;
             int it = 0, seg = 0;
             int st = 0;       // ring stage and use parity of tile `it`, stepped
             uint32_t ph = 0;
@@ -684,7 +694,8 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                     if (!b_ready) ok = mbar_wait(&b_full[st], ph, ctl, 4);
                     if (!ok) break;
                     b_ready = false;
-                    const uint32_t b_stage = b_addr + st * stage_bytes;
+                    const uint32_t b_lo_data = b_lo_data0 + st * stage_step, b_lo_norm = b_lo_norm0 + st * stage_step;
+#pragma unroll
                     for (int h = 0; h < MT; ++h) {
                         const int su = it * MT + h;  // accumulator buffers alternate per (tile, row tile)
                         const int buf = su & 1;
@@ -694,13 +705,12 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                         acc_ready = false;
                         tc_fence_after_sync();
                         const uint32_t d_tmem = tmem_base + buf * kAccStride;
-                        const uint32_t a_tile = a_addr + h * a_bytes;
                         // The descriptors of consecutive K steps differ only in the start-address field
                         // (16-byte units, low word): +2 inside a 64-column slice, then on to the next
                         // slice.  Stepping the low words keeps this thread's work per MMA to a few
                         // instructions; building each descriptor from scratch took about as long as the
                         // tensor core needs for the MMA itself.
-                        uint32_t a_lo = umma_desc_lo(a_tile), b_lo = umma_desc_lo(b_stage);
+                        uint32_t a_lo = a_lo_data[h], b_lo = b_lo_data;
                         for (int kk = 0; kk < p.ksteps; ++kk) {
                             umma_f16(d_tmem, umma_desc_join(a_lo, kDescHiSw128), umma_desc_join(b_lo, kDescHiSw128), idesc,
                                      kk > 0 ? 1u : 0u);
@@ -719,8 +729,8 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                                 b_ready = mbar_test_wait(&b_full[wrap ? 0 : st + 1], wrap ? ph ^ 1u : ph);
                             }
                         }
-                        umma_f16(d_tmem, umma_desc_join(umma_desc_lo(a_tile + a_data_bytes), kDescHiSw32),
-                                 umma_desc_join(umma_desc_lo(b_stage + b_data_bytes), kDescHiSw32), idesc, 1u);
+                        umma_f16(d_tmem, umma_desc_join(a_lo_norm[h], kDescHiSw32), umma_desc_join(b_lo_norm, kDescHiSw32), idesc,
+                                 1u);
                         umma_commit(&t_full[buf]);
                     }
                     if (!ok) break;
