@@ -118,12 +118,14 @@ __host__ __device__ inline int cta_of_unit(int64_t T, int G, int NT, int cross, 
     return static_cast<int>(((cu + 1) * G - 1) / C);
 }
 
+// (the radix histograms are used by the epilogues that keep a bounded candidate log, which always run
+// with one row tile per unit)
 __host__ __device__ inline size_t fused_smem_bytes(int kslices, int block_n, int nstage, int mtiles) {
     return 1024                                                                        // alignment slack
            + static_cast<size_t>(mtiles) * kBlockM * (kslices * kSliceRowBytes + kAugRowBytes)  // point tiles
            + static_cast<size_t>(nstage) * block_n * (kslices * kSliceRowBytes + kAugRowBytes)
            + 256                                                                       // barriers etc.
-           + kNumEpiWarps * 256 * sizeof(int);                                         // radix histograms
+           + (mtiles == 1 ? kNumEpiWarps * 256 * sizeof(int) : 0);                     // radix histograms
 }
 
 __device__ __forceinline__ uint32_t orderable(float v) {
