@@ -40,11 +40,11 @@ METRIC = "routed queries/s"
 UNIT = "queries/s"
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised in profiles/.
-# k = 1 kernel: captured at 262,144 rows (53.9 MB, profiles/fused_argmin_262144x65536x128.md) and
+# k = 1 kernel: captured at 262,144 rows (54.5 MB, profiles/fused_argmin_262144x65536x128.md) and
 # scaled by 4 to the bench's 1,048,576-row launch (an upper bound: the centroid copy does not grow).
-TRAFFIC_FUSED_ARGMIN_BYTES = 4 * (52.595456e6 + 1.256448e6)
+TRAFFIC_FUSED_ARGMIN_BYTES = 4 * (52.519424e6 + 1.968896e6)
 # k = 64 kernel: captured at the bench's own size (profiles/fused_groups_routing_c1_c2.md).
-TRAFFIC_FUSED_TOPK_BYTES = 94.215680e6 + 103.088640e6
+TRAFFIC_FUSED_TOPK_BYTES = 93.999360e6 + 104.450560e6
 
 
 def peaks():
