@@ -62,9 +62,11 @@ int fail(int code, const char* fmt, ...) {
 // programmatic-serialization attribute: the launch latency and the kernel's own set-up then overlap
 // the end of the kernel before it.  g_pdl = 0 falls back to ordinary launches (test hook).
 // Bit per kernel family: 1 prep, 2 fused, 4 threshold merge, 8 merge, 16 tail kernel (passed-on rows
-// and recomputation; 32 unused).  Measured: letting the fused kernel or the threshold merge start early costs time
-// (their waiting warps sit next to the running kernel), the other families gain 6-9 us per call.
-int g_pdl = 57;
+// and recomputation; 32 unused).  Measured per family on whole calls: every family gains except the
+// threshold merge (its waiting warps sit next to the running threshold pass: 256-query batches lose
+// 13 us), so that one is launched normally.  The fused kernel's set-up (TMEM allocation, barrier
+// initialisation, tensor-map prefetch) overlaps the end of its predecessor: 5-10 us per call.
+int g_pdl = 59;
 template <typename... KArgs, typename... Args>
 cudaError_t launch_dep(int cls, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
     cudaLaunchConfig_t cfg = {};
