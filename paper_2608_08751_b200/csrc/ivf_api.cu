@@ -62,11 +62,11 @@ int fail(int code, const char* fmt, ...) {
 // programmatic-serialization attribute: the launch latency and the kernel's own set-up then overlap
 // the end of the kernel before it.  g_pdl = 0 falls back to ordinary launches (test hook).
 // Bit per kernel family: 1 prep, 2 fused, 4 threshold merge, 8 merge, 16 tail kernel (passed-on rows
-// and recomputation; 32 unused).  Measured per family on whole calls: every family gains except the
+// and recomputation; 32 unused), 64 centroid update.  Measured per family on whole calls: every family gains except the
 // threshold merge (its waiting warps sit next to the running threshold pass: 256-query batches lose
 // 13 us), so that one is launched normally.  The fused kernel's set-up (TMEM allocation, barrier
 // initialisation, tensor-map prefetch) overlaps the end of its predecessor: 5-10 us per call.
-int g_pdl = 59;
+int g_pdl = 59 | 64;  // 64: the centroid-update family
 template <typename... KArgs, typename... Args>
 cudaError_t launch_dep(int cls, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
     cudaLaunchConfig_t cfg = {};
@@ -718,10 +718,15 @@ int update_device(DeviceCtx& ctx, const void* points, int ptype, const int32_t* 
     const int tk = timing_begin(TK_UPDATE, stream);
     CUDA_TRY(cudaMemsetAsync(cnt, 0, static_cast<size_t>(nlist) * sizeof(int), stream));
     const unsigned rb = static_cast<unsigned>((n + 255) / 256);
-    update_hist_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, cnt, ctx.status);
-    update_scan_local_kernel<<<scan_blocks, 1024, 0, stream>>>(cnt, nlist, off, block_sums);
-    update_scan_fix_kernel<<<scan_blocks, 1024, 0, stream>>>(nlist, off, block_sums, cur);
-    update_fill_kernel<<<rb, 256, 0, stream>>>(ids, n, nlist, off, cur, perm);
+    // (the kernels of this family start with griddepcontrol.wait and are launched as programmatic
+    // dependents of one another, family bit 64: their launch latencies overlap -- 0.123 -> 0.112 ms at
+    // 65,536 lists; with a few hundred lists the histogram's atomics are the bottleneck and early
+    // starters only get in its way (0.93 -> 1.01 ms at 256 lists), so those stay ordinary launches)
+    const int fam = (n / nlist >= 4096) ? 0 : 64;
+    LAUNCH_DEP(fam, update_hist_kernel, rb, 256, 0, stream, ids, n, nlist, cnt, ctx.status);
+    LAUNCH_DEP(fam, update_scan_local_kernel, scan_blocks, 1024, 0, stream, static_cast<const int*>(cnt), nlist, off, block_sums);
+    LAUNCH_DEP(fam, update_scan_fix_kernel, scan_blocks, 1024, 0, stream, nlist, off, static_cast<const int*>(block_sums), cur);
+    LAUNCH_DEP(fam, update_fill_kernel, rb, 256, 0, stream, ids, n, nlist, static_cast<const int*>(off), cur, perm);
     // few long lists: cut every list into pieces, one warp each, and add the pieces up in order
     const int64_t avg = n / nlist;
     int parts = avg >= 4096 ? static_cast<int>((avg + 2047) / 2048) : 1;
@@ -730,30 +735,32 @@ int update_device(DeviceCtx& ctx, const void* points, int ptype, const int32_t* 
         float* scratch;
         WS(WS_UPARTS, static_cast<size_t>(nlist) * parts * d * sizeof(float), scratch);
         const unsigned pb = static_cast<unsigned>((static_cast<int64_t>(nlist) * parts * 32 + 255) / 256);
+        const int* cperm = perm;
+        const int* coff = off;
         if (ptype == IVF_U8)
-            update_reduce_parts_kernel<uint8_t><<<pb, 256, 0, stream>>>(static_cast<const uint8_t*>(points), perm, off, nlist, d, parts, scratch);
+            LAUNCH_DEP(fam, update_reduce_parts_kernel<uint8_t>, pb, 256, 0, stream, static_cast<const uint8_t*>(points), cperm, coff, nlist, d, parts, scratch);
         else if (ptype == IVF_I8)
-            update_reduce_parts_kernel<int8_t><<<pb, 256, 0, stream>>>(static_cast<const int8_t*>(points), perm, off, nlist, d, parts, scratch);
+            LAUNCH_DEP(fam, update_reduce_parts_kernel<int8_t>, pb, 256, 0, stream, static_cast<const int8_t*>(points), cperm, coff, nlist, d, parts, scratch);
         else
-            update_reduce_parts_kernel<float><<<pb, 256, 0, stream>>>(static_cast<const float*>(points), perm, off, nlist, d, parts, scratch);
-        LAUNCH_CHECK();
+            LAUNCH_DEP(fam, update_reduce_parts_kernel<float>, pb, 256, 0, stream, static_cast<const float*>(points), cperm, coff, nlist, d, parts, scratch);
         const int64_t cells = static_cast<int64_t>(nlist) * d;
-        update_combine_parts_kernel<<<static_cast<unsigned>((cells + 255) / 256), 256, 0, stream>>>(
-            scratch, off, nlist, d, parts, sums, reinterpret_cast<long long*>(counts));
-        LAUNCH_CHECK();
+        LAUNCH_DEP(fam, update_combine_parts_kernel, static_cast<unsigned>((cells + 255) / 256), 256, 0, stream,
+                   static_cast<const float*>(scratch), coff, nlist, d, parts, sums, reinterpret_cast<long long*>(counts));
         timing_end(tk, stream);
         return IVF_OK;
     }
     const unsigned lb = static_cast<unsigned>((static_cast<int64_t>(nlist) * 32 + 255) / 256);
-    if (ptype == IVF_U8)
-        update_reduce_kernel<uint8_t><<<lb, 256, 0, stream>>>(static_cast<const uint8_t*>(points), perm, off, nlist, d,
-                                                              sums, reinterpret_cast<long long*>(counts));
-    else if (ptype == IVF_I8)
-        update_reduce_kernel<int8_t><<<lb, 256, 0, stream>>>(static_cast<const int8_t*>(points), perm, off, nlist, d,
-                                                             sums, reinterpret_cast<long long*>(counts));
-    else
-        update_reduce_kernel<float><<<lb, 256, 0, stream>>>(static_cast<const float*>(points), perm, off, nlist, d,
-                                                            sums, reinterpret_cast<long long*>(counts));
+    {
+        const int* cperm = perm;
+        const int* coff = off;
+        long long* lcounts = reinterpret_cast<long long*>(counts);
+        if (ptype == IVF_U8)
+            LAUNCH_DEP(fam, update_reduce_kernel<uint8_t>, lb, 256, 0, stream, static_cast<const uint8_t*>(points), cperm, coff, nlist, d, sums, lcounts);
+        else if (ptype == IVF_I8)
+            LAUNCH_DEP(fam, update_reduce_kernel<int8_t>, lb, 256, 0, stream, static_cast<const int8_t*>(points), cperm, coff, nlist, d, sums, lcounts);
+        else
+            LAUNCH_DEP(fam, update_reduce_kernel<float>, lb, 256, 0, stream, static_cast<const float*>(points), cperm, coff, nlist, d, sums, lcounts);
+    }
     timing_end(tk, stream);
     return IVF_OK;
 }

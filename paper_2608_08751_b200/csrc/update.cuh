@@ -8,12 +8,16 @@
 
 #include <type_traits>
 
+#include "ptx.cuh"
+
 namespace ivf {
 
 constexpr int kStatusBadId = -6;
 
 __global__ void update_hist_kernel(const int32_t* __restrict__ ids, int64_t n, int nlist, int* __restrict__ cnt,
                                    int* status) {
+    pdl_wait();
+    pdl_trigger();
     const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const int l = ids[i];
@@ -31,6 +35,8 @@ constexpr int kScanBlock = 4096;
 
 __global__ void __launch_bounds__(1024) update_scan_local_kernel(const int* __restrict__ cnt, int nlist,
                                                                  int* __restrict__ off, int* __restrict__ block_sums) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ int warp_sums[32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int i0 = blockIdx.x * kScanBlock + threadIdx.x * 4;
@@ -72,6 +78,8 @@ __global__ void __launch_bounds__(1024) update_scan_local_kernel(const int* __re
 __global__ void __launch_bounds__(1024) update_scan_fix_kernel(int nlist, int* __restrict__ off,
                                                                const int* __restrict__ block_sums,
                                                                int* __restrict__ cursor) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ int s_part[32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     int acc = 0;
@@ -96,6 +104,8 @@ __global__ void __launch_bounds__(1024) update_scan_fix_kernel(int nlist, int* _
 
 __global__ void update_fill_kernel(const int32_t* __restrict__ ids, int64_t n, int nlist,
                                    const int* __restrict__ off, int* __restrict__ cursor, int* __restrict__ perm) {
+    pdl_wait();
+    pdl_trigger();
     const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const int l = ids[i];
@@ -165,6 +175,8 @@ template <typename T>
 __global__ void update_reduce_kernel(const T* __restrict__ x, const int* __restrict__ perm,
                                      const int* __restrict__ off, int nlist, int d, float* __restrict__ sums,
                                      long long* __restrict__ counts) {
+    pdl_wait();
+    pdl_trigger();
     const int lane = threadIdx.x & 31;
     const int l = static_cast<int>((static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5);
     if (l >= nlist) return;
@@ -196,6 +208,8 @@ template <typename T>
 __global__ void update_reduce_parts_kernel(const T* __restrict__ x, const int* __restrict__ perm,
                                            const int* __restrict__ off, int nlist, int d, int parts,
                                            float* __restrict__ scratch) {
+    pdl_wait();
+    pdl_trigger();
     const int lane = threadIdx.x & 31;
     const int64_t w = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
     if (w >= static_cast<int64_t>(nlist) * parts) return;
@@ -215,6 +229,8 @@ __global__ void update_reduce_parts_kernel(const T* __restrict__ x, const int* _
 
 __global__ void update_combine_parts_kernel(const float* __restrict__ scratch, const int* __restrict__ off, int nlist, int d,
                                             int parts, float* __restrict__ sums, long long* __restrict__ counts) {
+    pdl_wait();
+    pdl_trigger();
     const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (i >= static_cast<int64_t>(nlist) * d) return;
     const int l = static_cast<int>(i / d), t = static_cast<int>(i - static_cast<int64_t>(l) * d);
