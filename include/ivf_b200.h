@@ -241,8 +241,8 @@ int ivf_debug_set_pq_groups(int groups);
 int ivf_debug_set_crossing_cost(int units);
 /* Test hook: mask of the kernel families of the routing path that may start while their predecessor
  * drains (programmatic dependent launch): 1 operand preparation, 2 fused kernel, 4 threshold merge,
- * 8 merge, 16 tail kernel (passed-on rows and recomputation; bit 32 is unused), 64 centroid update.
- * 0 = ordinary stream launches; default 123. */
+ * 8 merge, 16 tail kernel (passed-on rows and recomputation; bit 32 is unused), 64 centroid update,
+ * 128 residual-PQ search.  0 = ordinary stream launches; default 251. */
 int ivf_debug_set_dependent_launch(int mask);
 int ivf_debug_timing(int enable);
 int ivf_debug_timing_read(double ms[9], int64_t launches[9]);

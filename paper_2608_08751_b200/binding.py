@@ -467,7 +467,7 @@ def ivf_debug_set_crossing_cost(units: int) -> None:
 
 
 def ivf_debug_set_dependent_launch(on: bool) -> None:
-    lib().ivf_debug_set_dependent_launch(int(on) if not isinstance(on, bool) else (123 if on else 0))
+    lib().ivf_debug_set_dependent_launch(int(on) if not isinstance(on, bool) else (251 if on else 0))
 
 
 def ivf_debug_set_pq_groups(groups: int) -> None:

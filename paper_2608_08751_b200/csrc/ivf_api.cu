@@ -62,11 +62,11 @@ int fail(int code, const char* fmt, ...) {
 // programmatic-serialization attribute: the launch latency and the kernel's own set-up then overlap
 // the end of the kernel before it.  g_pdl = 0 falls back to ordinary launches (test hook).
 // Bit per kernel family: 1 prep, 2 fused, 4 threshold merge, 8 merge, 16 tail kernel (passed-on rows
-// and recomputation; 32 unused), 64 centroid update.  Measured per family on whole calls: every family gains except the
+// and recomputation; 32 unused), 64 centroid update, 128 residual-PQ search.  Measured per family on whole calls: every family gains except the
 // threshold merge (its waiting warps sit next to the running threshold pass: 256-query batches lose
 // 13 us), so that one is launched normally.  The fused kernel's set-up (TMEM allocation, barrier
 // initialisation, tensor-map prefetch) overlaps the end of its predecessor: 5-10 us per call.
-int g_pdl = 59 | 64;  // 64: the centroid-update family
+int g_pdl = 59 | 64 | 128;  // 64: the centroid-update family, 128: the residual-PQ search
 template <typename... KArgs, typename... Args>
 cudaError_t launch_dep(int cls, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
     cudaLaunchConfig_t cfg = {};
@@ -1212,12 +1212,12 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     float* cbt;
     WS(WS_PQ_CBT, static_cast<size_t>(d) * kPqK * sizeof(float), cbt);
     int tk = timing_begin(TK_PQ_SCAN, stream);
-    pq_transpose_codebooks_kernel<<<(d * kPqK + 255) / 256, 256, 0, stream>>>(codebooks, d, d / pq_m, cbt);
-    LAUNCH_CHECK();
-    pq_setup_query_kernel<<<static_cast<unsigned>(nq), 128, 0, stream>>>(
-        probe_ids, nprobe, nlist, reinterpret_cast<const long long*>(list_offsets), chunk_start,
-        reinterpret_cast<long long*>(out_counts), ctx.status);
-    LAUNCH_CHECK();
+    // (family bit 128 of the dependent-launch mask: the four kernels of a search overlap their launch
+    // latencies, which is a tenth of a small batch)
+    LAUNCH_DEP(128, pq_transpose_codebooks_kernel, (d * kPqK + 255) / 256, 256, 0, stream, codebooks, d, d / pq_m, cbt);
+    LAUNCH_DEP(128, pq_setup_query_kernel, static_cast<unsigned>(nq), 128, 0, stream, probe_ids, nprobe, nlist,
+               reinterpret_cast<const long long*>(list_offsets), chunk_start, reinterpret_cast<long long*>(out_counts),
+               ctx.status);
     PqScanParams sp;
     sp.q = queries;
     sp.q_type = qtype;
@@ -1243,13 +1243,12 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     if (teams) {
         const int64_t pairs = (total_groups + 1) / 2;
         const unsigned grid = static_cast<unsigned>(pairs < ctx.num_sms ? pairs : ctx.num_sms);
-        pq_scan_teams_kernel<<<grid, 2 * kPqScanThreads, pq_teams_smem_bytes(d, pq_m), stream>>>(sp);
+        LAUNCH_DEP(128, pq_scan_teams_kernel, grid, 2 * kPqScanThreads, pq_teams_smem_bytes(d, pq_m), stream, sp);
     } else {
         const int64_t resident = 2 * static_cast<int64_t>(ctx.num_sms);
         const unsigned grid = static_cast<unsigned>(total_groups < resident ? total_groups : resident);
-        pq_scan_kernel<<<grid, kPqScanThreads, pq_scan_smem_bytes(d, pq_m), stream>>>(sp);
+        LAUNCH_DEP(128, pq_scan_kernel, grid, kPqScanThreads, pq_scan_smem_bytes(d, pq_m), stream, sp);
     }
-    LAUNCH_CHECK();
     timing_end(tk, stream);
     tk = timing_begin(TK_PQ_MERGE, stream);
     PqMergeParams mp;
@@ -1263,10 +1262,9 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     mp.out_est = out_est;
     const int64_t slots = static_cast<int64_t>(ngroups) * n_rerank;
     if (slots > kPqBufKeys && slots <= static_cast<int64_t>(kPqMergeRegKeys) * kPqThreads)
-        pq_merge_kernel<true><<<static_cast<unsigned>(nq), kPqThreads, 0, stream>>>(mp);
+        LAUNCH_DEP(128, pq_merge_kernel<true>, static_cast<unsigned>(nq), kPqThreads, 0, stream, mp);
     else
-        pq_merge_kernel<false><<<static_cast<unsigned>(nq), kPqThreads, 0, stream>>>(mp);
-    LAUNCH_CHECK();
+        LAUNCH_DEP(128, pq_merge_kernel<false>, static_cast<unsigned>(nq), kPqThreads, 0, stream, mp);
     timing_end(tk, stream);
     return IVF_OK;
 }

@@ -239,6 +239,8 @@ __global__ void pq_residuals_kernel(const void* __restrict__ x, int x_type, int6
 
 // codebooks [pq_m][256][dsub] -> out[(m * dsub + t) * 256 + j] (coordinate-major), for the scan kernel
 __global__ void pq_transpose_codebooks_kernel(const float* __restrict__ codebooks, int d, int dsub, float* __restrict__ out) {
+    pdl_wait();
+    pdl_trigger();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;  // index in the output
     if (i >= d * kPqK) return;
     const int j = i & (kPqK - 1);
@@ -256,6 +258,8 @@ __global__ void __launch_bounds__(128) pq_setup_query_kernel(const int32_t* __re
                                                              const long long* __restrict__ offsets,
                                                              int* __restrict__ chunk_start,
                                                              long long* __restrict__ cand_count, int* status) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ int wsum[4];
     __shared__ long long wlen[4];
     __shared__ int carry_s;
@@ -677,6 +681,8 @@ __device__ __forceinline__ void pq_scan_groups(const PqScanParams& p, const PqTe
 // One team per CTA, two CTAs per SM; the codebook is read through L1 from its transposed copy.
 // Serves every shape (up to kPqMaxProbes probes) with little shared memory.
 __global__ void __launch_bounds__(kPqScanThreads, 2) pq_scan_kernel(const PqScanParams p) {
+    pdl_wait();
+    pdl_trigger();
     extern __shared__ __align__(16) uint8_t pq_smem_raw[];
     if (static_cast<int64_t>(blockIdx.x) >= p.nq * p.ngroups) return;
     const PqTeamSmem s = pq_team_carve(pq_smem_raw, p.pq_m, kPqMaxProbes);
@@ -687,6 +693,8 @@ __global__ void __launch_bounds__(kPqScanThreads, 2) pq_scan_kernel(const PqScan
 // memory and otherwise work on different groups with their own table, buffer and barrier, so one
 // team's table build (arithmetic) runs under the other's scan (shared-memory lookups).
 __global__ void __launch_bounds__(2 * kPqScanThreads, 1) pq_scan_teams_kernel(const PqScanParams p) {
+    pdl_wait();
+    pdl_trigger();
     extern __shared__ __align__(16) uint8_t pq_smem_raw[];
     if (2 * static_cast<int64_t>(blockIdx.x) >= p.nq * p.ngroups) return;
     float* cbt = reinterpret_cast<float*>(pq_smem_raw);
@@ -725,6 +733,8 @@ struct PqMergeParams {
 constexpr int kPqMergeRegKeys = 16;
 template <bool kRegs>
 __global__ void __launch_bounds__(kPqThreads, kRegs ? 1 : 2) pq_merge_kernel(const PqMergeParams p) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ uint64_t buf[kPqBufKeys];
     __shared__ int hist[256];
     __shared__ int misc[16];
