@@ -619,7 +619,9 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
             LAUNCH_DEP(4, merge_tau_warp_kernel, static_cast<unsigned>((n * 32 + 255) / 256), 256, 0, stream, ms);
         else {
             const int threads = pls.partials >= kTauThreads ? kTauThreads : (pls.partials + 31) / 32 * 32;
-            LAUNCH_DEP(4, merge_tau_kernel, static_cast<unsigned>(n), threads, 0, stream, ms);
+            // (a handful of rows: the few waiting CTAs of an early start do not disturb the threshold
+            // pass, B = 8: -2 us; hundreds of rows: they do, B = 256: +13 us)
+            LAUNCH_DEP(n <= 32 ? 1 : 4, merge_tau_kernel, static_cast<unsigned>(n), threads, 0, stream, ms);
         }
         LAUNCH_CHECK();
         timing_end(tk, stream);
