@@ -155,7 +155,9 @@ int ivf_centroid_finalize(const float* sums, const int64_t* counts, int nlist, i
  *   out_points   [n, d] (ptype), device: row p = points[out_order[p]]
  * The order of the rows inside a list is unspecified (every order is a valid layout; out_order tells
  * which one was taken).  A row whose id is outside [0, nlist) is dropped from the layout and flags
- * IVF_ERR_BAD_ID in the status word.  At most 2^31 - 1 rows per call.
+ * IVF_ERR_BAD_ID in the status word: the kept rows fill positions [0, out_offsets[nlist]); the
+ * positions after them get out_order = -1 and an all-zero row in out_points.  At most 2^31 - 1 rows
+ * per call.
  */
 int ivf_cluster_major_reorder(const void* points, ivf_dtype ptype, const int32_t* ids, int64_t n, int d,
                               int nlist, void* out_points, int64_t* out_offsets, int32_t* out_order,
@@ -203,6 +205,10 @@ int64_t ivf_launch_count(void);
  */
 int ivf_debug_plan(int64_t n, int nlist, int d, int k, int num_sms, int64_t out[9]);
 int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int64_t out[4]);
+/* Test hook (host only): the rotation of row group `row_group` in that schedule -- position p of the
+ * row group's sweep stands for centroid tile (p + rotation) mod col_tiles, so that the CTAs walk the
+ * centroid table as a few shared fronts.  Returns the rotation (>= 0) or a negative status. */
+int ivf_debug_rotation(int64_t n, int nlist, int d, int k, int num_sms, int64_t row_group);
 int ivf_debug_set_wait_limit_ns(int64_t ns);
 int ivf_debug_wait_probe(void* stream);
 /* Test hook: when on, the merge of a k > 1 call declares every row's candidate set insufficient, so

@@ -25,7 +25,7 @@ EXPORTS = (
     "ivf_route_prepared",
     "ivf_pq_encode", "ivf_pq_search", "ivf_pq_residuals", "ivf_assign_candidates",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
-    "ivf_debug_plan", "ivf_debug_span", "ivf_debug_set_wait_limit_ns",
+    "ivf_debug_plan", "ivf_debug_span", "ivf_debug_rotation", "ivf_debug_set_wait_limit_ns",
     "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_set_row_chunk", "ivf_debug_stats", "ivf_debug_set_pq_groups", "ivf_debug_set_dependent_launch", "ivf_debug_set_crossing_cost",
 )
 
@@ -67,6 +67,7 @@ def lib() -> ctypes.CDLL:
     L.ivf_launch_count.restype = i64
     L.ivf_debug_plan.argtypes = [i64, i32, i32, i32, i32, ctypes.POINTER(i64)]
     L.ivf_debug_span.argtypes = [i64, i32, i32, i32, i32, i32, ctypes.POINTER(i64)]
+    L.ivf_debug_rotation.argtypes = [i64, i32, i32, i32, i32, i64]
     L.ivf_debug_set_wait_limit_ns.argtypes = [i64]
     L.ivf_debug_timing.argtypes = [i32]
     L.ivf_debug_wait_probe.argtypes = [vp]
@@ -452,6 +453,13 @@ def ivf_debug_span(n: int, nlist: int, d: int, k: int, num_sms: int, cta: int):
     if int(out[2]) != cta or int(out[3]) != cta:
         raise AssertionError(f"unit-to-CTA mapping disagrees with the span of CTA {cta}: {list(out)}")
     return int(out[0]), int(out[1])
+
+
+def ivf_debug_rotation(n: int, nlist: int, d: int, k: int, num_sms: int, row_group: int) -> int:
+    rc = lib().ivf_debug_rotation(n, nlist, d, k, num_sms, row_group)
+    if rc < 0:
+        _raise(rc)
+    return int(rc)
 
 
 def ivf_debug_set_wait_limit_ns(ns: int) -> None:

@@ -118,6 +118,23 @@ __host__ __device__ inline int cta_of_unit(int64_t T, int G, int NT, int cross, 
     return static_cast<int>(((cu + 1) * G - 1) / C);
 }
 
+// Order of the centroid tiles inside a row group.  A CTA sweeps the positions of its span in order,
+// but position p of row group r stands for centroid tile (p + rot_r) mod NT, with rot_r = the time (in
+// cost units since the launch) at which position 0 of the row group is reached by the CTA that owns
+// it.  Every CTA therefore works on centroid tile (time + i * span length) mod NT for a small integer
+// i: the ~G CTAs sweep the table as a handful of fronts, each shared by the CTAs of many row groups,
+// instead of G different phases.  A centroid tile is then fetched from HBM once per front passage and
+// served to the other CTAs of the front from L2, however large the table is.  (With the positions
+// standing for their own tile index, a table larger than L2 was re-read from HBM once per row group.)
+__host__ __device__ inline int col_rotation(int64_t T, int G, int NT, int cross, int64_t r) {
+    const int64_t w = NT + cross;
+    const int first = cta_of_unit(T, G, NT, cross, r * NT);
+    const int64_t ub = span_begin(T, G, NT, cross, first);
+    const int64_t rb = ub / NT;
+    const int64_t arrive = (r * w + cross) - (rb * w + cross + (ub - rb * NT));
+    return static_cast<int>(arrive % NT);
+}
+
 // (the radix histograms are used by the epilogues that keep a bounded candidate log, which always run
 // with one row tile per unit)
 __host__ __device__ inline size_t fused_smem_bytes(int kslices, int block_n, int nstage, int mtiles) {
@@ -347,8 +364,7 @@ __device__ __forceinline__ void consume(uint32_t (&acc)[32], int jbase, RowState
         // which is the lowest id among equal keys.
         const float m0 = min8(acc, 0), m1 = min8(acc, 1), m2 = min8(acc, 2), m3 = min8(acc, 3);
         const float m = fminf(fminf(m0, m1), fminf(m2, m3));
-        if (m < st.tau) {
-            st.tau = m;
+        if (m <= st.tau) {
             const bool in0 = (m0 == m), in1 = (m1 == m), in2 = (m2 == m);
             const int g = in0 ? 0 : (in1 ? 1 : (in2 ? 2 : 3));
             int idx = 7;
@@ -357,7 +373,11 @@ __device__ __forceinline__ void consume(uint32_t (&acc)[32], int jbase, RowState
                 const float v = __uint_as_float(in0 ? acc[i] : (in1 ? acc[8 + i] : (in2 ? acc[16 + i] : acc[24 + i])));
                 if (v == m) idx = i;
             }
-            st.bestj = jbase + 8 * g + idx;
+            // (a sweep may wrap around to the low centroid ids, so an equal key with a lower id can
+            // come later: ties are settled by id)
+            const int j = jbase + 8 * g + idx;
+            if (m < st.tau || j < st.bestj) st.bestj = j;
+            st.tau = m;
         }
     } else if constexpr (EPI == EPI_GROUPS) {
         // One decision per group of 8 columns: if the group's minimum passes the threshold, the
@@ -642,7 +662,11 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 }
             }
             if (lane == 0) {
-                for (; t < t1 && ok; ++t) ok = load_b(t);
+                int col = (t0 + col_rotation(T, G, NT, p.cross, r)) % NT;  // centroid tile of position t
+                for (; t < t1 && ok; ++t) {
+                    ok = load_b(col);
+                    if (++col == NT) col = 0;
+                }
             }
             ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
             ++seg;
@@ -824,9 +848,11 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 }
             }
 
+            int col = (t0 + col_rotation(T, G, NT, p.cross, r)) % NT;  // centroid tile of position t
             for (int t = t0; t < t1 && ok; ++t) {
-                const bool ragged = (t + 1) * p.block_n > p.nlist;
-                const int tile_j0 = t * p.block_n;
+                const bool ragged = (col + 1) * p.block_n > p.nlist;
+                const int tile_j0 = col * p.block_n;
+                if (++col == NT) col = 0;
 #pragma unroll
                 for (int h = 0; h < MT; ++h) {
                     const int su = it * MT + h;

@@ -1019,12 +1019,12 @@ int ivf_cluster_major_reorder(const void* points, ivf_dtype ptype, const int32_t
             const int row_chunks = row_bytes / 16;
             const int64_t pieces = n * row_chunks;
             reorder_gather_kernel<uint4><<<static_cast<unsigned>((pieces + 255) / 256), 256, 0, stream>>>(
-                static_cast<const uint4*>(points), out_order, n, row_chunks, static_cast<uint4*>(out_points));
+                static_cast<const uint4*>(points), out_order, n, row_chunks, off + nlist, static_cast<uint4*>(out_points));
         } else {
             const int row_chunks = row_bytes / 4;
             const int64_t pieces = n * row_chunks;
             reorder_gather_kernel<uint32_t><<<static_cast<unsigned>((pieces + 255) / 256), 256, 0, stream>>>(
-                static_cast<const uint32_t*>(points), out_order, n, row_chunks, static_cast<uint32_t*>(out_points));
+                static_cast<const uint32_t*>(points), out_order, n, row_chunks, off + nlist, static_cast<uint32_t*>(out_points));
         }
         LAUNCH_CHECK();
     }
@@ -1338,6 +1338,16 @@ int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int
     out[2] = cta_of_unit(pl.total_units, pl.ctas, pl.col_tiles, pl.cross, out[0]);
     out[3] = cta_of_unit(pl.total_units, pl.ctas, pl.col_tiles, pl.cross, out[1] - 1);
     return IVF_OK;
+}
+
+int ivf_debug_rotation(int64_t n, int nlist, int d, int k, int num_sms, int64_t row_group) {
+    if (n < 1 || nlist < 1 || num_sms < 1) return fail(IVF_ERR_INVALID_ARG, "bad plan arguments");
+    Plan pl;
+    int stride = 1;
+    int rc = make_plan(n, nlist, d, k, num_sms, &pl, k > 1 && choose_rule(k, nlist, &stride) != TAU_GIVEN);
+    if (rc != IVF_OK) return rc;
+    if (row_group < 0 || row_group >= pl.row_tiles) return fail(IVF_ERR_INVALID_ARG, "row group outside the plan");
+    return col_rotation(pl.total_units, pl.ctas, pl.col_tiles, pl.cross, row_group);
 }
 
 int ivf_debug_timing(int enable) {

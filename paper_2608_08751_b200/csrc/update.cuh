@@ -241,14 +241,21 @@ __global__ void update_combine_parts_kernel(const float* __restrict__ scratch, c
 }
 
 // Cluster-major copy (Sec. 3.1 index layout): destination row p receives source row order[p];
-// one thread per 16-byte piece of a row (4-byte pieces when a row is not a multiple of 16 bytes).  Also widens the list offsets to 64 bits.
+// one thread per 16-byte piece of a row (4-byte pieces when a row is not a multiple of 16 bytes).
+// Rows whose id was outside [0, nlist) were left out by the fill, so only the first *kept positions
+// of `order` hold a source row: the positions after them get order = -1 and a zeroed row.
 template <typename Piece>
-__global__ void reorder_gather_kernel(const Piece* __restrict__ src, const int* __restrict__ order, int64_t n,
-                                      int row_chunks, Piece* __restrict__ dst) {
+__global__ void reorder_gather_kernel(const Piece* __restrict__ src, int* __restrict__ order, int64_t n,
+                                      int row_chunks, const int* __restrict__ kept, Piece* __restrict__ dst) {
     const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (i >= n * row_chunks) return;
     const int64_t p = i / row_chunks;
     const int c = static_cast<int>(i - p * row_chunks);
+    if (p >= *kept) {
+        if (c == 0) order[p] = -1;
+        dst[i] = Piece{};
+        return;
+    }
     dst[i] = src[static_cast<int64_t>(order[p]) * row_chunks + c];
 }
 

@@ -104,6 +104,45 @@ def _check_schedule(n, nlist, d, k, sms):
     assert 2 * max(per_row_tile.values()) <= pl["partials"]  # two epilogue warps share every row
 
 
+@pytest.mark.parametrize("n,nlist,d,k", [(10000, 65536, 128, 64), (10000, 262144, 96, 128), (9984, 1 << 20, 96, 256),
+                                        (1 << 20, 65536, 128, 1), (300, 100000, 64, 8), (40000, 3000, 128, 1)])
+def test_rotated_sweeps_walk_the_table_as_a_few_fronts(n, nlist, d, k):
+    # Position p of row group r stands for centroid tile (p + rot_r) mod NT.  With every CTA advancing
+    # one unit per step (a row-group change costs `cross` steps), the tile a CTA works on minus the
+    # step count must take only a handful of values over all CTAs and steps: the CTAs then share a
+    # few fronts and a tile is fetched from HBM once per front, not once per row group.
+    sms = 148
+    pl = binding.ivf_debug_plan(n, nlist, d, k, sms)
+    NT, R = pl["col_tiles"], pl["row_tiles"]
+    cross = 8 if k == 1 else 4
+    rot = {}
+    offsets = set()
+    for b in range(pl["ctas"]):
+        u0, u1 = binding.ivf_debug_span(n, nlist, d, k, sms, b)
+        t = 0
+        u = u0
+        while u < u1:
+            r = u // NT
+            if r not in rot:
+                rot[r] = binding.ivf_debug_rotation(n, nlist, d, k, sms, r)
+                assert 0 <= rot[r] < NT
+            p0 = u - r * NT
+            p1 = min(u1 - r * NT, NT)
+            offsets.add(((p0 + rot[r]) - t) % NT)   # constant along a segment: tile and time advance together
+            t += (p1 - p0) + cross
+            u = r * NT + p1
+    spans_per_sweep = -(-NT * R // pl["ctas"])
+    fronts = -(-NT // max(1, spans_per_sweep - 2 * cross)) + 2
+    # a front may be smeared by the rounding of the span boundaries and the crossing charge
+    centres = sorted(offsets)
+    groups = 1
+    for a, bb in zip(centres, centres[1:]):
+        if bb - a > 4 * cross + 4:
+            groups += 1
+    assert groups <= fronts + 1, (groups, fronts, len(offsets))
+    assert rot[0] == 0
+
+
 def test_threshold_rule_selection():
     assert binding.ivf_debug_rule(1, 65536) == (-1, 1)
     assert binding.ivf_debug_rule(16, 65536) == (1, 16)           # threshold pass, can never come up short

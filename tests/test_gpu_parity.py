@@ -298,6 +298,33 @@ def test_cluster_major_reorder(dtype, n, nlist, d):
     assert (out == x[order]).all()
 
 
+@pytest.mark.parametrize("dtype,d", [("u8", 128), ("f32", 36)])
+def test_cluster_major_reorder_drops_rows_with_bad_ids(dtype, d):
+    # rows whose id is outside [0, nlist) are left out: the kept rows fill the front of the layout, the
+    # positions after them read order = -1 and a zero row, and the status word reports the bad ids
+    n, nlist = 5000, 300
+    rng = np.random.default_rng(17)
+    x = rng.integers(1, 256, (n, d)).astype(np.uint8) if dtype == "u8" else (rng.standard_normal((n, d)).astype(np.float32) + 5)
+    ids = rng.integers(0, nlist, n).astype(np.int32)
+    bad = rng.choice(n, 37, replace=False)
+    ids[bad[:20]] = -1 - rng.integers(0, 1000, 20).astype(np.int32)
+    ids[bad[20:]] = nlist + rng.integers(0, 1000, 17).astype(np.int32)
+    out, offsets, order = B.ivf_cluster_major_reorder(_cuda(x), _cuda(ids), nlist)
+    with pytest.raises(B.IvfError) as e:
+        B.ivf_check()
+    assert e.value.code == B.IVF_ERR_BAD_ID
+    out, offsets, order = out.cpu().numpy(), offsets.cpu().numpy(), order.cpu().numpy()
+    good = np.flatnonzero((ids >= 0) & (ids < nlist))
+    o_off, _ = oracle.reorder(ids[good], nlist)
+    kept = n - 37
+    assert (offsets == o_off).all() and offsets[-1] == kept
+    assert (np.sort(order[:kept]) == good).all()
+    assert (ids[order[:kept]] == np.repeat(np.arange(nlist), np.diff(o_off))).all()
+    assert (out[:kept] == x[order[:kept]]).all()
+    assert (order[kept:] == -1).all() and (out[kept:] == 0).all()
+    B.ivf_check()
+
+
 # ---------------------------------------------------------------- host streaming
 def test_route_from_pinned_host_memory():
     x, c = _rand(3000, 2000, 128, "u8", 12)
