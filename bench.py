@@ -39,12 +39,18 @@ WORKLOAD = ("C1 SIFT-shaped routing (10000 u8 queries x 65536 f32 centroids, d=1
 METRIC = "routed queries/s"
 UNIT = "queries/s"
 
-# DRAM bytes (read + write) per launch from the ncu captures summarised in profiles/.
-# k = 1 kernel: captured at 262,144 rows (54.5 MB, profiles/fused_argmin_262144x65536x128.md) and
-# scaled by 4 to the bench's 1,048,576-row launch (an upper bound: the centroid copy does not grow).
+# DRAM bytes (read + write) per launch, from ncu captures of single launches (dram__bytes_read.sum +
+# dram__bytes_write.sum).  k = 1 kernel: captured at 262,144 rows and scaled by 4 to the bench's
+# 1,048,576-row launch (an upper bound: the centroid copy does not grow with the rows).
 TRAFFIC_FUSED_ARGMIN_BYTES = 4 * (52.519424e6 + 1.968896e6)
-# k = 64 kernel: captured at the bench's own size (profiles/fused_groups_routing_c1_c2.md).
+# k = 64 kernel at the C1 size, k = 128 kernel at the C2 size, k = 256 kernel on one 9,984-row chunk of C4
+# (each captured at that size; None until a capture of the current kernel exists).
 TRAFFIC_FUSED_TOPK_BYTES = 93.999360e6 + 104.450560e6
+TRAFFIC_FUSED_C2_BYTES = None
+TRAFFIC_FUSED_C4_CHUNK_BYTES = None
+# roofline rates of whole routing calls: the slower of 2 n nlist d FLOP at the measured burst peak and
+# the minimum bytes at the measured HBM rate (tensor-bound for every configuration here)
+ROOFLINE_QPS = {"C1": 9.78e7, "C2": 3.26e7, "C4": 8.15e6}
 
 
 def peaks():
@@ -215,6 +221,136 @@ def pq_side_measurement(dev, pk, sm_max_mhz):
     }
 
 
+def _time_calls(fn, reps, flush, dev):
+    """Median and minimum milliseconds of `reps` calls, CUDA events around each call, the L2 flushed
+    (a buffer larger than L2 rewritten) before every call."""
+    import torch
+    ts = []
+    for _ in range(reps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize(dev)
+        ts.append(e0.elapsed_time(e1))
+    return statistics.median(ts), min(ts)
+
+
+def _oracle_sample(q_np, c_np, k, g_ids, g_dists, rows, label):
+    """The oracle, as it stands, on `rows` seeded rows of a routing batch: its rate and the agreement
+    of the GPU's lists with its own by the stated rule."""
+    from oracle import compare, oracle
+    sel = np.sort(np.random.default_rng(1).choice(q_np.shape[0], rows, replace=False))
+    sample = np.ascontiguousarray(q_np[sel])
+    t0 = time.perf_counter()
+    o_ids, o_d, _ = oracle.route(sample, c_np, k)
+    dt = time.perf_counter() - t0
+    a = compare.route_agreement(sample, c_np, k, g_ids[sel], g_dists[sel], oracle_result=(o_ids, o_d))
+    out = {"value": rows / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+           "sample": f"{rows} seeded rows of the {label} routing batch, full centroid width, {dt:.1f} s"}
+    out.update(compare.summary(a))
+    return out
+
+
+def routing_config_entry(cfg, label, dev, pk, flush, reps, traffic, oracle_rows, prepared_too=False):
+    """One timed ivf_route call of a full routing configuration, outside the headline timing: whole
+    call (median of `reps`, L2 flushed before each), the fused main pass from per-kernel events, the
+    roofline fractions, and an oracle sample with the agreement figures."""
+    import torch
+    from paper_2608_08751_b200 import binding as B
+    from paper_2608_08751_b200 import synth
+    q_np, c_np = synth.routing_inputs(cfg)
+    q, c = torch.from_numpy(q_np).to(dev), torch.from_numpy(c_np).to(dev)
+    ids = torch.empty((cfg.nq, cfg.nprobe), dtype=torch.int32, device=dev)
+    dists = torch.empty((cfg.nq, cfg.nprobe), dtype=torch.float32, device=dev)
+    for _ in range(2):
+        B.ivf_route(q, c, cfg.nprobe, ids, dists)
+    B.ivf_check(dev)
+    l0 = B.ivf_launch_count()
+    med, best = _time_calls(lambda: B.ivf_route(q, c, cfg.nprobe, ids, dists), reps, flush, dev)
+    launches = (B.ivf_launch_count() - l0) // reps
+    B.ivf_debug_timing(True)
+    for _ in range(reps):
+        flush.zero_()
+        B.ivf_route(q, c, cfg.nprobe, ids, dists)
+    fam = B.ivf_debug_timing_read()
+    B.ivf_debug_timing(False)
+    B.ivf_debug_stats(True)
+    B.ivf_route(q, c, cfg.nprobe, ids, dists)
+    stats = B.ivf_debug_stats(False)
+    B.ivf_check(dev)
+    flops = 2.0 * cfg.nq * cfg.nlist * cfg.d
+    fused_ms_call = fam["fused_topk"][0] / reps          # all row-chunk launches of one call
+    fused_launches = fam["fused_topk"][1] // reps
+    ach = flops / (fused_ms_call / 1e3) / 1e12
+    qps = cfg.nq / (med / 1e3)
+    entry = {
+        "workload": f"{cfg.name}: {cfg.nq} {cfg.qtype} queries x {cfg.nlist} f32 centroids, d={cfg.d}, nprobe={cfg.nprobe}",
+        "call_ms_median": med, "call_ms_min": best, "queries_per_s": qps,
+        "call_frac_of_roofline_rate": qps / ROOFLINE_QPS[label], "roofline_rate_qps": ROOFLINE_QPS[label],
+        "reps": reps, "l2": "flushed before every call", "launches_per_call": int(launches),
+        "kernel_ms_per_call": {name: v[0] / reps for name, v in fam.items() if v[1]},
+        "rows_recomputed_exactly_per_call": stats["fallback_rows"],
+        "log_records_per_row": stats["log_entries"] / cfg.nq,
+        "roofline": {"kernel": f"fused_topk_kernel (k={cfg.nprobe}, main pass, {fused_launches} row-chunk launch(es) per call)",
+                     "bound": "tensor", "achieved": ach, "peak": pk["tf_burst"], "unit": "TFLOP/s",
+                     "frac": ach / pk["tf_burst"], "frac_of_sustained": ach / pk["tf_sustained"],
+                     "traffic": traffic, "algorithmic_flops_per_call": flops,
+                     "peak_source": f"{pk['source']}: 16-bit dense, burst"},
+    }
+    if prepared_too:
+        h = B.PreparedCentroids(c)
+        for _ in range(2):
+            B.ivf_route_prepared(h, q, cfg.nprobe, ids, dists)
+        pmed, pbest = _time_calls(lambda: B.ivf_route_prepared(h, q, cfg.nprobe, ids, dists), reps, flush, dev)
+        B.ivf_check(dev)
+        h.close()
+        entry["prepared_table_call_ms_median"] = pmed
+        entry["prepared_table_queries_per_s"] = cfg.nq / (pmed / 1e3)
+        entry["prepared_table_frac_of_roofline_rate"] = cfg.nq / (pmed / 1e3) / ROOFLINE_QPS[label]
+    if oracle_rows:
+        entry["cpu_baseline"] = _oracle_sample(q_np, c_np, cfg.nprobe, ids.cpu().numpy(), dists.cpu().numpy(),
+                                               oracle_rows, label)
+    del q, c, ids, dists
+    torch.cuda.empty_cache()
+    return entry
+
+
+def serving_entry(dev, flush):
+    """Serving-size batches against a prepared 524,288-list table (uint8, d = 128, nprobe = 64):
+    microseconds per batch, back-to-back calls (the table is the L2-resident working set of a
+    serving loop, so nothing is flushed here)."""
+    import torch
+    from paper_2608_08751_b200 import binding as B
+    from paper_2608_08751_b200 import synth
+    nlist, k = 524_288, 64
+    c = torch.from_numpy(synth.sift_like_centroids(nlist, D)).to(dev)
+    h = B.PreparedCentroids(c)
+    q_all = synth.sift_like_queries(2048, D)
+    out = {"workload": f"prepared table, {nlist} lists, u8 d={D}, nprobe={k}; 50 back-to-back calls per batch size"}
+    for bs in (8, 2048):
+        q = torch.from_numpy(q_all[:bs]).to(dev)
+        ids = torch.empty((bs, k), dtype=torch.int32, device=dev)
+        dists = torch.empty((bs, k), dtype=torch.float32, device=dev)
+        for _ in range(5):
+            B.ivf_route_prepared(h, q, k, ids, dists)
+        B.ivf_check(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(50):
+            B.ivf_route_prepared(h, q, k, ids, dists)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        us = e0.elapsed_time(e1) / 50 * 1e3
+        out[f"B={bs}"] = {"us_per_batch": us, "queries_per_s": bs / (us / 1e6)}
+    B.ivf_check(dev)
+    h.close()
+    del c
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -223,6 +359,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-pq", action="store_true", help="skip the residual-PQ candidate-reduction side measurement")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="skip the side measurements of the C2 / C4 routing configurations and the serving batches")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else max(args.warmup, 0)
 
@@ -402,7 +540,7 @@ def main():
     prep_ms, prep_n = fam["prep"]
     flops_assign = 2.0 * CHUNK * NLIST * D
     flops_route = 2.0 * NQ * NLIST * D
-    peak_tf = pk["tf_sustained"]
+    peak_tf = pk["tf_burst"]
     ach_arg = flops_assign / (arg_ms / max(arg_n, 1) / 1e3) / 1e12 if arg_n else None
     ach_top = flops_route / (top_ms / max(top_n, 1) / 1e3) / 1e12 if top_n else None
     upd_bytes = CHUNK * D + CHUNK * 4 * 3 + NLIST * D * 4 * 2 + NLIST * 8 * 2
@@ -421,8 +559,11 @@ def main():
             "centroid_update": upd_ms / max(upd_n, 1)},
         "roofline": {"kernel": "fused_topk_kernel (k=1, 1048576 x 65536 x 128)", "bound": "tensor",
                      "achieved": ach_arg, "peak": peak_tf, "unit": "TFLOP/s",
-                     "frac": (ach_arg / peak_tf) if ach_arg else None, "traffic": TRAFFIC_FUSED_ARGMIN_BYTES,
-                     "peak_source": f"{pk['source']}: 16-bit dense, sustained"},
+                     "frac": (ach_arg / peak_tf) if ach_arg else None,
+                     "frac_of_sustained": (ach_arg / pk["tf_sustained"]) if ach_arg else None,
+                     "traffic": TRAFFIC_FUSED_ARGMIN_BYTES,
+                     "flops_counted": "2 n nlist d (the 16 norm columns of the operand rows, K padding and tail tiles get no credit)",
+                     "peak_source": f"{pk['source']}: 16-bit dense, burst (the sustained figure is secondary)"},
         "roofline_route": {"kernel": "fused_topk_kernel (k=64, 10000 x 65536 x 128)", "bound": "tensor",
                            "achieved": ach_top, "peak": pk["tf_burst"], "unit": "TFLOP/s",
                            "frac": (ach_top / pk["tf_burst"]) if ach_top else None,
@@ -433,7 +574,10 @@ def main():
                             "frac": (upd_bytes / (upd_ms / max(upd_n, 1) / 1e3) / 1e9 / pk["hbm_gbs"]) if upd_n else None,
                             "traffic": None, "peak_source": pk["source"]},
         "e2e": {"value": world * NQ * K / (t_e2e / 1e3), "unit": UNIT, "h2d_bytes_per_step": NQ * D,
-                "d2h_bytes_per_step": NQ * NPROBE * 8},
+                "d2h_bytes_per_step": NQ * NPROBE * 8,
+                "note": "queries cross the host link inside ivf_route (host input through the C-ABI); the C-ABI writes "
+                        "results to device memory only, so the read-back to page-locked host memory is a torch copy "
+                        "on a second stream, outside the C-ABI, inside the timed region"},
         "e2e_assign": {"value": world * CHUNK * K / (t_e2e_a / 1e3), "unit": "vectors/s",
                        "h2d_bytes_per_step": CHUNK * D, "d2h_bytes_per_step": CHUNK * 4,
                        "host_link_GBps": CHUNK * D * K / (t_e2e_a / 1e3) / 1e9},
@@ -445,6 +589,22 @@ def main():
 
     if not args.no_pq and world == 1:
         line["pq"] = pq_side_measurement(dev, pk, clocks["sm_max_mhz"])
+
+    if not args.no_extra and world == 1:
+        # side measurements, outside the headline timing: the other routing configurations on this
+        # GPU (one timed call each, oracle samples beside them) and serving-size batches
+        from paper_2608_08751_b200 import synth
+        oc = 0 if args.no_cpu_baseline else 1
+        line["c1_call"] = routing_config_entry(synth.C1, "C1", dev, pk, flush, 10, TRAFFIC_FUSED_TOPK_BYTES, 0,
+                                               prepared_too=True)
+        line["c2"] = routing_config_entry(synth.C2, "C2", dev, pk, flush, 10, TRAFFIC_FUSED_C2_BYTES, 768 * oc,
+                                          prepared_too=True)
+        line["c4"] = routing_config_entry(synth.C4, "C4", dev, pk, flush, 5, TRAFFIC_FUSED_C4_CHUNK_BYTES, 384 * oc)
+        line["serving"] = serving_entry(dev, flush)
+        line["config"]["side_measurements"] = ("c1_call, c2, c4: one timed ivf_route call of the C1 / C2 (10000 x 262144 x 96, "
+                                               "nprobe 128) / C4 (100000 x 1048576 x 96, nprobe 256) configurations, CUDA "
+                                               "events, L2 flushed before each call; serving: B = 8 and 2048 against a "
+                                               "prepared 524288-list table; pq: residual-PQ candidate reduction")
 
     if not args.no_cpu_baseline and world == 1:
         from oracle import oracle
@@ -460,26 +620,16 @@ def main():
         t0 = time.perf_counter()
         o_ids, o_d, _ = oracle.route(sample, cent_np, NPROBE)
         dt = time.perf_counter() - t0
-        g_ids = out_ids.cpu().numpy()[sel]
+        from oracle import compare
+        B.ivf_route(queries, cent_route, NPROBE, out_ids, out_dists)
+        B.ivf_check(dev)
         # agreement with the oracle by the stated rule (outside the timed part): an id list may differ
         # from the oracle's only where the true distances involved lie within 1e-3 (|x|^2 + |c|^2)
-        xn, cn = oracle.sqnorms(sample), oracle.sqnorms(cent_np)
-        rr = np.repeat(np.arange(rows, dtype=np.int64), NPROBE)
-        d_true = oracle.pair_dists(sample, cent_np, rr, g_ids.ravel().astype(np.int64)).reshape(rows, NPROBE)
-        tol_g = 1e-3 * (xn[:, None] + cn[g_ids])
-        tol_o = 1e-3 * (xn[:, None] + cn[o_ids])
-        dk = o_d[:, -1]
-        must = o_d < (dk[:, None] - tol_o)
-        present = (o_ids[:, :, None] == g_ids[:, None, :]).any(-1)
-        differs = g_ids != o_ids
-        lower = np.maximum.accumulate(d_true - tol_g, axis=1)
-        row_ok = ((present | ~must).all(axis=1) & (d_true <= dk[:, None] + tol_g).all(axis=1)
-                  & (lower[:, :-1] <= (d_true + tol_g)[:, 1:]).all(axis=1))
+        a = compare.route_agreement(sample, cent_np, NPROBE, out_ids.cpu().numpy()[sel], out_dists.cpu().numpy()[sel],
+                                    oracle_result=(o_ids, o_d))
         line["cpu_baseline"] = {"value": rows / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "sample": f"{rows} seeded rows of the C1 routing batch, full centroid width, {dt:.1f} s",
-                                "rows_matching_oracle_by_tolerance_rule": float(row_ok.mean()),
-                                "rows_with_identical_id_lists": float((~differs).all(axis=1).mean()),
-                                "top_k_set_overlap": float(present.mean())}
+                                "sample": f"{rows} seeded rows of the C1 routing batch, full centroid width, {dt:.1f} s"}
+        line["cpu_baseline"].update(compare.summary(a))
     print(json.dumps(line), flush=True)
     if distributed:
         dist.destroy_process_group()

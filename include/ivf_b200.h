@@ -128,7 +128,11 @@ int ivf_centroid_update(const void* points, ivf_dtype ptype, const int32_t* ids,
  *            accumulation composes).  Other arguments, layouts and results are those of
  *            ivf_centroid_update.
  *   Set-up   the first call on each device looks up the array's device address (with that device
- *            current); make that first call before starting any stream capture.
+ *            current); make that first call before starting any stream capture.  The array is part
+ *            of the library image, and the CUDA runtime places an image on a device when the
+ *            library is first used there: so make that first call (or any other call into the
+ *            library) on each device before the device's free memory is handed to the serving
+ *            pool -- afterwards there may be no room left for the image itself.
  *   Sharing  all calls on a device use the one array, which still holds the previous call's
  *            contents (the call clears what it needs cleared).  Two calls whose kernels overlap on
  *            the GPU -- different streams without an ordering between them -- race on it: keep the
@@ -209,6 +213,9 @@ int ivf_debug_span(int64_t n, int nlist, int d, int k, int num_sms, int cta, int
  * row group's sweep stands for centroid tile (p + rotation) mod col_tiles, so that the CTAs walk the
  * centroid table as a few shared fronts.  Returns the rotation (>= 0) or a negative status. */
 int ivf_debug_rotation(int64_t n, int nlist, int d, int k, int num_sms, int64_t row_group);
+/* Measurement hook: 0 switches the rotation off (every position stands for its own tile index), so that
+ * the two sweep orders can be timed against each other; results do not depend on it.  Default 1. */
+int ivf_debug_set_rotation(int on);
 int ivf_debug_set_wait_limit_ns(int64_t ns);
 int ivf_debug_wait_probe(void* stream);
 /* Test hook: when on, the merge of a k > 1 call declares every row's candidate set insufficient, so
@@ -266,6 +273,22 @@ int ivf_debug_timing_read(double ms[9], int64_t launches[9]);
  */
 int ivf_assign_candidates(const void* points, int64_t n, int d, ivf_dtype ptype, const float* centroids, int nlist,
                           const int32_t* cand_ids, int m, int32_t* out_ids, float* out_dists, void* stream);
+
+/*
+ * Merge step of routing against a centroid table that is split over several GPUs (Sec. 4.1: finer
+ * partitions, N_list up to millions; Eq. 1: the P nearest centroids overall are the P smallest of
+ * the shards' P nearest).  Every GPU routes the queries against its own shard with ivf_route and
+ * adds its shard's first global id to the ids; the [nq, k] results of all shards are gathered
+ * (an all-gather) into
+ *   shard_ids    [parts][nq][k] int32, shard_dists [parts][nq][k] float32: device; each list
+ *                ascending by (distance, id); a shard with fewer than k centroids fills the unused
+ *                places with +inf;
+ * and this call writes the k smallest pairs by (distance, id) per query, ascending, to
+ *   out_ids [nq][k] int32, out_dists [nq][k] float32 (may be NULL): device.
+ * k <= 512; any number of parts.  Equal distances are settled by the lower global id.
+ */
+int ivf_merge_shards(const int32_t* shard_ids, const float* shard_dists, int parts, int64_t nq, int k,
+                     int32_t* out_ids, float* out_dists, void* stream);
 
 /*
  * Residual-PQ candidate reduction (Sec. 2.2 Eq. 3-5; Sec. 4.3; Sec. 4.4).  K = 256 codewords per

@@ -23,9 +23,9 @@ EXPORTS = (
     "ivf_route", "ivf_assign", "ivf_centroid_update", "ivf_centroid_update_noalloc", "ivf_centroid_finalize",
     "ivf_assign_update", "ivf_cluster_major_reorder", "ivf_centroids_create", "ivf_centroids_destroy",
     "ivf_route_prepared",
-    "ivf_pq_encode", "ivf_pq_search", "ivf_pq_residuals", "ivf_assign_candidates",
+    "ivf_pq_encode", "ivf_pq_search", "ivf_pq_residuals", "ivf_assign_candidates", "ivf_merge_shards",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
-    "ivf_debug_plan", "ivf_debug_span", "ivf_debug_rotation", "ivf_debug_set_wait_limit_ns",
+    "ivf_debug_plan", "ivf_debug_span", "ivf_debug_rotation", "ivf_debug_set_rotation", "ivf_debug_set_wait_limit_ns",
     "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_set_row_chunk", "ivf_debug_stats", "ivf_debug_set_pq_groups", "ivf_debug_set_dependent_launch", "ivf_debug_set_crossing_cost",
 )
 
@@ -76,6 +76,7 @@ def lib() -> ctypes.CDLL:
     L.ivf_debug_stats.argtypes = [i32, ctypes.POINTER(i64)]
     L.ivf_debug_rule.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_int)]
     L.ivf_assign_candidates.argtypes = [vp, i64, i32, i32, vp, i32, vp, i32, vp, vp, vp]
+    L.ivf_merge_shards.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
     L.ivf_pq_residuals.argtypes = [vp, i64, i32, i32, vp, vp, i32, vp, vp]
     L.ivf_pq_encode.argtypes = [vp, i64, i32, i32, vp, vp, i32, vp, i32, vp, vp]
     L.ivf_pq_search.argtypes = [vp, i64, i32, i32, vp, i32, vp, i32, vp, vp, i64, vp, i32, i32, vp, vp, vp, vp, vp]
@@ -303,6 +304,25 @@ def ivf_assign_candidates(points: torch.Tensor, centroids: torch.Tensor, cand_id
     return out_ids, out_dists
 
 
+def ivf_merge_shards(shard_ids: torch.Tensor, shard_dists: torch.Tensor):
+    """[parts, nq, k] per-shard routing results (global ids) -> (ids [nq, k] int32, dists [nq, k] float32):
+    the k smallest pairs by (distance, id) per query."""
+    _dev(shard_ids, "shard_ids", torch.int32)
+    _dev(shard_dists, "shard_dists", torch.float32)
+    if shard_ids.dim() != 3 or shard_ids.shape != shard_dists.shape:
+        raise ValueError("shard_ids and shard_dists must both be [parts, nq, k]")
+    parts, nq, k = shard_ids.shape
+    dev = shard_ids.device
+    out_ids = torch.empty((nq, k), dtype=torch.int32, device=dev)
+    out_dists = torch.empty((nq, k), dtype=torch.float32, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib().ivf_merge_shards(_ptr(shard_ids), _ptr(shard_dists), parts, nq, k, _ptr(out_ids), _ptr(out_dists),
+                                    _stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
+    return out_ids, out_dists
+
+
 def _codebooks(codebooks: torch.Tensor, d: int) -> int:
     _dev(codebooks, "codebooks", torch.float32)
     if codebooks.dim() != 3 or codebooks.shape[1] != 256 or codebooks.shape[0] * codebooks.shape[2] != d:
@@ -460,6 +480,10 @@ def ivf_debug_rotation(n: int, nlist: int, d: int, k: int, num_sms: int, row_gro
     if rc < 0:
         _raise(rc)
     return int(rc)
+
+
+def ivf_debug_set_rotation(on: bool) -> None:
+    lib().ivf_debug_set_rotation(1 if on else 0)
 
 
 def ivf_debug_set_wait_limit_ns(ns: int) -> None:

@@ -74,6 +74,7 @@ struct FusedParams {
     int col_tiles;        // centroid tiles per sweep
     int64_t total_units;  // row groups * col_tiles
     int cross;            // cost of a mid-span row-group crossing in units (span partition)
+    int rotate;           // 1: centroid tiles of a row group are swept in the rotated order (col_rotation)
     int partials;         // partial-result slots per row (CTAs sharing a row tile x kEpiHalves)
     int cap;              // candidate-log capacity per (row, slot), k > 1 only
     int rule;             // k > 1: TAU_RUNNING, TAU_GIVEN or TAU_BOUNDED
@@ -662,7 +663,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 }
             }
             if (lane == 0) {
-                int col = (t0 + col_rotation(T, G, NT, p.cross, r)) % NT;  // centroid tile of position t
+                int col = (t0 + (p.rotate ? col_rotation(T, G, NT, p.cross, r) : 0)) % NT;  // centroid tile of position t
                 for (; t < t1 && ok; ++t) {
                     ok = load_b(col);
                     if (++col == NT) col = 0;
@@ -848,7 +849,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 }
             }
 
-            int col = (t0 + col_rotation(T, G, NT, p.cross, r)) % NT;  // centroid tile of position t
+            int col = (t0 + (p.rotate ? col_rotation(T, G, NT, p.cross, r) : 0)) % NT;  // centroid tile of position t
             for (int t = t0; t < t1 && ok; ++t) {
                 const bool ragged = (col + 1) * p.block_n > p.nlist;
                 const int tile_j0 = col * p.block_n;

@@ -246,6 +246,7 @@ int choose_rule(int k, int nlist, int* stride) {
     return k <= kSampleM ? TAU_RUNNING : TAU_BOUNDED;
 }
 
+int g_rotate = 1;  // test hook (ivf_debug_set_rotation): 0 = every position of a sweep stands for its own tile index
 int g_cross = -1;  // crossing cost used by the span partition; -1 = by kernel variant (test hook: ivf_debug_set_crossing_cost)
 
 int make_plan(int64_t n, int nlist, int d, int k, int num_sms, Plan* pl, bool one_row_tile = false) {
@@ -462,6 +463,7 @@ int launch_fused(DeviceCtx& ctx, const Plan& pl, int64_t n, int nlist, int k, in
     fp.col_tiles = pl.col_tiles;
     fp.total_units = pl.total_units;
     fp.cross = pl.cross;
+    fp.rotate = g_rotate;
     fp.partials = pl.partials;
     fp.cap = pl.cap;
     fp.rule = rule;
@@ -1055,6 +1057,27 @@ int ivf_assign_update(const void* points, int64_t n, int d, ivf_dtype ptype, con
                       static_cast<cudaStream_t>(stream));
 }
 
+int ivf_merge_shards(const int32_t* shard_ids, const float* shard_dists, int parts, int64_t nq, int k,
+                     int32_t* out_ids, float* out_dists, void* stream_) {
+    if (nq < 0) return fail(IVF_ERR_INVALID_ARG, "negative query count %lld", (long long)nq);
+    if (parts < 1) return fail(IVF_ERR_INVALID_ARG, "parts = %d", parts);
+    if (k < 1 || k > kFallbackMaxK) return fail(IVF_ERR_UNSUPPORTED, "k = %d: must be in [1, %d]", k, kFallbackMaxK);
+    if (nq >= (int64_t(1) << 31)) return fail(IVF_ERR_UNSUPPORTED, "nq = %lld: at most 2^31 - 1 queries per call", (long long)nq);
+    if (nq == 0) return IVF_OK;
+    if (!shard_ids || !shard_dists || !out_ids) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
+    ShardMergeParams sp;
+    sp.nq = nq;
+    sp.k = k;
+    sp.parts = parts;
+    sp.ids = shard_ids;
+    sp.dists = shard_dists;
+    sp.out_ids = out_ids;
+    sp.out_dists = out_dists;
+    merge_shards_kernel<<<static_cast<unsigned>(nq), kMergeThreads, 0, static_cast<cudaStream_t>(stream_)>>>(sp);
+    LAUNCH_CHECK();
+    return IVF_OK;
+}
+
 int ivf_assign_candidates(const void* points, int64_t n, int d, ivf_dtype ptype, const float* centroids, int nlist,
                           const int32_t* cand_ids, int m, int32_t* out_ids, float* out_dists, void* stream_) {
     if (n < 0) return fail(IVF_ERR_INVALID_ARG, "negative row count %lld", (long long)n);
@@ -1414,6 +1437,11 @@ int ivf_debug_set_dependent_launch(int on) {
     return IVF_OK;
 }
 
+int ivf_debug_set_rotation(int on) {
+    g_rotate = on != 0;
+    return IVF_OK;
+}
+
 int ivf_debug_set_crossing_cost(int units) {
     g_cross = units;  // negative: chosen by kernel variant
     return IVF_OK;
@@ -1450,7 +1478,8 @@ int ivf_debug_set_wait_limit_ns(int64_t ns) {
 // ====================================================================== allocation-free update
 // Scratch of ivf_centroid_update_noalloc: lives in the module image, so every device that loads
 // the library holds these ~4.8 MB until the process exits.  Layout (ints):
-//   [0, 8)                         header: [0] = "an id was out of range" flag of the last call
+//   [0, 8)                         header: [0] = "an id was out of range" flag of the last call (written by
+//                                  the histogram kernel, read by nobody yet: reserved), [1..7] unused
 //   [8, 8 + L)                     per-list member counts of the call        (L = kNoAllocMaxLists)
 //   [8 + L, 8 + 2L + 1)            exclusive offsets of the list segments
 //   [8 + 2L + 8, 8 + 2L + 40)      partial totals of the offset scan (one per 4096 lists)

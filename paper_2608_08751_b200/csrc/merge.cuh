@@ -905,4 +905,44 @@ __global__ void __launch_bounds__(kMergeThreads) route_tail_kernel(const TailPar
     }
 }
 
+// ------------------------------------------------------------------ merge of centroid shards
+// When the centroid table is split over several GPUs (tables too large to replicate; Sec. 4.1 sweeps
+// N_list up to 4M), every GPU routes the queries against its own shard and the [nq, k] lists of all
+// shards are gathered: this kernel merges, per query, `parts` lists of k (distance, global id) pairs
+// -- each ascending, unused places holding (+inf, any id) -- into the k smallest by (distance, id).
+// One CTA per query; the running result and the next shard's list are sorted together in shared
+// memory (at most 2 * 512 keys), shard after shard, so any number of shards is taken.
+struct ShardMergeParams {
+    int64_t nq;
+    int k, parts;
+    const int32_t* ids;    // [parts][nq][k]
+    const float* dists;    // [parts][nq][k]
+    int32_t* out_ids;      // [nq][k]
+    float* out_dists;      // [nq][k] or nullptr
+};
+
+__global__ void __launch_bounds__(kMergeThreads) merge_shards_kernel(const ShardMergeParams p) {
+    __shared__ uint64_t keys[2 * kFallbackMaxK];
+    const int64_t q = blockIdx.x;
+    int m = 2;
+    while (m < 2 * p.k) m <<= 1;
+    auto load = [&](int part, int base) {
+        const size_t at = (static_cast<size_t>(part) * p.nq + q) * p.k;
+        for (int i = threadIdx.x; i < p.k; i += blockDim.x)
+            keys[base + i] = (static_cast<uint64_t>(orderable(p.dists[at + i])) << 32) | static_cast<uint32_t>(p.ids[at + i]);
+    };
+    load(0, 0);
+    for (int part = 1; part < p.parts; ++part) {
+        load(part, p.k);
+        for (int i = 2 * p.k + threadIdx.x; i < m; i += blockDim.x) keys[i] = ~0ull;
+        bitonic_sort_smem(keys, m);  // begins and ends with a barrier
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < p.k; i += blockDim.x) {
+        const uint64_t key = keys[i];
+        p.out_ids[q * p.k + i] = static_cast<int32_t>(key & 0xFFFFFFFFull);
+        if (p.out_dists) p.out_dists[q * p.k + i] = from_orderable(static_cast<uint32_t>(key >> 32));
+    }
+}
+
 }  // namespace ivf

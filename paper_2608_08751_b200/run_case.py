@@ -25,17 +25,39 @@ from . import binding as B
 from . import synth
 
 
-def stream_case(args):
+def _fill_chunks(host, args):
+    """Seeded rows into the page-locked buffer, chunk by chunk (the recipe of the full configuration);
+    numpy's generators release the interpreter lock, so a thread pool spreads the chunks over the cores."""
+    from concurrent.futures import ThreadPoolExecutor
+    import os
     chunk = synth.CHUNK_ROWS
     nchunks = -(-args.n // chunk)
-    host = torch.empty((args.n, args.d), dtype=torch.uint8 if args.dtype == "u8" else torch.float32).pin_memory()
-    for c in range(nchunks):  # the same seeded chunk recipe as the full configuration
+    view = host.numpy()
+
+    def fill(c):
         rows = min(chunk, args.n - c * chunk)
         if args.dtype == "u8":
-            blk = synth.sift_like_rows(c, rows=rows, d=args.d)
+            view[c * chunk:c * chunk + rows] = synth.sift_like_rows(c, rows=rows, d=args.d)
         else:
-            blk = synth.deep_like_rows(c, rows=rows, d=args.d)
-        host[c * chunk:c * chunk + rows] = torch.from_numpy(blk)
+            view[c * chunk:c * chunk + rows] = synth.deep_like_rows(c, rows=rows, d=args.d)
+
+    with ThreadPoolExecutor(max_workers=min(32, os.cpu_count() or 1)) as pool:
+        list(pool.map(fill, range(nchunks)))
+    return nchunks
+
+
+def stream_case(args, checker=None):
+    """The IVF-build configuration: rows in page-locked host memory, streamed in 1,048,576-row chunks
+    through assign + update, then the finalize, per Lloyd iteration.  Every iteration is timed on its
+    own with CUDA events.  `checker`, if given, is called between iterations (outside the timing) as
+    checker(sample_rows, centroids_used, ids_of_sample, dists_of_sample) -> dict on --check-rows seeded
+    rows; what it returns is added to the iteration's record (the test tree passes a checker that
+    re-assigns the rows on the CPU).  The per-list counts are compared with a bincount of all ids."""
+    import time
+    t_gen = time.perf_counter()
+    host = torch.empty((args.n, args.d), dtype=torch.uint8 if args.dtype == "u8" else torch.float32).pin_memory()
+    nchunks = _fill_chunks(host, args)
+    t_gen = time.perf_counter() - t_gen
     init = synth.init_sample(args.n, args.nlist)
     cent = host[torch.from_numpy(init)].to(torch.float32).cuda()
     sums = torch.zeros((args.nlist, args.d), dtype=torch.float32, device="cuda")
@@ -49,22 +71,47 @@ def stream_case(args):
         B.ivf_assign_update(host, cent, sums, counts, ids, dists)
         B.ivf_centroid_finalize(sums, counts, cent)
 
-    iteration()  # warm-up (workspace growth)
+    # warm-up on a few chunks (workspace growth), on a copy of the centroids
+    keep = cent.clone()
+    sums.zero_()
+    counts.zero_()
+    B.ivf_assign_update(host[:min(args.n, 4 * synth.CHUNK_ROWS)], cent, sums, counts, ids, dists)
     B.ivf_check()
-    inertia = []
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.iters):
+    cent.copy_(keep)
+    check_rows = min(args.check_rows, args.n) if checker is not None else 0
+    sel = np.sort(np.random.default_rng(33).choice(args.n, check_rows, replace=False)) if check_rows else None
+    sample = np.ascontiguousarray(host.numpy()[sel]) if check_rows else None
+    per_iter = []
+    for it in range(args.iters):
+        c_now = cent.cpu().numpy().copy() if check_rows else None
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
         iteration()
-        inertia.append(float(dists.double().sum().item()))
-    e1.record()
-    B.ivf_check()
-    ms = e0.elapsed_time(e1) / args.iters
-    esize = 1 if args.dtype == "u8" else 4
+        e1.record()
+        B.ivf_check()
+        ms = e0.elapsed_time(e1)
+        esize = 1 if args.dtype == "u8" else 4
+        rec = {"iteration": it, "ms": ms, "vectors_per_s": args.n / (ms / 1e3),
+               "host_link_GBps": args.n * args.d * esize / (ms / 1e3) / 1e9,
+               "tflops": 2.0 * args.n * args.nlist * args.d / (ms / 1e3) / 1e12,
+               "inertia": float(dists.double().sum().item()),
+               "counts_total": int(counts.sum().item()), "empty_lists": int((counts == 0).sum().item())}
+        if check_rows:
+            at = torch.from_numpy(sel).cuda()
+            rec.update(checker(sample, c_now, ids[at].cpu().numpy(), dists[at].cpu().numpy()))
+        rec["counts_equal_bincount_of_all_ids"] = bool(
+            (np.bincount(ids.cpu().numpy(), minlength=args.nlist) == counts.cpu().numpy()).all())
+        per_iter.append(rec)
+    total_ms = sum(r["ms"] for r in per_iter)
+    inertia = [r["inertia"] for r in per_iter]
     print(json.dumps({"op": "stream", "n": args.n, "nlist": args.nlist, "d": args.d, "dtype": args.dtype,
-                      "chunks": nchunks, "ms_per_iteration": ms, "vectors_per_s": args.n / (ms / 1e3),
-                      "host_link_GBps": args.n * args.d * esize / (ms / 1e3) / 1e9,
-                      "tflops": 2.0 * args.n * args.nlist * args.d / (ms / 1e3) / 1e12, "inertia": inertia}))
+                      "chunks": nchunks, "iterations": per_iter, "total_ms": total_ms,
+                      "ms_per_iteration": total_ms / args.iters, "vectors_per_s": args.n * args.iters / (total_ms / 1e3),
+                      "host_link_GBps": args.n * args.d * (1 if args.dtype == "u8" else 4) * args.iters / (total_ms / 1e3) / 1e9,
+                      "tflops": 2.0 * args.n * args.nlist * args.d * args.iters / (total_ms / 1e3) / 1e12,
+                      "inertia": inertia,
+                      "inertia_non_increasing": all(b <= a * (1 + 1e-6) for a, b in zip(inertia, inertia[1:])),
+                      "host_generation_s": t_gen}))
 
 
 def build_case(args):
@@ -75,10 +122,7 @@ def build_case(args):
     chunk = synth.CHUNK_ROWS
     nchunks = -(-args.n // chunk)
     host = torch.empty((args.n, args.d), dtype=torch.uint8 if args.dtype == "u8" else torch.float32).pin_memory()
-    for c in range(nchunks):
-        rows = min(chunk, args.n - c * chunk)
-        blk = synth.sift_like_rows(c, rows=rows, d=args.d) if args.dtype == "u8" else synth.deep_like_rows(c, rows, args.d)
-        host[c * chunk:c * chunk + rows] = torch.from_numpy(blk)
+    _fill_chunks(host, args)
     train_rows = min(args.train_rows, args.n)
     train = host[:train_rows]
     init = synth.init_sample(train_rows, args.nlist)
@@ -261,6 +305,8 @@ def main():
     ap.add_argument("--n-rerank", type=int, default=512, dest="n_rerank")
     ap.add_argument("--batches", default="8,32,256,2048", help="query batch sizes of --op serve")
     ap.add_argument("--iters", type=int, default=1, help="Lloyd iterations of --op stream")
+    ap.add_argument("--check-rows", type=int, default=0, dest="check_rows",
+                    help="--op stream: seeded rows per iteration handed to the checker callback, if one is given")
     ap.add_argument("--n", type=int, default=262144)
     ap.add_argument("--nlist", type=int, default=65536)
     ap.add_argument("--d", type=int, default=128)
@@ -269,7 +315,9 @@ def main():
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--dependent-launch", type=int, default=-1, help="kernel-family mask of dependent launches (0 = none)")
     ap.add_argument("--crossing-cost", type=int, default=-1, help="span-partition crossing cost in units (0 = equal counts)")
+    ap.add_argument("--rotation", type=int, default=1, help="0 = centroid tiles swept in index order (for comparison)")
     args = ap.parse_args()
+    B.ivf_debug_set_rotation(bool(args.rotation))
     if args.crossing_cost >= 0:
         B.ivf_debug_set_crossing_cost(args.crossing_cost)
     if args.dependent_launch >= 0:

@@ -193,29 +193,58 @@ def test_no_distances_requested():
     assert (ids.cpu().numpy() == ids2).all()
 
 
-# ---------------------------------------------------------------- full-size configurations, sampled rows
-def _sampled_full(cfg, sample):
+# ---------------------------------------------------------------- full-size configurations
+def _full_size(cfg, sample, stats=False):
+    """The whole configuration through the C-ABI in its production launch shape; the full oracle on
+    `sample` rows spread evenly over the batch (so every row chunk of a chunked call is hit) plus a
+    seeded random draw, and the definition re-checked for every returned (row, id) pair."""
     q, c = synth.routing_inputs(cfg)
+    if stats:
+        B.ivf_debug_stats(True)
     ids, dists = _route(q, c, cfg.nprobe)
-    rows = np.random.default_rng(cfg.index).choice(cfg.nq, sample, replace=False)
-    st = parity.check_route(q, c, cfg.nprobe, ids[rows], dists[rows], rows=rows)
-    # properties that hold at any size, for all rows
-    assert ((ids >= 0) & (ids < cfg.nlist)).all() and (np.diff(dists, axis=1) >= 0).all()
-    s = np.sort(ids, 1)
-    assert (s[:, 1:] != s[:, :-1]).all()
-    return st
+    st = B.ivf_debug_stats(False) if stats else None
+    even = np.linspace(0, cfg.nq - 1, sample // 2).astype(np.int64)
+    rnd = np.random.default_rng(cfg.index).choice(cfg.nq, sample - even.size, replace=False)
+    rows = np.unique(np.concatenate([even, rnd]))
+    res = parity.check_route(q, c, cfg.nprobe, ids[rows], dists[rows], rows=rows)
+    parity.check_all_row_distances(q, c, cfg.nprobe, ids, dists)
+    return res, st, (q, c, ids, dists)
 
 
-def test_config1_sift_shaped_full_size_sampled():
-    _sampled_full(synth.C1, 96)
+def test_config1_sift_shaped_full_size():
+    res, _, _ = _full_size(synth.C1, 2048)
+    assert res["rows"] >= 2000
 
 
-def test_config2_deep_shaped_full_size_sampled():
-    _sampled_full(synth.C2, 32)
+def test_config2_deep_shaped_full_size():
+    res, _, _ = _full_size(synth.C2, 1024)
+    assert res["rows"] >= 1000
 
 
-def test_config4_stress_full_size_sampled():
-    _sampled_full(synth.C4, 8)
+def test_config4_stress_full_size():
+    # 11 row chunks; 2,048 oracle rows spread over all of them
+    res, st, _ = _full_size(synth.C4, 2048, stats=True)
+    assert res["rows"] >= 2000
+    assert st["fallback_rows"] <= 0.001 * synth.C4.nq
+
+
+def test_config4_shape_rows_through_the_exact_recomputation():
+    # the recomputation path at the C4 table size (128 centroid slices per row): a C4-shaped subset
+    # of rows is forced through it and must agree with the oracle like any other result
+    cfg = synth.C4
+    q, c = synth.routing_inputs(cfg)
+    sub = np.ascontiguousarray(q[np.random.default_rng(44).choice(cfg.nq, 48, replace=False)])
+    B.ivf_debug_stats(True)
+    B.ivf_debug_force_fallback(True)
+    try:
+        ids, dists = _route(sub, c, cfg.nprobe)
+    finally:
+        B.ivf_debug_force_fallback(False)
+    st = B.ivf_debug_stats(False)
+    assert st["fallback_rows"] == 48
+    parity.check_route(sub, c, cfg.nprobe, ids, dists)
+    ids2, dists2 = _route(sub, c, cfg.nprobe)  # the regular path gives the same lists
+    assert (ids2 == ids).all()
 
 
 def test_config3_chunk_assignment_full_width_sampled():
