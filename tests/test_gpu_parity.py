@@ -203,9 +203,10 @@ def _full_size(cfg, sample, stats=False):
         B.ivf_debug_stats(True)
     ids, dists = _route(q, c, cfg.nprobe)
     st = B.ivf_debug_stats(False) if stats else None
-    even = np.linspace(0, cfg.nq - 1, sample // 2).astype(np.int64)
-    rnd = np.random.default_rng(cfg.index).choice(cfg.nq, sample - even.size, replace=False)
-    rows = np.unique(np.concatenate([even, rnd]))
+    even = np.unique(np.linspace(0, cfg.nq - 1, sample // 2).astype(np.int64))
+    rest = np.setdiff1d(np.arange(cfg.nq), even)
+    rnd = np.random.default_rng(cfg.index).choice(rest, sample - even.size, replace=False)
+    rows = np.sort(np.concatenate([even, rnd]))
     res = parity.check_route(q, c, cfg.nprobe, ids[rows], dists[rows], rows=rows)
     parity.check_all_row_distances(q, c, cfg.nprobe, ids, dists)
     return res, st, (q, c, ids, dists)
@@ -213,18 +214,18 @@ def _full_size(cfg, sample, stats=False):
 
 def test_config1_sift_shaped_full_size():
     res, _, _ = _full_size(synth.C1, 2048)
-    assert res["rows"] >= 2000
+    assert res["rows"] == 2048
 
 
 def test_config2_deep_shaped_full_size():
     res, _, _ = _full_size(synth.C2, 1024)
-    assert res["rows"] >= 1000
+    assert res["rows"] == 1024
 
 
 def test_config4_stress_full_size():
     # 11 row chunks; 2,048 oracle rows spread over all of them
     res, st, _ = _full_size(synth.C4, 2048, stats=True)
-    assert res["rows"] >= 2000
+    assert res["rows"] == 2048
     assert st["fallback_rows"] <= 0.001 * synth.C4.nq
 
 
@@ -243,8 +244,12 @@ def test_config4_shape_rows_through_the_exact_recomputation():
     st = B.ivf_debug_stats(False)
     assert st["fallback_rows"] == 48
     parity.check_route(sub, c, cfg.nprobe, ids, dists)
-    ids2, dists2 = _route(sub, c, cfg.nprobe)  # the regular path gives the same lists
-    assert (ids2 == ids).all()
+    # the regular path sums the same fp16 products in another order, so its lists may differ from the
+    # recomputed ones where keys are nearly equal -- both must satisfy the rule, and share nearly all ids
+    ids2, dists2 = _route(sub, c, cfg.nprobe)
+    parity.check_route(sub, c, cfg.nprobe, ids2, dists2)
+    same = (np.sort(ids2, 1) == np.sort(ids, 1)).mean()
+    assert same > 0.98
 
 
 def test_config3_chunk_assignment_full_width_sampled():
