@@ -248,8 +248,8 @@ def test_config4_shape_rows_through_the_exact_recomputation():
     # recomputed ones where keys are nearly equal -- both must satisfy the rule, and share nearly all ids
     ids2, dists2 = _route(sub, c, cfg.nprobe)
     parity.check_route(sub, c, cfg.nprobe, ids2, dists2)
-    same = (np.sort(ids2, 1) == np.sort(ids, 1)).mean()
-    assert same > 0.98
+    shared = np.mean([np.intersect1d(a, b).size for a, b in zip(ids, ids2)]) / cfg.nprobe
+    assert shared > 0.98
 
 
 def test_config3_chunk_assignment_full_width_sampled():
