@@ -58,7 +58,8 @@ typedef enum {
     IVF_ERR_ALLOC = -3,          /* workspace allocation failed                                   */
     IVF_ERR_CUDA = -4,           /* a CUDA runtime/driver call failed (see ivf_last_error)        */
     IVF_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait expired; results are invalid       */
-    IVF_ERR_BAD_ID = -6          /* ivf_centroid_update met an id outside [0, nlist); row skipped */
+    IVF_ERR_BAD_ID = -6,         /* ivf_centroid_update met an id outside [0, nlist); row skipped */
+    IVF_ERR_BOUNDS = -7          /* checked build only: an index check inside a kernel failed     */
 } ivf_status;
 
 /*
@@ -218,6 +219,17 @@ int ivf_debug_rotation(int64_t n, int nlist, int d, int k, int num_sms, int64_t 
 int ivf_debug_set_rotation(int on);
 int ivf_debug_set_wait_limit_ns(int64_t ns);
 int ivf_debug_wait_probe(void* stream);
+/* Test hook: the next `count` workspace allocations are refused (the call returns IVF_ERR_ALLOC
+ * before anything is freed or launched for that allocation); 0 switches the hook off. */
+int ivf_debug_fail_next_alloc(int count);
+/* 1 if this library was built with -DIVF_CHECK_BOUNDS (every kernel checks its shared-memory,
+ * tensor-memory and global indices, records the first violation as IVF_ERR_BOUNDS with a site number
+ * in the status word and skips the access -- a stand-in for a memory checker), else 0. */
+int ivf_debug_bounds_checked(void);
+/* Launches a one-thread kernel that evaluates one failing index check (index 5 against limit 3, site
+ * 999) and touches no memory: in the checked build ivf_check then reports IVF_ERR_BOUNDS, in the
+ * regular build nothing happens. */
+int ivf_debug_bounds_probe(void* stream);
 /* Test hook: when on, the merge of a k > 1 call declares every row's candidate set insufficient, so
  * that all rows take the exact brute-force recomputation that normally only catches rare rows. */
 int ivf_debug_force_fallback(int on);

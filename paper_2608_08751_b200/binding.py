@@ -17,7 +17,7 @@ from . import build as _build
 IVF_F32, IVF_U8, IVF_I8 = 0, 1, 2
 IVF_OK = 0
 IVF_ERR_INVALID_ARG, IVF_ERR_UNSUPPORTED, IVF_ERR_ALLOC = -1, -2, -3
-IVF_ERR_CUDA, IVF_ERR_DEVICE_TIMEOUT, IVF_ERR_BAD_ID = -4, -5, -6
+IVF_ERR_CUDA, IVF_ERR_DEVICE_TIMEOUT, IVF_ERR_BAD_ID, IVF_ERR_BOUNDS = -4, -5, -6, -7
 
 EXPORTS = (
     "ivf_route", "ivf_assign", "ivf_centroid_update", "ivf_centroid_update_noalloc", "ivf_centroid_finalize",
@@ -25,7 +25,7 @@ EXPORTS = (
     "ivf_route_prepared",
     "ivf_pq_encode", "ivf_pq_search", "ivf_pq_residuals", "ivf_assign_candidates", "ivf_merge_shards",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
-    "ivf_debug_plan", "ivf_debug_span", "ivf_debug_rotation", "ivf_debug_set_rotation", "ivf_debug_set_wait_limit_ns",
+    "ivf_debug_plan", "ivf_debug_span", "ivf_debug_rotation", "ivf_debug_set_rotation", "ivf_debug_fail_next_alloc", "ivf_debug_bounds_checked", "ivf_debug_bounds_probe", "ivf_debug_set_wait_limit_ns",
     "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_set_row_chunk", "ivf_debug_stats", "ivf_debug_set_pq_groups", "ivf_debug_set_dependent_launch", "ivf_debug_set_crossing_cost",
 )
 
@@ -43,10 +43,12 @@ def lib() -> ctypes.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    path = _build.LIB_PATH
-    if not os.path.exists(path) or _build._stale():
+    # IVF_B200_CHECKED=1 selects the build whose kernels check their indices (see ivf_debug_bounds_checked)
+    checked = os.environ.get("IVF_B200_CHECKED", "0") not in ("", "0")
+    path = _build.CHECKED_LIB_PATH if checked else _build.LIB_PATH
+    if not os.path.exists(path) or _build._stale(path):
         try:
-            path = _build.build()
+            path = _build.build(checked=checked)
         except Exception as exc:  # no nvcc on this machine: use what travelled with the tree
             if not os.path.exists(path):
                 raise RuntimeError(f"libivf_b200.so is missing and could not be built: {exc}") from exc
@@ -69,6 +71,8 @@ def lib() -> ctypes.CDLL:
     L.ivf_debug_span.argtypes = [i64, i32, i32, i32, i32, i32, ctypes.POINTER(i64)]
     L.ivf_debug_rotation.argtypes = [i64, i32, i32, i32, i32, i64]
     L.ivf_debug_set_wait_limit_ns.argtypes = [i64]
+    L.ivf_debug_fail_next_alloc.argtypes = [i32]
+    L.ivf_debug_bounds_probe.argtypes = [vp]
     L.ivf_debug_timing.argtypes = [i32]
     L.ivf_debug_wait_probe.argtypes = [vp]
     L.ivf_debug_force_fallback.argtypes = [i32]
@@ -484,6 +488,21 @@ def ivf_debug_rotation(n: int, nlist: int, d: int, k: int, num_sms: int, row_gro
 
 def ivf_debug_set_rotation(on: bool) -> None:
     lib().ivf_debug_set_rotation(1 if on else 0)
+
+
+def ivf_debug_fail_next_alloc(count: int) -> None:
+    lib().ivf_debug_fail_next_alloc(int(count))
+
+
+def ivf_debug_bounds_checked() -> bool:
+    return bool(lib().ivf_debug_bounds_checked())
+
+
+def ivf_debug_bounds_probe() -> None:
+    dev = torch.device("cuda", torch.cuda.current_device())
+    rc = lib().ivf_debug_bounds_probe(_stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
 
 
 def ivf_debug_set_wait_limit_ns(ns: int) -> None:

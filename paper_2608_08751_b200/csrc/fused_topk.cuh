@@ -248,7 +248,7 @@ __device__ __noinline__ float warp_select_k(Entry* log, int c, int k, int* hist,
             keep = (u < T) || (u == T && e.y <= J);
         }
         const uint32_t bal = __ballot_sync(0xFFFFFFFFu, keep);
-        if (keep) *reinterpret_cast<uint2*>(&log[base + __popc(bal & lt_mask)]) = e;
+        if (keep && IVF_IN_BOUNDS(101, base + __popc(bal & lt_mask), c)) *reinterpret_cast<uint2*>(&log[base + __popc(bal & lt_mask)]) = e;
         base += __popc(bal);
     }
     __syncwarp();
@@ -271,6 +271,12 @@ __global__ void wait_probe_kernel(int* status, uint64_t limit_ns) {
     ctl.status = status;
     ctl.limit_ns = limit_ns;
     (void)mbar_wait(&bar, 0, ctl, 99);
+}
+
+// Evaluates one failing index check and touches no memory: shows, in the checked build, that a
+// violation reaches the status word and that the context stays usable (a no-op in the regular build).
+__global__ void bounds_probe_kernel(int index, int limit, int* sink) {
+    if (IVF_IN_BOUNDS(999, index, limit) && sink != nullptr) *sink = index;
 }
 
 __device__ __forceinline__ float min3f(float a, float b, float c) {
@@ -521,8 +527,8 @@ __device__ __forceinline__ unsigned int widen_row_u8(const uint8_t* __restrict__
                 o.z = cvt2(w[i].y, 0x5140u);
                 o.w = cvt2(w[i].y, 0x5342u);
                 const int slice = c >> 3, j = c & 7;  // chunk j of the row goes to position j ^ (row % 8)
-                *reinterpret_cast<uint4*>(tile + slice * kBlockM * kSliceRowBytes + row * kSliceRowBytes +
-                                          ((j ^ (row & 7)) << 4)) = o;
+                const int toff = slice * kBlockM * kSliceRowBytes + row * kSliceRowBytes + ((j ^ (row & 7)) << 4);
+                if (IVF_IN_BOUNDS(110, toff, a_data_bytes - 15)) *reinterpret_cast<uint4*>(tile + toff) = o;
             }
         }
     }
@@ -530,8 +536,10 @@ __device__ __forceinline__ unsigned int widen_row_u8(const uint8_t* __restrict__
     const uint32_t a16 = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(A)));
     const uint4 aug0 = valid ? make_uint4(a16 | (a16 << 16), a16, 0u, 0u) : make_uint4(0u, 0u, 0u, 0u);
     const int sw = (row >> 2) & 1;
-    *reinterpret_cast<uint4*>(tile + a_data_bytes + row * kAugRowBytes + ((0 ^ sw) << 4)) = aug0;
-    *reinterpret_cast<uint4*>(tile + a_data_bytes + row * kAugRowBytes + ((1 ^ sw) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+    if (IVF_IN_BOUNDS(111, row, kBlockM)) {
+        *reinterpret_cast<uint4*>(tile + a_data_bytes + row * kAugRowBytes + ((0 ^ sw) << 4)) = aug0;
+        *reinterpret_cast<uint4*>(tile + a_data_bytes + row * kAugRowBytes + ((1 ^ sw) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+    }
     return sumsq;
 }
 
@@ -620,6 +628,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         uint32_t ph = 0;   // divided out of `it` (the stage count is a run-time value)
         bool ok = true;
         auto load_b = [&](int t) -> bool {  // lane 0: one centroid tile into the next ring stage
+            if (!IVF_IN_BOUNDS(120, st, p.nstage) || !IVF_IN_BOUNDS(121, t, NT)) return false;
             if (!mbar_wait(&b_empty[st], ph ^ 1u, ctl, 2)) return false;
             mbar_arrive_expect_tx(&b_full[st], stage_bytes);
             uint8_t* dst = smem_b + static_cast<size_t>(st) * stage_bytes;
@@ -732,6 +741,8 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                         acc_ready = false;
                         tc_fence_after_sync();
                         const uint32_t d_tmem = tmem_base + buf * kAccStride;
+                        (void)IVF_IN_BOUNDS(130, buf * kAccStride + p.block_n, kTmemCols + 1);
+                        (void)IVF_IN_BOUNDS(131, st, p.nstage);
                         // The descriptors of consecutive K steps differ only in the start-address field
                         // (16-byte units, low word): +2 inside a 64-column slice, then on to the next
                         // slice.  Stepping the low words keeps this thread's work per MMA to a few
@@ -805,6 +816,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             const int t0 = static_cast<int>(u - r * NT);
             const int t1 = static_cast<int>((u1 - r * NT < NT) ? (u1 - r * NT) : NT);
             const int slot = (b - cta_of_unit(T, G, NT, p.cross, r * NT)) * kEpiHalves + half;
+            if (!IVF_IN_BOUNDS(140, slot, p.partials)) break;  // (checked build only: a slot outside the row's partials)
 
             if (p.x_raw != nullptr && half < MT) {
                 // uint8 points: this thread widens its own row of point tile `half`.  The tile is free:
@@ -815,7 +827,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 const unsigned int sumsq =
                     widen_row_u8(p.x_raw + static_cast<size_t>(v ? grow : 0) * p.d, v, p.d, kd, smem_a + half * a_bytes,
                                  a_data_bytes, row_in_tile, raw_scales[0], raw_scales[3]);
-                if (v) p.xn_out[grow] = static_cast<float>(sumsq);
+                if (v && IVF_IN_BOUNDS(141, grow, p.n)) p.xn_out[grow] = static_cast<float>(sumsq);
                 fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's reads
                 __syncwarp();
                 if (lane == 0) mbar_arrive(a_full);
@@ -867,8 +879,10 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
 
                     // chunk q of this warp starts at column ((q/2) * halves + half) * 64 + (q%2) * 32
                     auto col_of = [&](int q) { return ((q >> 1) * kEpiHalves + half) * 64 + (q & 1) * 32; };
+                    (void)IVF_IN_BOUNDS(142, buf * kAccStride + col_of(nq - 1) + 32, kTmemCols + 1);
                     auto after_chunk = [&]() {
                         if constexpr (kHasLog) {
+                            (void)IVF_IN_BOUNDS(145, st[h].cnt, p.cap + 1);
                             if (__any_sync(0xFFFFFFFFu, st[h].cnt > p.cap - 32)) {
                                 __syncwarp();
                                 for (int rr = 0; rr < 32; ++rr) {
@@ -953,6 +967,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                         // checked once per tile (a tile appends at most 16 records per thread).  A full
                         // log cannot be compacted here (it holds raw groups): the row is flagged and
                         // recomputed by brute force after the merge
+                        (void)IVF_IN_BOUNDS(143, st[h].wp - st[h].base, static_cast<long long>(p.cap) * kRecordBytes + 1);
                         if (st[h].wp > st[h].limit) {
                             st[h].overflow = 1;
                             st[h].wp = st[h].base;
@@ -966,6 +981,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 for (int h = 0; h < MT; ++h) {
                     if (!valid[h]) continue;
                     const size_t at = static_cast<size_t>(row[h]) * p.partials + slot;
+                    if (!IVF_IN_BOUNDS(144, at, p.n * p.partials)) continue;
                     if constexpr (EPI == EPI_ARGMIN) {
                         Entry e;
                         e.v = st[h].tau;

@@ -176,6 +176,10 @@ int get_ctx(DeviceCtx** out) {
             CUDA_TRY(cudaEventCreateWithFlags(&c.ev_free[i], cudaEventDisableTiming));
         }
         CUDA_TRY(cudaEventCreateWithFlags(&c.ev_ready, cudaEventDisableTiming));
+#ifdef IVF_CHECK_BOUNDS
+        // checked build: the kernels' index checks report into this device's status word
+        CUDA_TRY(cudaMemcpyToSymbol(g_check_status, &c.status, sizeof(int*)));
+#endif
         c.init = true;
     }
     *out = &c;
@@ -183,9 +187,16 @@ int get_ctx(DeviceCtx** out) {
 }
 
 // Grow-only, stream-ordered.
+std::atomic<int> g_fail_allocs{0};  // test hook (ivf_debug_fail_next_alloc): workspace allocations to refuse
+
 int ws_get(DeviceCtx& c, WsSlot slot, size_t bytes, cudaStream_t stream, void** out) {
     Buf& b = c.bufs[slot];
     if (bytes > b.cap) {
+        if (g_fail_allocs.load() > 0) {
+            // refused before anything is freed: the workspace stays as it was
+            g_fail_allocs.fetch_sub(1);
+            return fail(IVF_ERR_ALLOC, "workspace allocation of %zu bytes refused by the test hook", bytes);
+        }
         if (b.p) CUDA_TRY(cudaFreeAsync(b.p, stream));
         b.p = nullptr;
         b.cap = 0;
@@ -1306,6 +1317,8 @@ int ivf_check(void* stream) {
         if (h[0] == IVF_ERR_DEVICE_TIMEOUT)
             return fail(IVF_ERR_DEVICE_TIMEOUT, "a device-side wait expired (wait site %d, block %d)", h[1], h[2]);
         if (h[0] == IVF_ERR_BAD_ID) return fail(IVF_ERR_BAD_ID, "ivf_centroid_update skipped ids outside [0, nlist)");
+        if (h[0] == IVF_ERR_BOUNDS)
+            return fail(IVF_ERR_BOUNDS, "an index check of the checked build failed (site %d, block %d, index %d)", h[1], h[2], h[3]);
         return fail(h[0], "device status %d", h[0]);
     }
     return IVF_OK;
@@ -1451,6 +1464,22 @@ int ivf_debug_set_pq_groups(int groups) {
     g_pq_kernel = groups < 0 ? 1 : 0;  // a negative count also selects the single-team kernel
     if (groups < 0) groups = -groups - 1;
     g_pq_groups = groups < 0 ? 0 : groups;
+    return IVF_OK;
+}
+
+int ivf_debug_fail_next_alloc(int count) {
+    g_fail_allocs.store(count > 0 ? count : 0);
+    return IVF_OK;
+}
+
+int ivf_debug_bounds_checked(void) { return kBoundsChecked ? 1 : 0; }
+
+int ivf_debug_bounds_probe(void* stream) {
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != IVF_OK) return rc;
+    bounds_probe_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(5, 3, nullptr);  // 5 is not below 3
+    LAUNCH_CHECK();
     return IVF_OK;
 }
 

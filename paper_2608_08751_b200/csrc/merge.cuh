@@ -50,7 +50,8 @@ __global__ void merge_argmin_kernel(const MergeParams p) {
     pdl_trigger();
     const int64_t row = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (row >= p.n) return;
-    const int ns = slots_of_row_tile(p, row / p.group_rows);
+    int ns = slots_of_row_tile(p, row / p.group_rows);
+    if (!IVF_IN_BOUNDS(201, ns, p.partials + 1)) ns = p.partials;
     const Entry* e = p.part + static_cast<size_t>(row) * p.partials;
     float bv = e[0].v;
     int bj = e[0].j;
@@ -97,6 +98,7 @@ __device__ __forceinline__ void merge_write_row(const MergeParams& p, int64_t ro
     const float inv = p.scal[2];
     for (int i = i0; i < p.k; i += istep) {
         const uint64_t key = keys[i];
+        if (!IVF_IN_BOUNDS(202, row * p.k + i, p.n * p.k)) continue;
         p.out_ids[row * p.k + i] = static_cast<int32_t>(key & 0xFFFFFFFFull);
         if (p.out_dists)
             p.out_dists[row * p.k + i] = fmaxf(fmaf(from_orderable(static_cast<uint32_t>(key >> 32)), inv, xn), 0.0f);
@@ -104,7 +106,7 @@ __device__ __forceinline__ void merge_write_row(const MergeParams& p, int64_t ro
 }
 __device__ __forceinline__ void merge_fail_row(const MergeParams& p, int64_t row) {
     const int at = atomicAdd(&p.fail[0], 1);
-    p.fail[1 + at] = static_cast<int>(row);
+    if (IVF_IN_BOUNDS(203, at, p.n)) p.fail[1 + at] = static_cast<int>(row);
     if (p.stats) atomicAdd(&p.stats[2], 1ull);
 }
 
@@ -196,7 +198,9 @@ __device__ __forceinline__ void merge_select_row(const MergeParams& p, int64_t r
                         const int mid = (lo + hi) >> 1;
                         if (pre[mid] <= idx) lo = mid; else hi = mid;
                     }
-                    if (p.records) {
+                    if (!IVF_IN_BOUNDS(210, lo, p.partials) || !IVF_IN_BOUNDS(211, idx - pre[lo], p.cap)) {
+                        nv = 0;
+                    } else if (p.records) {
                         const char* rec = reinterpret_cast<const char*>(p.part) +
                                           ((static_cast<size_t>(row) * p.partials + lo) * p.cap + (idx - pre[lo])) *
                                               kRecordBytes;
@@ -374,7 +378,7 @@ __global__ void __launch_bounds__(32 * WARPS) merge_warp_kernel(const MergeParam
                 const int t = __shfl_up_sync(FULL, v, off);
                 if (lane >= off) v += t;
             }
-            if (sidx < ns) sm.pre[sidx + 1] = v + carry;
+            if (sidx < ns && IVF_IN_BOUNDS(220, sidx + 1, kWarpSlots + 1)) sm.pre[sidx + 1] = v + carry;
             carry += __shfl_sync(FULL, v, 31);
         }
         if (lane == 0) sm.pre[0] = 0;
@@ -441,6 +445,7 @@ __global__ void __launch_bounds__(32 * WARPS) merge_warp_kernel(const MergeParam
                 if (sm.pre[mid] <= idx) lo = mid; else hi = mid;
             }
             const size_t at = (static_cast<size_t>(row) * p.partials + lo) * p.cap + (idx - sm.pre[lo]);
+            if (!IVF_IN_BOUNDS(221, lo, p.partials) || !IVF_IN_BOUNDS(222, idx - sm.pre[lo], p.cap)) return;
             if (p.records) {
                 const char* rec = reinterpret_cast<const char*>(p.part) + at * kRecordBytes;
                 na = *reinterpret_cast<const float4*>(rec);
@@ -502,7 +507,7 @@ __global__ void __launch_bounds__(32 * WARPS) merge_warp_kernel(const MergeParam
     if (pass_on) {
         if (lane == 0) {
             const int at = atomicAdd(&p.big[0], 1);
-            p.big[1 + at] = static_cast<int>(row);
+            if (IVF_IN_BOUNDS(223, at, p.n)) p.big[1 + at] = static_cast<int>(row);
         }
         return;
     }
@@ -556,7 +561,8 @@ __global__ void __launch_bounds__(kTauThreads) merge_tau_kernel(const MergeParam
         float v[kSampleM];
         const int slot = s0 + threadIdx.x;
 #pragma unroll
-        for (int i = 0; i < kSampleM; ++i) v[i] = slot < ns ? base[static_cast<size_t>(slot) * p.cap + i].v : INF;
+        for (int i = 0; i < kSampleM; ++i)
+            v[i] = (slot < ns && IVF_IN_BOUNDS(240, slot, p.partials)) ? base[static_cast<size_t>(slot) * p.cap + i].v : INF;
         float last;
         take16(v, lane, lists[warp], last);
         __syncthreads();
@@ -585,7 +591,8 @@ __global__ void __launch_bounds__(256) merge_tau_warp_kernel(const MergeParams p
     const Entry* base = p.part + static_cast<size_t>(row) * p.partials * p.cap;
     float v[kSampleM];
 #pragma unroll
-    for (int i = 0; i < kSampleM; ++i) v[i] = lane < ns ? base[static_cast<size_t>(lane) * p.cap + i].v : INF;
+    for (int i = 0; i < kSampleM; ++i)
+        v[i] = (lane < ns && IVF_IN_BOUNDS(241, lane, p.partials)) ? base[static_cast<size_t>(lane) * p.cap + i].v : INF;
     float result;
     take16(v, lane, nullptr, result);
     if (lane == 0) p.tau_out[row] = result;
@@ -675,7 +682,7 @@ __device__ __forceinline__ void fallback_slice_keys(const FallbackParams& p, con
         for (int u = 0; u < kInFlight; ++u) {
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) acc[u] += __shfl_xor_sync(0xFFFFFFFFu, acc[u], off);
-            if (lane == 0 && jb + u < j1) keys[jb + u - j0] = acc[u];
+            if (lane == 0 && jb + u < j1 && IVF_IN_BOUNDS(250, jb + u - j0, kFallbackSlice)) keys[jb + u - j0] = acc[u];
         }
     }
 }
@@ -740,7 +747,10 @@ __device__ __forceinline__ void fallback_slice(const FallbackParams& p, int slic
     const uint64_t bound = fallback_select_bound(get, len, p.k, sm);
     for (int i = threadIdx.x; i < len; i += blockDim.x) {
         const uint64_t v = get(i);
-        if (v <= bound) out[atomicAdd(&sm.cnt, 1)] = v;
+        if (v <= bound) {
+            const int at = atomicAdd(&sm.cnt, 1);
+            if (IVF_IN_BOUNDS(251, at, p.k)) out[at] = v;
+        }
     }
     __syncthreads();
 }
@@ -774,6 +784,7 @@ __device__ __forceinline__ void fallback_finish_row(const FallbackParams& p, con
     const float inv = p.scal[2];
     for (int i = threadIdx.x; i < p.k; i += blockDim.x) {
         const uint64_t key = sm.top[i];
+        if (!IVF_IN_BOUNDS(252, i, got)) continue;
         p.out_ids[row * p.k + i] = static_cast<int32_t>(key & 0xFFFFFFFFull);
         if (p.out_dists)
             p.out_dists[row * p.k + i] = fmaxf(fmaf(from_orderable(static_cast<uint32_t>(key >> 32)), inv, xn), 0.0f);
@@ -881,6 +892,7 @@ __global__ void __launch_bounds__(kMergeThreads) route_tail_kernel(const TailPar
             loaded = idx;
             __syncthreads();
         }
+        if (!IVF_IN_BOUNDS(260, idx, kFallbackFastRows) || !IVF_IN_BOUNDS(261, row, p.n)) break;
         fallback_slice(f, slice, f.cand + (static_cast<size_t>(idx) * f.slices + slice) * f.k, sm);
         __threadfence();
         __syncthreads();

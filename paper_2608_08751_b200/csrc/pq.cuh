@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(kPqThreads, 1) pq_encode_kernel(const PqEncode
                     bj = oj;
                 }
             }
-            if (lane == 0) p.codes[i * p.pq_m + m] = static_cast<uint8_t>(bj);
+            if (lane == 0 && IVF_IN_BOUNDS(430, bj, kPqK)) p.codes[i * p.pq_m + m] = static_cast<uint8_t>(bj);
         }
     }
 }
@@ -416,7 +416,10 @@ __device__ __forceinline__ uint64_t pq_cut_buffer(uint64_t* buf, int count, int 
     pq_group_sync<BAR, NT>();
 #pragma unroll
     for (int q = 0; q < kPer; ++q)
-        if (mine[q] <= bound && mine[q] != ~0ull) buf[atomicAdd(&misc[0], 1)] = mine[q];
+        if (mine[q] <= bound && mine[q] != ~0ull) {
+            const int at = atomicAdd(&misc[0], 1);
+            if (IVF_IN_BOUNDS(401, at, CAP)) buf[at] = mine[q];
+        }
     pq_group_sync<BAR, NT>();
     return bound;
 }
@@ -574,6 +577,7 @@ __device__ __forceinline__ void pq_scan_groups(const PqScanParams& p, const PqTe
         pq_group_sync<BAR, NT>();  // the previous group's descriptors, table and buffer are no longer in use
         // the query's probe descriptors, once per group: chunk prefix, list begin, list length
         for (int pr = tid; pr <= p.nprobe; pr += NT) {
+            if (!IVF_IN_BOUNDS(410, pr, kPqMaxProbes + 1)) continue;
             s.cs[pr] = cs_g[pr];
             if (pr < p.nprobe) {
                 const int l = p.probes[static_cast<size_t>(b) * p.nprobe + pr];
@@ -658,7 +662,7 @@ __device__ __forceinline__ void pq_scan_groups(const PqScanParams& p, const PqTe
                     int base = 0;
                     if (lane == 0) base = atomicAdd(&s.misc[0], __popc(bal));
                     base = __shfl_sync(0xFFFFFFFFu, base, 0);
-                    if (hit) s.buf[base + __popc(bal & lt_mask)] = key;
+                    if (hit && IVF_IN_BOUNDS(411, base + __popc(bal & lt_mask), kPqScanBufKeys)) s.buf[base + __popc(bal & lt_mask)] = key;
                 }
                 pq_group_sync<BAR, NT>();
                 const int count = s.misc[0];
@@ -673,7 +677,8 @@ __device__ __forceinline__ void pq_scan_groups(const PqScanParams& p, const PqTe
             count = p.n_rerank;
         }
         uint64_t* out = p.gcand + static_cast<size_t>(g) * p.n_rerank;
-        for (int i = tid; i < count; i += NT) out[i] = s.buf[i];
+        for (int i = tid; i < count; i += NT)
+            if (IVF_IN_BOUNDS(412, i, p.n_rerank)) out[i] = s.buf[i];
         if (tid == 0) p.gcand_count[g] = count;
     }
 }
@@ -772,7 +777,10 @@ __global__ void __launch_bounds__(kPqThreads, kRegs ? 1 : 2) pq_merge_kernel(con
         }
 #pragma unroll
         for (int q = 0; q < kRegKeys; ++q)
-            if (mine[q] != ~0ull && mine[q] <= bound) buf[atomicAdd(&misc[0], 1)] = mine[q];
+            if (mine[q] != ~0ull && mine[q] <= bound) {
+                const int at = atomicAdd(&misc[0], 1);
+                if (IVF_IN_BOUNDS(420, at, kPqBufKeys)) buf[at] = mine[q];
+            }
     } else {
         uint64_t bound = ~0ull;
         if (total > kPqBufKeys) {
@@ -782,7 +790,10 @@ __global__ void __launch_bounds__(kPqThreads, kRegs ? 1 : 2) pq_merge_kernel(con
         }
         for (int i = threadIdx.x; i < slots; i += blockDim.x) {
             const uint64_t v = get(i);
-            if (v != ~0ull && v <= bound) buf[atomicAdd(&misc[0], 1)] = v;
+            if (v != ~0ull && v <= bound) {
+                const int at = atomicAdd(&misc[0], 1);
+                if (IVF_IN_BOUNDS(421, at, kPqBufKeys)) buf[at] = v;
+            }
         }
     }
     __syncthreads();
@@ -818,6 +829,7 @@ __global__ void __launch_bounds__(kPqThreads, kRegs ? 1 : 2) pq_merge_kernel(con
         if (i < count) {
             const uint64_t key = buf[i];
             pos = static_cast<long long>(key & 0xFFFFFFFFull);
+            (void)IVF_IN_BOUNDS(422, i, kPqBufKeys);
             if (p.vec_ids) pos = p.vec_ids[pos];
             est = from_orderable(static_cast<uint32_t>(key >> 32));
         }

@@ -10,6 +10,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "check.cuh"
+
 namespace ivf {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

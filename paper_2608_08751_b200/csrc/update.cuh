@@ -111,7 +111,7 @@ __global__ void update_fill_kernel(const int32_t* __restrict__ ids, int64_t n, i
     const int l = ids[i];
     if (l < 0 || l >= nlist) return;
     const int pos = off[l] + atomicAdd(&cursor[l], 1);
-    perm[pos] = static_cast<int>(i);
+    if (IVF_IN_BOUNDS(301, pos, n)) perm[pos] = static_cast<int>(i);
 }
 
 // Sum of the member rows perm[beg .. end) for one warp: lane q owns columns [128*blk + 4*q, +4) for
@@ -182,6 +182,7 @@ __global__ void update_reduce_kernel(const T* __restrict__ x, const int* __restr
     if (l >= nlist) return;
     const int beg = off[l], end = off[l + 1];
     if (beg == end) return;
+    if (!IVF_IN_BOUNDS(302, end - beg, off[nlist] + 1) || !IVF_IN_BOUNDS(303, end, off[nlist] + 1)) return;
     float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
     reduce_members(x, perm, beg, end, d, lane, acc);
 #pragma unroll
