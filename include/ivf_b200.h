@@ -33,7 +33,13 @@
  *              Float inputs are scaled by an exact power of two (exponent clamped to +-40) before they are
  *              rounded to fp16: finite values with magnitude between about 1e-12 and 1e12 keep the stated
  *              tolerance (tested); beyond 2^51 the operands overflow and the results are undefined,
- *              as they are for non-finite inputs (always memory-safe).
+ *              as they are for non-finite inputs (always memory-safe).  The scale is one power of
+ *              two per matrix, taken from its largest magnitude M: inside one matrix the tolerance
+ *              1e-3 (|x|^2 + |c|^2) holds for every pair whose combined norm sqrt(|x|^2 + |c|^2) is at
+ *              least about 2^-9 M_centroids (tested down to 2^-7); for a pair of rows both far
+ *              smaller than that, next to much larger rows in the same matrices, the norm term
+ *              falls below fp16's smallest step and the error bound becomes the absolute
+ *              2^-30 M_centroids^2 instead.
  *              nlist < 2^31.  n == 0 is IVF_OK and enqueues nothing.
  *   Non-finite inputs give unspecified (but memory-safe) results.
  *
@@ -109,7 +115,10 @@ int ivf_assign(const void* points, int64_t n, int d, ivf_dtype ptype,
  * ACCUMULATES into sums/counts so that chunks of one iteration compose; the caller zeroes them
  * at the start of an iteration.  points [n, d] (ptype) and ids [n] int32 are device pointers.
  * A row whose id is outside [0, nlist) is skipped and flags IVF_ERR_BAD_ID in the status word.
- * For uint8 points the sums are exact while every list sum stays below 2^24.
+ * For uint8 and int8 points the sums are exact while every list sum stays below 2^24, hence
+ * bit-identical from run to run, like the counts.  Float points are added in an order that depends
+ * on scheduling: their sums are reproducible only up to the rounding of a different summation order
+ * (within 1e-5 of the sum of the members' magnitudes).
  */
 int ivf_centroid_update(const void* points, ivf_dtype ptype, const int32_t* ids, int64_t n, int d,
                         int nlist, float* sums, int64_t* counts, void* stream);

@@ -203,8 +203,11 @@ __global__ void update_reduce_kernel(const T* __restrict__ x, const int* __restr
 
 // Few long lists (k-means with a handful of clusters, PQ codebook training with 256): every list is
 // cut into `parts` equal pieces, one warp per piece writes its partial sum to scratch[l][part][d],
-// and update_combine_parts_kernel adds a list's partial sums in piece order (so the result does not
-// depend on scheduling).
+// and update_combine_parts_kernel adds a list's partial sums in piece order.
+// Reproducibility: the fill places a list's members with an atomic cursor, so their order inside the
+// list depends on scheduling.  Byte-typed rows are summed exactly (integers below 2^24), so their sums
+// and all counts are bit-identical from run to run; float sums are reproducible only within the
+// rounding of a different summation order (inside the 1e-5 bound the tests use).
 template <typename T>
 __global__ void update_reduce_parts_kernel(const T* __restrict__ x, const int* __restrict__ perm,
                                            const int* __restrict__ off, int nlist, int d, int parts,

@@ -157,6 +157,24 @@ def test_route_mixed_magnitudes_between_points_and_centroids():
         parity.check_route(x, c, 12, ids.cpu().numpy(), dists.cpu().numpy())
 
 
+@pytest.mark.parametrize("k", [1, 24])
+def test_route_mixed_magnitudes_inside_one_table(k):
+    # the operand scale is one power of two per matrix, so rows far below the matrix's largest
+    # magnitude lose bits: the header promises the tolerance for pairs whose combined norm is at
+    # least about 2^-9 of the largest centroid magnitude.  Here a tenth of the centroids and of the
+    # points are 2^-4, 2^-6 or 2^-7 of the rest (small-small pairs sit at about 2^-5 of the maximum).
+    rng = np.random.default_rng(91 + k)
+    x = rng.standard_normal((400, 64)).astype(np.float32)
+    c = rng.standard_normal((3000, 64)).astype(np.float32)
+    for arr in (x, c):
+        small = rng.choice(arr.shape[0], arr.shape[0] // 10, replace=False)
+        arr[small] *= rng.choice([2.0 ** -4, 2.0 ** -6, 2.0 ** -7], small.size)[:, None].astype(np.float32)
+    c[:40] = x[:40] * (1 + 1e-3)  # near neighbours, also among the small rows
+    ids, dists = (B.ivf_assign if k == 1 else lambda a, b: B.ivf_route(a, b, k))(_t(x), _t(c))
+    B.ivf_check()
+    parity.check_route(x, c, k, ids.cpu().numpy(), dists.cpu().numpy())
+
+
 @pytest.mark.parametrize("dtype,n,nlist,d,k", [
     ("u8", 2500, 4096, 32, 1), ("i8", 5000, 9000, 64, 1), ("u8", 1000, 40000, 16, 1),
     ("u8", 700, 4096, 128, 64), ("i8", 300, 1000, 100, 20),

@@ -298,6 +298,32 @@ def test_update_flags_and_skips_bad_ids():
     B.ivf_check()  # the status word was cleared
 
 
+def test_update_run_to_run_reproducibility():
+    # byte rows: sums and counts bit-identical over three runs; float rows: counts identical, sums
+    # within the rounding of a different summation order
+    rng = np.random.default_rng(12)
+    n, nlist, d = 60000, 900, 64
+    ids = _cuda(rng.integers(0, nlist, n).astype(np.int32))
+    for dtype in ("u8", "f32"):
+        x = rng.integers(0, 256, (n, d)).astype(np.uint8) if dtype == "u8" else rng.standard_normal((n, d)).astype(np.float32)
+        xt = _cuda(x)
+        runs = []
+        for _ in range(3):
+            sums = torch.zeros((nlist, d), dtype=torch.float32, device="cuda")
+            counts = torch.zeros((nlist,), dtype=torch.int64, device="cuda")
+            B.ivf_centroid_update(xt, ids, sums, counts)
+            B.ivf_check()
+            runs.append((sums.cpu().numpy(), counts.cpu().numpy()))
+        for s, c in runs[1:]:
+            assert (c == runs[0][1]).all()
+            if dtype == "u8":
+                assert (s == runs[0][0]).all()
+            else:
+                mag = np.zeros((nlist, d))
+                np.add.at(mag, ids.cpu().numpy(), np.abs(x.astype(np.float64)))
+                assert (np.abs(s.astype(np.float64) - runs[0][0]) <= 1e-5 * mag + 1e-30).all()
+
+
 def test_finalize_matches_oracle_and_keeps_empty_lists():
     rng = np.random.default_rng(1)
     sums = rng.standard_normal((50, 32)).astype(np.float32) * 100
