@@ -660,14 +660,17 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         // (both list counters were cleared by the fused kernel that just ran)
         mp.big = failbuf + n + 2;
         // three sizes of the warp-level kernel (the smaller the key buffer, the more warps per SM): up to
-        // 512 candidates in the buffer / 256 sorted (k <= 68 under the given rule), 1024 / 512 (k <= 280;
+        // 512 candidates in the buffer / 256 sorted (k <= 68 under the given rule; six CTAs of six warps
+        // per SM at 56 registers: a row is one serial chain of about 26 us, so the kernel's time is
+        // that chain times the number of rounds the rows need -- 10,000 rows: 3 rounds with 32 warps
+        // per SM, 2 with 36: 0.084 -> 0.073 ms), 1024 / 512 (k <= 280;
         // a row with more candidates than fit is cut down to its k smallest in mid-gather, which for
         // k = 256 costs less than the lower occupancy of the next size: C4 chunk 0.52 -> 0.40 ms),
         // 2048 / 1024 (k <= 340); beyond that everything goes to the general path of the tail kernel
         const int expect = given ? 5 * k : 2 * k;
         if (!ctx.merge_attr_set) {
-            CUDA_TRY(cudaFuncSetAttribute(merge_warp_kernel<512, 256, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          static_cast<int>(8 * sizeof(MergeWarpSmem<512>))));
+            CUDA_TRY(cudaFuncSetAttribute(merge_warp_kernel<512, 256, 6>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(6 * sizeof(MergeWarpSmem<512>))));
             CUDA_TRY(cudaFuncSetAttribute(merge_warp_kernel<1024, 512, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(8 * sizeof(MergeWarpSmem<1024>))));
             CUDA_TRY(cudaFuncSetAttribute(merge_warp_kernel<2048, 1024, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -679,7 +682,7 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
             // more partial logs than the warp-level kernel takes -- all rows go to the tail kernel)
             mp.big = nullptr;
         } else if (expect <= 340) {
-            LAUNCH_DEP(8, (merge_warp_kernel<512, 256, 8>), static_cast<unsigned>((n + 7) / 8), 256, 8 * sizeof(MergeWarpSmem<512>), stream, mp);
+            LAUNCH_DEP(8, (merge_warp_kernel<512, 256, 6>), static_cast<unsigned>((n + 5) / 6), 192, 6 * sizeof(MergeWarpSmem<512>), stream, mp);
         } else if (expect <= 1400) {
             LAUNCH_DEP(8, (merge_warp_kernel<1024, 512, 8>), static_cast<unsigned>((n + 7) / 8), 256, 8 * sizeof(MergeWarpSmem<1024>), stream, mp);
         } else if (expect <= 1700) {
