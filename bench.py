@@ -44,10 +44,10 @@ UNIT = "queries/s"
 # 1,048,576-row launch (an upper bound: the centroid copy does not grow with the rows).
 TRAFFIC_FUSED_ARGMIN_BYTES = 4 * (52.519424e6 + 1.968896e6)
 # k = 64 kernel at the C1 size, k = 128 kernel at the C2 size, k = 256 kernel on one 9,984-row chunk of C4
-# (each captured at that size; None until a capture of the current kernel exists).
-TRAFFIC_FUSED_TOPK_BYTES = 93.999360e6 + 104.450560e6
-TRAFFIC_FUSED_C2_BYTES = None
-TRAFFIC_FUSED_C4_CHUNK_BYTES = None
+# (each captured at that size).
+TRAFFIC_FUSED_TOPK_BYTES = 98.110208e6 + 109.510912e6
+TRAFFIC_FUSED_C2_BYTES = 257.216256e6 + 246.785280e6
+TRAFFIC_FUSED_C4_CHUNK_BYTES = 669.312768e6 + 503.178752e6   # per launch: one 9,728-row chunk of the 11 a C4 call makes
 # roofline rates of whole routing calls: the slower of 2 n nlist d FLOP at the measured burst peak and
 # the minimum bytes at the measured HBM rate (tensor-bound for every configuration here)
 ROOFLINE_QPS = {"C1": 9.78e7, "C2": 3.26e7, "C4": 8.15e6}
