@@ -343,7 +343,7 @@ __device__ __forceinline__ void warp_bitonic_sort(uint64_t* keys, int m, int lan
 }
 
 template <int KEYS, int SORT, int WARPS>
-__global__ void __launch_bounds__(32 * WARPS, KEYS <= 512 ? 6 : 1) merge_warp_kernel(const MergeParams p) {
+__global__ void __launch_bounds__(32 * WARPS, KEYS <= 512 ? 6 : (KEYS <= 1024 ? 3 : 2)) merge_warp_kernel(const MergeParams p) {
     pdl_wait();
     pdl_trigger();
     extern __shared__ __align__(16) uint8_t merge_smem_raw[];
