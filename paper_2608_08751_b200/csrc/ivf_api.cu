@@ -408,7 +408,8 @@ int convert_centroids(DeviceCtx& ctx, const float* centroids, int nlist, int d, 
     LAUNCH_DEP(1, maxabs_kernel, blocks, 256, 0, stream, centroids, count, cp->bits + 1);
     // the conversion derives the centroid scale from the magnitude word itself and publishes the scale
     // vector (with the byte-type point scale as a placeholder until the points are known)
-    const int64_t threads = static_cast<int64_t>(nlist) * 32;
+    const int rows_per_warp = pl.kd <= 64 ? 4 : (pl.kd <= 128 ? 2 : 1);  // the kernel's lane groups
+    const int64_t threads = (static_cast<int64_t>(nlist) + rows_per_warp - 1) / rows_per_warp * 32;
     LAUNCH_DEP(1, (convert_rows_kernel<float, true>), static_cast<unsigned>((threads + 255) / 256), 256, 0, stream,
                centroids, nlist, d, pl.kd, cp->scal, cp->c16, nullptr, cp->bits, 1);
     timing_end(tk, stream);
@@ -592,7 +593,8 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         // magnitude (float points only: byte types have a fixed bound), scales and the fp16 operand
         // copy with |x|^2
         tk = timing_begin(TK_PREP, stream);
-        const int64_t threads = n * 32;
+        const int rows_per_warp = pl.kd <= 64 ? 4 : (pl.kd <= 128 ? 2 : 1);
+        const int64_t threads = (n + rows_per_warp - 1) / rows_per_warp * 32;
         const unsigned cblocks = static_cast<unsigned>((threads + 255) / 256);
         if (ptype == IVF_F32) {
             CUDA_TRY(cudaMemsetAsync(cp.bits, 0, sizeof(unsigned int), stream));

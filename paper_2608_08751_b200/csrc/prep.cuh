@@ -25,8 +25,24 @@ __global__ void maxabs_kernel(const float* __restrict__ x, int64_t count, unsign
     pdl_trigger();
     float m = 0.0f;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
-    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < count; i += stride)
-        m = fmaxf(m, fabsf(x[i]));
+    const int64_t tid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    // 16-byte loads, four in flight per thread (the rows are 16-byte aligned and d is a multiple of 4,
+    // so the element count is a multiple of 4)
+    const float4* x4 = reinterpret_cast<const float4*>(x);
+    const int64_t count4 = count >> 2;
+    int64_t i = tid;
+    for (; i + 3 * stride < count4; i += 4 * stride) {
+        const float4 a = x4[i], b = x4[i + stride], c = x4[i + 2 * stride], e = x4[i + 3 * stride];
+        m = fmaxf(m, fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))));
+        m = fmaxf(m, fmaxf(fmaxf(fabsf(b.x), fabsf(b.y)), fmaxf(fabsf(b.z), fabsf(b.w))));
+        m = fmaxf(m, fmaxf(fmaxf(fabsf(c.x), fabsf(c.y)), fmaxf(fabsf(c.z), fabsf(c.w))));
+        m = fmaxf(m, fmaxf(fmaxf(fabsf(e.x), fabsf(e.y)), fmaxf(fabsf(e.z), fabsf(e.w))));
+    }
+    for (; i < count4; i += stride) {
+        const float4 a = x4[i];
+        m = fmaxf(m, fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))));
+    }
+    for (int64_t j = (count4 << 2) + tid; j < count; j += stride) m = fmaxf(m, fabsf(x[j]));
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
     __shared__ float wmax[32];
@@ -40,8 +56,9 @@ __global__ void maxabs_kernel(const float* __restrict__ x, int64_t count, unsign
     }
 }
 
-// One warp per row.  Lane g converts columns [8g, 8g+8) of the data part; after the norm is reduced
-// lanes 0 and 1 write the 16 extra columns.  If `bits` is given (point rows), the scales are derived
+// One lane group per row: 8 lanes for kd = 64 (four rows per warp), 16 for kd = 128 (two rows per warp),
+// the whole warp beyond.  Lane g of a group converts columns [8g, 8g+8) of the data part; after the norm
+// is reduced inside the group its lanes 0 and 1 write the 16 extra columns.  (rows_per_warp = 32 / group)  If `bits` is given (point rows), the scales are derived
 // here from the magnitude words instead of being read, and the first thread publishes them in `scal`
 // for the kernels that follow.
 template <typename T, bool CENTROID>
@@ -50,9 +67,11 @@ __global__ void convert_rows_kernel(const T* __restrict__ x, int64_t rows, int d
                                     const unsigned int* __restrict__ bits, int points_are_u8) {
     pdl_wait();
     pdl_trigger();
-    const int lane = threadIdx.x & 31;
-    const int64_t row = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
-    if (row >= rows) return;
+    const int group = kd <= 64 ? 8 : (kd <= 128 ? 16 : 32);
+    const int lane = threadIdx.x & (group - 1);
+    const int64_t warp = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    const int64_t row = warp * (32 / group) + ((threadIdx.x & 31) / group);
+    if (row >= rows) return;  // (a whole lane group leaves together: the shuffles below stay inside a group)
     const int kp = kd + 16;
     float sv[4];
     if (bits != nullptr) {
@@ -104,8 +123,11 @@ __global__ void convert_rows_kernel(const T* __restrict__ x, int64_t rows, int d
         }
         *reinterpret_cast<uint4*>(out + row * kp + c0) = *reinterpret_cast<const uint4*>(h);
     }
+    // (the mask names the lanes of this group only: groups whose row is past the end have returned)
+    const uint32_t gmask = group == 32 ? 0xFFFFFFFFu : (((1u << group) - 1u) << ((threadIdx.x & 31) / group * group));
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+    for (int off = 16; off > 0; off >>= 1)
+        if (off < group) acc += __shfl_xor_sync(gmask, acc, off);
     if (lane < 2) {
         __half a[8];
 #pragma unroll
