@@ -322,8 +322,8 @@ int ivf_merge_shards(const int32_t* shard_ids, const float* shard_dists, int par
  *     acc = fma(diff, diff, acc);   estimate: acc = 0, for m ascending: acc = acc + LUT_m[a_m].
  *
  * codebooks  [pq_m][256][d / pq_m] float32, row-major.  pq_m must divide d.  Encoding keeps the
- *            codebook in shared memory: 1024 * (d + pq_m) + 4 * d bytes must fit one SM's
- *            227 KB (d = 128 with pq_m = 32 does; d = 256 does not); searching needs
+ *            codebook in shared memory: 1024 * (d + pq_m) + 4 * d bytes (and 1024 * d + 8,704)
+ *            must fit one SM's 227 KB (d = 128 with pq_m = 32 does; d = 256 does not); searching needs
  *            1024 * pq_m + 21,584 bytes and d <= 256 -> IVF_ERR_UNSUPPORTED otherwise.
  *
  * ivf_pq_encode: out_codes[i][m] = arg-min over j of the table of x_i - centroids[ids[i]]

@@ -1131,7 +1131,8 @@ int pq_check_shape(int d, int pq_m, const float* codebooks, bool encode) {
     if (d < 1 || pq_m < 1 || d % pq_m != 0)
         return fail(IVF_ERR_INVALID_ARG, "d = %d, pq_m = %d: pq_m must divide d", d, pq_m);
     if (!codebooks) return fail(IVF_ERR_INVALID_ARG, "null pointer argument");
-    const size_t need = encode ? pq_smem_bytes(d, pq_m) : pq_scan_smem_bytes(d, pq_m);
+    size_t need = encode ? pq_smem_bytes(d, pq_m) : pq_scan_smem_bytes(d, pq_m);
+    if (encode && pq_encode_smem_bytes(d) > need) need = pq_encode_smem_bytes(d);
     if (need > kSmemLimit || d > 256)
         return fail(IVF_ERR_UNSUPPORTED, "d = %d, pq_m = %d: %zu bytes of shared memory needed (limit %zu), d at most 256", d,
                     pq_m, need, static_cast<size_t>(kSmemLimit));
@@ -1200,7 +1201,7 @@ int ivf_pq_encode(const void* points, int64_t n, int d, ivf_dtype ptype, const i
     p.status = ctx.status;
     const int tk = timing_begin(TK_PQ_ENCODE, stream);
     const unsigned grid = static_cast<unsigned>(n < ctx.num_sms ? n : ctx.num_sms);
-    pq_encode_kernel<<<grid, kPqThreads, pq_smem_bytes(d, pq_m), stream>>>(p);
+    pq_encode_kernel<<<grid, kPqThreads, pq_encode_smem_bytes(d), stream>>>(p);
     LAUNCH_CHECK();
     timing_end(tk, stream);
     return IVF_OK;

@@ -171,51 +171,185 @@ struct PqEncodeParams {
     int* status;
 };
 
+// Shared memory of the encode kernel: the codebook in its own layout [m][j][dsub] and two buffers of
+// kPqEncodeElems residual coordinates (a batch of vectors each).
+constexpr int kPqEncodeElems = kPqThreads;  // coordinates per batch = one per thread
+__host__ __device__ inline size_t pq_encode_smem_bytes(int d) {
+    return static_cast<size_t>(d) * kPqK * 4 + 2 * static_cast<size_t>(kPqEncodeElems) * 4 + 2 * 64 * 4;
+}
+
+// Codes of one (vector, subspace) pair by one warp: lane q takes codewords lane, lane + 32, ... (8 of
+// them), each table entry is the same chain of rounded operations as in the lookup-table build
+// (diff = r_t - p_t, acc = fma(diff, diff, acc), t ascending), the smallest entry wins, ties to the
+// lower codeword.  No table is written anywhere: the entries live in registers.  REGS: the lane's 8
+// codewords are already in registers (cwr), otherwise they are read from the shared-memory codebook.
+template <int DSUB, bool REGS>
+__device__ __forceinline__ int pq_encode_subspace(const float* __restrict__ rm, const float* __restrict__ cbm, int dsub,
+                                                  int lane, const float (&cwr)[kPqK / 32][DSUB > 0 ? DSUB : 1]) {
+    const int ds = DSUB > 0 ? DSUB : dsub;
+    float rv[DSUB > 0 ? DSUB : 1];
+    if constexpr (DSUB > 0) {
+        if constexpr ((DSUB & 3) == 0) {
+#pragma unroll
+            for (int t4 = 0; t4 < DSUB / 4; ++t4) {
+                const float4 v = reinterpret_cast<const float4*>(rm)[t4];
+                rv[4 * t4] = v.x; rv[4 * t4 + 1] = v.y; rv[4 * t4 + 2] = v.z; rv[4 * t4 + 3] = v.w;
+            }
+        } else {
+#pragma unroll
+            for (int t = 0; t < DSUB; ++t) rv[t] = rm[t];
+        }
+    }
+    float best = __int_as_float(0x7f800000);
+    int bj = 0x7fffffff;
+#pragma unroll
+    for (int q = 0; q < kPqK / 32; ++q) {
+        const int j = lane + 32 * q;
+        float acc = 0.0f;
+        if constexpr (REGS) {
+#pragma unroll
+            for (int t = 0; t < DSUB; ++t) {
+                const float diff = __fsub_rn(rv[t], cwr[q][t]);
+                acc = __fmaf_rn(diff, diff, acc);
+            }
+        } else {
+            const float* cw = cbm + j * ds;
+            if constexpr (DSUB > 0 && (DSUB & 3) == 0) {
+#pragma unroll
+                for (int t4 = 0; t4 < DSUB / 4; ++t4) {
+                    const float4 c = reinterpret_cast<const float4*>(cw)[t4];
+                    float diff = __fsub_rn(rv[4 * t4], c.x);
+                    acc = __fmaf_rn(diff, diff, acc);
+                    diff = __fsub_rn(rv[4 * t4 + 1], c.y);
+                    acc = __fmaf_rn(diff, diff, acc);
+                    diff = __fsub_rn(rv[4 * t4 + 2], c.z);
+                    acc = __fmaf_rn(diff, diff, acc);
+                    diff = __fsub_rn(rv[4 * t4 + 3], c.w);
+                    acc = __fmaf_rn(diff, diff, acc);
+                }
+            } else if constexpr (DSUB > 0) {
+#pragma unroll
+                for (int t = 0; t < DSUB; ++t) {
+                    const float diff = __fsub_rn(rv[t], cw[t]);
+                    acc = __fmaf_rn(diff, diff, acc);
+                }
+            } else {
+                for (int t = 0; t < ds; ++t) {
+                    const float diff = __fsub_rn(rm[t], cw[t]);
+                    acc = __fmaf_rn(diff, diff, acc);
+                }
+            }
+        }
+        if (acc < best) {  // codewords ascend within a lane, so an equal entry keeps the lower one
+            best = acc;
+            bj = j;
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float ov = __shfl_xor_sync(0xFFFFFFFFu, best, off);
+        const int oj = __shfl_xor_sync(0xFFFFFFFFu, bj, off);
+        if (ov < best || (ov == best && oj < bj)) {
+            best = ov;
+            bj = oj;
+        }
+    }
+    return bj;
+}
+
+// The batch loop of the encode kernel for one sub-vector width.  A CTA walks batches of V = 1024 / d
+// (rounded down to a power of two) vectors.  While the warps encode a batch -- one (vector, subspace)
+// pair per warp and step -- every thread already holds one residual coordinate of the next batch in a
+// register (row, id and centroid fetched from global memory under the arithmetic), so the kernel never
+// waits for memory between vectors.  REGS (the number of subspaces divides 32, sub-vectors of at most 4):
+// a warp then meets the same subspace at every step and keeps its 8 codewords per lane in registers for
+// the whole launch, so the shared-memory pipe carries only the residuals (the codebook reads were what
+// bounded the kernel: 1,024 wavefronts per vector).
+template <int DSUB, bool REGS>
+__device__ __forceinline__ void pq_encode_body(const PqEncodeParams& p, const float* cb, float* rbuf, int* badbuf) {
+    const int dsub = p.d / p.pq_m;
+    int V = kPqEncodeElems / p.d;
+    V = V >= 32 ? 32 : (V >= 16 ? 16 : (V >= 8 ? 8 : (V >= 4 ? 4 : (V >= 2 ? 2 : 1))));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const int e = threadIdx.x;                 // this thread's coordinate of a batch
+    const int ev = e / p.d, et = e - ev * p.d;  // vector within the batch, coordinate
+
+    // residual coordinate (ev, et) of the batch that starts at vector `base`; bad = the id is out of range
+    auto fetch = [&](int64_t base, float& r, int& bad) {
+        r = 0.0f;
+        bad = 0;
+        const int64_t i = base + ev;
+        if (ev < V && i < p.n) {
+            const int32_t l = p.ids[i];
+            if (l >= 0 && l < p.nlist) {
+                const float xv = pq_elem(p.x, p.x_type, i * p.d + et);
+                r = __fsub_rn(xv, p.centroids[static_cast<int64_t>(l) * p.d + et]);
+            } else {
+                bad = 1;
+            }
+        }
+    };
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * V;
+    int64_t base = static_cast<int64_t>(blockIdx.x) * V;
+    float r_next;
+    int bad_next;
+    fetch(base, r_next, bad_next);
+    __syncthreads();  // the codebook is in shared memory
+    float cwr[kPqK / 32][DSUB > 0 ? DSUB : 1];
+    if constexpr (REGS) {
+        const int m = warp % p.pq_m;  // the one subspace this warp ever meets
+#pragma unroll
+        for (int q = 0; q < kPqK / 32; ++q)
+#pragma unroll
+            for (int t = 0; t < DSUB; ++t) cwr[q][t] = cb[(static_cast<size_t>(m) * kPqK + lane + 32 * q) * DSUB + t];
+    }
+    int buf = 0;
+    for (; base < p.n; base += stride) {
+        rbuf[buf * kPqEncodeElems + e] = r_next;
+        if (et == 0 && ev < V) badbuf[buf * 64 + ev] = bad_next;
+        __syncthreads();  // this batch's residuals are in place
+        fetch(base + stride, r_next, bad_next);  // the next batch travels while this one is encoded
+        const int nv = static_cast<int>(p.n - base < V ? p.n - base : V);
+        const float* rb = rbuf + buf * kPqEncodeElems;
+        const int* bb = badbuf + buf * 64;
+        for (int item = warp; item < nv * p.pq_m; item += nwarps) {
+            const int vi = item / p.pq_m, m = item - vi * p.pq_m;
+            const int64_t i = base + vi;
+            int code = 0;
+            if (bb[vi]) {
+                if (lane == 0 && m == 0) atomicCAS(p.status, 0, kPqStatusBadId);
+            } else {
+                code = pq_encode_subspace<DSUB, REGS>(rb + vi * p.d + m * dsub, cb + static_cast<size_t>(m) * kPqK * dsub, dsub,
+                                                      lane, cwr);
+            }
+            if (lane == 0 && IVF_IN_BOUNDS(430, code, kPqK)) p.codes[i * p.pq_m + m] = static_cast<uint8_t>(code);
+        }
+        buf ^= 1;  // (the buffer written next was last read two batches ago: one barrier per batch is enough)
+    }
+}
+
+// Persistent: one CTA per SM keeps the codebook [m][j][dsub] in shared memory.
 __global__ void __launch_bounds__(kPqThreads, 1) pq_encode_kernel(const PqEncodeParams p) {
     extern __shared__ __align__(16) uint8_t pq_smem_raw[];
-    const PqSmem s = pq_carve(pq_smem_raw, p.d, p.pq_m);
+    float* cb = reinterpret_cast<float*>(pq_smem_raw);                       // [pq_m][256][dsub]
+    float* rbuf = cb + static_cast<size_t>(p.d) * kPqK;                      // [2][kPqEncodeElems]
+    int* badbuf = reinterpret_cast<int*>(rbuf + 2 * kPqEncodeElems);         // [2][64]
     const int dsub = p.d / p.pq_m;
-    pq_load_codebooks(p.codebooks, p.d, dsub, s.cbt);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    for (int64_t i = blockIdx.x; i < p.n; i += gridDim.x) {
-        const int32_t l = p.ids[i];
-        const bool ok = l >= 0 && l < p.nlist;
-        __syncthreads();  // the previous row's table has been consumed (and the codebook is in place)
-        if (!ok) {
-            if (threadIdx.x == 0) atomicCAS(p.status, 0, kPqStatusBadId);
-            for (int m = threadIdx.x; m < p.pq_m; m += blockDim.x) p.codes[i * p.pq_m + m] = 0;
-            continue;
-        }
-        for (int t = threadIdx.x; t < p.d; t += blockDim.x) {
-            const float xv = pq_elem(p.x, p.x_type, i * p.d + t);
-            s.r[t] = __fsub_rn(xv, p.centroids[static_cast<int64_t>(l) * p.d + t]);
-        }
-        __syncthreads();
-        pq_build_lut<false>(s.r, s.cbt, s.lut, p.pq_m, dsub, threadIdx.x, blockDim.x);
-        __syncthreads();
-        for (int m = warp; m < p.pq_m; m += nwarps) {
-            const float* row = s.lut + m * kPqK;
-            float best = row[lane];
-            int bj = lane;
-#pragma unroll
-            for (int q = 1; q < kPqK / 32; ++q) {
-                const float v = row[lane + 32 * q];
-                if (v < best) {
-                    best = v;
-                    bj = lane + 32 * q;
-                }
-            }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                const float ov = __shfl_xor_sync(0xFFFFFFFFu, best, off);
-                const int oj = __shfl_xor_sync(0xFFFFFFFFu, bj, off);
-                if (ov < best || (ov == best && oj < bj)) {
-                    best = ov;
-                    bj = oj;
-                }
-            }
-            if (lane == 0 && IVF_IN_BOUNDS(430, bj, kPqK)) p.codes[i * p.pq_m + m] = static_cast<uint8_t>(bj);
-        }
+    const int total_cb = p.d * kPqK;
+    if ((reinterpret_cast<uintptr_t>(p.codebooks) & 15) == 0) {
+        for (int i = threadIdx.x * 4; i < total_cb; i += blockDim.x * 4)    // d * 256 is a multiple of 4
+            *reinterpret_cast<float4*>(cb + i) = __ldg(reinterpret_cast<const float4*>(p.codebooks + i));
+    } else {
+        for (int i = threadIdx.x; i < total_cb; i += blockDim.x) cb[i] = __ldg(p.codebooks + i);
+    }
+    const bool regs = (32 % p.pq_m) == 0;  // every warp meets one subspace only
+    switch (dsub) {
+        case 2: return regs ? pq_encode_body<2, true>(p, cb, rbuf, badbuf) : pq_encode_body<2, false>(p, cb, rbuf, badbuf);
+        case 3: return regs ? pq_encode_body<3, true>(p, cb, rbuf, badbuf) : pq_encode_body<3, false>(p, cb, rbuf, badbuf);
+        case 4: return regs ? pq_encode_body<4, true>(p, cb, rbuf, badbuf) : pq_encode_body<4, false>(p, cb, rbuf, badbuf);
+        case 6: return pq_encode_body<6, false>(p, cb, rbuf, badbuf);
+        case 8: return pq_encode_body<8, false>(p, cb, rbuf, badbuf);
+        default: return pq_encode_body<0, false>(p, cb, rbuf, badbuf);
     }
 }
 
