@@ -618,6 +618,10 @@ def main():
                                           prepared_too=True)
         line["c4"] = routing_config_entry(synth.C4, "C4", dev, pk, flush, 5, TRAFFIC_FUSED_C4_CHUNK_BYTES, 384 * oc)
         line["serving"] = serving_entry(dev, flush)
+        # the same roofline objects under flat names
+        line["roofline_c1_call"] = line["c1_call"]["roofline"]
+        line["roofline_c2"] = line["c2"]["roofline"]
+        line["roofline_c4"] = line["c4"]["roofline"]
         line["config"]["side_measurements"] = ("c1_call, c2, c4: one timed ivf_route call of the C1 / C2 (10000 x 262144 x 96, "
                                                "nprobe 128) / C4 (100000 x 1048576 x 96, nprobe 256) configurations, CUDA "
                                                "events, L2 flushed before each call; serving: B = 8 and 2048 against a "
