@@ -543,6 +543,99 @@ __device__ __forceinline__ unsigned int widen_row_u8(const uint8_t* __restrict__
     return sumsq;
 }
 
+// The same for the 32 consecutive rows of one TMEM lane quadrant, by one warp with coalesced loads:
+// the rows are contiguous in memory, so lane l of step s takes the 16-byte chunk number 32 s + l of the
+// quadrant's 32 * d bytes (four steps in flight).  A chunk of 16 values becomes two 16-byte chunks of
+// the operand row, written where the swizzles put them.  The squares are summed per chunk and brought
+// to the lane that owns the row (lane = row within the quadrant), which also writes the norm columns
+// and |x|^2.  Rows at or beyond `n` become zero rows.
+__device__ __forceinline__ void widen_rows_u8_warp(const uint8_t* __restrict__ x_raw, int64_t grow0, int64_t n, int d, int kd,
+                                                   uint8_t* tile, int a_data_bytes, int row0, int lane, float sx, float A,
+                                                   float* __restrict__ xn_out) {
+    const __half2 k1024 = __floats2half2_rn(1024.0f, 1024.0f);
+    const __half2 sx2 = __floats2half2_rn(sx, sx);
+    auto cvt2 = [&](uint32_t w, uint32_t sel) {  // two bytes -> two fp16 (0x6400 | b is the half 1024 + b; all exact)
+        uint32_t q = __byte_perm(w, 0x64646464u, sel);
+        const __half2 t2 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&q), k1024), sx2);
+        return *reinterpret_cast<const uint32_t*>(&t2);
+    };
+    const int cpr = d >> 4;        // 16-byte chunks per row
+    const int total = 32 * cpr;    // chunks of the quadrant
+    const int64_t left = n - grow0;
+    const int rows_valid = left <= 0 ? 0 : (left < 32 ? static_cast<int>(left) : 32);
+    const uint4* src = reinterpret_cast<const uint4*>(x_raw + (rows_valid > 0 ? grow0 : 0) * d);
+    unsigned int sumsq = 0;        // of row `lane`
+    constexpr int U = 4;
+#pragma unroll 1
+    for (int g0 = 0; g0 < total; g0 += 32 * U) {
+        uint4 w[U];
+        int rr[U], cc[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int g = g0 + u * 32 + lane;
+            rr[u] = g / cpr;
+            cc[u] = g - rr[u] * cpr;
+            w[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (g < total && rr[u] < rows_valid) w[u] = src[g];
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int gb = g0 + u * 32;  // first chunk of this step
+            if (gb < total) {            // uniform over the warp
+                unsigned int part = __dp4a(w[u].x, w[u].x, 0u);
+                part = __dp4a(w[u].y, w[u].y, part);
+                part = __dp4a(w[u].z, w[u].z, part);
+                part = __dp4a(w[u].w, w[u].w, part);
+                if (gb + lane < total) {
+                    const int row = row0 + rr[u];
+                    uint4 o0, o1;
+                    o0.x = cvt2(w[u].x, 0x5140u); o0.y = cvt2(w[u].x, 0x5342u); o0.z = cvt2(w[u].y, 0x5140u); o0.w = cvt2(w[u].y, 0x5342u);
+                    o1.x = cvt2(w[u].z, 0x5140u); o1.y = cvt2(w[u].z, 0x5342u); o1.z = cvt2(w[u].w, 0x5140u); o1.w = cvt2(w[u].w, 0x5342u);
+                    const int c = 2 * cc[u];  // 8-value chunk index inside the row; c and c + 1 lie in the same 64-wide slice
+                    const int slice = c >> 3, j = c & 7;
+                    uint8_t* rowp = tile + slice * kBlockM * kSliceRowBytes + row * kSliceRowBytes;
+                    if (IVF_IN_BOUNDS(112, slice * kBlockM * kSliceRowBytes + row * kSliceRowBytes + (((j + 1) ^ (row & 7)) << 4),
+                                      a_data_bytes - 15)) {
+                        *reinterpret_cast<uint4*>(rowp + ((j ^ (row & 7)) << 4)) = o0;
+                        *reinterpret_cast<uint4*>(rowp + (((j + 1) ^ (row & 7)) << 4)) = o1;
+                    }
+                }
+                // the chunks of one row are neighbours: add them up towards the row's first lane ...
+                int rid = gb + lane < total ? rr[u] : -1;
+#pragma unroll
+                for (int off = 1; off < 16; off <<= 1) {
+                    const unsigned int t = __shfl_down_sync(0xFFFFFFFFu, part, off);
+                    const int tr = __shfl_down_sync(0xFFFFFFFFu, rid, off);
+                    if (lane + off < 32 && tr == rid) part += t;
+                }
+                // ... and hand the sum to the lane that owns the row (a row may continue from the step before)
+                const int first = lane * cpr - gb;  // step-relative chunk where row `lane` starts
+                const bool in_step = first < 32 && first + cpr > 0;
+                const unsigned int got = __shfl_sync(0xFFFFFFFFu, part, in_step ? (first > 0 ? first : 0) : 0);
+                if (in_step) sumsq += got;
+            }
+        }
+    }
+    // zero padding up to kd (rows whose length is not a multiple of 64)
+    const int pad = (kd - d) >> 3;  // 8-value chunks per row
+    for (int i = lane; i < 32 * pad; i += 32) {
+        const int rrow = i / pad, c = (d >> 3) + (i - rrow * pad);
+        const int row = row0 + rrow;
+        const int slice = c >> 3, j = c & 7;
+        *reinterpret_cast<uint4*>(tile + slice * kBlockM * kSliceRowBytes + row * kSliceRowBytes + ((j ^ (row & 7)) << 4)) =
+            make_uint4(0u, 0u, 0u, 0u);
+    }
+    // norm columns of the lane's own row: A A A 0 ... 0; chunk j of the row goes to position j ^ ((row / 4) % 2)
+    const int row = row0 + lane;
+    const bool valid = lane < rows_valid;
+    const uint32_t a16 = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(A)));
+    const uint4 aug0 = valid ? make_uint4(a16 | (a16 << 16), a16, 0u, 0u) : make_uint4(0u, 0u, 0u, 0u);
+    const int sw = (row >> 2) & 1;
+    *reinterpret_cast<uint4*>(tile + a_data_bytes + row * kAugRowBytes + ((0 ^ sw) << 4)) = aug0;
+    *reinterpret_cast<uint4*>(tile + a_data_bytes + row * kAugRowBytes + ((1 ^ sw) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+    if (valid && IVF_IN_BOUNDS(141, grow0 + lane, n)) xn_out[grow0 + lane] = static_cast<float>(sumsq);
+}
+
 template <int EPI, int MT>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_xa,
@@ -819,15 +912,11 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             if (!IVF_IN_BOUNDS(140, slot, p.partials)) break;  // (checked build only: a slot outside the row's partials)
 
             if (p.x_raw != nullptr && half < MT) {
-                // uint8 points: this thread widens its own row of point tile `half`.  The tile is free:
+                // uint8 points: this warp widens its 32 rows of point tile `half`.  The tile is free:
                 // the last accumulator of the previous row group could only be read after every MMA
                 // that used the old tile had completed.
-                const int64_t grow = (r * MT + half) * kBlockM + row_in_tile;
-                const bool v = grow < p.n;
-                const unsigned int sumsq =
-                    widen_row_u8(p.x_raw + static_cast<size_t>(v ? grow : 0) * p.d, v, p.d, kd, smem_a + half * a_bytes,
-                                 a_data_bytes, row_in_tile, raw_scales[0], raw_scales[3]);
-                if (v && IVF_IN_BOUNDS(141, grow, p.n)) p.xn_out[grow] = static_cast<float>(sumsq);
+                widen_rows_u8_warp(p.x_raw, (r * MT + half) * kBlockM + quad * 32, p.n, p.d, kd, smem_a + half * a_bytes,
+                                   a_data_bytes, quad * 32, lane, raw_scales[0], raw_scales[3], p.xn_out);
                 fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's reads
                 __syncwarp();
                 if (lane == 0) mbar_arrive(a_full);
