@@ -565,7 +565,7 @@ __device__ __forceinline__ void widen_rows_u8_warp(const uint8_t* __restrict__ x
     const int rows_valid = left <= 0 ? 0 : (left < 32 ? static_cast<int>(left) : 32);
     const uint4* src = reinterpret_cast<const uint4*>(x_raw + (rows_valid > 0 ? grow0 : 0) * d);
     unsigned int sumsq = 0;        // of row `lane`
-    constexpr int U = 4;
+    constexpr int U = 8;
 #pragma unroll 1
     for (int g0 = 0; g0 < total; g0 += 32 * U) {
         uint4 w[U];
