@@ -25,7 +25,7 @@ EXPORTS = (
     "ivf_route_prepared",
     "ivf_pq_encode", "ivf_pq_search", "ivf_pq_residuals", "ivf_assign_candidates", "ivf_merge_shards",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
-    "ivf_debug_plan", "ivf_debug_span", "ivf_debug_rotation", "ivf_debug_set_rotation", "ivf_debug_fail_next_alloc", "ivf_debug_bounds_checked", "ivf_debug_bounds_probe", "ivf_debug_set_wait_limit_ns",
+    "ivf_debug_plan", "ivf_debug_span", "ivf_debug_rotation", "ivf_debug_set_rotation", "ivf_debug_set_threshold_pass", "ivf_debug_fail_next_alloc", "ivf_debug_bounds_checked", "ivf_debug_bounds_probe", "ivf_debug_set_wait_limit_ns",
     "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_set_row_chunk", "ivf_debug_stats", "ivf_debug_set_pq_groups", "ivf_debug_set_dependent_launch", "ivf_debug_set_crossing_cost",
 )
 
@@ -484,6 +484,10 @@ def ivf_debug_rotation(n: int, nlist: int, d: int, k: int, num_sms: int, row_gro
     if rc < 0:
         _raise(rc)
     return int(rc)
+
+
+def ivf_debug_set_threshold_pass(split: bool) -> None:
+    lib().ivf_debug_set_threshold_pass(1 if split else 0)
 
 
 def ivf_debug_set_rotation(on: bool) -> None:

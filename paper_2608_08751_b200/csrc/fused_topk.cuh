@@ -79,6 +79,8 @@ struct FusedParams {
     int cap;              // candidate-log capacity per (row, slot), k > 1 only
     int rule;             // k > 1: TAU_RUNNING, TAU_GIVEN or TAU_BOUNDED
     const float* tau_in;  // given rule: threshold per row, in key units
+    float* tau_out;       // sketch rule with whole_rows: the row's threshold is finished inside the kernel
+    int whole_rows;       // 1: every CTA owns whole row groups (no row group is shared between CTAs)
     Entry* part;          // k = 1: [n][partials]; k > 1: [n][partials][cap] entries, or 48-byte group
                           // records for the given rule
     int2* part_meta;      // k > 1: [n][partials] {entries (records) in the log or -1 if it overflowed,
@@ -667,13 +669,25 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     const int b = blockIdx.x;
     const int64_t T = p.total_units;
     const int NT = p.col_tiles;
-    const int64_t u0 = span_begin(T, G, NT, p.cross, b);
-    const int64_t u1 = span_begin(T, G, NT, p.cross, b + 1);
+    int64_t u0 = span_begin(T, G, NT, p.cross, b);
+    int64_t u1 = span_begin(T, G, NT, p.cross, b + 1);
+    if (p.whole_rows) {  // row groups dealt out whole: CTA b takes row groups [R b / G, R (b + 1) / G)
+        const int64_t R = T / NT;
+        u0 = (R * b / G) * NT;
+        u1 = (R * (b + 1) / G) * NT;
+    }
+    // hand-over of the two epilogue warps of a lane quadrant (sketch rule with whole row groups)
+    uint64_t* x_full = bars + 24;   // [4]
+    uint64_t* x_empty = bars + 28;  // [4]
 
     if (threadIdx.x == 0) {
         mbar_init(a_full, p.x_raw != nullptr ? 4 * MT : 1);  // TMA bytes, or one arrival per widening warp
         mbar_init(a_empty, 1);
         mbar_init(drain, 1);
+        for (int i = 0; i < 4; ++i) {
+            mbar_init(&x_full[i], 1);
+            mbar_init(&x_empty[i], 1);
+        }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&t_full[i], 1);
             mbar_init(&t_empty[i], kNumEpiWarps);
@@ -765,7 +779,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 }
             }
             if (lane == 0) {
-                int col = (t0 + (p.rotate ? col_rotation(T, G, NT, p.cross, r) : 0)) % NT;  // centroid tile of position t
+                int col = (t0 + ((p.rotate && !p.whole_rows) ? col_rotation(T, G, NT, p.cross, r) : 0)) % NT;  // centroid tile of position t
                 for (; t < t1 && ok; ++t) {
                     ok = load_b(col);
                     if (++col == NT) col = 0;
@@ -903,12 +917,13 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             }
         }
         int it = 0;
+        [[maybe_unused]] int xseg = 0;  // row groups whose threshold this CTA has finished
         bool ok = true;
         for (int64_t u = u0; u < u1 && ok;) {
             const int64_t r = u / NT;  // row group
             const int t0 = static_cast<int>(u - r * NT);
             const int t1 = static_cast<int>((u1 - r * NT < NT) ? (u1 - r * NT) : NT);
-            const int slot = (b - cta_of_unit(T, G, NT, p.cross, r * NT)) * kEpiHalves + half;
+            const int slot = p.whole_rows ? half : (b - cta_of_unit(T, G, NT, p.cross, r * NT)) * kEpiHalves + half;
             if (!IVF_IN_BOUNDS(140, slot, p.partials)) break;  // (checked build only: a slot outside the row's partials)
 
             if (p.x_raw != nullptr && half < MT) {
@@ -950,7 +965,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 }
             }
 
-            int col = (t0 + (p.rotate ? col_rotation(T, G, NT, p.cross, r) : 0)) % NT;  // centroid tile of position t
+            int col = (t0 + ((p.rotate && !p.whole_rows) ? col_rotation(T, G, NT, p.cross, r) : 0)) % NT;  // centroid tile of position t
             for (int t = t0; t < t1 && ok; ++t) {
                 const bool ragged = (col + 1) * p.block_n > p.nlist;
                 const int tile_j0 = col * p.block_n;
@@ -1065,7 +1080,43 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 }
                 ++it;
             }
-            if (ok) {
+            if constexpr (EPI == EPI_SKETCH && MT == 1) {
+                if (ok && p.tau_out != nullptr) {
+                    // This CTA saw the row group's whole sample, split between the two warps of every lane
+                    // quadrant: the upper-half warp passes its 16 sorted minima through shared memory, the
+                    // lower-half warp finishes the threshold.  With a and b ascending, min(a[i], b[15 - i])
+                    // over i are the 16 smallest of the 32 values, so their maximum is the 16th smallest.
+                    float* xch = reinterpret_cast<float*>(hist_all) + row_in_tile * kSampleM;
+                    if (half == 1) {
+                        if (xseg > 0) ok = __all_sync(0xFFFFFFFFu, mbar_wait(&x_empty[quad], (xseg - 1) & 1, ctl, 7));
+                        if (ok) {
+#pragma unroll
+                            for (int i = 0; i < kSampleM; i += 4)
+                                *reinterpret_cast<float4*>(xch + i) = make_float4(st[0].net[i], st[0].net[i + 1], st[0].net[i + 2], st[0].net[i + 3]);
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&x_full[quad]);
+                        }
+                    } else {
+                        ok = __all_sync(0xFFFFFFFFu, mbar_wait(&x_full[quad], xseg & 1, ctl, 8));
+                        if (ok) {
+                            float other[kSampleM];
+#pragma unroll
+                            for (int i = 0; i < kSampleM; i += 4) {
+                                const float4 v = *reinterpret_cast<const float4*>(xch + i);
+                                other[i] = v.x; other[i + 1] = v.y; other[i + 2] = v.z; other[i + 3] = v.w;
+                            }
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&x_empty[quad]);
+                            float t16 = -INF;
+#pragma unroll
+                            for (int i = 0; i < kSampleM; ++i) t16 = fmaxf(t16, fminf(st[0].net[i], other[kSampleM - 1 - i]));
+                            if (valid[0]) p.tau_out[row[0]] = t16;
+                        }
+                    }
+                    ++xseg;
+                }
+            }
+            if (ok && !(EPI == EPI_SKETCH && p.tau_out != nullptr)) {
 #pragma unroll
                 for (int h = 0; h < MT; ++h) {
                     if (!valid[h]) continue;

@@ -257,6 +257,7 @@ int choose_rule(int k, int nlist, int* stride) {
     return k <= kSampleM ? TAU_RUNNING : TAU_BOUNDED;
 }
 
+int g_sketch_whole = 1;  // test hook (ivf_debug_set_threshold_pass): 0 = the threshold pass always as sketch kernel + merge
 int g_rotate = 1;  // test hook (ivf_debug_set_rotation): 0 = every position of a sweep stands for its own tile index
 int g_cross = -1;  // crossing cost used by the span partition; -1 = by kernel variant (test hook: ivf_debug_set_crossing_cost)
 
@@ -455,7 +456,7 @@ struct PointPrep {
 int launch_fused(DeviceCtx& ctx, const Plan& pl, int64_t n, int nlist, int k, int rule, const float* tau_in,
                  const PointPrep& pp, const CUtensorMap& tmap_c, const CUtensorMap& tmap_ca, Entry* part,
                  int2* part_meta, int kind, cudaStream_t stream, const unsigned int* bits, float* scal,
-                 int* clear0 = nullptr, int* clear1 = nullptr, int* clear32 = nullptr) {
+                 int* clear0 = nullptr, int* clear1 = nullptr, int* clear32 = nullptr, float* tau_out = nullptr) {
     FusedParams fp;
     fp.clear0 = clear0;
     fp.clear1 = clear1;
@@ -480,6 +481,8 @@ int launch_fused(DeviceCtx& ctx, const Plan& pl, int64_t n, int nlist, int k, in
     fp.cap = pl.cap;
     fp.rule = rule;
     fp.tau_in = tau_in;
+    fp.tau_out = tau_out;
+    fp.whole_rows = tau_out != nullptr ? 1 : 0;
     fp.part = part;
     fp.part_meta = part_meta;
     fp.status = ctx.status;
@@ -557,9 +560,21 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     if (given) pl.cap = (k <= kSampleM ? 384 : 4 * k) + kGroupLogMargin;
     size_t part_bytes = static_cast<size_t>(n) * pl.partials * pl.cap * (given ? kRecordBytes : sizeof(Entry));
     size_t meta_bytes = static_cast<size_t>(n) * pl.partials * sizeof(int2);
+    // Threshold pass in one kernel: with enough row tiles to occupy the GPU every CTA takes whole row tiles
+    // of 128 points across the entire centroid sample and finishes the rows' thresholds itself -- no
+    // partial sketches in global memory and no merge launch after it (C1: 36 + 17 us -> one kernel).
+    // Small batches keep the split schedule: a few CTAs walking the whole sample would take longer.
+    bool sketch_whole = false;
     if (given) {
-        rc = make_plan(n, cp.sample_rows, d, kSampleM, ctx.num_sms, &pls);
+        const int64_t row_tiles128 = (n + kBlockM - 1) / kBlockM;
+        const int sample_tiles = (cp.sample_rows + 255) / 256;
+        sketch_whole = g_sketch_whole && row_tiles128 >= 48 && sample_tiles <= 48;
+        rc = make_plan(n, cp.sample_rows, d, kSampleM, ctx.num_sms, &pls, sketch_whole);
         if (rc != IVF_OK) return rc;
+        if (sketch_whole) {
+            pls.ctas = static_cast<int>(pls.row_tiles < ctx.num_sms ? pls.row_tiles : ctx.num_sms);
+            pls.partials = kEpiHalves;
+        }
         const size_t pb = static_cast<size_t>(n) * pls.partials * pls.cap * sizeof(Entry);
         const size_t mb = static_cast<size_t>(n) * pls.partials * sizeof(int2);
         part_bytes = pb > part_bytes ? pb : part_bytes;
@@ -625,12 +640,15 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     if (given) {
         // threshold pass over every S-th centroid: the 16th smallest group minimum becomes the row's tau
         rc = launch_fused(ctx, pls, n, cp.sample_rows, kSampleM, TAU_SKETCH, nullptr, pp, cp.tmap_cs, cp.tmap_csa, part,
-                          part_meta, TK_THRESH, stream, cp.bits, cp.scal);
+                          part_meta, TK_THRESH, stream, cp.bits, cp.scal, nullptr, nullptr, nullptr,
+                          sketch_whole ? tau : nullptr);
         if (rc != IVF_OK) return rc;
         MergeParams ms = merge_params(pls, n, kSampleM, part, part_meta, pp, cp.scal);
         ms.tau_out = tau;
         tk = timing_begin(TK_THRESH, stream);
-        if (pls.partials <= 32)
+        if (sketch_whole) {
+            // the kernel wrote the thresholds itself
+        } else if (pls.partials <= 32)
             LAUNCH_DEP(4, merge_tau_warp_kernel, static_cast<unsigned>((n * 32 + 255) / 256), 256, 0, stream, ms);
         else {
             const int threads = pls.partials >= kTauThreads ? kTauThreads : (pls.partials + 31) / 32 * 32;
@@ -1453,6 +1471,11 @@ int ivf_debug_set_row_chunk(int64_t rows) {
 
 int ivf_debug_set_dependent_launch(int on) {
     g_pdl = on;
+    return IVF_OK;
+}
+
+int ivf_debug_set_threshold_pass(int split) {
+    g_sketch_whole = split ? 0 : 1;
     return IVF_OK;
 }
 

@@ -316,8 +316,11 @@ def main():
     ap.add_argument("--dependent-launch", type=int, default=-1, help="kernel-family mask of dependent launches (0 = none)")
     ap.add_argument("--crossing-cost", type=int, default=-1, help="span-partition crossing cost in units (0 = equal counts)")
     ap.add_argument("--rotation", type=int, default=1, help="0 = centroid tiles swept in index order (for comparison)")
+    ap.add_argument("--split-threshold-pass", type=int, default=0, dest="split_threshold",
+                    help="1 = threshold pass always as sketch kernel + merge launch (for comparison)")
     args = ap.parse_args()
     B.ivf_debug_set_rotation(bool(args.rotation))
+    B.ivf_debug_set_threshold_pass(bool(args.split_threshold))
     if args.crossing_cost >= 0:
         B.ivf_debug_set_crossing_cost(args.crossing_cost)
     if args.dependent_launch >= 0:

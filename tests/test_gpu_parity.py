@@ -145,6 +145,23 @@ def test_sampled_threshold_rarely_needs_the_exact_recomputation():
     parity.check_route(q, c, 64, ids[rows], dists[rows], rows=rows)
 
 
+@pytest.mark.parametrize("n,nlist,d,k,dtype", [(6200, 20000, 128, 40, "u8"), (7000, 70000, 96, 100, "f32"), (6145, 9000, 64, 17, "f32")])
+def test_threshold_pass_in_one_kernel_gives_the_same_results(n, nlist, d, k, dtype):
+    # from 48 row tiles on, every CTA of the threshold pass takes whole row tiles across the entire
+    # sample and finishes the thresholds itself; the split schedule (sketch kernel + merge launch)
+    # computes the same statistic, so ids and distances must agree bit for bit
+    x, c = _rand(n, nlist, d, dtype, seed=n)
+    ids, dists = _route(x, c, k)
+    B.ivf_debug_set_threshold_pass(True)
+    try:
+        ids2, dists2 = _route(x, c, k)
+    finally:
+        B.ivf_debug_set_threshold_pass(False)
+    assert (ids == ids2).all() and (dists == dists2).all()
+    rows = np.arange(0, n, 37)
+    parity.check_route(x, c, k, ids[rows], dists[rows], rows=rows)
+
+
 def test_duplicate_centroids_resolve_to_lower_id():
     _, c = _rand(1, 700, 128, "f32", 9)
     c[500] = c[20]
