@@ -145,7 +145,8 @@ def test_sampled_threshold_rarely_needs_the_exact_recomputation():
     parity.check_route(q, c, 64, ids[rows], dists[rows], rows=rows)
 
 
-@pytest.mark.parametrize("n,nlist,d,k,dtype", [(6200, 20000, 128, 40, "u8"), (7000, 70000, 96, 100, "f32"), (6145, 9000, 64, 17, "f32")])
+@pytest.mark.parametrize("n,nlist,d,k,dtype", [(6200, 20000, 128, 40, "u8"), (7000, 70000, 96, 100, "f32"), (6145, 9000, 64, 17, "f32"),
+                                               (20001, 20000, 64, 20, "u8")])  # the last: more row tiles than SMs
 def test_threshold_pass_in_one_kernel_gives_the_same_results(n, nlist, d, k, dtype):
     # from 48 row tiles on, every CTA of the threshold pass takes whole row tiles across the entire
     # sample and finishes the thresholds itself; the split schedule (sketch kernel + merge launch)
