@@ -1274,7 +1274,10 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     int tk = timing_begin(TK_PQ_SCAN, stream);
     // (family bit 128 of the dependent-launch mask: the four kernels of a search overlap their launch
     // latencies, which is a tenth of a small batch)
-    LAUNCH_DEP(128, pq_transpose_codebooks_kernel, (d * kPqK + 255) / 256, 256, 0, stream, codebooks, d, d / pq_m, cbt);
+    // the scan reads the codebook as given where one codeword is one aligned vector load
+    const bool cb_rows = pq_codebook_by_rows(d / pq_m) && (reinterpret_cast<uintptr_t>(codebooks) & 15) == 0;
+    if (!cb_rows)
+        LAUNCH_DEP(128, pq_transpose_codebooks_kernel, (d * kPqK + 255) / 256, 256, 0, stream, codebooks, d, d / pq_m, cbt);
     LAUNCH_DEP(128, pq_setup_query_kernel, static_cast<unsigned>(nq), 128, 0, stream, probe_ids, nprobe, nlist,
                reinterpret_cast<const long long*>(list_offsets), chunk_start, reinterpret_cast<long long*>(out_counts),
                ctx.status);
@@ -1289,7 +1292,8 @@ int ivf_pq_search(const void* queries, int64_t nq, int d, ivf_dtype qtype, const
     sp.n_rerank = n_rerank;
     sp.ngroups = ngroups;
     sp.centroids = centroids;
-    sp.cbt = cbt;
+    sp.cbt = cb_rows ? codebooks : cbt;
+    sp.cb_rows = cb_rows ? 1 : 0;
     sp.probes = probe_ids;
     sp.offsets = reinterpret_cast<const long long*>(list_offsets);
     sp.codes = codes;

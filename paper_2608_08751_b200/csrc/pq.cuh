@@ -124,11 +124,65 @@ __device__ __forceinline__ void pq_build_lut_fixed(const float* __restrict__ r, 
     }
 }
 
-// lut[m * 256 + j] for the residual r.  kGlobal: cbt points to the transposed codebook in global
-// memory (read through L1); otherwise to the copy in shared memory.
+// The same build from the codebook in its given layout [pq_m][256][dsub], for the widths whose
+// codeword is one 8- or 16-byte load (a warp's 32 codewords are then contiguous, so the load has as
+// many shared-memory wavefronts as the coordinate-major copy needs but a quarter or half of the
+// instructions).  Same operations in the same order as pq_build_lut_fixed: bit-identical tables.
+template <bool kGlobal, int DSUB>
+__device__ __forceinline__ void pq_build_lut_rows(const float* __restrict__ r, const float* __restrict__ cb,
+                                                  float* __restrict__ lut, int pq_m, int tid, int nthreads) {
+    static_assert(DSUB == 2 || DSUB == 4, "one vector load per codeword");
+    const int j = tid & (kPqK - 1);
+    const int first = tid >> 8;
+    const int step = nthreads >> 8;
+    const float* row = cb + (first * kPqK + j) * DSUB;
+    const float* rp = r + first * DSUB;
+    float* out = lut + first * kPqK + j;
+    const int row_step = step * kPqK * DSUB, r_step = step * DSUB, out_step = step * kPqK;
+#pragma unroll 4
+    for (int m = first; m < pq_m; m += step) {
+        float rv[DSUB], cv[DSUB];
+        if constexpr (DSUB == 4) {
+            const float4 v = *reinterpret_cast<const float4*>(rp);
+            rv[0] = v.x; rv[1] = v.y; rv[2] = v.z; rv[3] = v.w;
+            float4 c;
+            if constexpr (kGlobal) c = __ldg(reinterpret_cast<const float4*>(row));
+            else c = *reinterpret_cast<const float4*>(row);
+            cv[0] = c.x; cv[1] = c.y; cv[2] = c.z; cv[3] = c.w;
+        } else {
+            const float2 v = *reinterpret_cast<const float2*>(rp);
+            rv[0] = v.x; rv[1] = v.y;
+            float2 c;
+            if constexpr (kGlobal) c = __ldg(reinterpret_cast<const float2*>(row));
+            else c = *reinterpret_cast<const float2*>(row);
+            cv[0] = c.x; cv[1] = c.y;
+        }
+        float acc = 0.0f;
+#pragma unroll
+        for (int t = 0; t < DSUB; ++t) {
+            const float diff = __fsub_rn(rv[t], cv[t]);
+            acc = __fmaf_rn(diff, diff, acc);
+        }
+        *out = acc;
+        row += row_step;
+        rp += r_step;
+        out += out_step;
+    }
+}
+
+// true: the scan kernels can read the codebook in its given layout (pq_build_lut_rows), if it starts
+// on a 16-byte boundary; false: they need the coordinate-major copy
+__host__ __device__ inline bool pq_codebook_by_rows(int dsub) { return dsub == 2 || dsub == 4; }
+
+// lut[m * 256 + j] for the residual r.  cbt: the codebook, as given when by_rows, else coordinate-
+// major.  kGlobal: it is in global memory (read through L1); otherwise a copy in shared memory.
 template <bool kGlobal>
 __device__ __forceinline__ void pq_build_lut(const float* r, const float* cbt, float* lut, int pq_m, int dsub, int tid,
-                                             int nthreads) {
+                                             int nthreads, bool by_rows) {
+    if (by_rows) {
+        if (dsub == 4) return pq_build_lut_rows<kGlobal, 4>(r, cbt, lut, pq_m, tid, nthreads);
+        return pq_build_lut_rows<kGlobal, 2>(r, cbt, lut, pq_m, tid, nthreads);
+    }
     switch (dsub) {
         case 2: return pq_build_lut_fixed<kGlobal, 2>(r, cbt, lut, pq_m, tid, nthreads);
         case 3: return pq_build_lut_fixed<kGlobal, 3>(r, cbt, lut, pq_m, tid, nthreads);
@@ -566,7 +620,9 @@ struct PqScanParams {
     int d, pq_m, nlist, nprobe, n_rerank;
     int ngroups;             // groups per query
     const float* centroids;
-    const float* cbt;        // transposed codebook [d][256] in global memory (read through L1, or copied to shared memory)
+    const float* cbt;        // codebook in global memory (read through L1, or copied to shared memory): as given
+                             // ([pq_m][256][dsub]) when cb_rows, else transposed [d][256]
+    int cb_rows;
     const int32_t* probes;
     const long long* offsets;
     const uint8_t* codes;
@@ -769,7 +825,7 @@ __device__ __forceinline__ void pq_scan_groups(const PqScanParams& p, const PqTe
                     if (later < p.nprobe && s.cs[later] < chunk1 && tid < p.d)
                         cnext = p.centroids[static_cast<int64_t>(s.list_id[later]) * p.d + tid];
                     pq_group_sync<BAR, NT>();
-                    pq_build_lut<kGlobalCb>(s.r, cbt, s.lut, p.pq_m, dsub, tid, NT);
+                    pq_build_lut<kGlobalCb>(s.r, cbt, s.lut, p.pq_m, dsub, tid, NT, p.cb_rows != 0);
                     pq_group_sync<BAR, NT>();
                     built = pr;
                 }
@@ -837,7 +893,7 @@ __global__ void __launch_bounds__(2 * kPqScanThreads, 1) pq_scan_teams_kernel(co
     extern __shared__ __align__(16) uint8_t pq_smem_raw[];
     if (2 * static_cast<int64_t>(blockIdx.x) >= p.nq * p.ngroups) return;
     float* cbt = reinterpret_cast<float*>(pq_smem_raw);
-    {   // straight copy of the transposed codebook (d * 256 floats, 16-byte pieces)
+    {   // straight copy of the codebook (d * 256 floats, 16-byte pieces)
         const float4* src = reinterpret_cast<const float4*>(p.cbt);
         float4* dst = reinterpret_cast<float4*>(cbt);
         for (int i = threadIdx.x; i < p.d * (kPqK / 4); i += blockDim.x) dst[i] = __ldg(src + i);
