@@ -106,6 +106,31 @@ def test_every_group_count_gives_the_same_result(groups):
         B.ivf_debug_set_pq_groups(0)
 
 
+@pytest.mark.parametrize("d,pq_m", [(128, 32), (64, 32)])  # sub-vectors of 4 and of 2
+@pytest.mark.parametrize("groups", [0, -2])
+def test_codebook_on_any_four_byte_boundary(d, pq_m, groups):
+    # the table build reads these widths with vector loads when the codebook starts on a 16-byte
+    # boundary and from a coordinate-major copy otherwise: same candidates and estimates either way
+    q, c, cb, ids, offsets, x, probes = _problem(21, 30000, 50, d, pq_m, "u8", 11, 9)
+    codes = O.pq_encode(x, ids, c, cb)
+    flat = torch.zeros(cb.size + 4, dtype=torch.float32, device=DEV)
+    B.ivf_debug_set_pq_groups(groups)
+    try:
+        outs = []
+        for shift in (0, 1, 2):
+            view = flat[shift:shift + cb.size].view(cb.shape)
+            view.copy_(_t(cb))
+            assert (view.data_ptr() % 16 == 0) == (shift == 0)
+            got = B.ivf_pq_search(_t(q), _t(c), _t(probes), _t(offsets), _t(codes), view, 128)
+            outs.append([t.cpu().numpy() for t in got])
+        for o in outs[1:]:
+            for a, b in zip(outs[0], o):
+                assert (a == b).all()
+        _check_search(q, c, cb, offsets, codes, probes, 128)
+    finally:
+        B.ivf_debug_set_pq_groups(0)
+
+
 def test_large_batch_one_group_per_query():
     q, c, cb, ids, offsets, x, probes = _problem(8, 40000, 300, 64, 16, "f32", 3000, 16)
     codes = O.pq_encode(x, ids, c, cb)
