@@ -79,6 +79,13 @@ struct FusedParams {
     int cap;              // candidate-log capacity per (row, slot), k > 1 only
     int rule;             // k > 1: TAU_RUNNING, TAU_GIVEN or TAU_BOUNDED
     const float* tau_in;  // given rule: threshold per row, in key units
+    float* sketch_t;      // batches of at most kFoldRows rows, if set: the partial sketches of the threshold
+                          // pass as [n][16][sketch_pitch] floats (value i of slot s of row r at
+                          // (r * 16 + i) * sketch_pitch + s; ascending in i).  The sketch rule writes them
+                          // there instead of `part`; the given rule reads them: its epilogue warps finish
+                          // the thresholds themselves and tau_in is not read
+    int sketch_pitch;     // >= the slots of a row
+    int sketch_slots;     // slots that hold a sketch (given rule)
     float* tau_out;       // sketch rule with whole_rows: the row's threshold is finished inside the kernel
     int whole_rows;       // 1: every CTA owns whole row groups (no row group is shared between CTAs)
     Entry* part;          // k = 1: [n][partials]; k > 1: [n][partials][cap] entries, or 48-byte group
@@ -638,6 +645,63 @@ __device__ __forceinline__ void widen_rows_u8_warp(const uint8_t* __restrict__ x
     if (valid && IVF_IN_BOUNDS(141, grow0 + lane, n)) xn_out[grow0 + lane] = static_cast<float>(sumsq);
 }
 
+// ---------------------------------------------------------------- thresholds finished by the main pass
+// Serving-size batches (at most kFoldRows rows): every CTA of the main pass derives the rows'
+// thresholds from the partial sketches of the threshold pass itself, one epilogue warp per row
+// (two rows per warp at most), while its first tiles are computed -- no launch in between.
+constexpr int kFoldRows = 2 * kNumEpiWarps;
+
+// a, b ascending: a becomes the 16 smallest of the 32 values, ascending.  min(a[i], b[15 - i]) are
+// those 16 values as a bitonic sequence, which four half-cleaner stages sort.
+__device__ __forceinline__ void merge16_sorted(float (&a)[kSampleM], const float (&b)[kSampleM]) {
+    static_assert(kSampleM == 16, "network below is written for 16");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) a[i] = fminf(a[i], b[15 - i]);
+#pragma unroll
+    for (int stride = 8; stride > 0; stride >>= 1) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            if ((i & stride) == 0) {
+                const float lo = fminf(a[i], a[i + stride]), hi = fmaxf(a[i], a[i + stride]);
+                a[i] = lo;
+                a[i + stride] = hi;
+            }
+        }
+    }
+}
+
+// The 16th smallest of the values in `slots` ascending 16-entry lists (value i of list s at
+// base[i * pitch + s], so that a warp's loads are contiguous), computed by one warp; every lane
+// returns it.
+__device__ __forceinline__ float warp_threshold_of_sketches(const float* base, int slots, int pitch, int lane) {
+    const float INF = __int_as_float(0x7f800000);
+    float a[kSampleM];
+#pragma unroll
+    for (int i = 0; i < kSampleM; ++i) a[i] = INF;
+    // five lists per lane and memory round trip (the warp is alone on its scheduler half the time and
+    // the loads' latency, not their number, is what the batch waits for)
+    constexpr int kLists = 5;
+    for (int s0 = lane; s0 < slots; s0 += 32 * kLists) {
+        float v[kLists][kSampleM];
+#pragma unroll
+        for (int u = 0; u < kLists; ++u) {
+            const int s = s0 + 32 * u;
+#pragma unroll
+            for (int i = 0; i < kSampleM; ++i) v[u][i] = s < slots ? base[static_cast<size_t>(i) * pitch + s] : INF;
+        }
+#pragma unroll
+        for (int u = 0; u < kLists; ++u) merge16_sorted(a, v[u]);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        float b[kSampleM];
+#pragma unroll
+        for (int i = 0; i < kSampleM; ++i) b[i] = __shfl_xor_sync(0xFFFFFFFFu, a[i], off);
+        merge16_sorted(a, b);
+    }
+    return a[kSampleM - 1];
+}
+
 template <int EPI, int MT>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_xa,
@@ -919,6 +983,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         int it = 0;
         [[maybe_unused]] int xseg = 0;  // row groups whose threshold this CTA has finished
         bool ok = true;
+        [[maybe_unused]] const float* tau_fold = nullptr;
         for (int64_t u = u0; u < u1 && ok;) {
             const int64_t r = u / NT;  // row group
             const int t0 = static_cast<int>(u - r * NT);
@@ -935,6 +1000,21 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's reads
                 __syncwarp();
                 if (lane == 0) mbar_arrive(a_full);
+            }
+            if constexpr (EPI == EPI_GROUPS) {
+                if (p.sketch_t != nullptr && tau_fold == nullptr) {
+                    // (after the point tile is handed to the MMA warp, so that the first tiles are
+                    // computed meanwhile.)  Epilogue warp w finishes the thresholds of rows w, w + 8, ...:
+                    // the batch has at most kFoldRows rows
+                    float* ts = reinterpret_cast<float*>(hist_all);
+                    for (int e = warp - 2; e < p.n; e += kNumEpiWarps) {
+                        const float t = warp_threshold_of_sketches(p.sketch_t + static_cast<size_t>(e) * kSampleM * p.sketch_pitch,
+                                                                   p.sketch_slots, p.sketch_pitch, lane);
+                        if (lane == 0) ts[e] = t;
+                    }
+                    asm volatile("bar.sync 2, %0;" ::"n"(kNumEpiWarps * 32) : "memory");  // the epilogue warps only
+                    tau_fold = ts;
+                }
             }
 
             RowState<EPI> st[MT];
@@ -961,7 +1041,7 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                     st[h].wp = st[h].base;
                     st[h].limit = st[h].base + static_cast<size_t>(p.cap - kGroupLogMargin) * kRecordBytes;
                     st[h].overflow = 0;
-                    if (valid[h]) st[h].tau = p.tau_in[row[h]];
+                    if (valid[h]) st[h].tau = tau_fold != nullptr ? tau_fold[row[h]] : p.tau_in[row[h]];
                 }
             }
 
@@ -1129,10 +1209,19 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                         p.part[at] = e;
                     } else if constexpr (EPI == EPI_SKETCH) {
                         // the partial result of the threshold pass: the thread's 16 smallest group minima
-                        Entry* log = p.part + at * p.cap;
+                        if (p.sketch_t != nullptr) {
+                            // (a batch of a few rows, read back by the main pass with slot = lane)
+                            if (IVF_IN_BOUNDS(146, slot, p.sketch_pitch)) {
+                                float* out = p.sketch_t + static_cast<size_t>(row[h]) * kSampleM * p.sketch_pitch + slot;
 #pragma unroll
-                        for (int i = 0; i < kSampleM; ++i)
-                            *reinterpret_cast<uint2*>(&log[i]) = make_uint2(__float_as_uint(st[h].net[i]), 0u);
+                                for (int i = 0; i < kSampleM; ++i) out[static_cast<size_t>(i) * p.sketch_pitch] = st[h].net[i];
+                            }
+                        } else {
+                            Entry* log = p.part + at * p.cap;
+#pragma unroll
+                            for (int i = 0; i < kSampleM; ++i)
+                                *reinterpret_cast<uint2*>(&log[i]) = make_uint2(__float_as_uint(st[h].net[i]), 0u);
+                        }
                         p.part_meta[at] = make_int2(kSampleM, __float_as_int(INF));
                     } else if constexpr (EPI == EPI_GROUPS) {
                         const int recs = static_cast<int>((st[h].wp - st[h].base) / kRecordBytes);

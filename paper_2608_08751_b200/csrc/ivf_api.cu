@@ -129,7 +129,7 @@ void timing_end(int idx, cudaStream_t stream) {
 
 // ------------------------------------------------------------------ workspace
 enum WsSlot {
-    WS_X16, WS_C16, WS_XN, WS_SCAL, WS_BITS, WS_PART, WS_PARTMETA, WS_FAIL, WS_FBKEYS, WS_TAU,
+    WS_X16, WS_C16, WS_XN, WS_SCAL, WS_BITS, WS_PART, WS_PARTMETA, WS_FAIL, WS_FBKEYS, WS_TAU, WS_SKETCH,
     WS_UCNT, WS_UOFF, WS_UCUR, WS_UPERM, WS_IDS, WS_CHUNK0, WS_CHUNK1, WS_PQ_CHUNKS, WS_PQ_GCAND, WS_PQ_GCOUNT, WS_PQ_CBT, WS_UPARTS, WS_NUM
 };
 struct Buf {
@@ -258,6 +258,7 @@ int choose_rule(int k, int nlist, int* stride) {
 }
 
 int g_sketch_whole = 1;  // test hook (ivf_debug_set_threshold_pass): 0 = the threshold pass always as sketch kernel + merge
+int g_tau_fold = 1;      // same hook: 0 = thresholds of tiny batches by the merge kernel, not inside the main pass
 int g_rotate = 1;  // test hook (ivf_debug_set_rotation): 0 = every position of a sweep stands for its own tile index
 int g_cross = -1;  // crossing cost used by the span partition; -1 = by kernel variant (test hook: ivf_debug_set_crossing_cost)
 
@@ -456,8 +457,12 @@ struct PointPrep {
 int launch_fused(DeviceCtx& ctx, const Plan& pl, int64_t n, int nlist, int k, int rule, const float* tau_in,
                  const PointPrep& pp, const CUtensorMap& tmap_c, const CUtensorMap& tmap_ca, Entry* part,
                  int2* part_meta, int kind, cudaStream_t stream, const unsigned int* bits, float* scal,
-                 int* clear0 = nullptr, int* clear1 = nullptr, int* clear32 = nullptr, float* tau_out = nullptr) {
+                 int* clear0 = nullptr, int* clear1 = nullptr, int* clear32 = nullptr, float* tau_out = nullptr,
+                 float* sketch_t = nullptr, int sketch_pitch = 0, int sketch_slots = 0) {
     FusedParams fp;
+    fp.sketch_t = sketch_t;
+    fp.sketch_pitch = sketch_pitch;
+    fp.sketch_slots = sketch_slots;
     fp.clear0 = clear0;
     fp.clear1 = clear1;
     fp.clear32 = clear32;
@@ -580,6 +585,9 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         part_bytes = pb > part_bytes ? pb : part_bytes;
         meta_bytes = mb > meta_bytes ? mb : meta_bytes;
     }
+    // Batches of a few rows: the main pass finishes the thresholds from the partial sketches itself (one
+    // epilogue warp per row, while the first tiles load), so no merge kernel runs between the two passes.
+    const bool tau_fold = given && !sketch_whole && g_tau_fold && n <= kFoldRows;
     PointPrep pp;
     Entry* part;
     int2* part_meta = nullptr;
@@ -637,17 +645,28 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         pp.tmap_xa = cp.tmap_ca;
     }
 
+    float* fold_sketch = nullptr;
+    int fold_slots = 0;
     if (given) {
         // threshold pass over every S-th centroid: the 16th smallest group minimum becomes the row's tau
+        // (batches of at most kFoldRows rows: the sketches go to a buffer of their own, slot-minor, because
+        // the main pass, which finishes the thresholds itself, reads them while it fills `part`)
+        float* sketch_t = nullptr;
+        if (tau_fold) WS(WS_SKETCH, static_cast<size_t>(n) * kSampleM * pls.partials * sizeof(float), sketch_t);
         rc = launch_fused(ctx, pls, n, cp.sample_rows, kSampleM, TAU_SKETCH, nullptr, pp, cp.tmap_cs, cp.tmap_csa, part,
                           part_meta, TK_THRESH, stream, cp.bits, cp.scal, nullptr, nullptr, nullptr,
-                          sketch_whole ? tau : nullptr);
+                          sketch_whole ? tau : nullptr, sketch_t, pls.partials, 0);
         if (rc != IVF_OK) return rc;
         MergeParams ms = merge_params(pls, n, kSampleM, part, part_meta, pp, cp.scal);
         ms.tau_out = tau;
         tk = timing_begin(TK_THRESH, stream);
         if (sketch_whole) {
             // the kernel wrote the thresholds itself
+        } else if (tau_fold) {
+            // the main pass finishes them
+            fold_sketch = sketch_t;
+            fold_slots = (cta_of_unit(pls.total_units, pls.ctas, pls.col_tiles, pls.cross, pls.col_tiles - 1) -
+                          cta_of_unit(pls.total_units, pls.ctas, pls.col_tiles, pls.cross, 0) + 1) * kEpiHalves;
         } else if (pls.partials <= 32)
             LAUNCH_DEP(4, merge_tau_warp_kernel, static_cast<unsigned>((n * 32 + 255) / 256), 256, 0, stream, ms);
         else {
@@ -661,7 +680,8 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     }
     rc = launch_fused(ctx, pl, n, nlist, k, cp.rule, tau, pp, cp.tmap_c, cp.tmap_ca, part, part_meta,
                       k == 1 ? TK_FUSED_ARGMIN : TK_FUSED_TOPK, stream, cp.bits, cp.scal, failbuf,
-                      failbuf ? failbuf + n + 2 : nullptr, failbuf ? failbuf + 2 * (n + 2) : nullptr);
+                      failbuf ? failbuf + n + 2 : nullptr, failbuf ? failbuf + 2 * (n + 2) : nullptr, nullptr,
+                      fold_sketch, pls.partials, fold_slots);
     if (rc != IVF_OK) return rc;
 
     MergeParams mp = merge_params(pl, n, k, part, part_meta, pp, cp.scal);
@@ -1480,6 +1500,7 @@ int ivf_debug_set_dependent_launch(int on) {
 
 int ivf_debug_set_threshold_pass(int split) {
     g_sketch_whole = split ? 0 : 1;
+    g_tau_fold = split ? 0 : 1;
     return IVF_OK;
 }
 
