@@ -501,60 +501,11 @@ __device__ __forceinline__ void consume(uint32_t (&acc)[32], int jbase, RowState
     }
 }
 
-// One thread widens one uint8 point row into the fp16 operand tile in shared memory: 16-byte
-// chunks of 8 values at the positions the 128-byte swizzle (data) and the 32-byte swizzle (norm
-// columns) give them, exactly as a TMA load of the fp16 copy would have placed them.  Returns |x|^2.
-__device__ __forceinline__ unsigned int widen_row_u8(const uint8_t* __restrict__ src, bool valid, int d, int kd,
-                                                     uint8_t* tile, int a_data_bytes, int row, float sx, float A) {
-    const __half2 k1024 = __floats2half2_rn(1024.0f, 1024.0f);
-    const __half2 sx2 = __floats2half2_rn(sx, sx);
-    // two bytes -> two fp16: 0x6400 | b is the half 1024 + b; subtract 1024, scale (all exact)
-    auto cvt2 = [&](uint32_t w, uint32_t sel) {
-        uint32_t q = __byte_perm(w, 0x64646464u, sel);
-        const __half2 t2 = __hmul2(__hsub2(*reinterpret_cast<__half2*>(&q), k1024), sx2);
-        return *reinterpret_cast<const uint32_t*>(&t2);
-    };
-    unsigned int sumsq = 0;
-#pragma unroll 1
-    for (int c0 = 0; c0 < kd / 8; c0 += 16) {  // 16 chunks (128 columns) in flight
-        uint2 w[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int c = c0 + i;
-            w[i] = make_uint2(0u, 0u);
-            if (valid && c * 8 < d) w[i] = *reinterpret_cast<const uint2*>(src + c * 8);
-        }
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int c = c0 + i;
-            if (c < kd / 8) {
-                sumsq = __dp4a(w[i].x, w[i].x, sumsq);
-                sumsq = __dp4a(w[i].y, w[i].y, sumsq);
-                uint4 o;
-                o.x = cvt2(w[i].x, 0x5140u);
-                o.y = cvt2(w[i].x, 0x5342u);
-                o.z = cvt2(w[i].y, 0x5140u);
-                o.w = cvt2(w[i].y, 0x5342u);
-                const int slice = c >> 3, j = c & 7;  // chunk j of the row goes to position j ^ (row % 8)
-                const int toff = slice * kBlockM * kSliceRowBytes + row * kSliceRowBytes + ((j ^ (row & 7)) << 4);
-                if (IVF_IN_BOUNDS(110, toff, a_data_bytes - 15)) *reinterpret_cast<uint4*>(tile + toff) = o;
-            }
-        }
-    }
-    // norm columns: A A A 0 ... 0; chunk j of the row goes to position j ^ ((row / 4) % 2)
-    const uint32_t a16 = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(A)));
-    const uint4 aug0 = valid ? make_uint4(a16 | (a16 << 16), a16, 0u, 0u) : make_uint4(0u, 0u, 0u, 0u);
-    const int sw = (row >> 2) & 1;
-    if (IVF_IN_BOUNDS(111, row, kBlockM)) {
-        *reinterpret_cast<uint4*>(tile + a_data_bytes + row * kAugRowBytes + ((0 ^ sw) << 4)) = aug0;
-        *reinterpret_cast<uint4*>(tile + a_data_bytes + row * kAugRowBytes + ((1 ^ sw) << 4)) = make_uint4(0u, 0u, 0u, 0u);
-    }
-    return sumsq;
-}
-
-// The same for the 32 consecutive rows of one TMEM lane quadrant, by one warp with coalesced loads:
-// the rows are contiguous in memory, so lane l of step s takes the 16-byte chunk number 32 s + l of the
-// quadrant's 32 * d bytes (four steps in flight).  A chunk of 16 values becomes two 16-byte chunks of
+// One warp widens the 32 consecutive uint8 point rows of one TMEM lane quadrant into the fp16 operand
+// tile in shared memory, with coalesced loads: 16-byte chunks of 8 values go to the positions the
+// 128-byte swizzle (data) and the 32-byte swizzle (norm columns) give them, exactly as a TMA load of
+// an fp16 copy would have placed them.  The rows are contiguous in memory, so lane l of step s takes
+// the 16-byte chunk number 32 s + l of the quadrant's 32 * d bytes (four steps in flight).  A chunk of 16 values becomes two 16-byte chunks of
 // the operand row, written where the swizzles put them.  The squares are summed per chunk and brought
 // to the lane that owns the row (lane = row within the quadrant), which also writes the norm columns
 // and |x|^2.  Rows at or beyond `n` become zero rows.

@@ -34,25 +34,10 @@ constexpr int kPqMaxRerank = 1024;
 constexpr int kPqMaxProbes = 512;   // lists per query (the paper sweeps the probe count up to 512)
 constexpr int kPqStatusBadId = -6;
 
-// shared memory of the encode kernel: the transposed codebook, one lookup table, one residual
+// the stated bound on the encoder's shared memory (codebook, one lookup table, one residual); the
+// kernel itself asks for pq_encode_smem_bytes
 __host__ __device__ inline size_t pq_smem_bytes(int d, int pq_m) {
     return static_cast<size_t>(d) * kPqK * 4 + static_cast<size_t>(pq_m) * kPqK * 4 + static_cast<size_t>(d) * 4;
-}
-
-struct PqSmem {
-    float* cbt;  // [d][256]: coordinate-major codebook
-    float* lut;  // [pq_m][256]
-    float* r;    // [d]
-};
-
-__device__ __forceinline__ PqSmem pq_carve(uint8_t* raw, int d, int pq_m) {
-    PqSmem s;
-    s.cbt = reinterpret_cast<float*>(raw);
-    raw += static_cast<size_t>(d) * kPqK * 4;
-    s.lut = reinterpret_cast<float*>(raw);
-    raw += static_cast<size_t>(pq_m) * kPqK * 4;
-    s.r = reinterpret_cast<float*>(raw);
-    return s;
 }
 
 // A thread group: NT threads numbered tid that synchronise on hardware barrier BAR (BAR = 0 with
@@ -61,18 +46,6 @@ template <int BAR, int NT>
 __device__ __forceinline__ void pq_group_sync() {
     if constexpr (BAR == 0) __syncthreads();
     else asm volatile("bar.sync %0, %1;" ::"n"(BAR), "n"(NT) : "memory");
-}
-
-// codebooks [pq_m][256][dsub] in global memory -> cbt[(m * dsub + t) * 256 + j]
-__device__ __forceinline__ void pq_load_codebooks(const float* __restrict__ codebooks, int d, int dsub, float* cbt) {
-    const int total = d * kPqK;
-    for (int i = threadIdx.x; i < total; i += blockDim.x) {
-        // i walks the global layout: i = (m * 256 + j) * dsub + t
-        const int t = i % dsub;
-        const int mj = i / dsub;
-        const int j = mj & (kPqK - 1), m = mj >> 8;
-        cbt[(m * dsub + t) * kPqK + j] = codebooks[i];
-    }
 }
 
 // Lookup-table build.  Thread -> codeword j = tid & 255; the 256-thread slices of the CTA take
