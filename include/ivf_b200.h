@@ -76,10 +76,30 @@ typedef enum {
  *   out_ids    [nq, nprobe] int32, device: the nprobe nearest centroids of every query, ascending
  *              by (distance, id) -- equal distances are ordered by the lower id
  *   out_dists  [nq, nprobe] float32 squared L2 distances (clamped at 0), device; may be NULL
+ * Results in host memory (Sec. 4.1: what leaves the GPU is the O(B * P) list of selected lists, which
+ * the CPU-side search consumes): out_ids and out_dists may instead both be page-locked host memory.
+ * The kernels then write to staging buffers of the workspace and every row chunk is copied to the
+ * host on a stream of the library's own, under the next chunk's kernels; before the call returns it
+ * makes `stream` wait for the last copy, so in `stream` the call is complete when its results are in
+ * host memory -- ordinary stream semantics.  The same holds for ivf_route_prepared, ivf_assign and
+ * ivf_assign_update.  Pageable host memory -> IVF_ERR_INVALID_ARG.
  */
 int ivf_route(const void* queries, int64_t nq, int d, ivf_dtype qtype,
               const float* centroids, int nlist, int nprobe,
               int32_t* out_ids, float* out_dists, void* stream);
+
+/*
+ * Deferred read-back, for a serving loop that routes batch i + 1 while batch i's results travel to
+ * the host.  ivf_set_deferred_host_outputs(1) (per device; default 0): calls with host outputs no
+ * longer make `stream` wait for their read-back, so the next call's kernels start at once (two
+ * staging buffer pairs are used in turn; a pair is reused only after its read-back).  Read-backs
+ * finish in the order of the calls.  The host buffers of a call may be read after
+ * ivf_wait_host_outputs(stream) -- it makes `stream` wait for every read-back issued so far on the
+ * current device -- followed by whatever the caller uses to wait for `stream`, or after
+ * ivf_check(stream), which waits for them on the host.
+ */
+int ivf_set_deferred_host_outputs(int on);
+int ivf_wait_host_outputs(void* stream);
 
 /*
  * Routing against a centroid table that stays resident on the device (Sec. 3.1 / 4.1: the centroid

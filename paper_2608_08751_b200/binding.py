@@ -24,6 +24,7 @@ EXPORTS = (
     "ivf_assign_update", "ivf_cluster_major_reorder", "ivf_centroids_create", "ivf_centroids_destroy",
     "ivf_route_prepared",
     "ivf_pq_encode", "ivf_pq_search", "ivf_pq_residuals", "ivf_assign_candidates", "ivf_merge_shards",
+    "ivf_set_deferred_host_outputs", "ivf_wait_host_outputs",
     "ivf_check", "ivf_last_error", "ivf_release_workspace", "ivf_launch_count",
     "ivf_debug_plan", "ivf_debug_span", "ivf_debug_rotation", "ivf_debug_set_rotation", "ivf_debug_set_threshold_pass", "ivf_debug_fail_next_alloc", "ivf_debug_bounds_checked", "ivf_debug_bounds_probe", "ivf_debug_set_wait_limit_ns",
     "ivf_debug_timing", "ivf_debug_timing_read", "ivf_debug_wait_probe", "ivf_debug_force_fallback", "ivf_debug_rule", "ivf_debug_set_row_chunk", "ivf_debug_stats", "ivf_debug_set_pq_groups", "ivf_debug_set_dependent_launch", "ivf_debug_set_crossing_cost",
@@ -56,6 +57,8 @@ def lib() -> ctypes.CDLL:
     vp, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
     L.ivf_route.argtypes = [vp, i64, i32, i32, vp, i32, i32, vp, vp, vp]
     L.ivf_assign.argtypes = [vp, i64, i32, i32, vp, i32, vp, vp, vp]
+    L.ivf_set_deferred_host_outputs.argtypes = [i32]
+    L.ivf_wait_host_outputs.argtypes = [vp]
     L.ivf_centroid_update.argtypes = [vp, i32, vp, i64, i32, i32, vp, vp, vp]
     L.ivf_centroid_update_noalloc.argtypes = [vp, i32, vp, i64, i32, i32, vp, vp, vp]
     L.ivf_centroid_finalize.argtypes = [vp, vp, i32, i32, vp, vp]
@@ -123,6 +126,13 @@ def _dev(t: torch.Tensor, name: str, dtype: torch.dtype) -> torch.Tensor:
     return t
 
 
+def _out(t: torch.Tensor, name: str, dtype: torch.dtype) -> torch.Tensor:
+    """An output array: a contiguous CUDA tensor, or a pinned CPU tensor (results read back by the library)."""
+    if not (t.is_cuda or t.is_pinned()) or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA or pinned CPU tensor of {dtype}")
+    return t
+
+
 def _stream(device) -> int:
     return torch.cuda.current_stream(device).cuda_stream
 
@@ -147,8 +157,8 @@ def ivf_route(queries: torch.Tensor, centroids: torch.Tensor, nprobe: int,
         out_dists = torch.empty((nq, nprobe), dtype=torch.float32, device=dev)
     with torch.cuda.device(dev):
         rc = lib().ivf_route(_ptr(queries), nq, d, _dtype_code(queries), _ptr(centroids), nlist, nprobe,
-                             _ptr(_dev(out_ids, "out_ids", torch.int32)),
-                             _ptr(out_dists), _stream(dev))
+                             _ptr(_out(out_ids, "out_ids", torch.int32)),
+                             _ptr(None if out_dists is None else _out(out_dists, "out_dists", torch.float32)), _stream(dev))
     if rc != IVF_OK:
         _raise(rc)
     return out_ids, out_dists
@@ -196,7 +206,9 @@ def ivf_route_prepared(handle: PreparedCentroids, queries: torch.Tensor, nprobe:
         out_dists = torch.empty((nq, nprobe), dtype=torch.float32, device=dev)
     with torch.cuda.device(dev):
         rc = lib().ivf_route_prepared(handle._h, _ptr(queries), nq, _dtype_code(queries), nprobe,
-                                      _ptr(_dev(out_ids, "out_ids", torch.int32)), _ptr(out_dists), _stream(dev))
+                                      _ptr(_out(out_ids, "out_ids", torch.int32)),
+                                      _ptr(None if out_dists is None else _out(out_dists, "out_dists", torch.float32)),
+                                      _stream(dev))
     if rc != IVF_OK:
         _raise(rc)
     return out_ids, out_dists
@@ -216,10 +228,28 @@ def ivf_assign(points: torch.Tensor, centroids: torch.Tensor,
         out_dists = torch.empty((n,), dtype=torch.float32, device=dev)
     with torch.cuda.device(dev):
         rc = lib().ivf_assign(_ptr(points), n, d, _dtype_code(points), _ptr(centroids), centroids.shape[0],
-                              _ptr(_dev(out_ids, "out_ids", torch.int32)), _ptr(out_dists), _stream(dev))
+                              _ptr(_out(out_ids, "out_ids", torch.int32)),
+                              _ptr(None if out_dists is None else _out(out_dists, "out_dists", torch.float32)), _stream(dev))
     if rc != IVF_OK:
         _raise(rc)
     return out_ids, out_dists
+
+
+def ivf_set_deferred_host_outputs(on: bool, device=None) -> None:
+    """Calls with pinned-host outputs stop making the stream wait for their read-back (per device)."""
+    with torch.cuda.device(device if device is not None else torch.cuda.current_device()):
+        rc = lib().ivf_set_deferred_host_outputs(1 if on else 0)
+    if rc != IVF_OK:
+        _raise(rc)
+
+
+def ivf_wait_host_outputs(device=None) -> None:
+    """Makes the current stream wait for every read-back issued so far on the device."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    with torch.cuda.device(dev):
+        rc = lib().ivf_wait_host_outputs(_stream(dev))
+    if rc != IVF_OK:
+        _raise(rc)
 
 
 def ivf_centroid_update(points: torch.Tensor, ids: torch.Tensor, sums: torch.Tensor, counts: torch.Tensor):
@@ -430,9 +460,9 @@ def ivf_assign_update(points: torch.Tensor, centroids: torch.Tensor, sums: torch
     n, d = points.shape
     dev = centroids.device
     if out_ids is not None:
-        _dev(out_ids, "out_ids", torch.int32)
+        _out(out_ids, "out_ids", torch.int32)
     if out_dists is not None:
-        _dev(out_dists, "out_dists", torch.float32)
+        _out(out_dists, "out_dists", torch.float32)
     with torch.cuda.device(dev):
         rc = lib().ivf_assign_update(_ptr(points), n, d, _dtype_code(points), _ptr(centroids), centroids.shape[0],
                                      _ptr(out_ids), _ptr(out_dists), _ptr(sums), _ptr(counts), chunk_rows,

@@ -129,7 +129,7 @@ void timing_end(int idx, cudaStream_t stream) {
 
 // ------------------------------------------------------------------ workspace
 enum WsSlot {
-    WS_X16, WS_C16, WS_XN, WS_SCAL, WS_BITS, WS_PART, WS_PARTMETA, WS_FAIL, WS_FBKEYS, WS_TAU, WS_SKETCH,
+    WS_X16, WS_C16, WS_XN, WS_SCAL, WS_BITS, WS_PART, WS_PARTMETA, WS_FAIL, WS_FBKEYS, WS_TAU, WS_SKETCH, WS_OUT_IDS0, WS_OUT_IDS1, WS_OUT_DISTS0, WS_OUT_DISTS1,
     WS_UCNT, WS_UOFF, WS_UCUR, WS_UPERM, WS_IDS, WS_CHUNK0, WS_CHUNK1, WS_PQ_CHUNKS, WS_PQ_GCAND, WS_PQ_GCOUNT, WS_PQ_CBT, WS_UPARTS, WS_NUM
 };
 struct Buf {
@@ -146,6 +146,14 @@ struct DeviceCtx {
     cudaEvent_t ev_copied[2] = {nullptr, nullptr};
     cudaEvent_t ev_free[2] = {nullptr, nullptr};
     cudaEvent_t ev_ready = nullptr;
+    // results read back to page-locked host memory: a stream of its own (the host link carries both
+    // directions at once), two staging buffer pairs used in turn
+    cudaStream_t out_stream = nullptr;
+    cudaEvent_t ev_out_ready[2] = {nullptr, nullptr};  // the kernels that fill staging pair i are done
+    cudaEvent_t ev_out_done[2] = {nullptr, nullptr};   // the read-back of staging pair i is done
+    bool out_used[2] = {false, false};
+    unsigned out_seq = 0;
+    bool defer_outputs = false;  // ivf_set_deferred_host_outputs
     bool smem_attr_set = false;
     bool merge_attr_set = false;
     bool pq_attr_set = false;
@@ -176,6 +184,11 @@ int get_ctx(DeviceCtx** out) {
             CUDA_TRY(cudaEventCreateWithFlags(&c.ev_free[i], cudaEventDisableTiming));
         }
         CUDA_TRY(cudaEventCreateWithFlags(&c.ev_ready, cudaEventDisableTiming));
+        CUDA_TRY(cudaStreamCreateWithFlags(&c.out_stream, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+            CUDA_TRY(cudaEventCreateWithFlags(&c.ev_out_ready[i], cudaEventDisableTiming));
+            CUDA_TRY(cudaEventCreateWithFlags(&c.ev_out_done[i], cudaEventDisableTiming));
+        }
 #ifdef IVF_CHECK_BOUNDS
         // checked build: the kernels' index checks report into this device's status word
         CUDA_TRY(cudaMemcpyToSymbol(g_check_status, &c.status, sizeof(int*)));
@@ -847,6 +860,23 @@ int run_chunks(const void* points, int64_t n, int d, int ptype, const float* cen
     if (where < 0) return where;
     const bool host = where == 1;
     const size_t esize = dtype_size(ptype);
+    // results: device memory, or page-locked host memory (both arrays of the same kind)
+    bool out_host = false;
+    if (out_ids) {
+        const int ow = classify_pointer(out_ids);
+        if (ow < 0) return ow;
+        out_host = ow == 1;
+        if (out_dists) {
+            const int dw = classify_pointer(out_dists);
+            if (dw < 0) return dw;
+            if ((dw == 1) != out_host)
+                return fail(IVF_ERR_INVALID_ARG, "out_ids and out_dists must both be device memory or both page-locked host memory");
+        }
+    } else if (out_dists) {
+        const int dw = classify_pointer(out_dists);
+        if (dw < 0) return dw;
+        if (dw == 1) return fail(IVF_ERR_INVALID_ARG, "out_dists in host memory needs out_ids in host memory as well");
+    }
 
     int64_t rows = rows_per_launch(d, k);
     if (g_row_chunk_override.load() > 0) rows = g_row_chunk_override.load();
@@ -874,6 +904,24 @@ int run_chunks(const void* points, int64_t n, int d, int ptype, const float* cen
         CUDA_TRY(cudaStreamWaitEvent(ctx.copy_stream, ctx.ev_ready, 0));
     }
     if (with_update && !out_ids) WS(WS_IDS, static_cast<size_t>(rows) * sizeof(int32_t), tmp_ids);
+    int32_t* ostage_ids[2] = {nullptr, nullptr};
+    float* ostage_dists[2] = {nullptr, nullptr};
+    if (out_host) {
+        const size_t ob = static_cast<size_t>(rows) * k * sizeof(int32_t);
+        // a staging buffer about to grow is freed in `stream` order: no read-back may still be reading it
+        if (ctx.bufs[WS_OUT_IDS0].cap < ob || ctx.bufs[WS_OUT_IDS1].cap < ob ||
+            (out_dists && (ctx.bufs[WS_OUT_DISTS0].cap < ob || ctx.bufs[WS_OUT_DISTS1].cap < ob))) {
+            for (int i = 0; i < 2; ++i)
+                if (ctx.out_used[i]) CUDA_TRY(cudaStreamWaitEvent(stream, ctx.ev_out_done[i], 0));
+        }
+        WS(WS_OUT_IDS0, ob, ostage_ids[0]);
+        WS(WS_OUT_IDS1, ob, ostage_ids[1]);
+        if (out_dists) {
+            WS(WS_OUT_DISTS0, ob, ostage_dists[0]);
+            WS(WS_OUT_DISTS1, ob, ostage_dists[1]);
+        }
+    }
+    int last_out = -1;
 
     auto issue_copy = [&](int64_t c) -> int {
         const int64_t r0 = c * rows;
@@ -918,14 +966,36 @@ int run_chunks(const void* points, int64_t n, int d, int ptype, const float* cen
         }
         int32_t* ids_c = out_ids ? out_ids + r0 * k : tmp_ids;
         float* dists_c = out_dists ? out_dists + r0 * k : nullptr;
+        int so = 0;
+        if (out_host) {
+            // this chunk's results go to a staging pair; the pair's previous read-back must be over
+            so = static_cast<int>(ctx.out_seq++ & 1u);
+            if (ctx.out_used[so]) CUDA_TRY(cudaStreamWaitEvent(stream, ctx.ev_out_done[so], 0));
+            ids_c = ostage_ids[so];
+            dists_c = out_dists ? ostage_dists[so] : nullptr;
+        }
         rc = route_rows_device(ctx, chunk, nr, d, ptype, nlist, k, cp, ids_c, dists_c, stream);
         if (rc != IVF_OK) return rc;
+        if (out_host) {
+            // read-back on its own stream, under the next chunk's (or the next call's) kernels
+            const size_t nb = static_cast<size_t>(nr) * k * sizeof(int32_t);
+            CUDA_TRY(cudaEventRecord(ctx.ev_out_ready[so], stream));
+            CUDA_TRY(cudaStreamWaitEvent(ctx.out_stream, ctx.ev_out_ready[so], 0));
+            CUDA_TRY(cudaMemcpyAsync(out_ids + r0 * k, ids_c, nb, cudaMemcpyDeviceToHost, ctx.out_stream));
+            if (out_dists) CUDA_TRY(cudaMemcpyAsync(out_dists + r0 * k, dists_c, nb, cudaMemcpyDeviceToHost, ctx.out_stream));
+            CUDA_TRY(cudaEventRecord(ctx.ev_out_done[so], ctx.out_stream));
+            ctx.out_used[so] = true;
+            last_out = so;
+        }
         if (with_update) {
             rc = update_device(ctx, chunk, ptype, ids_c, nr, d, nlist, sums, counts, stream);
             if (rc != IVF_OK) return rc;
         }
         if (host) CUDA_TRY(cudaEventRecord(ctx.ev_free[sb], stream));
     }
+    // plain stream semantics unless the caller asked otherwise: the call is complete in `stream` only
+    // when its results are in host memory (the read-back stream is in order, so the last event covers all)
+    if (last_out >= 0 && !ctx.defer_outputs) CUDA_TRY(cudaStreamWaitEvent(stream, ctx.ev_out_done[last_out], 0));
     return IVF_OK;
 }
 
@@ -1358,6 +1428,7 @@ int ivf_check(void* stream) {
     int rc = get_ctx(&ctx);
     if (rc != IVF_OK) return rc;
     CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    if (ctx->out_used[0] || ctx->out_used[1]) CUDA_TRY(cudaStreamSynchronize(ctx->out_stream));  // deferred read-backs
     int h[4] = {0, 0, 0, 0};
     CUDA_TRY(cudaMemcpy(h, ctx->status, sizeof h, cudaMemcpyDeviceToHost));
     if (h[0] != 0) {
@@ -1369,6 +1440,24 @@ int ivf_check(void* stream) {
             return fail(IVF_ERR_BOUNDS, "an index check of the checked build failed (site %d, block %d, index %d)", h[1], h[2], h[3]);
         return fail(h[0], "device status %d", h[0]);
     }
+    return IVF_OK;
+}
+
+int ivf_set_deferred_host_outputs(int on) {
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != IVF_OK) return rc;
+    ctx->defer_outputs = on != 0;
+    return IVF_OK;
+}
+
+int ivf_wait_host_outputs(void* stream) {
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != IVF_OK) return rc;
+    // the read-back stream is in order: the younger of the two events covers every read-back issued
+    for (int i = 0; i < 2; ++i)
+        if (ctx->out_used[i]) CUDA_TRY(cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), ctx->ev_out_done[i], 0));
     return IVF_OK;
 }
 

@@ -451,6 +451,95 @@ def test_assign_update_streamed_in_chunks(host):
     assert (counts2 == counts).all() and (sums2 == sums).all()
 
 
+def _pinned(shape, dtype, fill):
+    t = torch.full(shape, fill, dtype=dtype).pin_memory()
+    return t
+
+
+@pytest.mark.parametrize("host_in", [False, True])
+@pytest.mark.parametrize("k,with_dists", [(1, True), (8, True), (40, False)])
+def test_results_in_pinned_host_memory(host_in, k, with_dists):
+    # the kernels write to staging buffers of the workspace; every row chunk is read back on the
+    # library's own stream and the caller's stream waits for the last copy before the call counts as done
+    n, nlist, d = 7000, 3000, 64
+    x, c = _rand(n, nlist, d, "f32", 77)
+    want_ids, want_d = _route(x, c, k)
+    xt = torch.from_numpy(x).pin_memory() if host_in else _cuda(x)
+    shape = (n,) if k == 1 else (n, k)
+    ids_h = _pinned(shape, torch.int32, -7)
+    d_h = _pinned(shape, torch.float32, -7.0) if with_dists else None
+    B.ivf_debug_set_row_chunk(1536)  # five chunks with a ragged tail: both staging pairs are reused
+    try:
+        if k == 1:
+            B.ivf_assign(xt, _cuda(c), ids_h, d_h, want_dists=with_dists)
+        else:
+            B.ivf_route(xt, _cuda(c), k, ids_h, d_h, want_dists=with_dists)
+        torch.cuda.current_stream().synchronize()  # no ivf_check here: the stream alone must cover the read-back
+    finally:
+        B.ivf_debug_set_row_chunk(0)
+    assert (ids_h.numpy() == want_ids).all()
+    if with_dists:
+        assert (d_h.numpy() == want_d).all()
+    B.ivf_check()
+
+
+def test_deferred_read_back_of_host_results():
+    # serving loop: with deferred read-back the calls do not wait for their copies; two staging pairs
+    # are used in turn, so a third call must wait for the first one's copy before it reuses the pair
+    n, nlist, d, k = 4000, 5000, 128, 32
+    c = _cuda(_rand(1, nlist, d, "u8", 5)[1])
+    batches = [_rand(n, nlist, d, "u8", 100 + i)[0] for i in range(5)]
+    want = []
+    for xb in batches:
+        ids, dd = B.ivf_route(_cuda(xb), c, k)
+        want.append((ids.cpu().numpy(), dd.cpu().numpy()))
+    hosts = [(_pinned((n, k), torch.int32, -1), _pinned((n, k), torch.float32, -1.0)) for _ in batches]
+    pinned_in = [torch.from_numpy(xb).pin_memory() for xb in batches]  # alive until the copies have run
+    B.ivf_set_deferred_host_outputs(True)
+    try:
+        for xt, (ih, dh) in zip(pinned_in, hosts):
+            B.ivf_route(xt, c, k, ih, dh)
+        B.ivf_wait_host_outputs()
+        torch.cuda.current_stream().synchronize()
+        for (wi, wd), (ih, dh) in zip(want, hosts):
+            assert (ih.numpy() == wi).all() and (dh.numpy() == wd).all()
+        # ivf_check alone waits for outstanding read-backs as well
+        ih, dh = _pinned((n, k), torch.int32, -1), _pinned((n, k), torch.float32, -1.0)
+        B.ivf_route(_cuda(batches[0]), c, k, ih, dh)
+        B.ivf_check()
+        assert (ih.numpy() == want[0][0]).all() and (dh.numpy() == want[0][1]).all()
+    finally:
+        B.ivf_set_deferred_host_outputs(False)
+
+
+def test_assign_update_with_ids_in_host_memory():
+    n, nlist, d = 9000, 300, 128
+    x = synth.sift_like_rows(3, rows=n)
+    c = synth.sift_like_centroids(nlist)
+    sums = torch.zeros((nlist, d), dtype=torch.float32, device="cuda")
+    counts = torch.zeros((nlist,), dtype=torch.int64, device="cuda")
+    ids_h = _pinned((n,), torch.int32, -1)
+    B.ivf_assign_update(torch.from_numpy(x).pin_memory(), _cuda(c), sums, counts, ids_h, None, chunk_rows=2048)
+    torch.cuda.current_stream().synchronize()
+    ids = ids_h.numpy().copy()
+    B.ivf_check()
+    want, _ = _route(x, c, 1)
+    assert (ids == want).all()
+    parity.check_update(x, ids, nlist, sums.cpu().numpy(), counts.cpu().numpy())
+
+
+def test_mixed_host_and_device_outputs_are_rejected():
+    x, c = _rand(100, 200, 64, "f32", 1)
+    ids_h = _pinned((100, 4), torch.int32, 0)
+    d_dev = torch.empty((100, 4), dtype=torch.float32, device="cuda")
+    with pytest.raises(B.IvfError) as e:
+        B.ivf_route(_cuda(x), _cuda(c), 4, ids_h, d_dev)
+    assert e.value.code == B.IVF_ERR_INVALID_ARG
+    ids_dev = torch.empty((100, 4), dtype=torch.int32, device="cuda")
+    with pytest.raises(B.IvfError):
+        B.ivf_route(_cuda(x), _cuda(c), 4, ids_dev, _pinned((100, 4), torch.float32, 0.0))
+
+
 def test_pageable_host_memory_is_rejected():
     x, c = _rand(100, 200, 64, "f32", 1)
     xt = torch.from_numpy(x)
