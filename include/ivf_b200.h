@@ -248,8 +248,9 @@ int ivf_debug_rotation(int64_t n, int nlist, int d, int k, int num_sms, int64_t 
 int ivf_debug_set_rotation(int on);
 /* Measurement / test hook: 1 makes the threshold pass of k > 16 calls always run as sketch kernel plus
  * merge launch; 0 (default) lets batches of at least 48 row tiles finish their thresholds inside the
- * sketch kernel, and batches of at most 16 rows inside the main pass (its epilogue warps merge the
- * partial sketches while the first tiles are computed).  All three give the same thresholds, hence
+ * sketch kernel, and batches of at most 16 rows (32 against tables of at least 4 x 256 centroids per
+ * SM) inside the main pass (its epilogue warps merge the partial sketches while the first tiles are
+ * computed).  All three give the same thresholds, hence
  * the same results. */
 int ivf_debug_set_threshold_pass(int split);
 int ivf_debug_set_wait_limit_ns(int64_t ns);

@@ -599,8 +599,8 @@ __device__ __forceinline__ void widen_rows_u8_warp(const uint8_t* __restrict__ x
 // ---------------------------------------------------------------- thresholds finished by the main pass
 // Serving-size batches (at most kFoldRows rows): every CTA of the main pass derives the rows'
 // thresholds from the partial sketches of the threshold pass itself, one epilogue warp per row
-// (two rows per warp at most), while its first tiles are computed -- no launch in between.
-constexpr int kFoldRows = 2 * kNumEpiWarps;
+// (four rows per warp at most), while its first tiles are computed -- no launch in between.
+constexpr int kFoldRows = 4 * kNumEpiWarps;
 
 // a, b ascending: a becomes the 16 smallest of the 32 values, ascending.  min(a[i], b[15 - i]) are
 // those 16 values as a bitonic sequence, which four half-cleaner stages sort.
@@ -1112,11 +1112,13 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 ++it;
             }
             if constexpr (EPI == EPI_SKETCH && MT == 1) {
-                if (ok && p.tau_out != nullptr) {
-                    // This CTA saw the row group's whole sample, split between the two warps of every lane
-                    // quadrant: the upper-half warp passes its 16 sorted minima through shared memory, the
-                    // lower-half warp finishes the threshold.  With a and b ascending, min(a[i], b[15 - i])
-                    // over i are the 16 smallest of the 32 values, so their maximum is the 16th smallest.
+                if (ok && (p.tau_out != nullptr || p.sketch_t != nullptr)) {
+                    // The two warps of every lane quadrant split the tiles' columns between them: the
+                    // upper-half warp passes its 16 sorted minima through shared memory to the lower-half
+                    // warp.  tau_out: this CTA saw the row group's whole sample and the lower-half warp
+                    // finishes the threshold -- with a and b ascending, min(a[i], b[15 - i]) over i are the
+                    // 16 smallest of the 32 values, so their maximum is the 16th smallest.  sketch_t: the
+                    // lower-half warp merges the two lists into the CTA's one partial sketch.
                     float* xch = reinterpret_cast<float*>(hist_all) + row_in_tile * kSampleM;
                     if (half == 1) {
                         if (xseg > 0) ok = __all_sync(0xFFFFFFFFu, mbar_wait(&x_empty[quad], (xseg - 1) & 1, ctl, 7));
@@ -1138,10 +1140,14 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                             }
                             __syncwarp();
                             if (lane == 0) mbar_arrive(&x_empty[quad]);
-                            float t16 = -INF;
+                            if (p.tau_out != nullptr) {
+                                float t16 = -INF;
 #pragma unroll
-                            for (int i = 0; i < kSampleM; ++i) t16 = fmaxf(t16, fminf(st[0].net[i], other[kSampleM - 1 - i]));
-                            if (valid[0]) p.tau_out[row[0]] = t16;
+                                for (int i = 0; i < kSampleM; ++i) t16 = fmaxf(t16, fminf(st[0].net[i], other[kSampleM - 1 - i]));
+                                if (valid[0]) p.tau_out[row[0]] = t16;
+                            } else {
+                                merge16_sorted(st[0].net, other);
+                            }
                         }
                     }
                     ++xseg;
@@ -1161,9 +1167,11 @@ fused_topk_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                     } else if constexpr (EPI == EPI_SKETCH) {
                         // the partial result of the threshold pass: the thread's 16 smallest group minima
                         if (p.sketch_t != nullptr) {
-                            // (a batch of a few rows, read back by the main pass with slot = lane)
-                            if (IVF_IN_BOUNDS(146, slot, p.sketch_pitch)) {
-                                float* out = p.sketch_t + static_cast<size_t>(row[h]) * kSampleM * p.sketch_pitch + slot;
+                            // (a batch of a few rows, read back by the main pass with slot = lane; with one
+                            // row tile per unit the lower-half warp holds the CTA's merged sketch)
+                            const int slot_out = MT == 1 ? slot >> 1 : slot;
+                            if ((MT != 1 || half == 0) && IVF_IN_BOUNDS(146, slot_out, p.sketch_pitch)) {
+                                float* out = p.sketch_t + static_cast<size_t>(row[h]) * kSampleM * p.sketch_pitch + slot_out;
 #pragma unroll
                                 for (int i = 0; i < kSampleM; ++i) out[static_cast<size_t>(i) * p.sketch_pitch] = st[h].net[i];
                             }

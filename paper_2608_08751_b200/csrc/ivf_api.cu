@@ -600,7 +600,10 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
     }
     // Batches of a few rows: the main pass finishes the thresholds from the partial sketches itself (one
     // epilogue warp per row, while the first tiles load), so no merge kernel runs between the two passes.
-    const bool tau_fold = given && !sketch_whole && g_tau_fold && n <= kFoldRows;
+    // (up to two rows per epilogue warp always; up to four when every CTA has enough tiles to compute
+    // meanwhile -- 524,288 lists, B = 32: 77.0 -> 72.6 us, but 65,536 lists: 45.5 -> 47.1)
+    const bool tau_fold = given && !sketch_whole && g_tau_fold &&
+                          (n <= kFoldRows / 2 || (n <= kFoldRows && pl.col_tiles >= 4 * ctx.num_sms));
     PointPrep pp;
     Entry* part;
     int2* part_meta = nullptr;
@@ -678,8 +681,11 @@ int route_rows_device(DeviceCtx& ctx, const void* points, int64_t n, int d, int 
         } else if (tau_fold) {
             // the main pass finishes them
             fold_sketch = sketch_t;
+            // (one sketch per CTA that took part of the row group's sample -- its two epilogue halves merge
+            // theirs in shared memory -- or one per half with two row tiles per unit)
             fold_slots = (cta_of_unit(pls.total_units, pls.ctas, pls.col_tiles, pls.cross, pls.col_tiles - 1) -
-                          cta_of_unit(pls.total_units, pls.ctas, pls.col_tiles, pls.cross, 0) + 1) * kEpiHalves;
+                          cta_of_unit(pls.total_units, pls.ctas, pls.col_tiles, pls.cross, 0) + 1) *
+                         (pls.mtiles == 1 ? 1 : kEpiHalves);
         } else if (pls.partials <= 32)
             LAUNCH_DEP(4, merge_tau_warp_kernel, static_cast<unsigned>((n * 32 + 255) / 256), 256, 0, stream, ms);
         else {

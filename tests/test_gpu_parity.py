@@ -163,11 +163,12 @@ def test_threshold_pass_in_one_kernel_gives_the_same_results(n, nlist, d, k, dty
     parity.check_route(x, c, k, ids[rows], dists[rows], rows=rows)
 
 
-@pytest.mark.parametrize("n", [1, 3, 8, 9, 16, 17])  # 17: one row more than the main pass takes on itself
+@pytest.mark.parametrize("n", [1, 3, 8, 9, 16, 17, 32, 33])  # main pass: up to 16 rows, up to 32 against the largest table
 @pytest.mark.parametrize("nlist,d,k,dtype", [(300000, 128, 64, "u8"), (90000, 96, 128, "f32"), (33000, 64, 17, "f32")])
 def test_thresholds_finished_by_the_main_pass_give_the_same_results(n, nlist, d, k, dtype):
-    # batches of at most 16 rows: the epilogue warps of the main pass merge the partial sketches of
-    # the threshold pass themselves (a warp per row, two rows per warp at most); the merge kernel computes the same order
+    # batches of at most 16 rows (32 when every CTA has tiles enough to compute meanwhile): the epilogue
+    # warps of the main pass merge the partial sketches of the threshold pass themselves (a warp per
+    # row, four rows per warp at most); the merge kernel computes the same order
     # statistic, so the two schedules must agree bit for bit -- with one or several sketches per lane
     x, c = _rand(n, nlist, d, dtype, seed=n + nlist)
     ids, dists = _route(x, c, k)
