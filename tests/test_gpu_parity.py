@@ -484,6 +484,21 @@ def test_results_in_pinned_host_memory(host_in, k, with_dists):
     B.ivf_check()
 
 
+def test_prepared_table_with_results_in_host_memory():
+    x, c = _rand(900, 40000, 128, "u8", 31)
+    want_ids, want_d = _route(x, c, 64)
+    h = B.PreparedCentroids(_cuda(c))
+    try:
+        ids_h, d_h = _pinned((900, 64), torch.int32, -1), _pinned((900, 64), torch.float32, -1.0)
+        xt = torch.from_numpy(x).pin_memory()  # alive until the copy has run
+        B.ivf_route_prepared(h, xt, 64, ids_h, d_h)
+        torch.cuda.current_stream().synchronize()
+        assert (ids_h.numpy() == want_ids).all() and (d_h.numpy() == want_d).all()
+        B.ivf_check()
+    finally:
+        h.close()
+
+
 def test_deferred_read_back_of_host_results():
     # serving loop: with deferred read-back the calls do not wait for their copies; two staging pairs
     # are used in turn, so a third call must wait for the first one's copy before it reuses the pair
@@ -520,7 +535,8 @@ def test_assign_update_with_ids_in_host_memory():
     sums = torch.zeros((nlist, d), dtype=torch.float32, device="cuda")
     counts = torch.zeros((nlist,), dtype=torch.int64, device="cuda")
     ids_h = _pinned((n,), torch.int32, -1)
-    B.ivf_assign_update(torch.from_numpy(x).pin_memory(), _cuda(c), sums, counts, ids_h, None, chunk_rows=2048)
+    xt = torch.from_numpy(x).pin_memory()  # alive until the copies have run
+    B.ivf_assign_update(xt, _cuda(c), sums, counts, ids_h, None, chunk_rows=2048)
     torch.cuda.current_stream().synchronize()
     ids = ids_h.numpy().copy()
     B.ivf_check()
