@@ -14,7 +14,9 @@
  * Conventions shared by all calls
  *   Layout     every matrix is dense row-major with contiguous rows (leading dimension = d).
  *   Pointers   "device" = memory of the current CUDA device; "host" = page-locked host memory.
- *              The caller owns every buffer; the library keeps none past stream completion.
+ *              The caller owns every buffer; the library keeps none past stream completion.  All work is
+ *              asynchronous: a buffer (host buffers above all) must stay allocated and unchanged until
+ *              the work the call enqueued has completed.
  *   Streams    work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = legacy default
  *              stream) and the call returns without waiting, except where stated.
  *   Workspace  the library keeps one grow-only device workspace per device; it grows with a
